@@ -1,0 +1,330 @@
+/*
+ * mpo.c -- CPU oracle for the mixed-precision training hot path.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain statement of what the
+ * path computes, used by the test-suite and by the benchmark's CPU-baseline leg.
+ * It shares no code with the CUDA library and the CUDA library never calls it.
+ *
+ * Recipe implemented (paper section 3; "pseudo FP16" mode of section 4):
+ *   - tensors are stored as IEEE binary16 (section 3.1);
+ *   - dot products multiply binary16 values and accumulate in binary32, the
+ *     result is converted to binary16 when written (section 3.3);
+ *   - reductions of the softmax are carried out in binary32 on binary16 data
+ *     (section 3.3);
+ *   - the loss is multiplied by a constant S before back-propagation, weight
+ *     gradients are multiplied by 1/S before the update, an inf/NaN in the
+ *     unscaled weight gradients skips the update (section 3.2);
+ *   - the update is applied to a binary32 master copy which is then rounded to
+ *     the binary16 working copy (section 3.1).
+ *
+ * The paper never names the rounding mode; round-to-nearest-even with gradual
+ * underflow is used throughout.  The paper's sentence that magnitudes below
+ * 2^-24 become zero (section 3.1) describes truncation; under round-to-nearest
+ * values in (2^-25, 2^-24) round up to 2^-24 and 2^-25 itself ties to zero.
+ *
+ * Pins: every function here is checked by tests that do not go through this
+ * file's own formulas (numpy's binary16 casts, exact rational arithmetic,
+ * closed forms, finite differences in double precision).  No function is
+ * "parity unpinned".
+ *
+ * Build: gcc -O2 -std=c11 -ffp-contract=off -fno-fast-math -fopenmp -shared -fPIC
+ * (-ffp-contract=off keeps every binary32 operation separately rounded).
+ * OpenMP is used over independent output rows / independent elements only, so
+ * no element's arithmetic depends on the thread count.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* ---------------------------------------------------------------- binary16 */
+
+static inline uint32_t f32_bits(float x) { uint32_t u; memcpy(&u, &x, 4); return u; }
+static inline float bits_f32(uint32_t u) { float x; memcpy(&x, &u, 4); return x; }
+
+/* binary16 -> binary32, exact for every pattern (section 3.1: FP16 storage). */
+float mpo_h2f(uint16_t h)
+{
+    uint32_t sign = (uint32_t)(h & 0x8000u) << 16;
+    uint32_t e = (h >> 10) & 0x1Fu;
+    uint32_t m = h & 0x3FFu;
+    if (e == 0x1Fu)                       /* inf / NaN */
+        return bits_f32(sign | 0x7F800000u | (m << 13));
+    if (e != 0)                           /* normal: exponent range [-14, 15] */
+        return bits_f32(sign | ((e + 112u) << 23) | (m << 13));
+    if (m == 0)
+        return bits_f32(sign);
+    /* subnormal: m * 2^-24 */
+    float mag = (float)m * 0x1p-24f;
+    return bits_f32(sign | f32_bits(mag));
+}
+
+/* binary32 -> binary16, round to nearest, ties to even, gradual underflow.
+ * Largest finite result 65504; |x| >= 65520 becomes infinity (section 3.2). */
+uint16_t mpo_f2h(float x)
+{
+    uint32_t u = f32_bits(x);
+    uint16_t sign = (uint16_t)((u >> 16) & 0x8000u);
+    uint32_t a = u & 0x7FFFFFFFu;
+    if (a > 0x7F800000u) return (uint16_t)(sign | 0x7E00u);       /* NaN -> quiet NaN */
+    if (a >= 0x477FF000u) return (uint16_t)(sign | 0x7C00u);      /* >= 65520, inf */
+    if (a >= 0x38800000u) {                                       /* >= 2^-14: normal */
+        uint32_t e = (a >> 23) - 112u;
+        uint32_t m = a & 0x7FFFFFu;
+        uint32_t h = (e << 10) | (m >> 13);
+        uint32_t rem = m & 0x1FFFu;
+        if (rem > 0x1000u || (rem == 0x1000u && (h & 1u))) h++;   /* carry may bump the exponent */
+        return (uint16_t)(sign | h);
+    }
+    /* result is subnormal or zero: round onto the 2^-24 grid */
+    uint32_t e = a >> 23;
+    if (e < 102u) return sign;                                    /* |x| < 2^-25 */
+    uint32_t m = (a & 0x7FFFFFu) | 0x800000u;
+    uint32_t shift = 126u - e;                                    /* 14 .. 24 */
+    uint32_t h = m >> shift;
+    uint32_t rem = m & ((1u << shift) - 1u);
+    uint32_t half = 1u << (shift - 1u);
+    if (rem > half || (rem == half && (h & 1u))) h++;
+    return (uint16_t)(sign | h);
+}
+
+void mpo_h2f_array(const uint16_t *h, float *f, size_t n)
+{
+#pragma omp parallel for schedule(static)
+    for (size_t i = 0; i < n; i++) f[i] = mpo_h2f(h[i]);
+}
+
+void mpo_f2h_array(const float *f, uint16_t *h, size_t n)
+{
+#pragma omp parallel for schedule(static)
+    for (size_t i = 0; i < n; i++) h[i] = mpo_f2h(f[i]);
+}
+
+/* f2h over a contiguous range of binary32 bit patterns (exhaustive pin). */
+void mpo_f2h_bits_range(uint32_t first, uint32_t count, uint16_t *h)
+{
+#pragma omp parallel for schedule(static)
+    for (uint32_t i = 0; i < count; i++) h[i] = mpo_f2h(bits_f32(first + i));
+}
+
+int mpo_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* -------------------------------------------------------------------- GEMM */
+/*
+ * C[m,n] = rn16( post( sum_{k ascending} A(m,k) * B(k,n) ) ), sum in binary32
+ * (section 3.3: FP16 dot product accumulated in FP32, converted on the store).
+ *
+ * The three linear-layer products of one training iteration (section 3.1) differ
+ * only in which index of each stored matrix is contracted:
+ *   op 0 forward  Y = X W^T : A stored [M,K] (a_trans=0), B stored [N,K] (b_trans=0)
+ *   op 1 dgrad    dX = dY W : A stored [M,K] (a_trans=0), B stored [K,N] (b_trans=1)
+ *   op 2 wgrad    dW = dY^T X: A stored [K,M] (a_trans=1), B stored [K,N] (b_trans=1)
+ * All stored matrices are row-major with leading dimensions lda/ldb/ldc.
+ *
+ * post: relu != 0 applies x>0 ? x : +0 to the binary32 sum before rounding
+ *       (NaN propagates).  mask != NULL zeroes (+0) the rounded output where
+ *       the stored binary16 value mask[m,n] is not > 0 (ReLU derivative taken
+ *       from the stored activation).
+ *
+ * Side channels (optional, may be NULL): exact[m,n] = the same sum accumulated
+ * in double (every product of two binary16 values is exact in double and the
+ * double sum is accurate far below binary16 resolution); absdot[m,n] = sum |a*b|.
+ *
+ * row_begin/row_end restrict the computed output rows (used to time a slab).
+ */
+void mpo_gemm_f16(int op, int M, int N, int K,
+                  const uint16_t *A, int lda, const uint16_t *B, int ldb,
+                  uint16_t *C, int ldc, int relu,
+                  const uint16_t *mask, int ldmask,
+                  double *exact, double *absdot,
+                  int row_begin, int row_end)
+{
+    const int a_trans = (op == 2);
+    const int b_trans = (op != 0);
+    if (row_begin < 0) row_begin = 0;
+    if (row_end > M || row_end < 0) row_end = M;
+    if (M <= 0 || N <= 0 || row_end <= row_begin) return;
+
+    /* binary32 copy of the second operand laid out [K][N] so that, for a fixed
+     * output row, the k loop is outermost and each output still sums k = 0..K-1
+     * in ascending order. */
+    float *Bf = (float *)malloc((size_t)(K > 0 ? K : 1) * (size_t)N * sizeof(float));
+#pragma omp parallel for schedule(static)
+    for (int k = 0; k < K; k++)
+        for (int n = 0; n < N; n++) {
+            uint16_t hb = b_trans ? B[(size_t)k * ldb + n] : B[(size_t)n * ldb + k];
+            Bf[(size_t)k * N + n] = mpo_h2f(hb);
+        }
+
+#pragma omp parallel
+    {
+        float *acc = (float *)malloc((size_t)N * sizeof(float));
+        double *dacc = exact ? (double *)malloc((size_t)N * sizeof(double)) : NULL;
+        double *aacc = absdot ? (double *)malloc((size_t)N * sizeof(double)) : NULL;
+#pragma omp for schedule(static)
+        for (int m = row_begin; m < row_end; m++) {
+            for (int n = 0; n < N; n++) acc[n] = 0.0f;
+            if (dacc) for (int n = 0; n < N; n++) dacc[n] = 0.0;
+            if (aacc) for (int n = 0; n < N; n++) aacc[n] = 0.0;
+            for (int k = 0; k < K; k++) {
+                uint16_t ha = a_trans ? A[(size_t)k * lda + m] : A[(size_t)m * lda + k];
+                float a = mpo_h2f(ha);
+                const float *brow = Bf + (size_t)k * N;
+                for (int n = 0; n < N; n++) {
+                    float p = a * brow[n];          /* exact: <= 22 significant bits */
+                    acc[n] = acc[n] + p;            /* one binary32 rounding per term */
+                }
+                if (dacc) for (int n = 0; n < N; n++) dacc[n] += (double)a * (double)brow[n];
+                if (aacc) for (int n = 0; n < N; n++) aacc[n] += fabs((double)a * (double)brow[n]);
+            }
+            for (int n = 0; n < N; n++) {
+                float s = acc[n];
+                if (relu) s = (s > 0.0f) ? s : ((s != s) ? s : 0.0f);
+                uint16_t h = mpo_f2h(s);
+                if (mask && !(mpo_h2f(mask[(size_t)m * ldmask + n]) > 0.0f)) h = 0;
+                C[(size_t)m * ldc + n] = h;
+            }
+            if (dacc) for (int n = 0; n < N; n++) exact[(size_t)m * N + n] = dacc[n];
+            if (aacc) for (int n = 0; n < N; n++) absdot[(size_t)m * N + n] = aacc[n];
+        }
+        free(acc); free(dacc); free(aacc);
+    }
+    free(Bf);
+}
+
+/* One output element of the same product, for sampled checks at sizes where the
+ * full product would take hours.  Returns the rounded binary16 (before mask). */
+uint16_t mpo_gemm_f16_element(int op, int K,
+                              const uint16_t *A, int lda, const uint16_t *B, int ldb,
+                              int m, int n, int relu, double *exact, double *absdot)
+{
+    const int a_trans = (op == 2);
+    const int b_trans = (op != 0);
+    float acc = 0.0f;
+    double d = 0.0, ad = 0.0;
+    for (int k = 0; k < K; k++) {
+        float a = mpo_h2f(a_trans ? A[(size_t)k * lda + m] : A[(size_t)m * lda + k]);
+        float b = mpo_h2f(b_trans ? B[(size_t)k * ldb + n] : B[(size_t)n * ldb + k]);
+        float p = a * b;
+        acc = acc + p;
+        d += (double)a * (double)b;
+        ad += fabs((double)a * (double)b);
+    }
+    if (relu) acc = (acc > 0.0f) ? acc : ((acc != acc) ? acc : 0.0f);
+    if (exact) *exact = d;
+    if (absdot) *absdot = ad;
+    return mpo_f2h(acc);
+}
+
+/* ------------------------------------------------ softmax cross-entropy */
+/*
+ * Per row i of binary16 logits z[i, 0..C-1] (section 3.3: reductions in FP32 on
+ * FP16 data), with the loss scale S applied to the gradient (section 3.2: scaling
+ * the loss scales every gradient by the chain rule):
+ *   m = max_j z_j ; e_j = expf(z_j - m) ; s = sum_j e_j (ascending)
+ *   loss_i = (m + logf(s)) - z_y
+ *   c = S / (float)B ; dz[i,j] = rn16( (e_j / s - [j == y]) * c )
+ * loss = (float)( sum_i (double)loss_i / B ), the unscaled mean.
+ * A label outside [0, C) contributes no loss and a zero gradient row and is
+ * counted in the return value.
+ */
+int mpo_softmax_ce(const uint16_t *z, int ldz, const int32_t *labels, int B, int C,
+                   float S, uint16_t *dz, int lddz, float *row_loss, float *loss)
+{
+    int bad = 0;
+    const float c = S / (float)B;
+    float *rl = row_loss ? row_loss : (float *)malloc((size_t)(B > 0 ? B : 1) * sizeof(float));
+#pragma omp parallel for schedule(static) reduction(+ : bad)
+    for (int i = 0; i < B; i++) {
+        const uint16_t *zi = z + (size_t)i * ldz;
+        uint16_t *dzi = dz ? dz + (size_t)i * lddz : NULL;
+        int y = labels[i];
+        if (y < 0 || y >= C) {
+            bad += 1;
+            rl[i] = 0.0f;
+            if (dzi) for (int j = 0; j < C; j++) dzi[j] = 0;
+            continue;
+        }
+        float m = mpo_h2f(zi[0]);
+        for (int j = 1; j < C; j++) {
+            float v = mpo_h2f(zi[j]);
+            if (v > m) m = v;                  /* a NaN logit reaches s through expf */
+        }
+        float s = 0.0f;
+        for (int j = 0; j < C; j++) s = s + expf(mpo_h2f(zi[j]) - m);
+        rl[i] = (m + logf(s)) - mpo_h2f(zi[y]);
+        if (dzi)
+            for (int j = 0; j < C; j++) {
+                float e = expf(mpo_h2f(zi[j]) - m);
+                float p = e / s;
+                float d = p - ((j == y) ? 1.0f : 0.0f);
+                dzi[j] = mpo_f2h(d * c);
+            }
+    }
+    if (loss) {
+        double acc = 0.0;
+        for (int i = 0; i < B; i++) acc += (double)rl[i];
+        *loss = (B > 0) ? (float)(acc / (double)B) : 0.0f;
+    }
+    if (!row_loss) free(rl);
+    return bad;
+}
+
+/* ------------------------------------------------------- master-weight pass */
+/*
+ * Overflow inspection (section 3.2): 1 if any unscaled weight gradient
+ * h2f(g[e]) * inv_S is inf or NaN.
+ */
+int mpo_grad_nonfinite(const uint16_t *g, size_t n, float inv_S)
+{
+    int flag = 0;
+#pragma omp parallel for schedule(static) reduction(| : flag)
+    for (size_t e = 0; e < n; e++) {
+        float v = mpo_h2f(g[e]) * inv_S;
+        if (!isfinite(v)) flag |= 1;
+    }
+    return flag;
+}
+
+/*
+ * Update of the binary32 master copy and re-rounding of the binary16 working
+ * copy (sections 3.1, 3.2).  Each line is one separately rounded binary32
+ * operation (no fused multiply-add, no flush to zero):
+ *   g = h2f(g16[e]) * inv_S
+ *   momentum:  t = mu * v[e] ; v[e] = t + g ; u = lr * v[e]
+ *   plain:     u = lr * g
+ *   w32[e] = w32[e] - u ; w16[e] = rn16(w32[e])
+ * The caller decides the skip: this function must only be called when
+ * mpo_grad_nonfinite over ALL layers returned 0.
+ */
+void mpo_update_apply(const uint16_t *g16, float *w32, float *v, uint16_t *w16,
+                      size_t n, float inv_S, float lr, float mu, int use_momentum)
+{
+#pragma omp parallel for schedule(static)
+    for (size_t e = 0; e < n; e++) {
+        float g = mpo_h2f(g16[e]) * inv_S;
+        float u;
+        if (use_momentum) {
+            float t = mu * v[e];
+            float nv = t + g;
+            v[e] = nv;
+            u = lr * nv;
+        } else {
+            u = lr * g;
+        }
+        float w = w32[e] - u;
+        w32[e] = w;
+        w16[e] = mpo_f2h(w);
+    }
+}

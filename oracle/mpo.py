@@ -1,0 +1,202 @@
+"""ctypes access to the CPU oracle (mpo.c).
+
+TEST INFRASTRUCTURE ONLY: imported by the tests, by the smoke check and by the
+benchmark's CPU-baseline leg.  The CUDA library and its Python binding never
+import this module, and this module never imports them.
+
+The shared object is compiled on first use with gcc (see ``build``).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "mpo.c")
+_LIB = os.path.join(_HERE, "libmpo.so")
+
+OP_FWD, OP_DGRAD, OP_WGRAD = 0, 1, 2
+
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile mpo.c into libmpo.so (gcc, separately rounded binary32 ops)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O2", "-std=c11", "-ffp-contract=off", "-fno-fast-math", "-fopenmp",
+               "-shared", "-fPIC", "-o", _LIB, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        build()
+        L = ctypes.CDLL(_LIB)
+        c = ctypes
+        L.mpo_h2f.restype = c.c_float
+        L.mpo_h2f.argtypes = [c.c_uint16]
+        L.mpo_f2h.restype = c.c_uint16
+        L.mpo_f2h.argtypes = [c.c_float]
+        L.mpo_h2f_array.restype = None
+        L.mpo_h2f_array.argtypes = [c.c_void_p, c.c_void_p, c.c_size_t]
+        L.mpo_f2h_array.restype = None
+        L.mpo_f2h_array.argtypes = [c.c_void_p, c.c_void_p, c.c_size_t]
+        L.mpo_f2h_bits_range.restype = None
+        L.mpo_f2h_bits_range.argtypes = [c.c_uint32, c.c_uint32, c.c_void_p]
+        L.mpo_num_threads.restype = c.c_int
+        L.mpo_num_threads.argtypes = []
+        L.mpo_gemm_f16.restype = None
+        L.mpo_gemm_f16.argtypes = [c.c_int, c.c_int, c.c_int, c.c_int,
+                                   c.c_void_p, c.c_int, c.c_void_p, c.c_int,
+                                   c.c_void_p, c.c_int, c.c_int,
+                                   c.c_void_p, c.c_int, c.c_void_p, c.c_void_p,
+                                   c.c_int, c.c_int]
+        L.mpo_gemm_f16_element.restype = c.c_uint16
+        L.mpo_gemm_f16_element.argtypes = [c.c_int, c.c_int, c.c_void_p, c.c_int, c.c_void_p, c.c_int,
+                                           c.c_int, c.c_int, c.c_int, c.c_void_p, c.c_void_p]
+        L.mpo_softmax_ce.restype = c.c_int
+        L.mpo_softmax_ce.argtypes = [c.c_void_p, c.c_int, c.c_void_p, c.c_int, c.c_int, c.c_float,
+                                     c.c_void_p, c.c_int, c.c_void_p, c.c_void_p]
+        L.mpo_grad_nonfinite.restype = c.c_int
+        L.mpo_grad_nonfinite.argtypes = [c.c_void_p, c.c_size_t, c.c_float]
+        L.mpo_update_apply.restype = None
+        L.mpo_update_apply.argtypes = [c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_size_t,
+                                       c.c_float, c.c_float, c.c_float, c.c_int]
+        _lib = L
+    return _lib
+
+
+def num_threads() -> int:
+    return int(lib().mpo_num_threads())
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _u16(a) -> np.ndarray:
+    """View/convert an array of binary16 values as contiguous uint16 bit patterns."""
+    a = np.asarray(a)
+    if a.dtype == np.float16:
+        a = a.view(np.uint16)
+    if a.dtype != np.uint16:
+        raise TypeError("expected float16 or uint16 bit patterns, got %s" % a.dtype)
+    return a
+
+
+def h2f(h) -> np.ndarray:
+    h = np.ascontiguousarray(_u16(h))
+    out = np.empty(h.shape, dtype=np.float32)
+    lib().mpo_h2f_array(_ptr(h), _ptr(out), h.size)
+    return out
+
+
+def f2h(f) -> np.ndarray:
+    """binary32 -> binary16 bit patterns (uint16), round to nearest even."""
+    f = np.ascontiguousarray(np.asarray(f, dtype=np.float32))
+    out = np.empty(f.shape, dtype=np.uint16)
+    lib().mpo_f2h_array(_ptr(f), _ptr(out), f.size)
+    return out
+
+
+def f2h_bits_range(first: int, count: int) -> np.ndarray:
+    out = np.empty(count, dtype=np.uint16)
+    lib().mpo_f2h_bits_range(first, count, _ptr(out))
+    return out
+
+
+def gemm_f16(op, A, B, relu=False, mask=None, want_exact=False, rows=None):
+    """Linear-layer product in the mixed-precision recipe (paper section 3.3).
+
+    op 0: C[M,N] = A[M,K] . B[N,K]^T ; op 1: C[M,N] = A[M,K] . B[K,N] ;
+    op 2: C[M,N] = A[K,M]^T . B[K,N].  A, B, mask: 2-D uint16/float16 arrays (row
+    strides may exceed the row length).  Returns uint16 bit patterns, plus
+    (exact, absdot) float64 arrays when want_exact.
+    """
+    A = _u16(A)
+    B = _u16(B)
+    assert A.ndim == 2 and B.ndim == 2
+    assert A.strides[1] == 2 and B.strides[1] == 2
+    if op == OP_FWD:
+        M, K = A.shape
+        N, K2 = B.shape
+    elif op == OP_DGRAD:
+        M, K = A.shape
+        K2, N = B.shape
+    elif op == OP_WGRAD:
+        K, M = A.shape
+        K2, N = B.shape
+    else:
+        raise ValueError("op")
+    assert K == K2, (A.shape, B.shape, op)
+    lda = A.strides[0] // 2 if A.shape[0] > 1 else A.shape[1]
+    ldb = B.strides[0] // 2 if B.shape[0] > 1 else B.shape[1]
+    C = np.zeros((M, N), dtype=np.uint16)
+    ex = np.zeros((M, N), dtype=np.float64) if want_exact else None
+    ab = np.zeros((M, N), dtype=np.float64) if want_exact else None
+    mk = None
+    ldm = 0
+    if mask is not None:
+        mk = _u16(mask)
+        assert mk.shape == (M, N) and mk.strides[1] == 2
+        ldm = mk.strides[0] // 2 if M > 1 else N
+    r0, r1 = (0, M) if rows is None else rows
+    lib().mpo_gemm_f16(op, M, N, K, _ptr(A), lda, _ptr(B), ldb, _ptr(C), N, int(bool(relu)),
+                       _ptr(mk), ldm, _ptr(ex), _ptr(ab), r0, r1)
+    if want_exact:
+        return C, ex, ab
+    return C
+
+
+def gemm_f16_element(op, A, B, m, n, relu=False):
+    """One output element (rounded bits, exact double sum, sum of |products|)."""
+    A = _u16(A)
+    B = _u16(B)
+    K = A.shape[0] if op == OP_WGRAD else A.shape[1]
+    lda = A.strides[0] // 2
+    ldb = B.strides[0] // 2
+    ex = ctypes.c_double(0.0)
+    ab = ctypes.c_double(0.0)
+    h = lib().mpo_gemm_f16_element(op, K, _ptr(A), lda, _ptr(B), ldb, int(m), int(n), int(bool(relu)),
+                                   ctypes.byref(ex), ctypes.byref(ab))
+    return int(h), ex.value, ab.value
+
+
+def softmax_ce(z, labels, S):
+    """Softmax cross-entropy forward + scaled backward (paper sections 3.2, 3.3).
+
+    Returns (dz uint16 [B,C], row_loss float32 [B], mean loss float, n_bad_labels).
+    """
+    z = _u16(z)
+    assert z.ndim == 2 and z.strides[1] == 2
+    Bn, C = z.shape
+    ldz = z.strides[0] // 2 if Bn > 1 else C
+    labels = np.ascontiguousarray(labels, dtype=np.int32)
+    dz = np.zeros((Bn, C), dtype=np.uint16)
+    rl = np.zeros(Bn, dtype=np.float32)
+    loss = ctypes.c_float(0.0)
+    bad = lib().mpo_softmax_ce(_ptr(z), ldz, _ptr(labels), Bn, C, float(S), _ptr(dz), C, _ptr(rl),
+                               ctypes.byref(loss))
+    return dz, rl, float(loss.value), int(bad)
+
+
+def grad_nonfinite(g16, inv_S) -> int:
+    g = np.ascontiguousarray(_u16(g16)).reshape(-1)
+    return int(lib().mpo_grad_nonfinite(_ptr(g), g.size, float(inv_S)))
+
+
+def update_apply(g16, w32, v, w16, inv_S, lr, mu, use_momentum) -> None:
+    """In-place master update on contiguous arrays (caller has checked the flag)."""
+    g = _u16(g16)
+    for a in (g, w32, w16) + ((v,) if v is not None else ()):
+        assert a.flags["C_CONTIGUOUS"]
+    assert w32.dtype == np.float32 and w16.dtype == np.uint16
+    if use_momentum:
+        assert v is not None and v.dtype == np.float32
+    lib().mpo_update_apply(_ptr(g), _ptr(w32), _ptr(v) if use_momentum else None, _ptr(w16), g.size,
+                           float(inv_S), float(lr), float(mu), int(bool(use_momentum)))
