@@ -1,0 +1,233 @@
+/*
+ * mpt.h -- C ABI of the B200 (sm_100a) mixed-precision training hot path.
+ *
+ * The library implements one training iteration of a stack of bias-free linear
+ * layers in the recipe of "Mixed Precision Training" (arXiv 1710.03740):
+ *
+ *   section 3.1  weights, activations and gradients are stored as FP16; an FP32
+ *                master copy of the weights receives the update and is rounded
+ *                to the FP16 working copy used by forward and backward;
+ *   section 3.2  the loss is multiplied by a constant S before back-propagation;
+ *                weight gradients are multiplied by 1/S before the update and
+ *                inspected for inf/NaN, in which case the update is skipped;
+ *   section 3.3  dot products take FP16 operands, accumulate in FP32 and convert
+ *                to FP16 on the store; softmax reductions run in FP32 on FP16
+ *                data; point-wise ops (ReLU) are fused into the producers.
+ *
+ * Conventions
+ *   - Every tensor is row-major, last index contiguous.  FP16 values cross this
+ *     boundary as uint16_t bit patterns (IEEE binary16).  Rounding FP32 -> FP16
+ *     is round-to-nearest-even with gradual underflow everywhere.
+ *   - "_dev" pointers are CUDA device pointers, "_host" pointers are host
+ *     pointers (pageable or pinned).  Nothing in a signature is a torch type.
+ *   - The library never allocates or frees device memory, never creates a
+ *     stream, and keeps no global state.  The caller owns the workspace, the
+ *     inputs, the stream and all host buffers; the library owns only its
+ *     host-side context object.
+ *   - Every call returns MPT_OK (0) or a negative MPT_ERR_* code and never
+ *     throws.  A null context or a null required pointer gives
+ *     MPT_ERR_INVALID_ARG with nothing dereferenced.  Calls are asynchronous on
+ *     the context's stream unless a host out-pointer is passed, in which case
+ *     the call synchronises the stream before writing it.
+ *   - After MPT_ERR_CUDA or MPT_ERR_TIMEOUT the context is poisoned: only
+ *     mpt_last_error and mpt_destroy succeed.
+ *   - A context is not thread-safe; distinct contexts are independent.
+ */
+#ifndef MPT_H_
+#define MPT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define MPT_OK 0
+#define MPT_ERR_INVALID_ARG (-1) /* null pointer, bad enum, bad scalar */
+#define MPT_ERR_SHAPE (-2)       /* dimensions inconsistent or out of range */
+#define MPT_ERR_STATE (-3)       /* call order violated (e.g. backward before forward) */
+#define MPT_ERR_WORKSPACE (-4)   /* workspace too small or misaligned */
+#define MPT_ERR_CUDA (-5)        /* a CUDA runtime/driver call failed */
+#define MPT_ERR_TIMEOUT (-6)     /* a bounded device-side wait expired */
+#define MPT_ERR_INTERNAL (-7)    /* internal consistency check failed */
+
+/* Which index of the stored operands is contracted (section 3.3; the three
+ * products of one layer's iteration, section 3.1):
+ *   FWD    C[M,N] = A[M,K] . B[N,K]^T     Y  = X  W^T
+ *   DGRAD  C[M,N] = A[M,K] . B[K,N]       dX = dY W
+ *   WGRAD  C[M,N] = A[K,M]^T . B[K,N]     dW = dY^T X                      */
+#define MPT_OP_FWD 0
+#define MPT_OP_DGRAD 1
+#define MPT_OP_WGRAD 2
+
+/* mpt_gemm_f16 flags */
+#define MPT_GEMM_RELU 1u      /* apply x > 0 ? x : +0 to the FP32 sum before rounding */
+#define MPT_GEMM_FORCE_SIMT 2u /* use the plain CUDA-core kernel (sequential-k FP32 sum) */
+#define MPT_GEMM_FORCE_TC 4u   /* require the tcgen05 kernel; MPT_ERR_SHAPE if the operands
+                                  do not meet its alignment rules */
+
+/* mpt_get_tensor kinds */
+#define MPT_T_W16 0        /* FP16 working weights   [out, in]            */
+#define MPT_T_GRAD16 1     /* FP16 weight gradients  [out, in] (scaled by S) */
+#define MPT_T_ACT16 2      /* FP16 activation a_l    [batch, out_l]       */
+#define MPT_T_DACT16 3     /* FP16 gradient dz_l     [batch, out_l] (scaled by S) */
+#define MPT_T_MOMENTUM32 4 /* FP32 momentum buffer   [out, in]            */
+#define MPT_T_MASTER32 5   /* FP32 master weights    [out, in]            */
+
+typedef struct mpt_ctx mpt_ctx;
+
+typedef struct mpt_layer_desc {
+    int32_t in_features;
+    int32_t out_features;
+    int32_t relu; /* 1: ReLU after this layer (hidden layers); the last layer must be 0 */
+} mpt_layer_desc;
+
+/* ------------------------------------------------------------ model-level calls */
+
+/* Size in bytes of the single device workspace a context needs (section 3.1:
+ * FP32 master + FP16 weights + FP16 gradients, optional FP32 momentum, FP16
+ * activations and activation gradients for max_batch rows, an input staging
+ * buffer, per-row losses and status words).  Host-only; no CUDA call. */
+int mpt_workspace_bytes(const mpt_layer_desc *layers, int n_layers, int max_batch,
+                        int use_momentum, size_t *bytes_out);
+
+/* Create a context over a caller-allocated workspace (section 3.1, 3.2: the
+ * iteration's state: master weights, loss scale S, learning rate).
+ *   layers/n_layers  chain of linear layers, out_l == in_{l+1}, last layer relu == 0
+ *   S                constant loss scale, finite, 2^-100 <= S <= 2^120
+ *   lr               learning rate, finite
+ *   momentum         0 <= momentum < 1; 0 selects plain SGD (no momentum buffer)
+ *   max_batch        largest batch later passed to mpt_forward
+ *   workspace_dev    device memory, 256-byte aligned, >= mpt_workspace_bytes(...)
+ *   cuda_stream      a cudaStream_t (may be 0 for the default stream); all work
+ *                    of this context is issued on it
+ * Zeroes the momentum and gradient buffers.  Master weights are undefined until
+ * mpt_set_master has been called for every layer. */
+int mpt_create(const mpt_layer_desc *layers, int n_layers, float S, float lr, float momentum,
+               int max_batch, void *workspace_dev, size_t workspace_bytes, void *cuda_stream,
+               mpt_ctx **out);
+
+/* Upload one layer's FP32 master weights [out, in] from the host and round them
+ * to the FP16 working copy (section 3.1).  n must equal out*in.  Synchronous. */
+int mpt_set_master(mpt_ctx *ctx, int layer, const float *src_host, size_t n);
+
+/* Forward pass (section 3.3): for l = 1..L
+ *   a_l[i,j] = rn16( act( sum_k a_{l-1}[i,k] * w16_l[j,k] ) ), sum in FP32.
+ * x_dev: FP16 [batch, in_1] with row pitch in_1, read-only, caller-owned; it must
+ * stay valid and unchanged until the stream work of the following
+ * mpt_backward_scaled has completed (the first layer's weight gradient reads it).
+ * 1 <= batch <= max_batch.  The logits are a_L (MPT_T_ACT16, layer L-1). */
+int mpt_forward(mpt_ctx *ctx, const uint16_t *x_dev, int batch);
+
+/* Scaled backward pass (sections 3.2, 3.3).  Softmax cross-entropy over the
+ * logits in FP32: loss = mean_i (logsumexp(z_i) - z_i[y_i]), logit gradient
+ * dz_L = rn16((softmax(z_i) - onehot(y_i)) * S / batch); then for l = L..1
+ *   gW_l[j,k]   = rn16( sum_i dz_l[i,j] * a_{l-1}[i,k] )
+ *   dz_{l-1}[i,k] = [a_{l-1}[i,k] > 0] * rn16( sum_j dz_l[i,j] * w16_l[j,k] )  (l > 1)
+ * The gradient buffers are overwritten, not accumulated into.
+ * labels_dev: int32 [batch] on the device.  A label outside [0, C) contributes
+ * neither loss nor gradient; it is reported as MPT_ERR_INVALID_ARG by the next
+ * call that synchronises.  loss_host_or_null: if non-null the stream is
+ * synchronised and the unscaled mean loss is stored.  MPT_ERR_STATE if no
+ * mpt_forward preceded it. */
+int mpt_backward_scaled(mpt_ctx *ctx, const int32_t *labels_dev, float *loss_host_or_null);
+
+/* Master-weight pass (sections 3.1, 3.2).  With inv = 1.0f / S (one FP32 division on
+ * the host): overflow = any element of any layer with non-finite f32(gW) * inv.
+ * If overflow: nothing is modified.  Otherwise, per element, each operation rounded
+ * separately in FP32 (no fused multiply-add):
+ *   g = f32(gW) * inv ; [momentum: v = mu*v + g ; u = lr*v]  [plain: u = lr*g]
+ *   w32 = w32 - u ; w16 = rn16(w32)
+ * The skip decision is taken on the device.  overflow_host_or_null: if non-null
+ * the stream is synchronised and 0/1 is stored.  Overflow is not an error: the
+ * return value stays MPT_OK. */
+int mpt_step(mpt_ctx *ctx, int *overflow_host_or_null);
+
+/* Download one layer's FP32 master weights [out, in] (section 3.1).  Synchronous. */
+int mpt_get_master(mpt_ctx *ctx, int layer, float *dst_host, size_t n);
+
+/* One whole iteration from HOST buffers (figure 1 / section 3.1-3.2 in sequence):
+ * copies x_host (FP16 [batch, in_1]) and labels_host (int32 [batch]) to the device
+ * staging area, runs mpt_forward, mpt_backward_scaled and mpt_step, and returns
+ * the loss and the overflow flag.  Synchronises the stream before returning. */
+int mpt_train_step_host(mpt_ctx *ctx, const uint16_t *x_host, const int32_t *labels_host, int batch,
+                        float *loss_host, int *overflow_host);
+
+/* Change the loss scale (section 3.2) / learning rate; takes effect at the next
+ * mpt_backward_scaled / mpt_step.  Same range checks as mpt_create. */
+int mpt_set_scale(mpt_ctx *ctx, float S);
+int mpt_set_lr(mpt_ctx *ctx, float lr);
+
+/* Test and checkpoint hooks.  mpt_get_tensor downloads an internal tensor without
+ * padding (bytes must equal rows*cols*element size; ACT16/DACT16 use the batch of
+ * the last forward; ACT16 layer l is a_{l+1}, the output of layer l).
+ * mpt_set_grad overwrites one layer's FP16 weight gradient and refreshes the
+ * device overflow flag over all layers.  mpt_set_momentum uploads an FP32
+ * momentum buffer (checkpoint restore).  All synchronous. */
+int mpt_get_tensor(mpt_ctx *ctx, int kind, int layer, void *dst_host, size_t bytes);
+int mpt_set_grad(mpt_ctx *ctx, int layer, const uint16_t *src_host, size_t n);
+int mpt_set_momentum(mpt_ctx *ctx, int layer, const float *src_host, size_t n);
+
+/* Number of kernels this context has launched since creation (bookkeeping for
+ * benchmarks). */
+int mpt_launch_count(mpt_ctx *ctx, long long *count_out);
+
+/* Message for the last non-OK status of this context (never null). */
+const char *mpt_last_error(mpt_ctx *ctx);
+
+/* Releases the host-side context.  Does not touch device memory. */
+void mpt_destroy(mpt_ctx *ctx);
+
+/* ------------------------------------------------- stateless kernel launchers */
+
+/* One FP16 product with FP32 accumulation and FP16 store (section 3.3).
+ * op selects the stored layouts (see MPT_OP_*).  lda/ldb/ldc/ldmask are row
+ * pitches in elements.  mask_dev (may be null): FP16 [M,N]; outputs where the
+ * stored value is not > 0 are written as +0 (ReLU derivative from the stored
+ * activation).  nonfinite_flag_dev (may be null): a uint32 that is OR-ed with 1 if
+ * any stored output is inf or NaN (section 3.2: overflow shows up in the weight
+ * gradients).  The tcgen05 kernel needs 16-byte aligned base pointers and pitches
+ * that are multiples of 8 elements; other operands run on the CUDA-core kernel.
+ * Results do not depend on the launch and are run-to-run identical.
+ * status_dev: device uint32[4] scratch the kernel writes its error word into
+ * (index 0: 0 = fine, else a timeout code); may be null to skip reporting. */
+int mpt_gemm_f16(int op, int M, int N, int K, const uint16_t *A_dev, int lda, const uint16_t *B_dev,
+                 int ldb, uint16_t *C_dev, int ldc, unsigned flags, const uint16_t *mask_dev,
+                 int ldmask, uint32_t *nonfinite_flag_dev, uint32_t *status_dev, void *cuda_stream);
+
+/* w16[e] = rn16(w32[e]) (section 3.1: the FP16 copy is made by rounding). */
+int mpt_recast(const float *w32_dev, uint16_t *w16_dev, size_t n, void *cuda_stream);
+
+/* Overflow inspection alone (section 3.2): *flag_dev |= 1 if any f32(g16[e]) * inv_S
+ * is inf/NaN.  flag_dev must have been zeroed by the caller. */
+int mpt_grad_nonfinite(const uint16_t *g16_dev, size_t n, float inv_S, uint32_t *flag_dev,
+                       void *cuda_stream);
+
+/* Master-weight pass over flat arrays (sections 3.1, 3.2), arithmetic as in mpt_step.
+ * flags_dev: device uint32[2] scratch.  If detect != 0 the call first zeroes
+ * flags_dev[0] and runs the inspection over g16 (an extra 2 bytes/element read);
+ * if detect == 0 the caller has already produced flags_dev[0].  The update kernel
+ * returns at once when flags_dev[0] != 0, otherwise updates in a single pass that
+ * reads g16, w32, (v) once and writes w32, (v), w16 once, and stores its own
+ * inspection result in flags_dev[1].  v_dev may be null iff use_momentum == 0. */
+int mpt_update_flat(const uint16_t *g16_dev, float *w32_dev, float *v_dev, uint16_t *w16_dev, size_t n,
+                    float inv_S, float lr, float mu, int use_momentum, int detect, uint32_t *flags_dev,
+                    void *cuda_stream);
+
+/* Softmax cross-entropy forward and scaled backward (sections 3.2, 3.3), arithmetic
+ * as in mpt_backward_scaled.  z_dev/dz_dev: FP16 [B, C] with pitches ldz/lddz
+ * (the two must not overlap).  row_loss_dev: float [B] scratch; loss_dev: one float,
+ * receives the unscaled mean; bad_labels_dev: one uint32, receives the number of
+ * labels outside [0, C) (may be null). */
+int mpt_softmax_ce(const uint16_t *z_dev, int ldz, const int32_t *labels_dev, int B, int C, float S,
+                   uint16_t *dz_dev, int lddz, float *row_loss_dev, float *loss_dev,
+                   uint32_t *bad_labels_dev, void *cuda_stream);
+
+/* Library build identification, e.g. "mpt 0.1 sm_100a". */
+const char *mpt_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MPT_H_ */

@@ -1,0 +1,254 @@
+"""Thin ctypes binding over libmpt.so (the C ABI declared in include/mpt.h).
+
+Argument marshalling only: every arithmetic step runs in the CUDA library.  PyTorch
+is used for device memory (the workspace and the tensors handed in) and streams.
+There is no fallback: if the shared library is missing or a call fails, an
+exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmpt.so")
+
+OK = 0
+ERR = {-1: "MPT_ERR_INVALID_ARG", -2: "MPT_ERR_SHAPE", -3: "MPT_ERR_STATE", -4: "MPT_ERR_WORKSPACE",
+       -5: "MPT_ERR_CUDA", -6: "MPT_ERR_TIMEOUT", -7: "MPT_ERR_INTERNAL"}
+OP_FWD, OP_DGRAD, OP_WGRAD = 0, 1, 2
+GEMM_RELU, GEMM_FORCE_SIMT, GEMM_FORCE_TC = 1, 2, 4
+T_W16, T_GRAD16, T_ACT16, T_DACT16, T_MOMENTUM32, T_MASTER32 = range(6)
+
+# every symbol include/mpt.h declares
+EXPORTS = ["mpt_workspace_bytes", "mpt_create", "mpt_set_master", "mpt_forward", "mpt_backward_scaled",
+           "mpt_step", "mpt_get_master", "mpt_train_step_host", "mpt_set_scale", "mpt_set_lr",
+           "mpt_get_tensor", "mpt_set_grad", "mpt_set_momentum", "mpt_launch_count", "mpt_last_error",
+           "mpt_destroy", "mpt_gemm_f16", "mpt_recast", "mpt_grad_nonfinite", "mpt_update_flat",
+           "mpt_softmax_ce", "mpt_version"]
+
+
+class MptError(RuntimeError):
+    def __init__(self, code, msg=""):
+        self.code = code
+        super().__init__("%s (%d) %s" % (ERR.get(code, "MPT_ERR_?"), code, msg))
+
+
+class LayerDesc(C.Structure):
+    _fields_ = [("in_features", C.c_int32), ("out_features", C.c_int32), ("relu", C.c_int32)]
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Load libmpt.so; raises if it has not been built (python -m paper_1710_03740_b200.build)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError("CUDA library %s not found: run `python -m paper_1710_03740_b200.build`" % LIB_PATH)
+    L = C.CDLL(LIB_PATH)
+    vp, i32, u32, f32, sz = C.c_void_p, C.c_int, C.c_uint, C.c_float, C.c_size_t
+    L.mpt_workspace_bytes.argtypes = [C.POINTER(LayerDesc), i32, i32, i32, C.POINTER(sz)]
+    L.mpt_create.argtypes = [C.POINTER(LayerDesc), i32, f32, f32, f32, i32, vp, sz, vp, C.POINTER(vp)]
+    L.mpt_set_master.argtypes = [vp, i32, vp, sz]
+    L.mpt_forward.argtypes = [vp, vp, i32]
+    L.mpt_backward_scaled.argtypes = [vp, vp, C.POINTER(f32)]
+    L.mpt_step.argtypes = [vp, C.POINTER(i32)]
+    L.mpt_get_master.argtypes = [vp, i32, vp, sz]
+    L.mpt_train_step_host.argtypes = [vp, vp, vp, i32, C.POINTER(f32), C.POINTER(i32)]
+    L.mpt_set_scale.argtypes = [vp, f32]
+    L.mpt_set_lr.argtypes = [vp, f32]
+    L.mpt_get_tensor.argtypes = [vp, i32, i32, vp, sz]
+    L.mpt_set_grad.argtypes = [vp, i32, vp, sz]
+    L.mpt_set_momentum.argtypes = [vp, i32, vp, sz]
+    L.mpt_launch_count.argtypes = [vp, C.POINTER(C.c_longlong)]
+    L.mpt_last_error.argtypes = [vp]
+    L.mpt_last_error.restype = C.c_char_p
+    L.mpt_destroy.argtypes = [vp]
+    L.mpt_destroy.restype = None
+    L.mpt_gemm_f16.argtypes = [i32, i32, i32, i32, vp, i32, vp, i32, vp, i32, u32, vp, i32, vp, vp, vp]
+    L.mpt_recast.argtypes = [vp, vp, sz, vp]
+    L.mpt_grad_nonfinite.argtypes = [vp, sz, f32, vp, vp]
+    L.mpt_update_flat.argtypes = [vp, vp, vp, vp, sz, f32, f32, f32, i32, i32, vp, vp]
+    L.mpt_softmax_ce.argtypes = [vp, i32, vp, i32, i32, f32, vp, i32, vp, vp, vp, vp]
+    L.mpt_version.restype = C.c_char_p
+    L.mpt_version.argtypes = []
+    _lib = L
+    return L
+
+
+def _check(code, ctx=None):
+    if code != OK:
+        msg = ""
+        if ctx:
+            msg = lib().mpt_last_error(ctx).decode()
+        raise MptError(code, msg)
+
+
+def _stream_ptr(stream=None):
+    import torch
+    s = torch.cuda.current_stream() if stream is None else stream
+    return C.c_void_p(s.cuda_stream)
+
+
+def _dptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _hptr(a):
+    """Host pointer of a numpy array or a CPU torch tensor."""
+    if isinstance(a, np.ndarray):
+        return C.c_void_p(a.ctypes.data)
+    return C.c_void_p(a.data_ptr())
+
+
+def _layer_array(layers):
+    arr = (LayerDesc * len(layers))()
+    for k, (i, o, r) in enumerate(layers):
+        arr[k].in_features, arr[k].out_features, arr[k].relu = int(i), int(o), int(r)
+    return arr
+
+
+def mpt_workspace_bytes(layers, max_batch, use_momentum) -> int:
+    out = C.c_size_t(0)
+    _check(lib().mpt_workspace_bytes(_layer_array(layers), len(layers), int(max_batch), int(bool(use_momentum)),
+                                     C.byref(out)))
+    return int(out.value)
+
+
+class Context:
+    """One mpt_ctx over a torch-allocated workspace.  Method names follow the C calls."""
+
+    def __init__(self, layers, S, lr, momentum=0.0, max_batch=1, device="cuda:0", stream=None):
+        import torch
+        self.layers = [(int(i), int(o), int(r)) for (i, o, r) in layers]
+        self.device = torch.device(device)
+        self.stream = stream
+        nbytes = mpt_workspace_bytes(self.layers, max_batch, momentum != 0.0)
+        with torch.cuda.device(self.device):
+            self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
+            base = self.workspace.data_ptr()
+            self._ws_ptr = (base + 255) // 256 * 256
+            self._ctx = C.c_void_p()
+            _check(lib().mpt_create(_layer_array(self.layers), len(self.layers), float(S), float(lr), float(momentum),
+                                    int(max_batch), C.c_void_p(self._ws_ptr), nbytes, _stream_ptr(stream),
+                                    C.byref(self._ctx)))
+        self.workspace_bytes = nbytes
+        self.batch = 0
+
+    def close(self):
+        if getattr(self, "_ctx", None):
+            lib().mpt_destroy(self._ctx)
+            self._ctx = None
+
+    __del__ = close
+
+    def set_master(self, layer, w32):
+        w = np.ascontiguousarray(w32, dtype=np.float32)
+        _check(lib().mpt_set_master(self._ctx, layer, _hptr(w), w.size), self._ctx)
+
+    def get_master(self, layer):
+        i, o, _ = self.layers[layer]
+        out = np.empty((o, i), dtype=np.float32)
+        _check(lib().mpt_get_master(self._ctx, layer, _hptr(out), out.size), self._ctx)
+        return out
+
+    def forward(self, x_dev):
+        """x_dev: torch float16 CUDA tensor [batch, in_1], contiguous; kept alive by the caller."""
+        assert x_dev.is_cuda and x_dev.is_contiguous() and x_dev.element_size() == 2
+        self.batch = int(x_dev.shape[0])
+        _check(lib().mpt_forward(self._ctx, _dptr(x_dev), self.batch), self._ctx)
+
+    def backward_scaled(self, labels_dev, want_loss=True):
+        assert labels_dev.is_cuda and labels_dev.is_contiguous() and labels_dev.element_size() == 4
+        if want_loss:
+            loss = C.c_float(0.0)
+            _check(lib().mpt_backward_scaled(self._ctx, _dptr(labels_dev), C.byref(loss)), self._ctx)
+            return float(loss.value)
+        _check(lib().mpt_backward_scaled(self._ctx, _dptr(labels_dev), None), self._ctx)
+        return None
+
+    def step(self, want_flag=True):
+        if want_flag:
+            flag = C.c_int(0)
+            _check(lib().mpt_step(self._ctx, C.byref(flag)), self._ctx)
+            return int(flag.value)
+        _check(lib().mpt_step(self._ctx, None), self._ctx)
+        return None
+
+    def train_step_host(self, x_host, labels_host):
+        """x_host: float16/uint16 [batch, in_1] host array (numpy or pinned torch); labels int32 [batch]."""
+        batch = int(x_host.shape[0])
+        loss, flag = C.c_float(0.0), C.c_int(0)
+        _check(lib().mpt_train_step_host(self._ctx, _hptr(x_host), _hptr(labels_host), batch, C.byref(loss),
+                                         C.byref(flag)), self._ctx)
+        self.batch = batch
+        return float(loss.value), int(flag.value)
+
+    def set_scale(self, S):
+        _check(lib().mpt_set_scale(self._ctx, float(S)), self._ctx)
+
+    def set_lr(self, lr):
+        _check(lib().mpt_set_lr(self._ctx, float(lr)), self._ctx)
+
+    def get_tensor(self, kind, layer):
+        i, o, _ = self.layers[layer]
+        if kind in (T_W16, T_GRAD16):
+            out = np.empty((o, i), dtype=np.uint16)
+        elif kind in (T_MOMENTUM32, T_MASTER32):
+            out = np.empty((o, i), dtype=np.float32)
+        else:
+            out = np.empty((self.batch, o), dtype=np.uint16)
+        _check(lib().mpt_get_tensor(self._ctx, kind, layer, _hptr(out), out.nbytes), self._ctx)
+        return out
+
+    def set_grad(self, layer, g16):
+        g = np.ascontiguousarray(g16)
+        if g.dtype == np.float16:
+            g = g.view(np.uint16)
+        assert g.dtype == np.uint16
+        _check(lib().mpt_set_grad(self._ctx, layer, _hptr(g), g.size), self._ctx)
+
+    def set_momentum(self, layer, v):
+        v = np.ascontiguousarray(v, dtype=np.float32)
+        _check(lib().mpt_set_momentum(self._ctx, layer, _hptr(v), v.size), self._ctx)
+
+    def launch_count(self):
+        n = C.c_longlong(0)
+        _check(lib().mpt_launch_count(self._ctx, C.byref(n)), self._ctx)
+        return int(n.value)
+
+
+# ------------------------------------------------------------ stateless calls
+
+def mpt_gemm_f16(op, M, N, K, A, lda, B, ldb, Cout, ldc, flags=0, mask=None, ldmask=0, nonfinite_flag=None,
+                 status=None, stream=None):
+    """Arguments are torch CUDA tensors (any 2-byte dtype) used as raw device pointers."""
+    _check(lib().mpt_gemm_f16(op, M, N, K, _dptr(A), lda, _dptr(B), ldb, _dptr(Cout), ldc, flags, _dptr(mask), ldmask,
+                              _dptr(nonfinite_flag), _dptr(status), _stream_ptr(stream)))
+
+
+def mpt_recast(w32, w16, n, stream=None):
+    _check(lib().mpt_recast(_dptr(w32), _dptr(w16), n, _stream_ptr(stream)))
+
+
+def mpt_grad_nonfinite(g16, n, inv_S, flag, stream=None):
+    _check(lib().mpt_grad_nonfinite(_dptr(g16), n, float(inv_S), _dptr(flag), _stream_ptr(stream)))
+
+
+def mpt_update_flat(g16, w32, v, w16, n, inv_S, lr, mu, use_momentum, detect, flags, stream=None):
+    _check(lib().mpt_update_flat(_dptr(g16), _dptr(w32), _dptr(v), _dptr(w16), n, float(inv_S), float(lr), float(mu),
+                                 int(bool(use_momentum)), int(bool(detect)), _dptr(flags), _stream_ptr(stream)))
+
+
+def mpt_softmax_ce(z, ldz, labels, B, Cn, S, dz, lddz, row_loss, loss, bad_labels=None, stream=None):
+    _check(lib().mpt_softmax_ce(_dptr(z), ldz, _dptr(labels), B, Cn, float(S), _dptr(dz), lddz, _dptr(row_loss),
+                                _dptr(loss), _dptr(bad_labels), _stream_ptr(stream)))
+
+
+def mpt_version() -> str:
+    return lib().mpt_version().decode()

@@ -1,0 +1,485 @@
+// Tensor-core FP16 GEMM for sm_100a (paper section 3.3: FP16 operands, FP32
+// accumulation, FP16 on the store), with the point-wise work fused into the
+// epilogue (ReLU, the ReLU-derivative mask of the backward pass, and the inf/NaN
+// inspection of weight gradients of section 3.2).
+//
+// Structure: persistent kernel, one CTA per SM, 192 threads in three roles
+//   warp 0      TMA producer: cp.async.bulk.tensor loads of 128x64 (A) and 256x64 (B)
+//               FP16 tiles into a 4-stage shared-memory ring (128-byte swizzle)
+//   warp 1      MMA issuer: tcgen05.mma.kind::f16, 128x256x16 per instruction,
+//               FP32 accumulators in tensor memory (2 x 256 columns, double buffered)
+//   warps 2..5  epilogue: tcgen05.ld the accumulator, ReLU / mask / round to FP16 /
+//               inspect, 128-bit stores to C
+// Operand layouts are taken as stored (no transposed copies): a "K-major" operand has
+// the contraction index contiguous, an "MN-major" operand has the output index
+// contiguous; the forward product is K x K, dgrad is K x MN, wgrad is MN x MN.
+// Ragged M, N, K are handled by TMA zero fill on loads and by predicated stores.
+//
+// Every wait on an mbarrier is bounded: after ~2 s the waiting role records an error
+// word, raises a CTA-wide abort flag and all roles fall through to the common exit,
+// which frees the tensor memory.
+#include <cuda.h>
+
+#include "mpt_common.cuh"
+
+namespace mpt {
+
+static constexpr int BLOCK_M = 128, BLOCK_N = 256, BLOCK_K = 64, UMMA_K = 16, STAGES = 4;
+static constexpr int A_STAGE_BYTES = BLOCK_M * BLOCK_K * 2;  // 16 KB
+static constexpr int B_STAGE_BYTES = BLOCK_N * BLOCK_K * 2;  // 32 KB
+static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+static constexpr int MN_BOX_BYTES = 64 * BLOCK_K * 2;        // one 64(mn) x 64(k) box of an MN-major operand
+static constexpr int TMEM_COLS = 512;
+static constexpr int NUM_THREADS = 192;
+static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+static constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
+
+// ----------------------------------------------------------------- PTX wrappers
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok;
+}
+__device__ __forceinline__ unsigned long long global_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Bounded wait.  Returns false when the CTA is aborting or the time limit expired.
+__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag)
+{
+    unsigned long long t0 = 0;
+    for (uint32_t it = 0;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 127u) == 127u) {
+            if (*abort_flag) return false;
+            unsigned long long now = global_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > WAIT_LIMIT_NS) return false;
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tc_mma_f16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                           uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor (tcgen05): start address, leading/stride byte
+// offsets (all >> 4), descriptor version 1, 128-byte swizzle.
+//   K-major  operand: rows of 128 bytes (64 k), 8-row groups 1024 bytes apart (stride offset);
+//                     the leading offset is unused with swizzling.
+//   MN-major operand: 64 k-rows of 128 bytes (64 mn) per box, 8-k groups 1024 bytes apart
+//                     (stride offset), the next 64 mn one box (8192 bytes) further (leading offset).
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+    d |= (uint64_t)1 << 46;  // descriptor version (Blackwell)
+    d |= (uint64_t)2 << 61;  // SWIZZLE_128B
+    return d;
+}
+
+// Instruction descriptor, kind::f16: D = F32, A = B = F16, majors, N >> 3, M >> 4.
+__host__ __device__ constexpr uint32_t make_idesc(bool a_mn, bool b_mn)
+{
+    return (1u << 4) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) | ((uint32_t)(BLOCK_N >> 3) << 17) |
+           ((uint32_t)(BLOCK_M >> 4) << 24);
+}
+
+struct TcParams {
+    int M, N, K;
+    uint16_t *C;
+    int ldc;
+    const uint16_t *mask;
+    int ldmask;
+    int relu;
+    uint32_t *nonfinite_flag;
+    uint32_t *status;  // may be null
+    int tiles_m, tiles_n, group_m;
+};
+
+__device__ __forceinline__ void tile_coords(const TcParams &p, int tile, int &mb, int &nb)
+{
+    // groups of group_m row-blocks, row-block fastest inside a group: concurrently
+    // running CTAs share B tiles and a bounded set of A tiles in L2
+    int per_group = p.group_m * p.tiles_n;
+    int g = tile / per_group;
+    int first_m = g * p.group_m;
+    int gsz = min(p.group_m, p.tiles_m - first_m);
+    int r = tile - g * per_group;
+    mb = first_m + r % gsz;
+    nb = r / gsz;
+}
+
+__device__ __forceinline__ void report(const TcParams &p, volatile uint32_t *abort_flag, uint32_t code)
+{
+    *abort_flag = 1u;
+    if (p.status) atomicCAS(p.status, 0u, code | ((uint32_t)blockIdx.x << 8));
+}
+
+template <bool A_MN, bool B_MN>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;   // swizzled tiles need 1024-byte alignment
+    uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
+    const uint32_t bars = base + STAGES * STAGE_BYTES;
+    // barrier words: full[STAGES], empty[STAGES], acc_full[2], acc_empty[2], then tmem slot + abort flag
+    auto full_bar = [&](int s) { return bars + 8u * s; };
+    auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
+    auto accf_bar = [&](int b) { return bars + 8u * (2 * STAGES + b); };
+    auto acce_bar = [&](int b) { return bars + 8u * (2 * STAGES + 2 + b); };
+    volatile uint32_t *tmem_slot = (volatile uint32_t *)(base_ptr + STAGES * STAGE_BYTES + 8 * (2 * STAGES + 4));
+    volatile uint32_t *abort_flag = tmem_slot + 1;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int num_tiles = p.tiles_m * p.tiles_n;
+    const int nkb = (p.K + BLOCK_K - 1) / BLOCK_K;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; s++) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int b = 0; b < 2; b++) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), 4); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void *)tmem_slot)),
+                     "r"((uint32_t)TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t issued = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+                int mb, nb;
+                tile_coords(p, tile, mb, nb);
+                const int m0 = mb * BLOCK_M, n0 = nb * BLOCK_N;
+                for (int kb = 0; kb < nkb; kb++, issued++) {
+                    const int s = issued % STAGES;
+                    const uint32_t ph = (issued / STAGES) & 1u;
+                    if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) {
+                        if (!*abort_flag) report(p, abort_flag, KERR_WAIT_EMPTY);
+                        ok = false;
+                        break;
+                    }
+                    const uint32_t sa = base + s * STAGE_BYTES, sb = sa + A_STAGE_BYTES;
+                    mbar_arrive_expect_tx(full_bar(s), STAGE_BYTES);
+                    const int k0 = kb * BLOCK_K;
+                    if (A_MN) {
+#pragma unroll
+                        for (int j = 0; j < BLOCK_M / 64; j++) tma_load_2d(sa + j * MN_BOX_BYTES, &tmA, m0 + 64 * j, k0, full_bar(s));
+                    } else {
+                        tma_load_2d(sa, &tmA, k0, m0, full_bar(s));
+                    }
+                    if (B_MN) {
+#pragma unroll
+                        for (int j = 0; j < BLOCK_N / 64; j++) tma_load_2d(sb + j * MN_BOX_BYTES, &tmB, n0 + 64 * j, k0, full_bar(s));
+                    } else {
+                        tma_load_2d(sb, &tmB, k0, n0, full_bar(s));
+                    }
+                }
+            }
+            if (!ok) {
+                // let the copies already in flight land before the CTA exits (bounded)
+                uint32_t first = issued > (uint32_t)STAGES ? issued - STAGES : 0;
+                for (uint32_t i = first; i < issued; i++) {
+                    unsigned long long t0 = global_ns();
+                    while (!mbar_try_wait(full_bar(i % STAGES), (i / STAGES) & 1u) && global_ns() - t0 < 1000000ull) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // -------------------------------------------------------------- MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc(A_MN, B_MN);
+            uint32_t consumed = 0;
+            bool ok = true;
+            int t = 0;
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, t++) {
+                const int buf = t & 1;
+                const uint32_t acc_ph = (t >> 1) & 1u;
+                if (!mbar_wait(acce_bar(buf), acc_ph ^ 1u, abort_flag)) {
+                    if (!*abort_flag) report(p, abort_flag, KERR_WAIT_ACC_FREE);
+                    ok = false;
+                    break;
+                }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BLOCK_N);
+                for (int kb = 0; kb < nkb; kb++, consumed++) {
+                    const int s = consumed % STAGES;
+                    const uint32_t ph = (consumed / STAGES) & 1u;
+                    if (!mbar_wait(full_bar(s), ph, abort_flag)) {
+                        if (!*abort_flag) report(p, abort_flag, KERR_WAIT_FULL);
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint32_t sa = base + s * STAGE_BYTES, sb = sa + A_STAGE_BYTES;
+#pragma unroll
+                    for (int k = 0; k < BLOCK_K / UMMA_K; k++) {
+                        // K-major: 16 k = 32 bytes along the swizzled row; MN-major: 16 k-rows of 128 bytes
+                        const uint64_t ad = A_MN ? make_desc(sa + k * (UMMA_K * 128), MN_BOX_BYTES, 1024)
+                                                 : make_desc(sa + k * (UMMA_K * 2), 16, 1024);
+                        const uint64_t bd = B_MN ? make_desc(sb + k * (UMMA_K * 128), MN_BOX_BYTES, 1024)
+                                                 : make_desc(sb + k * (UMMA_K * 2), 16, 1024);
+                        tc_mma_f16(d_tmem, ad, bd, idesc, (kb | k) != 0 ? 1u : 0u);
+                    }
+                    tc_commit(empty_bar(s));       // frees the stage when these MMAs have read it
+                }
+                if (ok) tc_commit(accf_bar(buf));  // accumulator complete
+            }
+        }
+    } else {
+        // ---------------------------------------------------------------- epilogue
+        const int q = warp & 3;                    // TMEM lane quadrant this warp may access
+        bool ok = true;
+        int t = 0;
+        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, t++) {
+            int mb, nb;
+            tile_coords(p, tile, mb, nb);
+            const int buf = t & 1;
+            const uint32_t acc_ph = (t >> 1) & 1u;
+            if (!mbar_wait(accf_bar(buf), acc_ph, abort_flag)) {
+                if (!*abort_flag && lane == 0) report(p, abort_flag, KERR_WAIT_ACC);
+                ok = false;
+                break;
+            }
+            tc_fence_after();
+            const int row = mb * BLOCK_M + q * 32 + lane;
+            const bool row_ok = row < p.M;
+            uint16_t *crow = p.C + (size_t)row * p.ldc;
+            const uint16_t *mrow = p.mask ? p.mask + (size_t)row * p.ldmask : nullptr;
+            bool bad = false;
+#pragma unroll 1
+            for (int c = 0; c < BLOCK_N / 32; c++) {
+                uint32_t r[32];
+                tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BLOCK_N + c * 32), r);
+                tc_wait_ld();
+                const int col0 = nb * BLOCK_N + c * 32;
+                if (row_ok && col0 < p.N) {
+#pragma unroll
+                    for (int g8 = 0; g8 < 4; g8++) {
+                        const int col = col0 + g8 * 8;
+                        uint32_t h[8];
+#pragma unroll
+                        for (int e = 0; e < 8; e++) {
+                            float s = __uint_as_float(r[g8 * 8 + e]);
+                            if (p.relu) s = (s > 0.0f || s != s) ? s : 0.0f;
+                            h[e] = (uint32_t)__half_as_ushort(__float2half_rn(s));
+                        }
+                        if (col + 8 <= p.N) {
+                            if (mrow) {
+                                uint4 mk = *(const uint4 *)(mrow + col);
+                                uint32_t mw[4] = {mk.x, mk.y, mk.z, mk.w};
+#pragma unroll
+                                for (int e = 0; e < 8; e++) {
+                                    uint32_t mh = (e & 1) ? (mw[e >> 1] >> 16) : (mw[e >> 1] & 0xFFFFu);
+                                    // stored activation > 0  <=>  sign clear, non-zero, not NaN
+                                    bool keep = (mh & 0x8000u) == 0 && mh != 0 && mh <= 0x7C00u;
+                                    if (!keep) h[e] = 0;
+                                }
+                            }
+#pragma unroll
+                            for (int e = 0; e < 8; e++) bad |= half_bits_nonfinite(h[e]);
+                            uint4 o = make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), h[4] | (h[5] << 16),
+                                                 h[6] | (h[7] << 16));
+                            *(uint4 *)(crow + col) = o;
+                        } else {
+                            for (int e = 0; e < 8 && col + e < p.N; e++) {
+                                uint32_t v = h[e];
+                                if (mrow) {
+                                    uint32_t mh = mrow[col + e];
+                                    bool keep = (mh & 0x8000u) == 0 && mh != 0 && mh <= 0x7C00u;
+                                    if (!keep) v = 0;
+                                }
+                                bad |= half_bits_nonfinite(v);
+                                crow[col + e] = (uint16_t)v;
+                            }
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acce_bar(buf));
+            if (p.nonfinite_flag && __any_sync(0xFFFFFFFFu, bad) && lane == 0) atomicOr(p.nonfinite_flag, 1u);
+        }
+    }
+
+    // common exit: every role gets here (all waits are bounded)
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS) : "memory");
+    }
+}
+
+// ------------------------------------------------------------------ host side
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn get_encode()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)sym;
+    }
+    return fn;
+}
+
+// 2-D FP16 tensor map over a row-major matrix [rows, cols] with pitch ld (elements);
+// box = box_cols x box_rows, 128-byte swizzle, zero fill outside the matrix.
+static bool encode_map(CUtensorMap *map, const void *ptr, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_cols,
+                       uint32_t box_rows)
+{
+    EncodeTiledFn fn = get_encode();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {ld * 2};
+    cuuint32_t box[2] = {box_cols, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void *>(ptr), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+bool tc_gemm_supported(int op, int M, int N, int K, const void *A, int lda, const void *B, int ldb, const void *C,
+                       int ldc, const void *mask, int ldmask)
+{
+    (void)op;
+    if (M <= 0 || N <= 0 || K <= 0) return false;
+    uintptr_t bits = (uintptr_t)A | (uintptr_t)B | (uintptr_t)C | (uintptr_t)mask;
+    if (bits & 15) return false;
+    if ((lda % 8) || (ldb % 8) || (ldc % 8) || (mask && (ldmask % 8))) return false;
+    return true;
+}
+
+template <bool A_MN, bool B_MN>
+static cudaError_t launch_variant(const CUtensorMap &ta, const CUtensorMap &tb, const TcParams &p, int grid,
+                                  cudaStream_t st)
+{
+    static bool configured = false;
+    auto kern = k_gemm_tc<A_MN, B_MN>;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    kern<<<grid, NUM_THREADS, SMEM_BYTES, st>>>(ta, tb, p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_gemm_tc(int op, int M, int N, int K, const uint16_t *A, int lda, const uint16_t *B, int ldb,
+                           uint16_t *C, int ldc, bool relu, const uint16_t *mask, int ldmask, uint32_t *nonfinite_flag,
+                           uint32_t *status, cudaStream_t st)
+{
+    CUtensorMap ta, tb;
+    bool ok;
+    // A: stored [M,K] (K-major) for fwd/dgrad, stored [K,M] (MN-major) for wgrad
+    if (op == MPT_OP_WGRAD) ok = encode_map(&ta, A, (uint64_t)K, (uint64_t)M, (uint64_t)lda, 64, BLOCK_K);
+    else ok = encode_map(&ta, A, (uint64_t)M, (uint64_t)K, (uint64_t)lda, BLOCK_K, BLOCK_M);
+    // B: stored [N,K] (K-major) for fwd, stored [K,N] (MN-major) for dgrad/wgrad
+    if (op == MPT_OP_FWD) ok = ok && encode_map(&tb, B, (uint64_t)N, (uint64_t)K, (uint64_t)ldb, BLOCK_K, BLOCK_N);
+    else ok = ok && encode_map(&tb, B, (uint64_t)K, (uint64_t)N, (uint64_t)ldb, 64, BLOCK_K);
+    if (!ok) return cudaErrorInvalidValue;
+
+    TcParams p;
+    p.M = M; p.N = N; p.K = K;
+    p.C = C; p.ldc = ldc;
+    p.mask = mask; p.ldmask = ldmask;
+    p.relu = relu ? 1 : 0;
+    p.nonfinite_flag = nonfinite_flag;
+    p.status = status;
+    p.tiles_m = (M + BLOCK_M - 1) / BLOCK_M;
+    p.tiles_n = (N + BLOCK_N - 1) / BLOCK_N;
+    p.group_m = 16;
+    int tiles = p.tiles_m * p.tiles_n;
+    int grid = tiles < 148 ? tiles : 148;
+    if (op == MPT_OP_FWD) return launch_variant<false, false>(ta, tb, p, grid, st);
+    if (op == MPT_OP_DGRAD) return launch_variant<false, true>(ta, tb, p, grid, st);
+    return launch_variant<true, true>(ta, tb, p, grid, st);
+}
+
+}  // namespace mpt

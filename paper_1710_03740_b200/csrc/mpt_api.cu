@@ -1,0 +1,557 @@
+// C ABI of the library (include/mpt.h): host-side context, workspace carving,
+// launch sequencing of one mixed-precision training iteration (paper sections
+// 3.1-3.3), status handling.  No device memory is allocated here.
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "mpt_common.cuh"
+
+using namespace mpt;
+
+namespace {
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct Layer {
+    int in, out, relu;
+    size_t off;      // element offset of this layer inside the flat parameter arenas
+    size_t n;        // out * in
+    int ld_out;      // row pitch (elements) of a_l / dz_l buffers
+    uint16_t *act;   // a_{l+1}  [max_batch, ld_out]
+    uint16_t *dact;  // dz_{l+1} [max_batch, ld_out]
+};
+
+struct Plan {
+    size_t total = 0, P_pad = 0;
+    size_t off_status = 0, off_master = 0, off_mom = 0, off_w16 = 0, off_g16 = 0, off_x = 0, off_labels = 0,
+           off_rowloss = 0;
+    std::vector<size_t> off_act, off_dact, lay_off;
+    std::vector<int> ld_out;
+};
+
+bool valid_scale(float S)
+{
+    return std::isfinite(S) && S >= 0x1p-100f && S <= 0x1p120f;
+}
+
+int validate_layers(const mpt_layer_desc *layers, int n_layers, int max_batch)
+{
+    if (!layers) return MPT_ERR_INVALID_ARG;
+    if (n_layers < 1 || n_layers > 1024 || max_batch < 1) return MPT_ERR_SHAPE;
+    for (int l = 0; l < n_layers; l++) {
+        if (layers[l].in_features < 1 || layers[l].out_features < 1) return MPT_ERR_SHAPE;
+        if (layers[l].relu != 0 && layers[l].relu != 1) return MPT_ERR_INVALID_ARG;
+        if (l > 0 && layers[l].in_features != layers[l - 1].out_features) return MPT_ERR_SHAPE;
+    }
+    if (layers[n_layers - 1].relu != 0) return MPT_ERR_SHAPE;
+    return MPT_OK;
+}
+
+void make_plan(const mpt_layer_desc *layers, int L, int max_batch, bool mom, Plan &pl)
+{
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    pl.off_status = take(ST_WORDS * sizeof(uint32_t));
+    size_t P = 0;
+    pl.lay_off.resize(L);
+    for (int l = 0; l < L; l++) {
+        pl.lay_off[l] = P;
+        P += align_up((size_t)layers[l].in_features * layers[l].out_features, 128);
+    }
+    pl.P_pad = P;
+    pl.off_master = take(P * 4);
+    pl.off_mom = mom ? take(P * 4) : 0;
+    pl.off_w16 = take(P * 2);
+    pl.off_g16 = take(P * 2);
+    pl.off_act.resize(L); pl.off_dact.resize(L); pl.ld_out.resize(L);
+    for (int l = 0; l < L; l++) {
+        pl.ld_out[l] = (int)align_up((size_t)layers[l].out_features, 8);
+        pl.off_act[l] = take((size_t)max_batch * pl.ld_out[l] * 2);
+    }
+    for (int l = 0; l < L; l++) pl.off_dact[l] = take((size_t)max_batch * pl.ld_out[l] * 2);
+    pl.off_x = take((size_t)max_batch * layers[0].in_features * 2);
+    pl.off_labels = take((size_t)max_batch * 4);
+    pl.off_rowloss = take((size_t)max_batch * 4);
+    pl.total = off;
+}
+
+}  // namespace
+
+struct mpt_ctx {
+    std::vector<Layer> layers;
+    float S, lr, mu;
+    bool use_momentum;
+    int max_batch;
+    cudaStream_t stream;
+    uint8_t *ws;
+    Plan plan;
+    uint32_t *status;
+    float *master, *mom;
+    uint16_t *w16, *g16, *x_stage;
+    int32_t *labels_stage;
+    float *row_loss;
+    const uint16_t *x_cur = nullptr;
+    int batch = 0;
+    bool forward_done = false, have_grads = false, poisoned = false;
+    long long launches = 0;
+    bool disable_tc = false;
+    std::string err;
+};
+
+namespace {
+
+int fail(mpt_ctx *c, int code, const char *fmt, const char *detail = "")
+{
+    char buf[512];
+    snprintf(buf, sizeof buf, fmt, detail);
+    c->err = buf;
+    if (code == MPT_ERR_CUDA || code == MPT_ERR_TIMEOUT) c->poisoned = true;
+    return code;
+}
+
+int cuda_fail(mpt_ctx *c, cudaError_t e, const char *what)
+{
+    char buf[512];
+    snprintf(buf, sizeof buf, "%s: %s", what, cudaGetErrorString(e));
+    c->err = buf;
+    c->poisoned = true;
+    return MPT_ERR_CUDA;
+}
+
+#define CK(call, what)                                            \
+    do {                                                          \
+        cudaError_t e__ = (call);                                 \
+        if (e__ != cudaSuccess) return cuda_fail(c, e__, what);   \
+    } while (0)
+
+int usable(mpt_ctx *c)
+{
+    if (!c) return MPT_ERR_INVALID_ARG;
+    if (c->poisoned) return MPT_ERR_STATE;
+    return MPT_OK;
+}
+
+// One product of the iteration, on the tensor-core kernel when the operands allow it.
+int gemm(mpt_ctx *c, int op, int M, int N, int K, const uint16_t *A, int lda, const uint16_t *B, int ldb, uint16_t *C,
+         int ldc, bool relu, const uint16_t *mask, int ldmask, uint32_t *nonfinite)
+{
+    cudaError_t e;
+    if (!c->disable_tc && tc_gemm_supported(op, M, N, K, A, lda, B, ldb, C, ldc, mask, ldmask))
+        e = launch_gemm_tc(op, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite,
+                           c->status + ST_KERNEL_ERR, c->stream);
+    else
+        e = launch_gemm_simt(op, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite, c->stream);
+    c->launches++;
+    if (e != cudaSuccess) return cuda_fail(c, e, "gemm launch");
+    return MPT_OK;
+}
+
+// After a stream synchronisation: read the status block once and turn device-side
+// conditions into return codes.
+int read_status(mpt_ctx *c, uint32_t (&st)[ST_WORDS])
+{
+    CK(cudaMemcpyAsync(st, c->status, sizeof st, cudaMemcpyDeviceToHost, c->stream), "status copy");
+    CK(cudaStreamSynchronize(c->stream), "stream synchronize");
+    if (st[ST_KERNEL_ERR] != 0) {
+        char buf[64];
+        snprintf(buf, sizeof buf, "0x%x", st[ST_KERNEL_ERR]);
+        return fail(c, MPT_ERR_TIMEOUT, "a device-side bounded wait expired (code|cta<<8 = %s)", buf);
+    }
+    return MPT_OK;
+}
+
+int do_forward(mpt_ctx *c, const uint16_t *x_dev, int batch)
+{
+    if (batch < 1 || batch > c->max_batch) return fail(c, MPT_ERR_SHAPE, "batch outside [1, max_batch]");
+    const uint16_t *a = x_dev;
+    int lda = c->layers[0].in;
+    for (size_t l = 0; l < c->layers.size(); l++) {
+        Layer &ly = c->layers[l];
+        int r = gemm(c, MPT_OP_FWD, batch, ly.out, ly.in, a, lda, c->w16 + ly.off, ly.in, ly.act, ly.ld_out, ly.relu != 0,
+                     nullptr, 0, nullptr);
+        if (r != MPT_OK) return r;
+        a = ly.act;
+        lda = ly.ld_out;
+    }
+    c->x_cur = x_dev;
+    c->batch = batch;
+    c->forward_done = true;
+    return MPT_OK;
+}
+
+int do_backward(mpt_ctx *c, const int32_t *labels_dev)
+{
+    if (!c->forward_done) return fail(c, MPT_ERR_STATE, "mpt_backward_scaled needs a preceding mpt_forward");
+    const int L = (int)c->layers.size(), B = c->batch;
+    // status words 0..2 (overflow, overflow seen, bad labels) start the backward at zero
+    CK(cudaMemsetAsync(c->status, 0, 3 * sizeof(uint32_t), c->stream), "status clear");
+    Layer &last = c->layers[L - 1];
+    int nl = 0;
+    cudaError_t e = launch_softmax_ce(last.act, last.ld_out, labels_dev, B, last.out, c->S, last.dact, last.ld_out,
+                                      c->row_loss, (float *)(c->status + ST_LOSS), c->status + ST_BAD_LABELS, c->stream,
+                                      &nl);
+    c->launches += nl;
+    if (e != cudaSuccess) return cuda_fail(c, e, "softmax launch");
+    for (int l = L - 1; l >= 0; l--) {
+        Layer &ly = c->layers[l];
+        const uint16_t *a_prev = l ? c->layers[l - 1].act : c->x_cur;
+        const int ld_prev = l ? c->layers[l - 1].ld_out : ly.in;
+        int r = gemm(c, MPT_OP_WGRAD, ly.out, ly.in, B, ly.dact, ly.ld_out, a_prev, ld_prev, c->g16 + ly.off, ly.in, false,
+                     nullptr, 0, c->status + ST_OVERFLOW);
+        if (r != MPT_OK) return r;
+        if (l > 0) {
+            Layer &pv = c->layers[l - 1];
+            r = gemm(c, MPT_OP_DGRAD, B, ly.in, ly.out, ly.dact, ly.ld_out, c->w16 + ly.off, ly.in, pv.dact, pv.ld_out, false,
+                     pv.relu ? pv.act : nullptr, pv.ld_out, nullptr);
+            if (r != MPT_OK) return r;
+        }
+    }
+    c->forward_done = false;
+    c->have_grads = true;
+    return MPT_OK;
+}
+
+int do_step(mpt_ctx *c)
+{
+    if (!c->have_grads) return fail(c, MPT_ERR_STATE, "mpt_step needs gradients (mpt_backward_scaled or mpt_set_grad)");
+    const float inv = 1.0f / c->S;
+    CK(cudaMemsetAsync(c->status + ST_OVERFLOW_SEEN, 0, sizeof(uint32_t), c->stream), "status clear");
+    cudaError_t e = launch_update(c->g16, c->master, c->mom, c->w16, c->plan.P_pad, inv, c->lr, c->mu, c->use_momentum,
+                                  c->status + ST_OVERFLOW, c->stream);
+    c->launches++;
+    if (e != cudaSuccess) return cuda_fail(c, e, "update launch");
+    return MPT_OK;
+}
+
+int finish_step(mpt_ctx *c, const uint32_t (&st)[ST_WORDS], int *overflow_host)
+{
+    if (st[ST_OVERFLOW] == 0 && st[ST_OVERFLOW_SEEN] != 0)
+        return fail(c, MPT_ERR_INTERNAL, "update kernel saw a non-finite gradient the producer did not flag");
+    if (overflow_host) *overflow_host = st[ST_OVERFLOW] ? 1 : 0;
+    return MPT_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *mpt_version(void) { return "mpt 0.1 sm_100a"; }
+
+int mpt_workspace_bytes(const mpt_layer_desc *layers, int n_layers, int max_batch, int use_momentum, size_t *bytes_out)
+{
+    if (!bytes_out) return MPT_ERR_INVALID_ARG;
+    int r = validate_layers(layers, n_layers, max_batch);
+    if (r != MPT_OK) return r;
+    Plan pl;
+    make_plan(layers, n_layers, max_batch, use_momentum != 0, pl);
+    *bytes_out = pl.total;
+    return MPT_OK;
+}
+
+int mpt_create(const mpt_layer_desc *layers, int n_layers, float S, float lr, float momentum, int max_batch,
+               void *workspace_dev, size_t workspace_bytes, void *cuda_stream, mpt_ctx **out)
+{
+    if (!out) return MPT_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!workspace_dev) return MPT_ERR_INVALID_ARG;
+    int r = validate_layers(layers, n_layers, max_batch);
+    if (r != MPT_OK) return r;
+    if (!valid_scale(S) || !std::isfinite(lr) || !(momentum >= 0.0f && momentum < 1.0f)) return MPT_ERR_INVALID_ARG;
+    if ((uintptr_t)workspace_dev % 256) return MPT_ERR_WORKSPACE;
+    mpt_ctx *c = new (std::nothrow) mpt_ctx();
+    if (!c) return MPT_ERR_INTERNAL;
+    c->use_momentum = momentum != 0.0f;
+    make_plan(layers, n_layers, max_batch, c->use_momentum, c->plan);
+    if (workspace_bytes < c->plan.total) { delete c; return MPT_ERR_WORKSPACE; }
+    c->S = S; c->lr = lr; c->mu = momentum; c->max_batch = max_batch;
+    c->stream = (cudaStream_t)cuda_stream;
+    c->ws = (uint8_t *)workspace_dev;
+    const Plan &pl = c->plan;
+    c->status = (uint32_t *)(c->ws + pl.off_status);
+    c->master = (float *)(c->ws + pl.off_master);
+    c->mom = c->use_momentum ? (float *)(c->ws + pl.off_mom) : nullptr;
+    c->w16 = (uint16_t *)(c->ws + pl.off_w16);
+    c->g16 = (uint16_t *)(c->ws + pl.off_g16);
+    c->x_stage = (uint16_t *)(c->ws + pl.off_x);
+    c->labels_stage = (int32_t *)(c->ws + pl.off_labels);
+    c->row_loss = (float *)(c->ws + pl.off_rowloss);
+    c->layers.resize(n_layers);
+    for (int l = 0; l < n_layers; l++) {
+        Layer &ly = c->layers[l];
+        ly.in = layers[l].in_features; ly.out = layers[l].out_features; ly.relu = layers[l].relu;
+        ly.off = pl.lay_off[l];
+        ly.n = (size_t)ly.in * ly.out;
+        ly.ld_out = pl.ld_out[l];
+        ly.act = (uint16_t *)(c->ws + pl.off_act[l]);
+        ly.dact = (uint16_t *)(c->ws + pl.off_dact[l]);
+    }
+    const char *env = getenv("MPT_DISABLE_TC");
+    c->disable_tc = env && env[0] == '1';
+    // Parameter arenas (including the padding between layers), activations and status start at zero.
+    cudaError_t e = cudaMemsetAsync(c->ws, 0, pl.total, c->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
+    if (e != cudaSuccess) { delete c; return MPT_ERR_CUDA; }
+    *out = c;
+    return MPT_OK;
+}
+
+void mpt_destroy(mpt_ctx *c) { delete c; }
+
+const char *mpt_last_error(mpt_ctx *c) { return c ? c->err.c_str() : "null context"; }
+
+int mpt_launch_count(mpt_ctx *c, long long *count_out)
+{
+    if (!c || !count_out) return MPT_ERR_INVALID_ARG;
+    *count_out = c->launches;
+    return MPT_OK;
+}
+
+int mpt_set_scale(mpt_ctx *c, float S)
+{
+    int r = usable(c);
+    if (r != MPT_OK) return r;
+    if (!valid_scale(S)) return fail(c, MPT_ERR_INVALID_ARG, "loss scale out of range");
+    c->S = S;
+    return MPT_OK;
+}
+
+int mpt_set_lr(mpt_ctx *c, float lr)
+{
+    int r = usable(c);
+    if (r != MPT_OK) return r;
+    if (!std::isfinite(lr)) return fail(c, MPT_ERR_INVALID_ARG, "learning rate not finite");
+    c->lr = lr;
+    return MPT_OK;
+}
+
+int mpt_set_master(mpt_ctx *c, int layer, const float *src_host, size_t n)
+{
+    int r = usable(c);
+    if (r != MPT_OK) return r;
+    if (!src_host) return fail(c, MPT_ERR_INVALID_ARG, "null source");
+    if (layer < 0 || layer >= (int)c->layers.size()) return fail(c, MPT_ERR_INVALID_ARG, "layer index");
+    Layer &ly = c->layers[layer];
+    if (n != ly.n) return fail(c, MPT_ERR_SHAPE, "n must equal out*in");
+    CK(cudaMemcpyAsync(c->master + ly.off, src_host, n * 4, cudaMemcpyHostToDevice, c->stream), "master upload");
+    cudaError_t e = launch_recast(c->master + ly.off, c->w16 + ly.off, n, c->stream);
+    c->launches++;
+    if (e != cudaSuccess) return cuda_fail(c, e, "recast launch");
+    CK(cudaStreamSynchronize(c->stream), "stream synchronize");
+    return MPT_OK;
+}
+
+int mpt_get_master(mpt_ctx *c, int layer, float *dst_host, size_t n)
+{
+    int r = usable(c);
+    if (r != MPT_OK) return r;
+    if (!dst_host) return fail(c, MPT_ERR_INVALID_ARG, "null destination");
+    if (layer < 0 || layer >= (int)c->layers.size()) return fail(c, MPT_ERR_INVALID_ARG, "layer index");
+    Layer &ly = c->layers[layer];
+    if (n != ly.n) return fail(c, MPT_ERR_SHAPE, "n must equal out*in");
+    CK(cudaMemcpyAsync(dst_host, c->master + ly.off, n * 4, cudaMemcpyDeviceToHost, c->stream), "master download");
+    CK(cudaStreamSynchronize(c->stream), "stream synchronize");
+    return MPT_OK;
+}
+
+int mpt_forward(mpt_ctx *c, const uint16_t *x_dev, int batch)
+{
+    int r = usable(c);
+    if (r != MPT_OK) return r;
+    if (!x_dev) return fail(c, MPT_ERR_INVALID_ARG, "null input");
+    return do_forward(c, x_dev, batch);
+}
+
+int mpt_backward_scaled(mpt_ctx *c, const int32_t *labels_dev, float *loss_host_or_null)
+{
+    int r = usable(c);
+    if (r != MPT_OK) return r;
+    if (!labels_dev) return fail(c, MPT_ERR_INVALID_ARG, "null labels");
+    r = do_backward(c, labels_dev);
+    if (r != MPT_OK) return r;
+    if (loss_host_or_null) {
+        uint32_t st[ST_WORDS];
+        r = read_status(c, st);
+        if (r != MPT_OK) return r;
+        memcpy(loss_host_or_null, &st[ST_LOSS], 4);
+        if (st[ST_BAD_LABELS]) return fail(c, MPT_ERR_INVALID_ARG, "labels outside [0, C) were ignored");
+    }
+    return MPT_OK;
+}
+
+int mpt_step(mpt_ctx *c, int *overflow_host_or_null)
+{
+    int r = usable(c);
+    if (r != MPT_OK) return r;
+    r = do_step(c);
+    if (r != MPT_OK) return r;
+    if (overflow_host_or_null) {
+        uint32_t st[ST_WORDS];
+        r = read_status(c, st);
+        if (r != MPT_OK) return r;
+        return finish_step(c, st, overflow_host_or_null);
+    }
+    return MPT_OK;
+}
+
+int mpt_train_step_host(mpt_ctx *c, const uint16_t *x_host, const int32_t *labels_host, int batch, float *loss_host,
+                        int *overflow_host)
+{
+    int r = usable(c);
+    if (r != MPT_OK) return r;
+    if (!x_host || !labels_host) return fail(c, MPT_ERR_INVALID_ARG, "null host input");
+    if (batch < 1 || batch > c->max_batch) return fail(c, MPT_ERR_SHAPE, "batch outside [1, max_batch]");
+    CK(cudaMemcpyAsync(c->x_stage, x_host, (size_t)batch * c->layers[0].in * 2, cudaMemcpyHostToDevice, c->stream),
+       "input upload");
+    CK(cudaMemcpyAsync(c->labels_stage, labels_host, (size_t)batch * 4, cudaMemcpyHostToDevice, c->stream), "label upload");
+    r = do_forward(c, c->x_stage, batch);
+    if (r != MPT_OK) return r;
+    r = do_backward(c, c->labels_stage);
+    if (r != MPT_OK) return r;
+    r = do_step(c);
+    if (r != MPT_OK) return r;
+    uint32_t st[ST_WORDS];
+    r = read_status(c, st);
+    if (r != MPT_OK) return r;
+    if (loss_host) memcpy(loss_host, &st[ST_LOSS], 4);
+    r = finish_step(c, st, overflow_host);
+    if (r != MPT_OK) return r;
+    if (st[ST_BAD_LABELS]) return fail(c, MPT_ERR_INVALID_ARG, "labels outside [0, C) were ignored");
+    return MPT_OK;
+}
+
+int mpt_get_tensor(mpt_ctx *c, int kind, int layer, void *dst_host, size_t bytes)
+{
+    int r = usable(c);
+    if (r != MPT_OK) return r;
+    if (!dst_host) return fail(c, MPT_ERR_INVALID_ARG, "null destination");
+    if (layer < 0 || layer >= (int)c->layers.size()) return fail(c, MPT_ERR_INVALID_ARG, "layer index");
+    Layer &ly = c->layers[layer];
+    const void *src = nullptr;
+    size_t rows = 0, row_bytes = 0, pitch = 0;
+    switch (kind) {
+        case MPT_T_W16: src = c->w16 + ly.off; rows = 1; row_bytes = ly.n * 2; pitch = row_bytes; break;
+        case MPT_T_GRAD16: src = c->g16 + ly.off; rows = 1; row_bytes = ly.n * 2; pitch = row_bytes; break;
+        case MPT_T_MASTER32: src = c->master + ly.off; rows = 1; row_bytes = ly.n * 4; pitch = row_bytes; break;
+        case MPT_T_MOMENTUM32:
+            if (!c->use_momentum) return fail(c, MPT_ERR_STATE, "context has no momentum buffer");
+            src = c->mom + ly.off; rows = 1; row_bytes = ly.n * 4; pitch = row_bytes; break;
+        case MPT_T_ACT16:
+        case MPT_T_DACT16:
+            if (c->batch < 1) return fail(c, MPT_ERR_STATE, "no forward pass yet");
+            src = kind == MPT_T_ACT16 ? ly.act : ly.dact;
+            rows = (size_t)c->batch; row_bytes = (size_t)ly.out * 2; pitch = (size_t)ly.ld_out * 2; break;
+        default: return fail(c, MPT_ERR_INVALID_ARG, "tensor kind");
+    }
+    if (bytes != rows * row_bytes) return fail(c, MPT_ERR_SHAPE, "byte count does not match the tensor");
+    CK(cudaMemcpy2DAsync(dst_host, row_bytes, src, pitch, row_bytes, rows, cudaMemcpyDeviceToHost, c->stream), "tensor download");
+    CK(cudaStreamSynchronize(c->stream), "stream synchronize");
+    return MPT_OK;
+}
+
+int mpt_set_grad(mpt_ctx *c, int layer, const uint16_t *src_host, size_t n)
+{
+    int r = usable(c);
+    if (r != MPT_OK) return r;
+    if (!src_host) return fail(c, MPT_ERR_INVALID_ARG, "null source");
+    if (layer < 0 || layer >= (int)c->layers.size()) return fail(c, MPT_ERR_INVALID_ARG, "layer index");
+    Layer &ly = c->layers[layer];
+    if (n != ly.n) return fail(c, MPT_ERR_SHAPE, "n must equal out*in");
+    CK(cudaMemcpyAsync(c->g16 + ly.off, src_host, n * 2, cudaMemcpyHostToDevice, c->stream), "gradient upload");
+    // the overflow word must describe all layers' gradients as they now stand
+    CK(cudaMemsetAsync(c->status + ST_OVERFLOW, 0, sizeof(uint32_t), c->stream), "status clear");
+    cudaError_t e = launch_grad_nonfinite(c->g16, c->plan.P_pad, 1.0f / c->S, c->status + ST_OVERFLOW, c->stream);
+    c->launches++;
+    if (e != cudaSuccess) return cuda_fail(c, e, "inspection launch");
+    CK(cudaStreamSynchronize(c->stream), "stream synchronize");
+    c->have_grads = true;
+    return MPT_OK;
+}
+
+int mpt_set_momentum(mpt_ctx *c, int layer, const float *src_host, size_t n)
+{
+    int r = usable(c);
+    if (r != MPT_OK) return r;
+    if (!src_host) return fail(c, MPT_ERR_INVALID_ARG, "null source");
+    if (layer < 0 || layer >= (int)c->layers.size()) return fail(c, MPT_ERR_INVALID_ARG, "layer index");
+    if (!c->use_momentum) return fail(c, MPT_ERR_STATE, "context has no momentum buffer");
+    Layer &ly = c->layers[layer];
+    if (n != ly.n) return fail(c, MPT_ERR_SHAPE, "n must equal out*in");
+    CK(cudaMemcpyAsync(c->mom + ly.off, src_host, n * 4, cudaMemcpyHostToDevice, c->stream), "momentum upload");
+    CK(cudaStreamSynchronize(c->stream), "stream synchronize");
+    return MPT_OK;
+}
+
+// ---------------------------------------------------------- stateless launchers
+
+int mpt_gemm_f16(int op, int M, int N, int K, const uint16_t *A, int lda, const uint16_t *B, int ldb, uint16_t *C, int ldc,
+                 unsigned flags, const uint16_t *mask, int ldmask, uint32_t *nonfinite_flag, uint32_t *status_dev,
+                 void *cuda_stream)
+{
+    if (!A || !B || !C) return MPT_ERR_INVALID_ARG;
+    if (op != MPT_OP_FWD && op != MPT_OP_DGRAD && op != MPT_OP_WGRAD) return MPT_ERR_INVALID_ARG;
+    if (M < 0 || N < 0 || K < 0) return MPT_ERR_SHAPE;
+    if (M == 0 || N == 0) return MPT_OK;
+    const int a_cols = op == MPT_OP_WGRAD ? M : K, b_cols = op == MPT_OP_FWD ? K : N;
+    if (lda < a_cols || ldb < b_cols || ldc < N || (mask && ldmask < N)) return MPT_ERR_SHAPE;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const bool relu = (flags & MPT_GEMM_RELU) != 0;
+    bool tc_ok = K > 0 && tc_gemm_supported(op, M, N, K, A, lda, B, ldb, C, ldc, mask, ldmask);
+    if ((flags & MPT_GEMM_FORCE_TC) && !tc_ok) return MPT_ERR_SHAPE;
+    cudaError_t e;
+    if (tc_ok && !(flags & MPT_GEMM_FORCE_SIMT))
+        e = launch_gemm_tc(op, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite_flag, status_dev, st);
+    else
+        e = launch_gemm_simt(op, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite_flag, st);
+    return e == cudaSuccess ? MPT_OK : MPT_ERR_CUDA;
+}
+
+int mpt_recast(const float *w32_dev, uint16_t *w16_dev, size_t n, void *cuda_stream)
+{
+    if (!w32_dev || !w16_dev) return MPT_ERR_INVALID_ARG;
+    return launch_recast(w32_dev, w16_dev, n, (cudaStream_t)cuda_stream) == cudaSuccess ? MPT_OK : MPT_ERR_CUDA;
+}
+
+int mpt_grad_nonfinite(const uint16_t *g16_dev, size_t n, float inv_S, uint32_t *flag_dev, void *cuda_stream)
+{
+    if (!g16_dev || !flag_dev) return MPT_ERR_INVALID_ARG;
+    return launch_grad_nonfinite(g16_dev, n, inv_S, flag_dev, (cudaStream_t)cuda_stream) == cudaSuccess ? MPT_OK
+                                                                                                       : MPT_ERR_CUDA;
+}
+
+int mpt_update_flat(const uint16_t *g16_dev, float *w32_dev, float *v_dev, uint16_t *w16_dev, size_t n, float inv_S,
+                    float lr, float mu, int use_momentum, int detect, uint32_t *flags_dev, void *cuda_stream)
+{
+    if (!g16_dev || !w32_dev || !w16_dev || !flags_dev) return MPT_ERR_INVALID_ARG;
+    if (use_momentum && !v_dev) return MPT_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    cudaError_t e;
+    if (detect) {
+        e = cudaMemsetAsync(flags_dev, 0, 2 * sizeof(uint32_t), st);
+        if (e == cudaSuccess) e = launch_grad_nonfinite(g16_dev, n, inv_S, flags_dev, st);
+    } else {
+        e = cudaMemsetAsync(flags_dev + 1, 0, sizeof(uint32_t), st);
+    }
+    if (e == cudaSuccess) e = launch_update(g16_dev, w32_dev, v_dev, w16_dev, n, inv_S, lr, mu, use_momentum != 0, flags_dev, st);
+    return e == cudaSuccess ? MPT_OK : MPT_ERR_CUDA;
+}
+
+int mpt_softmax_ce(const uint16_t *z_dev, int ldz, const int32_t *labels_dev, int B, int C, float S, uint16_t *dz_dev,
+                   int lddz, float *row_loss_dev, float *loss_dev, uint32_t *bad_labels_dev, void *cuda_stream)
+{
+    if (!z_dev || !labels_dev || !dz_dev || !row_loss_dev || !loss_dev) return MPT_ERR_INVALID_ARG;
+    if (B < 0 || C < 0 || ldz < C || lddz < C) return MPT_ERR_SHAPE;
+    if (z_dev == dz_dev) return MPT_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    cudaError_t e = cudaSuccess;
+    if (bad_labels_dev) e = cudaMemsetAsync(bad_labels_dev, 0, sizeof(uint32_t), st);
+    if (e == cudaSuccess)
+        e = launch_softmax_ce(z_dev, ldz, labels_dev, B, C, S, dz_dev, lddz, row_loss_dev, loss_dev, bad_labels_dev, st, nullptr);
+    return e == cudaSuccess ? MPT_OK : MPT_ERR_CUDA;
+}
+
+}  // extern "C"

@@ -1,0 +1,60 @@
+// Shared declarations of the CUDA library: kernel launcher prototypes and small
+// device helpers.  Internal; the public boundary is include/mpt.h.
+#pragma once
+
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "mpt.h"
+
+namespace mpt {
+
+// Device status block (uint32 words) inside a context's workspace.
+enum StatusWord : int {
+    ST_OVERFLOW = 0,      // OR of "weight gradient is inf/NaN" (wgrad epilogues, detect kernel)
+    ST_OVERFLOW_SEEN = 1, // the update kernel's own inspection of the gradients it streamed
+    ST_BAD_LABELS = 2,    // labels outside [0, C) seen by the last softmax
+    ST_KERNEL_ERR = 3,    // first device-side error (bounded wait expired): code | where<<8
+    ST_LOSS = 4,          // float: unscaled mean loss of the last backward
+    ST_WORDS = 16
+};
+
+// Device-side error codes written to ST_KERNEL_ERR.
+enum KernelErr : uint32_t {
+    KERR_NONE = 0,
+    KERR_WAIT_FULL = 1,   // consumer gave up waiting for a TMA-filled stage
+    KERR_WAIT_EMPTY = 2,  // producer gave up waiting for a free stage
+    KERR_WAIT_ACC = 3,    // epilogue gave up waiting for the accumulator
+    KERR_WAIT_ACC_FREE = 4, // MMA issuer gave up waiting for a drained accumulator
+    KERR_TMEM_ALLOC = 5
+};
+
+__device__ __forceinline__ bool half_bits_nonfinite(uint32_t h) { return (h & 0x7C00u) == 0x7C00u; }
+__device__ __forceinline__ bool f32_nonfinite(float x)
+{
+    return (__float_as_uint(x) & 0x7F800000u) == 0x7F800000u;
+}
+
+// Launchers (each returns a cudaError_t from the launch; all asynchronous on `st`).
+cudaError_t launch_recast(const float *w32, uint16_t *w16, size_t n, cudaStream_t st);
+cudaError_t launch_grad_nonfinite(const uint16_t *g16, size_t n, float inv_S, uint32_t *flag,
+                                  cudaStream_t st);
+cudaError_t launch_update(const uint16_t *g16, float *w32, float *v, uint16_t *w16, size_t n, float inv_S,
+                          float lr, float mu, bool use_momentum, uint32_t *flags, cudaStream_t st);
+cudaError_t launch_softmax_ce(const uint16_t *z, int ldz, const int32_t *labels, int B, int C, float S,
+                              uint16_t *dz, int lddz, float *row_loss, float *loss, uint32_t *bad_labels,
+                              cudaStream_t st, int *n_launches);
+cudaError_t launch_gemm_simt(int op, int M, int N, int K, const uint16_t *A, int lda, const uint16_t *B,
+                             int ldb, uint16_t *C, int ldc, bool relu, const uint16_t *mask, int ldmask,
+                             uint32_t *nonfinite_flag, cudaStream_t st);
+
+// tcgen05 path.  tc_gemm_supported: alignment/shape rules; launch_gemm_tc builds the
+// TMA descriptors on the host and launches the persistent kernel.
+bool tc_gemm_supported(int op, int M, int N, int K, const void *A, int lda, const void *B, int ldb,
+                       const void *C, int ldc, const void *mask, int ldmask);
+cudaError_t launch_gemm_tc(int op, int M, int N, int K, const uint16_t *A, int lda, const uint16_t *B,
+                           int ldb, uint16_t *C, int ldc, bool relu, const uint16_t *mask, int ldmask,
+                           uint32_t *nonfinite_flag, uint32_t *status, cudaStream_t st);
+
+}  // namespace mpt

@@ -1,0 +1,176 @@
+// Fused softmax cross-entropy forward + loss-scaled backward (paper sections 3.2, 3.3):
+// FP16 logits in, FP32 max / sum-of-exponentials / log, FP16 logit gradient out with
+// the factor S/B applied.  One CTA per row; the row is read from HBM once (kept in
+// shared memory as FP16) and written once: 4 bytes per logit.
+#include "mpt_common.cuh"
+
+namespace mpt {
+
+static constexpr int kMaxSmemRowBytes = 200 * 1024;
+
+__device__ __forceinline__ float hbits2f(uint32_t h) { return __half2float(__ushort_as_half((unsigned short)h)); }
+__device__ __forceinline__ uint32_t f2hbits(float x) { return (uint32_t)__half_as_ushort(__float2half_rn(x)); }
+
+__device__ __forceinline__ float block_reduce(float v, bool is_max, float *red)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        float other = __shfl_xor_sync(0xFFFFFFFFu, v, o);
+        v = is_max ? fmaxf(v, other) : v + other;
+    }
+    __syncthreads();  // protect red[] from the previous use
+    if (lane == 0) red[warp] = v;
+    __syncthreads();
+    float r = red[0];
+    for (int w = 1; w < nw; w++) r = is_max ? fmaxf(r, red[w]) : r + red[w];   // fixed order
+    return r;
+}
+
+// VEC: rows are 16-byte aligned and C % 8 == 0 is NOT required (tail handled scalar).
+// CACHE: the row fits the dynamic shared-memory buffer.
+template <bool VEC, bool CACHE>
+__global__ void __launch_bounds__(1024) k_softmax_ce(const uint16_t *__restrict__ z, int ldz,
+                                                     const int32_t *__restrict__ labels, int B, int C, float c,
+                                                     uint16_t *dz, int lddz, float *__restrict__ row_loss,
+                                                     uint32_t *bad_labels)
+{
+    extern __shared__ __align__(16) uint16_t srow[];
+    __shared__ float red[32];
+    const int tid = threadIdx.x, nt = blockDim.x;
+    const int C8 = VEC ? (C / 8) : 0;
+
+    for (int row = blockIdx.x; row < B; row += gridDim.x) {
+        const uint16_t *zr = z + (size_t)row * ldz;
+        uint16_t *dr = dz + (size_t)row * lddz;
+        const int y = labels[row];
+        if (y < 0 || y >= C) {  // contributes neither loss nor gradient
+            for (int j = tid; j < C; j += nt) dr[j] = 0;
+            if (tid == 0) {
+                row_loss[row] = 0.0f;
+                if (bad_labels) atomicAdd(bad_labels, 1u);
+            }
+            continue;
+        }
+        // pass 1: read the row once, keep it on chip, running max
+        float m = -INFINITY;
+        bool first_nan = false;
+        if (VEC) {
+            const uint4 *zv = (const uint4 *)zr;
+            for (int i = tid; i < C8; i += nt) {
+                uint4 x = __ldcs(zv + i);
+                if (CACHE) ((uint4 *)srow)[i] = x;
+                uint32_t w[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+                for (int q = 0; q < 4; q++) {
+                    m = fmaxf(m, hbits2f(w[q] & 0xFFFFu));
+                    m = fmaxf(m, hbits2f(w[q] >> 16));
+                }
+            }
+        }
+        for (int j = C8 * 8 + tid; j < C; j += nt) {
+            uint16_t h = zr[j];
+            if (CACHE) srow[j] = h;
+            m = fmaxf(m, hbits2f(h));
+        }
+        (void)first_nan;
+        m = block_reduce(m, true, red);   // also orders the srow writes before the reads below
+
+        // pass 2: sum of exponentials in FP32
+        float s = 0.0f;
+        for (int j = tid; j < C; j += nt) {
+            float v = hbits2f(CACHE ? srow[j] : zr[j]);
+            s += expf(v - m);
+        }
+        s = block_reduce(s, false, red);
+        if (tid == 0) {
+            float zy = hbits2f(CACHE ? srow[y] : zr[y]);
+            row_loss[row] = (m + logf(s)) - zy;
+        }
+        // pass 3: gradient (e/s - onehot) * c, rounded to FP16
+        if (VEC) {
+            uint4 *dv = (uint4 *)dr;
+            for (int i = tid; i < C8; i += nt) {
+                uint4 x = CACHE ? ((const uint4 *)srow)[i] : ((const uint4 *)zr)[i];
+                uint32_t w[4] = {x.x, x.y, x.z, x.w};
+                uint32_t o[4];
+#pragma unroll
+                for (int q = 0; q < 4; q++) {
+                    int j = i * 8 + q * 2;
+                    float p0 = __fdiv_rn(expf(hbits2f(w[q] & 0xFFFFu) - m), s);
+                    float p1 = __fdiv_rn(expf(hbits2f(w[q] >> 16) - m), s);
+                    float d0 = __fmul_rn(__fsub_rn(p0, (j == y) ? 1.0f : 0.0f), c);
+                    float d1 = __fmul_rn(__fsub_rn(p1, (j + 1 == y) ? 1.0f : 0.0f), c);
+                    o[q] = f2hbits(d0) | (f2hbits(d1) << 16);
+                }
+                __stcs(dv + i, make_uint4(o[0], o[1], o[2], o[3]));
+            }
+        }
+        for (int j = C8 * 8 + tid; j < C; j += nt) {
+            float p = __fdiv_rn(expf(hbits2f(CACHE ? srow[j] : zr[j]) - m), s);
+            dr[j] = (uint16_t)f2hbits(__fmul_rn(__fsub_rn(p, (j == y) ? 1.0f : 0.0f), c));
+        }
+        __syncthreads();  // srow is reused by the next row
+    }
+}
+
+// loss = (float)( sum_i (double)row_loss[i] / B ), fixed reduction order.
+__global__ void __launch_bounds__(256) k_loss_mean(const float *__restrict__ row_loss, int B, float *loss)
+{
+    __shared__ double red[256];
+    double acc = 0.0;
+    for (int i = threadIdx.x; i < B; i += 256) acc += (double)row_loss[i];
+    red[threadIdx.x] = acc;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) {
+        if ((int)threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) *loss = (B > 0) ? (float)(red[0] / (double)B) : 0.0f;
+}
+
+template <bool VEC, bool CACHE>
+static cudaError_t launch_variant(const uint16_t *z, int ldz, const int32_t *labels, int B, int C, float c,
+                                  uint16_t *dz, int lddz, float *row_loss, uint32_t *bad_labels, int threads,
+                                  int grid, size_t smem, cudaStream_t st)
+{
+    auto kern = k_softmax_ce<VEC, CACHE>;
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+    }
+    kern<<<grid, threads, smem, st>>>(z, ldz, labels, B, C, c, dz, lddz, row_loss, bad_labels);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_softmax_ce(const uint16_t *z, int ldz, const int32_t *labels, int B, int C, float S,
+                              uint16_t *dz, int lddz, float *row_loss, float *loss, uint32_t *bad_labels,
+                              cudaStream_t st, int *n_launches)
+{
+    if (n_launches) *n_launches = 0;
+    if (B <= 0 || C <= 0) return cudaSuccess;
+    const float c = S / (float)B;  // one FP32 division
+    const bool vec = ((((uintptr_t)z | (uintptr_t)dz) & 15) == 0) && (ldz % 8 == 0) && (lddz % 8 == 0) && C >= 8;
+    const size_t row_bytes = ((size_t)C * 2 + 15) & ~(size_t)15;
+    const bool cache = row_bytes <= (size_t)kMaxSmemRowBytes;
+    int threads = vec ? (C / 8) : C;
+    threads = ((threads + 31) / 32) * 32;
+    if (threads > 1024) threads = 1024;
+    if (threads < 32) threads = 32;
+    int grid = B < 148 * 16 ? B : 148 * 16;
+    size_t smem = cache ? row_bytes : 0;
+    cudaError_t e;
+    if (vec && cache) e = launch_variant<true, true>(z, ldz, labels, B, C, c, dz, lddz, row_loss, bad_labels, threads, grid, smem, st);
+    else if (vec) e = launch_variant<true, false>(z, ldz, labels, B, C, c, dz, lddz, row_loss, bad_labels, threads, grid, smem, st);
+    else if (cache) e = launch_variant<false, true>(z, ldz, labels, B, C, c, dz, lddz, row_loss, bad_labels, threads, grid, smem, st);
+    else e = launch_variant<false, false>(z, ldz, labels, B, C, c, dz, lddz, row_loss, bad_labels, threads, grid, smem, st);
+    if (e != cudaSuccess) return e;
+    if (n_launches) *n_launches = 1;
+    if (loss) {
+        k_loss_mean<<<1, 256, 0, st>>>(row_loss, B, loss);
+        if (n_launches) *n_launches = 2;
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace mpt

@@ -1,0 +1,236 @@
+// Master-weight pass (paper sections 3.1, 3.2): recast, overflow inspection, and the
+// fused unscale / inspect / FP32 SGD(+momentum) / FP16 re-round kernel.
+//
+// All three are streaming kernels bound by HBM bandwidth: 128-bit accesses, a grid
+// of 148 SMs x 8 resident CTAs of 256 threads, two independent 8-element vectors in
+// flight per thread.  The update reads g16, w32, (v) once and writes w32, (v), w16
+// once: 12 bytes/parameter (plain SGD) or 20 bytes/parameter (momentum).
+//
+// Bit-exactness contract: every FP32 operation is rounded separately (the __f*_rn
+// intrinsics are never contracted into a fused multiply-add), no flush-to-zero.
+#include "mpt_common.cuh"
+
+namespace mpt {
+
+static constexpr int kThreads = 256;
+static constexpr int kSMs = 148;
+static constexpr int kCtasPerSM = 8;
+
+__device__ __forceinline__ float h2f_bits(uint32_t h) { return __half2float(__ushort_as_half((unsigned short)h)); }
+__device__ __forceinline__ uint32_t f2h_bits(float x) { return (uint32_t)__half_as_ushort(__float2half_rn(x)); }
+
+static inline int grid_for(size_t work_items)
+{
+    size_t blocks = (work_items + kThreads - 1) / kThreads;
+    size_t cap = (size_t)kSMs * kCtasPerSM;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    return (int)blocks;
+}
+
+// ------------------------------------------------------------------ recast
+
+__global__ void __launch_bounds__(kThreads) k_recast_vec(const float4 *__restrict__ w32, uint4 *__restrict__ w16,
+                                                         size_t n8)
+{
+    size_t stride = (size_t)gridDim.x * blockDim.x;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n8; i += stride) {
+        float4 a = __ldcs(w32 + 2 * i), b = __ldcs(w32 + 2 * i + 1);
+        uint4 o;
+        o.x = f2h_bits(a.x) | (f2h_bits(a.y) << 16);
+        o.y = f2h_bits(a.z) | (f2h_bits(a.w) << 16);
+        o.z = f2h_bits(b.x) | (f2h_bits(b.y) << 16);
+        o.w = f2h_bits(b.z) | (f2h_bits(b.w) << 16);
+        w16[i] = o;
+    }
+}
+
+__global__ void k_recast_scalar(const float *__restrict__ w32, uint16_t *__restrict__ w16, size_t begin, size_t n)
+{
+    size_t stride = (size_t)gridDim.x * blockDim.x;
+    for (size_t i = begin + (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride)
+        w16[i] = (uint16_t)f2h_bits(w32[i]);
+}
+
+cudaError_t launch_recast(const float *w32, uint16_t *w16, size_t n, cudaStream_t st)
+{
+    if (n == 0) return cudaSuccess;
+    bool aligned = (((uintptr_t)w32 | (uintptr_t)w16) & 15) == 0;
+    size_t n8 = aligned ? n / 8 : 0;
+    if (n8) k_recast_vec<<<grid_for(n8), kThreads, 0, st>>>((const float4 *)w32, (uint4 *)w16, n8);
+    if (n8 * 8 < n) k_recast_scalar<<<grid_for(n - n8 * 8), kThreads, 0, st>>>(w32, w16, n8 * 8, n);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------- overflow inspection
+
+__device__ __forceinline__ bool pair_nonfinite(uint32_t two_halfs, float inv)
+{
+    return f32_nonfinite(__fmul_rn(h2f_bits(two_halfs & 0xFFFFu), inv)) ||
+           f32_nonfinite(__fmul_rn(h2f_bits(two_halfs >> 16), inv));
+}
+
+__global__ void __launch_bounds__(kThreads) k_nonfinite_vec(const uint4 *__restrict__ g, size_t n8, float inv,
+                                                            uint32_t *flag)
+{
+    size_t stride = (size_t)gridDim.x * blockDim.x;
+    bool bad = false;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n8; i += stride) {
+        uint4 x = __ldcs(g + i);
+        bad |= pair_nonfinite(x.x, inv) | pair_nonfinite(x.y, inv) | pair_nonfinite(x.z, inv) |
+               pair_nonfinite(x.w, inv);
+    }
+    // warp vote, then at most one atomic per warp and only when something was found
+    if (__any_sync(0xFFFFFFFFu, bad) && (threadIdx.x & 31) == 0) atomicOr(flag, 1u);
+}
+
+__global__ void k_nonfinite_scalar(const uint16_t *__restrict__ g, size_t begin, size_t n, float inv, uint32_t *flag)
+{
+    size_t stride = (size_t)gridDim.x * blockDim.x;
+    bool bad = false;
+    for (size_t i = begin + (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride)
+        bad |= f32_nonfinite(__fmul_rn(h2f_bits(g[i]), inv));
+    if (__any_sync(0xFFFFFFFFu, bad) && (threadIdx.x & 31) == 0) atomicOr(flag, 1u);
+}
+
+cudaError_t launch_grad_nonfinite(const uint16_t *g16, size_t n, float inv_S, uint32_t *flag, cudaStream_t st)
+{
+    if (n == 0) return cudaSuccess;
+    bool aligned = ((uintptr_t)g16 & 15) == 0;
+    size_t n8 = aligned ? n / 8 : 0;
+    if (n8) k_nonfinite_vec<<<grid_for(n8), kThreads, 0, st>>>((const uint4 *)g16, n8, inv_S, flag);
+    if (n8 * 8 < n) k_nonfinite_scalar<<<grid_for(n - n8 * 8), kThreads, 0, st>>>(g16, n8 * 8, n, inv_S, flag);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------- update
+
+// One element: g = f32(g16) * inv ; [v = mu*v + g ; u = lr*v] or [u = lr*g] ; w -= u.
+template <bool MOM>
+__device__ __forceinline__ void upd1(uint32_t gh, float &w, float &v, float inv, float lr, float mu, bool &bad)
+{
+    float g = __fmul_rn(h2f_bits(gh), inv);
+    bad |= f32_nonfinite(g);
+    float u;
+    if (MOM) {
+        float t = __fmul_rn(mu, v);
+        v = __fadd_rn(t, g);
+        u = __fmul_rn(lr, v);
+    } else {
+        u = __fmul_rn(lr, g);
+    }
+    w = __fsub_rn(w, u);
+}
+
+template <bool MOM>
+__device__ __forceinline__ void upd8(const uint4 &g, float4 &w0, float4 &w1, float4 &v0, float4 &v1, uint4 &h,
+                                     float inv, float lr, float mu, bool &bad)
+{
+    upd1<MOM>(g.x & 0xFFFFu, w0.x, v0.x, inv, lr, mu, bad);
+    upd1<MOM>(g.x >> 16, w0.y, v0.y, inv, lr, mu, bad);
+    upd1<MOM>(g.y & 0xFFFFu, w0.z, v0.z, inv, lr, mu, bad);
+    upd1<MOM>(g.y >> 16, w0.w, v0.w, inv, lr, mu, bad);
+    upd1<MOM>(g.z & 0xFFFFu, w1.x, v1.x, inv, lr, mu, bad);
+    upd1<MOM>(g.z >> 16, w1.y, v1.y, inv, lr, mu, bad);
+    upd1<MOM>(g.w & 0xFFFFu, w1.z, v1.z, inv, lr, mu, bad);
+    upd1<MOM>(g.w >> 16, w1.w, v1.w, inv, lr, mu, bad);
+    h.x = f2h_bits(w0.x) | (f2h_bits(w0.y) << 16);
+    h.y = f2h_bits(w0.z) | (f2h_bits(w0.w) << 16);
+    h.z = f2h_bits(w1.x) | (f2h_bits(w1.y) << 16);
+    h.w = f2h_bits(w1.z) | (f2h_bits(w1.w) << 16);
+}
+
+// flags[0]: overflow decided by the producer of the gradients (read, never written);
+// flags[1]: this kernel's own inspection (written).  When flags[0] is set the whole
+// grid returns before touching a parameter: a skipped step moves no parameter byte.
+template <bool MOM>
+__global__ void __launch_bounds__(kThreads) k_update_vec(const uint4 *__restrict__ g16, float4 *__restrict__ w32,
+                                                         float4 *__restrict__ v32, uint4 *__restrict__ w16, size_t n8,
+                                                         float inv, float lr, float mu, uint32_t *flags)
+{
+    if (*(volatile const uint32_t *)flags != 0u) return;
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    bool bad = false;
+    // two vectors per trip: all loads of both are issued before the first use
+    for (; i + stride < n8; i += 2 * stride) {
+        const size_t j = i + stride;
+        uint4 ga = __ldcs(g16 + i), gb = __ldcs(g16 + j);
+        float4 wa0 = __ldcs(w32 + 2 * i), wa1 = __ldcs(w32 + 2 * i + 1);
+        float4 wb0 = __ldcs(w32 + 2 * j), wb1 = __ldcs(w32 + 2 * j + 1);
+        float4 va0 = {}, va1 = {}, vb0 = {}, vb1 = {};
+        if (MOM) {
+            va0 = __ldcs(v32 + 2 * i); va1 = __ldcs(v32 + 2 * i + 1);
+            vb0 = __ldcs(v32 + 2 * j); vb1 = __ldcs(v32 + 2 * j + 1);
+        }
+        uint4 ha, hb;
+        upd8<MOM>(ga, wa0, wa1, va0, va1, ha, inv, lr, mu, bad);
+        upd8<MOM>(gb, wb0, wb1, vb0, vb1, hb, inv, lr, mu, bad);
+        __stcs(w32 + 2 * i, wa0); __stcs(w32 + 2 * i + 1, wa1);
+        __stcs(w32 + 2 * j, wb0); __stcs(w32 + 2 * j + 1, wb1);
+        if (MOM) {
+            __stcs(v32 + 2 * i, va0); __stcs(v32 + 2 * i + 1, va1);
+            __stcs(v32 + 2 * j, vb0); __stcs(v32 + 2 * j + 1, vb1);
+        }
+        w16[i] = ha;
+        w16[j] = hb;
+    }
+    if (i < n8) {
+        uint4 ga = __ldcs(g16 + i);
+        float4 wa0 = __ldcs(w32 + 2 * i), wa1 = __ldcs(w32 + 2 * i + 1);
+        float4 va0 = {}, va1 = {};
+        if (MOM) { va0 = __ldcs(v32 + 2 * i); va1 = __ldcs(v32 + 2 * i + 1); }
+        uint4 ha;
+        upd8<MOM>(ga, wa0, wa1, va0, va1, ha, inv, lr, mu, bad);
+        __stcs(w32 + 2 * i, wa0); __stcs(w32 + 2 * i + 1, wa1);
+        if (MOM) { __stcs(v32 + 2 * i, va0); __stcs(v32 + 2 * i + 1, va1); }
+        w16[i] = ha;
+    }
+    if (__any_sync(0xFFFFFFFFu, bad) && (threadIdx.x & 31) == 0) atomicOr(flags + 1, 1u);
+}
+
+template <bool MOM>
+__global__ void k_update_scalar(const uint16_t *__restrict__ g16, float *__restrict__ w32, float *__restrict__ v32,
+                                uint16_t *__restrict__ w16, size_t begin, size_t n, float inv, float lr, float mu,
+                                uint32_t *flags)
+{
+    if (*(volatile const uint32_t *)flags != 0u) return;
+    size_t stride = (size_t)gridDim.x * blockDim.x;
+    bool bad = false;
+    for (size_t i = begin + (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
+        float w = w32[i], v = MOM ? v32[i] : 0.0f;
+        upd1<MOM>(g16[i], w, v, inv, lr, mu, bad);
+        w32[i] = w;
+        if (MOM) v32[i] = v;
+        w16[i] = (uint16_t)f2h_bits(w);
+    }
+    if (__any_sync(0xFFFFFFFFu, bad) && (threadIdx.x & 31) == 0) atomicOr(flags + 1, 1u);
+}
+
+cudaError_t launch_update(const uint16_t *g16, float *w32, float *v, uint16_t *w16, size_t n, float inv_S, float lr,
+                          float mu, bool use_momentum, uint32_t *flags, cudaStream_t st)
+{
+    if (n == 0) return cudaSuccess;
+    uintptr_t bits = (uintptr_t)g16 | (uintptr_t)w32 | (uintptr_t)w16 | (use_momentum ? (uintptr_t)v : 0);
+    size_t n8 = (bits & 15) == 0 ? n / 8 : 0;
+    if (n8) {
+        // each thread owns two vectors per trip
+        int grid = grid_for((n8 + 1) / 2);
+        if (use_momentum)
+            k_update_vec<true><<<grid, kThreads, 0, st>>>((const uint4 *)g16, (float4 *)w32, (float4 *)v, (uint4 *)w16,
+                                                          n8, inv_S, lr, mu, flags);
+        else
+            k_update_vec<false><<<grid, kThreads, 0, st>>>((const uint4 *)g16, (float4 *)w32, nullptr, (uint4 *)w16, n8,
+                                                           inv_S, lr, mu, flags);
+    }
+    if (n8 * 8 < n) {
+        int grid = grid_for(n - n8 * 8);
+        if (use_momentum)
+            k_update_scalar<true><<<grid, kThreads, 0, st>>>(g16, w32, v, w16, n8 * 8, n, inv_S, lr, mu, flags);
+        else
+            k_update_scalar<false><<<grid, kThreads, 0, st>>>(g16, w32, nullptr, w16, n8 * 8, n, inv_S, lr, mu, flags);
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace mpt

@@ -1,0 +1,151 @@
+"""Parity of the FP16 GEMMs (FP32 accumulate, FP16 store; paper section 3.3) with the oracle.
+
+The CUDA-core kernel sums in the oracle's order and must match bit for bit; the
+tensor-core kernel sums in hardware order and is held to the acceptance rule
+(2 FP16 ulp / 1e-2 relative / a-priori summation bound near zero)."""
+import numpy as np
+import pytest
+
+from oracle import mpo
+from paper_1710_03740_b200 import inputs
+from parity import gemm_accept
+from gpu_util import dev, host_u16, require_gpu, torch
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _gpu():
+    require_gpu()
+
+
+def _pad(a, ld):
+    rows, cols = a.shape
+    out = np.zeros((rows, ld), dtype=np.uint16)
+    out[:, :cols] = a.view(np.uint16)
+    return out
+
+
+def run_gemm(op, A, B, M, N, K, flags=0, mask=None, pad=0, want_flag=False):
+    """A, B: stored float16 operands.  pad: extra columns added to every pitch."""
+    from paper_1710_03740_b200 import binding as b
+    lda, ldb, ldc = A.shape[1] + pad, B.shape[1] + pad, N + pad
+    Ad, Bd = dev(_pad(A, lda)), dev(_pad(B, ldb))
+    Cd = torch.full((M, ldc), 0x5555, dtype=torch.int16, device="cuda")
+    md = dev(_pad(mask, ldc)) if mask is not None else None
+    flag = torch.zeros(1, dtype=torch.int32, device="cuda")
+    status = torch.zeros(4, dtype=torch.int32, device="cuda")
+    b.mpt_gemm_f16(op, M, N, K, Ad, lda, Bd, ldb, Cd, ldc, flags, md, ldc if mask is not None else 0,
+                   flag if want_flag else None, status)
+    torch.cuda.synchronize()
+    assert int(status[0].item()) == 0, "device-side wait expired: 0x%x" % int(status[0].item())
+    out = host_u16(Cd)
+    if pad:
+        assert np.all(out[:, N:] == 0x5555)
+    return out[:, :N], int(flag.item())
+
+
+SIMT_SHAPES = [(1, 1, 1), (5, 7, 3), (64, 10, 512), (70, 130, 33), (129, 65, 100), (256, 256, 64)]
+
+
+@pytest.mark.parametrize("op", [0, 1, 2])
+@pytest.mark.parametrize("M,N,K", SIMT_SHAPES)
+def test_simt_gemm_bit_exact(op, M, N, K):
+    from paper_1710_03740_b200 import binding as b
+    A, B = inputs.gemm_operands(op, M, N, K, seed=11, scale_a=1.0, scale_b=1.0)
+    ref = mpo.gemm_f16(op, A, B)
+    got, _ = run_gemm(op, A, B, M, N, K, flags=b.GEMM_FORCE_SIMT, pad=3)
+    assert np.array_equal(got, ref)
+
+
+def test_simt_gemm_relu_mask_flag():
+    from paper_1710_03740_b200 import binding as b
+    M, N, K = 50, 40, 64
+    A, B = inputs.gemm_operands(0, M, N, K, seed=12, scale_a=1.0, scale_b=1.0)
+    ref = mpo.gemm_f16(0, A, B, relu=True)
+    got, _ = run_gemm(0, A, B, M, N, K, flags=b.GEMM_FORCE_SIMT | b.GEMM_RELU)
+    assert np.array_equal(got, ref)
+    rng = np.random.default_rng(1)
+    mask = rng.standard_normal((M, N)).astype(np.float16)
+    mask[0, :4] = [0.0, -0.0, np.nan, np.inf]
+    A, B = inputs.gemm_operands(1, M, N, K, seed=13, scale_a=1.0, scale_b=1.0)
+    ref = mpo.gemm_f16(1, A, B, mask=mask)
+    got, flag = run_gemm(1, A, B, M, N, K, flags=b.GEMM_FORCE_SIMT, mask=mask, want_flag=True)
+    assert np.array_equal(got, ref) and flag == 0
+    A2 = (A.astype(np.float32) * 3000).astype(np.float16)
+    B2 = (B.astype(np.float32) * 3000).astype(np.float16)
+    ref = mpo.gemm_f16(1, A2, B2)
+    got, flag = run_gemm(1, A2, B2, M, N, K, flags=b.GEMM_FORCE_SIMT, want_flag=True)
+    assert np.array_equal(got, ref)
+    assert flag == 1 and (~np.isfinite(ref.view(np.float16).astype(np.float32))).any()
+
+
+def _check_tc(op, M, N, K, flags=0, mask=None, seed=21, scale=None, want_flag=False):
+    from paper_1710_03740_b200 import binding as b
+    sa = sb = scale
+    A, B = inputs.gemm_operands(op, M, N, K, seed=seed, scale_a=sa, scale_b=sb)
+    ref, ex, ab = mpo.gemm_f16(op, A, B, relu=bool(flags & b.GEMM_RELU), mask=mask, want_exact=True)
+    got, flag = run_gemm(op, A, B, M, N, K, flags=flags | b.GEMM_FORCE_TC, mask=mask,
+                         pad=(8 if (M * N) % 3 == 0 else 0), want_flag=want_flag)
+    ok, stats = gemm_accept(got, ref, K=K, absdot=ab)
+    assert ok.all(), (op, M, N, K, stats, np.argwhere(~ok)[:8].tolist())
+    assert stats["by_abs_only"] <= max(2, stats["n"] // 1000), stats
+    # both sides within the summation bound of the exactly rounded sum
+    if not flags and mask is None:
+        exact16 = ex.astype(np.float32).astype(np.float16).view(np.uint16)
+        ok2, st2 = gemm_accept(got, exact16, K=K, absdot=ab)
+        assert ok2.all(), st2
+    return got, ref, flag, stats
+
+
+TC_SHAPES = [(128, 256, 64), (128, 256, 256), (256, 512, 128), (128, 256, 72), (200, 304, 136),
+             (64, 16, 512), (8, 8, 8), (384, 768, 1024), (1024, 1024, 1024)]
+
+
+@pytest.mark.parametrize("op", [0, 1, 2])
+@pytest.mark.parametrize("M,N,K", TC_SHAPES)
+def test_tc_gemm_parity(op, M, N, K):
+    _check_tc(op, M, N, K)
+
+
+@pytest.mark.parametrize("op", [0, 1, 2])
+def test_tc_gemm_run_to_run_identical(op):
+    M, N, K = 304, 520, 392
+    a, _, _, _ = _check_tc(op, M, N, K)
+    b2, _, _, _ = _check_tc(op, M, N, K)
+    assert np.array_equal(a, b2)
+
+
+def test_tc_gemm_relu_mask_flag_subnormals():
+    from paper_1710_03740_b200 import binding as b
+    M, N, K = 256, 512, 320
+    _check_tc(0, M, N, K, flags=b.GEMM_RELU)
+    rng = np.random.default_rng(4)
+    mask = rng.standard_normal((M, N)).astype(np.float16)
+    mask[0, :4] = [0.0, -0.0, np.nan, np.inf]
+    _check_tc(1, M, N, K, mask=mask)
+    # subnormal operands and outputs (config 2: head weights scaled by 2^-16)
+    got, ref, _, stats = _check_tc(0, M, N, K, scale=2.0 ** -9)
+    sub = (ref & 0x7C00) == 0
+    assert sub.mean() > 0.5 and (ref[sub] != 0).any()
+    # overflow on the store raises the flag (section 3.2)
+    got, ref, flag, _ = _check_tc(2, M, N, K, scale=60.0, want_flag=True)
+    assert flag == 1 and ((ref & 0x7FFF) == 0x7C00).any()
+    got, ref, flag, _ = _check_tc(2, M, N, K, want_flag=True)
+    assert flag == 0
+
+
+def test_tc_gemm_rejects_unaligned():
+    from paper_1710_03740_b200 import binding as b
+    A = torch.zeros((16, 10), dtype=torch.int16, device="cuda")
+    Bm = torch.zeros((16, 10), dtype=torch.int16, device="cuda")
+    Cm = torch.zeros((16, 16), dtype=torch.int16, device="cuda")
+    with pytest.raises(b.MptError) as e:
+        b.mpt_gemm_f16(0, 16, 16, 10, A, 10, Bm, 10, Cm, 16, b.GEMM_FORCE_TC)
+    assert e.value.code == -2
+    b.mpt_gemm_f16(0, 16, 16, 10, A, 10, Bm, 10, Cm, 16, 0)     # falls back to the CUDA-core kernel
+    torch.cuda.synchronize()
+    with pytest.raises(b.MptError):
+        b.mpt_gemm_f16(7, 16, 16, 10, A, 10, Bm, 10, Cm, 16, 0)
+    with pytest.raises(b.MptError):
+        b.mpt_gemm_f16(0, 16, 16, 10, A, 8, Bm, 10, Cm, 16, 0)  # pitch shorter than the row

@@ -1,0 +1,199 @@
+"""End-to-end parity of the training iteration with the oracle (configs 1 and 2a and the
+reduced twin of config 5): every tensor of every step under the GEMM acceptance rule,
+overflow flags equal, loss trajectories within 1e-3 relative, and the master update
+bit-exact when both sides are fed identical gradient bits."""
+import numpy as np
+import pytest
+
+from oracle import mpo
+from oracle.mlp import OracleMLP
+from paper_1710_03740_b200 import inputs
+from parity import gemm_accept
+from gpu_util import dev, require_gpu, torch
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _gpu():
+    require_gpu()
+
+
+def _make(cfg, S, masters):
+    from paper_1710_03740_b200 import binding as b
+    net = b.Context(cfg["layers"], S, cfg["lr"], cfg["momentum"], cfg["batch"])
+    ora = OracleMLP(cfg["layers"], S, cfg["lr"], cfg["momentum"])
+    for l, w in enumerate(masters):
+        net.set_master(l, w)
+        ora.set_master(l, w)
+    return net, ora
+
+
+def _teacher_forced_update_check(b, net, ora_layers, cfg, S):
+    """Feed the GPU's own gradient bits to a fresh oracle state and compare the step bit-exactly."""
+    L = len(cfg["layers"])
+    chk = OracleMLP(cfg["layers"], S, cfg["lr"], cfg["momentum"])
+    for l in range(L):
+        chk.set_master(l, net.get_master(l))
+        if cfg["momentum"]:
+            chk.v[l] = net.get_tensor(b.T_MOMENTUM32, l)
+        chk.set_grad(l, net.get_tensor(b.T_GRAD16, l))
+    return chk
+
+
+def _teacher_forced_kernel_checks(b, net, cfg, x16, labels, S):
+    """Every kernel output of this iteration against the oracle applied to the very inputs
+    that kernel read on the device (downloaded), under the GEMM acceptance rule."""
+    L = len(cfg["layers"])
+    acts = [x16.view(np.uint16)] + [net.get_tensor(b.T_ACT16, l) for l in range(L)]
+    dzs = [net.get_tensor(b.T_DACT16, l) for l in range(L)]
+    w16 = [net.get_tensor(b.T_W16, l) for l in range(L)]
+    g16 = [net.get_tensor(b.T_GRAD16, l) for l in range(L)]
+
+    def check(got, ref, ab, K, what):
+        ok, stats = gemm_accept(got, ref, K=K, absdot=ab)
+        assert ok.all(), (what, stats)
+
+    for l, (fin, fout, relu) in enumerate(cfg["layers"]):
+        ref, _, ab = mpo.gemm_f16(mpo.OP_FWD, acts[l], w16[l], relu=bool(relu), want_exact=True)
+        check(acts[l + 1], ref, ab, fin, ("fwd", l))
+    ref, _, _, _ = mpo.softmax_ce(acts[L], labels, S)
+    check(dzs[L - 1], ref, None, None, "softmax")
+    B = x16.shape[0]
+    for l in range(L - 1, -1, -1):
+        ref, _, ab = mpo.gemm_f16(mpo.OP_WGRAD, dzs[l], acts[l], want_exact=True)
+        check(g16[l], ref, ab, B, ("wgrad", l))
+        if l > 0:
+            mask = acts[l] if cfg["layers"][l - 1][2] else None
+            ref, _, ab = mpo.gemm_f16(mpo.OP_DGRAD, dzs[l], w16[l], mask=mask, want_exact=True)
+            check(dzs[l - 1], ref, ab, cfg["layers"][l][1], ("dgrad", l))
+
+
+def _free_run(cfg, S, steps, check_tensors=True):
+    from paper_1710_03740_b200 import binding as b
+    masters = inputs.mlp_masters(cfg)
+    net, ora = _make(cfg, S, masters)
+    X, Y = inputs.mlp_batches(cfg, steps)
+    L = len(cfg["layers"])
+    losses_g, losses_o, flags_g, flags_o = [], [], [], []
+    for t in range(steps):
+        xd, yd = dev(X[t].view(np.uint16)), dev(Y[t])
+        net.forward(xd)
+        lg = net.backward_scaled(yd)
+        ora.forward(X[t])
+        lo = ora.backward_scaled(Y[t])
+        if check_tensors:
+            _teacher_forced_kernel_checks(b, net, cfg, X[t], Y[t], S)
+        chk = _teacher_forced_update_check(b, net, ora.layers, cfg, S)
+        fg = net.step()
+        fc = chk.step()
+        assert fg == fc
+        for l in range(L):
+            assert net.get_master(l).tobytes() == chk.w32[l].tobytes(), (t, l)
+            assert net.get_tensor(b.T_W16, l).tobytes() == chk.w16[l].tobytes()
+            if cfg["momentum"]:
+                assert net.get_tensor(b.T_MOMENTUM32, l).tobytes() == chk.v[l].tobytes()
+        fo = ora.step()
+        losses_g.append(lg); losses_o.append(lo); flags_g.append(fg); flags_o.append(fo)
+    return net, ora, masters, losses_g, losses_o, flags_g, flags_o
+
+
+def test_tiny_config_trajectory():
+    cfg = inputs.MLP_CONFIGS["tiny"]
+    net, ora, _, lg, lo, fg, fo = _free_run(cfg, cfg["S"], cfg["steps"])
+    assert fg == fo == [0] * 10
+    for a, c in zip(lg, lo):
+        assert abs(a - c) <= 1e-3 * abs(c), (lg, lo)
+    assert net.launch_count() > 0
+
+
+@pytest.mark.parametrize("S", inputs.SCALE_SWEEP)
+def test_scale_sweep_config(S):
+    cfg = inputs.MLP_CONFIGS["scale_sweep"]
+    steps = cfg["steps"] if S == 2.0 ** 24 else 6
+    net, ora, masters, lg, lo, fg, fo = _free_run(cfg, S, steps, check_tensors=(S != 2.0 ** 24))
+    assert fg == fo
+    for a, c in zip(lg, lo):
+        assert abs(a - c) <= 1e-3 * abs(c)
+    if S == 2.0 ** 24:
+        assert fg == [1] * steps                      # overflows and skips every step
+        for l, w in enumerate(masters):
+            assert net.get_master(l).tobytes() == w.tobytes()
+    else:
+        assert fg == [0] * steps
+    if S == 1.0:
+        # hidden layers received nothing on the first step ... checked in the run above via parity;
+        # their masters have not moved at all after step 1 only, so just check zero fractions agree
+        from paper_1710_03740_b200 import binding as b
+        for l in range(4):
+            g, r = net.get_tensor(b.T_GRAD16, l), ora.g16[l]
+            assert abs(float((g == 0).mean()) - float((r == 0).mean())) < 0.02
+
+
+def test_large_twin_trajectory_with_momentum():
+    cfg = inputs.MLP_CONFIGS["large_twin"]
+    net, ora, _, lg, lo, fg, fo = _free_run(cfg, cfg["S"], cfg["steps"])
+    assert fg == fo == [0] * cfg["steps"]
+    for a, c in zip(lg, lo):
+        assert abs(a - c) <= 1e-3 * abs(c), (lg, lo)
+
+
+def test_train_step_host_matches_device_calls_and_checkpoint_resume():
+    from paper_1710_03740_b200 import binding as b
+    cfg = inputs.MLP_CONFIGS["tiny"]
+    masters = inputs.mlp_masters(cfg)
+    X, Y = inputs.mlp_batches(cfg, 4)
+    net1, _ = _make(cfg, cfg["S"], masters)
+    net2, _ = _make(cfg, cfg["S"], masters)
+    for t in range(2):
+        xd, yd = dev(X[t].view(np.uint16)), dev(Y[t])
+        net1.forward(xd)
+        l1 = net1.backward_scaled(yd)
+        f1 = net1.step()
+        l2, f2 = net2.train_step_host(X[t].view(np.uint16), Y[t])
+        assert l1 == l2 and f1 == f2
+    for l in range(2):
+        assert net1.get_master(l).tobytes() == net2.get_master(l).tobytes()
+    # checkpoint: masters out, new context, masters in, identical next step
+    saved = [net1.get_master(l) for l in range(2)]
+    net3, _ = _make(cfg, cfg["S"], saved)
+    la, fa = net1.train_step_host(X[2].view(np.uint16), Y[2])
+    lb, fb = net3.train_step_host(X[2].view(np.uint16), Y[2])
+    assert la == lb and fa == fb
+    for l in range(2):
+        assert net1.get_master(l).tobytes() == net3.get_master(l).tobytes()
+
+
+def test_error_paths():
+    from paper_1710_03740_b200 import binding as b
+    cfg = inputs.MLP_CONFIGS["tiny"]
+    net, _ = _make(cfg, cfg["S"], inputs.mlp_masters(cfg))
+    X, Y = inputs.mlp_batches(cfg, 1)
+    yd = dev(Y[0])
+    with pytest.raises(b.MptError) as e:
+        net.backward_scaled(yd)                       # no forward yet
+    assert e.value.code == -3
+    with pytest.raises(b.MptError) as e:
+        net.step()                                    # no gradients yet
+    assert e.value.code == -3
+    big = torch.zeros((cfg["batch"] + 1, 256), dtype=torch.float16, device="cuda")
+    with pytest.raises(b.MptError) as e:
+        net.forward(big)
+    assert e.value.code == -2
+    with pytest.raises(b.MptError):
+        net.set_master(0, np.zeros(5, dtype=np.float32))
+    # labels out of range are reported, and the context stays usable
+    net.forward(dev(X[0].view(np.uint16)))
+    bad = Y[0].copy()
+    bad[3] = 10
+    with pytest.raises(b.MptError) as e:
+        net.backward_scaled(dev(bad))
+    assert e.value.code == -1
+    assert net.step() == 0
+    # injected inf gradient: flag, nothing moves
+    before = net.get_master(1)
+    g = net.get_tensor(b.T_GRAD16, 1)
+    g[0, 0] = 0x7C00
+    net.set_grad(1, g)
+    assert net.step() == 1
+    assert net.get_master(1).tobytes() == before.tobytes()

@@ -1,0 +1,143 @@
+"""Parity of the master-weight pass with the oracle: bit-exact (paper sections 3.1, 3.2)."""
+import numpy as np
+import pytest
+
+from oracle import mpo
+from paper_1710_03740_b200 import inputs
+from gpu_util import dev, host_u16, require_gpu, torch
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _gpu():
+    require_gpu()
+
+
+def _binding():
+    from paper_1710_03740_b200 import binding
+    return binding
+
+
+@pytest.mark.parametrize("n", [0, 1, 7, 8, 1000, 4096 + 3, (1 << 20) + 5])
+def test_recast_matches_oracle(n):
+    b = _binding()
+    rng = np.random.default_rng(n)
+    w = (rng.standard_normal(n) * 10.0 ** rng.integers(-9, 6, n)).astype(np.float32)
+    if n >= 8:
+        w[:8] = [65504.0, 65519.9, 65520.0, 2.0 ** -24, 2.0 ** -25, 3 * 2.0 ** -26, -2.0 ** -26, np.inf]
+    wd = dev(np.concatenate([w, np.zeros(1, np.float32)]))      # never an empty (null) buffer
+    out = torch.zeros(n + 1, dtype=torch.int16, device="cuda")
+    b.mpt_recast(wd, out, n)
+    torch.cuda.synchronize()
+    assert np.array_equal(host_u16(out)[:n], mpo.f2h(w))
+
+
+def _run_update(n, use_momentum, S, lr, mu, g16, w, v, misalign=0, detect=True):
+    b = _binding()
+    pad = misalign
+    gd = torch.zeros(n + 8, dtype=torch.int16, device="cuda")
+    wd = torch.zeros(n + 8, dtype=torch.float32, device="cuda")
+    vd = torch.zeros(n + 8, dtype=torch.float32, device="cuda")
+    hd = torch.zeros(n + 8, dtype=torch.int16, device="cuda")
+    gd[pad:pad + n] = dev(g16.view(np.uint16))
+    wd[pad:pad + n] = dev(w)
+    vd[pad:pad + n] = dev(v)
+    flags = torch.zeros(2, dtype=torch.int32, device="cuda")
+    inv = float(np.float32(1.0) / np.float32(S))
+    b.mpt_update_flat(gd[pad:], wd[pad:], vd[pad:] if use_momentum else None, hd[pad:], n, inv, lr, mu,
+                      use_momentum, detect, flags)
+    torch.cuda.synchronize()
+    return (wd[pad:pad + n].cpu().numpy(), vd[pad:pad + n].cpu().numpy(), host_u16(hd[pad:pad + n]),
+            flags.cpu().numpy())
+
+
+@pytest.mark.parametrize("use_momentum", [False, True])
+@pytest.mark.parametrize("n,misalign", [(1, 0), (13, 0), (8 * 256 * 3 + 5, 0), ((1 << 21) + 11, 0), (5000, 1)])
+def test_update_bit_exact(use_momentum, n, misalign):
+    rng = np.random.default_rng(n + 17 * use_momentum)
+    S, lr, mu = 512.0, 0.01, 0.9
+    g16 = (rng.standard_normal(n) * 40.0).astype(np.float16)
+    w = rng.standard_normal(n).astype(np.float32)
+    v = (rng.standard_normal(n) * 0.1).astype(np.float32)
+    if n > 100:
+        g16[:6] = np.array([65504.0, -65504.0, 2.0 ** -24, -2.0 ** -24, 0.0, 6e-5], dtype=np.float16)
+    w_ref, v_ref = w.copy(), v.copy()
+    h_ref = np.zeros(n, dtype=np.uint16)
+    inv = np.float32(1.0) / np.float32(S)
+    assert mpo.grad_nonfinite(g16, inv) == 0
+    mpo.update_apply(g16, w_ref, v_ref, h_ref, inv, np.float32(lr), np.float32(mu), use_momentum)
+    w_g, v_g, h_g, flags = _run_update(n, use_momentum, S, lr, mu, g16, w, v, misalign)
+    assert flags.tolist() == [0, 0]
+    assert np.array_equal(w_g.view(np.uint32), w_ref.view(np.uint32))
+    if use_momentum:
+        assert np.array_equal(v_g.view(np.uint32), v_ref.view(np.uint32))
+    else:
+        assert np.array_equal(v_g.view(np.uint32), v.view(np.uint32))
+    assert np.array_equal(h_g, h_ref)
+
+
+def test_update_golden_fma_pairs():
+    """Operands for which a fused multiply-add would change the last bit."""
+    import os
+    import struct
+    rows = [l.split() for l in open(os.path.join(os.path.dirname(__file__), "golden", "fma_pairs.txt"))
+            if not l.startswith("#")]
+    for kind, x, c, g, sep, fused in rows:
+        x, c, g = (struct.unpack("<f", struct.pack("<I", int(t, 16)))[0] for t in (x, c, g))
+        g16 = np.array([g] * 9, dtype=np.float16)
+        if kind == "sub":
+            w_g, _, _, _ = _run_update(9, False, 1.0, c, 0.0, g16, np.full(9, x, np.float32), np.zeros(9, np.float32))
+            assert all(int(t) == int(sep, 16) for t in w_g.view(np.uint32))
+        else:
+            _, v_g, _, _ = _run_update(9, True, 1.0, 0.0, c, g16, np.zeros(9, np.float32), np.full(9, x, np.float32))
+            assert all(int(t) == int(sep, 16) for t in v_g.view(np.uint32))
+
+
+@pytest.mark.parametrize("bad", [np.inf, -np.inf, np.nan])
+@pytest.mark.parametrize("pos", [0, 4097, -1])
+def test_overflow_skips_everything(bad, pos):
+    n = 10007
+    rng = np.random.default_rng(3)
+    g16 = rng.standard_normal(n).astype(np.float16)
+    g16[pos] = bad
+    w = rng.standard_normal(n).astype(np.float32)
+    v = rng.standard_normal(n).astype(np.float32)
+    assert mpo.grad_nonfinite(g16, 1.0) == 1
+    w_g, v_g, h_g, flags = _run_update(n, True, 1.0, 0.1, 0.9, g16, w, v)
+    assert flags[0] == 1
+    assert w_g.tobytes() == w.tobytes() and v_g.tobytes() == v.tobytes() and not h_g.any()
+
+
+def test_nonfinite_flag_matches_oracle_on_loguniform():
+    b = _binding()
+    n = 1 << 22
+    for S in inputs.SCALE_SWEEP:
+        g = inputs.loguniform_grads(n, S)
+        inv = float(np.float32(1.0) / np.float32(S))
+        flag = torch.zeros(1, dtype=torch.int32, device="cuda")
+        b.mpt_grad_nonfinite(dev(g.view(np.uint16)), n, inv, flag)
+        torch.cuda.synchronize()
+        assert int(flag.item()) == mpo.grad_nonfinite(g, inv) == 0
+    g = inputs.loguniform_grads(n, 1.0)
+    g[-3] = np.inf
+    flag = torch.zeros(1, dtype=torch.int32, device="cuda")
+    b.mpt_grad_nonfinite(dev(g.view(np.uint16)), n, 1.0, flag)
+    assert int(flag.item()) == 1
+
+
+def test_update_loguniform_config_2b_bit_exact():
+    """Config 2b: 2^24 log-uniform gradients on a 4096x4096 layer, every scale of the sweep."""
+    n = 1 << 24
+    rng = np.random.default_rng(5)
+    w = (rng.standard_normal(n) / 64).astype(np.float32)
+    for S in inputs.SCALE_SWEEP:
+        g16 = inputs.loguniform_grads(n, S)
+        inv = np.float32(1.0) / np.float32(S)
+        w_ref = w.copy()
+        h_ref = np.zeros(n, dtype=np.uint16)
+        mpo.update_apply(g16, w_ref, None, h_ref, inv, np.float32(0.01), np.float32(0.0), False)
+        w_g, _, h_g, flags = _run_update(n, False, S, 0.01, 0.0, g16, w, np.zeros(1, np.float32).repeat(n))
+        assert flags.tolist() == [0, 0]
+        assert np.array_equal(w_g.view(np.uint32), w_ref.view(np.uint32))
+        assert np.array_equal(h_g, h_ref)
