@@ -1,0 +1,338 @@
+#!/usr/bin/env python
+"""Benchmark of the mixed-precision training step (forward GEMMs, scaled softmax-CE,
+backward GEMMs, FP32 master update) on synthetic data.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl mine|reference] [--workload NAME]
+
+One "step" is one pass of the whole hot path over one batch: mpt_forward,
+mpt_backward_scaled, mpt_step.  The default workload "large" is the large-MLP
+configuration (8 x 12288^2 ReLU layers + 12288 -> 32000 head, batch 4096, S = 8192,
+SGD momentum 0.9); "large_twin" and "tiny" are small cases.  Prints ONE JSON line on
+rank 0.  With N > 1 (launched by torch.distributed.run) every rank runs an independent
+replica of the step on its own GPU (the path has no exchange step); the time is the
+maximum over ranks and the value the sum of all ranks' work over that time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_1710_03740_b200 import inputs  # noqa: E402
+
+METRIC = "train_step_tflops"
+UNIT = "TFLOP/s"
+NOMINAL_FP16_TFLOPS = 2250.0
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def step_flops(cfg):
+    """GEMM flop of one iteration: forward + wgrad for every layer, dgrad for all but the first."""
+    B = cfg["batch"]
+    tot = 0
+    for l, (fin, fout, _) in enumerate(cfg["layers"]):
+        tot += 2 * B * fin * fout * (2 if l == 0 else 3)
+    return float(tot)
+
+
+def n_params(cfg):
+    return sum(fin * fout for fin, fout, _ in cfg["layers"])
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            d = json.load(open(p))
+            return {k: float(d[k]) for k in FALLBACK_PEAKS}, "measured"
+        except Exception:
+            pass
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU with nvidia-smi while a region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); smax.append(float(f[1])); power.append(float(f[2]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        # keep samples taken under load (clock above idle)
+        busy = [c for c in sm if c > 500] or sm
+        return {"sm_mhz": float(np.median(busy)) if busy else None,
+                "sm_max_mhz": max(smax) if smax else None,
+                "power_w_max": max(power) if power else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def oracle_operands(cfg, seconds_target):
+    from oracle import mpo
+    B = cfg["batch"]
+    fin, fout, _ = max(cfg["layers"], key=lambda l: l[0] * l[1])
+    cores = mpo.num_threads()
+    # ~1.3 GFLOP/s per core is typical for the plain loops; aim for `seconds_target`
+    rows = int(seconds_target * 1.3e9 * cores / (2.0 * fin * fout))
+    rows = max(cores, min(B, rows))
+    return inputs.gemm_operands(0, rows, fout, fin, seed=2, fast=True)
+
+
+def oracle_sample(cfg, seconds_target=12.0, operands=None):
+    """Times the CPU oracle, as it stands, on a slab of output rows of the dominant GEMM of
+    this workload (a hidden-layer forward product) and returns TFLOP/s."""
+    from oracle import mpo
+    B = cfg["batch"]
+    A, W = operands if operands is not None else oracle_operands(cfg, seconds_target)
+    rows, fin = A.shape
+    fout = W.shape[0]
+    cores = mpo.num_threads()
+    t0 = time.perf_counter()
+    mpo.gemm_f16(mpo.OP_FWD, A, W, relu=True)
+    dt = time.perf_counter() - t0
+    flops = 2.0 * rows * fin * fout
+    return {"value": flops / dt / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": "forward GEMM slab: %d of %d rows x N=%d x K=%d in %.1f s" % (rows, B, fout, fin, dt)}
+
+
+def run_reference(args, cfg, rank):
+    """Reference arm: the CPU oracle on the host cores, bounded sample per step."""
+    if rank != 0:
+        return
+    vals = []
+    ops = oracle_operands(cfg, 4.0)
+    for i in range(args.warmup + args.steps):
+        r = oracle_sample(cfg, operands=ops)
+        if i >= args.warmup:
+            vals.append(r)
+    v = float(np.mean([r["value"] for r in vals]))
+    sample = vals[-1]["sample"]
+    # time one full step would take at this rate
+    ms = step_flops(cfg) / (v * 1e12) * 1e3
+    out = {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+           "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+           "vs_baseline": None, "dtype": "f16", "data": "synthetic",
+           "config": {"workload": args.workload, "note": "CPU oracle, bounded sample per step, extrapolated"},
+           "cpu_baseline": {"value": v, "unit": UNIT, "cores": vals[-1]["cores"], "kind": "oracle", "sample": sample},
+           "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+           "gpu_launches": 0}
+    print(json.dumps(out), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="mine", choices=["mine", "reference"])
+    ap.add_argument("--workload", default="large", choices=sorted(inputs.MLP_CONFIGS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "mine" else args.warmup
+    cfg = inputs.MLP_CONFIGS[args.workload]
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    if args.impl == "reference":
+        run_reference(args, cfg, rank)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_1710_03740_b200 import binding as mpt   # raises if the CUDA library is missing
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    # ---- synthetic inputs (seeded; rank r uses seed + 100 r so replicas differ)
+    cfg = dict(cfg)
+    cfg["seed"] = cfg["seed"] + 100 * rank
+    big = n_params(cfg) > (1 << 26)
+    L = len(cfg["layers"])
+    net = mpt.Context(cfg["layers"], cfg["S"], cfg["lr"], cfg["momentum"], cfg["batch"], device=dev)
+    seqs = np.random.SeedSequence(cfg["seed"]).spawn(L + 2 * cfg["steps"])
+    for l, (fin, fout, _) in enumerate(cfg["layers"]):
+        scale = fin ** -0.5 * (cfg["head_scale"] if l == L - 1 else 1.0)
+        if big:
+            w16 = inputs.normal_f16_fast(seqs[l], (fout, fin), scale, threads=min(32, os.cpu_count() or 8))
+        else:
+            w16 = inputs.normal_f16(np.random.default_rng(seqs[l]), (fout, fin), scale)
+        net.set_master(l, w16.astype(np.float32))
+        del w16
+    X, Y = inputs.mlp_batches(cfg)
+    nb = X.shape[0]
+    Xd = [torch.from_numpy(X[t].view(np.int16)).to(dev) for t in range(nb)]
+    Yd = [torch.from_numpy(Y[t]).to(dev) for t in range(nb)]
+    Xp = [torch.from_numpy(X[t].view(np.int16)).pin_memory() for t in range(nb)]
+    Yp = [torch.from_numpy(Y[t]).pin_memory() for t in range(nb)]
+
+    def step_dev(t):
+        net.forward(Xd[t % nb])
+        net.backward_scaled(Yd[t % nb], want_loss=False)
+        net.step(want_flag=False)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident throughput
+    for t in range(args.warmup):
+        step_dev(t)
+    barrier()
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    if sampler:
+        sampler.start()
+        time.sleep(0.15)
+    n0 = net.launch_count()
+    net.profile(True)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record()
+    for t in range(args.steps):
+        step_dev(args.warmup + t)
+    ev1.record()
+    barrier()
+    ms_total = ev0.elapsed_time(ev1)
+    prof = net.profile_read()
+    net.profile(False)
+    launches = net.launch_count() - n0
+    clocks = sampler.stop() if sampler else None
+    # loss and flag of one more step, to show the job is live (outside the timed region)
+    net.forward(Xd[0])
+    loss = net.backward_scaled(Yd[0], want_loss=True)
+    flag = net.step(want_flag=True)
+
+    # ---- end to end through the host-buffer entry point (H2D of the batch, D2H of loss/flag per step)
+    for t in range(2):
+        net.train_step_host(Xp[t % nb], Yp[t % nb])
+    barrier()
+    t0 = time.perf_counter()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for t in range(args.steps):
+        net.train_step_host(Xp[t % nb], Yp[t % nb])
+    e1.record()
+    barrier()
+    # every call synchronises, so host wall-clock and device events bracket the same work
+    ms_e2e = max(e0.elapsed_time(e1), (time.perf_counter() - t0) * 1e3)
+
+    if world > 1:
+        tt = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms_total, ms_e2e = float(tt[0]), float(tt[1])
+
+    if rank == 0:
+        peaks, peak_src = measured_peaks()
+        fl = step_flops(cfg)
+        ms_step = ms_total / args.steps
+        value = fl * world / (ms_step * 1e-3) / 1e12
+        e2e_val = fl * world / (ms_e2e / args.steps * 1e-3) / 1e12
+        g_ms, g_work, g_n = prof["gemm"]
+        u_ms, u_work, u_n = prof["update"]
+        s_ms, s_work, s_n = prof["softmax"]
+        gemm_tflops = g_work / (g_ms * 1e-3) / 1e12 if g_ms > 0 else None
+        upd_gbs = u_work / (u_ms * 1e-3) / 1e9 if u_ms > 0 else None
+        sm_gbs = s_work / (s_ms * 1e-3) / 1e9 if s_ms > 0 else None
+        peak_t = peaks["bf16_tflops_sustained"]
+        traffic = None
+        tp = os.path.join(ROOT, "profiles", "traffic.json")
+        if os.path.exists(tp):
+            try:
+                traffic = json.load(open(tp)).get(args.workload, {}).get("gemm_dram_bytes_per_launch")
+            except Exception:
+                traffic = None
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f16", "data": "synthetic",
+            "config": {"workload": args.workload, "layers": L, "batch": cfg["batch"], "params": n_params(cfg),
+                       "S": cfg["S"], "momentum": cfg["momentum"], "parallelism": "replicas only",
+                       "l2": "inputs larger than L2 (weights %.1f GB per pass)" % (n_params(cfg) * 2 / 1e9),
+                       "flop_per_step": fl},
+            "frac_of_nominal_fp16_peak": value / world / NOMINAL_FP16_TFLOPS,
+            "roofline": {"bound": "tensor", "kernel": "k_gemm_tc (all GEMM launches of the step)",
+                         "achieved": gemm_tflops, "peak": peak_t, "peak_source": peak_src + " (sustained bf16 GEMM; fp16 has the same nominal rate)",
+                         "unit": "TFLOP/s", "frac": (gemm_tflops / peak_t) if gemm_tflops else None,
+                         "frac_of_nominal": (gemm_tflops / NOMINAL_FP16_TFLOPS) if gemm_tflops else None,
+                         "launches": g_n, "avg_launch_ms": g_ms / g_n if g_n else None, "traffic": traffic},
+            "update": {"bound": "hbm", "kernel": "k_update_vec", "achieved": upd_gbs, "peak": peaks["hbm_gbs"],
+                       "peak_source": peak_src, "unit": "GB/s", "frac": (upd_gbs / peaks["hbm_gbs"]) if upd_gbs else None,
+                       "frac_of_nominal": (upd_gbs / NOMINAL_HBM_GBS) if upd_gbs else None,
+                       "bytes_per_param": 20 if cfg["momentum"] else 12, "avg_launch_ms": u_ms / u_n if u_n else None},
+            "softmax": {"bound": "hbm", "achieved": sm_gbs, "unit": "GB/s", "avg_launch_ms": s_ms / s_n if s_n else None},
+            "phase_ms_per_step": {"gemm": g_ms / args.steps, "update": u_ms / args.steps, "softmax": s_ms / args.steps},
+            "e2e": {"value": e2e_val, "unit": UNIT, "ms_per_step": ms_e2e / args.steps,
+                    "h2d_bytes_per_step": int(X[0].nbytes + Y[0].nbytes), "d2h_bytes_per_step": 64},
+            "gpu_launches": int(launches),
+            "clocks": clocks,
+            "last_loss": loss, "last_overflow": flag,
+        }
+        if not args.no_cpu_baseline:
+            try:
+                out["cpu_baseline"] = oracle_sample(cfg)
+            except Exception as ex:  # the oracle is a reported baseline; never fatal for the bench line
+                out["cpu_baseline"] = {"value": None, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
+                                       "sample": "failed: %r" % (ex,)}
+        print(json.dumps(out), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -173,6 +173,22 @@ int mpt_set_momentum(mpt_ctx *ctx, int layer, const float *src_host, size_t n);
  * benchmarks). */
 int mpt_launch_count(mpt_ctx *ctx, long long *count_out);
 
+/* Per-kernel timing with CUDA events on the context's stream, for benchmarks.
+ * mpt_profile(ctx, 1) synchronises, clears the counters and starts bracketing every
+ * kernel launch of this context with a pair of events; mpt_profile(ctx, 0) stops.
+ * mpt_profile_read synchronises and returns, per kernel class (MPT_PROF_*), the
+ * summed device time in milliseconds, the summed algorithmic work (GEMM: 2*M*N*K
+ * flop; update: 12 or 20 bytes per parameter; softmax: 4 bytes per logit) and the
+ * number of launches since profiling was enabled.  Each array has
+ * MPT_PROF_CLASSES entries. */
+#define MPT_PROF_GEMM 0
+#define MPT_PROF_UPDATE 1
+#define MPT_PROF_SOFTMAX 2
+#define MPT_PROF_OTHER 3
+#define MPT_PROF_CLASSES 4
+int mpt_profile(mpt_ctx *ctx, int enable);
+int mpt_profile_read(mpt_ctx *ctx, double *ms_out, double *work_out, long long *launches_out);
+
 /* Message for the last non-OK status of this context (never null). */
 const char *mpt_last_error(mpt_ctx *ctx);
 

@@ -25,7 +25,8 @@ T_W16, T_GRAD16, T_ACT16, T_DACT16, T_MOMENTUM32, T_MASTER32 = range(6)
 # every symbol include/mpt.h declares
 EXPORTS = ["mpt_workspace_bytes", "mpt_create", "mpt_set_master", "mpt_forward", "mpt_backward_scaled",
            "mpt_step", "mpt_get_master", "mpt_train_step_host", "mpt_set_scale", "mpt_set_lr",
-           "mpt_get_tensor", "mpt_set_grad", "mpt_set_momentum", "mpt_launch_count", "mpt_last_error",
+           "mpt_get_tensor", "mpt_set_grad", "mpt_set_momentum", "mpt_launch_count", "mpt_profile",
+           "mpt_profile_read", "mpt_last_error",
            "mpt_destroy", "mpt_gemm_f16", "mpt_recast", "mpt_grad_nonfinite", "mpt_update_flat",
            "mpt_softmax_ce", "mpt_version"]
 
@@ -66,6 +67,8 @@ def lib() -> C.CDLL:
     L.mpt_set_grad.argtypes = [vp, i32, vp, sz]
     L.mpt_set_momentum.argtypes = [vp, i32, vp, sz]
     L.mpt_launch_count.argtypes = [vp, C.POINTER(C.c_longlong)]
+    L.mpt_profile.argtypes = [vp, i32]
+    L.mpt_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_longlong)]
     L.mpt_last_error.argtypes = [vp]
     L.mpt_last_error.restype = C.c_char_p
     L.mpt_destroy.argtypes = [vp]
@@ -216,6 +219,16 @@ class Context:
     def set_momentum(self, layer, v):
         v = np.ascontiguousarray(v, dtype=np.float32)
         _check(lib().mpt_set_momentum(self._ctx, layer, _hptr(v), v.size), self._ctx)
+
+    def profile(self, enable):
+        _check(lib().mpt_profile(self._ctx, int(bool(enable))), self._ctx)
+
+    def profile_read(self):
+        """{class name: (milliseconds, algorithmic work, launches)} since profile(True)."""
+        ms, work, n = (C.c_double * 4)(), (C.c_double * 4)(), (C.c_longlong * 4)()
+        _check(lib().mpt_profile_read(self._ctx, ms, work, n), self._ctx)
+        names = ("gemm", "update", "softmax", "other")
+        return {names[k]: (float(ms[k]), float(work[k]), int(n[k])) for k in range(4)}
 
     def launch_count(self):
         n = C.c_longlong(0)

@@ -101,6 +101,14 @@ struct mpt_ctx {
     long long launches = 0;
     bool disable_tc = false;
     std::string err;
+    // optional per-kernel timing with CUDA events (mpt_profile)
+    bool profiling = false;
+    struct Span { cudaEvent_t a, b; int cls; };
+    std::vector<Span> spans;
+    std::vector<Span> pool;
+    double prof_ms[MPT_PROF_CLASSES] = {0, 0, 0, 0};
+    double prof_work[MPT_PROF_CLASSES] = {0, 0, 0, 0};
+    long long prof_launches[MPT_PROF_CLASSES] = {0, 0, 0, 0};
 };
 
 namespace {
@@ -136,11 +144,35 @@ int usable(mpt_ctx *c)
     return MPT_OK;
 }
 
+// Brackets one kernel launch with CUDA events on the context's stream when profiling.
+struct ProfSpan {
+    mpt_ctx *c;
+    bool on;
+    mpt_ctx::Span sp;
+    ProfSpan(mpt_ctx *ctx, int cls, double work) : c(ctx), on(ctx->profiling)
+    {
+        if (!on) return;
+        if (!c->pool.empty()) { sp = c->pool.back(); c->pool.pop_back(); }
+        else if (cudaEventCreate(&sp.a) != cudaSuccess || cudaEventCreate(&sp.b) != cudaSuccess) { on = false; return; }
+        sp.cls = cls;
+        c->prof_work[cls] += work;
+        c->prof_launches[cls] += 1;
+        cudaEventRecord(sp.a, c->stream);
+    }
+    ~ProfSpan()
+    {
+        if (!on) return;
+        cudaEventRecord(sp.b, c->stream);
+        c->spans.push_back(sp);
+    }
+};
+
 // One product of the iteration, on the tensor-core kernel when the operands allow it.
 int gemm(mpt_ctx *c, int op, int M, int N, int K, const uint16_t *A, int lda, const uint16_t *B, int ldb, uint16_t *C,
          int ldc, bool relu, const uint16_t *mask, int ldmask, uint32_t *nonfinite)
 {
     cudaError_t e;
+    ProfSpan span(c, MPT_PROF_GEMM, 2.0 * M * N * K);
     if (!c->disable_tc && tc_gemm_supported(op, M, N, K, A, lda, B, ldb, C, ldc, mask, ldmask))
         e = launch_gemm_tc(op, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite,
                            c->status + ST_KERNEL_ERR, c->stream);
@@ -192,9 +224,12 @@ int do_backward(mpt_ctx *c, const int32_t *labels_dev)
     CK(cudaMemsetAsync(c->status, 0, 3 * sizeof(uint32_t), c->stream), "status clear");
     Layer &last = c->layers[L - 1];
     int nl = 0;
-    cudaError_t e = launch_softmax_ce(last.act, last.ld_out, labels_dev, B, last.out, c->S, last.dact, last.ld_out,
-                                      c->row_loss, (float *)(c->status + ST_LOSS), c->status + ST_BAD_LABELS, c->stream,
-                                      &nl);
+    cudaError_t e;
+    {
+        ProfSpan span(c, MPT_PROF_SOFTMAX, 4.0 * B * last.out);
+        e = launch_softmax_ce(last.act, last.ld_out, labels_dev, B, last.out, c->S, last.dact, last.ld_out, c->row_loss,
+                              (float *)(c->status + ST_LOSS), c->status + ST_BAD_LABELS, c->stream, &nl);
+    }
     c->launches += nl;
     if (e != cudaSuccess) return cuda_fail(c, e, "softmax launch");
     for (int l = L - 1; l >= 0; l--) {
@@ -221,8 +256,12 @@ int do_step(mpt_ctx *c)
     if (!c->have_grads) return fail(c, MPT_ERR_STATE, "mpt_step needs gradients (mpt_backward_scaled or mpt_set_grad)");
     const float inv = 1.0f / c->S;
     CK(cudaMemsetAsync(c->status + ST_OVERFLOW_SEEN, 0, sizeof(uint32_t), c->stream), "status clear");
-    cudaError_t e = launch_update(c->g16, c->master, c->mom, c->w16, c->plan.P_pad, inv, c->lr, c->mu, c->use_momentum,
-                                  c->status + ST_OVERFLOW, c->stream);
+    cudaError_t e;
+    {
+        ProfSpan span(c, MPT_PROF_UPDATE, (c->use_momentum ? 20.0 : 12.0) * (double)c->plan.P_pad);
+        e = launch_update(c->g16, c->master, c->mom, c->w16, c->plan.P_pad, inv, c->lr, c->mu, c->use_momentum,
+                          c->status + ST_OVERFLOW, c->stream);
+    }
     c->launches++;
     if (e != cudaSuccess) return cuda_fail(c, e, "update launch");
     return MPT_OK;
@@ -300,7 +339,44 @@ int mpt_create(const mpt_layer_desc *layers, int n_layers, float S, float lr, fl
     return MPT_OK;
 }
 
-void mpt_destroy(mpt_ctx *c) { delete c; }
+void mpt_destroy(mpt_ctx *c)
+{
+    if (!c) return;
+    for (auto &sp : c->spans) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
+    for (auto &sp : c->pool) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
+    delete c;
+}
+
+int mpt_profile(mpt_ctx *c, int enable)
+{
+    int r = usable(c);
+    if (r != MPT_OK) return r;
+    CK(cudaStreamSynchronize(c->stream), "stream synchronize");
+    for (auto &sp : c->spans) c->pool.push_back(sp);
+    c->spans.clear();
+    for (int k = 0; k < MPT_PROF_CLASSES; k++) { c->prof_ms[k] = 0; c->prof_work[k] = 0; c->prof_launches[k] = 0; }
+    c->profiling = enable != 0;
+    return MPT_OK;
+}
+
+int mpt_profile_read(mpt_ctx *c, double *ms_out, double *work_out, long long *launches_out)
+{
+    int r = usable(c);
+    if (r != MPT_OK) return r;
+    if (!ms_out || !work_out || !launches_out) return fail(c, MPT_ERR_INVALID_ARG, "null output");
+    CK(cudaStreamSynchronize(c->stream), "stream synchronize");
+    for (auto &sp : c->spans) {
+        float ms = 0.0f;
+        CK(cudaEventElapsedTime(&ms, sp.a, sp.b), "event elapsed time");
+        c->prof_ms[sp.cls] += ms;
+        c->pool.push_back(sp);
+    }
+    c->spans.clear();
+    for (int k = 0; k < MPT_PROF_CLASSES; k++) {
+        ms_out[k] = c->prof_ms[k]; work_out[k] = c->prof_work[k]; launches_out[k] = c->prof_launches[k];
+    }
+    return MPT_OK;
+}
 
 const char *mpt_last_error(mpt_ctx *c) { return c ? c->err.c_str() : "null context"; }
 
