@@ -1,0 +1,132 @@
+"""Per-kernel timing through the C ABI (CUDA events, synthetic data): the isolated GEMM
+sweep, the bigLSTM-shaped products, the master-update pass and the softmax cross-entropy.
+
+    python -m paper_1710_03740_b200.kernel_bench gemm   [--shape MxNxK ...] [--op 0 1 2] [--iters 20]
+    python -m paper_1710_03740_b200.kernel_bench update [--params N] [--momentum 0|1] [--iters 20]
+    python -m paper_1710_03740_b200.kernel_bench softmax [--rows B] [--classes C] [--iters 20]
+
+Prints one JSON line per case: best-of and back-to-back ("sustained") rates.  Working sets
+are larger than the 126 MB L2 unless the shape itself is smaller; small cases say so.
+`--compare-library` adds torch.matmul (cuBLAS) on the same operands as context.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+
+import torch
+
+from . import binding as mpt
+from . import inputs
+
+OPS = {0: "fwd", 1: "dgrad", 2: "wgrad"}
+
+
+def _time(fn, iters, warmup=3):
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    best = float("inf")
+    for _ in range(min(iters, 5)):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        torch.cuda.synchronize()
+        best = min(best, e0.elapsed_time(e1))
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return best, e0.elapsed_time(e1) / iters
+
+
+def bench_gemm(M, N, K, op, iters, compare=False, flags=mpt.GEMM_FORCE_TC):
+    sa = (K, M) if op == 2 else (M, K)
+    sb = (N, K) if op == 0 else (K, N)
+    g = torch.Generator(device="cuda").manual_seed(2)
+    A = (torch.randn(sa, device="cuda", generator=g) * K ** -0.5).half()
+    B = (torch.randn(sb, device="cuda", generator=g) * K ** -0.5).half()
+    C = torch.empty((M, N), dtype=torch.half, device="cuda")
+    st = torch.zeros(4, dtype=torch.int32, device="cuda")
+    fn = lambda: mpt.mpt_gemm_f16(op, M, N, K, A, sa[1], B, sb[1], C, N, flags, None, 0, None, st)  # noqa: E731
+    best, sus = _time(fn, iters)
+    fl = 2.0 * M * N * K
+    out = {"kernel": "gemm", "op": OPS[op], "M": M, "N": N, "K": K, "best_ms": best, "sustained_ms": sus,
+           "best_tflops": fl / best / 1e9, "sustained_tflops": fl / sus / 1e9, "device_error": int(st[0]),
+           "working_set_mb": (A.numel() + B.numel() + C.numel()) * 2 / 1e6}
+    if compare:
+        if op == 0:
+            ref = lambda: torch.matmul(A, B.t())  # noqa: E731
+        elif op == 1:
+            ref = lambda: torch.matmul(A, B)  # noqa: E731
+        else:
+            ref = lambda: torch.matmul(A.t(), B)  # noqa: E731
+        rb, rs = _time(ref, iters)
+        out["library_best_tflops"] = fl / rb / 1e9
+        out["library_sustained_tflops"] = fl / rs / 1e9
+    return out
+
+
+def bench_update(n, momentum, iters):
+    g = torch.Generator(device="cuda").manual_seed(3)
+    g16 = (torch.randn(n, device="cuda", generator=g) * 37).half()
+    w32 = torch.randn(n, device="cuda", generator=g)
+    v = torch.zeros(n, device="cuda") if momentum else None
+    w16 = torch.empty(n, dtype=torch.half, device="cuda")
+    flags = torch.zeros(2, dtype=torch.int32, device="cuda")
+    fn = lambda: mpt.mpt_update_flat(g16, w32, v, w16, n, 1.0 / 512, 1e-4, 0.9, momentum, False, flags)  # noqa: E731
+    best, sus = _time(fn, iters)
+    bpp = 20 if momentum else 12
+    return {"kernel": "update", "params": n, "momentum": bool(momentum), "bytes_per_param": bpp, "best_ms": best,
+            "sustained_ms": sus, "best_gbs": bpp * n / best / 1e6, "sustained_gbs": bpp * n / sus / 1e6,
+            "working_set_mb": bpp * n / 2e6, "flags": flags.tolist()}
+
+
+def bench_softmax(B, Cn, iters):
+    g = torch.Generator(device="cuda").manual_seed(4)
+    z = (torch.randn((B, Cn), device="cuda", generator=g) * 3).half()
+    y = torch.randint(0, Cn, (B,), device="cuda", generator=g, dtype=torch.int32)
+    dz = torch.empty_like(z)
+    rl = torch.empty(B, device="cuda")
+    loss = torch.empty(1, device="cuda")
+    fn = lambda: mpt.mpt_softmax_ce(z, Cn, y, B, Cn, 8192.0, dz, Cn, rl, loss, None)  # noqa: E731
+    best, sus = _time(fn, iters)
+    by = 4.0 * B * Cn
+    return {"kernel": "softmax_ce", "rows": B, "classes": Cn, "best_ms": best, "sustained_ms": sus,
+            "best_gbs": by / best / 1e6, "sustained_gbs": by / sus / 1e6, "loss": float(loss.item())}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    sub = ap.add_subparsers(dest="cmd", required=True)
+    g = sub.add_parser("gemm")
+    g.add_argument("--shape", nargs="*", default=None, help="MxNxK; default: the sweep and the bigLSTM shapes")
+    g.add_argument("--op", nargs="*", type=int, default=[0, 1, 2])
+    g.add_argument("--iters", type=int, default=20)
+    g.add_argument("--compare-library", action="store_true")
+    u = sub.add_parser("update")
+    u.add_argument("--params", type=int, default=150994944)
+    u.add_argument("--momentum", type=int, default=1)
+    u.add_argument("--iters", type=int, default=20)
+    s = sub.add_parser("softmax")
+    s.add_argument("--rows", type=int, default=4096)
+    s.add_argument("--classes", type=int, default=32000)
+    s.add_argument("--iters", type=int, default=20)
+    args = ap.parse_args()
+    if args.cmd == "gemm":
+        shapes = ([tuple(int(x) for x in t.split("x")) for t in args.shape] if args.shape
+                  else inputs.GEMM_SWEEP + [inputs.LSTM_GATE, inputs.LSTM_PROJ])
+        for (M, N, K) in shapes:
+            for op in args.op:
+                print(json.dumps(bench_gemm(M, N, K, op, args.iters, args.compare_library)), flush=True)
+    elif args.cmd == "update":
+        print(json.dumps(bench_update(args.params, args.momentum, args.iters)), flush=True)
+    else:
+        print(json.dumps(bench_softmax(args.rows, args.classes, args.iters)), flush=True)
+
+
+if __name__ == "__main__":
+    main()
