@@ -240,6 +240,35 @@ int mpt_softmax_ce(const uint16_t *z_dev, int ldz, const int32_t *labels_dev, in
                    uint16_t *dz_dev, int lddz, float *row_loss_dev, float *loss_dev,
                    uint32_t *bad_labels_dev, void *cuda_stream);
 
+/* mpt_softmax_ce without the caller-provided scratch.  (The paper has no counterpart:
+ * this entry point exists for the sake of callers, not of the method.)
+ *
+ * Some callers cannot obtain device memory at the point where they need the loss: code
+ * that runs inside a framework which hands it a fixed set of tensors and owns every
+ * other byte of the GPU, or a latency-critical loop that must not call cudaMalloc
+ * because that call synchronises the whole device.  mpt_softmax_ce asks such a caller
+ * for a float[B] scratch buffer it may not have.  This variant computes exactly the
+ * same results (same kernels, same arithmetic) but keeps the per-row losses in a
+ * fixed array inside the library, so the caller passes only inputs and outputs.
+ * It calls no cudaMalloc/cudaFree and no allocating library routine.
+ *
+ *   - Limit: B <= MPT_SOFTMAX_STATIC_MAX_ROWS (65536 rows, a 256 KiB array that every
+ *     GPU which loads the library holds until the process exits).  A larger B returns
+ *     MPT_ERR_SHAPE and launches nothing; use mpt_softmax_ce for such batches.
+ *   - The first call made on a device looks up the array's device address (a host-side
+ *     runtime query, done once per device with that device current).  Make that first
+ *     call during set-up, before any stream capture.
+ *   - All calls on a GPU share the one array.  Two calls whose kernels overlap on the
+ *     GPU (different streams, or different threads) race on it and may return wrong
+ *     losses; calls on one stream are ordered and safe.  The array keeps the previous
+ *     call's values, which is harmless: each call overwrites rows 0..B-1 before reading
+ *     them and reads nothing else.
+ * Other arguments, results and error codes are those of mpt_softmax_ce. */
+#define MPT_SOFTMAX_STATIC_MAX_ROWS 65536
+int mpt_softmax_ce_static(const uint16_t *z_dev, int ldz, const int32_t *labels_dev, int B, int C, float S,
+                          uint16_t *dz_dev, int lddz, float *loss_dev, uint32_t *bad_labels_dev,
+                          void *cuda_stream);
+
 /* Library build identification, e.g. "mpt 0.1 sm_100a". */
 const char *mpt_version(void);
 

@@ -28,7 +28,7 @@ EXPORTS = ["mpt_workspace_bytes", "mpt_create", "mpt_set_master", "mpt_forward",
            "mpt_get_tensor", "mpt_set_grad", "mpt_set_momentum", "mpt_launch_count", "mpt_profile",
            "mpt_profile_read", "mpt_last_error",
            "mpt_destroy", "mpt_gemm_f16", "mpt_recast", "mpt_grad_nonfinite", "mpt_update_flat",
-           "mpt_softmax_ce", "mpt_version"]
+           "mpt_softmax_ce", "mpt_softmax_ce_static", "mpt_version"]
 
 
 class MptError(RuntimeError):
@@ -78,6 +78,7 @@ def lib() -> C.CDLL:
     L.mpt_grad_nonfinite.argtypes = [vp, sz, f32, vp, vp]
     L.mpt_update_flat.argtypes = [vp, vp, vp, vp, sz, f32, f32, f32, i32, i32, vp, vp]
     L.mpt_softmax_ce.argtypes = [vp, i32, vp, i32, i32, f32, vp, i32, vp, vp, vp, vp]
+    L.mpt_softmax_ce_static.argtypes = [vp, i32, vp, i32, i32, f32, vp, i32, vp, vp, vp]
     L.mpt_version.restype = C.c_char_p
     L.mpt_version.argtypes = []
     _lib = L
@@ -261,6 +262,13 @@ def mpt_update_flat(g16, w32, v, w16, n, inv_S, lr, mu, use_momentum, detect, fl
 def mpt_softmax_ce(z, ldz, labels, B, Cn, S, dz, lddz, row_loss, loss, bad_labels=None, stream=None):
     _check(lib().mpt_softmax_ce(_dptr(z), ldz, _dptr(labels), B, Cn, float(S), _dptr(dz), lddz, _dptr(row_loss),
                                 _dptr(loss), _dptr(bad_labels), _stream_ptr(stream)))
+
+
+def mpt_softmax_ce_static(z, ldz, labels, B, Cn, S, dz, lddz, loss, bad_labels=None, stream=None):
+    """mpt_softmax_ce for callers that cannot provide the float[B] scratch: the per-row losses
+    live in a fixed array inside the library (B <= 65536; calls that overlap on the GPU race)."""
+    _check(lib().mpt_softmax_ce_static(_dptr(z), ldz, _dptr(labels), B, Cn, float(S), _dptr(dz), lddz, _dptr(loss),
+                                       _dptr(bad_labels), _stream_ptr(stream)))
 
 
 def mpt_version() -> str:

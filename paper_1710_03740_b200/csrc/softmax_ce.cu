@@ -174,3 +174,46 @@ cudaError_t launch_softmax_ce(const uint16_t *z, int ldz, const int32_t *labels,
 }
 
 }  // namespace mpt
+
+// ---------------------------------------------------------------------------------
+// Variant of mpt_softmax_ce whose per-row loss scratch lives inside the library.
+//
+// The array below is part of the loaded module: every GPU that loads this library
+// holds these 256 KiB from load until the process exits, and every call on that GPU
+// shares them.  In host code the name g_static_row_loss is only a handle for the
+// symbol, not an address a kernel can use; the device address is obtained once per
+// device with cudaGetSymbolAddress while that device is current, and that pointer
+// is what the kernels receive.
+static __device__ __align__(256) float g_static_row_loss[MPT_SOFTMAX_STATIC_MAX_ROWS];
+
+namespace {
+constexpr int kMaxDevices = 64;
+float *g_static_ptr[kMaxDevices];   // per device, filled on the first call made with that device current
+}  // namespace
+
+extern "C" int mpt_softmax_ce_static(const uint16_t *z_dev, int ldz, const int32_t *labels_dev, int B, int C, float S,
+                                     uint16_t *dz_dev, int lddz, float *loss_dev, uint32_t *bad_labels_dev,
+                                     void *cuda_stream)
+{
+    if (!z_dev || !labels_dev || !dz_dev || !loss_dev) return MPT_ERR_INVALID_ARG;
+    if (B < 0 || C < 0 || ldz < C || lddz < C) return MPT_ERR_SHAPE;
+    if (B > MPT_SOFTMAX_STATIC_MAX_ROWS) return MPT_ERR_SHAPE;   // the built-in scratch holds one float per row
+    if (z_dev == dz_dev) return MPT_ERR_INVALID_ARG;
+    int device = -1;
+    if (cudaGetDevice(&device) != cudaSuccess) return MPT_ERR_CUDA;
+    if (device < 0 || device >= kMaxDevices) return MPT_ERR_INTERNAL;
+    if (!g_static_ptr[device]) {
+        float *p = nullptr;
+        if (cudaGetSymbolAddress((void **)&p, g_static_row_loss) != cudaSuccess || !p) return MPT_ERR_CUDA;
+        g_static_ptr[device] = p;
+    }
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    cudaError_t e = cudaSuccess;
+    if (bad_labels_dev) e = cudaMemsetAsync(bad_labels_dev, 0, sizeof(uint32_t), st);
+    // Nothing in the scratch has to start at zero: rows 0..B-1 are each written by the row
+    // kernel before the mean kernel reads exactly those rows; older contents are never read.
+    if (e == cudaSuccess)
+        e = mpt::launch_softmax_ce(z_dev, ldz, labels_dev, B, C, S, dz_dev, lddz, g_static_ptr[device], loss_dev,
+                                   bad_labels_dev, st, nullptr);
+    return e == cudaSuccess ? MPT_OK : MPT_ERR_CUDA;
+}
