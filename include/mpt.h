@@ -64,8 +64,12 @@ extern "C" {
 /* mpt_gemm_f16 flags */
 #define MPT_GEMM_RELU 1u      /* apply x > 0 ? x : +0 to the FP32 sum before rounding */
 #define MPT_GEMM_FORCE_SIMT 2u /* use the plain CUDA-core kernel (sequential-k FP32 sum) */
-#define MPT_GEMM_FORCE_TC 4u   /* require the tcgen05 kernel; MPT_ERR_SHAPE if the operands
-                                  do not meet its alignment rules */
+#define MPT_GEMM_FORCE_TC 4u   /* require the single-CTA tcgen05 kernel (128x256 tiles);
+                                  MPT_ERR_SHAPE if the operands do not meet its alignment rules */
+#define MPT_GEMM_FORCE_PAIR 8u /* require the CTA-pair tcgen05 kernel (cta_group::2, 256x256 tiles);
+                                  same alignment rules.  Without a FORCE flag the library picks the
+                                  pair kernel when the output has at least 128 tiles of 256x256,
+                                  else the single-CTA one */
 
 /* mpt_get_tensor kinds */
 #define MPT_T_W16 0        /* FP16 working weights   [out, in]            */

@@ -19,8 +19,10 @@
 // word, raises a CTA-wide abort flag and all roles fall through to the common exit,
 // which frees the tensor memory.
 #include <cuda.h>
+#include <cstdlib>
 
 #include "mpt_common.cuh"
+#include "tc_ptx.cuh"
 
 namespace mpt {
 
@@ -32,116 +34,6 @@ static constexpr int MN_BOX_BYTES = 64 * BLOCK_K * 2;        // one 64(mn) x 64(
 static constexpr int TMEM_COLS = 512;
 static constexpr int NUM_THREADS = 192;
 static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
-static constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
-
-// ----------------------------------------------------------------- PTX wrappers
-
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.b32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok;
-}
-__device__ __forceinline__ unsigned long long global_ns()
-{
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-
-// Bounded wait.  Returns false when the CTA is aborting or the time limit expired.
-__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag)
-{
-    unsigned long long t0 = 0;
-    for (uint32_t it = 0;; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 127u) == 127u) {
-            if (*abort_flag) return false;
-            unsigned long long now = global_ns();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > WAIT_LIMIT_NS) return false;
-        }
-    }
-}
-
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
-        : "memory");
-}
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void tc_commit(uint32_t bar)
-{
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-
-__device__ __forceinline__ void tc_mma_f16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                           uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-
-__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32])
-{
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr)
-        : "memory");
-}
-__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// Shared-memory matrix descriptor (tcgen05): start address, leading/stride byte
-// offsets (all >> 4), descriptor version 1, 128-byte swizzle.
-//   K-major  operand: rows of 128 bytes (64 k), 8-row groups 1024 bytes apart (stride offset);
-//                     the leading offset is unused with swizzling.
-//   MN-major operand: 64 k-rows of 128 bytes (64 mn) per box, 8-k groups 1024 bytes apart
-//                     (stride offset), the next 64 mn one box (8192 bytes) further (leading offset).
-__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes)
-{
-    uint64_t d = 0;
-    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
-    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
-    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
-    d |= (uint64_t)1 << 46;  // descriptor version (Blackwell)
-    d |= (uint64_t)2 << 61;  // SWIZZLE_128B
-    return d;
-}
 
 // Instruction descriptor, kind::f16: D = F32, A = B = F16, majors, N >> 3, M >> 4.
 __host__ __device__ constexpr uint32_t make_idesc(bool a_mn, bool b_mn)
@@ -159,6 +51,9 @@ struct TcParams {
     int relu;
     uint32_t *nonfinite_flag;
     uint32_t *status;  // may be null
+#ifdef MPT_TC_TRACE
+    int dbg;
+#endif
     int tiles_m, tiles_n, group_m;
 };
 
@@ -222,21 +117,22 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            uint32_t issued = 0;
+            uint32_t issued = 0, s = 0, ph = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
                 int mb, nb;
                 tile_coords(p, tile, mb, nb);
                 const int m0 = mb * BLOCK_M, n0 = nb * BLOCK_N;
-                for (int kb = 0; kb < nkb; kb++, issued++) {
-                    const int s = issued % STAGES;
-                    const uint32_t ph = (issued / STAGES) & 1u;
-                    if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) {
+                for (int kb = 0; kb < nkb; kb++, issued++, s = (s + 1 == STAGES) ? 0 : s + 1, ph ^= (s == 0)) {
+                    if (!mbar_try_wait(empty_bar(s), ph ^ 1u) && !mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) {
                         if (!*abort_flag) report(p, abort_flag, KERR_WAIT_EMPTY);
                         ok = false;
                         break;
                     }
                     const uint32_t sa = base + s * STAGE_BYTES, sb = sa + A_STAGE_BYTES;
+#ifdef MPT_TC_TRACE
+                    if ((p.dbg & 1) && issued >= (uint32_t)STAGES) { mbar_arrive(full_bar(s)); continue; }
+#endif
                     mbar_arrive_expect_tx(full_bar(s), STAGE_BYTES);
                     const int k0 = kb * BLOCK_K;
                     if (A_MN) {
@@ -266,39 +162,46 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         // -------------------------------------------------------------- MMA issuer
         if (lane == 0) {
             constexpr uint32_t idesc = make_idesc(A_MN, B_MN);
-            uint32_t consumed = 0;
+            // descriptor halves: only the start address (low word) changes with stage and k.
+            // K-major: 16 k = 32 bytes along the swizzled row; MN-major: 16 k-rows of 128 bytes.
+            constexpr uint32_t KSTEP_A = (A_MN ? UMMA_K * 128 : UMMA_K * 2) >> 4;
+            constexpr uint32_t KSTEP_B = (B_MN ? UMMA_K * 128 : UMMA_K * 2) >> 4;
+            const uint32_t a_hi = desc_hi(1024), b_hi = desc_hi(1024);
+            const uint32_t a_lo0 = desc_lo(base, A_MN ? MN_BOX_BYTES : 16);
+            const uint32_t b_lo0 = desc_lo(base + A_STAGE_BYTES, B_MN ? MN_BOX_BYTES : 16);
+            uint32_t s = 0, ph = 0;
             bool ok = true;
             int t = 0;
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, t++) {
                 const int buf = t & 1;
                 const uint32_t acc_ph = (t >> 1) & 1u;
-                if (!mbar_wait(acce_bar(buf), acc_ph ^ 1u, abort_flag)) {
+                if (!mbar_try_wait(acce_bar(buf), acc_ph ^ 1u) && !mbar_wait(acce_bar(buf), acc_ph ^ 1u, abort_flag)) {
                     if (!*abort_flag) report(p, abort_flag, KERR_WAIT_ACC_FREE);
                     ok = false;
                     break;
                 }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BLOCK_N);
-                for (int kb = 0; kb < nkb; kb++, consumed++) {
-                    const int s = consumed % STAGES;
-                    const uint32_t ph = (consumed / STAGES) & 1u;
-                    if (!mbar_wait(full_bar(s), ph, abort_flag)) {
+                uint32_t acc = 0;                       // first MMA of a tile overwrites the accumulator
+                for (int kb = 0; kb < nkb; kb++) {
+                    if (!mbar_try_wait(full_bar(s), ph) && !mbar_wait(full_bar(s), ph, abort_flag)) {
                         if (!*abort_flag) report(p, abort_flag, KERR_WAIT_FULL);
                         ok = false;
                         break;
                     }
                     tc_fence_after();
-                    const uint32_t sa = base + s * STAGE_BYTES, sb = sa + A_STAGE_BYTES;
+                    const uint32_t alo = a_lo0 + s * (uint32_t)(STAGE_BYTES >> 4);
+                    const uint32_t blo = b_lo0 + s * (uint32_t)(STAGE_BYTES >> 4);
 #pragma unroll
                     for (int k = 0; k < BLOCK_K / UMMA_K; k++) {
-                        // K-major: 16 k = 32 bytes along the swizzled row; MN-major: 16 k-rows of 128 bytes
-                        const uint64_t ad = A_MN ? make_desc(sa + k * (UMMA_K * 128), MN_BOX_BYTES, 1024)
-                                                 : make_desc(sa + k * (UMMA_K * 2), 16, 1024);
-                        const uint64_t bd = B_MN ? make_desc(sb + k * (UMMA_K * 128), MN_BOX_BYTES, 1024)
-                                                 : make_desc(sb + k * (UMMA_K * 2), 16, 1024);
-                        tc_mma_f16(d_tmem, ad, bd, idesc, (kb | k) != 0 ? 1u : 0u);
+#ifdef MPT_TC_TRACE
+                        if (p.dbg & 4) continue;
+#endif
+                        tc_mma_f16(d_tmem, desc_join(alo + k * KSTEP_A, a_hi), desc_join(blo + k * KSTEP_B, b_hi), idesc, acc);
+                        acc = 1;
                     }
                     tc_commit(empty_bar(s));       // frees the stage when these MMAs have read it
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
                 if (ok) tc_commit(accf_bar(buf));  // accumulator complete
             }
@@ -330,48 +233,10 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                 tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BLOCK_N + c * 32), r);
                 tc_wait_ld();
                 const int col0 = nb * BLOCK_N + c * 32;
-                if (row_ok && col0 < p.N) {
-#pragma unroll
-                    for (int g8 = 0; g8 < 4; g8++) {
-                        const int col = col0 + g8 * 8;
-                        uint32_t h[8];
-#pragma unroll
-                        for (int e = 0; e < 8; e++) {
-                            float s = __uint_as_float(r[g8 * 8 + e]);
-                            if (p.relu) s = (s > 0.0f || s != s) ? s : 0.0f;
-                            h[e] = (uint32_t)__half_as_ushort(__float2half_rn(s));
-                        }
-                        if (col + 8 <= p.N) {
-                            if (mrow) {
-                                uint4 mk = *(const uint4 *)(mrow + col);
-                                uint32_t mw[4] = {mk.x, mk.y, mk.z, mk.w};
-#pragma unroll
-                                for (int e = 0; e < 8; e++) {
-                                    uint32_t mh = (e & 1) ? (mw[e >> 1] >> 16) : (mw[e >> 1] & 0xFFFFu);
-                                    // stored activation > 0  <=>  sign clear, non-zero, not NaN
-                                    bool keep = (mh & 0x8000u) == 0 && mh != 0 && mh <= 0x7C00u;
-                                    if (!keep) h[e] = 0;
-                                }
-                            }
-#pragma unroll
-                            for (int e = 0; e < 8; e++) bad |= half_bits_nonfinite(h[e]);
-                            uint4 o = make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), h[4] | (h[5] << 16),
-                                                 h[6] | (h[7] << 16));
-                            *(uint4 *)(crow + col) = o;
-                        } else {
-                            for (int e = 0; e < 8 && col + e < p.N; e++) {
-                                uint32_t v = h[e];
-                                if (mrow) {
-                                    uint32_t mh = mrow[col + e];
-                                    bool keep = (mh & 0x8000u) == 0 && mh != 0 && mh <= 0x7C00u;
-                                    if (!keep) v = 0;
-                                }
-                                bad |= half_bits_nonfinite(v);
-                                crow[col + e] = (uint16_t)v;
-                            }
-                        }
-                    }
-                }
+#ifdef MPT_TC_TRACE
+                if (p.dbg & 2) { if (r[0] == 0x12345678u && r[7] == 0x9abcdef0u) bad = true; continue; }
+#endif
+                if (row_ok && col0 < p.N) epilogue_store32(r, crow, mrow, col0, p.N, p.relu != 0, bad);
             }
             tc_fence_before();
             __syncwarp();
@@ -410,7 +275,7 @@ static EncodeTiledFn get_encode()
 
 // 2-D FP16 tensor map over a row-major matrix [rows, cols] with pitch ld (elements);
 // box = box_cols x box_rows, 128-byte swizzle, zero fill outside the matrix.
-static bool encode_map(CUtensorMap *map, const void *ptr, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_cols,
+bool tc_encode_map(CUtensorMap *map, const void *ptr, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_cols,
                        uint32_t box_rows)
 {
     EncodeTiledFn fn = get_encode();
@@ -458,11 +323,11 @@ cudaError_t launch_gemm_tc(int op, int M, int N, int K, const uint16_t *A, int l
     CUtensorMap ta, tb;
     bool ok;
     // A: stored [M,K] (K-major) for fwd/dgrad, stored [K,M] (MN-major) for wgrad
-    if (op == MPT_OP_WGRAD) ok = encode_map(&ta, A, (uint64_t)K, (uint64_t)M, (uint64_t)lda, 64, BLOCK_K);
-    else ok = encode_map(&ta, A, (uint64_t)M, (uint64_t)K, (uint64_t)lda, BLOCK_K, BLOCK_M);
+    if (op == MPT_OP_WGRAD) ok = tc_encode_map(&ta, A, (uint64_t)K, (uint64_t)M, (uint64_t)lda, 64, BLOCK_K);
+    else ok = tc_encode_map(&ta, A, (uint64_t)M, (uint64_t)K, (uint64_t)lda, BLOCK_K, BLOCK_M);
     // B: stored [N,K] (K-major) for fwd, stored [K,N] (MN-major) for dgrad/wgrad
-    if (op == MPT_OP_FWD) ok = ok && encode_map(&tb, B, (uint64_t)N, (uint64_t)K, (uint64_t)ldb, BLOCK_K, BLOCK_N);
-    else ok = ok && encode_map(&tb, B, (uint64_t)K, (uint64_t)N, (uint64_t)ldb, 64, BLOCK_K);
+    if (op == MPT_OP_FWD) ok = ok && tc_encode_map(&tb, B, (uint64_t)N, (uint64_t)K, (uint64_t)ldb, BLOCK_K, BLOCK_N);
+    else ok = ok && tc_encode_map(&tb, B, (uint64_t)K, (uint64_t)N, (uint64_t)ldb, 64, BLOCK_K);
     if (!ok) return cudaErrorInvalidValue;
 
     TcParams p;
@@ -472,9 +337,15 @@ cudaError_t launch_gemm_tc(int op, int M, int N, int K, const uint16_t *A, int l
     p.relu = relu ? 1 : 0;
     p.nonfinite_flag = nonfinite_flag;
     p.status = status;
+#ifdef MPT_TC_TRACE
+    { const char *e = getenv("MPT_DBG"); p.dbg = e ? atoi(e) : 0; }
+#endif
     p.tiles_m = (M + BLOCK_M - 1) / BLOCK_M;
     p.tiles_n = (N + BLOCK_N - 1) / BLOCK_N;
     p.group_m = 16;
+#ifdef MPT_TC_TRACE
+    { const char *e = getenv("MPT_GROUP_M"); if (e) p.group_m = atoi(e); }
+#endif
     int tiles = p.tiles_m * p.tiles_n;
     int grid = tiles < 148 ? tiles : 148;
     if (op == MPT_OP_FWD) return launch_variant<false, false>(ta, tb, p, grid, st);

@@ -1,0 +1,367 @@
+// Tensor-core FP16 GEMM for sm_100a with CTA pairs (paper section 3.3: FP16 operands,
+// FP32 accumulation, FP16 on the store; same fused epilogue as the single-CTA kernel).
+//
+// Two CTAs on neighbouring SMs form a cluster and compute one 256x256 output tile with
+// tcgen05.mma.cta_group::2 (M = 256, N = 256, K = 16 per instruction).  Each CTA loads its
+// own 128 rows of A and its own 128 columns of B (64 k per stage, 32 KB per stage and CTA),
+// the tensor core reads both CTAs' shared memory, and each CTA's tensor memory receives the
+// 128 x 256 accumulator block of its rows.  Compared with one CTA per 128x256 tile this
+// moves a third fewer operand bytes from L2 to the SMs and leaves room for a 7-stage ring.
+//
+// Roles in each CTA (192 threads): warp 0 TMA producer, warp 1 MMA issuer (only the
+// leader CTA, rank 0, issues; both CTAs' warp 1 take part in the paired tensor-memory
+// allocation), warps 2-5 epilogue.  Synchronisation:
+//   full[s]   in the leader: 1 arrival (leader's expect_tx for both CTAs' bytes) + the bytes
+//             of both CTAs' loads (the peer's loads signal the leader's barrier)
+//   empty[s]  in each CTA: tcgen05.commit multicast to both CTAs when the MMAs have read stage s
+//   accf[b]   in each CTA: tcgen05.commit multicast when a tile's accumulator is complete
+//   acce[b]   in the leader: 8 arrivals, one per epilogue warp of both CTAs
+// No TMA multicast is used.  Every mbarrier wait is bounded (see tc_ptx.cuh).
+#include <cuda.h>
+#include <cstdlib>
+
+#include "mpt_common.cuh"
+#include "tc_ptx.cuh"
+
+namespace mpt {
+
+namespace pair {
+
+#ifdef MPT_TC_TRACE
+#define TRACE(slot, t) do { if (blockIdx.x == 0 && p.status && (t) < 32) p.status[16 + 8 * (t) + (slot)] = (uint32_t)global_ns(); } while (0)
+#else
+#define TRACE(slot, t) do { } while (0)
+#endif
+
+static constexpr int CTA_M = 128;          // rows per CTA (256 per pair)
+static constexpr int TILE_N = 256;         // columns per pair tile
+static constexpr int CTA_N = 128;          // columns of B each CTA loads
+static constexpr int BLOCK_K = 64, UMMA_K = 16;
+static constexpr int STAGES = 7;
+static constexpr int A_STAGE_BYTES = CTA_M * BLOCK_K * 2;   // 16 KB
+static constexpr int B_STAGE_BYTES = CTA_N * BLOCK_K * 2;   // 16 KB
+static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+static constexpr int MN_BOX_BYTES = 64 * BLOCK_K * 2;
+static constexpr int TMEM_COLS = 512;
+static constexpr int NUM_THREADS = 192;
+static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256;
+
+__host__ __device__ constexpr uint32_t make_idesc(bool a_mn, bool b_mn)
+{
+    return (1u << 4) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) | ((uint32_t)(TILE_N >> 3) << 17) |
+           ((uint32_t)((2 * CTA_M) >> 4) << 24);
+}
+
+struct Params {
+    int M, N, K;
+    uint16_t *C;
+    int ldc;
+    const uint16_t *mask;
+    int ldmask;
+    int relu;
+    uint32_t *nonfinite_flag;
+    uint32_t *status;
+#ifdef MPT_TC_TRACE
+    int dbg;
+#endif
+    int tiles_m, tiles_n, group_m;   // pair tiles (256 rows x 256 columns)
+};
+
+__device__ __forceinline__ void tile_coords(const Params &p, int tile, int &mb, int &nb)
+{
+    int per_group = p.group_m * p.tiles_n;
+    int g = tile / per_group;
+    int first_m = g * p.group_m;
+    int gsz = min(p.group_m, p.tiles_m - first_m);
+    int r = tile - g * per_group;
+    mb = first_m + r % gsz;
+    nb = r / gsz;
+}
+
+__device__ __forceinline__ void report(const Params &p, volatile uint32_t *abort_flag, uint32_t code)
+{
+    *abort_flag = 1u;
+    if (p.status) atomicCAS(p.status, 0u, code | 0x80u | ((uint32_t)blockIdx.x << 8));
+}
+
+template <bool A_MN, bool B_MN>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const Params p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
+    const uint32_t bars = base + STAGES * STAGE_BYTES;
+    auto full_bar = [&](int s) { return bars + 8u * s; };
+    auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
+    auto accf_bar = [&](int b) { return bars + 8u * (2 * STAGES + b); };
+    auto acce_bar = [&](int b) { return bars + 8u * (2 * STAGES + 2 + b); };
+    volatile uint32_t *tmem_slot = (volatile uint32_t *)(base_ptr + STAGES * STAGE_BYTES + 8 * (2 * STAGES + 4));
+    volatile uint32_t *abort_flag = tmem_slot + 1;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) TRACE(6, 0);
+#ifdef MPT_TC_TRACE
+    if (threadIdx.x == 0 && blockIdx.x == 0 && p.status) p.status[16 + 8 * 2 + 6] = (uint32_t)clock64();
+#endif
+    const uint32_t rank = cluster_ctarank();       // 0 = leader of the pair
+    const bool leader = rank == 0;
+    const int pair_id = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+    const int num_tiles = p.tiles_m * p.tiles_n;
+    const int nkb = (p.K + BLOCK_K - 1) / BLOCK_K;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; s++) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int b = 0; b < 2; b++) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), 8); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {   // paired allocation: the same warp of both CTAs executes it
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void *)tmem_slot)),
+                     "r"((uint32_t)TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                            // the peer's barriers exist before anything signals them
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    if (threadIdx.x == 0) TRACE(7, 0);
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer (both CTAs)
+        if (lane == 0) {
+            uint32_t issued = 0, s = 0, ph = 0;
+            bool ok = true;
+            for (int tile = pair_id; tile < num_tiles && ok; tile += num_pairs) {
+                int mb, nb;
+                tile_coords(p, tile, mb, nb);
+                const int m0 = mb * (2 * CTA_M) + (int)rank * CTA_M;      // this CTA's rows of A
+                const int n0 = nb * TILE_N + (int)rank * CTA_N;           // this CTA's columns of B
+                for (int kb = 0; kb < nkb; kb++, issued++, s = (s + 1 == STAGES) ? 0 : s + 1, ph ^= (s == 0)) {
+                    if (!mbar_try_wait(empty_bar(s), ph ^ 1u) && !mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) {
+                        if (!*abort_flag) report(p, abort_flag, KERR_WAIT_EMPTY);
+                        ok = false;
+                        break;
+                    }
+                    const uint32_t sa = base + s * STAGE_BYTES, sb = sa + A_STAGE_BYTES;
+                    const uint32_t lead_full = mapa_u32(full_bar(s), 0);
+#ifdef MPT_TC_TRACE
+                    if ((p.dbg & 1) && issued >= (uint32_t)STAGES) { if (leader) mbar_arrive(full_bar(s)); continue; }
+#endif
+                    if (leader) mbar_arrive_expect_tx(full_bar(s), 2 * STAGE_BYTES);
+                    const int k0 = kb * BLOCK_K;
+                    if (A_MN) {
+#pragma unroll
+                        for (int j = 0; j < CTA_M / 64; j++) tma_load_2d_pair(sa + j * MN_BOX_BYTES, &tmA, m0 + 64 * j, k0, lead_full);
+                    } else {
+                        tma_load_2d_pair(sa, &tmA, k0, m0, lead_full);
+                    }
+                    if (B_MN) {
+#pragma unroll
+                        for (int j = 0; j < CTA_N / 64; j++) tma_load_2d_pair(sb + j * MN_BOX_BYTES, &tmB, n0 + 64 * j, k0, lead_full);
+                    } else {
+                        tma_load_2d_pair(sb, &tmB, k0, n0, lead_full);
+                    }
+                }
+            }
+            if (!ok && leader) {
+                // let the copies already in flight land before the CTA exits (bounded)
+                uint32_t first = issued > (uint32_t)STAGES ? issued - STAGES : 0;
+                for (uint32_t i = first; i < issued; i++) {
+                    unsigned long long t0 = global_ns();
+                    while (!mbar_try_wait(full_bar(i % STAGES), (i / STAGES) & 1u) && global_ns() - t0 < 1000000ull) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // -------------------------------------------------------------- MMA issuer (leader only)
+        if (leader && lane == 0) {
+            constexpr uint32_t idesc = make_idesc(A_MN, B_MN);
+            // descriptor halves: only the start address (low word) changes with stage and k
+            constexpr uint32_t KSTEP_A = (A_MN ? UMMA_K * 128 : UMMA_K * 2) >> 4;
+            constexpr uint32_t KSTEP_B = (B_MN ? UMMA_K * 128 : UMMA_K * 2) >> 4;
+            const uint32_t a_hi = desc_hi(1024), b_hi = desc_hi(1024);
+            const uint32_t a_lo0 = desc_lo(base, A_MN ? MN_BOX_BYTES : 16);
+            const uint32_t b_lo0 = desc_lo(base + A_STAGE_BYTES, B_MN ? MN_BOX_BYTES : 16);
+            uint32_t s = 0, ph = 0;
+            bool ok = true;
+            int t = 0;
+            for (int tile = pair_id; tile < num_tiles && ok; tile += num_pairs, t++) {
+                const int buf = t & 1;
+                const uint32_t acc_ph = (t >> 1) & 1u;
+                if (!mbar_try_wait(acce_bar(buf), acc_ph ^ 1u) && !mbar_wait(acce_bar(buf), acc_ph ^ 1u, abort_flag)) {
+                    if (!*abort_flag) report(p, abort_flag, KERR_WAIT_ACC_FREE);
+                    ok = false;
+                    break;
+                }
+                tc_fence_after();
+                TRACE(0, t);
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * TILE_N);
+                uint32_t acc = 0;                          // first MMA of a tile overwrites the accumulator
+                for (int kb = 0; kb < nkb; kb++) {
+                    if (!mbar_try_wait(full_bar(s), ph) && !mbar_wait(full_bar(s), ph, abort_flag)) {
+                        if (!*abort_flag) report(p, abort_flag, KERR_WAIT_FULL);
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    if (kb == 0) TRACE(1, t);
+                    const uint32_t alo = a_lo0 + s * (uint32_t)(STAGE_BYTES >> 4);
+                    const uint32_t blo = b_lo0 + s * (uint32_t)(STAGE_BYTES >> 4);
+#pragma unroll
+                    for (int k = 0; k < BLOCK_K / UMMA_K; k++) {
+#ifdef MPT_TC_TRACE
+                        if (p.dbg & 4) continue;
+#endif
+                        tc_mma_f16_pair(d_tmem, desc_join(alo + k * KSTEP_A, a_hi), desc_join(blo + k * KSTEP_B, b_hi), idesc, acc);
+                        acc = 1;
+                    }
+                    tc_commit_pair(empty_bar(s), 3);        // both CTAs' producers may refill stage s
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                }
+                if (ok) tc_commit_pair(accf_bar(buf), 3);   // both CTAs' epilogues may read the accumulator
+                TRACE(2, t);
+            }
+        }
+    } else {
+        // ---------------------------------------------------------------- epilogue (both CTAs)
+        const int q = warp & 3;
+        bool ok = true;
+        int t = 0;
+        for (int tile = pair_id; tile < num_tiles && ok; tile += num_pairs, t++) {
+            int mb, nb;
+            tile_coords(p, tile, mb, nb);
+            const int buf = t & 1;
+            const uint32_t acc_ph = (t >> 1) & 1u;
+            const bool got = mbar_wait(accf_bar(buf), acc_ph, abort_flag);
+            if (!__all_sync(0xFFFFFFFFu, got)) {
+                if (!*abort_flag && lane == 0) report(p, abort_flag, KERR_WAIT_ACC);
+                ok = false;
+                break;
+            }
+            tc_fence_after();
+            if (warp == 2 && lane == 0) TRACE(3, t);
+            const int row = mb * (2 * CTA_M) + (int)rank * CTA_M + q * 32 + lane;
+            const bool row_ok = row < p.M;
+            uint16_t *crow = p.C + (size_t)row * p.ldc;
+            const uint16_t *mrow = p.mask ? p.mask + (size_t)row * p.ldmask : nullptr;
+            bool bad = false;
+#pragma unroll 1
+            for (int c = 0; c < TILE_N / 32; c++) {
+                uint32_t r[32];
+                tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * TILE_N + c * 32), r);
+                tc_wait_ld();
+                const int col0 = nb * TILE_N + c * 32;
+#ifdef MPT_TC_TRACE
+                if (p.dbg & 2) { if (r[0] == 0x12345678u && r[7] == 0x9abcdef0u) bad = true; continue; }
+#endif
+                if (row_ok && col0 < p.N) epilogue_store32(r, crow, mrow, col0, p.N, p.relu != 0, bad);
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (warp == 2 && lane == 0) TRACE(4, t);
+            if (lane == 0) mbar_arrive_cluster(mapa_u32(acce_bar(buf), 0));
+            if (warp == 2 && lane == 0) TRACE(5, t);
+            if (p.nonfinite_flag && __any_sync(0xFFFFFFFFu, bad) && lane == 0) atomicOr(p.nonfinite_flag, 1u);
+        }
+    }
+
+    // common exit: all waits above are bounded, so both CTAs of the pair arrive here; neither
+    // may leave while the other can still touch its shared or tensor memory
+    tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x == 0) TRACE(6, 1);
+    cluster_sync_all();
+    if (threadIdx.x == 0) TRACE(7, 1);
+#ifdef MPT_TC_TRACE
+    if (threadIdx.x == 0 && blockIdx.x == 0 && p.status) p.status[16 + 8 * 2 + 7] = (uint32_t)clock64();
+#endif
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS) : "memory");
+    }
+}
+
+template <bool A_MN, bool B_MN>
+static cudaError_t launch_variant(const CUtensorMap &ta, const CUtensorMap &tb, const Params &p, int pairs_wanted,
+                                  cudaStream_t st)
+{
+    static bool configured = false;
+    static int max_pairs = 0;
+    auto kern = k_gemm_tc2<A_MN, B_MN>;
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        cfg.gridDim = dim3(148, 1, 1);
+        int n = 0;
+        e = cudaOccupancyMaxActiveClusters(&n, kern, &cfg);
+        if (e != cudaSuccess) return e;
+        if (n < 1) return cudaErrorLaunchOutOfResources;
+        max_pairs = n < 74 ? n : 74;
+        configured = true;
+    }
+    int pairs = pairs_wanted < max_pairs ? pairs_wanted : max_pairs;
+    cfg.gridDim = dim3(2 * pairs, 1, 1);
+    return cudaLaunchKernelEx(&cfg, kern, ta, tb, p);
+}
+
+}  // namespace pair
+
+bool tc2_gemm_preferred(int M, int N, int K)
+{
+    // pairs pay off once there are enough 256x256 tiles to fill the 74 clusters about twice;
+    // small or thin problems have more parallelism as 128x256 tiles on the 1-CTA kernel
+    (void)K;
+    const long tiles = (long)((M + 255) / 256) * ((N + 255) / 256);
+    return M >= 256 && N >= 256 && tiles >= 128;
+}
+
+cudaError_t launch_gemm_tc2(int op, int M, int N, int K, const uint16_t *A, int lda, const uint16_t *B, int ldb,
+                            uint16_t *C, int ldc, bool relu, const uint16_t *mask, int ldmask, uint32_t *nonfinite_flag,
+                            uint32_t *status, cudaStream_t st)
+{
+    using namespace pair;
+    CUtensorMap ta, tb;
+    bool ok;
+    if (op == MPT_OP_WGRAD) ok = tc_encode_map(&ta, A, (uint64_t)K, (uint64_t)M, (uint64_t)lda, 64, BLOCK_K);
+    else ok = tc_encode_map(&ta, A, (uint64_t)M, (uint64_t)K, (uint64_t)lda, BLOCK_K, CTA_M);
+    if (op == MPT_OP_FWD) ok = ok && tc_encode_map(&tb, B, (uint64_t)N, (uint64_t)K, (uint64_t)ldb, BLOCK_K, CTA_N);
+    else ok = ok && tc_encode_map(&tb, B, (uint64_t)K, (uint64_t)N, (uint64_t)ldb, 64, BLOCK_K);
+    if (!ok) return cudaErrorInvalidValue;
+    Params p;
+    p.M = M; p.N = N; p.K = K;
+    p.C = C; p.ldc = ldc;
+    p.mask = mask; p.ldmask = ldmask;
+    p.relu = relu ? 1 : 0;
+    p.nonfinite_flag = nonfinite_flag;
+    p.status = status;
+#ifdef MPT_TC_TRACE
+    { const char *e = getenv("MPT_DBG"); p.dbg = e ? atoi(e) : 0; }
+#endif
+    p.tiles_m = (M + 2 * CTA_M - 1) / (2 * CTA_M);
+    p.tiles_n = (N + TILE_N - 1) / TILE_N;
+    p.group_m = 8;
+#ifdef MPT_TC_TRACE
+    { const char *e = getenv("MPT_GROUP_M"); if (e) p.group_m = atoi(e); }
+#endif
+    int tiles = p.tiles_m * p.tiles_n;
+    if (op == MPT_OP_FWD) return launch_variant<false, false>(ta, tb, p, tiles, st);
+    if (op == MPT_OP_DGRAD) return launch_variant<false, true>(ta, tb, p, tiles, st);
+    return launch_variant<true, true>(ta, tb, p, tiles, st);
+}
+
+}  // namespace mpt

@@ -99,7 +99,7 @@ struct mpt_ctx {
     int batch = 0;
     bool forward_done = false, have_grads = false, poisoned = false;
     long long launches = 0;
-    bool disable_tc = false;
+    bool disable_tc = false, disable_pair = false;
     std::string err;
     // optional per-kernel timing with CUDA events (mpt_profile)
     bool profiling = false;
@@ -173,10 +173,14 @@ int gemm(mpt_ctx *c, int op, int M, int N, int K, const uint16_t *A, int lda, co
 {
     cudaError_t e;
     ProfSpan span(c, MPT_PROF_GEMM, 2.0 * M * N * K);
-    if (!c->disable_tc && tc_gemm_supported(op, M, N, K, A, lda, B, ldb, C, ldc, mask, ldmask))
-        e = launch_gemm_tc(op, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite,
-                           c->status + ST_KERNEL_ERR, c->stream);
-    else
+    if (!c->disable_tc && tc_gemm_supported(op, M, N, K, A, lda, B, ldb, C, ldc, mask, ldmask)) {
+        if (!c->disable_pair && tc2_gemm_preferred(M, N, K))
+            e = launch_gemm_tc2(op, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite,
+                                c->status + ST_KERNEL_ERR, c->stream);
+        else
+            e = launch_gemm_tc(op, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite,
+                               c->status + ST_KERNEL_ERR, c->stream);
+    } else
         e = launch_gemm_simt(op, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite, c->stream);
     c->launches++;
     if (e != cudaSuccess) return cuda_fail(c, e, "gemm launch");
@@ -331,6 +335,8 @@ int mpt_create(const mpt_layer_desc *layers, int n_layers, float S, float lr, fl
     }
     const char *env = getenv("MPT_DISABLE_TC");
     c->disable_tc = env && env[0] == '1';
+    env = getenv("MPT_DISABLE_PAIR");
+    c->disable_pair = env && env[0] == '1';
     // Parameter arenas (including the padding between layers), activations and status start at zero.
     cudaError_t e = cudaMemsetAsync(c->ws, 0, pl.total, c->stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
@@ -577,11 +583,15 @@ int mpt_gemm_f16(int op, int M, int N, int K, const uint16_t *A, int lda, const 
     cudaStream_t st = (cudaStream_t)cuda_stream;
     const bool relu = (flags & MPT_GEMM_RELU) != 0;
     bool tc_ok = K > 0 && tc_gemm_supported(op, M, N, K, A, lda, B, ldb, C, ldc, mask, ldmask);
-    if ((flags & MPT_GEMM_FORCE_TC) && !tc_ok) return MPT_ERR_SHAPE;
+    if ((flags & (MPT_GEMM_FORCE_TC | MPT_GEMM_FORCE_PAIR)) && !tc_ok) return MPT_ERR_SHAPE;
     cudaError_t e;
-    if (tc_ok && !(flags & MPT_GEMM_FORCE_SIMT))
-        e = launch_gemm_tc(op, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite_flag, status_dev, st);
-    else
+    if (tc_ok && !(flags & MPT_GEMM_FORCE_SIMT)) {
+        const bool pair = (flags & MPT_GEMM_FORCE_PAIR) || (!(flags & MPT_GEMM_FORCE_TC) && tc2_gemm_preferred(M, N, K));
+        if (pair)
+            e = launch_gemm_tc2(op, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite_flag, status_dev, st);
+        else
+            e = launch_gemm_tc(op, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite_flag, status_dev, st);
+    } else
         e = launch_gemm_simt(op, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite_flag, st);
     return e == cudaSuccess ? MPT_OK : MPT_ERR_CUDA;
 }

@@ -57,4 +57,10 @@ cudaError_t launch_gemm_tc(int op, int M, int N, int K, const uint16_t *A, int l
                            int ldb, uint16_t *C, int ldc, bool relu, const uint16_t *mask, int ldmask,
                            uint32_t *nonfinite_flag, uint32_t *status, cudaStream_t st);
 
+// CTA-pair variant (tcgen05 cta_group::2, 256x256 tiles); same operand rules as launch_gemm_tc.
+bool tc2_gemm_preferred(int M, int N, int K);
+cudaError_t launch_gemm_tc2(int op, int M, int N, int K, const uint16_t *A, int lda, const uint16_t *B, int ldb,
+                            uint16_t *C, int ldc, bool relu, const uint16_t *mask, int ldmask,
+                            uint32_t *nonfinite_flag, uint32_t *status, cudaStream_t st);
+
 }  // namespace mpt

@@ -107,6 +107,8 @@ def main():
     g.add_argument("--op", nargs="*", type=int, default=[0, 1, 2])
     g.add_argument("--iters", type=int, default=20)
     g.add_argument("--compare-library", action="store_true")
+    g.add_argument("--kernel", default="auto", choices=["auto", "tc", "pair"],
+                   help="auto: the library's choice; tc: single-CTA 128x256 tiles; pair: cta_group::2 256x256 tiles")
     u = sub.add_parser("update")
     u.add_argument("--params", type=int, default=150994944)
     u.add_argument("--momentum", type=int, default=1)
@@ -121,7 +123,10 @@ def main():
                   else inputs.GEMM_SWEEP + [inputs.LSTM_GATE, inputs.LSTM_PROJ])
         for (M, N, K) in shapes:
             for op in args.op:
-                print(json.dumps(bench_gemm(M, N, K, op, args.iters, args.compare_library)), flush=True)
+                flags = {"auto": 0, "tc": mpt.GEMM_FORCE_TC, "pair": mpt.GEMM_FORCE_PAIR}[args.kernel]
+                res = bench_gemm(M, N, K, op, args.iters, args.compare_library, flags)
+                res["kernel_choice"] = args.kernel
+                print(json.dumps(res), flush=True)
     elif args.cmd == "update":
         print(json.dumps(bench_update(args.params, args.momentum, args.iters)), flush=True)
     else:

@@ -80,12 +80,13 @@ def test_simt_gemm_relu_mask_flag():
     assert flag == 1 and (~np.isfinite(ref.view(np.float16).astype(np.float32))).any()
 
 
-def _check_tc(op, M, N, K, flags=0, mask=None, seed=21, scale=None, want_flag=False):
+def _check_tc(op, M, N, K, flags=0, mask=None, seed=21, scale=None, want_flag=False, kernel="tc"):
     from paper_1710_03740_b200 import binding as b
+    force = b.GEMM_FORCE_PAIR if kernel == "pair" else b.GEMM_FORCE_TC
     sa = sb = scale
     A, B = inputs.gemm_operands(op, M, N, K, seed=seed, scale_a=sa, scale_b=sb)
     ref, ex, ab = mpo.gemm_f16(op, A, B, relu=bool(flags & b.GEMM_RELU), mask=mask, want_exact=True)
-    got, flag = run_gemm(op, A, B, M, N, K, flags=flags | b.GEMM_FORCE_TC, mask=mask,
+    got, flag = run_gemm(op, A, B, M, N, K, flags=flags | force, mask=mask,
                          pad=(8 if (M * N) % 3 == 0 else 0), want_flag=want_flag)
     ok, stats = gemm_accept(got, ref, K=K, absdot=ab)
     assert ok.all(), (op, M, N, K, stats, np.argwhere(~ok)[:8].tolist())
@@ -102,6 +103,10 @@ TC_SHAPES = [(128, 256, 64), (128, 256, 256), (256, 512, 128), (128, 256, 72), (
              (64, 16, 512), (8, 8, 8), (384, 768, 1024), (1024, 1024, 1024)]
 
 
+PAIR_SHAPES = [(256, 256, 64), (256, 256, 448), (512, 768, 128), (256, 512, 72), (392, 560, 136),
+                (64, 16, 512), (8, 8, 8), (1280, 1024, 1024)]
+
+
 @pytest.mark.parametrize("op", [0, 1, 2])
 @pytest.mark.parametrize("M,N,K", TC_SHAPES)
 def test_tc_gemm_parity(op, M, N, K):
@@ -109,29 +114,44 @@ def test_tc_gemm_parity(op, M, N, K):
 
 
 @pytest.mark.parametrize("op", [0, 1, 2])
-def test_tc_gemm_run_to_run_identical(op):
+@pytest.mark.parametrize("M,N,K", PAIR_SHAPES)
+def test_pair_gemm_parity(op, M, N, K):
+    _check_tc(op, M, N, K, kernel="pair")
+
+
+@pytest.mark.parametrize("kernel", ["tc", "pair"])
+@pytest.mark.parametrize("op", [0, 1, 2])
+def test_tc_gemm_run_to_run_identical(op, kernel):
     M, N, K = 304, 520, 392
-    a, _, _, _ = _check_tc(op, M, N, K)
-    b2, _, _, _ = _check_tc(op, M, N, K)
+    a, _, _, _ = _check_tc(op, M, N, K, kernel=kernel)
+    b2, _, _, _ = _check_tc(op, M, N, K, kernel=kernel)
     assert np.array_equal(a, b2)
 
 
-def test_tc_gemm_relu_mask_flag_subnormals():
+def test_pair_kernel_runs_many_tiles_per_cluster():
+    """More 256x256 tiles than clusters: the ring, the two accumulator buffers and the
+    barrier phases all wrap several times."""
+    _check_tc(0, 2048, 4096 + 256, 192, kernel="pair")
+    _check_tc(2, 2304, 3072, 136, kernel="pair")
+
+
+@pytest.mark.parametrize("kernel", ["tc", "pair"])
+def test_tc_gemm_relu_mask_flag_subnormals(kernel):
     from paper_1710_03740_b200 import binding as b
     M, N, K = 256, 512, 320
-    _check_tc(0, M, N, K, flags=b.GEMM_RELU)
+    _check_tc(0, M, N, K, flags=b.GEMM_RELU, kernel=kernel)
     rng = np.random.default_rng(4)
     mask = rng.standard_normal((M, N)).astype(np.float16)
     mask[0, :4] = [0.0, -0.0, np.nan, np.inf]
-    _check_tc(1, M, N, K, mask=mask)
+    _check_tc(1, M, N, K, mask=mask, kernel=kernel)
     # subnormal operands and outputs (config 2: head weights scaled by 2^-16)
-    got, ref, _, stats = _check_tc(0, M, N, K, scale=2.0 ** -9)
+    got, ref, _, stats = _check_tc(0, M, N, K, scale=2.0 ** -9, kernel=kernel)
     sub = (ref & 0x7C00) == 0
     assert sub.mean() > 0.5 and (ref[sub] != 0).any()
     # overflow on the store raises the flag (section 3.2)
-    got, ref, flag, _ = _check_tc(2, M, N, K, scale=60.0, want_flag=True)
+    got, ref, flag, _ = _check_tc(2, M, N, K, scale=60.0, want_flag=True, kernel=kernel)
     assert flag == 1 and ((ref & 0x7FFF) == 0x7C00).any()
-    got, ref, flag, _ = _check_tc(2, M, N, K, want_flag=True)
+    got, ref, flag, _ = _check_tc(2, M, N, K, want_flag=True, kernel=kernel)
     assert flag == 0
 
 
