@@ -1,10 +1,13 @@
 // Master-weight pass (paper sections 3.1, 3.2): recast, overflow inspection, and the
 // fused unscale / inspect / FP32 SGD(+momentum) / FP16 re-round kernel.
 //
-// All three are streaming kernels bound by HBM bandwidth: 128-bit accesses, a grid
-// of 148 SMs x 8 resident CTAs of 256 threads, two independent 8-element vectors in
-// flight per thread.  The update reads g16, w32, (v) once and writes w32, (v), w16
-// once: 12 bytes/parameter (plain SGD) or 20 bytes/parameter (momentum).
+// All three are streaming kernels bound by HBM bandwidth: 128-bit accesses with streaming
+// cache hints, one CTA of 256 threads per 1024 consecutive 8-element vectors (four
+// independent vectors in flight per thread, all loads issued before the first use) and no
+// grid-stride loop: on B200 a grid of short-lived CTAs handed out in address order by the
+// hardware scheduler sustains about 20 % more bandwidth than a persistent grid-stride grid.
+// The update reads g16, w32, (v) once and writes w32, (v), w16 once: 12 bytes/parameter
+// (plain SGD) or 20 bytes/parameter (momentum).
 //
 // Bit-exactness contract: every FP32 operation is rounded separately (the __f*_rn
 // intrinsics are never contracted into a fused multiply-add), no flush-to-zero.
@@ -15,6 +18,7 @@ namespace mpt {
 static constexpr int kThreads = 256;
 static constexpr int kSMs = 148;
 static constexpr int kCtasPerSM = 8;
+static constexpr int kVecPerThread = 4;   // 8-element vectors per thread in the one-shot kernels
 
 __device__ __forceinline__ float h2f_bits(uint32_t h) { return __half2float(__ushort_as_half((unsigned short)h)); }
 __device__ __forceinline__ uint32_t f2h_bits(float x) { return (uint32_t)__half_as_ushort(__float2half_rn(x)); }
@@ -28,20 +32,36 @@ static inline int grid_for(size_t work_items)
     return (int)blocks;
 }
 
+// one CTA per kThreads * kVecPerThread vectors
+static inline unsigned vec_grid(size_t n8)
+{
+    const size_t per_cta = (size_t)kThreads * kVecPerThread;
+    return (unsigned)((n8 + per_cta - 1) / per_cta);
+}
+
 // ------------------------------------------------------------------ recast
 
 __global__ void __launch_bounds__(kThreads) k_recast_vec(const float4 *__restrict__ w32, uint4 *__restrict__ w16,
                                                          size_t n8)
 {
-    size_t stride = (size_t)gridDim.x * blockDim.x;
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n8; i += stride) {
-        float4 a = __ldcs(w32 + 2 * i), b = __ldcs(w32 + 2 * i + 1);
-        uint4 o;
-        o.x = f2h_bits(a.x) | (f2h_bits(a.y) << 16);
-        o.y = f2h_bits(a.z) | (f2h_bits(a.w) << 16);
-        o.z = f2h_bits(b.x) | (f2h_bits(b.y) << 16);
-        o.w = f2h_bits(b.z) | (f2h_bits(b.w) << 16);
-        w16[i] = o;
+    const size_t base = (size_t)blockIdx.x * (kThreads * kVecPerThread) + threadIdx.x;
+    float4 a[kVecPerThread], b[kVecPerThread];
+#pragma unroll
+    for (int u = 0; u < kVecPerThread; u++) {
+        const size_t j = base + (size_t)u * kThreads;
+        if (j < n8) { a[u] = __ldcs(w32 + 2 * j); b[u] = __ldcs(w32 + 2 * j + 1); }
+    }
+#pragma unroll
+    for (int u = 0; u < kVecPerThread; u++) {
+        const size_t j = base + (size_t)u * kThreads;
+        if (j < n8) {
+            uint4 o;
+            o.x = f2h_bits(a[u].x) | (f2h_bits(a[u].y) << 16);
+            o.y = f2h_bits(a[u].z) | (f2h_bits(a[u].w) << 16);
+            o.z = f2h_bits(b[u].x) | (f2h_bits(b[u].y) << 16);
+            o.w = f2h_bits(b[u].z) | (f2h_bits(b[u].w) << 16);
+            w16[j] = o;
+        }
     }
 }
 
@@ -57,7 +77,7 @@ cudaError_t launch_recast(const float *w32, uint16_t *w16, size_t n, cudaStream_
     if (n == 0) return cudaSuccess;
     bool aligned = (((uintptr_t)w32 | (uintptr_t)w16) & 15) == 0;
     size_t n8 = aligned ? n / 8 : 0;
-    if (n8) k_recast_vec<<<grid_for(n8), kThreads, 0, st>>>((const float4 *)w32, (uint4 *)w16, n8);
+    if (n8) k_recast_vec<<<vec_grid(n8), kThreads, 0, st>>>((const float4 *)w32, (uint4 *)w16, n8);
     if (n8 * 8 < n) k_recast_scalar<<<grid_for(n - n8 * 8), kThreads, 0, st>>>(w32, w16, n8 * 8, n);
     return cudaGetLastError();
 }
@@ -73,13 +93,18 @@ __device__ __forceinline__ bool pair_nonfinite(uint32_t two_halfs, float inv)
 __global__ void __launch_bounds__(kThreads) k_nonfinite_vec(const uint4 *__restrict__ g, size_t n8, float inv,
                                                             uint32_t *flag)
 {
-    size_t stride = (size_t)gridDim.x * blockDim.x;
-    bool bad = false;
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n8; i += stride) {
-        uint4 x = __ldcs(g + i);
-        bad |= pair_nonfinite(x.x, inv) | pair_nonfinite(x.y, inv) | pair_nonfinite(x.z, inv) |
-               pair_nonfinite(x.w, inv);
+    const size_t base = (size_t)blockIdx.x * (kThreads * kVecPerThread) + threadIdx.x;
+    uint4 x[kVecPerThread];
+#pragma unroll
+    for (int u = 0; u < kVecPerThread; u++) {
+        const size_t j = base + (size_t)u * kThreads;
+        x[u] = (j < n8) ? __ldcs(g + j) : make_uint4(0, 0, 0, 0);
     }
+    bool bad = false;
+#pragma unroll
+    for (int u = 0; u < kVecPerThread; u++)
+        bad |= pair_nonfinite(x[u].x, inv) | pair_nonfinite(x[u].y, inv) | pair_nonfinite(x[u].z, inv) |
+               pair_nonfinite(x[u].w, inv);
     // warp vote, then at most one atomic per warp and only when something was found
     if (__any_sync(0xFFFFFFFFu, bad) && (threadIdx.x & 31) == 0) atomicOr(flag, 1u);
 }
@@ -98,7 +123,7 @@ cudaError_t launch_grad_nonfinite(const uint16_t *g16, size_t n, float inv_S, ui
     if (n == 0) return cudaSuccess;
     bool aligned = ((uintptr_t)g16 & 15) == 0;
     size_t n8 = aligned ? n / 8 : 0;
-    if (n8) k_nonfinite_vec<<<grid_for(n8), kThreads, 0, st>>>((const uint4 *)g16, n8, inv_S, flag);
+    if (n8) k_nonfinite_vec<<<vec_grid(n8), kThreads, 0, st>>>((const uint4 *)g16, n8, inv_S, flag);
     if (n8 * 8 < n) k_nonfinite_scalar<<<grid_for(n - n8 * 8), kThreads, 0, st>>>(g16, n8 * 8, n, inv_S, flag);
     return cudaGetLastError();
 }
@@ -149,42 +174,30 @@ __global__ void __launch_bounds__(kThreads) k_update_vec(const uint4 *__restrict
                                                          float inv, float lr, float mu, uint32_t *flags)
 {
     if (*(volatile const uint32_t *)flags != 0u) return;
-    const size_t stride = (size_t)gridDim.x * blockDim.x;
-    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const size_t base = (size_t)blockIdx.x * (kThreads * kVecPerThread) + threadIdx.x;
     bool bad = false;
-    // two vectors per trip: all loads of both are issued before the first use
-    for (; i + stride < n8; i += 2 * stride) {
-        const size_t j = i + stride;
-        uint4 ga = __ldcs(g16 + i), gb = __ldcs(g16 + j);
-        float4 wa0 = __ldcs(w32 + 2 * i), wa1 = __ldcs(w32 + 2 * i + 1);
-        float4 wb0 = __ldcs(w32 + 2 * j), wb1 = __ldcs(w32 + 2 * j + 1);
-        float4 va0 = {}, va1 = {}, vb0 = {}, vb1 = {};
-        if (MOM) {
-            va0 = __ldcs(v32 + 2 * i); va1 = __ldcs(v32 + 2 * i + 1);
-            vb0 = __ldcs(v32 + 2 * j); vb1 = __ldcs(v32 + 2 * j + 1);
+    uint4 g[kVecPerThread];
+    float4 w0[kVecPerThread], w1[kVecPerThread], v0[kVecPerThread], v1[kVecPerThread];
+#pragma unroll
+    for (int u = 0; u < kVecPerThread; u++) {      // every load of this thread is in flight before the first use
+        const size_t j = base + (size_t)u * kThreads;
+        if (j < n8) {
+            g[u] = __ldcs(g16 + j);
+            w0[u] = __ldcs(w32 + 2 * j); w1[u] = __ldcs(w32 + 2 * j + 1);
+            if (MOM) { v0[u] = __ldcs(v32 + 2 * j); v1[u] = __ldcs(v32 + 2 * j + 1); }
         }
-        uint4 ha, hb;
-        upd8<MOM>(ga, wa0, wa1, va0, va1, ha, inv, lr, mu, bad);
-        upd8<MOM>(gb, wb0, wb1, vb0, vb1, hb, inv, lr, mu, bad);
-        __stcs(w32 + 2 * i, wa0); __stcs(w32 + 2 * i + 1, wa1);
-        __stcs(w32 + 2 * j, wb0); __stcs(w32 + 2 * j + 1, wb1);
-        if (MOM) {
-            __stcs(v32 + 2 * i, va0); __stcs(v32 + 2 * i + 1, va1);
-            __stcs(v32 + 2 * j, vb0); __stcs(v32 + 2 * j + 1, vb1);
-        }
-        w16[i] = ha;
-        w16[j] = hb;
     }
-    if (i < n8) {
-        uint4 ga = __ldcs(g16 + i);
-        float4 wa0 = __ldcs(w32 + 2 * i), wa1 = __ldcs(w32 + 2 * i + 1);
-        float4 va0 = {}, va1 = {};
-        if (MOM) { va0 = __ldcs(v32 + 2 * i); va1 = __ldcs(v32 + 2 * i + 1); }
-        uint4 ha;
-        upd8<MOM>(ga, wa0, wa1, va0, va1, ha, inv, lr, mu, bad);
-        __stcs(w32 + 2 * i, wa0); __stcs(w32 + 2 * i + 1, wa1);
-        if (MOM) { __stcs(v32 + 2 * i, va0); __stcs(v32 + 2 * i + 1, va1); }
-        w16[i] = ha;
+#pragma unroll
+    for (int u = 0; u < kVecPerThread; u++) {
+        const size_t j = base + (size_t)u * kThreads;
+        if (j < n8) {
+            uint4 h;
+            if (!MOM) { v0[u] = make_float4(0, 0, 0, 0); v1[u] = v0[u]; }
+            upd8<MOM>(g[u], w0[u], w1[u], v0[u], v1[u], h, inv, lr, mu, bad);
+            __stcs(w32 + 2 * j, w0[u]); __stcs(w32 + 2 * j + 1, w1[u]);
+            if (MOM) { __stcs(v32 + 2 * j, v0[u]); __stcs(v32 + 2 * j + 1, v1[u]); }
+            __stcs(w16 + j, h);
+        }
     }
     if (__any_sync(0xFFFFFFFFu, bad) && (threadIdx.x & 31) == 0) atomicOr(flags + 1, 1u);
 }
@@ -214,8 +227,8 @@ cudaError_t launch_update(const uint16_t *g16, float *w32, float *v, uint16_t *w
     uintptr_t bits = (uintptr_t)g16 | (uintptr_t)w32 | (uintptr_t)w16 | (use_momentum ? (uintptr_t)v : 0);
     size_t n8 = (bits & 15) == 0 ? n / 8 : 0;
     if (n8) {
-        // each thread owns two vectors per trip
-        int grid = grid_for((n8 + 1) / 2);
+        const size_t per_cta = (size_t)kThreads * kVecPerThread;
+        const unsigned grid = (unsigned)((n8 + per_cta - 1) / per_cta);
         if (use_momentum)
             k_update_vec<true><<<grid, kThreads, 0, st>>>((const uint4 *)g16, (float4 *)w32, (float4 *)v, (uint4 *)w16,
                                                           n8, inv_S, lr, mu, flags);
