@@ -26,19 +26,26 @@
 
 namespace mpt {
 
-static constexpr int BLOCK_M = 128, BLOCK_N = 256, BLOCK_K = 64, UMMA_K = 16, STAGES = 4;
+static constexpr int BLOCK_M = 128, BLOCK_K = 64, UMMA_K = 16;
 static constexpr int A_STAGE_BYTES = BLOCK_M * BLOCK_K * 2;  // 16 KB
-static constexpr int B_STAGE_BYTES = BLOCK_N * BLOCK_K * 2;  // 32 KB
-static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
 static constexpr int MN_BOX_BYTES = 64 * BLOCK_K * 2;        // one 64(mn) x 64(k) box of an MN-major operand
-static constexpr int TMEM_COLS = 512;
 static constexpr int NUM_THREADS = 192;
-static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+
+// Tile width BN is 256 (four 48 KB stages) or, for outputs with too few 128x256 tiles to fill
+// the SMs, 128 (six 32 KB stages).  The two accumulator buffers take 2 * BN tensor-memory columns.
+template <int BN>
+struct TileCfg {
+    static constexpr int B_STAGE_BYTES = BN * BLOCK_K * 2;
+    static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+    static constexpr int STAGES = BN == 256 ? 4 : 6;
+    static constexpr int TMEM_COLS = 2 * BN;
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+};
 
 // Instruction descriptor, kind::f16: D = F32, A = B = F16, majors, N >> 3, M >> 4.
-__host__ __device__ constexpr uint32_t make_idesc(bool a_mn, bool b_mn)
+__host__ __device__ constexpr uint32_t make_idesc(bool a_mn, bool b_mn, int bn)
 {
-    return (1u << 4) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) | ((uint32_t)(BLOCK_N >> 3) << 17) |
+    return (1u << 4) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) | ((uint32_t)(bn >> 3) << 17) |
            ((uint32_t)(BLOCK_M >> 4) << 24);
 }
 
@@ -76,10 +83,13 @@ __device__ __forceinline__ void report(const TcParams &p, volatile uint32_t *abo
     if (p.status) atomicCAS(p.status, 0u, code | ((uint32_t)blockIdx.x << 8));
 }
 
-template <bool A_MN, bool B_MN>
+template <bool A_MN, bool B_MN, int BLOCK_N>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcParams p)
 {
+    constexpr int STAGES = TileCfg<BLOCK_N>::STAGES;
+    constexpr int STAGE_BYTES = TileCfg<BLOCK_N>::STAGE_BYTES;
+    constexpr int TMEM_COLS = TileCfg<BLOCK_N>::TMEM_COLS;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;   // swizzled tiles need 1024-byte alignment
     uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
@@ -161,7 +171,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     } else if (warp == 1) {
         // -------------------------------------------------------------- MMA issuer
         if (lane == 0) {
-            constexpr uint32_t idesc = make_idesc(A_MN, B_MN);
+            constexpr uint32_t idesc = make_idesc(A_MN, B_MN, BLOCK_N);
             // descriptor halves: only the start address (low word) changes with stage and k.
             // K-major: 16 k = 32 bytes along the swizzled row; MN-major: 16 k-rows of 128 bytes.
             constexpr uint32_t KSTEP_A = (A_MN ? UMMA_K * 128 : UMMA_K * 2) >> 4;
@@ -301,12 +311,13 @@ bool tc_gemm_supported(int op, int M, int N, int K, const void *A, int lda, cons
     return true;
 }
 
-template <bool A_MN, bool B_MN>
+template <bool A_MN, bool B_MN, int BN>
 static cudaError_t launch_variant(const CUtensorMap &ta, const CUtensorMap &tb, const TcParams &p, int grid,
                                   cudaStream_t st)
 {
     static bool configured = false;
-    auto kern = k_gemm_tc<A_MN, B_MN>;
+    constexpr int SMEM_BYTES = TileCfg<BN>::SMEM_BYTES;
+    auto kern = k_gemm_tc<A_MN, B_MN, BN>;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
         if (e != cudaSuccess) return e;
@@ -316,9 +327,9 @@ static cudaError_t launch_variant(const CUtensorMap &ta, const CUtensorMap &tb, 
     return cudaGetLastError();
 }
 
-cudaError_t launch_gemm_tc(int op, int M, int N, int K, const uint16_t *A, int lda, const uint16_t *B, int ldb,
-                           uint16_t *C, int ldc, bool relu, const uint16_t *mask, int ldmask, uint32_t *nonfinite_flag,
-                           uint32_t *status, cudaStream_t st)
+template <int BN>
+static cudaError_t launch_bn(int op, int M, int N, int K, const uint16_t *A, int lda, const uint16_t *B, int ldb,
+                             TcParams p, cudaStream_t st)
 {
     CUtensorMap ta, tb;
     bool ok;
@@ -326,10 +337,26 @@ cudaError_t launch_gemm_tc(int op, int M, int N, int K, const uint16_t *A, int l
     if (op == MPT_OP_WGRAD) ok = tc_encode_map(&ta, A, (uint64_t)K, (uint64_t)M, (uint64_t)lda, 64, BLOCK_K);
     else ok = tc_encode_map(&ta, A, (uint64_t)M, (uint64_t)K, (uint64_t)lda, BLOCK_K, BLOCK_M);
     // B: stored [N,K] (K-major) for fwd, stored [K,N] (MN-major) for dgrad/wgrad
-    if (op == MPT_OP_FWD) ok = ok && tc_encode_map(&tb, B, (uint64_t)N, (uint64_t)K, (uint64_t)ldb, BLOCK_K, BLOCK_N);
+    if (op == MPT_OP_FWD) ok = ok && tc_encode_map(&tb, B, (uint64_t)N, (uint64_t)K, (uint64_t)ldb, BLOCK_K, BN);
     else ok = ok && tc_encode_map(&tb, B, (uint64_t)K, (uint64_t)N, (uint64_t)ldb, 64, BLOCK_K);
     if (!ok) return cudaErrorInvalidValue;
+    p.tiles_m = (M + BLOCK_M - 1) / BLOCK_M;
+    p.tiles_n = (N + BN - 1) / BN;
+    p.group_m = 16;
+#ifdef MPT_TC_TRACE
+    { const char *e = getenv("MPT_GROUP_M"); if (e) p.group_m = atoi(e); }
+#endif
+    int tiles = p.tiles_m * p.tiles_n;
+    int grid = tiles < 148 ? tiles : 148;
+    if (op == MPT_OP_FWD) return launch_variant<false, false, BN>(ta, tb, p, grid, st);
+    if (op == MPT_OP_DGRAD) return launch_variant<false, true, BN>(ta, tb, p, grid, st);
+    return launch_variant<true, true, BN>(ta, tb, p, grid, st);
+}
 
+cudaError_t launch_gemm_tc(int op, int M, int N, int K, const uint16_t *A, int lda, const uint16_t *B, int ldb,
+                           uint16_t *C, int ldc, bool relu, const uint16_t *mask, int ldmask, uint32_t *nonfinite_flag,
+                           uint32_t *status, cudaStream_t st)
+{
     TcParams p;
     p.M = M; p.N = N; p.K = K;
     p.C = C; p.ldc = ldc;
@@ -340,17 +367,11 @@ cudaError_t launch_gemm_tc(int op, int M, int N, int K, const uint16_t *A, int l
 #ifdef MPT_TC_TRACE
     { const char *e = getenv("MPT_DBG"); p.dbg = e ? atoi(e) : 0; }
 #endif
-    p.tiles_m = (M + BLOCK_M - 1) / BLOCK_M;
-    p.tiles_n = (N + BLOCK_N - 1) / BLOCK_N;
-    p.group_m = 16;
-#ifdef MPT_TC_TRACE
-    { const char *e = getenv("MPT_GROUP_M"); if (e) p.group_m = atoi(e); }
-#endif
-    int tiles = p.tiles_m * p.tiles_n;
-    int grid = tiles < 148 ? tiles : 148;
-    if (op == MPT_OP_FWD) return launch_variant<false, false>(ta, tb, p, grid, st);
-    if (op == MPT_OP_DGRAD) return launch_variant<false, true>(ta, tb, p, grid, st);
-    return launch_variant<true, true>(ta, tb, p, grid, st);
+    // 128-wide tiles when 256-wide ones would leave more than a fifth of the SMs without work
+    const long tm = (M + BLOCK_M - 1) / BLOCK_M;
+    const long tiles256 = tm * ((N + 255) / 256);
+    if (tiles256 < 118 && N > 128) return launch_bn<128>(op, M, N, K, A, lda, B, ldb, p, st);
+    return launch_bn<256>(op, M, N, K, A, lda, B, ldb, p, st);
 }
 
 }  // namespace mpt
