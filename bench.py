@@ -50,8 +50,8 @@ def n_params(cfg):
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum of the representative GEMM launch of each workload
-# (ncu capture summarised in profiles/k_gemm_tc_fwd_4096x12288x12288.md), bytes per launch.
-NCU_GEMM_TRAFFIC = {"large": {"launch": "forward 4096x12288x12288", "bytes": 1.345e9, "algorithmic_bytes": 0.503e9}}
+# (ncu capture summarised in profiles/k_gemm_tc2_pair_4096x12288x12288.md), bytes per launch.
+NCU_GEMM_TRAFFIC = {"large": {"launch": "forward 4096x12288x12288", "bytes": 1.652e9, "algorithmic_bytes": 0.503e9}}
 
 
 def max_over_ranks(vals, device=None):
@@ -318,7 +318,7 @@ def main():
                        "l2": "inputs larger than L2 (weights %.1f GB per pass)" % (n_params(cfg) * 2 / 1e9),
                        "flop_per_step": fl},
             "frac_of_nominal_fp16_peak": value / world / NOMINAL_FP16_TFLOPS,
-            "roofline": {"bound": "tensor", "kernel": "k_gemm_tc (all GEMM launches of the step)",
+            "roofline": {"bound": "tensor", "kernel": "pair::k_gemm_tc2 (all GEMM launches of the step)",
                          "achieved": gemm_tflops, "peak": peak_t, "peak_source": peak_src + " (sustained bf16 GEMM; fp16 has the same nominal rate)",
                          "unit": "TFLOP/s", "frac": (gemm_tflops / peak_t) if gemm_tflops else None,
                          "frac_of_nominal": (gemm_tflops / NOMINAL_FP16_TFLOPS) if gemm_tflops else None,
