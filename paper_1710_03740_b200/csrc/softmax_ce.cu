@@ -1,7 +1,9 @@
 // Fused softmax cross-entropy forward + loss-scaled backward (paper sections 3.2, 3.3):
 // FP16 logits in, FP32 max / sum-of-exponentials / log, FP16 logit gradient out with
-// the factor S/B applied.  One CTA per row; the row is read from HBM once (kept in
-// shared memory as FP16) and written once: 4 bytes per logit.
+// the factor S/B applied.  One CTA per row; the row is read from HBM once and written
+// once: 4 bytes per logit.  Rows of up to 65536 classes with 16-byte aligned pitches stay
+// in registers (k_softmax_ce_reg); other rows go through shared memory or are re-read
+// (k_softmax_ce).
 #include "mpt_common.cuh"
 
 namespace mpt {
@@ -114,6 +116,96 @@ __global__ void __launch_bounds__(1024) k_softmax_ce(const uint16_t *__restrict_
     }
 }
 
+// Register-resident variant: thread t holds the 8-element vectors t, t + T, t + 2T, ... of its
+// row (T = blockDim.x, at most VPT of them) and, for rows whose length is not a multiple of 8,
+// threads 0..6 hold one tail element each.  Exponentials are 2^((z - m) * log2 e) on the
+// special-function unit: z - m is exact near the maximum, so the rounding of the argument
+// only touches terms far below it, and is far below FP16 resolution after the store.  Non-label outputs are e_j * (c / s); the label's output is
+// (e_y / s - 1) * c, evaluated separately because of the cancellation.
+template <int VPT>
+__global__ void __launch_bounds__(1024) k_softmax_ce_reg(const uint16_t *__restrict__ z, int ldz,
+                                                         const int32_t *__restrict__ labels, int C, float c,
+                                                         uint16_t *__restrict__ dz, int lddz,
+                                                         float *__restrict__ row_loss, uint32_t *bad_labels)
+{
+    __shared__ float red[32];
+    const int tid = threadIdx.x, nt = blockDim.x, row = blockIdx.x;
+    const int C8 = C >> 3, tail = C & 7;
+    const uint16_t *zr = z + (size_t)row * ldz;
+    uint16_t *dr = dz + (size_t)row * lddz;
+    const int y = labels[row];
+    if (y < 0 || y >= C) {  // contributes neither loss nor gradient
+        for (int j = tid; j < C; j += nt) dr[j] = 0;
+        if (tid == 0) {
+            row_loss[row] = 0.0f;
+            if (bad_labels) atomicAdd(bad_labels, 1u);
+        }
+        return;
+    }
+    constexpr float LOG2E = 1.4426950408889634f;
+    uint4 x[VPT];
+#pragma unroll
+    for (int u = 0; u < VPT; u++) {
+        const int i = tid + u * nt;
+        if (i < C8) x[u] = __ldcs((const uint4 *)zr + i);
+    }
+    float tv = 0.0f;
+    const bool has_tail = tid < tail;
+    if (has_tail) tv = hbits2f(zr[C8 * 8 + tid]);
+
+    float m = -INFINITY;
+#pragma unroll
+    for (int u = 0; u < VPT; u++) {
+        if (tid + u * nt < C8) {
+            const uint32_t w[4] = {x[u].x, x[u].y, x[u].z, x[u].w};
+#pragma unroll
+            for (int q = 0; q < 4; q++) m = fmaxf(m, fmaxf(hbits2f(w[q] & 0xFFFFu), hbits2f(w[q] >> 16)));
+        }
+    }
+    if (has_tail) m = fmaxf(m, tv);
+    m = block_reduce(m, true, red);
+
+    float s = 0.0f;
+#pragma unroll
+    for (int u = 0; u < VPT; u++) {
+        if (tid + u * nt < C8) {
+            const uint32_t w[4] = {x[u].x, x[u].y, x[u].z, x[u].w};
+#pragma unroll
+            for (int q = 0; q < 4; q++) {
+                s += exp2f((hbits2f(w[q] & 0xFFFFu) - m) * LOG2E);
+                s += exp2f((hbits2f(w[q] >> 16) - m) * LOG2E);
+            }
+        }
+    }
+    if (has_tail) s += exp2f((tv - m) * LOG2E);
+    s = block_reduce(s, false, red);
+    const float inv_s = __fdiv_rn(1.0f, s);
+    const float k = inv_s * c;
+    if (tid == 0) row_loss[row] = (m + logf(s)) - hbits2f(zr[y]);
+
+#pragma unroll
+    for (int u = 0; u < VPT; u++) {
+        const int i = tid + u * nt;
+        if (i < C8) {
+            const uint32_t w[4] = {x[u].x, x[u].y, x[u].z, x[u].w};
+            uint32_t o[4];
+#pragma unroll
+            for (int q = 0; q < 4; q++) {
+                const float d0 = exp2f((hbits2f(w[q] & 0xFFFFu) - m) * LOG2E) * k;
+                const float d1 = exp2f((hbits2f(w[q] >> 16) - m) * LOG2E) * k;
+                o[q] = f2hbits(d0) | (f2hbits(d1) << 16);
+            }
+            __stcs((uint4 *)dr + i, make_uint4(o[0], o[1], o[2], o[3]));
+        }
+    }
+    if (has_tail) dr[C8 * 8 + tid] = (uint16_t)f2hbits(exp2f((tv - m) * LOG2E) * k);
+    __syncthreads();  // the row's stores are done before the label element is patched
+    if (tid == 0) {
+        const float ey = exp2f((hbits2f(zr[y]) - m) * LOG2E);
+        dr[y] = (uint16_t)f2hbits(__fmul_rn(__fsub_rn(ey * inv_s, 1.0f), c));
+    }
+}
+
 // loss = (float)( sum_i (double)row_loss[i] / B ), fixed reduction order.
 __global__ void __launch_bounds__(256) k_loss_mean(const float *__restrict__ row_loss, int B, float *loss)
 {
@@ -151,6 +243,29 @@ cudaError_t launch_softmax_ce(const uint16_t *z, int ldz, const int32_t *labels,
     if (B <= 0 || C <= 0) return cudaSuccess;
     const float c = S / (float)B;  // one FP32 division
     const bool vec = ((((uintptr_t)z | (uintptr_t)dz) & 15) == 0) && (ldz % 8 == 0) && (lddz % 8 == 0) && C >= 8;
+    if (vec && (C >> 3) <= 8 * 1024) {
+        // register-resident rows: T threads x VPT vectors cover C / 8 vectors
+        const int C8 = C >> 3;
+        int vpt = 1;
+        while (vpt < 8 && (long)vpt * 1024 < C8) vpt *= 2;
+        int threads = (C8 + vpt - 1) / vpt;
+        threads = ((threads + 31) / 32) * 32;
+        if (threads < 32) threads = 32;
+        switch (vpt) {
+            case 1: k_softmax_ce_reg<1><<<B, threads, 0, st>>>(z, ldz, labels, C, c, dz, lddz, row_loss, bad_labels); break;
+            case 2: k_softmax_ce_reg<2><<<B, threads, 0, st>>>(z, ldz, labels, C, c, dz, lddz, row_loss, bad_labels); break;
+            case 4: k_softmax_ce_reg<4><<<B, threads, 0, st>>>(z, ldz, labels, C, c, dz, lddz, row_loss, bad_labels); break;
+            default: k_softmax_ce_reg<8><<<B, threads, 0, st>>>(z, ldz, labels, C, c, dz, lddz, row_loss, bad_labels); break;
+        }
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+        if (n_launches) *n_launches = 1;
+        if (loss) {
+            k_loss_mean<<<1, 256, 0, st>>>(row_loss, B, loss);
+            if (n_launches) *n_launches = 2;
+        }
+        return cudaGetLastError();
+    }
     const size_t row_bytes = ((size_t)C * 2 + 15) & ~(size_t)15;
     const bool cache = row_bytes <= (size_t)kMaxSmemRowBytes;
     int threads = vec ? (C / 8) : C;
