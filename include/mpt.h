@@ -91,8 +91,8 @@ typedef struct mpt_layer_desc {
 
 /* Size in bytes of the single device workspace a context needs (section 3.1:
  * FP32 master + FP16 weights + FP16 gradients, optional FP32 momentum, FP16
- * activations and activation gradients for max_batch rows, an input staging
- * buffer, per-row losses and status words).  Host-only; no CUDA call. */
+ * activations and activation gradients for max_batch rows, two input staging
+ * slots, per-row losses and status words).  Host-only; no CUDA call. */
 int mpt_workspace_bytes(const mpt_layer_desc *layers, int n_layers, int max_batch,
                         int use_momentum, size_t *bytes_out);
 
@@ -157,6 +157,20 @@ int mpt_get_master(mpt_ctx *ctx, int layer, float *dst_host, size_t n);
  * the loss and the overflow flag.  Synchronises the stream before returning. */
 int mpt_train_step_host(mpt_ctx *ctx, const uint16_t *x_host, const int32_t *labels_host, int batch,
                         float *loss_host, int *overflow_host);
+
+/* The same iteration with the host-to-device copy of a batch overlapped with the compute of
+ * the previous one (the method's steps and arithmetic are those of mpt_train_step_host).
+ * mpt_stage_batch_host copies x_host / labels_host into one of two staging slots on
+ * copy_stream (a cudaStream_t of the caller, normally different from the context's stream) and
+ * returns at once; host buffers must stay valid until that copy has run (use pinned memory for a
+ * truly asynchronous copy).  mpt_train_step_staged makes the context's stream wait for the
+ * oldest staged batch, runs forward, scaled backward and the master-weight pass on it,
+ * synchronises and returns loss and overflow flag.  At most two batches can be staged;
+ * staging a third, or stepping with none staged, returns MPT_ERR_STATE.  Typical loop:
+ *   stage(batch 0); for t: stage(batch t+1); train_step_staged();                      */
+int mpt_stage_batch_host(mpt_ctx *ctx, const uint16_t *x_host, const int32_t *labels_host, int batch,
+                         void *copy_stream);
+int mpt_train_step_staged(mpt_ctx *ctx, float *loss_host, int *overflow_host);
 
 /* Change the loss scale (section 3.2) / learning rate; takes effect at the next
  * mpt_backward_scaled / mpt_step.  Same range checks as mpt_create. */

@@ -24,7 +24,8 @@ T_W16, T_GRAD16, T_ACT16, T_DACT16, T_MOMENTUM32, T_MASTER32 = range(6)
 
 # every symbol include/mpt.h declares
 EXPORTS = ["mpt_workspace_bytes", "mpt_create", "mpt_set_master", "mpt_forward", "mpt_backward_scaled",
-           "mpt_step", "mpt_get_master", "mpt_train_step_host", "mpt_set_scale", "mpt_set_lr",
+           "mpt_step", "mpt_get_master", "mpt_train_step_host", "mpt_stage_batch_host",
+           "mpt_train_step_staged", "mpt_set_scale", "mpt_set_lr",
            "mpt_get_tensor", "mpt_set_grad", "mpt_set_momentum", "mpt_launch_count", "mpt_profile",
            "mpt_profile_read", "mpt_last_error",
            "mpt_destroy", "mpt_gemm_f16", "mpt_recast", "mpt_grad_nonfinite", "mpt_update_flat",
@@ -61,6 +62,8 @@ def lib() -> C.CDLL:
     L.mpt_step.argtypes = [vp, C.POINTER(i32)]
     L.mpt_get_master.argtypes = [vp, i32, vp, sz]
     L.mpt_train_step_host.argtypes = [vp, vp, vp, i32, C.POINTER(f32), C.POINTER(i32)]
+    L.mpt_stage_batch_host.argtypes = [vp, vp, vp, i32, vp]
+    L.mpt_train_step_staged.argtypes = [vp, C.POINTER(f32), C.POINTER(i32)]
     L.mpt_set_scale.argtypes = [vp, f32]
     L.mpt_set_lr.argtypes = [vp, f32]
     L.mpt_get_tensor.argtypes = [vp, i32, i32, vp, sz]
@@ -191,6 +194,16 @@ class Context:
         _check(lib().mpt_train_step_host(self._ctx, _hptr(x_host), _hptr(labels_host), batch, C.byref(loss),
                                          C.byref(flag)), self._ctx)
         self.batch = batch
+        return float(loss.value), int(flag.value)
+
+    def stage_batch_host(self, x_host, labels_host, copy_stream):
+        """Start the host-to-device copy of one batch on `copy_stream` (a torch.cuda.Stream)."""
+        _check(lib().mpt_stage_batch_host(self._ctx, _hptr(x_host), _hptr(labels_host), int(x_host.shape[0]),
+                                          C.c_void_p(copy_stream.cuda_stream)), self._ctx)
+
+    def train_step_staged(self):
+        loss, flag = C.c_float(0.0), C.c_int(0)
+        _check(lib().mpt_train_step_staged(self._ctx, C.byref(loss), C.byref(flag)), self._ctx)
         return float(loss.value), int(flag.value)
 
     def set_scale(self, S):

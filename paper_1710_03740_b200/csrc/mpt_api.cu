@@ -28,8 +28,8 @@ struct Layer {
 
 struct Plan {
     size_t total = 0, P_pad = 0;
-    size_t off_status = 0, off_master = 0, off_mom = 0, off_w16 = 0, off_g16 = 0, off_x = 0, off_labels = 0,
-           off_rowloss = 0;
+    size_t off_status = 0, off_master = 0, off_mom = 0, off_w16 = 0, off_g16 = 0, off_x[2] = {0, 0},
+           off_labels[2] = {0, 0}, off_rowloss = 0;
     std::vector<size_t> off_act, off_dact, lay_off;
     std::vector<int> ld_out;
 };
@@ -74,8 +74,10 @@ void make_plan(const mpt_layer_desc *layers, int L, int max_batch, bool mom, Pla
         pl.off_act[l] = take((size_t)max_batch * pl.ld_out[l] * 2);
     }
     for (int l = 0; l < L; l++) pl.off_dact[l] = take((size_t)max_batch * pl.ld_out[l] * 2);
-    pl.off_x = take((size_t)max_batch * layers[0].in_features * 2);
-    pl.off_labels = take((size_t)max_batch * 4);
+    for (int k = 0; k < 2; k++) {   // two staging slots: one being consumed, one being filled
+        pl.off_x[k] = take((size_t)max_batch * layers[0].in_features * 2);
+        pl.off_labels[k] = take((size_t)max_batch * 4);
+    }
     pl.off_rowloss = take((size_t)max_batch * 4);
     pl.total = off;
 }
@@ -92,8 +94,13 @@ struct mpt_ctx {
     Plan plan;
     uint32_t *status;
     float *master, *mom;
-    uint16_t *w16, *g16, *x_stage;
-    int32_t *labels_stage;
+    uint16_t *w16, *g16, *x_stage[2];
+    int32_t *labels_stage[2];
+    // staged (pipelined) host batches: slot state and the events that order copies against compute
+    cudaEvent_t staged_ev[2] = {nullptr, nullptr}, used_ev[2] = {nullptr, nullptr};
+    bool staged_valid[2] = {false, false}, used_recorded[2] = {false, false};
+    int staged_batch[2] = {0, 0};
+    int stage_w = 0, stage_r = 0;
     float *row_loss;
     const uint16_t *x_cur = nullptr;
     int batch = 0;
@@ -320,8 +327,10 @@ int mpt_create(const mpt_layer_desc *layers, int n_layers, float S, float lr, fl
     c->mom = c->use_momentum ? (float *)(c->ws + pl.off_mom) : nullptr;
     c->w16 = (uint16_t *)(c->ws + pl.off_w16);
     c->g16 = (uint16_t *)(c->ws + pl.off_g16);
-    c->x_stage = (uint16_t *)(c->ws + pl.off_x);
-    c->labels_stage = (int32_t *)(c->ws + pl.off_labels);
+    for (int k = 0; k < 2; k++) {
+        c->x_stage[k] = (uint16_t *)(c->ws + pl.off_x[k]);
+        c->labels_stage[k] = (int32_t *)(c->ws + pl.off_labels[k]);
+    }
     c->row_loss = (float *)(c->ws + pl.off_rowloss);
     c->layers.resize(n_layers);
     for (int l = 0; l < n_layers; l++) {
@@ -340,7 +349,11 @@ int mpt_create(const mpt_layer_desc *layers, int n_layers, float S, float lr, fl
     // Parameter arenas (including the padding between layers), activations and status start at zero.
     cudaError_t e = cudaMemsetAsync(c->ws, 0, pl.total, c->stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
-    if (e != cudaSuccess) { delete c; return MPT_ERR_CUDA; }
+    for (int k = 0; k < 2 && e == cudaSuccess; k++) {
+        e = cudaEventCreateWithFlags(&c->staged_ev[k], cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->used_ev[k], cudaEventDisableTiming);
+    }
+    if (e != cudaSuccess) { mpt_destroy(c); return MPT_ERR_CUDA; }
     *out = c;
     return MPT_OK;
 }
@@ -350,6 +363,10 @@ void mpt_destroy(mpt_ctx *c)
     if (!c) return;
     for (auto &sp : c->spans) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
     for (auto &sp : c->pool) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
+    for (int k = 0; k < 2; k++) {
+        if (c->staged_ev[k]) cudaEventDestroy(c->staged_ev[k]);
+        if (c->used_ev[k]) cudaEventDestroy(c->used_ev[k]);
+    }
     delete c;
 }
 
@@ -487,15 +504,64 @@ int mpt_train_step_host(mpt_ctx *c, const uint16_t *x_host, const int32_t *label
     if (r != MPT_OK) return r;
     if (!x_host || !labels_host) return fail(c, MPT_ERR_INVALID_ARG, "null host input");
     if (batch < 1 || batch > c->max_batch) return fail(c, MPT_ERR_SHAPE, "batch outside [1, max_batch]");
-    CK(cudaMemcpyAsync(c->x_stage, x_host, (size_t)batch * c->layers[0].in * 2, cudaMemcpyHostToDevice, c->stream),
+    if (c->staged_valid[0] || c->staged_valid[1])
+        return fail(c, MPT_ERR_STATE, "a staged batch is pending: use mpt_train_step_staged");
+    CK(cudaMemcpyAsync(c->x_stage[0], x_host, (size_t)batch * c->layers[0].in * 2, cudaMemcpyHostToDevice, c->stream),
        "input upload");
-    CK(cudaMemcpyAsync(c->labels_stage, labels_host, (size_t)batch * 4, cudaMemcpyHostToDevice, c->stream), "label upload");
-    r = do_forward(c, c->x_stage, batch);
+    CK(cudaMemcpyAsync(c->labels_stage[0], labels_host, (size_t)batch * 4, cudaMemcpyHostToDevice, c->stream), "label upload");
+    r = do_forward(c, c->x_stage[0], batch);
     if (r != MPT_OK) return r;
-    r = do_backward(c, c->labels_stage);
+    r = do_backward(c, c->labels_stage[0]);
     if (r != MPT_OK) return r;
     r = do_step(c);
     if (r != MPT_OK) return r;
+    uint32_t st[ST_WORDS];
+    r = read_status(c, st);
+    if (r != MPT_OK) return r;
+    if (loss_host) memcpy(loss_host, &st[ST_LOSS], 4);
+    r = finish_step(c, st, overflow_host);
+    if (r != MPT_OK) return r;
+    if (st[ST_BAD_LABELS]) return fail(c, MPT_ERR_INVALID_ARG, "labels outside [0, C) were ignored");
+    return MPT_OK;
+}
+
+int mpt_stage_batch_host(mpt_ctx *c, const uint16_t *x_host, const int32_t *labels_host, int batch, void *copy_stream)
+{
+    int r = usable(c);
+    if (r != MPT_OK) return r;
+    if (!x_host || !labels_host) return fail(c, MPT_ERR_INVALID_ARG, "null host input");
+    if (batch < 1 || batch > c->max_batch) return fail(c, MPT_ERR_SHAPE, "batch outside [1, max_batch]");
+    const int k = c->stage_w;
+    if (c->staged_valid[k]) return fail(c, MPT_ERR_STATE, "both staging slots hold unconsumed batches");
+    cudaStream_t cs = (cudaStream_t)copy_stream;
+    // the slot's previous consumer (the step that read it) must have finished before it is overwritten
+    if (c->used_recorded[k]) CK(cudaStreamWaitEvent(cs, c->used_ev[k], 0), "wait for the slot's last consumer");
+    CK(cudaMemcpyAsync(c->x_stage[k], x_host, (size_t)batch * c->layers[0].in * 2, cudaMemcpyHostToDevice, cs), "input upload");
+    CK(cudaMemcpyAsync(c->labels_stage[k], labels_host, (size_t)batch * 4, cudaMemcpyHostToDevice, cs), "label upload");
+    CK(cudaEventRecord(c->staged_ev[k], cs), "event record");
+    c->staged_valid[k] = true;
+    c->staged_batch[k] = batch;
+    c->stage_w ^= 1;
+    return MPT_OK;
+}
+
+int mpt_train_step_staged(mpt_ctx *c, float *loss_host, int *overflow_host)
+{
+    int r = usable(c);
+    if (r != MPT_OK) return r;
+    const int k = c->stage_r;
+    if (!c->staged_valid[k]) return fail(c, MPT_ERR_STATE, "no staged batch: call mpt_stage_batch_host first");
+    CK(cudaStreamWaitEvent(c->stream, c->staged_ev[k], 0), "wait for the staged batch");
+    r = do_forward(c, c->x_stage[k], c->staged_batch[k]);
+    if (r != MPT_OK) return r;
+    r = do_backward(c, c->labels_stage[k]);
+    if (r != MPT_OK) return r;
+    r = do_step(c);
+    if (r != MPT_OK) return r;
+    CK(cudaEventRecord(c->used_ev[k], c->stream), "event record");
+    c->used_recorded[k] = true;
+    c->staged_valid[k] = false;
+    c->stage_r ^= 1;
     uint32_t st[ST_WORDS];
     r = read_status(c, st);
     if (r != MPT_OK) return r;

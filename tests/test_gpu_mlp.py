@@ -164,6 +164,44 @@ def test_train_step_host_matches_device_calls_and_checkpoint_resume():
         assert net1.get_master(l).tobytes() == net3.get_master(l).tobytes()
 
 
+def test_staged_pipeline_matches_plain_host_steps():
+    """Copy of batch t+1 overlapped with the compute of batch t: same losses, flags and masters."""
+    from paper_1710_03740_b200 import binding as b
+    cfg = inputs.MLP_CONFIGS["tiny"]
+    masters = inputs.mlp_masters(cfg)
+    X, Y = inputs.mlp_batches(cfg, 5)
+    net1, _ = _make(cfg, cfg["S"], masters)
+    net2, _ = _make(cfg, cfg["S"], masters)
+    Xp = [torch.from_numpy(X[t].view(np.int16)).pin_memory() for t in range(5)]
+    Yp = [torch.from_numpy(Y[t]).pin_memory() for t in range(5)]
+    ref = [net1.train_step_host(Xp[t], Yp[t]) for t in range(5)]
+    cs = torch.cuda.Stream()
+    with pytest.raises(b.MptError) as e:
+        net2.train_step_staged()                         # nothing staged yet
+    assert e.value.code == -3
+    net2.stage_batch_host(Xp[0], Yp[0], cs)
+    got = []
+    for t in range(5):
+        if t + 1 < 5:
+            net2.stage_batch_host(Xp[t + 1], Yp[t + 1], cs)
+        got.append(net2.train_step_staged())
+    assert got == ref
+    for l in range(2):
+        assert net1.get_master(l).tobytes() == net2.get_master(l).tobytes()
+    # a third staged batch is refused; mixing with the unstaged call is refused while one is pending
+    net2.stage_batch_host(Xp[0], Yp[0], cs)
+    net2.stage_batch_host(Xp[1], Yp[1], cs)
+    with pytest.raises(b.MptError) as e:
+        net2.stage_batch_host(Xp[2], Yp[2], cs)
+    assert e.value.code == -3
+    with pytest.raises(b.MptError) as e:
+        net2.train_step_host(Xp[2], Yp[2])
+    assert e.value.code == -3
+    net2.train_step_staged()
+    net2.train_step_staged()
+    cs.synchronize()
+
+
 def test_error_paths():
     from paper_1710_03740_b200 import binding as b
     cfg = inputs.MLP_CONFIGS["tiny"]
