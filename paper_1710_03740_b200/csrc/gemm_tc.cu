@@ -19,7 +19,6 @@
 // word, raises a CTA-wide abort flag and all roles fall through to the common exit,
 // which frees the tensor memory.
 #include <cuda.h>
-#include <cstdlib>
 
 #include "mpt_common.cuh"
 #include "tc_ptx.cuh"
@@ -58,9 +57,6 @@ struct TcParams {
     int relu;
     uint32_t *nonfinite_flag;
     uint32_t *status;  // may be null
-#ifdef MPT_TC_TRACE
-    int dbg;
-#endif
     int tiles_m, tiles_n, group_m;
 };
 
@@ -140,9 +136,6 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                         break;
                     }
                     const uint32_t sa = base + s * STAGE_BYTES, sb = sa + A_STAGE_BYTES;
-#ifdef MPT_TC_TRACE
-                    if ((p.dbg & 1) && issued >= (uint32_t)STAGES) { mbar_arrive(full_bar(s)); continue; }
-#endif
                     mbar_arrive_expect_tx(full_bar(s), STAGE_BYTES);
                     const int k0 = kb * BLOCK_K;
                     if (A_MN) {
@@ -204,9 +197,6 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                     const uint32_t blo = b_lo0 + s * (uint32_t)(STAGE_BYTES >> 4);
 #pragma unroll
                     for (int k = 0; k < BLOCK_K / UMMA_K; k++) {
-#ifdef MPT_TC_TRACE
-                        if (p.dbg & 4) continue;
-#endif
                         tc_mma_f16(d_tmem, desc_join(alo + k * KSTEP_A, a_hi), desc_join(blo + k * KSTEP_B, b_hi), idesc, acc);
                         acc = 1;
                     }
@@ -243,9 +233,6 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                 tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BLOCK_N + c * 32), r);
                 tc_wait_ld();
                 const int col0 = nb * BLOCK_N + c * 32;
-#ifdef MPT_TC_TRACE
-                if (p.dbg & 2) { if (r[0] == 0x12345678u && r[7] == 0x9abcdef0u) bad = true; continue; }
-#endif
                 if (row_ok && col0 < p.N) epilogue_store32(r, crow, mrow, col0, p.N, p.relu != 0, bad);
             }
             tc_fence_before();
@@ -343,9 +330,6 @@ static cudaError_t launch_bn(int op, int M, int N, int K, const uint16_t *A, int
     p.tiles_m = (M + BLOCK_M - 1) / BLOCK_M;
     p.tiles_n = (N + BN - 1) / BN;
     p.group_m = 16;
-#ifdef MPT_TC_TRACE
-    { const char *e = getenv("MPT_GROUP_M"); if (e) p.group_m = atoi(e); }
-#endif
     int tiles = p.tiles_m * p.tiles_n;
     int grid = tiles < 148 ? tiles : 148;
     if (op == MPT_OP_FWD) return launch_variant<false, false, BN>(ta, tb, p, grid, st);
@@ -364,9 +348,6 @@ cudaError_t launch_gemm_tc(int op, int M, int N, int K, const uint16_t *A, int l
     p.relu = relu ? 1 : 0;
     p.nonfinite_flag = nonfinite_flag;
     p.status = status;
-#ifdef MPT_TC_TRACE
-    { const char *e = getenv("MPT_DBG"); p.dbg = e ? atoi(e) : 0; }
-#endif
     // 128-wide tiles when 256-wide ones would leave more than a fifth of the SMs without work
     const long tm = (M + BLOCK_M - 1) / BLOCK_M;
     const long tiles256 = tm * ((N + 255) / 256);

@@ -18,7 +18,6 @@
 //   acce[b]   in the leader: 8 arrivals, one per epilogue warp of both CTAs
 // No TMA multicast is used.  Every mbarrier wait is bounded (see tc_ptx.cuh).
 #include <cuda.h>
-#include <cstdlib>
 
 #include "mpt_common.cuh"
 #include "tc_ptx.cuh"
@@ -27,11 +26,6 @@ namespace mpt {
 
 namespace pair {
 
-#ifdef MPT_TC_TRACE
-#define TRACE(slot, t) do { if (blockIdx.x == 0 && p.status && (t) < 32) p.status[16 + 8 * (t) + (slot)] = (uint32_t)global_ns(); } while (0)
-#else
-#define TRACE(slot, t) do { } while (0)
-#endif
 
 static constexpr int CTA_M = 128;          // rows per CTA (256 per pair)
 static constexpr int TILE_N = 256;         // columns per pair tile
@@ -61,9 +55,6 @@ struct Params {
     int relu;
     uint32_t *nonfinite_flag;
     uint32_t *status;
-#ifdef MPT_TC_TRACE
-    int dbg;
-#endif
     int tiles_m, tiles_n, group_m;   // pair tiles (256 rows x 256 columns)
 };
 
@@ -100,10 +91,6 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
     volatile uint32_t *abort_flag = tmem_slot + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (threadIdx.x == 0) TRACE(6, 0);
-#ifdef MPT_TC_TRACE
-    if (threadIdx.x == 0 && blockIdx.x == 0 && p.status) p.status[16 + 8 * 2 + 6] = (uint32_t)clock64();
-#endif
     const uint32_t rank = cluster_ctarank();       // 0 = leader of the pair
     const bool leader = rank == 0;
     const int pair_id = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
@@ -128,7 +115,6 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
     cluster_sync_all();                            // the peer's barriers exist before anything signals them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    if (threadIdx.x == 0) TRACE(7, 0);
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer (both CTAs)
@@ -148,9 +134,6 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
                     }
                     const uint32_t sa = base + s * STAGE_BYTES, sb = sa + A_STAGE_BYTES;
                     const uint32_t lead_full = mapa_u32(full_bar(s), 0);
-#ifdef MPT_TC_TRACE
-                    if ((p.dbg & 1) && issued >= (uint32_t)STAGES) { if (leader) mbar_arrive(full_bar(s)); continue; }
-#endif
                     if (leader) mbar_arrive_expect_tx(full_bar(s), 2 * STAGE_BYTES);
                     const int k0 = kb * BLOCK_K;
                     if (A_MN) {
@@ -198,7 +181,6 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
                     break;
                 }
                 tc_fence_after();
-                TRACE(0, t);
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * TILE_N);
                 uint32_t acc = 0;                          // first MMA of a tile overwrites the accumulator
                 for (int kb = 0; kb < nkb; kb++) {
@@ -208,14 +190,10 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
                         break;
                     }
                     tc_fence_after();
-                    if (kb == 0) TRACE(1, t);
                     const uint32_t alo = a_lo0 + s * (uint32_t)(STAGE_BYTES >> 4);
                     const uint32_t blo = b_lo0 + s * (uint32_t)(STAGE_BYTES >> 4);
 #pragma unroll
                     for (int k = 0; k < BLOCK_K / UMMA_K; k++) {
-#ifdef MPT_TC_TRACE
-                        if (p.dbg & 4) continue;
-#endif
                         tc_mma_f16_pair(d_tmem, desc_join(alo + k * KSTEP_A, a_hi), desc_join(blo + k * KSTEP_B, b_hi), idesc, acc);
                         acc = 1;
                     }
@@ -223,7 +201,6 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
                 if (ok) tc_commit_pair(accf_bar(buf), 3);   // both CTAs' epilogues may read the accumulator
-                TRACE(2, t);
             }
         }
     } else {
@@ -243,7 +220,6 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
                 break;
             }
             tc_fence_after();
-            if (warp == 2 && lane == 0) TRACE(3, t);
             const int row = mb * (2 * CTA_M) + (int)rank * CTA_M + q * 32 + lane;
             const bool row_ok = row < p.M;
             uint16_t *crow = p.C + (size_t)row * p.ldc;
@@ -255,16 +231,11 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
                 tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * TILE_N + c * 32), r);
                 tc_wait_ld();
                 const int col0 = nb * TILE_N + c * 32;
-#ifdef MPT_TC_TRACE
-                if (p.dbg & 2) { if (r[0] == 0x12345678u && r[7] == 0x9abcdef0u) bad = true; continue; }
-#endif
                 if (row_ok && col0 < p.N) epilogue_store32(r, crow, mrow, col0, p.N, p.relu != 0, bad);
             }
             tc_fence_before();
             __syncwarp();
-            if (warp == 2 && lane == 0) TRACE(4, t);
             if (lane == 0) mbar_arrive_cluster(mapa_u32(acce_bar(buf), 0));
-            if (warp == 2 && lane == 0) TRACE(5, t);
             if (p.nonfinite_flag && __any_sync(0xFFFFFFFFu, bad) && lane == 0) atomicOr(p.nonfinite_flag, 1u);
         }
     }
@@ -273,12 +244,7 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
     // may leave while the other can still touch its shared or tensor memory
     tc_fence_before();
     __syncthreads();
-    if (threadIdx.x == 0) TRACE(6, 1);
     cluster_sync_all();
-    if (threadIdx.x == 0) TRACE(7, 1);
-#ifdef MPT_TC_TRACE
-    if (threadIdx.x == 0 && blockIdx.x == 0 && p.status) p.status[16 + 8 * 2 + 7] = (uint32_t)clock64();
-#endif
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS) : "memory");
@@ -349,15 +315,9 @@ cudaError_t launch_gemm_tc2(int op, int M, int N, int K, const uint16_t *A, int 
     p.relu = relu ? 1 : 0;
     p.nonfinite_flag = nonfinite_flag;
     p.status = status;
-#ifdef MPT_TC_TRACE
-    { const char *e = getenv("MPT_DBG"); p.dbg = e ? atoi(e) : 0; }
-#endif
     p.tiles_m = (M + 2 * CTA_M - 1) / (2 * CTA_M);
     p.tiles_n = (N + TILE_N - 1) / TILE_N;
     p.group_m = 8;
-#ifdef MPT_TC_TRACE
-    { const char *e = getenv("MPT_GROUP_M"); if (e) p.group_m = atoi(e); }
-#endif
     int tiles = p.tiles_m * p.tiles_n;
     if (op == MPT_OP_FWD) return launch_variant<false, false>(ta, tb, p, tiles, st);
     if (op == MPT_OP_DGRAD) return launch_variant<false, true>(ta, tb, p, tiles, st);
