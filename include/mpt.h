@@ -177,6 +177,18 @@ int mpt_train_step_staged(mpt_ctx *ctx, float *loss_host, int *overflow_host);
 int mpt_set_scale(mpt_ctx *ctx, float S);
 int mpt_set_lr(mpt_ctx *ctx, float lr);
 
+/* Dynamic loss scaling (the paper's closing section: the scale "could be dynamically increased
+ * or decreased by inspecting the weight gradients for overflow, skipping weight updates when
+ * an overflow is detected"; no schedule is given there).  The schedule taken here: after a
+ * step that overflowed (and was skipped) S <- max(S/2, min_scale); after growth_interval
+ * consecutive steps without overflow S <- min(2*S, max_scale); either event restarts the
+ * count.  S stays a power of two if it starts as one, so scaling remains exact.  The scale
+ * lives in device memory and is adjusted by a one-thread kernel at the end of mpt_step: no host
+ * synchronisation is added.  enable = 0 returns to a constant scale (the current value).
+ * mpt_get_scale synchronises and returns the scale the next backward pass will use. */
+int mpt_set_dynamic_scale(mpt_ctx *ctx, int enable, int growth_interval, float min_scale, float max_scale);
+int mpt_get_scale(mpt_ctx *ctx, float *S_out);
+
 /* Test and checkpoint hooks.  mpt_get_tensor downloads an internal tensor without
  * padding (bytes must equal rows*cols*element size; ACT16/DACT16 use the batch of
  * the last forward; ACT16 layer l is a_{l+1}, the output of layer l).

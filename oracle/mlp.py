@@ -9,6 +9,11 @@ paper describes for a layer (section 3.1, figure 1 caption; section 3.2):
   unscale by 1/S while inspecting for inf/NaN -> skip, or FP32 SGD(+momentum)
   on the master copy and re-round the FP16 copy.
 
+Dynamic loss scaling (the paper's closing section only says the factor could be raised or
+lowered by inspecting the weight gradients for overflow while skipping overflowing updates):
+after an overflowing step S <- max(S * backoff, min); after `growth_interval` consecutive
+clean steps S <- min(S * growth, max); either event restarts the count.
+
 Readings where the paper is silent: no bias; mean loss over the batch; momentum
 form v <- mu*v + g, w <- w - lr*v with v in FP32 starting at zero; a skipped step
 leaves master, momentum and FP16 weights untouched; the ReLU derivative is taken
@@ -36,6 +41,8 @@ class OracleMLP:
         self.w16 = [None] * len(self.layers)
         self.v = [np.zeros((o, i), dtype=np.float32) for (i, o, _) in self.layers]
         self.g16 = [np.zeros((o, i), dtype=np.uint16) for (i, o, _) in self.layers]
+        self.dynamic = None    # (growth_interval, backoff, growth, min_scale, max_scale) or None
+        self.clean_steps = 0
         self.acts = None       # [a_0 .. a_L], uint16
         self.dz = None         # dz_l for l = 1..L (index l-1), uint16
         self.loss = None
@@ -75,18 +82,33 @@ class OracleMLP:
                                               mask=self.acts[l] if self.layers[l - 1][2] else None)
         return loss
 
+    def set_dynamic_scale(self, growth_interval, min_scale, max_scale, backoff=0.5, growth=2.0):
+        self.dynamic = (int(growth_interval), np.float32(backoff), np.float32(growth), np.float32(min_scale),
+                        np.float32(max_scale))
+        self.clean_steps = 0
+        self.S = np.float32(min(max(self.S, np.float32(min_scale)), np.float32(max_scale)))
+
     # -- sections 3.1, 3.2: unscale, inspect, skip or update
     def step(self):
         inv = np.float32(1.0) / self.S
         overflow = 0
         for g in self.g16:
             overflow |= mpo.grad_nonfinite(g, inv)
-        if overflow:
-            return 1
-        for l in range(len(self.layers)):
-            mpo.update_apply(self.g16[l], self.w32[l], self.v[l], self.w16[l], inv, self.lr, self.mu,
-                             self.use_momentum)
-        return 0
+        if not overflow:
+            for l in range(len(self.layers)):
+                mpo.update_apply(self.g16[l], self.w32[l], self.v[l], self.w16[l], inv, self.lr, self.mu,
+                                 self.use_momentum)
+        if self.dynamic is not None:
+            interval, backoff, growth, smin, smax = self.dynamic
+            if overflow:
+                self.S = np.float32(max(np.float32(self.S * backoff), smin))
+                self.clean_steps = 0
+            else:
+                self.clean_steps += 1
+                if self.clean_steps >= interval:
+                    self.S = np.float32(min(np.float32(self.S * growth), smax))
+                    self.clean_steps = 0
+        return 1 if overflow else 0
 
     def set_grad(self, l, g16):
         i, o, _ = self.layers[l]

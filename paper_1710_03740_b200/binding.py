@@ -25,7 +25,7 @@ T_W16, T_GRAD16, T_ACT16, T_DACT16, T_MOMENTUM32, T_MASTER32 = range(6)
 # every symbol include/mpt.h declares
 EXPORTS = ["mpt_workspace_bytes", "mpt_create", "mpt_set_master", "mpt_forward", "mpt_backward_scaled",
            "mpt_step", "mpt_get_master", "mpt_train_step_host", "mpt_stage_batch_host",
-           "mpt_train_step_staged", "mpt_set_scale", "mpt_set_lr",
+           "mpt_train_step_staged", "mpt_set_scale", "mpt_set_lr", "mpt_set_dynamic_scale", "mpt_get_scale",
            "mpt_get_tensor", "mpt_set_grad", "mpt_set_momentum", "mpt_launch_count", "mpt_profile",
            "mpt_profile_read", "mpt_last_error",
            "mpt_destroy", "mpt_gemm_f16", "mpt_recast", "mpt_grad_nonfinite", "mpt_update_flat",
@@ -66,6 +66,8 @@ def lib() -> C.CDLL:
     L.mpt_train_step_staged.argtypes = [vp, C.POINTER(f32), C.POINTER(i32)]
     L.mpt_set_scale.argtypes = [vp, f32]
     L.mpt_set_lr.argtypes = [vp, f32]
+    L.mpt_set_dynamic_scale.argtypes = [vp, i32, i32, f32, f32]
+    L.mpt_get_scale.argtypes = [vp, C.POINTER(f32)]
     L.mpt_get_tensor.argtypes = [vp, i32, i32, vp, sz]
     L.mpt_set_grad.argtypes = [vp, i32, vp, sz]
     L.mpt_set_momentum.argtypes = [vp, i32, vp, sz]
@@ -208,6 +210,15 @@ class Context:
 
     def set_scale(self, S):
         _check(lib().mpt_set_scale(self._ctx, float(S)), self._ctx)
+
+    def set_dynamic_scale(self, enable, growth_interval=2000, min_scale=2.0 ** -14, max_scale=2.0 ** 24):
+        _check(lib().mpt_set_dynamic_scale(self._ctx, int(bool(enable)), int(growth_interval), float(min_scale),
+                                           float(max_scale)), self._ctx)
+
+    def get_scale(self):
+        S = C.c_float(0.0)
+        _check(lib().mpt_get_scale(self._ctx, C.byref(S)), self._ctx)
+        return float(S.value)
 
     def set_lr(self, lr):
         _check(lib().mpt_set_lr(self._ctx, float(lr)), self._ctx)

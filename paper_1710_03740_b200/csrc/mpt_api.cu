@@ -107,6 +107,10 @@ struct mpt_ctx {
     bool forward_done = false, have_grads = false, poisoned = false;
     long long launches = 0;
     bool disable_tc = false, disable_pair = false;
+    // dynamic loss scaling (off by default: constant S)
+    bool dynamic_scale = false;
+    int growth_interval = 2000;
+    float scale_backoff = 0.5f, scale_growth = 2.0f, scale_min = 0x1p-100f, scale_max = 0x1p120f;
     std::string err;
     // optional per-kernel timing with CUDA events (mpt_profile)
     bool profiling = false;
@@ -148,6 +152,20 @@ int usable(mpt_ctx *c)
 {
     if (!c) return MPT_ERR_INVALID_ARG;
     if (c->poisoned) return MPT_ERR_STATE;
+    return MPT_OK;
+}
+
+// The loss scale lives in the status block (S, 1/S, clean-step counter): kernels read it from
+// there, so it can change on the device (dynamic scaling) without a host round trip.
+int push_scale(mpt_ctx *c)
+{
+    uint32_t w[3];
+    const float inv = 1.0f / c->S;
+    memcpy(&w[0], &c->S, 4);
+    memcpy(&w[1], &inv, 4);
+    w[2] = 0;
+    CK(cudaMemcpyAsync(c->status + ST_SCALE, w, sizeof w, cudaMemcpyHostToDevice, c->stream), "scale upload");
+    CK(cudaStreamSynchronize(c->stream), "stream synchronize");
     return MPT_OK;
 }
 
@@ -239,7 +257,8 @@ int do_backward(mpt_ctx *c, const int32_t *labels_dev)
     {
         ProfSpan span(c, MPT_PROF_SOFTMAX, 4.0 * B * last.out);
         e = launch_softmax_ce(last.act, last.ld_out, labels_dev, B, last.out, c->S, last.dact, last.ld_out, c->row_loss,
-                              (float *)(c->status + ST_LOSS), c->status + ST_BAD_LABELS, c->stream, &nl);
+                              (float *)(c->status + ST_LOSS), c->status + ST_BAD_LABELS, c->stream, &nl,
+                              (const float *)(c->status + ST_SCALE));
     }
     c->launches += nl;
     if (e != cudaSuccess) return cuda_fail(c, e, "softmax launch");
@@ -271,10 +290,17 @@ int do_step(mpt_ctx *c)
     {
         ProfSpan span(c, MPT_PROF_UPDATE, (c->use_momentum ? 20.0 : 12.0) * (double)c->plan.P_pad);
         e = launch_update(c->g16, c->master, c->mom, c->w16, c->plan.P_pad, inv, c->lr, c->mu, c->use_momentum,
-                          c->status + ST_OVERFLOW, c->stream);
+                          c->status + ST_OVERFLOW, c->stream, (const float *)(c->status + ST_INV_SCALE));
     }
     c->launches++;
     if (e != cudaSuccess) return cuda_fail(c, e, "update launch");
+    if (c->dynamic_scale) {
+        ProfSpan span(c, MPT_PROF_OTHER, 0.0);
+        e = launch_scale_adjust(c->status, c->growth_interval, c->scale_backoff, c->scale_growth, c->scale_min,
+                                c->scale_max, c->stream);
+        c->launches++;
+        if (e != cudaSuccess) return cuda_fail(c, e, "scale adjust launch");
+    }
     return MPT_OK;
 }
 
@@ -349,6 +375,7 @@ int mpt_create(const mpt_layer_desc *layers, int n_layers, float S, float lr, fl
     // Parameter arenas (including the padding between layers), activations and status start at zero.
     cudaError_t e = cudaMemsetAsync(c->ws, 0, pl.total, c->stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
+    if (e == cudaSuccess && push_scale(c) != MPT_OK) e = cudaErrorUnknown;
     for (int k = 0; k < 2 && e == cudaSuccess; k++) {
         e = cudaEventCreateWithFlags(&c->staged_ev[k], cudaEventDisableTiming);
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->used_ev[k], cudaEventDisableTiming);
@@ -416,7 +443,45 @@ int mpt_set_scale(mpt_ctx *c, float S)
     if (r != MPT_OK) return r;
     if (!valid_scale(S)) return fail(c, MPT_ERR_INVALID_ARG, "loss scale out of range");
     c->S = S;
+    return push_scale(c);
+}
+
+int mpt_get_scale(mpt_ctx *c, float *S_out)
+{
+    int r = usable(c);
+    if (r != MPT_OK) return r;
+    if (!S_out) return fail(c, MPT_ERR_INVALID_ARG, "null output");
+    uint32_t st[ST_WORDS];
+    r = read_status(c, st);
+    if (r != MPT_OK) return r;
+    memcpy(S_out, &st[ST_SCALE], 4);
+    c->S = *S_out;
     return MPT_OK;
+}
+
+int mpt_set_dynamic_scale(mpt_ctx *c, int enable, int growth_interval, float min_scale, float max_scale)
+{
+    int r = usable(c);
+    if (r != MPT_OK) return r;
+    if (enable) {
+        if (growth_interval < 1) return fail(c, MPT_ERR_INVALID_ARG, "growth interval must be >= 1");
+        if (!valid_scale(min_scale) || !valid_scale(max_scale) || min_scale > max_scale)
+            return fail(c, MPT_ERR_INVALID_ARG, "scale bounds out of range");
+        c->growth_interval = growth_interval;
+        c->scale_min = min_scale;
+        c->scale_max = max_scale;
+    }
+    c->dynamic_scale = enable != 0;
+    // the counter of clean steps restarts; S itself is kept (read it back so the host copy is current)
+    float S = 0.0f;
+    r = mpt_get_scale(c, &S);
+    if (r != MPT_OK) return r;
+    if (enable) {
+        if (S < min_scale) S = min_scale;
+        if (S > max_scale) S = max_scale;
+    }
+    c->S = S;
+    return push_scale(c);
 }
 
 int mpt_set_lr(mpt_ctx *c, float lr)

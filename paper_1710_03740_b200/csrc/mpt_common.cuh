@@ -17,6 +17,9 @@ enum StatusWord : int {
     ST_BAD_LABELS = 2,    // labels outside [0, C) seen by the last softmax
     ST_KERNEL_ERR = 3,    // first device-side error (bounded wait expired): code | where<<8
     ST_LOSS = 4,          // float: unscaled mean loss of the last backward
+    ST_SCALE = 5,         // float: loss scale S the next backward / master pass will use
+    ST_INV_SCALE = 6,     // float: 1.0f / S (one FP32 division)
+    ST_CLEAN_STEPS = 7,   // consecutive steps without overflow since S last changed (dynamic scaling)
     ST_WORDS = 16
 };
 
@@ -40,11 +43,19 @@ __device__ __forceinline__ bool f32_nonfinite(float x)
 cudaError_t launch_recast(const float *w32, uint16_t *w16, size_t n, cudaStream_t st);
 cudaError_t launch_grad_nonfinite(const uint16_t *g16, size_t n, float inv_S, uint32_t *flag,
                                   cudaStream_t st);
+// inv_S_dev / S_dev (may be null): when given, the kernel reads 1/S resp. S from device memory
+// instead of taking the by-value argument (the scale can then change without a host round trip).
 cudaError_t launch_update(const uint16_t *g16, float *w32, float *v, uint16_t *w16, size_t n, float inv_S,
-                          float lr, float mu, bool use_momentum, uint32_t *flags, cudaStream_t st);
+                          float lr, float mu, bool use_momentum, uint32_t *flags, cudaStream_t st,
+                          const float *inv_S_dev = nullptr);
 cudaError_t launch_softmax_ce(const uint16_t *z, int ldz, const int32_t *labels, int B, int C, float S,
                               uint16_t *dz, int lddz, float *row_loss, float *loss, uint32_t *bad_labels,
-                              cudaStream_t st, int *n_launches);
+                              cudaStream_t st, int *n_launches, const float *S_dev = nullptr);
+// Dynamic loss scaling (one thread): on overflow S <- max(S * backoff, min_S) and the clean-step
+// counter restarts; after `interval` clean steps S <- min(S * growth, max_S).  Rewrites the
+// ST_SCALE / ST_INV_SCALE / ST_CLEAN_STEPS words of the status block.
+cudaError_t launch_scale_adjust(uint32_t *status, int interval, float backoff, float growth, float min_S,
+                                float max_S, cudaStream_t st);
 cudaError_t launch_gemm_simt(int op, int M, int N, int K, const uint16_t *A, int lda, const uint16_t *B,
                              int ldb, uint16_t *C, int ldc, bool relu, const uint16_t *mask, int ldmask,
                              uint32_t *nonfinite_flag, cudaStream_t st);

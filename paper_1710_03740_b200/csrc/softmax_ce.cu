@@ -35,9 +35,10 @@ template <bool VEC, bool CACHE>
 __global__ void __launch_bounds__(1024) k_softmax_ce(const uint16_t *__restrict__ z, int ldz,
                                                      const int32_t *__restrict__ labels, int B, int C, float c,
                                                      uint16_t *dz, int lddz, float *__restrict__ row_loss,
-                                                     uint32_t *bad_labels)
+                                                     uint32_t *bad_labels, const float *__restrict__ scale_dev)
 {
     extern __shared__ __align__(16) uint16_t srow[];
+    if (scale_dev) c = __fdiv_rn(*scale_dev, (float)B);
     __shared__ float red[32];
     const int tid = threadIdx.x, nt = blockDim.x;
     const int C8 = VEC ? (C / 8) : 0;
@@ -126,9 +127,11 @@ template <int VPT>
 __global__ void __launch_bounds__(1024) k_softmax_ce_reg(const uint16_t *__restrict__ z, int ldz,
                                                          const int32_t *__restrict__ labels, int C, float c,
                                                          uint16_t *__restrict__ dz, int lddz,
-                                                         float *__restrict__ row_loss, uint32_t *bad_labels)
+                                                         float *__restrict__ row_loss, uint32_t *bad_labels,
+                                                         const float *__restrict__ scale_dev)
 {
     __shared__ float red[32];
+    if (scale_dev) c = __fdiv_rn(*scale_dev, (float)gridDim.x);   // one CTA per row: gridDim.x is the batch
     const int tid = threadIdx.x, nt = blockDim.x, row = blockIdx.x;
     const int C8 = C >> 3, tail = C & 7;
     const uint16_t *zr = z + (size_t)row * ldz;
@@ -224,20 +227,20 @@ __global__ void __launch_bounds__(256) k_loss_mean(const float *__restrict__ row
 template <bool VEC, bool CACHE>
 static cudaError_t launch_variant(const uint16_t *z, int ldz, const int32_t *labels, int B, int C, float c,
                                   uint16_t *dz, int lddz, float *row_loss, uint32_t *bad_labels, int threads,
-                                  int grid, size_t smem, cudaStream_t st)
+                                  int grid, size_t smem, cudaStream_t st, const float *S_dev)
 {
     auto kern = k_softmax_ce<VEC, CACHE>;
     if (smem > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
     }
-    kern<<<grid, threads, smem, st>>>(z, ldz, labels, B, C, c, dz, lddz, row_loss, bad_labels);
+    kern<<<grid, threads, smem, st>>>(z, ldz, labels, B, C, c, dz, lddz, row_loss, bad_labels, S_dev);
     return cudaGetLastError();
 }
 
 cudaError_t launch_softmax_ce(const uint16_t *z, int ldz, const int32_t *labels, int B, int C, float S,
                               uint16_t *dz, int lddz, float *row_loss, float *loss, uint32_t *bad_labels,
-                              cudaStream_t st, int *n_launches)
+                              cudaStream_t st, int *n_launches, const float *S_dev)
 {
     if (n_launches) *n_launches = 0;
     if (B <= 0 || C <= 0) return cudaSuccess;
@@ -252,10 +255,10 @@ cudaError_t launch_softmax_ce(const uint16_t *z, int ldz, const int32_t *labels,
         threads = ((threads + 31) / 32) * 32;
         if (threads < 32) threads = 32;
         switch (vpt) {
-            case 1: k_softmax_ce_reg<1><<<B, threads, 0, st>>>(z, ldz, labels, C, c, dz, lddz, row_loss, bad_labels); break;
-            case 2: k_softmax_ce_reg<2><<<B, threads, 0, st>>>(z, ldz, labels, C, c, dz, lddz, row_loss, bad_labels); break;
-            case 4: k_softmax_ce_reg<4><<<B, threads, 0, st>>>(z, ldz, labels, C, c, dz, lddz, row_loss, bad_labels); break;
-            default: k_softmax_ce_reg<8><<<B, threads, 0, st>>>(z, ldz, labels, C, c, dz, lddz, row_loss, bad_labels); break;
+            case 1: k_softmax_ce_reg<1><<<B, threads, 0, st>>>(z, ldz, labels, C, c, dz, lddz, row_loss, bad_labels, S_dev); break;
+            case 2: k_softmax_ce_reg<2><<<B, threads, 0, st>>>(z, ldz, labels, C, c, dz, lddz, row_loss, bad_labels, S_dev); break;
+            case 4: k_softmax_ce_reg<4><<<B, threads, 0, st>>>(z, ldz, labels, C, c, dz, lddz, row_loss, bad_labels, S_dev); break;
+            default: k_softmax_ce_reg<8><<<B, threads, 0, st>>>(z, ldz, labels, C, c, dz, lddz, row_loss, bad_labels, S_dev); break;
         }
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
@@ -275,10 +278,10 @@ cudaError_t launch_softmax_ce(const uint16_t *z, int ldz, const int32_t *labels,
     int grid = B < 148 * 16 ? B : 148 * 16;
     size_t smem = cache ? row_bytes : 0;
     cudaError_t e;
-    if (vec && cache) e = launch_variant<true, true>(z, ldz, labels, B, C, c, dz, lddz, row_loss, bad_labels, threads, grid, smem, st);
-    else if (vec) e = launch_variant<true, false>(z, ldz, labels, B, C, c, dz, lddz, row_loss, bad_labels, threads, grid, smem, st);
-    else if (cache) e = launch_variant<false, true>(z, ldz, labels, B, C, c, dz, lddz, row_loss, bad_labels, threads, grid, smem, st);
-    else e = launch_variant<false, false>(z, ldz, labels, B, C, c, dz, lddz, row_loss, bad_labels, threads, grid, smem, st);
+    if (vec && cache) e = launch_variant<true, true>(z, ldz, labels, B, C, c, dz, lddz, row_loss, bad_labels, threads, grid, smem, st, S_dev);
+    else if (vec) e = launch_variant<true, false>(z, ldz, labels, B, C, c, dz, lddz, row_loss, bad_labels, threads, grid, smem, st, S_dev);
+    else if (cache) e = launch_variant<false, true>(z, ldz, labels, B, C, c, dz, lddz, row_loss, bad_labels, threads, grid, smem, st, S_dev);
+    else e = launch_variant<false, false>(z, ldz, labels, B, C, c, dz, lddz, row_loss, bad_labels, threads, grid, smem, st, S_dev);
     if (e != cudaSuccess) return e;
     if (n_launches) *n_launches = 1;
     if (loss) {

@@ -171,9 +171,11 @@ __device__ __forceinline__ void upd8(const uint4 &g, float4 &w0, float4 &w1, flo
 template <bool MOM>
 __global__ void __launch_bounds__(kThreads) k_update_vec(const uint4 *__restrict__ g16, float4 *__restrict__ w32,
                                                          float4 *__restrict__ v32, uint4 *__restrict__ w16, size_t n8,
-                                                         float inv, float lr, float mu, uint32_t *flags)
+                                                         float inv, float lr, float mu, uint32_t *flags,
+                                                         const float *__restrict__ inv_dev)
 {
     if (*(volatile const uint32_t *)flags != 0u) return;
+    if (inv_dev) inv = *inv_dev;
     const size_t base = (size_t)blockIdx.x * (kThreads * kVecPerThread) + threadIdx.x;
     bool bad = false;
     uint4 g[kVecPerThread];
@@ -205,9 +207,10 @@ __global__ void __launch_bounds__(kThreads) k_update_vec(const uint4 *__restrict
 template <bool MOM>
 __global__ void k_update_scalar(const uint16_t *__restrict__ g16, float *__restrict__ w32, float *__restrict__ v32,
                                 uint16_t *__restrict__ w16, size_t begin, size_t n, float inv, float lr, float mu,
-                                uint32_t *flags)
+                                uint32_t *flags, const float *__restrict__ inv_dev)
 {
     if (*(volatile const uint32_t *)flags != 0u) return;
+    if (inv_dev) inv = *inv_dev;
     size_t stride = (size_t)gridDim.x * blockDim.x;
     bool bad = false;
     for (size_t i = begin + (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
@@ -221,7 +224,7 @@ __global__ void k_update_scalar(const uint16_t *__restrict__ g16, float *__restr
 }
 
 cudaError_t launch_update(const uint16_t *g16, float *w32, float *v, uint16_t *w16, size_t n, float inv_S, float lr,
-                          float mu, bool use_momentum, uint32_t *flags, cudaStream_t st)
+                          float mu, bool use_momentum, uint32_t *flags, cudaStream_t st, const float *inv_S_dev)
 {
     if (n == 0) return cudaSuccess;
     uintptr_t bits = (uintptr_t)g16 | (uintptr_t)w32 | (uintptr_t)w16 | (use_momentum ? (uintptr_t)v : 0);
@@ -231,18 +234,47 @@ cudaError_t launch_update(const uint16_t *g16, float *w32, float *v, uint16_t *w
         const unsigned grid = (unsigned)((n8 + per_cta - 1) / per_cta);
         if (use_momentum)
             k_update_vec<true><<<grid, kThreads, 0, st>>>((const uint4 *)g16, (float4 *)w32, (float4 *)v, (uint4 *)w16,
-                                                          n8, inv_S, lr, mu, flags);
+                                                          n8, inv_S, lr, mu, flags, inv_S_dev);
         else
             k_update_vec<false><<<grid, kThreads, 0, st>>>((const uint4 *)g16, (float4 *)w32, nullptr, (uint4 *)w16, n8,
-                                                           inv_S, lr, mu, flags);
+                                                           inv_S, lr, mu, flags, inv_S_dev);
     }
     if (n8 * 8 < n) {
         int grid = grid_for(n - n8 * 8);
         if (use_momentum)
-            k_update_scalar<true><<<grid, kThreads, 0, st>>>(g16, w32, v, w16, n8 * 8, n, inv_S, lr, mu, flags);
+            k_update_scalar<true><<<grid, kThreads, 0, st>>>(g16, w32, v, w16, n8 * 8, n, inv_S, lr, mu, flags, inv_S_dev);
         else
-            k_update_scalar<false><<<grid, kThreads, 0, st>>>(g16, w32, nullptr, w16, n8 * 8, n, inv_S, lr, mu, flags);
+            k_update_scalar<false><<<grid, kThreads, 0, st>>>(g16, w32, nullptr, w16, n8 * 8, n, inv_S, lr, mu, flags, inv_S_dev);
     }
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------- dynamic loss scale
+
+// The paper's closing section proposes raising or lowering the scale by inspecting the weight
+// gradients for overflow while skipping the overflowing updates; it gives no schedule.  Taken
+// here: multiply by `backoff` on overflow, by `growth` after `interval` clean steps in a row,
+// clamp to [min_S, max_S].  With power-of-two factors every scale stays a power of two.
+__global__ void k_scale_adjust(uint32_t *status, int interval, float backoff, float growth, float min_S, float max_S)
+{
+    float S = __uint_as_float(status[ST_SCALE]);
+    uint32_t clean = status[ST_CLEAN_STEPS];
+    if (status[ST_OVERFLOW] != 0u) {
+        S = fmaxf(__fmul_rn(S, backoff), min_S);
+        clean = 0;
+    } else if (++clean >= (uint32_t)interval) {
+        S = fminf(__fmul_rn(S, growth), max_S);
+        clean = 0;
+    }
+    status[ST_SCALE] = __float_as_uint(S);
+    status[ST_INV_SCALE] = __float_as_uint(__fdiv_rn(1.0f, S));
+    status[ST_CLEAN_STEPS] = clean;
+}
+
+cudaError_t launch_scale_adjust(uint32_t *status, int interval, float backoff, float growth, float min_S, float max_S,
+                                cudaStream_t st)
+{
+    k_scale_adjust<<<1, 1, 0, st>>>(status, interval, backoff, growth, min_S, max_S);
     return cudaGetLastError();
 }
 

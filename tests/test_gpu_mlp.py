@@ -202,6 +202,71 @@ def test_staged_pipeline_matches_plain_host_steps():
     cs.synchronize()
 
 
+def test_dynamic_scale_hand_trace_on_device():
+    """The schedule pinned by hand for the oracle (interval 3, bounds [2, 64], start 16), on the device:
+    the scale lives in device memory and is adjusted at the end of mpt_step."""
+    from paper_1710_03740_b200 import binding as b
+    net = b.Context([(1, 1, 0)], 16.0, 0.5, 0.0, 1)
+    net.set_master(0, np.array([[1.0]], dtype=np.float32))
+    net.set_dynamic_scale(True, 3, 2.0, 64.0)
+    inf, ok = np.float16(np.inf), np.float16(16.0)
+    seq = [ok, ok, ok, ok, inf, ok, ok, inf, inf, inf, inf, ok, ok, ok, ok, ok, ok, ok, ok, ok]
+    want_S_after = [16, 16, 32, 32, 16, 16, 16, 8, 4, 2, 2, 2, 2, 4, 4, 4, 8, 8, 8, 16]
+    want_flag = [0, 0, 0, 0, 1, 0, 0, 1, 1, 1, 1, 0, 0, 0, 0, 0, 0, 0, 0, 0]
+    ora = OracleMLP([(1, 1, 0)], 16.0, 0.5, 0.0)
+    ora.set_master(0, np.array([[1.0]], dtype=np.float32))
+    ora.set_dynamic_scale(3, 2.0, 64.0)
+    for t, g in enumerate(seq):
+        net.set_grad(0, np.array([[g]], dtype=np.float16))
+        ora.set_grad(0, np.array([[g]], dtype=np.float16))
+        assert net.step() == ora.step() == want_flag[t]
+        assert net.get_scale() == float(ora.S) == want_S_after[t]
+        assert net.get_master(0).tobytes() == ora.w32[0].tobytes()
+    net.set_dynamic_scale(False)
+    assert net.get_scale() == 16.0
+
+
+def test_dynamic_scale_recovers_from_overflowing_start():
+    """Scale-sweep network started at S = 2^24 with dynamic scaling: same skip sequence, same
+    scales and (within 1e-3) same losses as the oracle; no host synchronisation inside a step."""
+    from paper_1710_03740_b200 import binding as b
+    cfg = inputs.MLP_CONFIGS["scale_sweep"]
+    masters = inputs.mlp_masters(cfg)
+    steps = 12
+    X, Y = inputs.mlp_batches(cfg, steps)
+    net, ora = _make(cfg, 2.0 ** 24, masters)
+    net.set_dynamic_scale(True, 4, 1.0, 2.0 ** 24)
+    ora.set_dynamic_scale(4, 1.0, 2.0 ** 24)
+    xs = [dev(X[t].view(np.uint16)) for t in range(steps)]
+    ys = [dev(Y[t]) for t in range(steps)]
+    flags_o, scales_o, losses_o = [], [], []
+    for t in range(steps):
+        ora.forward(X[t])
+        losses_o.append(ora.backward_scaled(Y[t]))
+        flags_o.append(ora.step())
+        scales_o.append(float(ora.S))
+    flags_g, scales_g, losses_g = [], [], []
+    for t in range(steps):
+        net.forward(xs[t])
+        losses_g.append(net.backward_scaled(ys[t]))
+        flags_g.append(net.step())
+        scales_g.append(net.get_scale())
+    assert flags_g == flags_o and scales_g == scales_o
+    assert flags_o[0] == 1 and 0 in flags_o and max(scales_o) > min(scales_o)
+    for a, c in zip(losses_g, losses_o):
+        assert abs(a - c) <= 1e-3 * abs(c)
+    # fully asynchronous use: no host read between steps, then one check at the end
+    net2, _ = _make(cfg, 2.0 ** 24, masters)
+    net2.set_dynamic_scale(True, 4, 1.0, 2.0 ** 24)
+    for t in range(steps):
+        net2.forward(xs[t])
+        net2.backward_scaled(ys[t], want_loss=False)
+        net2.step(want_flag=False)
+    assert net2.get_scale() == scales_o[-1]
+    for l in range(len(masters)):
+        assert net2.get_master(l).tobytes() == net.get_master(l).tobytes()
+
+
 def test_error_paths():
     from paper_1710_03740_b200 import binding as b
     cfg = inputs.MLP_CONFIGS["tiny"]

@@ -646,6 +646,69 @@ def test_overflowing_scale_skips_every_step_twin():
     assert losses[-1] < losses[0]
 
 
+def test_dynamic_scale_schedule_hand_trace():
+    """Dynamic loss scaling (paper section 5: raise or lower the factor by inspecting the weight
+    gradients for overflow, skipping overflowing updates).  One weight, injected gradients: the
+    scale after each step is worked out by hand for interval 3, bounds [2, 64], start 16."""
+    net = OracleMLP([(1, 1, 0)], 16.0, 0.5, 0.0)
+    net.set_master(0, np.array([[1.0]], dtype=np.float32))
+    net.set_dynamic_scale(3, 2.0, 64.0)
+    inf, ok = np.float16(np.inf), np.float16(16.0)          # 16/S is the unscaled gradient
+    seq = [ok, ok, ok, ok, inf, ok, ok, inf, inf, inf, inf, ok, ok, ok, ok, ok, ok, ok, ok, ok]
+    # S used by each step:    16  16  16  32  32   16  16  16   8    4    2   2   2   2   4   4   4   8   8   8
+    want_S_after = [16, 16, 32, 32, 16, 16, 16, 8, 4, 2, 2, 2, 2, 4, 4, 4, 8, 8, 8, 16]
+    want_flag = [0, 0, 0, 0, 1, 0, 0, 1, 1, 1, 1, 0, 0, 0, 0, 0, 0, 0, 0, 0]
+    w = 1.0
+    for t, g in enumerate(seq):
+        S_used = float(net.S)
+        net.set_grad(0, np.array([[g]], dtype=np.float16))
+        flag = net.step()
+        assert flag == want_flag[t] and float(net.S) == want_S_after[t], (t, flag, float(net.S))
+        if not flag:
+            w = float(np.float32(w) - np.float32(0.5) * np.float32(16.0 / S_used))
+        assert float(net.w32[0][0, 0]) == w                 # skipped steps leave the master alone
+    # clamp at the upper bound
+    net2 = OracleMLP([(1, 1, 0)], 32.0, 0.5, 0.0)
+    net2.set_master(0, np.array([[1.0]], dtype=np.float32))
+    net2.set_dynamic_scale(1, 2.0, 64.0)
+    for want in (64, 64, 64):
+        net2.set_grad(0, np.array([[1.0]], dtype=np.float16))
+        net2.step()
+        assert float(net2.S) == want
+
+
+def test_dynamic_scale_recovers_from_an_overflowing_start():
+    """Twin of the scale-sweep network started at S = 2^24 (overflows, section 3.2): the scale
+    backs off until steps go through, no skipped step moves the master, and from then on the
+    run is bit-identical to a constant-scale run started at the settled scale from the same
+    masters (power-of-two scales only change exponents)."""
+    cfg = dict(inputs.MLP_CONFIGS["scale_sweep_twin"])
+    masters = inputs.mlp_masters(cfg)
+    X, Y = inputs.mlp_batches(cfg, 12)
+    net = OracleMLP(cfg["layers"], 2.0 ** 24, cfg["lr"], cfg["momentum"])
+    for l, w in enumerate(masters):
+        net.set_master(l, w)
+    net.set_dynamic_scale(1000, 1.0, 2.0 ** 24)
+    flags, scales = [], []
+    for t in range(12):
+        net.forward(X[t])
+        net.backward_scaled(Y[t])
+        scales.append(float(net.S))
+        flags.append(net.step())
+    n_skip = flags.index(0)
+    assert n_skip >= 1 and flags[:n_skip] == [1] * n_skip and flags[n_skip:] == [0] * (12 - n_skip)
+    assert scales[:n_skip + 1] == [2.0 ** (24 - i) for i in range(n_skip + 1)]
+    ref = OracleMLP(cfg["layers"], scales[n_skip], cfg["lr"], cfg["momentum"])
+    for l, w in enumerate(masters):
+        ref.set_master(l, w)
+    for t in range(n_skip, 12):
+        ref.forward(X[t])
+        ref.backward_scaled(Y[t])
+        assert ref.step() == 0
+    for l in range(len(masters)):
+        assert ref.w32[l].tobytes() == net.w32[l].tobytes()
+
+
 def test_tiny_config_trains():
     cfg = inputs.MLP_CONFIGS["tiny"]
     net, flags, losses, _ = _run(cfg, cfg["S"], cfg["steps"])
