@@ -16,6 +16,10 @@
 //   empty[s]  in each CTA: tcgen05.commit multicast to both CTAs when the MMAs have read stage s
 //   accf[b]   in each CTA: tcgen05.commit multicast when a tile's accumulator is complete
 //   acce[b]   in the leader: 8 arrivals, one per epilogue warp of both CTAs
+// Work units: every cluster first takes the same number of full 256x256 tiles; the tiles left
+// over for a last, partly filled round are cut into two 256x128 halves when that lets every
+// half run at once (the last round then takes about half as long).  A half unit is the same
+// pipeline with 64 columns of B per CTA and N = 128 instructions.
 // No TMA multicast is used.  Every mbarrier wait is bounded (see tc_ptx.cuh).
 #include <cuda.h>
 
@@ -40,10 +44,10 @@ static constexpr int TMEM_COLS = 512;
 static constexpr int NUM_THREADS = 192;
 static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256;
 
+// instruction descriptor without the N field (N >> 3 goes to bits 17..22)
 __host__ __device__ constexpr uint32_t make_idesc(bool a_mn, bool b_mn)
 {
-    return (1u << 4) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) | ((uint32_t)(TILE_N >> 3) << 17) |
-           ((uint32_t)((2 * CTA_M) >> 4) << 24);
+    return (1u << 4) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) | ((uint32_t)((2 * CTA_M) >> 4) << 24);
 }
 
 struct Params {
@@ -56,6 +60,13 @@ struct Params {
     uint32_t *nonfinite_flag;
     uint32_t *status;
     int tiles_m, tiles_n, group_m;   // pair tiles (256 rows x 256 columns)
+    int full_units, num_units;       // units [0, full_units) are whole tiles, the rest are half tiles
+};
+
+struct Unit {
+    int mb, nb;      // tile coordinates
+    int n_off;       // first column of the unit inside its tile (0 or 128)
+    int width;       // 256 (whole tile) or 128 (half)
 };
 
 __device__ __forceinline__ void tile_coords(const Params &p, int tile, int &mb, int &nb)
@@ -69,6 +80,22 @@ __device__ __forceinline__ void tile_coords(const Params &p, int tile, int &mb, 
     nb = r / gsz;
 }
 
+__device__ __forceinline__ Unit unit_of(const Params &p, int u)
+{
+    Unit w;
+    int tile = u;
+    w.n_off = 0;
+    w.width = TILE_N;
+    if (u >= p.full_units) {
+        const int h = u - p.full_units;
+        tile = p.full_units + (h >> 1);
+        w.n_off = (h & 1) * (TILE_N / 2);
+        w.width = TILE_N / 2;
+    }
+    tile_coords(p, tile, w.mb, w.nb);
+    return w;
+}
+
 __device__ __forceinline__ void report(const Params &p, volatile uint32_t *abort_flag, uint32_t code)
 {
     *abort_flag = 1u;
@@ -77,7 +104,8 @@ __device__ __forceinline__ void report(const Params &p, volatile uint32_t *abort
 
 template <bool A_MN, bool B_MN>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const Params p)
+k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+           const __grid_constant__ CUtensorMap tmBh, const Params p)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -94,7 +122,7 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
     const uint32_t rank = cluster_ctarank();       // 0 = leader of the pair
     const bool leader = rank == 0;
     const int pair_id = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
-    const int num_tiles = p.tiles_m * p.tiles_n;
+    const int num_units = p.num_units;
     const int nkb = (p.K + BLOCK_K - 1) / BLOCK_K;
 
     if (threadIdx.x == 0) {
@@ -121,11 +149,12 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
         if (lane == 0) {
             uint32_t issued = 0, s = 0, ph = 0;
             bool ok = true;
-            for (int tile = pair_id; tile < num_tiles && ok; tile += num_pairs) {
-                int mb, nb;
-                tile_coords(p, tile, mb, nb);
-                const int m0 = mb * (2 * CTA_M) + (int)rank * CTA_M;      // this CTA's rows of A
-                const int n0 = nb * TILE_N + (int)rank * CTA_N;           // this CTA's columns of B
+            for (int u = pair_id; u < num_units && ok; u += num_pairs) {
+                const Unit w = unit_of(p, u);
+                const int cta_n = w.width >> 1;                            // columns of B this CTA loads
+                const int m0 = w.mb * (2 * CTA_M) + (int)rank * CTA_M;    // this CTA's rows of A
+                const int n0 = w.nb * TILE_N + w.n_off + (int)rank * cta_n;
+                const uint32_t tx_bytes = 2u * (uint32_t)(A_STAGE_BYTES + cta_n * BLOCK_K * 2);
                 for (int kb = 0; kb < nkb; kb++, issued++, s = (s + 1 == STAGES) ? 0 : s + 1, ph ^= (s == 0)) {
                     if (!mbar_try_wait(empty_bar(s), ph ^ 1u) && !mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) {
                         if (!*abort_flag) report(p, abort_flag, KERR_WAIT_EMPTY);
@@ -134,7 +163,7 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
                     }
                     const uint32_t sa = base + s * STAGE_BYTES, sb = sa + A_STAGE_BYTES;
                     const uint32_t lead_full = mapa_u32(full_bar(s), 0);
-                    if (leader) mbar_arrive_expect_tx(full_bar(s), 2 * STAGE_BYTES);
+                    if (leader) mbar_arrive_expect_tx(full_bar(s), tx_bytes);
                     const int k0 = kb * BLOCK_K;
                     if (A_MN) {
 #pragma unroll
@@ -143,10 +172,10 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
                         tma_load_2d_pair(sa, &tmA, k0, m0, lead_full);
                     }
                     if (B_MN) {
-#pragma unroll
-                        for (int j = 0; j < CTA_N / 64; j++) tma_load_2d_pair(sb + j * MN_BOX_BYTES, &tmB, n0 + 64 * j, k0, lead_full);
+                        tma_load_2d_pair(sb, &tmB, n0, k0, lead_full);
+                        if (cta_n == CTA_N) tma_load_2d_pair(sb + MN_BOX_BYTES, &tmB, n0 + 64, k0, lead_full);
                     } else {
-                        tma_load_2d_pair(sb, &tmB, k0, n0, lead_full);
+                        tma_load_2d_pair(sb, cta_n == CTA_N ? &tmB : &tmBh, k0, n0, lead_full);
                     }
                 }
             }
@@ -162,7 +191,7 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
     } else if (warp == 1) {
         // -------------------------------------------------------------- MMA issuer (leader only)
         if (leader && lane == 0) {
-            constexpr uint32_t idesc = make_idesc(A_MN, B_MN);
+            constexpr uint32_t idesc_base = make_idesc(A_MN, B_MN);
             // descriptor halves: only the start address (low word) changes with stage and k
             constexpr uint32_t KSTEP_A = (A_MN ? UMMA_K * 128 : UMMA_K * 2) >> 4;
             constexpr uint32_t KSTEP_B = (B_MN ? UMMA_K * 128 : UMMA_K * 2) >> 4;
@@ -172,7 +201,8 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
             uint32_t s = 0, ph = 0;
             bool ok = true;
             int t = 0;
-            for (int tile = pair_id; tile < num_tiles && ok; tile += num_pairs, t++) {
+            for (int u = pair_id; u < num_units && ok; u += num_pairs, t++) {
+                const uint32_t idesc = idesc_base | ((uint32_t)((u < p.full_units ? TILE_N : TILE_N / 2) >> 3) << 17);
                 const int buf = t & 1;
                 const uint32_t acc_ph = (t >> 1) & 1u;
                 if (!mbar_try_wait(acce_bar(buf), acc_ph ^ 1u) && !mbar_wait(acce_bar(buf), acc_ph ^ 1u, abort_flag)) {
@@ -208,9 +238,8 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
         const int q = warp & 3;
         bool ok = true;
         int t = 0;
-        for (int tile = pair_id; tile < num_tiles && ok; tile += num_pairs, t++) {
-            int mb, nb;
-            tile_coords(p, tile, mb, nb);
+        for (int u = pair_id; u < num_units && ok; u += num_pairs, t++) {
+            const Unit w = unit_of(p, u);
             const int buf = t & 1;
             const uint32_t acc_ph = (t >> 1) & 1u;
             const bool got = mbar_wait(accf_bar(buf), acc_ph, abort_flag);
@@ -220,17 +249,17 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
                 break;
             }
             tc_fence_after();
-            const int row = mb * (2 * CTA_M) + (int)rank * CTA_M + q * 32 + lane;
+            const int row = w.mb * (2 * CTA_M) + (int)rank * CTA_M + q * 32 + lane;
             const bool row_ok = row < p.M;
             uint16_t *crow = p.C + (size_t)row * p.ldc;
             const uint16_t *mrow = p.mask ? p.mask + (size_t)row * p.ldmask : nullptr;
             bool bad = false;
 #pragma unroll 1
-            for (int c = 0; c < TILE_N / 32; c++) {
+            for (int c = 0; c < w.width / 32; c++) {
                 uint32_t r[32];
                 tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * TILE_N + c * 32), r);
                 tc_wait_ld();
-                const int col0 = nb * TILE_N + c * 32;
+                const int col0 = w.nb * TILE_N + w.n_off + c * 32;
                 if (row_ok && col0 < p.N) epilogue_store32(r, crow, mrow, col0, p.N, p.relu != 0, bad);
             }
             tc_fence_before();
@@ -252,7 +281,7 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
 }
 
 template <bool A_MN, bool B_MN>
-static cudaError_t launch_variant(const CUtensorMap &ta, const CUtensorMap &tb, const Params &p, int pairs_wanted,
+static cudaError_t launch_variant(const CUtensorMap &ta, const CUtensorMap &tb, const CUtensorMap &tbh, Params p,
                                   cudaStream_t st)
 {
     static bool configured = false;
@@ -280,9 +309,21 @@ static cudaError_t launch_variant(const CUtensorMap &ta, const CUtensorMap &tb, 
         max_pairs = n < 74 ? n : 74;
         configured = true;
     }
-    int pairs = pairs_wanted < max_pairs ? pairs_wanted : max_pairs;
-    cfg.gridDim = dim3(2 * pairs, 1, 1);
-    return cudaLaunchKernelEx(&cfg, kern, ta, tb, p);
+    // every cluster takes tiles / pairs whole tiles; what is left over is cut into halves when all
+    // halves fit into one round
+    const int tiles = p.tiles_m * p.tiles_n;
+    const int pairs = tiles < max_pairs ? tiles : max_pairs;
+    const int full = (tiles / pairs) * pairs, rest = tiles - full;
+    if (rest > 0 && 2 * rest <= max_pairs) {
+        p.full_units = full;
+        p.num_units = full + 2 * rest;
+    } else {
+        p.full_units = tiles;
+        p.num_units = tiles;
+    }
+    const int grid_pairs = p.num_units < max_pairs ? p.num_units : max_pairs;
+    cfg.gridDim = dim3(2 * grid_pairs, 1, 1);
+    return cudaLaunchKernelEx(&cfg, kern, ta, tb, tbh, p);
 }
 
 }  // namespace pair
@@ -301,12 +342,18 @@ cudaError_t launch_gemm_tc2(int op, int M, int N, int K, const uint16_t *A, int 
                             uint32_t *status, cudaStream_t st)
 {
     using namespace pair;
-    CUtensorMap ta, tb;
+    CUtensorMap ta, tb, tbh;
     bool ok;
     if (op == MPT_OP_WGRAD) ok = tc_encode_map(&ta, A, (uint64_t)K, (uint64_t)M, (uint64_t)lda, 64, BLOCK_K);
     else ok = tc_encode_map(&ta, A, (uint64_t)M, (uint64_t)K, (uint64_t)lda, BLOCK_K, CTA_M);
-    if (op == MPT_OP_FWD) ok = ok && tc_encode_map(&tb, B, (uint64_t)N, (uint64_t)K, (uint64_t)ldb, BLOCK_K, CTA_N);
-    else ok = ok && tc_encode_map(&tb, B, (uint64_t)K, (uint64_t)N, (uint64_t)ldb, 64, BLOCK_K);
+    if (op == MPT_OP_FWD) {
+        // K-major B: one box of 128 rows per CTA for whole tiles, of 64 rows for half tiles
+        ok = ok && tc_encode_map(&tb, B, (uint64_t)N, (uint64_t)K, (uint64_t)ldb, BLOCK_K, CTA_N);
+        ok = ok && tc_encode_map(&tbh, B, (uint64_t)N, (uint64_t)K, (uint64_t)ldb, BLOCK_K, CTA_N / 2);
+    } else {
+        ok = ok && tc_encode_map(&tb, B, (uint64_t)K, (uint64_t)N, (uint64_t)ldb, 64, BLOCK_K);
+        tbh = tb;
+    }
     if (!ok) return cudaErrorInvalidValue;
     Params p;
     p.M = M; p.N = N; p.K = K;
@@ -318,10 +365,10 @@ cudaError_t launch_gemm_tc2(int op, int M, int N, int K, const uint16_t *A, int 
     p.tiles_m = (M + 2 * CTA_M - 1) / (2 * CTA_M);
     p.tiles_n = (N + TILE_N - 1) / TILE_N;
     p.group_m = 8;
-    int tiles = p.tiles_m * p.tiles_n;
-    if (op == MPT_OP_FWD) return launch_variant<false, false>(ta, tb, p, tiles, st);
-    if (op == MPT_OP_DGRAD) return launch_variant<false, true>(ta, tb, p, tiles, st);
-    return launch_variant<true, true>(ta, tb, p, tiles, st);
+    p.full_units = p.num_units = 0;
+    if (op == MPT_OP_FWD) return launch_variant<false, false>(ta, tb, tbh, p, st);
+    if (op == MPT_OP_DGRAD) return launch_variant<false, true>(ta, tb, tbh, p, st);
+    return launch_variant<true, true>(ta, tb, tbh, p, st);
 }
 
 }  // namespace mpt

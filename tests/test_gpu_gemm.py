@@ -135,6 +135,14 @@ def test_pair_kernel_runs_many_tiles_per_cluster():
     _check_tc(2, 2304, 3072, 136, kernel="pair")
 
 
+@pytest.mark.parametrize("op", [0, 1, 2])
+@pytest.mark.parametrize("M,N,K", [(1280, 4000, 136), (1280, 3944, 72), (2304, 3072, 200)])
+def test_pair_kernel_half_width_tail_units(op, M, N, K):
+    """A few more tiles than clusters: the left-over tiles run as two 256x128 halves, including
+    halves that are partly or wholly outside a ragged N."""
+    _check_tc(op, M, N, K, kernel="pair")
+
+
 @pytest.mark.parametrize("kernel", ["tc", "pair"])
 def test_tc_gemm_relu_mask_flag_subnormals(kernel):
     from paper_1710_03740_b200 import binding as b
