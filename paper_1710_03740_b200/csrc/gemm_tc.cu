@@ -302,13 +302,15 @@ template <bool A_MN, bool B_MN, int BN>
 static cudaError_t launch_variant(const CUtensorMap &ta, const CUtensorMap &tb, const TcParams &p, int grid,
                                   cudaStream_t st)
 {
-    static bool configured = false;
+    static bool configured[kMaxDevices] = {};
     constexpr int SMEM_BYTES = TileCfg<BN>::SMEM_BYTES;
     auto kern = k_gemm_tc<A_MN, B_MN, BN>;
-    if (!configured) {
+    const int dev = current_device_slot();
+    if (dev < 0) return cudaErrorInvalidDevice;
+    if (!configured[dev]) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
         if (e != cudaSuccess) return e;
-        configured = true;
+        configured[dev] = true;
     }
     kern<<<grid, NUM_THREADS, SMEM_BYTES, st>>>(ta, tb, p);
     return cudaGetLastError();

@@ -284,9 +284,10 @@ template <bool A_MN, bool B_MN>
 static cudaError_t launch_variant(const CUtensorMap &ta, const CUtensorMap &tb, const CUtensorMap &tbh, Params p,
                                   cudaStream_t st)
 {
-    static bool configured = false;
-    static int max_pairs = 0;
+    static int max_pairs_dev[kMaxDevices] = {};     // 0 = this device not configured yet
     auto kern = k_gemm_tc2<A_MN, B_MN>;
+    const int dev = current_device_slot();
+    if (dev < 0) return cudaErrorInvalidDevice;
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -298,7 +299,7 @@ static cudaError_t launch_variant(const CUtensorMap &ta, const CUtensorMap &tb, 
     cfg.stream = st;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (!configured) {
+    if (max_pairs_dev[dev] == 0) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
         if (e != cudaSuccess) return e;
         cfg.gridDim = dim3(148, 1, 1);
@@ -306,9 +307,9 @@ static cudaError_t launch_variant(const CUtensorMap &ta, const CUtensorMap &tb, 
         e = cudaOccupancyMaxActiveClusters(&n, kern, &cfg);
         if (e != cudaSuccess) return e;
         if (n < 1) return cudaErrorLaunchOutOfResources;
-        max_pairs = n < 74 ? n : 74;
-        configured = true;
+        max_pairs_dev[dev] = n < 74 ? n : 74;
     }
+    const int max_pairs = max_pairs_dev[dev];
     // every cluster takes tiles / pairs whole tiles; what is left over is cut into halves when all
     // halves fit into one round
     const int tiles = p.tiles_m * p.tiles_n;

@@ -33,6 +33,16 @@ enum KernelErr : uint32_t {
     KERR_TMEM_ALLOC = 5
 };
 
+// Kernel attributes (opt-in shared memory size, cluster occupancy) are per device: launchers
+// keep one "configured" slot per device ordinal.
+static constexpr int kMaxDevices = 64;
+inline int current_device_slot()
+{
+    int d = 0;
+    if (cudaGetDevice(&d) != cudaSuccess || d < 0 || d >= kMaxDevices) return -1;
+    return d;
+}
+
 __device__ __forceinline__ bool half_bits_nonfinite(uint32_t h) { return (h & 0x7C00u) == 0x7C00u; }
 __device__ __forceinline__ bool f32_nonfinite(float x)
 {

@@ -305,8 +305,7 @@ cudaError_t launch_softmax_ce(const uint16_t *z, int ldz, const int32_t *labels,
 static __device__ __align__(256) float g_static_row_loss[MPT_SOFTMAX_STATIC_MAX_ROWS];
 
 namespace {
-constexpr int kMaxDevices = 64;
-float *g_static_ptr[kMaxDevices];   // per device, filled on the first call made with that device current
+float *g_static_ptr[mpt::kMaxDevices];   // per device, filled on the first call made with that device current
 }  // namespace
 
 extern "C" int mpt_softmax_ce_static(const uint16_t *z_dev, int ldz, const int32_t *labels_dev, int B, int C, float S,
@@ -319,7 +318,7 @@ extern "C" int mpt_softmax_ce_static(const uint16_t *z_dev, int ldz, const int32
     if (z_dev == dz_dev) return MPT_ERR_INVALID_ARG;
     int device = -1;
     if (cudaGetDevice(&device) != cudaSuccess) return MPT_ERR_CUDA;
-    if (device < 0 || device >= kMaxDevices) return MPT_ERR_INTERNAL;
+    if (device < 0 || device >= mpt::kMaxDevices) return MPT_ERR_INTERNAL;
     if (!g_static_ptr[device]) {
         float *p = nullptr;
         if (cudaGetSymbolAddress((void **)&p, g_static_row_loss) != cudaSuccess || !p) return MPT_ERR_CUDA;

@@ -4,6 +4,7 @@ sweep, the bigLSTM-shaped products, the master-update pass and the softmax cross
     python -m paper_1710_03740_b200.kernel_bench gemm   [--shape MxNxK ...] [--op 0 1 2] [--iters 20]
     python -m paper_1710_03740_b200.kernel_bench update [--params N] [--momentum 0|1] [--iters 20]
     python -m paper_1710_03740_b200.kernel_bench softmax [--rows B] [--classes C] [--iters 20]
+    python -m paper_1710_03740_b200.kernel_bench step    [--workload tiny|scale_sweep|large_twin] [--iters 50]
 
 Prints one JSON line per case: best-of and back-to-back ("sustained") rates.  Working sets
 are larger than the 126 MB L2 unless the shape itself is smaller; small cases say so.
@@ -99,6 +100,50 @@ def bench_softmax(B, Cn, iters):
             "best_gbs": by / best / 1e6, "sustained_gbs": by / sus / 1e6, "loss": float(loss.item())}
 
 
+def bench_step(workload, iters):
+    """Latency of one whole iteration (forward, scaled backward, master pass) of a small
+    configuration: calls issued one by one, and the same calls replayed from a CUDA graph."""
+    import numpy as np
+    cfg = inputs.MLP_CONFIGS[workload]
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        net = mpt.Context(cfg["layers"], cfg["S"], cfg["lr"], cfg["momentum"], cfg["batch"], stream=side)
+        for l, w in enumerate(inputs.mlp_masters(cfg)):
+            net.set_master(l, w)
+        X, Y = inputs.mlp_batches(cfg, 1)
+        x = torch.from_numpy(X[0].view(np.int16)).cuda()
+        y = torch.from_numpy(Y[0]).cuda()
+
+        def one():
+            net.forward(x)
+            net.backward_scaled(y, want_loss=False)
+            net.step(want_flag=False)
+
+        def timed(fn):
+            for _ in range(5):
+                fn()
+            side.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(side)
+            for _ in range(iters):
+                fn()
+            e1.record(side)
+            side.synchronize()
+            return e0.elapsed_time(e1) / iters * 1e3
+
+        n0 = net.launch_count()
+        one()
+        launches = net.launch_count() - n0
+        eager_us = timed(one)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            one()
+        graph_us = timed(graph.replay)
+    fl = sum(2.0 * cfg["batch"] * i * o * (2 if l == 0 else 3) for l, (i, o, _) in enumerate(cfg["layers"]))
+    return {"kernel": "step", "workload": workload, "kernel_launches": launches, "eager_us": eager_us,
+            "graph_us": graph_us, "gflop_per_step": fl / 1e9, "graph_tflops": fl / graph_us / 1e6}
+
+
 def main():
     ap = argparse.ArgumentParser()
     sub = ap.add_subparsers(dest="cmd", required=True)
@@ -117,8 +162,13 @@ def main():
     s.add_argument("--rows", type=int, default=4096)
     s.add_argument("--classes", type=int, default=32000)
     s.add_argument("--iters", type=int, default=20)
+    t = sub.add_parser("step")
+    t.add_argument("--workload", default="tiny", choices=["tiny", "scale_sweep", "scale_sweep_twin", "large_twin"])
+    t.add_argument("--iters", type=int, default=50)
     args = ap.parse_args()
-    if args.cmd == "gemm":
+    if args.cmd == "step":
+        print(json.dumps(bench_step(args.workload, args.iters)), flush=True)
+    elif args.cmd == "gemm":
         shapes = ([tuple(int(x) for x in t.split("x")) for t in args.shape] if args.shape
                   else inputs.GEMM_SWEEP + [inputs.LSTM_GATE, inputs.LSTM_PROJ])
         for (M, N, K) in shapes:

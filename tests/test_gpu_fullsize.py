@@ -142,8 +142,9 @@ def test_large_mlp_step_teacher_forced():
         w16_host.append(w)                                   # masters are FP16-representable at t = 0
     X, Y = inputs.mlp_batches(cfg, 1)
     x16 = X[0].view(np.uint16)
-    net.forward(dev(x16))
-    loss = net.backward_scaled(dev(Y[0]))
+    x_dev, y_dev = dev(x16), dev(Y[0])          # must stay alive until the backward pass has run
+    net.forward(x_dev)
+    loss = net.backward_scaled(y_dev)
     B = cfg["batch"]
 
     # forward products, layer by layer, from the activations the device actually consumed

@@ -267,6 +267,50 @@ def test_dynamic_scale_recovers_from_overflowing_start():
         assert net2.get_master(l).tobytes() == net.get_master(l).tobytes()
 
 
+def test_step_replayed_from_a_cuda_graph_matches_eager():
+    """The three calls of an iteration only enqueue work on the context's stream, so a caller can
+    record them once in a CUDA graph and replay it per batch (launch-bound small configs)."""
+    cfg = inputs.MLP_CONFIGS["tiny"]
+    masters = inputs.mlp_masters(cfg)
+    X, Y = inputs.mlp_batches(cfg, 5)
+    eager, _ = _make(cfg, cfg["S"], masters)
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        from paper_1710_03740_b200 import binding as b
+        net = b.Context(cfg["layers"], cfg["S"], cfg["lr"], cfg["momentum"], cfg["batch"], stream=side)
+        for l, w in enumerate(masters):
+            net.set_master(l, w)
+        x_static = torch.zeros((cfg["batch"], 256), dtype=torch.int16, device="cuda")
+        y_static = torch.zeros(cfg["batch"], dtype=torch.int32, device="cuda")
+        # one eager step first: kernel attributes are set outside the capture
+        x_static.copy_(dev(X[0].view(np.uint16)))
+        y_static.copy_(dev(Y[0]))
+        net.forward(x_static)
+        net.backward_scaled(y_static, want_loss=False)
+        net.step(want_flag=False)
+        side.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            net.forward(x_static)
+            net.backward_scaled(y_static, want_loss=False)
+            net.step(want_flag=False)
+        for t in range(1, 5):
+            x_static.copy_(dev(X[t].view(np.uint16)))
+            y_static.copy_(dev(Y[t]))
+            graph.replay()
+        side.synchronize()
+    keep = []                                       # inputs must outlive the backward pass that reads them
+    for t in range(5):
+        xd, yd = dev(X[t].view(np.uint16)), dev(Y[t])
+        keep.append((xd, yd))
+        eager.forward(xd)
+        eager.backward_scaled(yd, want_loss=False)
+        eager.step(want_flag=False)
+    torch.cuda.synchronize()
+    for l in range(2):
+        assert net.get_master(l).tobytes() == eager.get_master(l).tobytes()
+
+
 def test_error_paths():
     from paper_1710_03740_b200 import binding as b
     cfg = inputs.MLP_CONFIGS["tiny"]
@@ -286,7 +330,8 @@ def test_error_paths():
     with pytest.raises(b.MptError):
         net.set_master(0, np.zeros(5, dtype=np.float32))
     # labels out of range are reported, and the context stays usable
-    net.forward(dev(X[0].view(np.uint16)))
+    x_dev = dev(X[0].view(np.uint16))
+    net.forward(x_dev)
     bad = Y[0].copy()
     bad[3] = 10
     with pytest.raises(b.MptError) as e:
