@@ -68,7 +68,7 @@ extern "C" {
                                   MPT_ERR_SHAPE if the operands do not meet its alignment rules */
 #define MPT_GEMM_FORCE_PAIR 8u /* require the CTA-pair tcgen05 kernel (cta_group::2, 256x256 tiles);
                                   same alignment rules.  Without a FORCE flag the library picks the
-                                  pair kernel when the output has at least 128 tiles of 256x256,
+                                  pair kernel when the output has at least 48 tiles of 256x256,
                                   else the single-CTA one */
 
 /* mpt_get_tensor kinds */
@@ -241,6 +241,19 @@ void mpt_destroy(mpt_ctx *ctx);
 int mpt_gemm_f16(int op, int M, int N, int K, const uint16_t *A_dev, int lda, const uint16_t *B_dev,
                  int ldb, uint16_t *C_dev, int ldc, unsigned flags, const uint16_t *mask_dev,
                  int ldmask, uint32_t *nonfinite_flag_dev, uint32_t *status_dev, void *cuda_stream);
+
+/* The same product with a caller-provided scratch buffer that allows the contraction to be
+ * split (section 3.3 arithmetic unchanged except for the order of the FP32 additions: the
+ * parts are added in ascending order by a second kernel, so results stay run-to-run
+ * identical).  Outputs with few tiles and a long contraction (for instance 2048 x 1024 with
+ * K = 8192) otherwise leave most SMs idle.  mpt_gemm_workspace_bytes returns the scratch size
+ * the library would like for a shape (0 when it would not split); a smaller or null buffer
+ * simply disables or narrows the split.  splitk_ws_dev must be 16-byte aligned. */
+int mpt_gemm_workspace_bytes(int op, int M, int N, int K, size_t *bytes_out);
+int mpt_gemm_f16_ws(int op, int M, int N, int K, const uint16_t *A_dev, int lda, const uint16_t *B_dev, int ldb,
+                    uint16_t *C_dev, int ldc, unsigned flags, const uint16_t *mask_dev, int ldmask,
+                    uint32_t *nonfinite_flag_dev, uint32_t *status_dev, void *splitk_ws_dev, size_t splitk_ws_bytes,
+                    void *cuda_stream);
 
 /* w16[e] = rn16(w32[e]) (section 3.1: the FP16 copy is made by rounding). */
 int mpt_recast(const float *w32_dev, uint16_t *w16_dev, size_t n, void *cuda_stream);

@@ -28,7 +28,7 @@ EXPORTS = ["mpt_workspace_bytes", "mpt_create", "mpt_set_master", "mpt_forward",
            "mpt_train_step_staged", "mpt_set_scale", "mpt_set_lr", "mpt_set_dynamic_scale", "mpt_get_scale",
            "mpt_get_tensor", "mpt_set_grad", "mpt_set_momentum", "mpt_launch_count", "mpt_profile",
            "mpt_profile_read", "mpt_last_error",
-           "mpt_destroy", "mpt_gemm_f16", "mpt_recast", "mpt_grad_nonfinite", "mpt_update_flat",
+           "mpt_destroy", "mpt_gemm_f16", "mpt_gemm_f16_ws", "mpt_gemm_workspace_bytes", "mpt_recast", "mpt_grad_nonfinite", "mpt_update_flat",
            "mpt_softmax_ce", "mpt_softmax_ce_static", "mpt_version"]
 
 
@@ -79,6 +79,8 @@ def lib() -> C.CDLL:
     L.mpt_destroy.argtypes = [vp]
     L.mpt_destroy.restype = None
     L.mpt_gemm_f16.argtypes = [i32, i32, i32, i32, vp, i32, vp, i32, vp, i32, u32, vp, i32, vp, vp, vp]
+    L.mpt_gemm_f16_ws.argtypes = [i32, i32, i32, i32, vp, i32, vp, i32, vp, i32, u32, vp, i32, vp, vp, vp, sz, vp]
+    L.mpt_gemm_workspace_bytes.argtypes = [i32, i32, i32, i32, C.POINTER(sz)]
     L.mpt_recast.argtypes = [vp, vp, sz, vp]
     L.mpt_grad_nonfinite.argtypes = [vp, sz, f32, vp, vp]
     L.mpt_update_flat.argtypes = [vp, vp, vp, vp, sz, f32, f32, f32, i32, i32, vp, vp]
@@ -268,6 +270,20 @@ def mpt_gemm_f16(op, M, N, K, A, lda, B, ldb, Cout, ldc, flags=0, mask=None, ldm
     """Arguments are torch CUDA tensors (any 2-byte dtype) used as raw device pointers."""
     _check(lib().mpt_gemm_f16(op, M, N, K, _dptr(A), lda, _dptr(B), ldb, _dptr(Cout), ldc, flags, _dptr(mask), ldmask,
                               _dptr(nonfinite_flag), _dptr(status), _stream_ptr(stream)))
+
+
+def mpt_gemm_workspace_bytes(op, M, N, K) -> int:
+    out = C.c_size_t(0)
+    _check(lib().mpt_gemm_workspace_bytes(op, M, N, K, C.byref(out)))
+    return int(out.value)
+
+
+def mpt_gemm_f16_ws(op, M, N, K, A, lda, B, ldb, Cout, ldc, flags=0, mask=None, ldmask=0, nonfinite_flag=None,
+                    status=None, workspace=None, stream=None):
+    """mpt_gemm_f16 with a scratch tensor (any dtype, 16-byte aligned) that permits split-K."""
+    nbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib().mpt_gemm_f16_ws(op, M, N, K, _dptr(A), lda, _dptr(B), ldb, _dptr(Cout), ldc, flags, _dptr(mask), ldmask,
+                                 _dptr(nonfinite_flag), _dptr(status), _dptr(workspace), nbytes, _stream_ptr(stream)))
 
 
 def mpt_recast(w32, w16, n, stream=None):

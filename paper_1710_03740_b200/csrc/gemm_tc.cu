@@ -58,6 +58,12 @@ struct TcParams {
     uint32_t *nonfinite_flag;
     uint32_t *status;  // may be null
     int tiles_m, tiles_n, group_m;
+    // split-K: the contraction range of every tile is cut into split_k parts, each part is a
+    // work unit that leaves its raw FP32 accumulator in `partial` [split_k][M][ldp]; a second
+    // kernel adds the parts in a fixed order and applies the epilogue.  split_k == 1: off.
+    int split_k;
+    float *partial;
+    int ldp;
 };
 
 __device__ __forceinline__ void tile_coords(const TcParams &p, int tile, int &mb, int &nb)
@@ -100,7 +106,12 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int num_tiles = p.tiles_m * p.tiles_n;
+    const int num_units = num_tiles * p.split_k;   // unit u: tile u % num_tiles, contraction part u / num_tiles
     const int nkb = (p.K + BLOCK_K - 1) / BLOCK_K;
+    // k-block range of contraction part `part` (32-bit arithmetic: nkb * split_k is far below 2^31)
+    auto kb_begin = [&](int part) { return p.split_k == 1 ? part * nkb : (int)((unsigned)(nkb * part) / (unsigned)p.split_k); };
+    auto unit_tile = [&](int u) { return p.split_k == 1 ? u : u % num_tiles; };
+    auto unit_part = [&](int u) { return p.split_k == 1 ? 0 : u / num_tiles; };
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; s++) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
@@ -125,11 +136,12 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         if (lane == 0) {
             uint32_t issued = 0, s = 0, ph = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+            for (int u = blockIdx.x; u < num_units && ok; u += gridDim.x) {
                 int mb, nb;
-                tile_coords(p, tile, mb, nb);
+                tile_coords(p, unit_tile(u), mb, nb);
+                const int part = unit_part(u), kb1 = kb_begin(part + 1);
                 const int m0 = mb * BLOCK_M, n0 = nb * BLOCK_N;
-                for (int kb = 0; kb < nkb; kb++, issued++, s = (s + 1 == STAGES) ? 0 : s + 1, ph ^= (s == 0)) {
+                for (int kb = kb_begin(part); kb < kb1; kb++, issued++, s = (s + 1 == STAGES) ? 0 : s + 1, ph ^= (s == 0)) {
                     if (!mbar_try_wait(empty_bar(s), ph ^ 1u) && !mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) {
                         if (!*abort_flag) report(p, abort_flag, KERR_WAIT_EMPTY);
                         ok = false;
@@ -175,7 +187,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
             uint32_t s = 0, ph = 0;
             bool ok = true;
             int t = 0;
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, t++) {
+            for (int u = blockIdx.x; u < num_units && ok; u += gridDim.x, t++) {
+                const int part = unit_part(u), kb0 = kb_begin(part), kb1 = kb_begin(part + 1);
                 const int buf = t & 1;
                 const uint32_t acc_ph = (t >> 1) & 1u;
                 if (!mbar_try_wait(acce_bar(buf), acc_ph ^ 1u) && !mbar_wait(acce_bar(buf), acc_ph ^ 1u, abort_flag)) {
@@ -185,8 +198,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                 }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BLOCK_N);
-                uint32_t acc = 0;                       // first MMA of a tile overwrites the accumulator
-                for (int kb = 0; kb < nkb; kb++) {
+                uint32_t acc = 0;                       // first MMA of a unit overwrites the accumulator
+                for (int kb = kb0; kb < kb1; kb++) {
                     if (!mbar_try_wait(full_bar(s), ph) && !mbar_wait(full_bar(s), ph, abort_flag)) {
                         if (!*abort_flag) report(p, abort_flag, KERR_WAIT_FULL);
                         ok = false;
@@ -211,9 +224,10 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         const int q = warp & 3;                    // TMEM lane quadrant this warp may access
         bool ok = true;
         int t = 0;
-        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, t++) {
+        for (int u = blockIdx.x; u < num_units && ok; u += gridDim.x, t++) {
             int mb, nb;
-            tile_coords(p, tile, mb, nb);
+            tile_coords(p, unit_tile(u), mb, nb);
+            const int part = unit_part(u);
             const int buf = t & 1;
             const uint32_t acc_ph = (t >> 1) & 1u;
             if (!mbar_wait(accf_bar(buf), acc_ph, abort_flag)) {
@@ -233,7 +247,18 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                 tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BLOCK_N + c * 32), r);
                 tc_wait_ld();
                 const int col0 = nb * BLOCK_N + c * 32;
-                if (row_ok && col0 < p.N) epilogue_store32(r, crow, mrow, col0, p.N, p.relu != 0, bad);
+                if (p.split_k > 1) {
+                    // raw FP32 partial sums; ldp is a multiple of 32, so a started chunk is always whole
+                    if (row_ok && col0 < p.ldp) {
+                        float4 *dst = (float4 *)(p.partial + ((size_t)part * p.M + row) * p.ldp + col0);
+#pragma unroll
+                        for (int v = 0; v < 8; v++)
+                            dst[v] = make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
+                                                 __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
+                    }
+                } else if (row_ok && col0 < p.N) {
+                    epilogue_store32(r, crow, mrow, col0, p.N, p.relu != 0, bad);
+                }
             }
             tc_fence_before();
             __syncwarp();
@@ -249,6 +274,42 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS) : "memory");
     }
+}
+
+// Second step of a split-K product: C = epilogue(partial[0] + partial[1] + ... ) with the parts
+// added in ascending order (FP32, one rounding per add), eight columns per thread.
+__global__ void __launch_bounds__(256) k_splitk_reduce(const float *__restrict__ partial, int split_k, int M, int N,
+                                                       int ldp, uint16_t *__restrict__ C, int ldc, int relu,
+                                                       const uint16_t *__restrict__ mask, int ldmask,
+                                                       uint32_t *nonfinite_flag)
+{
+    const int groups = (N + 7) / 8;
+    const size_t total = (size_t)M * groups;
+    bool bad = false;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const int row = (int)(i / groups), col = (int)(i % groups) * 8;
+        const float *src = partial + (size_t)row * ldp + col;
+        float4 a = *(const float4 *)src, b = *(const float4 *)(src + 4);
+        for (int sp = 1; sp < split_k; sp++) {
+            const float *q = src + (size_t)sp * M * ldp;
+            const float4 c = *(const float4 *)q, d = *(const float4 *)(q + 4);
+            a.x += c.x; a.y += c.y; a.z += c.z; a.w += c.w;
+            b.x += d.x; b.y += d.y; b.z += d.z; b.w += d.w;
+        }
+        const float v[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+        for (int e = 0; e < 8 && col + e < N; e++) {
+            float s = v[e];
+            if (relu) s = (s > 0.0f || s != s) ? s : 0.0f;
+            uint32_t h = (uint32_t)__half_as_ushort(__float2half_rn(s));
+            if (mask) {
+                const uint32_t mh = mask[(size_t)row * ldmask + col + e];
+                if (!((mh & 0x8000u) == 0 && mh != 0 && mh <= 0x7C00u)) h = 0;
+            }
+            bad |= (h & 0x7C00u) == 0x7C00u;
+            C[(size_t)row * ldc + col + e] = (uint16_t)h;
+        }
+    }
+    if (nonfinite_flag && __any_sync(0xFFFFFFFFu, bad) && (threadIdx.x & 31) == 0) atomicOr(nonfinite_flag, 1u);
 }
 
 // ------------------------------------------------------------------ host side
@@ -332,16 +393,58 @@ static cudaError_t launch_bn(int op, int M, int N, int K, const uint16_t *A, int
     p.tiles_m = (M + BLOCK_M - 1) / BLOCK_M;
     p.tiles_n = (N + BN - 1) / BN;
     p.group_m = 16;
-    int tiles = p.tiles_m * p.tiles_n;
-    int grid = tiles < 148 ? tiles : 148;
-    if (op == MPT_OP_FWD) return launch_variant<false, false, BN>(ta, tb, p, grid, st);
-    if (op == MPT_OP_DGRAD) return launch_variant<false, true, BN>(ta, tb, p, grid, st);
-    return launch_variant<true, true, BN>(ta, tb, p, grid, st);
+    int units = p.tiles_m * p.tiles_n * p.split_k;
+    int grid = units < 148 ? units : 148;
+    cudaError_t e;
+    if (op == MPT_OP_FWD) e = launch_variant<false, false, BN>(ta, tb, p, grid, st);
+    else if (op == MPT_OP_DGRAD) e = launch_variant<false, true, BN>(ta, tb, p, grid, st);
+    else e = launch_variant<true, true, BN>(ta, tb, p, grid, st);
+    if (e != cudaSuccess || p.split_k == 1) return e;
+    const size_t work = (size_t)M * ((N + 7) / 8);
+    size_t blocks = (work + 255) / 256;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    k_splitk_reduce<<<(unsigned)blocks, 256, 0, st>>>(p.partial, p.split_k, M, N, p.ldp, p.C, p.ldc, p.relu, p.mask,
+                                                      p.ldmask, p.nonfinite_flag);
+    return cudaGetLastError();
+}
+
+// Tile width and split factor for the single-CTA kernel.  Cost model in tensor-pipe cycles: a
+// 128x256 tile needs 512 cycles per 64-deep k-block; a 128x128 tile needs 256 but runs at about
+// 0.6 of that rate (operand reads from shared memory bound it); measured per k-block: about 600
+// and 437 cycles.  The epilogue of a tile costs about 400 cycles per 32 columns and is exposed
+// for the last tile of a CTA; a launch costs about 14000 cycles; a split adds a second, mostly
+// overlapped launch (about 4000) and one FP32 write and read of the output per part, which
+// stays in L2 (about 64 bytes per cycle and SM).  Calibrated with launches replayed from a CUDA
+// graph on 2048x1024x8192, 1024x1024x4096, 512x256x4096 and the tiny-MLP products.  The split
+// is only considered when a workspace is available.
+void tc_gemm_plan(int M, int N, int K, size_t ws_bytes, int *bn_out, int *split_out, size_t *ws_needed)
+{
+    const long tm = (M + BLOCK_M - 1) / BLOCK_M;
+    const int nkb = (K + BLOCK_K - 1) / BLOCK_K;
+    double best = 1e30;
+    int best_bn = 256, best_s = 1;
+    for (int bn : {256, 128}) {
+        if (bn == 128 && N <= 128) continue;
+        const long tiles = tm * ((N + bn - 1) / bn);
+        const double cyc = bn == 256 ? 600.0 : 437.0;
+        for (int s = 1; s <= 8; s++) {
+            if (s > 1 && (nkb / s < 8)) break;
+            const size_t need = s > 1 ? (size_t)s * M * (((size_t)N + 31) / 32 * 32) * 4 : 0;
+            if (need > ws_bytes) break;
+            const long rounds = (tiles * s + 147) / 148;
+            double cost = rounds * ((double)nkb / s) * cyc + (bn / 32) * 400.0 + 14000.0;   // + exposed epilogue + launch
+            if (s > 1) cost += 4000.0 + (double)need * 2.0 / 148.0 / 64.0;                  // second launch + partial traffic
+            if (cost < best * 0.99) { best = cost; best_bn = bn; best_s = s; }
+        }
+    }
+    *bn_out = best_bn;
+    *split_out = best_s;
+    if (ws_needed) *ws_needed = best_s > 1 ? (size_t)best_s * M * (((size_t)N + 31) / 32 * 32) * 4 : 0;
 }
 
 cudaError_t launch_gemm_tc(int op, int M, int N, int K, const uint16_t *A, int lda, const uint16_t *B, int ldb,
                            uint16_t *C, int ldc, bool relu, const uint16_t *mask, int ldmask, uint32_t *nonfinite_flag,
-                           uint32_t *status, cudaStream_t st)
+                           uint32_t *status, cudaStream_t st, float *splitk_ws, size_t splitk_ws_bytes)
 {
     TcParams p;
     p.M = M; p.N = N; p.K = K;
@@ -350,10 +453,12 @@ cudaError_t launch_gemm_tc(int op, int M, int N, int K, const uint16_t *A, int l
     p.relu = relu ? 1 : 0;
     p.nonfinite_flag = nonfinite_flag;
     p.status = status;
-    // 128-wide tiles when 256-wide ones would leave more than a fifth of the SMs without work
-    const long tm = (M + BLOCK_M - 1) / BLOCK_M;
-    const long tiles256 = tm * ((N + 255) / 256);
-    if (tiles256 < 118 && N > 128) return launch_bn<128>(op, M, N, K, A, lda, B, ldb, p, st);
+    int bn = 256, split = 1;
+    tc_gemm_plan(M, N, K, (splitk_ws && (((uintptr_t)splitk_ws) & 15) == 0) ? splitk_ws_bytes : 0, &bn, &split, nullptr);
+    p.split_k = split;
+    p.partial = splitk_ws;
+    p.ldp = (N + 31) / 32 * 32;
+    if (bn == 128) return launch_bn<128>(op, M, N, K, A, lda, B, ldb, p, st);
     return launch_bn<256>(op, M, N, K, A, lda, B, ldb, p, st);
 }
 

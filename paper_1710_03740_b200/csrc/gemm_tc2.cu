@@ -314,7 +314,8 @@ static cudaError_t launch_variant(const CUtensorMap &ta, const CUtensorMap &tb, 
     // halves fit into one round
     const int tiles = p.tiles_m * p.tiles_n;
     const int pairs = tiles < max_pairs ? tiles : max_pairs;
-    const int full = (tiles / pairs) * pairs, rest = tiles - full;
+    int full = (tiles / pairs) * pairs, rest = tiles - full;
+    if (2 * tiles <= max_pairs) { full = 0; rest = tiles; }   // too few tiles for the clusters: halves all the way
     if (rest > 0 && 2 * rest <= max_pairs) {
         p.full_units = full;
         p.num_units = full + 2 * rest;
@@ -331,11 +332,12 @@ static cudaError_t launch_variant(const CUtensorMap &ta, const CUtensorMap &tb, 
 
 bool tc2_gemm_preferred(int M, int N, int K)
 {
-    // pairs pay off once there are enough 256x256 tiles to fill the 74 clusters about twice;
-    // small or thin problems have more parallelism as 128x256 tiles on the 1-CTA kernel
+    // measured on B200 with launches replayed from a CUDA graph: from about 48 tiles of 256x256
+    // (two thirds of the 74 clusters) the pair kernel wins; below that the single-CTA kernel
+    // with narrower tiles or a split contraction has more parallelism
     (void)K;
     const long tiles = (long)((M + 255) / 256) * ((N + 255) / 256);
-    return M >= 256 && N >= 256 && tiles >= 128;
+    return M >= 256 && N >= 256 && tiles >= 48;
 }
 
 cudaError_t launch_gemm_tc2(int op, int M, int N, int K, const uint16_t *A, int lda, const uint16_t *B, int ldb,

@@ -29,7 +29,7 @@ struct Layer {
 struct Plan {
     size_t total = 0, P_pad = 0;
     size_t off_status = 0, off_master = 0, off_mom = 0, off_w16 = 0, off_g16 = 0, off_x[2] = {0, 0},
-           off_labels[2] = {0, 0}, off_rowloss = 0;
+           off_labels[2] = {0, 0}, off_rowloss = 0, off_splitk = 0, splitk_bytes = 0;
     std::vector<size_t> off_act, off_dact, lay_off;
     std::vector<int> ld_out;
 };
@@ -79,6 +79,23 @@ void make_plan(const mpt_layer_desc *layers, int L, int max_batch, bool mom, Pla
         pl.off_labels[k] = take((size_t)max_batch * 4);
     }
     pl.off_rowloss = take((size_t)max_batch * 4);
+    // scratch for split-K partial sums: the largest need of any product of the step that runs on
+    // the single-CTA tensor-core kernel (small or thin outputs), capped at 256 MB
+    size_t need_max = 0;
+    for (int l = 0; l < L; l++) {
+        const int B = max_batch, in = layers[l].in_features, out = layers[l].out_features;
+        const int shapes[3][3] = {{B, out, in}, {out, in, B}, {B, in, out}};   // forward, wgrad, dgrad as (M, N, K)
+        for (int k = 0; k < 3; k++) {
+            if (k == 2 && l == 0) continue;
+            if (tc2_gemm_preferred(shapes[k][0], shapes[k][1], shapes[k][2])) continue;
+            int bn, split;
+            size_t need = 0;
+            tc_gemm_plan(shapes[k][0], shapes[k][1], shapes[k][2], (size_t)256 << 20, &bn, &split, &need);
+            if (need > need_max) need_max = need;
+        }
+    }
+    pl.splitk_bytes = need_max;
+    pl.off_splitk = need_max ? take(need_max) : 0;
     pl.total = off;
 }
 
@@ -96,6 +113,7 @@ struct mpt_ctx {
     float *master, *mom;
     uint16_t *w16, *g16, *x_stage[2];
     int32_t *labels_stage[2];
+    float *splitk_ws = nullptr;
     // staged (pipelined) host batches: slot state and the events that order copies against compute
     cudaEvent_t staged_ev[2] = {nullptr, nullptr}, used_ev[2] = {nullptr, nullptr};
     bool staged_valid[2] = {false, false}, used_recorded[2] = {false, false};
@@ -204,7 +222,7 @@ int gemm(mpt_ctx *c, int op, int M, int N, int K, const uint16_t *A, int lda, co
                                 c->status + ST_KERNEL_ERR, c->stream);
         else
             e = launch_gemm_tc(op, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite,
-                               c->status + ST_KERNEL_ERR, c->stream);
+                               c->status + ST_KERNEL_ERR, c->stream, c->splitk_ws, c->plan.splitk_bytes);
     } else
         e = launch_gemm_simt(op, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite, c->stream);
     c->launches++;
@@ -358,6 +376,7 @@ int mpt_create(const mpt_layer_desc *layers, int n_layers, float S, float lr, fl
         c->labels_stage[k] = (int32_t *)(c->ws + pl.off_labels[k]);
     }
     c->row_loss = (float *)(c->ws + pl.off_rowloss);
+    c->splitk_ws = pl.splitk_bytes ? (float *)(c->ws + pl.off_splitk) : nullptr;
     c->layers.resize(n_layers);
     for (int l = 0; l < n_layers; l++) {
         Layer &ly = c->layers[l];
@@ -701,9 +720,29 @@ int mpt_set_momentum(mpt_ctx *c, int layer, const float *src_host, size_t n)
 
 // ---------------------------------------------------------- stateless launchers
 
+int mpt_gemm_workspace_bytes(int op, int M, int N, int K, size_t *bytes_out)
+{
+    if (!bytes_out) return MPT_ERR_INVALID_ARG;
+    if (op != MPT_OP_FWD && op != MPT_OP_DGRAD && op != MPT_OP_WGRAD) return MPT_ERR_INVALID_ARG;
+    if (M < 0 || N < 0 || K < 0) return MPT_ERR_SHAPE;
+    *bytes_out = 0;
+    if (M == 0 || N == 0 || K == 0 || tc2_gemm_preferred(M, N, K)) return MPT_OK;
+    int bn, split;
+    tc_gemm_plan(M, N, K, (size_t)256 << 20, &bn, &split, bytes_out);
+    return MPT_OK;
+}
+
 int mpt_gemm_f16(int op, int M, int N, int K, const uint16_t *A, int lda, const uint16_t *B, int ldb, uint16_t *C, int ldc,
                  unsigned flags, const uint16_t *mask, int ldmask, uint32_t *nonfinite_flag, uint32_t *status_dev,
                  void *cuda_stream)
+{
+    return mpt_gemm_f16_ws(op, M, N, K, A, lda, B, ldb, C, ldc, flags, mask, ldmask, nonfinite_flag, status_dev, nullptr, 0,
+                           cuda_stream);
+}
+
+int mpt_gemm_f16_ws(int op, int M, int N, int K, const uint16_t *A, int lda, const uint16_t *B, int ldb, uint16_t *C,
+                    int ldc, unsigned flags, const uint16_t *mask, int ldmask, uint32_t *nonfinite_flag,
+                    uint32_t *status_dev, void *splitk_ws_dev, size_t splitk_ws_bytes, void *cuda_stream)
 {
     if (!A || !B || !C) return MPT_ERR_INVALID_ARG;
     if (op != MPT_OP_FWD && op != MPT_OP_DGRAD && op != MPT_OP_WGRAD) return MPT_ERR_INVALID_ARG;
@@ -721,7 +760,8 @@ int mpt_gemm_f16(int op, int M, int N, int K, const uint16_t *A, int lda, const 
         if (pair)
             e = launch_gemm_tc2(op, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite_flag, status_dev, st);
         else
-            e = launch_gemm_tc(op, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite_flag, status_dev, st);
+            e = launch_gemm_tc(op, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite_flag, status_dev, st,
+                               (float *)splitk_ws_dev, splitk_ws_bytes);
     } else
         e = launch_gemm_simt(op, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite_flag, st);
     return e == cudaSuccess ? MPT_OK : MPT_ERR_CUDA;

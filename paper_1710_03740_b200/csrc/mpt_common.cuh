@@ -74,9 +74,14 @@ cudaError_t launch_gemm_simt(int op, int M, int N, int K, const uint16_t *A, int
 // TMA descriptors on the host and launches the persistent kernel.
 bool tc_gemm_supported(int op, int M, int N, int K, const void *A, int lda, const void *B, int ldb,
                        const void *C, int ldc, const void *mask, int ldmask);
+// splitk_ws (may be null): 16-byte aligned device scratch for split-K partial sums; without it
+// the contraction is never split.  tc_gemm_plan tells which tile width / split factor the
+// launcher will pick and how much scratch that needs.
 cudaError_t launch_gemm_tc(int op, int M, int N, int K, const uint16_t *A, int lda, const uint16_t *B,
                            int ldb, uint16_t *C, int ldc, bool relu, const uint16_t *mask, int ldmask,
-                           uint32_t *nonfinite_flag, uint32_t *status, cudaStream_t st);
+                           uint32_t *nonfinite_flag, uint32_t *status, cudaStream_t st, float *splitk_ws = nullptr,
+                           size_t splitk_ws_bytes = 0);
+void tc_gemm_plan(int M, int N, int K, size_t ws_bytes, int *bn_out, int *split_out, size_t *ws_needed);
 
 // CTA-pair variant (tcgen05 cta_group::2, 256x256 tiles); same operand rules as launch_gemm_tc.
 bool tc2_gemm_preferred(int M, int N, int K);

@@ -26,7 +26,7 @@ def _pad(a, ld):
     return out
 
 
-def run_gemm(op, A, B, M, N, K, flags=0, mask=None, pad=0, want_flag=False):
+def run_gemm(op, A, B, M, N, K, flags=0, mask=None, pad=0, want_flag=False, workspace=False):
     """A, B: stored float16 operands.  pad: extra columns added to every pitch."""
     from paper_1710_03740_b200 import binding as b
     lda, ldb, ldc = A.shape[1] + pad, B.shape[1] + pad, N + pad
@@ -35,8 +35,16 @@ def run_gemm(op, A, B, M, N, K, flags=0, mask=None, pad=0, want_flag=False):
     md = dev(_pad(mask, ldc)) if mask is not None else None
     flag = torch.zeros(1, dtype=torch.int32, device="cuda")
     status = torch.zeros(4, dtype=torch.int32, device="cuda")
-    b.mpt_gemm_f16(op, M, N, K, Ad, lda, Bd, ldb, Cd, ldc, flags, md, ldc if mask is not None else 0,
-                   flag if want_flag else None, status)
+    if workspace:
+        nbytes = b.mpt_gemm_workspace_bytes(op, M, N, K)
+        if nbytes == 0:
+            pytest.skip("the library does not split this shape")
+        ws = torch.full((nbytes // 4,), float("nan"), dtype=torch.float32, device="cuda")
+        b.mpt_gemm_f16_ws(op, M, N, K, Ad, lda, Bd, ldb, Cd, ldc, flags, md, ldc if mask is not None else 0,
+                          flag if want_flag else None, status, ws)
+    else:
+        b.mpt_gemm_f16(op, M, N, K, Ad, lda, Bd, ldb, Cd, ldc, flags, md, ldc if mask is not None else 0,
+                       flag if want_flag else None, status)
     torch.cuda.synchronize()
     assert int(status[0].item()) == 0, "device-side wait expired: 0x%x" % int(status[0].item())
     out = host_u16(Cd)
@@ -80,14 +88,14 @@ def test_simt_gemm_relu_mask_flag():
     assert flag == 1 and (~np.isfinite(ref.view(np.float16).astype(np.float32))).any()
 
 
-def _check_tc(op, M, N, K, flags=0, mask=None, seed=21, scale=None, want_flag=False, kernel="tc"):
+def _check_tc(op, M, N, K, flags=0, mask=None, seed=21, scale=None, want_flag=False, kernel="tc", workspace=False):
     from paper_1710_03740_b200 import binding as b
     force = b.GEMM_FORCE_PAIR if kernel == "pair" else b.GEMM_FORCE_TC
     sa = sb = scale
     A, B = inputs.gemm_operands(op, M, N, K, seed=seed, scale_a=sa, scale_b=sb)
     ref, ex, ab = mpo.gemm_f16(op, A, B, relu=bool(flags & b.GEMM_RELU), mask=mask, want_exact=True)
     got, flag = run_gemm(op, A, B, M, N, K, flags=flags | force, mask=mask,
-                         pad=(8 if (M * N) % 3 == 0 else 0), want_flag=want_flag)
+                         pad=(8 if (M * N) % 3 == 0 else 0), want_flag=want_flag, workspace=workspace)
     ok, stats = gemm_accept(got, ref, K=K, absdot=ab)
     assert ok.all(), (op, M, N, K, stats, np.argwhere(~ok)[:8].tolist())
     assert stats["by_abs_only"] <= max(2, stats["n"] // 1000), stats
@@ -141,6 +149,25 @@ def test_pair_kernel_half_width_tail_units(op, M, N, K):
     """A few more tiles than clusters: the left-over tiles run as two 256x128 halves, including
     halves that are partly or wholly outside a ragged N."""
     _check_tc(op, M, N, K, kernel="pair")
+
+
+@pytest.mark.parametrize("op", [0, 1, 2])
+@pytest.mark.parametrize("M,N,K", [(512, 256, 4096), (256, 264, 8192), (136, 96, 8192), (384, 1024, 6144)])
+def test_split_k_parity_and_determinism(op, M, N, K):
+    """Few output tiles and a long contraction: the contraction is split over CTAs, FP32 parts are
+    added in a fixed order by a second kernel.  Same acceptance rule; identical bits on a rerun;
+    ReLU, mask and the overflow flag go through the reduce kernel."""
+    from paper_1710_03740_b200 import binding as b
+    if (M, N, K) == (512, 256, 4096):
+        assert b.mpt_gemm_workspace_bytes(op, M, N, K) > 0      # the canonical few-tiles / long-K case must split
+    got, ref, _, _ = _check_tc(op, M, N, K, workspace=True)
+    again, _, _, _ = _check_tc(op, M, N, K, workspace=True)
+    assert np.array_equal(got, again)
+    _check_tc(op, M, N, K, flags=b.GEMM_RELU, workspace=True)
+    mask = np.random.default_rng(8).standard_normal((M, N)).astype(np.float16)
+    _check_tc(op, M, N, K, mask=mask, workspace=True)
+    _, ref, flag, _ = _check_tc(op, M, N, K, scale=30.0, want_flag=True, workspace=True)
+    assert flag == int(((ref & 0x7FFF) >= 0x7C00).any()) == 1
 
 
 @pytest.mark.parametrize("kernel", ["tc", "pair"])
