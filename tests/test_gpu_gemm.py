@@ -170,6 +170,24 @@ def test_split_k_parity_and_determinism(op, M, N, K):
     assert flag == int(((ref & 0x7FFF) >= 0x7C00).any()) == 1
 
 
+@pytest.mark.parametrize("op", [0, 1, 2])
+def test_random_ragged_shapes_all_kernels(op):
+    """Seeded random shapes with ragged M, N, K (pitches are multiples of 8): every kernel choice the
+    library can make (single CTA, pair, automatic with and without a split-K workspace)."""
+    from paper_1710_03740_b200 import binding as b
+    rng = np.random.default_rng(1000 + op)
+    for trial in range(14):
+        M = int(rng.integers(1, 90)) * 8
+        N = int(rng.integers(1, 90)) * 8
+        K = int(rng.choice([8, 24, 64, 72, 200, 520, 1032, 2056, 4104]))
+        relu = bool(rng.integers(0, 2))
+        for kernel, ws in (("tc", False), ("pair", False), ("tc", True)):
+            if ws and b.mpt_gemm_workspace_bytes(op, M, N, K) == 0:
+                continue
+            _check_tc(op, M, N, K, flags=b.GEMM_RELU if relu else 0, seed=int(rng.integers(1 << 30)), kernel=kernel,
+                      workspace=ws)
+
+
 @pytest.mark.parametrize("kernel", ["tc", "pair"])
 def test_tc_gemm_relu_mask_flag_subnormals(kernel):
     from paper_1710_03740_b200 import binding as b
