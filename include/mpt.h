@@ -78,6 +78,36 @@ extern "C" {
 #define MPT_T_DACT16 3     /* FP16 gradient dz_l     [batch, out_l] (scaled by S) */
 #define MPT_T_MOMENTUM32 4 /* FP32 momentum buffer   [out, in]            */
 #define MPT_T_MASTER32 5   /* FP32 master weights    [out, in]            */
+#define MPT_T_STATE2_32 6  /* FP32 second optimizer state [out, in] (Adam's second moment) */
+
+/* Optimizer step applied to the FP32 master copy (section 3.1: the update is computed in FP32;
+ * the paper's experiments use plain and Nesterov momentum SGD, Adagrad and Adam, sections 4.3,
+ * 4.5, 4.6, without giving formulas: the textbook forms are used).  With g the UNSCALED
+ * gradient (section 3.2: decay and the like act after unscaling), every line one separately
+ * rounded FP32 operation, states starting at zero:
+ *   weight_decay != 0:  g = g + weight_decay * w
+ *   MPT_OPT_SGD       momentum == 0: u = lr*g ;  else  s1 = momentum*s1 + g ; u = lr*s1
+ *   MPT_OPT_NESTEROV  s1 = momentum*s1 + g ; u = lr*(g + momentum*s1)
+ *   MPT_OPT_ADAGRAD   s1 = s1 + g*g ; u = lr*(g / (sqrt(s1) + eps))
+ *   MPT_OPT_ADAM      s1 = b1*s1 + (1-b1)*g ; s2 = b2*s2 + (1-b2)*(g*g) ;
+ *                     u = lr*((s1/(1-b1^t)) / (sqrt(s2/(1-b2^t)) + eps))   (b1 = momentum field)
+ *                     where b^t are running FP32 products over the steps that were applied
+ *                     (a step skipped for overflow does not advance them)
+ *   w = w - u ; w16 = rn16(w)
+ * Bytes moved per parameter: 12 (plain SGD), 20 (one state), 28 (Adam). */
+#define MPT_OPT_SGD 0
+#define MPT_OPT_NESTEROV 1
+#define MPT_OPT_ADAGRAD 2
+#define MPT_OPT_ADAM 3
+
+typedef struct mpt_optimizer {
+    int32_t kind;       /* MPT_OPT_* */
+    float lr;
+    float momentum;     /* SGD / Nesterov momentum, Adam beta1; in [0, 1) */
+    float beta2;        /* Adam beta2 in [0, 1); ignored otherwise */
+    float eps;          /* Adagrad / Adam epsilon >= 0; ignored otherwise */
+    float weight_decay; /* >= 0; 0 disables */
+} mpt_optimizer;
 
 typedef struct mpt_ctx mpt_ctx;
 
@@ -111,6 +141,13 @@ int mpt_workspace_bytes(const mpt_layer_desc *layers, int n_layers, int max_batc
 int mpt_create(const mpt_layer_desc *layers, int n_layers, float S, float lr, float momentum,
                int max_batch, void *workspace_dev, size_t workspace_bytes, void *cuda_stream,
                mpt_ctx **out);
+
+/* mpt_workspace_bytes / mpt_create for any optimizer of the list above (mpt_create is the SGD
+ * case: kind MPT_OPT_SGD with the given lr and momentum). */
+int mpt_workspace_bytes_opt(const mpt_layer_desc *layers, int n_layers, int max_batch, const mpt_optimizer *opt,
+                            size_t *bytes_out);
+int mpt_create_opt(const mpt_layer_desc *layers, int n_layers, float S, const mpt_optimizer *opt, int max_batch,
+                   void *workspace_dev, size_t workspace_bytes, void *cuda_stream, mpt_ctx **out);
 
 /* Upload one layer's FP32 master weights [out, in] from the host and round them
  * to the FP16 working copy (section 3.1).  n must equal out*in.  Synchronous. */
@@ -198,6 +235,11 @@ int mpt_get_scale(mpt_ctx *ctx, float *S_out);
 int mpt_get_tensor(mpt_ctx *ctx, int kind, int layer, void *dst_host, size_t bytes);
 int mpt_set_grad(mpt_ctx *ctx, int layer, const uint16_t *src_host, size_t n);
 int mpt_set_momentum(mpt_ctx *ctx, int layer, const float *src_host, size_t n);
+/* Checkpoint hooks for Adam: the second state of a layer, and the running products beta1^t,
+ * beta2^t (both 1 before the first applied step).  Synchronous. */
+int mpt_set_state2(mpt_ctx *ctx, int layer, const float *src_host, size_t n);
+int mpt_get_adam_products(mpt_ctx *ctx, float *b1t_out, float *b2t_out);
+int mpt_set_adam_products(mpt_ctx *ctx, float b1t, float b2t);
 
 /* Number of kernels this context has launched since creation (bookkeeping for
  * benchmarks). */
@@ -273,6 +315,13 @@ int mpt_grad_nonfinite(const uint16_t *g16_dev, size_t n, float inv_S, uint32_t 
 int mpt_update_flat(const uint16_t *g16_dev, float *w32_dev, float *v_dev, uint16_t *w16_dev, size_t n,
                     float inv_S, float lr, float mu, int use_momentum, int detect, uint32_t *flags_dev,
                     void *cuda_stream);
+
+/* The same pass for any optimizer of mpt_optimizer (kind, weight decay).  s1_dev / s2_dev: FP32
+ * states (null when the kind does not use them).  b1t / b2t: for Adam, beta1^t and beta2^t
+ * INCLUDING this step (the caller keeps the products); ignored otherwise. */
+int mpt_update_flat_opt(const mpt_optimizer *opt, const uint16_t *g16_dev, float *w32_dev, float *s1_dev, float *s2_dev,
+                        uint16_t *w16_dev, size_t n, float inv_S, float b1t, float b2t, int detect, uint32_t *flags_dev,
+                        void *cuda_stream);
 
 /* Softmax cross-entropy forward and scaled backward (sections 3.2, 3.3), arithmetic
  * as in mpt_backward_scaled.  z_dev/dz_dev: FP16 [B, C] with pitches ldz/lddz

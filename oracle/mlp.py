@@ -41,6 +41,11 @@ class OracleMLP:
         self.w16 = [None] * len(self.layers)
         self.v = [np.zeros((o, i), dtype=np.float32) for (i, o, _) in self.layers]
         self.g16 = [np.zeros((o, i), dtype=np.uint16) for (i, o, _) in self.layers]
+        # optimizer: kind 0 SGD(+momentum) by default; set_optimizer switches (state s1/s2 start at zero)
+        self.opt = dict(kind=mpo.OPT_SGD, b2=np.float32(0.0), eps=np.float32(0.0), wd=np.float32(0.0))
+        self.s2 = [np.zeros((o, i), dtype=np.float32) for (i, o, _) in self.layers]
+        self.b1t = np.float32(1.0)     # running products beta1^t, beta2^t over applied steps (Adam)
+        self.b2t = np.float32(1.0)
         self.dynamic = None    # (growth_interval, backoff, growth, min_scale, max_scale) or None
         self.clean_steps = 0
         self.acts = None       # [a_0 .. a_L], uint16
@@ -82,6 +87,13 @@ class OracleMLP:
                                               mask=self.acts[l] if self.layers[l - 1][2] else None)
         return loss
 
+    def set_optimizer(self, kind, lr, mu=0.0, b2=0.0, eps=0.0, wd=0.0):
+        """kind: mpo.OPT_*; mu is the momentum (SGD, Nesterov) or beta1 (Adam)."""
+        self.opt = dict(kind=int(kind), b2=np.float32(b2), eps=np.float32(eps), wd=np.float32(wd))
+        self.lr = np.float32(lr)
+        self.mu = np.float32(mu)
+        self.use_momentum = (kind == mpo.OPT_SGD and float(mu) != 0.0) or kind != mpo.OPT_SGD
+
     def set_dynamic_scale(self, growth_interval, min_scale, max_scale, backoff=0.5, growth=2.0):
         self.dynamic = (int(growth_interval), np.float32(backoff), np.float32(growth), np.float32(min_scale),
                         np.float32(max_scale))
@@ -95,9 +107,22 @@ class OracleMLP:
         for g in self.g16:
             overflow |= mpo.grad_nonfinite(g, inv)
         if not overflow:
-            for l in range(len(self.layers)):
-                mpo.update_apply(self.g16[l], self.w32[l], self.v[l], self.w16[l], inv, self.lr, self.mu,
-                                 self.use_momentum)
+            kind = self.opt["kind"]
+            if kind == mpo.OPT_SGD and float(self.opt["wd"]) == 0.0:
+                for l in range(len(self.layers)):
+                    mpo.update_apply(self.g16[l], self.w32[l], self.v[l], self.w16[l], inv, self.lr, self.mu,
+                                     self.use_momentum)
+            else:
+                if kind == mpo.OPT_ADAM:       # bias corrections use the products including this step
+                    self.b1t = np.float32(self.b1t * self.mu)
+                    self.b2t = np.float32(self.b2t * self.opt["b2"])
+                bc1 = np.float32(1.0) - self.b1t
+                bc2 = np.float32(1.0) - self.b2t
+                for l in range(len(self.layers)):
+                    s1 = self.v[l] if (kind != mpo.OPT_SGD or self.use_momentum) else None
+                    s2 = self.s2[l] if kind == mpo.OPT_ADAM else None
+                    mpo.update_apply_opt(kind, self.g16[l], self.w32[l], s1, s2, self.w16[l], inv, self.lr, self.mu,
+                                         self.opt["b2"], self.opt["eps"], self.opt["wd"], bc1, bc2)
         if self.dynamic is not None:
             interval, backoff, growth, smin, smax = self.dynamic
             if overflow:

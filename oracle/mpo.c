@@ -328,3 +328,78 @@ void mpo_update_apply(const uint16_t *g16, float *w32, float *v, uint16_t *w16,
         w16[e] = mpo_f2h(w);
     }
 }
+
+/*
+ * Other optimizer steps on the binary32 master copy (the paper's experiments use Nesterov
+ * momentum for the speech models, section 4.3; Adagrad for bigLSTM, section 4.5; Adam for
+ * DCGAN, section 4.6; section 3.2 requires weight decay and other gradient-related terms to
+ * act on the UNSCALED gradient).  The paper gives no formulas; the textbook forms are used,
+ * every line one separately rounded binary32 operation, in this order:
+ *   g = h2f(g16) * inv_S
+ *   if wd != 0:          t = wd * w ; g = g + t                       (L2 weight decay)
+ *   kind 1 Nesterov:     a = mu * s1 ; s1 = a + g ; b = mu * s1 ; c = g + b ; u = lr * c
+ *   kind 2 Adagrad:      q = g * g ; s1 = s1 + q ; r = sqrtf(s1) ; d = r + eps ; c = g / d ; u = lr * c
+ *   kind 3 Adam:         a = b1 * s1 ; b = omb1 * g ; s1 = a + b
+ *                        q = g * g ; c = b2 * s2 ; d = omb2 * q ; s2 = c + d
+ *                        mh = s1 / bc1 ; vh = s2 / bc2 ; r = sqrtf(vh) ; e = r + eps ; f = mh / e ; u = lr * f
+ *     with omb1 = 1 - b1, omb2 = 1 - b2, bc1 = 1 - b1^t, bc2 = 1 - b2^t, where b1^t, b2^t are
+ *     running binary32 products passed in by the caller (t counts applied, not skipped, steps)
+ *   kind 0 SGD:          momentum (s1 != NULL): a = mu * s1 ; s1 = a + g ; u = lr * s1 ; else u = lr * g
+ *   w = w - u ; w16 = rn16(w)
+ * mu doubles as b1.  s1 / s2 may be NULL when the kind does not use them.
+ */
+void mpo_update_apply_opt(int kind, const uint16_t *g16, float *w32, float *s1, float *s2, uint16_t *w16,
+                          size_t n, float inv_S, float lr, float mu, float b2, float eps, float wd,
+                          float bc1, float bc2)
+{
+    const float omb1 = 1.0f - mu, omb2 = 1.0f - b2;
+#pragma omp parallel for schedule(static)
+    for (size_t i = 0; i < n; i++) {
+        float w = w32[i];
+        float g = mpo_h2f(g16[i]) * inv_S;
+        if (wd != 0.0f) { float t = wd * w; g = g + t; }
+        float u;
+        if (kind == 1) {
+            float a = mu * s1[i];
+            float v = a + g;
+            s1[i] = v;
+            float b = mu * v;
+            float c = g + b;
+            u = lr * c;
+        } else if (kind == 2) {
+            float q = g * g;
+            float h = s1[i] + q;
+            s1[i] = h;
+            float r = sqrtf(h);
+            float d = r + eps;
+            float c = g / d;
+            u = lr * c;
+        } else if (kind == 3) {
+            float a = mu * s1[i];
+            float b = omb1 * g;
+            float m = a + b;
+            s1[i] = m;
+            float q = g * g;
+            float c = b2 * s2[i];
+            float d = omb2 * q;
+            float v = c + d;
+            s2[i] = v;
+            float mh = m / bc1;
+            float vh = v / bc2;
+            float r = sqrtf(vh);
+            float e = r + eps;
+            float f = mh / e;
+            u = lr * f;
+        } else if (s1) {
+            float a = mu * s1[i];
+            float v = a + g;
+            s1[i] = v;
+            u = lr * v;
+        } else {
+            u = lr * g;
+        }
+        w = w - u;
+        w32[i] = w;
+        w16[i] = mpo_f2h(w);
+    }
+}

@@ -67,6 +67,9 @@ def lib() -> ctypes.CDLL:
         L.mpo_update_apply.restype = None
         L.mpo_update_apply.argtypes = [c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_size_t,
                                        c.c_float, c.c_float, c.c_float, c.c_int]
+        L.mpo_update_apply_opt.restype = None
+        L.mpo_update_apply_opt.argtypes = [c.c_int, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p,
+                                           c.c_size_t] + [c.c_float] * 8
         _lib = L
     return _lib
 
@@ -200,3 +203,16 @@ def update_apply(g16, w32, v, w16, inv_S, lr, mu, use_momentum) -> None:
         assert v is not None and v.dtype == np.float32
     lib().mpo_update_apply(_ptr(g), _ptr(w32), _ptr(v) if use_momentum else None, _ptr(w16), g.size,
                            float(inv_S), float(lr), float(mu), int(bool(use_momentum)))
+
+
+OPT_SGD, OPT_NESTEROV, OPT_ADAGRAD, OPT_ADAM = 0, 1, 2, 3
+
+
+def update_apply_opt(kind, g16, w32, s1, s2, w16, inv_S, lr, mu, b2=0.0, eps=0.0, wd=0.0, bc1=1.0, bc2=1.0) -> None:
+    """In-place optimizer step of the given kind on contiguous arrays (see mpo.c for the op order)."""
+    g = _u16(g16)
+    for a in (g, w32, w16, s1, s2):
+        if a is not None:
+            assert a.flags["C_CONTIGUOUS"]
+    lib().mpo_update_apply_opt(int(kind), _ptr(g), _ptr(w32), _ptr(s1), _ptr(s2), _ptr(w16), g.size, float(inv_S),
+                               float(lr), float(mu), float(b2), float(eps), float(wd), float(bc1), float(bc2))

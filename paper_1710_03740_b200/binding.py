@@ -20,10 +20,12 @@ ERR = {-1: "MPT_ERR_INVALID_ARG", -2: "MPT_ERR_SHAPE", -3: "MPT_ERR_STATE", -4: 
        -5: "MPT_ERR_CUDA", -6: "MPT_ERR_TIMEOUT", -7: "MPT_ERR_INTERNAL"}
 OP_FWD, OP_DGRAD, OP_WGRAD = 0, 1, 2
 GEMM_RELU, GEMM_FORCE_SIMT, GEMM_FORCE_TC, GEMM_FORCE_PAIR = 1, 2, 4, 8
-T_W16, T_GRAD16, T_ACT16, T_DACT16, T_MOMENTUM32, T_MASTER32 = range(6)
+T_W16, T_GRAD16, T_ACT16, T_DACT16, T_MOMENTUM32, T_MASTER32, T_STATE2_32 = range(7)
+OPT_SGD, OPT_NESTEROV, OPT_ADAGRAD, OPT_ADAM = 0, 1, 2, 3
 
 # every symbol include/mpt.h declares
-EXPORTS = ["mpt_workspace_bytes", "mpt_create", "mpt_set_master", "mpt_forward", "mpt_backward_scaled",
+EXPORTS = ["mpt_workspace_bytes", "mpt_create", "mpt_workspace_bytes_opt", "mpt_create_opt", "mpt_set_state2",
+           "mpt_get_adam_products", "mpt_set_adam_products", "mpt_update_flat_opt", "mpt_set_master", "mpt_forward", "mpt_backward_scaled",
            "mpt_step", "mpt_get_master", "mpt_train_step_host", "mpt_stage_batch_host",
            "mpt_train_step_staged", "mpt_set_scale", "mpt_set_lr", "mpt_set_dynamic_scale", "mpt_get_scale",
            "mpt_get_tensor", "mpt_set_grad", "mpt_set_momentum", "mpt_launch_count", "mpt_profile",
@@ -42,6 +44,12 @@ class LayerDesc(C.Structure):
     _fields_ = [("in_features", C.c_int32), ("out_features", C.c_int32), ("relu", C.c_int32)]
 
 
+class Optimizer(C.Structure):
+    """mpt_optimizer: kind (OPT_*), lr, momentum (or Adam beta1), beta2, eps, weight_decay."""
+    _fields_ = [("kind", C.c_int32), ("lr", C.c_float), ("momentum", C.c_float), ("beta2", C.c_float),
+                ("eps", C.c_float), ("weight_decay", C.c_float)]
+
+
 _lib = None
 
 
@@ -56,6 +64,12 @@ def lib() -> C.CDLL:
     vp, i32, u32, f32, sz = C.c_void_p, C.c_int, C.c_uint, C.c_float, C.c_size_t
     L.mpt_workspace_bytes.argtypes = [C.POINTER(LayerDesc), i32, i32, i32, C.POINTER(sz)]
     L.mpt_create.argtypes = [C.POINTER(LayerDesc), i32, f32, f32, f32, i32, vp, sz, vp, C.POINTER(vp)]
+    L.mpt_workspace_bytes_opt.argtypes = [C.POINTER(LayerDesc), i32, i32, C.POINTER(Optimizer), C.POINTER(sz)]
+    L.mpt_create_opt.argtypes = [C.POINTER(LayerDesc), i32, f32, C.POINTER(Optimizer), i32, vp, sz, vp, C.POINTER(vp)]
+    L.mpt_set_state2.argtypes = [vp, i32, vp, sz]
+    L.mpt_get_adam_products.argtypes = [vp, C.POINTER(f32), C.POINTER(f32)]
+    L.mpt_set_adam_products.argtypes = [vp, f32, f32]
+    L.mpt_update_flat_opt.argtypes = [C.POINTER(Optimizer), vp, vp, vp, vp, vp, sz, f32, f32, f32, i32, vp, vp]
     L.mpt_set_master.argtypes = [vp, i32, vp, sz]
     L.mpt_forward.argtypes = [vp, vp, i32]
     L.mpt_backward_scaled.argtypes = [vp, vp, C.POINTER(f32)]
@@ -134,20 +148,26 @@ def mpt_workspace_bytes(layers, max_batch, use_momentum) -> int:
 class Context:
     """One mpt_ctx over a torch-allocated workspace.  Method names follow the C calls."""
 
-    def __init__(self, layers, S, lr, momentum=0.0, max_batch=1, device="cuda:0", stream=None):
+    def __init__(self, layers, S, lr, momentum=0.0, max_batch=1, device="cuda:0", stream=None, optimizer=None):
+        """optimizer: an Optimizer struct; default SGD with the given lr and momentum."""
         import torch
         self.layers = [(int(i), int(o), int(r)) for (i, o, r) in layers]
         self.device = torch.device(device)
         self.stream = stream
-        nbytes = mpt_workspace_bytes(self.layers, max_batch, momentum != 0.0)
+        opt = optimizer if optimizer is not None else Optimizer(OPT_SGD, float(lr), float(momentum), 0.0, 0.0, 0.0)
+        self.optimizer = opt
+        out = C.c_size_t(0)
+        _check(lib().mpt_workspace_bytes_opt(_layer_array(self.layers), len(self.layers), int(max_batch), C.byref(opt),
+                                             C.byref(out)))
+        nbytes = int(out.value)
         with torch.cuda.device(self.device):
             self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
             base = self.workspace.data_ptr()
             self._ws_ptr = (base + 255) // 256 * 256
             self._ctx = C.c_void_p()
-            _check(lib().mpt_create(_layer_array(self.layers), len(self.layers), float(S), float(lr), float(momentum),
-                                    int(max_batch), C.c_void_p(self._ws_ptr), nbytes, _stream_ptr(stream),
-                                    C.byref(self._ctx)))
+            _check(lib().mpt_create_opt(_layer_array(self.layers), len(self.layers), float(S), C.byref(opt),
+                                        int(max_batch), C.c_void_p(self._ws_ptr), nbytes, _stream_ptr(stream),
+                                        C.byref(self._ctx)))
         self.workspace_bytes = nbytes
         self.batch = 0
 
@@ -229,7 +249,7 @@ class Context:
         i, o, _ = self.layers[layer]
         if kind in (T_W16, T_GRAD16):
             out = np.empty((o, i), dtype=np.uint16)
-        elif kind in (T_MOMENTUM32, T_MASTER32):
+        elif kind in (T_MOMENTUM32, T_MASTER32, T_STATE2_32):
             out = np.empty((o, i), dtype=np.float32)
         else:
             out = np.empty((self.batch, o), dtype=np.uint16)
@@ -256,6 +276,18 @@ class Context:
         _check(lib().mpt_profile_read(self._ctx, ms, work, n), self._ctx)
         names = ("gemm", "update", "softmax", "other")
         return {names[k]: (float(ms[k]), float(work[k]), int(n[k])) for k in range(4)}
+
+    def set_state2(self, layer, v):
+        v = np.ascontiguousarray(v, dtype=np.float32)
+        _check(lib().mpt_set_state2(self._ctx, layer, _hptr(v), v.size), self._ctx)
+
+    def get_adam_products(self):
+        a, b = C.c_float(0.0), C.c_float(0.0)
+        _check(lib().mpt_get_adam_products(self._ctx, C.byref(a), C.byref(b)), self._ctx)
+        return float(a.value), float(b.value)
+
+    def set_adam_products(self, b1t, b2t):
+        _check(lib().mpt_set_adam_products(self._ctx, float(b1t), float(b2t)), self._ctx)
 
     def launch_count(self):
         n = C.c_longlong(0)
@@ -297,6 +329,12 @@ def mpt_grad_nonfinite(g16, n, inv_S, flag, stream=None):
 def mpt_update_flat(g16, w32, v, w16, n, inv_S, lr, mu, use_momentum, detect, flags, stream=None):
     _check(lib().mpt_update_flat(_dptr(g16), _dptr(w32), _dptr(v), _dptr(w16), n, float(inv_S), float(lr), float(mu),
                                  int(bool(use_momentum)), int(bool(detect)), _dptr(flags), _stream_ptr(stream)))
+
+
+def mpt_update_flat_opt(opt, g16, w32, s1, s2, w16, n, inv_S, b1t, b2t, detect, flags, stream=None):
+    _check(lib().mpt_update_flat_opt(C.byref(opt), _dptr(g16), _dptr(w32), _dptr(s1), _dptr(s2), _dptr(w16), n,
+                                     float(inv_S), float(b1t), float(b2t), int(bool(detect)), _dptr(flags),
+                                     _stream_ptr(stream)))
 
 
 def mpt_softmax_ce(z, ldz, labels, B, Cn, S, dz, lddz, row_loss, loss, bad_labels=None, stream=None):

@@ -28,11 +28,33 @@ struct Layer {
 
 struct Plan {
     size_t total = 0, P_pad = 0;
-    size_t off_status = 0, off_master = 0, off_mom = 0, off_w16 = 0, off_g16 = 0, off_x[2] = {0, 0},
+    size_t off_status = 0, off_master = 0, off_mom = 0, off_state2 = 0, off_w16 = 0, off_g16 = 0, off_x[2] = {0, 0},
            off_labels[2] = {0, 0}, off_rowloss = 0, off_splitk = 0, splitk_bytes = 0;
     std::vector<size_t> off_act, off_dact, lay_off;
     std::vector<int> ld_out;
 };
+
+int opt_states(const mpt_optimizer &o)
+{
+    switch (o.kind) {
+        case MPT_OPT_SGD: return o.momentum != 0.0f ? 1 : 0;
+        case MPT_OPT_NESTEROV:
+        case MPT_OPT_ADAGRAD: return 1;
+        default: return 2;
+    }
+}
+
+bool valid_optimizer(const mpt_optimizer *o)
+{
+    if (!o) return false;
+    if (o->kind < MPT_OPT_SGD || o->kind > MPT_OPT_ADAM) return false;
+    if (!std::isfinite(o->lr)) return false;
+    if (!(o->momentum >= 0.0f && o->momentum < 1.0f)) return false;
+    if (!(o->weight_decay >= 0.0f) || !std::isfinite(o->weight_decay)) return false;
+    if (o->kind == MPT_OPT_ADAM && !(o->beta2 >= 0.0f && o->beta2 < 1.0f)) return false;
+    if ((o->kind == MPT_OPT_ADAM || o->kind == MPT_OPT_ADAGRAD) && (!(o->eps >= 0.0f) || !std::isfinite(o->eps))) return false;
+    return true;
+}
 
 bool valid_scale(float S)
 {
@@ -52,7 +74,7 @@ int validate_layers(const mpt_layer_desc *layers, int n_layers, int max_batch)
     return MPT_OK;
 }
 
-void make_plan(const mpt_layer_desc *layers, int L, int max_batch, bool mom, Plan &pl)
+void make_plan(const mpt_layer_desc *layers, int L, int max_batch, int n_states, Plan &pl)
 {
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
@@ -65,7 +87,8 @@ void make_plan(const mpt_layer_desc *layers, int L, int max_batch, bool mom, Pla
     }
     pl.P_pad = P;
     pl.off_master = take(P * 4);
-    pl.off_mom = mom ? take(P * 4) : 0;
+    pl.off_mom = n_states >= 1 ? take(P * 4) : 0;
+    pl.off_state2 = n_states >= 2 ? take(P * 4) : 0;
     pl.off_w16 = take(P * 2);
     pl.off_g16 = take(P * 2);
     pl.off_act.resize(L); pl.off_dact.resize(L); pl.ld_out.resize(L);
@@ -104,7 +127,10 @@ void make_plan(const mpt_layer_desc *layers, int L, int max_batch, bool mom, Pla
 struct mpt_ctx {
     std::vector<Layer> layers;
     float S, lr, mu;
-    bool use_momentum;
+    bool use_momentum;          // first optimizer state in use
+    int opt_kind = MPT_OPT_SGD;
+    float beta2 = 0.0f, eps = 0.0f, wd = 0.0f;
+    float *state2 = nullptr;
     int max_batch;
     cudaStream_t stream;
     uint8_t *ws;
@@ -183,6 +209,16 @@ int push_scale(mpt_ctx *c)
     memcpy(&w[1], &inv, 4);
     w[2] = 0;
     CK(cudaMemcpyAsync(c->status + ST_SCALE, w, sizeof w, cudaMemcpyHostToDevice, c->stream), "scale upload");
+    CK(cudaStreamSynchronize(c->stream), "stream synchronize");
+    return MPT_OK;
+}
+
+int push_adam_products(mpt_ctx *c, float b1t, float b2t)
+{
+    uint32_t w[2];
+    memcpy(&w[0], &b1t, 4);
+    memcpy(&w[1], &b2t, 4);
+    CK(cudaMemcpyAsync(c->status + ST_B1T, w, sizeof w, cudaMemcpyHostToDevice, c->stream), "optimizer state upload");
     CK(cudaStreamSynchronize(c->stream), "stream synchronize");
     return MPT_OK;
 }
@@ -306,18 +342,26 @@ int do_step(mpt_ctx *c)
     CK(cudaMemsetAsync(c->status + ST_OVERFLOW_SEEN, 0, sizeof(uint32_t), c->stream), "status clear");
     cudaError_t e;
     {
-        ProfSpan span(c, MPT_PROF_UPDATE, (c->use_momentum ? 20.0 : 12.0) * (double)c->plan.P_pad);
-        e = launch_update(c->g16, c->master, c->mom, c->w16, c->plan.P_pad, inv, c->lr, c->mu, c->use_momentum,
-                          c->status + ST_OVERFLOW, c->stream, (const float *)(c->status + ST_INV_SCALE));
+        const double bytes_per_param = 12.0 + 8.0 * (c->use_momentum ? 1 : 0) + 8.0 * (c->state2 ? 1 : 0);
+        ProfSpan span(c, MPT_PROF_UPDATE, bytes_per_param * (double)c->plan.P_pad);
+        if (c->opt_kind == MPT_OPT_SGD && c->wd == 0.0f)
+            e = launch_update(c->g16, c->master, c->mom, c->w16, c->plan.P_pad, inv, c->lr, c->mu, c->use_momentum,
+                              c->status + ST_OVERFLOW, c->stream, (const float *)(c->status + ST_INV_SCALE));
+        else
+            e = launch_update_opt(c->opt_kind, c->g16, c->master, c->mom, c->state2, c->w16, c->plan.P_pad, inv, c->lr, c->mu,
+                                  c->beta2, c->eps, c->wd, 1.0f, 1.0f, c->status + ST_OVERFLOW, c->stream,
+                                  (const float *)(c->status + ST_INV_SCALE),
+                                  c->opt_kind == MPT_OPT_ADAM ? (const float *)(c->status + ST_B1T) : nullptr);
     }
     c->launches++;
     if (e != cudaSuccess) return cuda_fail(c, e, "update launch");
-    if (c->dynamic_scale) {
+    if (c->dynamic_scale || c->opt_kind == MPT_OPT_ADAM) {
+        // end-of-step bookkeeping on the device: loss scale and Adam's beta^t move only on applied steps
         ProfSpan span(c, MPT_PROF_OTHER, 0.0);
-        e = launch_scale_adjust(c->status, c->growth_interval, c->scale_backoff, c->scale_growth, c->scale_min,
-                                c->scale_max, c->stream);
+        e = launch_post_step(c->status, c->dynamic_scale ? c->growth_interval : 0, c->scale_backoff, c->scale_growth,
+                             c->scale_min, c->scale_max, c->opt_kind == MPT_OPT_ADAM ? 1 : 0, c->mu, c->beta2, c->stream);
         c->launches++;
-        if (e != cudaSuccess) return cuda_fail(c, e, "scale adjust launch");
+        if (e != cudaSuccess) return cuda_fail(c, e, "post-step launch");
     }
     return MPT_OK;
 }
@@ -342,7 +386,20 @@ int mpt_workspace_bytes(const mpt_layer_desc *layers, int n_layers, int max_batc
     int r = validate_layers(layers, n_layers, max_batch);
     if (r != MPT_OK) return r;
     Plan pl;
-    make_plan(layers, n_layers, max_batch, use_momentum != 0, pl);
+    make_plan(layers, n_layers, max_batch, use_momentum != 0 ? 1 : 0, pl);
+    *bytes_out = pl.total;
+    return MPT_OK;
+}
+
+int mpt_workspace_bytes_opt(const mpt_layer_desc *layers, int n_layers, int max_batch, const mpt_optimizer *opt,
+                            size_t *bytes_out)
+{
+    if (!bytes_out || !opt) return MPT_ERR_INVALID_ARG;
+    int r = validate_layers(layers, n_layers, max_batch);
+    if (r != MPT_OK) return r;
+    if (!valid_optimizer(opt)) return MPT_ERR_INVALID_ARG;
+    Plan pl;
+    make_plan(layers, n_layers, max_batch, opt_states(*opt), pl);
     *bytes_out = pl.total;
     return MPT_OK;
 }
@@ -350,18 +407,28 @@ int mpt_workspace_bytes(const mpt_layer_desc *layers, int n_layers, int max_batc
 int mpt_create(const mpt_layer_desc *layers, int n_layers, float S, float lr, float momentum, int max_batch,
                void *workspace_dev, size_t workspace_bytes, void *cuda_stream, mpt_ctx **out)
 {
+    mpt_optimizer opt = {MPT_OPT_SGD, lr, momentum, 0.0f, 0.0f, 0.0f};
+    return mpt_create_opt(layers, n_layers, S, &opt, max_batch, workspace_dev, workspace_bytes, cuda_stream, out);
+}
+
+int mpt_create_opt(const mpt_layer_desc *layers, int n_layers, float S, const mpt_optimizer *opt, int max_batch,
+                   void *workspace_dev, size_t workspace_bytes, void *cuda_stream, mpt_ctx **out)
+{
     if (!out) return MPT_ERR_INVALID_ARG;
     *out = nullptr;
     if (!workspace_dev) return MPT_ERR_INVALID_ARG;
     int r = validate_layers(layers, n_layers, max_batch);
     if (r != MPT_OK) return r;
-    if (!valid_scale(S) || !std::isfinite(lr) || !(momentum >= 0.0f && momentum < 1.0f)) return MPT_ERR_INVALID_ARG;
+    if (!valid_scale(S) || !valid_optimizer(opt)) return MPT_ERR_INVALID_ARG;
     if ((uintptr_t)workspace_dev % 256) return MPT_ERR_WORKSPACE;
     mpt_ctx *c = new (std::nothrow) mpt_ctx();
     if (!c) return MPT_ERR_INTERNAL;
-    c->use_momentum = momentum != 0.0f;
-    make_plan(layers, n_layers, max_batch, c->use_momentum, c->plan);
+    const int n_states = opt_states(*opt);
+    c->use_momentum = n_states >= 1;
+    c->opt_kind = opt->kind; c->beta2 = opt->beta2; c->eps = opt->eps; c->wd = opt->weight_decay;
+    make_plan(layers, n_layers, max_batch, n_states, c->plan);
     if (workspace_bytes < c->plan.total) { delete c; return MPT_ERR_WORKSPACE; }
+    const float lr = opt->lr, momentum = opt->momentum;
     c->S = S; c->lr = lr; c->mu = momentum; c->max_batch = max_batch;
     c->stream = (cudaStream_t)cuda_stream;
     c->ws = (uint8_t *)workspace_dev;
@@ -369,6 +436,7 @@ int mpt_create(const mpt_layer_desc *layers, int n_layers, float S, float lr, fl
     c->status = (uint32_t *)(c->ws + pl.off_status);
     c->master = (float *)(c->ws + pl.off_master);
     c->mom = c->use_momentum ? (float *)(c->ws + pl.off_mom) : nullptr;
+    c->state2 = n_states >= 2 ? (float *)(c->ws + pl.off_state2) : nullptr;
     c->w16 = (uint16_t *)(c->ws + pl.off_w16);
     c->g16 = (uint16_t *)(c->ws + pl.off_g16);
     for (int k = 0; k < 2; k++) {
@@ -395,6 +463,7 @@ int mpt_create(const mpt_layer_desc *layers, int n_layers, float S, float lr, fl
     cudaError_t e = cudaMemsetAsync(c->ws, 0, pl.total, c->stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
     if (e == cudaSuccess && push_scale(c) != MPT_OK) e = cudaErrorUnknown;
+    if (e == cudaSuccess && push_adam_products(c, 1.0f, 1.0f) != MPT_OK) e = cudaErrorUnknown;
     for (int k = 0; k < 2 && e == cudaSuccess; k++) {
         e = cudaEventCreateWithFlags(&c->staged_ev[k], cudaEventDisableTiming);
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->used_ev[k], cudaEventDisableTiming);
@@ -672,6 +741,9 @@ int mpt_get_tensor(mpt_ctx *c, int kind, int layer, void *dst_host, size_t bytes
         case MPT_T_MOMENTUM32:
             if (!c->use_momentum) return fail(c, MPT_ERR_STATE, "context has no momentum buffer");
             src = c->mom + ly.off; rows = 1; row_bytes = ly.n * 4; pitch = row_bytes; break;
+        case MPT_T_STATE2_32:
+            if (!c->state2) return fail(c, MPT_ERR_STATE, "context has no second optimizer state");
+            src = c->state2 + ly.off; rows = 1; row_bytes = ly.n * 4; pitch = row_bytes; break;
         case MPT_T_ACT16:
         case MPT_T_DACT16:
             if (c->batch < 1) return fail(c, MPT_ERR_STATE, "no forward pass yet");
@@ -716,6 +788,41 @@ int mpt_set_momentum(mpt_ctx *c, int layer, const float *src_host, size_t n)
     CK(cudaMemcpyAsync(c->mom + ly.off, src_host, n * 4, cudaMemcpyHostToDevice, c->stream), "momentum upload");
     CK(cudaStreamSynchronize(c->stream), "stream synchronize");
     return MPT_OK;
+}
+
+int mpt_set_state2(mpt_ctx *c, int layer, const float *src_host, size_t n)
+{
+    int r = usable(c);
+    if (r != MPT_OK) return r;
+    if (!src_host) return fail(c, MPT_ERR_INVALID_ARG, "null source");
+    if (layer < 0 || layer >= (int)c->layers.size()) return fail(c, MPT_ERR_INVALID_ARG, "layer index");
+    if (!c->state2) return fail(c, MPT_ERR_STATE, "context has no second optimizer state");
+    Layer &ly = c->layers[layer];
+    if (n != ly.n) return fail(c, MPT_ERR_SHAPE, "n must equal out*in");
+    CK(cudaMemcpyAsync(c->state2 + ly.off, src_host, n * 4, cudaMemcpyHostToDevice, c->stream), "state upload");
+    CK(cudaStreamSynchronize(c->stream), "stream synchronize");
+    return MPT_OK;
+}
+
+int mpt_get_adam_products(mpt_ctx *c, float *b1t_out, float *b2t_out)
+{
+    int r = usable(c);
+    if (r != MPT_OK) return r;
+    if (!b1t_out || !b2t_out) return fail(c, MPT_ERR_INVALID_ARG, "null output");
+    uint32_t st[ST_WORDS];
+    r = read_status(c, st);
+    if (r != MPT_OK) return r;
+    memcpy(b1t_out, &st[ST_B1T], 4);
+    memcpy(b2t_out, &st[ST_B2T], 4);
+    return MPT_OK;
+}
+
+int mpt_set_adam_products(mpt_ctx *c, float b1t, float b2t)
+{
+    int r = usable(c);
+    if (r != MPT_OK) return r;
+    if (!std::isfinite(b1t) || !std::isfinite(b2t)) return fail(c, MPT_ERR_INVALID_ARG, "products must be finite");
+    return push_adam_products(c, b1t, b2t);
 }
 
 // ---------------------------------------------------------- stateless launchers
@@ -794,6 +901,29 @@ int mpt_update_flat(const uint16_t *g16_dev, float *w32_dev, float *v_dev, uint1
         e = cudaMemsetAsync(flags_dev + 1, 0, sizeof(uint32_t), st);
     }
     if (e == cudaSuccess) e = launch_update(g16_dev, w32_dev, v_dev, w16_dev, n, inv_S, lr, mu, use_momentum != 0, flags_dev, st);
+    return e == cudaSuccess ? MPT_OK : MPT_ERR_CUDA;
+}
+
+int mpt_update_flat_opt(const mpt_optimizer *opt, const uint16_t *g16_dev, float *w32_dev, float *s1_dev, float *s2_dev,
+                        uint16_t *w16_dev, size_t n, float inv_S, float b1t, float b2t, int detect, uint32_t *flags_dev,
+                        void *cuda_stream)
+{
+    if (!g16_dev || !w32_dev || !w16_dev || !flags_dev) return MPT_ERR_INVALID_ARG;
+    if (!valid_optimizer(opt)) return MPT_ERR_INVALID_ARG;
+    const int ns = opt_states(*opt);
+    if ((ns >= 1 && !s1_dev) || (ns >= 2 && !s2_dev)) return MPT_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    cudaError_t e;
+    if (detect) {
+        e = cudaMemsetAsync(flags_dev, 0, 2 * sizeof(uint32_t), st);
+        if (e == cudaSuccess) e = launch_grad_nonfinite(g16_dev, n, inv_S, flags_dev, st);
+    } else {
+        e = cudaMemsetAsync(flags_dev + 1, 0, sizeof(uint32_t), st);
+    }
+    if (e == cudaSuccess)
+        e = launch_update_opt(opt->kind, g16_dev, w32_dev, ns >= 1 ? s1_dev : nullptr, ns >= 2 ? s2_dev : nullptr, w16_dev, n,
+                              inv_S, opt->lr, opt->momentum, opt->beta2, opt->eps, opt->weight_decay, b1t, b2t, flags_dev, st,
+                              nullptr, nullptr);
     return e == cudaSuccess ? MPT_OK : MPT_ERR_CUDA;
 }
 

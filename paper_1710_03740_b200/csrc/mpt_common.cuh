@@ -20,6 +20,8 @@ enum StatusWord : int {
     ST_SCALE = 5,         // float: loss scale S the next backward / master pass will use
     ST_INV_SCALE = 6,     // float: 1.0f / S (one FP32 division)
     ST_CLEAN_STEPS = 7,   // consecutive steps without overflow since S last changed (dynamic scaling)
+    ST_B1T = 8,           // float: beta1^t over the applied (not skipped) steps (Adam)
+    ST_B2T = 9,           // float: beta2^t
     ST_WORDS = 16
 };
 
@@ -61,6 +63,19 @@ cudaError_t launch_update(const uint16_t *g16, float *w32, float *v, uint16_t *w
 cudaError_t launch_softmax_ce(const uint16_t *z, int ldz, const int32_t *labels, int B, int C, float S,
                               uint16_t *dz, int lddz, float *row_loss, float *loss, uint32_t *bad_labels,
                               cudaStream_t st, int *n_launches, const float *S_dev = nullptr);
+// Optimizer steps other than SGD(+momentum), and weight decay (see mpt.h MPT_OPT_*).  s1 / s2:
+// FP32 state arrays (momentum or squared-gradient sum; Adam's second moment).  For Adam the
+// bias corrections are 1 - beta^t with beta^t either passed by value (b1t, b2t: the products
+// INCLUDING this step) or, when betat_dev is given, read as the products of the previous applied
+// steps from device memory and multiplied by beta once more in the kernel.
+cudaError_t launch_update_opt(int kind, const uint16_t *g16, float *w32, float *s1, float *s2, uint16_t *w16, size_t n,
+                              float inv_S, float lr, float mu, float b2, float eps, float wd, float b1t, float b2t,
+                              uint32_t *flags, cudaStream_t st, const float *inv_S_dev, const float *betat_dev);
+// End-of-step bookkeeping on the device (one thread): dynamic loss scale (if interval > 0) and
+// Adam's running products beta^t (if adam != 0); both only move on a step that was applied.
+cudaError_t launch_post_step(uint32_t *status, int interval, float backoff, float growth, float min_S, float max_S,
+                             int adam, float b1, float b2, cudaStream_t st);
+
 // Dynamic loss scaling (one thread): on overflow S <- max(S * backoff, min_S) and the clean-step
 // counter restarts; after `interval` clean steps S <- min(S * growth, max_S).  Rewrites the
 // ST_SCALE / ST_INV_SCALE / ST_CLEAN_STEPS words of the status block.

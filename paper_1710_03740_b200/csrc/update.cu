@@ -249,6 +249,194 @@ cudaError_t launch_update(const uint16_t *g16, float *w32, float *v, uint16_t *w
     return cudaGetLastError();
 }
 
+// ------------------------------------------- other optimizer steps, weight decay
+
+// One element; every operation rounded separately, in the order documented in mpt.h.
+template <int KIND, bool WD>
+__device__ __forceinline__ void opt1(uint32_t gh, float &w, float &s1, float &s2, float inv, float lr, float mu, float b2,
+                                     float omb1, float omb2, float eps, float wd, float bc1, float bc2, bool &bad)
+{
+    float g = __fmul_rn(h2f_bits(gh), inv);
+    bad |= f32_nonfinite(g);
+    if (WD) g = __fadd_rn(g, __fmul_rn(wd, w));
+    float u;
+    if (KIND == MPT_OPT_NESTEROV) {
+        s1 = __fadd_rn(__fmul_rn(mu, s1), g);
+        u = __fmul_rn(lr, __fadd_rn(g, __fmul_rn(mu, s1)));
+    } else if (KIND == MPT_OPT_ADAGRAD) {
+        s1 = __fadd_rn(s1, __fmul_rn(g, g));
+        u = __fmul_rn(lr, __fdiv_rn(g, __fadd_rn(__fsqrt_rn(s1), eps)));
+    } else if (KIND == MPT_OPT_ADAM) {
+        s1 = __fadd_rn(__fmul_rn(mu, s1), __fmul_rn(omb1, g));
+        s2 = __fadd_rn(__fmul_rn(b2, s2), __fmul_rn(omb2, __fmul_rn(g, g)));
+        const float mh = __fdiv_rn(s1, bc1), vh = __fdiv_rn(s2, bc2);
+        u = __fmul_rn(lr, __fdiv_rn(mh, __fadd_rn(__fsqrt_rn(vh), eps)));
+    } else {  // SGD with weight decay: momentum iff s1 is in use (mu != 0)
+        if (mu != 0.0f) {
+            s1 = __fadd_rn(__fmul_rn(mu, s1), g);
+            u = __fmul_rn(lr, s1);
+        } else {
+            u = __fmul_rn(lr, g);
+        }
+    }
+    w = __fsub_rn(w, u);
+}
+
+static constexpr int kOptVec = 2;   // vectors per thread (up to 72 bytes of loads each)
+
+template <int KIND, bool WD>
+__global__ void __launch_bounds__(kThreads) k_update_opt(const uint4 *__restrict__ g16, float4 *__restrict__ w32,
+                                                         float4 *__restrict__ s1p, float4 *__restrict__ s2p,
+                                                         uint4 *__restrict__ w16, size_t n8, float inv, float lr, float mu,
+                                                         float b2, float eps, float wd, float b1t, float b2t,
+                                                         uint32_t *flags, const float *__restrict__ inv_dev,
+                                                         const float *__restrict__ betat_dev)
+{
+    if (*(volatile const uint32_t *)flags != 0u) return;
+    if (inv_dev) inv = *inv_dev;
+    if (betat_dev) { b1t = __fmul_rn(betat_dev[0], mu); b2t = __fmul_rn(betat_dev[1], b2); }
+    const float bc1 = __fsub_rn(1.0f, b1t), bc2 = __fsub_rn(1.0f, b2t);
+    const float omb1 = __fsub_rn(1.0f, mu), omb2 = __fsub_rn(1.0f, b2);
+    constexpr bool S1 = true;                      // every kind handled here may use the first state
+    constexpr bool S2 = KIND == MPT_OPT_ADAM;
+    const bool use_s1 = KIND != MPT_OPT_SGD || mu != 0.0f;
+    const size_t base = (size_t)blockIdx.x * (kThreads * kOptVec) + threadIdx.x;
+    bool bad = false;
+    uint4 g[kOptVec];
+    float4 w0[kOptVec], w1[kOptVec], a0[kOptVec], a1[kOptVec], b0[kOptVec], b1[kOptVec];
+#pragma unroll
+    for (int u = 0; u < kOptVec; u++) {
+        const size_t j = base + (size_t)u * kThreads;
+        a0[u] = a1[u] = b0[u] = b1[u] = make_float4(0, 0, 0, 0);
+        if (j < n8) {
+            g[u] = __ldcs(g16 + j);
+            w0[u] = __ldcs(w32 + 2 * j); w1[u] = __ldcs(w32 + 2 * j + 1);
+            if (S1 && use_s1) { a0[u] = __ldcs(s1p + 2 * j); a1[u] = __ldcs(s1p + 2 * j + 1); }
+            if (S2) { b0[u] = __ldcs(s2p + 2 * j); b1[u] = __ldcs(s2p + 2 * j + 1); }
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < kOptVec; u++) {
+        const size_t j = base + (size_t)u * kThreads;
+        if (j < n8) {
+            const uint32_t gw[4] = {g[u].x, g[u].y, g[u].z, g[u].w};
+            float *wf[2] = {&w0[u].x, &w1[u].x}, *af[2] = {&a0[u].x, &a1[u].x}, *bf[2] = {&b0[u].x, &b1[u].x};
+#pragma unroll
+            for (int e = 0; e < 8; e++) {
+                const uint32_t gh = (e & 1) ? (gw[e >> 1] >> 16) : (gw[e >> 1] & 0xFFFFu);
+                opt1<KIND, WD>(gh, wf[e >> 2][e & 3], af[e >> 2][e & 3], bf[e >> 2][e & 3], inv, lr, mu, b2, omb1, omb2, eps,
+                               wd, bc1, bc2, bad);
+            }
+            uint4 h;
+            h.x = f2h_bits(w0[u].x) | (f2h_bits(w0[u].y) << 16);
+            h.y = f2h_bits(w0[u].z) | (f2h_bits(w0[u].w) << 16);
+            h.z = f2h_bits(w1[u].x) | (f2h_bits(w1[u].y) << 16);
+            h.w = f2h_bits(w1[u].z) | (f2h_bits(w1[u].w) << 16);
+            __stcs(w32 + 2 * j, w0[u]); __stcs(w32 + 2 * j + 1, w1[u]);
+            if (S1 && use_s1) { __stcs(s1p + 2 * j, a0[u]); __stcs(s1p + 2 * j + 1, a1[u]); }
+            if (S2) { __stcs(s2p + 2 * j, b0[u]); __stcs(s2p + 2 * j + 1, b1[u]); }
+            __stcs(w16 + j, h);
+        }
+    }
+    if (__any_sync(0xFFFFFFFFu, bad) && (threadIdx.x & 31) == 0) atomicOr(flags + 1, 1u);
+}
+
+template <int KIND, bool WD>
+__global__ void k_update_opt_scalar(const uint16_t *__restrict__ g16, float *__restrict__ w32, float *__restrict__ s1p,
+                                    float *__restrict__ s2p, uint16_t *__restrict__ w16, size_t begin, size_t n, float inv,
+                                    float lr, float mu, float b2, float eps, float wd, float b1t, float b2t, uint32_t *flags,
+                                    const float *__restrict__ inv_dev, const float *__restrict__ betat_dev)
+{
+    if (*(volatile const uint32_t *)flags != 0u) return;
+    if (inv_dev) inv = *inv_dev;
+    if (betat_dev) { b1t = __fmul_rn(betat_dev[0], mu); b2t = __fmul_rn(betat_dev[1], b2); }
+    const float bc1 = __fsub_rn(1.0f, b1t), bc2 = __fsub_rn(1.0f, b2t);
+    const float omb1 = __fsub_rn(1.0f, mu), omb2 = __fsub_rn(1.0f, b2);
+    const bool use_s1 = KIND != MPT_OPT_SGD || mu != 0.0f;
+    size_t stride = (size_t)gridDim.x * blockDim.x;
+    bool bad = false;
+    for (size_t i = begin + (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
+        float w = w32[i], a = use_s1 ? s1p[i] : 0.0f, b = KIND == MPT_OPT_ADAM ? s2p[i] : 0.0f;
+        opt1<KIND, WD>(g16[i], w, a, b, inv, lr, mu, b2, omb1, omb2, eps, wd, bc1, bc2, bad);
+        w32[i] = w;
+        if (use_s1) s1p[i] = a;
+        if (KIND == MPT_OPT_ADAM) s2p[i] = b;
+        w16[i] = (uint16_t)f2h_bits(w);
+    }
+    if (__any_sync(0xFFFFFFFFu, bad) && (threadIdx.x & 31) == 0) atomicOr(flags + 1, 1u);
+}
+
+template <int KIND, bool WD>
+static cudaError_t launch_opt_variant(const uint16_t *g16, float *w32, float *s1, float *s2, uint16_t *w16, size_t n,
+                                      float inv_S, float lr, float mu, float b2, float eps, float wd, float b1t, float b2t,
+                                      uint32_t *flags, cudaStream_t st, const float *inv_dev, const float *betat_dev)
+{
+    uintptr_t bits = (uintptr_t)g16 | (uintptr_t)w32 | (uintptr_t)w16 | (uintptr_t)s1 | (uintptr_t)s2;
+    size_t n8 = (bits & 15) == 0 ? n / 8 : 0;
+    if (n8) {
+        const size_t per_cta = (size_t)kThreads * kOptVec;
+        k_update_opt<KIND, WD><<<(unsigned)((n8 + per_cta - 1) / per_cta), kThreads, 0, st>>>(
+            (const uint4 *)g16, (float4 *)w32, (float4 *)s1, (float4 *)s2, (uint4 *)w16, n8, inv_S, lr, mu, b2, eps, wd, b1t, b2t,
+            flags, inv_dev, betat_dev);
+    }
+    if (n8 * 8 < n)
+        k_update_opt_scalar<KIND, WD><<<grid_for(n - n8 * 8), kThreads, 0, st>>>(g16, w32, s1, s2, w16, n8 * 8, n, inv_S, lr, mu, b2,
+                                                                                eps, wd, b1t, b2t, flags, inv_dev, betat_dev);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_update_opt(int kind, const uint16_t *g16, float *w32, float *s1, float *s2, uint16_t *w16, size_t n,
+                              float inv_S, float lr, float mu, float b2, float eps, float wd, float b1t, float b2t,
+                              uint32_t *flags, cudaStream_t st, const float *inv_dev, const float *betat_dev)
+{
+    if (n == 0) return cudaSuccess;
+#define MPT_OPT_CASE(K)                                                                                                     \
+    case K:                                                                                                                 \
+        return wd != 0.0f ? launch_opt_variant<K, true>(g16, w32, s1, s2, w16, n, inv_S, lr, mu, b2, eps, wd, b1t, b2t, flags, \
+                                                        st, inv_dev, betat_dev)                                             \
+                          : launch_opt_variant<K, false>(g16, w32, s1, s2, w16, n, inv_S, lr, mu, b2, eps, wd, b1t, b2t, flags, \
+                                                         st, inv_dev, betat_dev);
+    switch (kind) {
+        MPT_OPT_CASE(MPT_OPT_SGD)
+        MPT_OPT_CASE(MPT_OPT_NESTEROV)
+        MPT_OPT_CASE(MPT_OPT_ADAGRAD)
+        MPT_OPT_CASE(MPT_OPT_ADAM)
+        default: return cudaErrorInvalidValue;
+    }
+#undef MPT_OPT_CASE
+}
+
+__global__ void k_post_step(uint32_t *status, int interval, float backoff, float growth, float min_S, float max_S, int adam,
+                            float b1, float b2)
+{
+    const bool overflow = status[ST_OVERFLOW] != 0u;
+    if (adam && !overflow) {
+        status[ST_B1T] = __float_as_uint(__fmul_rn(__uint_as_float(status[ST_B1T]), b1));
+        status[ST_B2T] = __float_as_uint(__fmul_rn(__uint_as_float(status[ST_B2T]), b2));
+    }
+    if (interval > 0) {
+        float S = __uint_as_float(status[ST_SCALE]);
+        uint32_t clean = status[ST_CLEAN_STEPS];
+        if (overflow) {
+            S = fmaxf(__fmul_rn(S, backoff), min_S);
+            clean = 0;
+        } else if (++clean >= (uint32_t)interval) {
+            S = fminf(__fmul_rn(S, growth), max_S);
+            clean = 0;
+        }
+        status[ST_SCALE] = __float_as_uint(S);
+        status[ST_INV_SCALE] = __float_as_uint(__fdiv_rn(1.0f, S));
+        status[ST_CLEAN_STEPS] = clean;
+    }
+}
+
+cudaError_t launch_post_step(uint32_t *status, int interval, float backoff, float growth, float min_S, float max_S, int adam,
+                             float b1, float b2, cudaStream_t st)
+{
+    k_post_step<<<1, 1, 0, st>>>(status, interval, backoff, growth, min_S, max_S, adam, b1, b2);
+    return cudaGetLastError();
+}
+
 // ------------------------------------------------------- dynamic loss scale
 
 // The paper's closing section proposes raising or lowering the scale by inspecting the weight

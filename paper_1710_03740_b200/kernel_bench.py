@@ -116,6 +116,24 @@ def bench_update(n, momentum, iters):
             "working_set_mb": bpp * n / 2e6, "flags": flags.tolist()}
 
 
+def bench_update_opt(n, kind, wd, iters):
+    """Master pass with Nesterov (1), Adagrad (2) or Adam (3), optional weight decay."""
+    g = torch.Generator(device="cuda").manual_seed(3)
+    g16 = (torch.randn(n, device="cuda", generator=g) * 37).half()
+    w32 = torch.randn(n, device="cuda", generator=g)
+    s1 = torch.zeros(n, device="cuda")
+    s2 = torch.zeros(n, device="cuda") if kind == mpt.OPT_ADAM else None
+    w16 = torch.empty(n, dtype=torch.half, device="cuda")
+    flags = torch.zeros(2, dtype=torch.int32, device="cuda")
+    opt = mpt.Optimizer(kind, 1e-4, 0.9, 0.999, 1e-8, wd)
+    fn = lambda: mpt.mpt_update_flat_opt(opt, g16, w32, s1, s2, w16, n, 1.0 / 512, 0.81, 0.998, False, flags)  # noqa: E731
+    best, sus = _time(fn, iters)
+    bpp = 28 if kind == mpt.OPT_ADAM else 20
+    return {"kernel": "update_opt", "optimizer": ["sgd", "nesterov", "adagrad", "adam"][kind], "weight_decay": wd,
+            "params": n, "bytes_per_param": bpp, "best_ms": best, "sustained_ms": sus, "best_gbs": bpp * n / best / 1e6,
+            "sustained_gbs": bpp * n / sus / 1e6, "flags": flags.tolist()}
+
+
 def bench_softmax(B, Cn, iters):
     g = torch.Generator(device="cuda").manual_seed(4)
     z = (torch.randn((B, Cn), device="cuda", generator=g) * 3).half()
@@ -188,6 +206,8 @@ def main():
     u = sub.add_parser("update")
     u.add_argument("--params", type=int, default=150994944)
     u.add_argument("--momentum", type=int, default=1)
+    u.add_argument("--optimizer", default="sgd", choices=["sgd", "nesterov", "adagrad", "adam"])
+    u.add_argument("--weight-decay", type=float, default=0.0)
     u.add_argument("--iters", type=int, default=20)
     s = sub.add_parser("softmax")
     s.add_argument("--rows", type=int, default=4096)
@@ -209,7 +229,11 @@ def main():
                 res["kernel_choice"] = args.kernel
                 print(json.dumps(res), flush=True)
     elif args.cmd == "update":
-        print(json.dumps(bench_update(args.params, args.momentum, args.iters)), flush=True)
+        kind = ["sgd", "nesterov", "adagrad", "adam"].index(args.optimizer)
+        if kind == 0 and args.weight_decay == 0.0:
+            print(json.dumps(bench_update(args.params, args.momentum, args.iters)), flush=True)
+        else:
+            print(json.dumps(bench_update_opt(args.params, kind, args.weight_decay, args.iters)), flush=True)
     else:
         print(json.dumps(bench_softmax(args.rows, args.classes, args.iters)), flush=True)
 

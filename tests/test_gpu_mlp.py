@@ -311,6 +311,51 @@ def test_step_replayed_from_a_cuda_graph_matches_eager():
         assert net.get_master(l).tobytes() == eager.get_master(l).tobytes()
 
 
+@pytest.mark.parametrize("kind", [1, 2, 3])
+def test_optimizer_variants_end_to_end(kind):
+    """Whole iterations with Nesterov / Adagrad / Adam (+ weight decay, + an injected overflow that
+    must not advance Adam's step count): flags equal, losses within 1e-3, and the update bit-exact
+    when the oracle is fed the device's own gradient bits."""
+    from paper_1710_03740_b200 import binding as b
+    cfg = dict(inputs.MLP_CONFIGS["tiny"])
+    lr = {1: 0.01, 2: 0.05, 3: 0.001}[kind]
+    opt = b.Optimizer(kind, lr, 0.9, 0.999, 1e-8, 1e-3)
+    masters = inputs.mlp_masters(cfg)
+    X, Y = inputs.mlp_batches(cfg, 6)
+    net = b.Context(cfg["layers"], cfg["S"], lr, 0.9, cfg["batch"], optimizer=opt)
+    ora = OracleMLP(cfg["layers"], cfg["S"], lr, 0.9)
+    ora.set_optimizer(kind, lr, mu=0.9, b2=0.999, eps=1e-8, wd=1e-3)
+    chk = OracleMLP(cfg["layers"], cfg["S"], lr, 0.9)            # teacher-forced twin of the device state
+    chk.set_optimizer(kind, lr, mu=0.9, b2=0.999, eps=1e-8, wd=1e-3)
+    for l, w in enumerate(masters):
+        net.set_master(l, w); ora.set_master(l, w); chk.set_master(l, w)
+    for t in range(6):
+        xd, yd = dev(X[t].view(np.uint16)), dev(Y[t])
+        net.forward(xd)
+        lg = net.backward_scaled(yd)
+        ora.forward(X[t])
+        lo = ora.backward_scaled(Y[t])
+        assert abs(lg - lo) <= 1e-3 * abs(lo)
+        if t == 2:                                               # overflow: skipped everywhere
+            g = net.get_tensor(b.T_GRAD16, 0)
+            g[0, 0] = 0x7C00
+            net.set_grad(0, g)
+            ora.set_grad(0, g)
+        for l in range(2):
+            chk.set_grad(l, net.get_tensor(b.T_GRAD16, l))
+        fg, fo, fc = net.step(), ora.step(), chk.step()
+        assert fg == fo == fc == (1 if t == 2 else 0)
+        for l in range(2):
+            assert net.get_master(l).tobytes() == chk.w32[l].tobytes(), (t, l)
+            assert net.get_tensor(b.T_MOMENTUM32, l).tobytes() == chk.v[l].tobytes()
+            if kind == 3:
+                assert net.get_tensor(b.T_STATE2_32, l).tobytes() == chk.s2[l].tobytes()
+    if kind == 3:
+        b1t, b2t = net.get_adam_products()
+        assert b1t == float(chk.b1t) and b2t == float(chk.b2t)
+        assert abs(b1t - 0.9 ** 5) < 1e-6                        # five applied steps out of six
+
+
 def test_error_paths():
     from paper_1710_03740_b200 import binding as b
     cfg = inputs.MLP_CONFIGS["tiny"]

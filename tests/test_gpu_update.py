@@ -141,3 +141,44 @@ def test_update_loguniform_config_2b_bit_exact():
         assert flags.tolist() == [0, 0]
         assert np.array_equal(w_g.view(np.uint32), w_ref.view(np.uint32))
         assert np.array_equal(h_g, h_ref)
+
+
+@pytest.mark.parametrize("kind", [0, 1, 2, 3])
+@pytest.mark.parametrize("wd", [0.0, 1e-2])
+@pytest.mark.parametrize("n,misalign", [(8 * 256 * 5 + 3, 0), (4097, 1)])
+def test_optimizer_variants_bit_exact(kind, wd, n, misalign):
+    """Nesterov, Adagrad, Adam and weight decay on the master pass: bit for bit with the oracle."""
+    b = _binding()
+    if kind == 0 and wd == 0.0:
+        pytest.skip("plain SGD(+momentum) is covered above")
+    rng = np.random.default_rng(50 + kind)
+    f = np.float32
+    S, lr, mu, b2, eps = 256.0, 0.01, 0.9, 0.999, 1e-8
+    g16 = (rng.standard_normal(n) * 30.0).astype(np.float16)
+    w = rng.standard_normal(n).astype(np.float32)
+    s1 = (np.abs(rng.standard_normal(n)) * 0.1).astype(np.float32)
+    s2 = (np.abs(rng.standard_normal(n)) * 0.01).astype(np.float32)
+    b1t, b2t = f(f(0.9) * f(0.9)), f(f(0.999) * f(0.999))                 # second applied step
+    inv = f(1.0) / f(S)
+    w_ref, a_ref, c_ref = w.copy(), s1.copy(), s2.copy()
+    h_ref = np.zeros(n, dtype=np.uint16)
+    mpo.update_apply_opt(kind, g16, w_ref, a_ref, c_ref if kind == 3 else None, h_ref, inv, f(lr), f(mu), f(b2), f(eps),
+                         f(wd), f(1.0) - b1t, f(1.0) - b2t)
+    pad = misalign
+    gd = torch.zeros(n + 8, dtype=torch.int16, device="cuda")
+    wd_ = torch.zeros(n + 8, dtype=torch.float32, device="cuda")
+    ad = torch.zeros(n + 8, dtype=torch.float32, device="cuda")
+    cd = torch.zeros(n + 8, dtype=torch.float32, device="cuda")
+    hd = torch.zeros(n + 8, dtype=torch.int16, device="cuda")
+    gd[pad:pad + n] = dev(g16.view(np.uint16)); wd_[pad:pad + n] = dev(w); ad[pad:pad + n] = dev(s1); cd[pad:pad + n] = dev(s2)
+    flags = torch.zeros(2, dtype=torch.int32, device="cuda")
+    opt = b.Optimizer(kind, lr, mu, b2, eps, wd)
+    b.mpt_update_flat_opt(opt, gd[pad:], wd_[pad:], ad[pad:], cd[pad:] if kind == 3 else None, hd[pad:], n, float(inv),
+                          float(b1t), float(b2t), True, flags)
+    torch.cuda.synchronize()
+    assert flags.tolist() == [0, 0]
+    assert np.array_equal(wd_[pad:pad + n].cpu().numpy().view(np.uint32), w_ref.view(np.uint32))
+    assert np.array_equal(ad[pad:pad + n].cpu().numpy().view(np.uint32), a_ref.view(np.uint32))
+    if kind == 3:
+        assert np.array_equal(cd[pad:pad + n].cpu().numpy().view(np.uint32), c_ref.view(np.uint32))
+    assert np.array_equal(host_u16(hd[pad:pad + n]), h_ref)

@@ -460,6 +460,89 @@ def test_update_vs_numpy_float32_ops(use_momentum):
     assert np.array_equal(w16, w_ref.astype(np.float16).view(np.uint16))
 
 
+@pytest.mark.parametrize("kind", [0, 1, 2, 3])
+@pytest.mark.parametrize("wd", [0.0, 1e-2])
+def test_optimizer_variants_vs_numpy_float32_ops(kind, wd):
+    """Nesterov / Adagrad / Adam / weight decay on the master copy (optimizers the paper's
+    experiments use, sections 4.3, 4.5, 4.6; section 3.2: decay acts on the unscaled gradient):
+    numpy float32 array arithmetic rounds every operation separately, in the same order."""
+    rng = np.random.default_rng(40 + kind)
+    n = 1 << 18
+    w = rng.standard_normal(n).astype(np.float32)
+    s1 = (np.abs(rng.standard_normal(n)) * 0.1).astype(np.float32)
+    s2 = (np.abs(rng.standard_normal(n)) * 0.01).astype(np.float32)
+    if kind in (0, 1):
+        s1 = (rng.standard_normal(n) * 0.1).astype(np.float32)
+    g16 = (rng.standard_normal(n) * 37.0).astype(np.float16)
+    f = np.float32
+    S, lr, mu, b2, eps, wdf = f(128.0), f(0.01), f(0.9), f(0.999), f(1e-8), f(wd)
+    bc1, bc2 = f(1.0) - f(0.9) ** 3, f(1.0) - f(0.999) ** 3
+    inv = f(1.0) / S
+    g = g16.astype(np.float32) * inv
+    if wd:
+        g = g + wdf * w
+    s1r, s2r = s1.copy(), s2.copy()
+    if kind == 0:
+        s1r = mu * s1 + g
+        u = lr * s1r
+    elif kind == 1:
+        s1r = mu * s1 + g
+        u = lr * (g + mu * s1r)
+    elif kind == 2:
+        s1r = s1 + g * g
+        u = lr * (g / (np.sqrt(s1r) + eps))
+    else:
+        s1r = mu * s1 + (f(1.0) - mu) * g
+        s2r = b2 * s2 + (f(1.0) - b2) * (g * g)
+        u = lr * ((s1r / bc1) / (np.sqrt(s2r / bc2) + eps))
+    w_ref = w - u
+    w2, a1, a2 = w.copy(), s1.copy(), s2.copy()
+    h = np.zeros(n, dtype=np.uint16)
+    mpo.update_apply_opt(kind, g16, w2, a1, a2 if kind == 3 else None, h, inv, lr, mu, b2, eps, wdf, bc1, bc2)
+    assert np.array_equal(w2.view(np.uint32), w_ref.view(np.uint32))
+    assert np.array_equal(a1.view(np.uint32), s1r.astype(np.float32).view(np.uint32))
+    if kind == 3:
+        assert np.array_equal(a2.view(np.uint32), s2r.astype(np.float32).view(np.uint32))
+    assert np.array_equal(h, w_ref.astype(np.float16).view(np.uint16))
+    if kind == 0 and not wd:     # the generic entry point agrees with the SGD+momentum one
+        w3, v3, h3 = w.copy(), s1.copy(), np.zeros(n, dtype=np.uint16)
+        mpo.update_apply(g16, w3, v3, h3, inv, lr, mu, True)
+        assert w3.tobytes() == w2.tobytes() and v3.tobytes() == a1.tobytes() and h3.tobytes() == h.tobytes()
+
+
+def test_optimizer_first_step_closed_forms():
+    """From zero state: Adam's bias-corrected first update is lr*g/(|g|+eps), Adagrad's is the
+    same expression, Nesterov's is lr*(1+mu)*g, and decay adds wd*w to the unscaled gradient."""
+    g16 = np.array([0.5, -2.0, 3.0, -0.125], dtype=np.float16)
+    g = g16.astype(np.float64)
+    lr, eps = 0.01, 1e-8
+    for kind, want in ((3, lr * g / (np.abs(g) + eps)), (2, lr * g / (np.abs(g) + eps)), (1, lr * 1.9 * g)):
+        net = OracleMLP([(4, 1, 0)], 1.0, lr, 0.0)
+        net.set_master(0, np.zeros((1, 4), dtype=np.float32))
+        net.set_optimizer(kind, lr, mu=0.9, b2=0.999, eps=eps)
+        net.set_grad(0, g16.reshape(1, 4))
+        assert net.step() == 0
+        assert np.allclose(-net.w32[0][0].astype(np.float64), want, rtol=2e-6, atol=0)
+    net = OracleMLP([(4, 1, 0)], 1.0, lr, 0.0)
+    w0 = np.array([[1.0, -2.0, 4.0, 8.0]], dtype=np.float32)
+    net.set_master(0, w0)
+    net.set_optimizer(0, lr, wd=0.5)
+    net.set_grad(0, g16.reshape(1, 4))
+    net.step()
+    assert np.allclose(net.w32[0][0].astype(np.float64), w0[0] - lr * (g + 0.5 * w0[0]), rtol=1e-6)
+    # Adam's bias correction uses the number of APPLIED steps: a skipped step does not advance it
+    net = OracleMLP([(4, 1, 0)], 1.0, lr, 0.0)
+    net.set_master(0, np.zeros((1, 4), dtype=np.float32))
+    net.set_optimizer(3, lr, mu=0.9, b2=0.999, eps=eps)
+    bad = g16.copy()
+    bad[0] = np.inf
+    net.set_grad(0, bad.reshape(1, 4))
+    assert net.step() == 1 and float(net.b1t) == 1.0 and not net.w32[0].any()
+    net.set_grad(0, g16.reshape(1, 4))
+    assert net.step() == 0
+    assert np.allclose(-net.w32[0][0].astype(np.float64), lr * g / (np.abs(g) + eps), rtol=2e-6)
+
+
 def test_overflow_detect_and_skip():
     """Section 3.2: an inf/NaN in any weight gradient skips the update."""
     layers = [(8, 6, 1), (6, 4, 0)]
