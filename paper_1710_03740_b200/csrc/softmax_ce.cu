@@ -124,7 +124,7 @@ __global__ void __launch_bounds__(1024) k_softmax_ce(const uint16_t *__restrict_
 // only touches terms far below it, and is far below FP16 resolution after the store.  Non-label outputs are e_j * (c / s); the label's output is
 // (e_y / s - 1) * c, evaluated separately because of the cancellation.
 template <int VPT>
-__global__ void __launch_bounds__(1024) k_softmax_ce_reg(const uint16_t *__restrict__ z, int ldz,
+__global__ void __launch_bounds__(1024, VPT <= 4 ? 2 : 1) k_softmax_ce_reg(const uint16_t *__restrict__ z, int ldz,
                                                          const int32_t *__restrict__ labels, int C, float c,
                                                          uint16_t *__restrict__ dz, int lddz,
                                                          float *__restrict__ row_loss, uint32_t *bad_labels,
