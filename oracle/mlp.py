@@ -42,7 +42,8 @@ class OracleMLP:
         self.v = [np.zeros((o, i), dtype=np.float32) for (i, o, _) in self.layers]
         self.g16 = [np.zeros((o, i), dtype=np.uint16) for (i, o, _) in self.layers]
         # optimizer: kind 0 SGD(+momentum) by default; set_optimizer switches (state s1/s2 start at zero)
-        self.opt = dict(kind=mpo.OPT_SGD, b2=np.float32(0.0), eps=np.float32(0.0), wd=np.float32(0.0))
+        self.opt = dict(kind=mpo.OPT_SGD, b2=np.float32(0.0), eps=np.float32(0.0), wd=np.float32(0.0), clip=0.0)
+        self.last_coef = np.float32(1.0)
         self.s2 = [np.zeros((o, i), dtype=np.float32) for (i, o, _) in self.layers]
         self.b1t = np.float32(1.0)     # running products beta1^t, beta2^t over applied steps (Adam)
         self.b2t = np.float32(1.0)
@@ -87,9 +88,10 @@ class OracleMLP:
                                               mask=self.acts[l] if self.layers[l - 1][2] else None)
         return loss
 
-    def set_optimizer(self, kind, lr, mu=0.0, b2=0.0, eps=0.0, wd=0.0):
-        """kind: mpo.OPT_*; mu is the momentum (SGD, Nesterov) or beta1 (Adam)."""
-        self.opt = dict(kind=int(kind), b2=np.float32(b2), eps=np.float32(eps), wd=np.float32(wd))
+    def set_optimizer(self, kind, lr, mu=0.0, b2=0.0, eps=0.0, wd=0.0, clip=0.0):
+        """kind: mpo.OPT_*; mu is the momentum (SGD, Nesterov) or beta1 (Adam); clip: global-norm
+        bound on the unscaled gradients (0 = off)."""
+        self.opt = dict(kind=int(kind), b2=np.float32(b2), eps=np.float32(eps), wd=np.float32(wd), clip=float(clip))
         self.lr = np.float32(lr)
         self.mu = np.float32(mu)
         self.use_momentum = (kind == mpo.OPT_SGD and float(mu) != 0.0) or kind != mpo.OPT_SGD
@@ -108,7 +110,11 @@ class OracleMLP:
             overflow |= mpo.grad_nonfinite(g, inv)
         if not overflow:
             kind = self.opt["kind"]
-            if kind == mpo.OPT_SGD and float(self.opt["wd"]) == 0.0:
+            clip = self.opt["clip"]
+            if clip > 0.0:      # section 3.2: clipping acts on the unscaled gradients of all layers together
+                total = sum(mpo.grad_sqnorm(g, inv) for g in self.g16)
+                self.last_coef = mpo.clip_coef(total, clip)
+            if kind == mpo.OPT_SGD and float(self.opt["wd"]) == 0.0 and clip <= 0.0:
                 for l in range(len(self.layers)):
                     mpo.update_apply(self.g16[l], self.w32[l], self.v[l], self.w16[l], inv, self.lr, self.mu,
                                      self.use_momentum)
@@ -121,8 +127,12 @@ class OracleMLP:
                 for l in range(len(self.layers)):
                     s1 = self.v[l] if (kind != mpo.OPT_SGD or self.use_momentum) else None
                     s2 = self.s2[l] if kind == mpo.OPT_ADAM else None
-                    mpo.update_apply_opt(kind, self.g16[l], self.w32[l], s1, s2, self.w16[l], inv, self.lr, self.mu,
-                                         self.opt["b2"], self.opt["eps"], self.opt["wd"], bc1, bc2)
+                    if clip > 0.0:
+                        mpo.update_apply_clip(kind, self.g16[l], self.w32[l], s1, s2, self.w16[l], inv, self.last_coef,
+                                              self.lr, self.mu, self.opt["b2"], self.opt["eps"], self.opt["wd"], bc1, bc2)
+                    else:
+                        mpo.update_apply_opt(kind, self.g16[l], self.w32[l], s1, s2, self.w16[l], inv, self.lr, self.mu,
+                                             self.opt["b2"], self.opt["eps"], self.opt["wd"], bc1, bc2)
         if self.dynamic is not None:
             interval, backoff, growth, smin, smax = self.dynamic
             if overflow:

@@ -70,6 +70,11 @@ def lib() -> ctypes.CDLL:
         L.mpo_update_apply_opt.restype = None
         L.mpo_update_apply_opt.argtypes = [c.c_int, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p,
                                            c.c_size_t] + [c.c_float] * 8
+        L.mpo_grad_sqnorm.restype = c.c_double
+        L.mpo_grad_sqnorm.argtypes = [c.c_void_p, c.c_size_t, c.c_float]
+        L.mpo_update_apply_clip.restype = None
+        L.mpo_update_apply_clip.argtypes = [c.c_int, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p,
+                                            c.c_size_t] + [c.c_float] * 9
         _lib = L
     return _lib
 
@@ -216,3 +221,20 @@ def update_apply_opt(kind, g16, w32, s1, s2, w16, inv_S, lr, mu, b2=0.0, eps=0.0
             assert a.flags["C_CONTIGUOUS"]
     lib().mpo_update_apply_opt(int(kind), _ptr(g), _ptr(w32), _ptr(s1), _ptr(s2), _ptr(w16), g.size, float(inv_S),
                                float(lr), float(mu), float(b2), float(eps), float(wd), float(bc1), float(bc2))
+
+
+def grad_sqnorm(g16, inv_S) -> float:
+    """Sum of squares of the unscaled gradients, accumulated in double."""
+    g = np.ascontiguousarray(_u16(g16)).reshape(-1)
+    return float(lib().mpo_grad_sqnorm(_ptr(g), g.size, float(inv_S)))
+
+
+def clip_coef(total_sq, clip_norm) -> np.float32:
+    """coef = min(1, clip / (sqrt(total) + 1e-6)), rounded to binary32."""
+    return np.float32(min(1.0, float(clip_norm) / (float(np.sqrt(total_sq)) + 1e-6)))
+
+
+def update_apply_clip(kind, g16, w32, s1, s2, w16, inv_S, coef, lr, mu, b2=0.0, eps=0.0, wd=0.0, bc1=1.0, bc2=1.0) -> None:
+    g = _u16(g16)
+    lib().mpo_update_apply_clip(int(kind), _ptr(g), _ptr(w32), _ptr(s1), _ptr(s2), _ptr(w16), g.size, float(inv_S),
+                                float(coef), float(lr), float(mu), float(b2), float(eps), float(wd), float(bc1), float(bc2))

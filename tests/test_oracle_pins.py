@@ -543,6 +543,51 @@ def test_optimizer_first_step_closed_forms():
     assert np.allclose(-net.w32[0][0].astype(np.float64), lr * g / (np.abs(g) + eps), rtol=2e-6)
 
 
+def test_global_norm_clipping_closed_forms():
+    """Section 3.2: clipping acts on the unscaled gradients.  Known norm (3-4-5 triangle spread
+    over two layers), coefficient min(1, clip/norm), update equal to numpy float32 arithmetic,
+    and independence from the loss scale."""
+    f = np.float32
+    for S in (1.0, 256.0):
+        net = OracleMLP([(2, 1, 1), (1, 1, 0)], S, 0.5, 0.0)
+        net.set_master(0, np.array([[1.0, 2.0]], dtype=np.float32))
+        net.set_master(1, np.array([[3.0]], dtype=np.float32))
+        net.set_optimizer(0, 0.5, clip=2.5)
+        net.set_grad(0, (np.array([[3.0, 0.0]]) * S).astype(np.float16))
+        net.set_grad(1, (np.array([[4.0]]) * S).astype(np.float16))
+        assert net.step() == 0
+        coef = f(2.5 / (5.0 + 1e-6))
+        assert float(net.last_coef) == float(coef)
+        assert float(net.w32[0][0, 0]) == float(f(1.0) - f(0.5) * (f(3.0) * coef))
+        assert float(net.w32[0][0, 1]) == 2.0
+        assert float(net.w32[1][0, 0]) == float(f(3.0) - f(0.5) * (f(4.0) * coef))
+    # a norm under the bound leaves the gradient alone (coefficient exactly 1)
+    net = OracleMLP([(2, 1, 0)], 1.0, 0.5, 0.0)
+    net.set_master(0, np.zeros((1, 2), dtype=np.float32))
+    net.set_optimizer(0, 0.5, clip=10.0)
+    net.set_grad(0, np.array([[3.0, 4.0]], dtype=np.float16))
+    net.step()
+    assert float(net.last_coef) == 1.0 and net.w32[0].tolist() == [[-1.5, -2.0]]
+    # the sum of squares against numpy float64 on random data, and the generic step against numpy
+    rng = np.random.default_rng(77)
+    n = 1 << 16
+    g16 = (rng.standard_normal(n) * 20).astype(np.float16)
+    inv = f(1.0) / f(64.0)
+    ref = float(((g16.astype(np.float32) * inv).astype(np.float64) ** 2).sum())
+    got = mpo.grad_sqnorm(g16, inv)
+    assert abs(got - ref) <= 1e-12 * ref
+    coef = mpo.clip_coef(got, 1.0)
+    w = rng.standard_normal(n).astype(np.float32)
+    v = (rng.standard_normal(n) * 0.1).astype(np.float32)
+    g = (g16.astype(np.float32) * inv) * coef
+    g = g + f(1e-2) * w
+    v_ref = f(0.9) * v + g
+    w_ref = w - f(0.01) * (g + f(0.9) * v_ref)
+    w2, v2, h = w.copy(), v.copy(), np.zeros(n, dtype=np.uint16)
+    mpo.update_apply_clip(1, g16, w2, v2, None, h, inv, coef, f(0.01), f(0.9), wd=f(1e-2))
+    assert np.array_equal(w2.view(np.uint32), w_ref.view(np.uint32)) and np.array_equal(v2.view(np.uint32), v_ref.view(np.uint32))
+
+
 def test_overflow_detect_and_skip():
     """Section 3.2: an inf/NaN in any weight gradient skips the update."""
     layers = [(8, 6, 1), (6, 4, 0)]
