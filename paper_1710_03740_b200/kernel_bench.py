@@ -14,6 +14,8 @@ from __future__ import annotations
 
 import argparse
 import json
+import subprocess
+import time
 
 import torch
 
@@ -21,6 +23,46 @@ from . import binding as mpt
 from . import inputs
 
 OPS = {0: "fwd", 1: "dgrad", 2: "wgrad"}
+
+
+def _sustained(fn, seconds):
+    """Rate over a loop of at least `seconds` of back-to-back launches, with the SM clock and power
+    sampled by nvidia-smi every 100 ms meanwhile (the GPU settles under its power cap)."""
+    q = "clocks.sm,power.draw,clocks_event_reasons.sw_power_cap,clocks_event_reasons.hw_slowdown,clocks_event_reasons.sw_thermal_slowdown"
+    try:
+        smi = subprocess.Popen(["nvidia-smi", "-i", str(torch.cuda.current_device()), "--query-gpu=" + q,
+                                "--format=csv,noheader,nounits", "-lms", "100"], stdout=subprocess.PIPE, text=True)
+    except OSError:
+        smi = None
+    for _ in range(3):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n, t0 = 0, time.time()
+    e0.record()
+    while time.time() - t0 < seconds:
+        for _ in range(50):
+            fn()
+        n += 50
+        torch.cuda.synchronize()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / n
+    clocks, power, reasons = [], [], set()
+    if smi is not None:
+        smi.terminate()
+        for line in smi.stdout.read().strip().splitlines()[3:]:
+            f = [x.strip() for x in line.split(",")]
+            try:
+                clocks.append(float(f[0])); power.append(float(f[1]))
+            except (ValueError, IndexError):
+                continue
+            for name, v in zip(("sw_power_cap", "hw_slowdown", "sw_thermal_slowdown"), f[2:5]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+    clocks.sort(); power.sort()
+    return ms, {"sm_mhz_median": clocks[len(clocks) // 2] if clocks else None,
+                "power_w_median": power[len(power) // 2] if power else None, "reasons": sorted(reasons)}
 
 
 def _time_graph(fn, iters):
@@ -65,7 +107,7 @@ def _time(fn, iters, warmup=3):
     return best, e0.elapsed_time(e1) / iters
 
 
-def bench_gemm(M, N, K, op, iters, compare=False, flags=mpt.GEMM_FORCE_TC, use_workspace=True):
+def bench_gemm(M, N, K, op, iters, compare=False, flags=mpt.GEMM_FORCE_TC, use_workspace=True, sustain_s=0.0):
     sa = (K, M) if op == 2 else (M, K)
     sb = (N, K) if op == 0 else (K, N)
     g = torch.Generator(device="cuda").manual_seed(2)
@@ -86,6 +128,10 @@ def bench_gemm(M, N, K, op, iters, compare=False, flags=mpt.GEMM_FORCE_TC, use_w
     out = {"kernel": "gemm", "op": OPS[op], "M": M, "N": N, "K": K, "best_ms": best, "sustained_ms": sus,
            "best_tflops": fl / best / 1e9, "sustained_tflops": fl / sus / 1e9, "device_error": int(st[0]), "splitk_workspace_mb": nws / 1e6,
            "working_set_mb": (A.numel() + B.numel() + C.numel()) * 2 / 1e6}
+    if sustain_s > 0:
+        ms, clk = _sustained(fn, sustain_s)
+        out["sustained_%gs_tflops" % sustain_s] = fl / ms / 1e9
+        out["sustained_clocks"] = clk
     if compare:
         if op == 0:
             ref = lambda: torch.matmul(A, B.t())  # noqa: E731
@@ -98,6 +144,10 @@ def bench_gemm(M, N, K, op, iters, compare=False, flags=mpt.GEMM_FORCE_TC, use_w
             rs = min(rs, _time_graph(ref, iters))
         out["library_best_tflops"] = fl / rb / 1e9
         out["library_sustained_tflops"] = fl / rs / 1e9
+        if sustain_s > 0:
+            ms, clk = _sustained(ref, sustain_s)
+            out["library_sustained_%gs_tflops" % sustain_s] = fl / ms / 1e9
+            out["library_sustained_clocks"] = clk
     return out
 
 
@@ -201,6 +251,8 @@ def main():
     g.add_argument("--iters", type=int, default=20)
     g.add_argument("--compare-library", action="store_true")
     g.add_argument("--no-workspace", action="store_true", help="do not offer a split-K scratch buffer")
+    g.add_argument("--sustain", type=float, default=0.0, metavar="SECONDS",
+                   help="also time a loop of at least this many seconds with clocks and power sampled")
     g.add_argument("--kernel", default="auto", choices=["auto", "tc", "pair"],
                    help="auto: the library's choice; tc: single-CTA 128x256 tiles; pair: cta_group::2 256x256 tiles")
     u = sub.add_parser("update")
@@ -225,7 +277,7 @@ def main():
         for (M, N, K) in shapes:
             for op in args.op:
                 flags = {"auto": 0, "tc": mpt.GEMM_FORCE_TC, "pair": mpt.GEMM_FORCE_PAIR}[args.kernel]
-                res = bench_gemm(M, N, K, op, args.iters, args.compare_library, flags, not args.no_workspace)
+                res = bench_gemm(M, N, K, op, args.iters, args.compare_library, flags, not args.no_workspace, args.sustain)
                 res["kernel_choice"] = args.kernel
                 print(json.dumps(res), flush=True)
     elif args.cmd == "update":
