@@ -83,8 +83,11 @@ extern "C" {
 /* Optimizer step applied to the FP32 master copy (section 3.1: the update is computed in FP32;
  * the paper's experiments use plain and Nesterov momentum SGD, Adagrad and Adam, sections 4.3,
  * 4.5, 4.6, without giving formulas: the textbook forms are used).  With g the UNSCALED
- * gradient (section 3.2: decay and the like act after unscaling), every line one separately
- * rounded FP32 operation, states starting at zero:
+ * gradient (section 3.2: clipping, decay and the like act after unscaling), every line one
+ * separately rounded FP32 operation, states starting at zero:
+ *   clip_norm > 0:      g = g * coef, coef = min(1, clip_norm / (norm + 1e-6)) rounded to FP32,
+ *                       norm = sqrt(sum over ALL layers of g*g), sum, sqrt and quotient in double
+ *                       (one extra read of the FP16 gradients: +2 bytes per parameter)
  *   weight_decay != 0:  g = g + weight_decay * w
  *   MPT_OPT_SGD       momentum == 0: u = lr*g ;  else  s1 = momentum*s1 + g ; u = lr*s1
  *   MPT_OPT_NESTEROV  s1 = momentum*s1 + g ; u = lr*(g + momentum*s1)
@@ -107,6 +110,7 @@ typedef struct mpt_optimizer {
     float beta2;        /* Adam beta2 in [0, 1); ignored otherwise */
     float eps;          /* Adagrad / Adam epsilon >= 0; ignored otherwise */
     float weight_decay; /* >= 0; 0 disables */
+    float clip_norm;    /* >= 0; bound on the global norm of the unscaled gradients; 0 disables */
 } mpt_optimizer;
 
 typedef struct mpt_ctx mpt_ctx;
@@ -240,6 +244,10 @@ int mpt_set_momentum(mpt_ctx *ctx, int layer, const float *src_host, size_t n);
 int mpt_set_state2(mpt_ctx *ctx, int layer, const float *src_host, size_t n);
 int mpt_get_adam_products(mpt_ctx *ctx, float *b1t_out, float *b2t_out);
 int mpt_set_adam_products(mpt_ctx *ctx, float b1t, float b2t);
+/* Norm of the unscaled gradients and clipping coefficient of the last mpt_step (contexts created
+ * with clip_norm > 0; MPT_ERR_STATE otherwise).  After an overflowing step the norm is inf or NaN
+ * and the step was skipped.  Synchronous. */
+int mpt_get_grad_norm(mpt_ctx *ctx, float *norm_out, float *coef_out);
 
 /* Number of kernels this context has launched since creation (bookkeeping for
  * benchmarks). */
@@ -316,12 +324,16 @@ int mpt_update_flat(const uint16_t *g16_dev, float *w32_dev, float *v_dev, uint1
                     float inv_S, float lr, float mu, int use_momentum, int detect, uint32_t *flags_dev,
                     void *cuda_stream);
 
-/* The same pass for any optimizer of mpt_optimizer (kind, weight decay).  s1_dev / s2_dev: FP32
- * states (null when the kind does not use them).  b1t / b2t: for Adam, beta1^t and beta2^t
- * INCLUDING this step (the caller keeps the products); ignored otherwise. */
+/* The same pass for any optimizer of mpt_optimizer (kind, weight decay, clipping).  s1_dev /
+ * s2_dev: FP32 states (null when the kind does not use them).  b1t / b2t: for Adam, beta1^t and
+ * beta2^t INCLUDING this step (the caller keeps the products); ignored otherwise.
+ * clip_scratch_dev: needed iff opt->clip_norm > 0 (else may be null): MPT_CLIP_SCRATCH_BYTES of
+ * device memory, 256-byte aligned, owned by the caller; the norm is taken over g16[0..n) and on
+ * return (stream order) its first two floats hold the coefficient and the norm. */
+#define MPT_CLIP_SCRATCH_BYTES 16384
 int mpt_update_flat_opt(const mpt_optimizer *opt, const uint16_t *g16_dev, float *w32_dev, float *s1_dev, float *s2_dev,
                         uint16_t *w16_dev, size_t n, float inv_S, float b1t, float b2t, int detect, uint32_t *flags_dev,
-                        void *cuda_stream);
+                        void *clip_scratch_dev, void *cuda_stream);
 
 /* Softmax cross-entropy forward and scaled backward (sections 3.2, 3.3), arithmetic
  * as in mpt_backward_scaled.  z_dev/dz_dev: FP16 [B, C] with pitches ldz/lddz

@@ -230,8 +230,9 @@ def grad_sqnorm(g16, inv_S) -> float:
 
 
 def clip_coef(total_sq, clip_norm) -> np.float32:
-    """coef = min(1, clip / (sqrt(total) + 1e-6)), rounded to binary32."""
-    return np.float32(min(1.0, float(clip_norm) / (float(np.sqrt(total_sq)) + 1e-6)))
+    """coef = min(1, clip / (sqrt(total) + 1e-6)), rounded to binary32.  The bound is a binary32
+    parameter of the optimizer: the quotient is formed in double from its binary32 value."""
+    return np.float32(min(1.0, float(np.float32(clip_norm)) / (float(np.sqrt(total_sq)) + 1e-6)))
 
 
 def update_apply_clip(kind, g16, w32, s1, s2, w16, inv_S, coef, lr, mu, b2=0.0, eps=0.0, wd=0.0, bc1=1.0, bc2=1.0) -> None:

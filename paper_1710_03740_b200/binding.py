@@ -25,7 +25,7 @@ OPT_SGD, OPT_NESTEROV, OPT_ADAGRAD, OPT_ADAM = 0, 1, 2, 3
 
 # every symbol include/mpt.h declares
 EXPORTS = ["mpt_workspace_bytes", "mpt_create", "mpt_workspace_bytes_opt", "mpt_create_opt", "mpt_set_state2",
-           "mpt_get_adam_products", "mpt_set_adam_products", "mpt_update_flat_opt", "mpt_set_master", "mpt_forward", "mpt_backward_scaled",
+           "mpt_get_adam_products", "mpt_set_adam_products", "mpt_get_grad_norm", "mpt_update_flat_opt", "mpt_set_master", "mpt_forward", "mpt_backward_scaled",
            "mpt_step", "mpt_get_master", "mpt_train_step_host", "mpt_stage_batch_host",
            "mpt_train_step_staged", "mpt_set_scale", "mpt_set_lr", "mpt_set_dynamic_scale", "mpt_get_scale",
            "mpt_get_tensor", "mpt_set_grad", "mpt_set_momentum", "mpt_launch_count", "mpt_profile",
@@ -45,9 +45,9 @@ class LayerDesc(C.Structure):
 
 
 class Optimizer(C.Structure):
-    """mpt_optimizer: kind (OPT_*), lr, momentum (or Adam beta1), beta2, eps, weight_decay."""
+    """mpt_optimizer: kind (OPT_*), lr, momentum (or Adam beta1), beta2, eps, weight_decay, clip_norm."""
     _fields_ = [("kind", C.c_int32), ("lr", C.c_float), ("momentum", C.c_float), ("beta2", C.c_float),
-                ("eps", C.c_float), ("weight_decay", C.c_float)]
+                ("eps", C.c_float), ("weight_decay", C.c_float), ("clip_norm", C.c_float)]
 
 
 _lib = None
@@ -69,7 +69,8 @@ def lib() -> C.CDLL:
     L.mpt_set_state2.argtypes = [vp, i32, vp, sz]
     L.mpt_get_adam_products.argtypes = [vp, C.POINTER(f32), C.POINTER(f32)]
     L.mpt_set_adam_products.argtypes = [vp, f32, f32]
-    L.mpt_update_flat_opt.argtypes = [C.POINTER(Optimizer), vp, vp, vp, vp, vp, sz, f32, f32, f32, i32, vp, vp]
+    L.mpt_update_flat_opt.argtypes = [C.POINTER(Optimizer), vp, vp, vp, vp, vp, sz, f32, f32, f32, i32, vp, vp, vp]
+    L.mpt_get_grad_norm.argtypes = [vp, C.POINTER(f32), C.POINTER(f32)]
     L.mpt_set_master.argtypes = [vp, i32, vp, sz]
     L.mpt_forward.argtypes = [vp, vp, i32]
     L.mpt_backward_scaled.argtypes = [vp, vp, C.POINTER(f32)]
@@ -286,6 +287,12 @@ class Context:
         _check(lib().mpt_get_adam_products(self._ctx, C.byref(a), C.byref(b)), self._ctx)
         return float(a.value), float(b.value)
 
+    def get_grad_norm(self):
+        """(norm of the unscaled gradients, clipping coefficient) of the last step."""
+        a, b = C.c_float(0.0), C.c_float(0.0)
+        _check(lib().mpt_get_grad_norm(self._ctx, C.byref(a), C.byref(b)), self._ctx)
+        return float(a.value), float(b.value)
+
     def set_adam_products(self, b1t, b2t):
         _check(lib().mpt_set_adam_products(self._ctx, float(b1t), float(b2t)), self._ctx)
 
@@ -331,10 +338,13 @@ def mpt_update_flat(g16, w32, v, w16, n, inv_S, lr, mu, use_momentum, detect, fl
                                  int(bool(use_momentum)), int(bool(detect)), _dptr(flags), _stream_ptr(stream)))
 
 
-def mpt_update_flat_opt(opt, g16, w32, s1, s2, w16, n, inv_S, b1t, b2t, detect, flags, stream=None):
+CLIP_SCRATCH_BYTES = 16384
+
+
+def mpt_update_flat_opt(opt, g16, w32, s1, s2, w16, n, inv_S, b1t, b2t, detect, flags, clip_scratch=None, stream=None):
     _check(lib().mpt_update_flat_opt(C.byref(opt), _dptr(g16), _dptr(w32), _dptr(s1), _dptr(s2), _dptr(w16), n,
                                      float(inv_S), float(b1t), float(b2t), int(bool(detect)), _dptr(flags),
-                                     _stream_ptr(stream)))
+                                     _dptr(clip_scratch), _stream_ptr(stream)))
 
 
 def mpt_softmax_ce(z, ldz, labels, B, Cn, S, dz, lddz, row_loss, loss, bad_labels=None, stream=None):

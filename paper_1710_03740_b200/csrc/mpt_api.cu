@@ -29,7 +29,7 @@ struct Layer {
 struct Plan {
     size_t total = 0, P_pad = 0;
     size_t off_status = 0, off_master = 0, off_mom = 0, off_state2 = 0, off_w16 = 0, off_g16 = 0, off_x[2] = {0, 0},
-           off_labels[2] = {0, 0}, off_rowloss = 0, off_splitk = 0, splitk_bytes = 0;
+           off_labels[2] = {0, 0}, off_rowloss = 0, off_norm = 0, off_splitk = 0, splitk_bytes = 0;
     std::vector<size_t> off_act, off_dact, lay_off;
     std::vector<int> ld_out;
 };
@@ -51,6 +51,7 @@ bool valid_optimizer(const mpt_optimizer *o)
     if (!std::isfinite(o->lr)) return false;
     if (!(o->momentum >= 0.0f && o->momentum < 1.0f)) return false;
     if (!(o->weight_decay >= 0.0f) || !std::isfinite(o->weight_decay)) return false;
+    if (!(o->clip_norm >= 0.0f) || !std::isfinite(o->clip_norm)) return false;
     if (o->kind == MPT_OPT_ADAM && !(o->beta2 >= 0.0f && o->beta2 < 1.0f)) return false;
     if ((o->kind == MPT_OPT_ADAM || o->kind == MPT_OPT_ADAGRAD) && (!(o->eps >= 0.0f) || !std::isfinite(o->eps))) return false;
     return true;
@@ -102,6 +103,7 @@ void make_plan(const mpt_layer_desc *layers, int L, int max_batch, int n_states,
         pl.off_labels[k] = take((size_t)max_batch * 4);
     }
     pl.off_rowloss = take((size_t)max_batch * 4);
+    pl.off_norm = take((size_t)kNormParts * sizeof(double));
     // scratch for split-K partial sums: the largest need of any product of the step that runs on
     // the single-CTA tensor-core kernel (small or thin outputs), capped at 256 MB
     size_t need_max = 0;
@@ -129,7 +131,7 @@ struct mpt_ctx {
     float S, lr, mu;
     bool use_momentum;          // first optimizer state in use
     int opt_kind = MPT_OPT_SGD;
-    float beta2 = 0.0f, eps = 0.0f, wd = 0.0f;
+    float beta2 = 0.0f, eps = 0.0f, wd = 0.0f, clip = 0.0f;
     float *state2 = nullptr;
     int max_batch;
     cudaStream_t stream;
@@ -146,6 +148,7 @@ struct mpt_ctx {
     int staged_batch[2] = {0, 0};
     int stage_w = 0, stage_r = 0;
     float *row_loss;
+    double *norm_parts;   // fixed-partition partial sums of the gradient norm (clipping)
     const uint16_t *x_cur = nullptr;
     int batch = 0;
     bool forward_done = false, have_grads = false, poisoned = false;
@@ -342,16 +345,24 @@ int do_step(mpt_ctx *c)
     CK(cudaMemsetAsync(c->status + ST_OVERFLOW_SEEN, 0, sizeof(uint32_t), c->stream), "status clear");
     cudaError_t e;
     {
-        const double bytes_per_param = 12.0 + 8.0 * (c->use_momentum ? 1 : 0) + 8.0 * (c->state2 ? 1 : 0);
+        const double bytes_per_param = 12.0 + 8.0 * (c->use_momentum ? 1 : 0) + 8.0 * (c->state2 ? 1 : 0) + (c->clip > 0.0f ? 2.0 : 0.0);
         ProfSpan span(c, MPT_PROF_UPDATE, bytes_per_param * (double)c->plan.P_pad);
-        if (c->opt_kind == MPT_OPT_SGD && c->wd == 0.0f)
+        if (c->clip > 0.0f) {
+            // norm over the whole gradient arena (layer padding holds zeros) and the coefficient
+            e = launch_clip_coef(c->g16, c->plan.P_pad, inv, (const float *)(c->status + ST_INV_SCALE), c->clip, c->norm_parts,
+                                 (float *)(c->status + ST_CLIP_COEF), c->stream);
+            c->launches += 2;
+            if (e != cudaSuccess) return cuda_fail(c, e, "clip launch");
+        }
+        if (c->opt_kind == MPT_OPT_SGD && c->wd == 0.0f && c->clip <= 0.0f)
             e = launch_update(c->g16, c->master, c->mom, c->w16, c->plan.P_pad, inv, c->lr, c->mu, c->use_momentum,
                               c->status + ST_OVERFLOW, c->stream, (const float *)(c->status + ST_INV_SCALE));
         else
             e = launch_update_opt(c->opt_kind, c->g16, c->master, c->mom, c->state2, c->w16, c->plan.P_pad, inv, c->lr, c->mu,
                                   c->beta2, c->eps, c->wd, 1.0f, 1.0f, c->status + ST_OVERFLOW, c->stream,
                                   (const float *)(c->status + ST_INV_SCALE),
-                                  c->opt_kind == MPT_OPT_ADAM ? (const float *)(c->status + ST_B1T) : nullptr);
+                                  c->opt_kind == MPT_OPT_ADAM ? (const float *)(c->status + ST_B1T) : nullptr,
+                                  c->clip > 0.0f ? (const float *)(c->status + ST_CLIP_COEF) : nullptr);
     }
     c->launches++;
     if (e != cudaSuccess) return cuda_fail(c, e, "update launch");
@@ -407,7 +418,7 @@ int mpt_workspace_bytes_opt(const mpt_layer_desc *layers, int n_layers, int max_
 int mpt_create(const mpt_layer_desc *layers, int n_layers, float S, float lr, float momentum, int max_batch,
                void *workspace_dev, size_t workspace_bytes, void *cuda_stream, mpt_ctx **out)
 {
-    mpt_optimizer opt = {MPT_OPT_SGD, lr, momentum, 0.0f, 0.0f, 0.0f};
+    mpt_optimizer opt = {MPT_OPT_SGD, lr, momentum, 0.0f, 0.0f, 0.0f, 0.0f};
     return mpt_create_opt(layers, n_layers, S, &opt, max_batch, workspace_dev, workspace_bytes, cuda_stream, out);
 }
 
@@ -425,7 +436,7 @@ int mpt_create_opt(const mpt_layer_desc *layers, int n_layers, float S, const mp
     if (!c) return MPT_ERR_INTERNAL;
     const int n_states = opt_states(*opt);
     c->use_momentum = n_states >= 1;
-    c->opt_kind = opt->kind; c->beta2 = opt->beta2; c->eps = opt->eps; c->wd = opt->weight_decay;
+    c->opt_kind = opt->kind; c->beta2 = opt->beta2; c->eps = opt->eps; c->wd = opt->weight_decay; c->clip = opt->clip_norm;
     make_plan(layers, n_layers, max_batch, n_states, c->plan);
     if (workspace_bytes < c->plan.total) { delete c; return MPT_ERR_WORKSPACE; }
     const float lr = opt->lr, momentum = opt->momentum;
@@ -444,6 +455,7 @@ int mpt_create_opt(const mpt_layer_desc *layers, int n_layers, float S, const mp
         c->labels_stage[k] = (int32_t *)(c->ws + pl.off_labels[k]);
     }
     c->row_loss = (float *)(c->ws + pl.off_rowloss);
+    c->norm_parts = (double *)(c->ws + pl.off_norm);
     c->splitk_ws = pl.splitk_bytes ? (float *)(c->ws + pl.off_splitk) : nullptr;
     c->layers.resize(n_layers);
     for (int l = 0; l < n_layers; l++) {
@@ -817,6 +829,20 @@ int mpt_get_adam_products(mpt_ctx *c, float *b1t_out, float *b2t_out)
     return MPT_OK;
 }
 
+int mpt_get_grad_norm(mpt_ctx *c, float *norm_out, float *coef_out)
+{
+    int r = usable(c);
+    if (r != MPT_OK) return r;
+    if (!norm_out || !coef_out) return fail(c, MPT_ERR_INVALID_ARG, "null output");
+    if (c->clip <= 0.0f) return fail(c, MPT_ERR_STATE, "the context was created without gradient clipping");
+    uint32_t st[ST_WORDS];
+    r = read_status(c, st);
+    if (r != MPT_OK) return r;
+    memcpy(norm_out, &st[ST_GRAD_NORM], 4);
+    memcpy(coef_out, &st[ST_CLIP_COEF], 4);
+    return MPT_OK;
+}
+
 int mpt_set_adam_products(mpt_ctx *c, float b1t, float b2t)
 {
     int r = usable(c);
@@ -906,10 +932,12 @@ int mpt_update_flat(const uint16_t *g16_dev, float *w32_dev, float *v_dev, uint1
 
 int mpt_update_flat_opt(const mpt_optimizer *opt, const uint16_t *g16_dev, float *w32_dev, float *s1_dev, float *s2_dev,
                         uint16_t *w16_dev, size_t n, float inv_S, float b1t, float b2t, int detect, uint32_t *flags_dev,
-                        void *cuda_stream)
+                        void *clip_scratch_dev, void *cuda_stream)
 {
     if (!g16_dev || !w32_dev || !w16_dev || !flags_dev) return MPT_ERR_INVALID_ARG;
     if (!valid_optimizer(opt)) return MPT_ERR_INVALID_ARG;
+    const bool clip = opt->clip_norm > 0.0f;
+    if (clip && (!clip_scratch_dev || ((uintptr_t)clip_scratch_dev & 255) != 0)) return MPT_ERR_INVALID_ARG;
     const int ns = opt_states(*opt);
     if ((ns >= 1 && !s1_dev) || (ns >= 2 && !s2_dev)) return MPT_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)cuda_stream;
@@ -920,10 +948,15 @@ int mpt_update_flat_opt(const mpt_optimizer *opt, const uint16_t *g16_dev, float
     } else {
         e = cudaMemsetAsync(flags_dev + 1, 0, sizeof(uint32_t), st);
     }
+    float *coef_dev = nullptr;
+    if (e == cudaSuccess && clip) {   // scratch: two floats (coefficient, norm), then the partial sums at byte 256
+        coef_dev = (float *)clip_scratch_dev;
+        e = launch_clip_coef(g16_dev, n, inv_S, nullptr, opt->clip_norm, (double *)((char *)clip_scratch_dev + 256), coef_dev, st);
+    }
     if (e == cudaSuccess)
         e = launch_update_opt(opt->kind, g16_dev, w32_dev, ns >= 1 ? s1_dev : nullptr, ns >= 2 ? s2_dev : nullptr, w16_dev, n,
                               inv_S, opt->lr, opt->momentum, opt->beta2, opt->eps, opt->weight_decay, b1t, b2t, flags_dev, st,
-                              nullptr, nullptr);
+                              nullptr, nullptr, coef_dev);
     return e == cudaSuccess ? MPT_OK : MPT_ERR_CUDA;
 }
 

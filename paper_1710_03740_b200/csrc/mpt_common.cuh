@@ -22,6 +22,8 @@ enum StatusWord : int {
     ST_CLEAN_STEPS = 7,   // consecutive steps without overflow since S last changed (dynamic scaling)
     ST_B1T = 8,           // float: beta1^t over the applied (not skipped) steps (Adam)
     ST_B2T = 9,           // float: beta2^t
+    ST_CLIP_COEF = 10,    // float: clipping coefficient of the last step (global-norm clipping)
+    ST_GRAD_NORM = 11,    // float: norm of the unscaled gradients of the last step
     ST_WORDS = 16
 };
 
@@ -70,7 +72,14 @@ cudaError_t launch_softmax_ce(const uint16_t *z, int ldz, const int32_t *labels,
 // steps from device memory and multiplied by beta once more in the kernel.
 cudaError_t launch_update_opt(int kind, const uint16_t *g16, float *w32, float *s1, float *s2, uint16_t *w16, size_t n,
                               float inv_S, float lr, float mu, float b2, float eps, float wd, float b1t, float b2t,
-                              uint32_t *flags, cudaStream_t st, const float *inv_S_dev, const float *betat_dev);
+                              uint32_t *flags, cudaStream_t st, const float *inv_S_dev, const float *betat_dev,
+                              const float *coef_dev = nullptr);
+// Global-norm clipping of the unscaled gradients: a fixed-partition double-precision sum of
+// squares over g16[0..n) into parts[kNormParts], then out2[0] = min(1, clip/(norm + 1e-6)) and
+// out2[1] = norm as FP32.  launch_update_opt multiplies every unscaled gradient by *coef_dev.
+static constexpr int kNormParts = 1184;
+cudaError_t launch_clip_coef(const uint16_t *g16, size_t n, float inv_S, const float *inv_S_dev, float clip, double *parts,
+                             float *out2, cudaStream_t st);
 // End-of-step bookkeeping on the device (one thread): dynamic loss scale (if interval > 0) and
 // Adam's running products beta^t (if adam != 0); both only move on a step that was applied.
 cudaError_t launch_post_step(uint32_t *status, int interval, float backoff, float growth, float min_S, float max_S,

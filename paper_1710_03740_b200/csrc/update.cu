@@ -254,10 +254,11 @@ cudaError_t launch_update(const uint16_t *g16, float *w32, float *v, uint16_t *w
 // One element; every operation rounded separately, in the order documented in mpt.h.
 template <int KIND, bool WD>
 __device__ __forceinline__ void opt1(uint32_t gh, float &w, float &s1, float &s2, float inv, float lr, float mu, float b2,
-                                     float omb1, float omb2, float eps, float wd, float bc1, float bc2, bool &bad)
+                                     float omb1, float omb2, float eps, float wd, float bc1, float bc2, float coef, bool &bad)
 {
     float g = __fmul_rn(h2f_bits(gh), inv);
     bad |= f32_nonfinite(g);
+    g = __fmul_rn(g, coef);     // global-norm clipping coefficient (exactly 1.0f when clipping is off)
     if (WD) g = __fadd_rn(g, __fmul_rn(wd, w));
     float u;
     if (KIND == MPT_OPT_NESTEROV) {
@@ -290,10 +291,12 @@ __global__ void __launch_bounds__(kThreads) k_update_opt(const uint4 *__restrict
                                                          uint4 *__restrict__ w16, size_t n8, float inv, float lr, float mu,
                                                          float b2, float eps, float wd, float b1t, float b2t,
                                                          uint32_t *flags, const float *__restrict__ inv_dev,
-                                                         const float *__restrict__ betat_dev)
+                                                         const float *__restrict__ betat_dev,
+                                                         const float *__restrict__ coef_dev)
 {
     if (*(volatile const uint32_t *)flags != 0u) return;
     if (inv_dev) inv = *inv_dev;
+    const float coef = coef_dev ? *coef_dev : 1.0f;
     if (betat_dev) { b1t = __fmul_rn(betat_dev[0], mu); b2t = __fmul_rn(betat_dev[1], b2); }
     const float bc1 = __fsub_rn(1.0f, b1t), bc2 = __fsub_rn(1.0f, b2t);
     const float omb1 = __fsub_rn(1.0f, mu), omb2 = __fsub_rn(1.0f, b2);
@@ -325,7 +328,7 @@ __global__ void __launch_bounds__(kThreads) k_update_opt(const uint4 *__restrict
             for (int e = 0; e < 8; e++) {
                 const uint32_t gh = (e & 1) ? (gw[e >> 1] >> 16) : (gw[e >> 1] & 0xFFFFu);
                 opt1<KIND, WD>(gh, wf[e >> 2][e & 3], af[e >> 2][e & 3], bf[e >> 2][e & 3], inv, lr, mu, b2, omb1, omb2, eps,
-                               wd, bc1, bc2, bad);
+                               wd, bc1, bc2, coef, bad);
             }
             uint4 h;
             h.x = f2h_bits(w0[u].x) | (f2h_bits(w0[u].y) << 16);
@@ -345,10 +348,12 @@ template <int KIND, bool WD>
 __global__ void k_update_opt_scalar(const uint16_t *__restrict__ g16, float *__restrict__ w32, float *__restrict__ s1p,
                                     float *__restrict__ s2p, uint16_t *__restrict__ w16, size_t begin, size_t n, float inv,
                                     float lr, float mu, float b2, float eps, float wd, float b1t, float b2t, uint32_t *flags,
-                                    const float *__restrict__ inv_dev, const float *__restrict__ betat_dev)
+                                    const float *__restrict__ inv_dev, const float *__restrict__ betat_dev,
+                                    const float *__restrict__ coef_dev)
 {
     if (*(volatile const uint32_t *)flags != 0u) return;
     if (inv_dev) inv = *inv_dev;
+    const float coef = coef_dev ? *coef_dev : 1.0f;
     if (betat_dev) { b1t = __fmul_rn(betat_dev[0], mu); b2t = __fmul_rn(betat_dev[1], b2); }
     const float bc1 = __fsub_rn(1.0f, b1t), bc2 = __fsub_rn(1.0f, b2t);
     const float omb1 = __fsub_rn(1.0f, mu), omb2 = __fsub_rn(1.0f, b2);
@@ -357,7 +362,7 @@ __global__ void k_update_opt_scalar(const uint16_t *__restrict__ g16, float *__r
     bool bad = false;
     for (size_t i = begin + (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
         float w = w32[i], a = use_s1 ? s1p[i] : 0.0f, b = KIND == MPT_OPT_ADAM ? s2p[i] : 0.0f;
-        opt1<KIND, WD>(g16[i], w, a, b, inv, lr, mu, b2, omb1, omb2, eps, wd, bc1, bc2, bad);
+        opt1<KIND, WD>(g16[i], w, a, b, inv, lr, mu, b2, omb1, omb2, eps, wd, bc1, bc2, coef, bad);
         w32[i] = w;
         if (use_s1) s1p[i] = a;
         if (KIND == MPT_OPT_ADAM) s2p[i] = b;
@@ -369,7 +374,8 @@ __global__ void k_update_opt_scalar(const uint16_t *__restrict__ g16, float *__r
 template <int KIND, bool WD>
 static cudaError_t launch_opt_variant(const uint16_t *g16, float *w32, float *s1, float *s2, uint16_t *w16, size_t n,
                                       float inv_S, float lr, float mu, float b2, float eps, float wd, float b1t, float b2t,
-                                      uint32_t *flags, cudaStream_t st, const float *inv_dev, const float *betat_dev)
+                                      uint32_t *flags, cudaStream_t st, const float *inv_dev, const float *betat_dev,
+                                      const float *coef_dev)
 {
     uintptr_t bits = (uintptr_t)g16 | (uintptr_t)w32 | (uintptr_t)w16 | (uintptr_t)s1 | (uintptr_t)s2;
     size_t n8 = (bits & 15) == 0 ? n / 8 : 0;
@@ -377,25 +383,26 @@ static cudaError_t launch_opt_variant(const uint16_t *g16, float *w32, float *s1
         const size_t per_cta = (size_t)kThreads * kOptVec;
         k_update_opt<KIND, WD><<<(unsigned)((n8 + per_cta - 1) / per_cta), kThreads, 0, st>>>(
             (const uint4 *)g16, (float4 *)w32, (float4 *)s1, (float4 *)s2, (uint4 *)w16, n8, inv_S, lr, mu, b2, eps, wd, b1t, b2t,
-            flags, inv_dev, betat_dev);
+            flags, inv_dev, betat_dev, coef_dev);
     }
     if (n8 * 8 < n)
         k_update_opt_scalar<KIND, WD><<<grid_for(n - n8 * 8), kThreads, 0, st>>>(g16, w32, s1, s2, w16, n8 * 8, n, inv_S, lr, mu, b2,
-                                                                                eps, wd, b1t, b2t, flags, inv_dev, betat_dev);
+                                                                                eps, wd, b1t, b2t, flags, inv_dev, betat_dev, coef_dev);
     return cudaGetLastError();
 }
 
 cudaError_t launch_update_opt(int kind, const uint16_t *g16, float *w32, float *s1, float *s2, uint16_t *w16, size_t n,
                               float inv_S, float lr, float mu, float b2, float eps, float wd, float b1t, float b2t,
-                              uint32_t *flags, cudaStream_t st, const float *inv_dev, const float *betat_dev)
+                              uint32_t *flags, cudaStream_t st, const float *inv_dev, const float *betat_dev,
+                              const float *coef_dev)
 {
     if (n == 0) return cudaSuccess;
 #define MPT_OPT_CASE(K)                                                                                                     \
     case K:                                                                                                                 \
         return wd != 0.0f ? launch_opt_variant<K, true>(g16, w32, s1, s2, w16, n, inv_S, lr, mu, b2, eps, wd, b1t, b2t, flags, \
-                                                        st, inv_dev, betat_dev)                                             \
+                                                        st, inv_dev, betat_dev, coef_dev)                                   \
                           : launch_opt_variant<K, false>(g16, w32, s1, s2, w16, n, inv_S, lr, mu, b2, eps, wd, b1t, b2t, flags, \
-                                                         st, inv_dev, betat_dev);
+                                                         st, inv_dev, betat_dev, coef_dev);
     switch (kind) {
         MPT_OPT_CASE(MPT_OPT_SGD)
         MPT_OPT_CASE(MPT_OPT_NESTEROV)
@@ -463,6 +470,79 @@ cudaError_t launch_scale_adjust(uint32_t *status, int interval, float backoff, f
                                 cudaStream_t st)
 {
     k_scale_adjust<<<1, 1, 0, st>>>(status, interval, backoff, growth, min_S, max_S);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------- global-norm gradient clipping
+
+// Section 3.2: clipping thresholds act on the UNSCALED gradients.  The squared norm is accumulated
+// in double (section 3.3: reductions in higher precision than the stored values) with a fixed
+// partition, so the same input gives the same bits on every run: thread t of CTA b sums the
+// vectors b*kThreads + t + k*kNormParts*kThreads in increasing k, a CTA combines its threads with
+// a fixed shuffle/shared tree into parts[b], and one CTA combines the parts the same way.
+__device__ __forceinline__ double block_sum_fixed(double v, double *sh)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    const int warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    if ((threadIdx.x & 31) == 0) sh[warp] = v;
+    __syncthreads();
+    double total = 0.0;
+    if (threadIdx.x == 0)
+        for (int w = 0; w < nwarps; w++) total += sh[w];
+    return total;   // valid in thread 0
+}
+
+__global__ void __launch_bounds__(kThreads) k_grad_sqnorm(const uint16_t *__restrict__ g16, size_t n, size_t n8, float inv,
+                                                          const float *__restrict__ inv_dev, double *__restrict__ parts)
+{
+    __shared__ double sh[kThreads / 32];
+    if (inv_dev) inv = *inv_dev;
+    double acc = 0.0;
+    const uint4 *gv = (const uint4 *)g16;
+    const size_t stride = (size_t)gridDim.x * kThreads;
+    for (size_t j = (size_t)blockIdx.x * kThreads + threadIdx.x; j < n8; j += stride) {
+        const uint4 q = __ldcs(gv + j);
+        const uint32_t gw[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+        for (int e = 0; e < 8; e++) {
+            const uint32_t gh = (e & 1) ? (gw[e >> 1] >> 16) : (gw[e >> 1] & 0xFFFFu);
+            const double v = (double)__fmul_rn(h2f_bits(gh), inv);
+            acc += v * v;
+        }
+    }
+    if (blockIdx.x == 0)      // elements past the last whole vector (or everything, for unaligned input)
+        for (size_t i = n8 * 8 + threadIdx.x; i < n; i += kThreads) {
+            const double v = (double)__fmul_rn(h2f_bits(g16[i]), inv);
+            acc += v * v;
+        }
+    const double total = block_sum_fixed(acc, sh);
+    if (threadIdx.x == 0) parts[blockIdx.x] = total;
+}
+
+// coef = min(1, clip / (sqrt(total) + 1e-6)) rounded to FP32; out[0] = coef, out[1] = norm (FP32).
+__global__ void __launch_bounds__(1024) k_clip_coef(const double *__restrict__ parts, int count, float clip,
+                                                    float *__restrict__ out)
+{
+    __shared__ double sh[32];
+    double acc = 0.0;
+    for (int i = threadIdx.x; i < count; i += 1024) acc += parts[i];
+    const double total = block_sum_fixed(acc, sh);
+    if (threadIdx.x == 0) {
+        const double norm = sqrt(total);
+        out[0] = (float)fmin(1.0, (double)clip / (norm + 1e-6));
+        out[1] = (float)norm;
+    }
+}
+
+cudaError_t launch_clip_coef(const uint16_t *g16, size_t n, float inv_S, const float *inv_dev, float clip, double *parts,
+                             float *out2, cudaStream_t st)
+{
+    const size_t n8 = ((uintptr_t)g16 & 15) == 0 ? n / 8 : 0;
+    size_t want = (n8 + kThreads - 1) / kThreads;
+    const int grid = (int)(want < 1 ? 1 : (want > (size_t)kNormParts ? (size_t)kNormParts : want));
+    k_grad_sqnorm<<<grid, kThreads, 0, st>>>(g16, n, n8, inv_S, inv_dev, parts);
+    k_clip_coef<<<1, 1024, 0, st>>>(parts, grid, clip, out2);
     return cudaGetLastError();
 }
 

@@ -166,8 +166,9 @@ def bench_update(n, momentum, iters):
             "working_set_mb": bpp * n / 2e6, "flags": flags.tolist()}
 
 
-def bench_update_opt(n, kind, wd, iters):
-    """Master pass with Nesterov (1), Adagrad (2) or Adam (3), optional weight decay."""
+def bench_update_opt(n, kind, wd, iters, clip=0.0):
+    """Master pass with Nesterov (1), Adagrad (2) or Adam (3), optional weight decay and global-norm
+    clipping (one more read of the FP16 gradients: +2 bytes per parameter)."""
     g = torch.Generator(device="cuda").manual_seed(3)
     g16 = (torch.randn(n, device="cuda", generator=g) * 37).half()
     w32 = torch.randn(n, device="cuda", generator=g)
@@ -175,11 +176,14 @@ def bench_update_opt(n, kind, wd, iters):
     s2 = torch.zeros(n, device="cuda") if kind == mpt.OPT_ADAM else None
     w16 = torch.empty(n, dtype=torch.half, device="cuda")
     flags = torch.zeros(2, dtype=torch.int32, device="cuda")
-    opt = mpt.Optimizer(kind, 1e-4, 0.9, 0.999, 1e-8, wd)
-    fn = lambda: mpt.mpt_update_flat_opt(opt, g16, w32, s1, s2, w16, n, 1.0 / 512, 0.81, 0.998, False, flags)  # noqa: E731
+    opt = mpt.Optimizer(kind, 1e-4, 0.9, 0.999, 1e-8, wd, clip)
+    scratch = torch.zeros(mpt.CLIP_SCRATCH_BYTES // 4, device="cuda") if clip > 0 else None
+    fn = lambda: mpt.mpt_update_flat_opt(opt, g16, w32, s1, s2, w16, n, 1.0 / 512, 0.81, 0.998, False, flags,  # noqa: E731
+                                         clip_scratch=scratch)
     best, sus = _time(fn, iters)
-    bpp = 28 if kind == mpt.OPT_ADAM else 20
+    bpp = (28 if kind == mpt.OPT_ADAM else 20) + (2 if clip > 0 else 0)
     return {"kernel": "update_opt", "optimizer": ["sgd", "nesterov", "adagrad", "adam"][kind], "weight_decay": wd,
+            "clip_norm": clip,
             "params": n, "bytes_per_param": bpp, "best_ms": best, "sustained_ms": sus, "best_gbs": bpp * n / best / 1e6,
             "sustained_gbs": bpp * n / sus / 1e6, "flags": flags.tolist()}
 
@@ -260,6 +264,7 @@ def main():
     u.add_argument("--momentum", type=int, default=1)
     u.add_argument("--optimizer", default="sgd", choices=["sgd", "nesterov", "adagrad", "adam"])
     u.add_argument("--weight-decay", type=float, default=0.0)
+    u.add_argument("--clip-norm", type=float, default=0.0)
     u.add_argument("--iters", type=int, default=20)
     s = sub.add_parser("softmax")
     s.add_argument("--rows", type=int, default=4096)
@@ -282,10 +287,10 @@ def main():
                 print(json.dumps(res), flush=True)
     elif args.cmd == "update":
         kind = ["sgd", "nesterov", "adagrad", "adam"].index(args.optimizer)
-        if kind == 0 and args.weight_decay == 0.0:
+        if kind == 0 and args.weight_decay == 0.0 and args.clip_norm == 0.0:
             print(json.dumps(bench_update(args.params, args.momentum, args.iters)), flush=True)
         else:
-            print(json.dumps(bench_update_opt(args.params, kind, args.weight_decay, args.iters)), flush=True)
+            print(json.dumps(bench_update_opt(args.params, kind, args.weight_decay, args.iters, args.clip_norm)), flush=True)
     else:
         print(json.dumps(bench_softmax(args.rows, args.classes, args.iters)), flush=True)
 

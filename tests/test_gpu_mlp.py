@@ -356,6 +356,54 @@ def test_optimizer_variants_end_to_end(kind):
         assert abs(b1t - 0.9 ** 5) < 1e-6                        # five applied steps out of six
 
 
+@pytest.mark.parametrize("kind,clip", [(0, 0.05), (3, 0.05), (1, 1e6)])
+def test_global_norm_clipping_end_to_end(kind, clip):
+    """Clipping of the unscaled gradients by their global norm (section 3.2), with dynamic scaling
+    changing S under it: norm and coefficient equal to the oracle's on the device's own gradient
+    bits, update bit-exact, and a bound far above the norm leaves the trajectory of the unclipped
+    run untouched (coefficient exactly 1)."""
+    from paper_1710_03740_b200 import binding as b
+    cfg = dict(inputs.MLP_CONFIGS["tiny"])
+    lr = 0.001 if kind == 3 else 0.05
+    opt = b.Optimizer(kind, lr, 0.9, 0.999, 1e-8, 1e-4, clip)
+    masters = inputs.mlp_masters(cfg)
+    X, Y = inputs.mlp_batches(cfg, 6)
+    net = b.Context(cfg["layers"], 2.0 ** 12, lr, 0.9, cfg["batch"], optimizer=opt)
+    net.set_dynamic_scale(True, 2, 1.0, 2.0 ** 20)
+    chk = OracleMLP(cfg["layers"], 2.0 ** 12, lr, 0.9)
+    chk.set_optimizer(kind, lr, mu=0.9, b2=0.999, eps=1e-8, wd=1e-4, clip=clip)
+    chk.set_dynamic_scale(2, 1.0, 2.0 ** 20)
+    plain = None
+    if clip >= 1e6:
+        plain = b.Context(cfg["layers"], 2.0 ** 12, lr, 0.9, cfg["batch"], optimizer=b.Optimizer(kind, lr, 0.9, 0.999, 1e-8, 1e-4))
+        plain.set_dynamic_scale(True, 2, 1.0, 2.0 ** 20)
+    for l, w in enumerate(masters):
+        net.set_master(l, w); chk.set_master(l, w)
+        if plain is not None:
+            plain.set_master(l, w)
+    seen_clipped = False
+    for t in range(6):
+        xd, yd = dev(X[t].view(np.uint16)), dev(Y[t])
+        net.forward(xd)
+        net.backward_scaled(yd)
+        for l in range(2):
+            chk.set_grad(l, net.get_tensor(b.T_GRAD16, l))
+        assert net.step() == chk.step() == 0
+        norm, coef = net.get_grad_norm()
+        assert coef == float(chk.last_coef), (t, coef, float(chk.last_coef))
+        seen_clipped |= coef < 1.0
+        assert net.get_scale() == float(chk.S)
+        for l in range(2):
+            assert net.get_master(l).tobytes() == chk.w32[l].tobytes(), (t, l)
+        if plain is not None:
+            plain.forward(xd)
+            plain.backward_scaled(yd)
+            assert plain.step() == 0
+            for l in range(2):
+                assert net.get_master(l).tobytes() == plain.get_master(l).tobytes()
+    assert seen_clipped == (clip < 1e6)
+
+
 def test_error_paths():
     from paper_1710_03740_b200 import binding as b
     cfg = inputs.MLP_CONFIGS["tiny"]

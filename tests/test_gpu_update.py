@@ -182,3 +182,51 @@ def test_optimizer_variants_bit_exact(kind, wd, n, misalign):
     if kind == 3:
         assert np.array_equal(cd[pad:pad + n].cpu().numpy().view(np.uint32), c_ref.view(np.uint32))
     assert np.array_equal(host_u16(hd[pad:pad + n]), h_ref)
+
+
+@pytest.mark.parametrize("kind", [0, 1, 2, 3])
+@pytest.mark.parametrize("n,misalign", [(1 << 20, 0), (300007, 0), (4099, 3), (5, 0)])
+def test_clipped_update_bit_exact(kind, n, misalign):
+    """Global-norm clipping in the stateless pass: the coefficient (double-precision norm over a
+    fixed partition, rounded to FP32) equals the oracle's, and the update with it is bit-exact;
+    unaligned arrays take the scalar path of both kernels."""
+    from paper_1710_03740_b200 import binding as b
+    f = np.float32
+    rng = np.random.default_rng(1000 + n + kind)
+    S, lr, clip = 1024.0, 0.01, 0.5
+    g16 = (rng.standard_normal(n) * 30).astype(np.float16)
+    w = rng.standard_normal(n).astype(np.float32)
+    s1 = (np.abs(rng.standard_normal(n)) * 0.01).astype(np.float32)
+    s2 = (np.abs(rng.standard_normal(n)) * 0.01).astype(np.float32)
+    inv = f(1.0) / f(S)
+    coef = mpo.clip_coef(mpo.grad_sqnorm(g16, inv), clip)
+    assert coef < 1.0 or n == 5
+    w_ref, a_ref, c_ref, h_ref = w.copy(), s1.copy(), s2.copy(), np.zeros(n, dtype=np.uint16)
+    b1t, b2t = f(0.9), f(0.999)
+    mpo.update_apply_clip(kind, g16, w_ref, a_ref, c_ref if kind == 3 else None, h_ref, inv, coef, f(lr), f(0.9), f(0.999),
+                          f(1e-8), f(1e-3), f(1.0) - b1t, f(1.0) - b2t)
+    pad = misalign
+    gd = torch.zeros(n + 8, dtype=torch.int16, device="cuda")
+    wd_ = torch.zeros(n + 8, dtype=torch.float32, device="cuda")
+    ad = torch.zeros(n + 8, dtype=torch.float32, device="cuda")
+    cd = torch.zeros(n + 8, dtype=torch.float32, device="cuda")
+    hd = torch.zeros(n + 8, dtype=torch.int16, device="cuda")
+    gd[pad:pad + n] = dev(g16.view(np.uint16)); wd_[pad:pad + n] = dev(w); ad[pad:pad + n] = dev(s1); cd[pad:pad + n] = dev(s2)
+    flags = torch.zeros(2, dtype=torch.int32, device="cuda")
+    scratch = torch.zeros(b.CLIP_SCRATCH_BYTES // 4, dtype=torch.float32, device="cuda")
+    opt = b.Optimizer(kind, lr, 0.9, 0.999, 1e-8, 1e-3, clip)
+    for _ in range(2):          # the second call checks that the result does not depend on leftover scratch
+        wd_[pad:pad + n] = dev(w); ad[pad:pad + n] = dev(s1); cd[pad:pad + n] = dev(s2)
+        b.mpt_update_flat_opt(opt, gd[pad:], wd_[pad:], ad[pad:], cd[pad:] if kind == 3 else None, hd[pad:], n, float(inv),
+                              float(b1t), float(b2t), True, flags, clip_scratch=scratch)
+        torch.cuda.synchronize()
+        assert flags.tolist() == [0, 0]
+        got = scratch[:2].cpu().numpy()
+        assert got[0] == coef
+        ref_norm = np.sqrt(((g16.astype(np.float32) * inv).astype(np.float64) ** 2).sum())
+        assert abs(float(got[1]) - ref_norm) <= 1e-6 * ref_norm
+        assert np.array_equal(wd_[pad:pad + n].cpu().numpy().view(np.uint32), w_ref.view(np.uint32))
+        assert np.array_equal(ad[pad:pad + n].cpu().numpy().view(np.uint32), a_ref.view(np.uint32))
+        assert np.array_equal(host_u16(hd[pad:pad + n]), h_ref)
+    with pytest.raises(b.MptError):     # clipping without the scratch is refused
+        b.mpt_update_flat_opt(opt, gd[pad:], wd_[pad:], ad[pad:], cd[pad:], hd[pad:], n, float(inv), 0.9, 0.999, True, flags)
