@@ -456,3 +456,153 @@ void mpo_update_apply_clip(int kind, const uint16_t *g16, float *w32, float *s1,
         w16[i] = mpo_f2h(w);
     }
 }
+
+/* ------------------------------------------------------------------------
+ * LSTM cell with fused gate arithmetic (sections 3.3 and 4.6: recurrent matrix products on
+ * FP16 inputs with FP32 accumulation; point-wise gate arithmetic is memory-bound and may run
+ * in either precision - here FP32 arithmetic on FP16 storage).
+ *
+ * Row b of XR holds [x_t ; r_{t-1}] (K values).  Wg is [4H][K], row 4j+q = gate q of cell j
+ * with q: 0 input, 1 forget, 2 candidate, 3 output; bias16 [4H] in the same order.
+ *   pre_q = (sum_k XR[b,k]*Wg[4j+q,k], ascending k, binary32) + h2f(bias16[4j+q])
+ *   i = sig(pre_0)  f = sig(pre_1)  g = tanh(pre_2)  o = sig(pre_3),  sig(x) = 1/(1+exp(-x))
+ *   acts[b,4j+q] = rn16(gate value)
+ *   c = f*c_prev + i*g  (two products, one sum, each rounded to binary32);  c16 = rn16(c)
+ *   h16 = rn16(o * tanh(h2f(c16)))     (consumers only ever see the stored cell state)
+ * pre32 (optional) receives the binary32 pre-activations, absdot (optional) sum |a*b| per gate.
+ */
+static float mpo_sigmoid(float x)
+{
+    float e = expf(-x);
+    float d = 1.0f + e;
+    return 1.0f / d;
+}
+
+void mpo_lstm_cell_fwd(int B, int H, int K, const uint16_t *XR, int ldxr, const uint16_t *Wg, int ldw,
+                       const uint16_t *bias16, const uint16_t *c_prev, int ldcp, uint16_t *acts, int ldacts,
+                       uint16_t *c_out, int ldco, uint16_t *h_out, int ldh, float *pre32, double *absdot)
+{
+    const int N = 4 * H;
+    float *Wf = (float *)malloc((size_t)(K > 0 ? K : 1) * (size_t)N * sizeof(float));   /* [K][N] */
+#pragma omp parallel for schedule(static)
+    for (int k = 0; k < K; k++)
+        for (int n = 0; n < N; n++) Wf[(size_t)k * N + n] = mpo_h2f(Wg[(size_t)n * ldw + k]);
+#pragma omp parallel
+    {
+        float *acc = (float *)malloc((size_t)N * sizeof(float));
+        double *aacc = (double *)malloc((size_t)N * sizeof(double));
+#pragma omp for schedule(static)
+        for (int b = 0; b < B; b++) {
+            for (int n = 0; n < N; n++) { acc[n] = 0.0f; aacc[n] = 0.0; }
+            for (int k = 0; k < K; k++) {
+                float a = mpo_h2f(XR[(size_t)b * ldxr + k]);
+                const float *wrow = Wf + (size_t)k * N;
+                for (int n = 0; n < N; n++) {
+                    float p = a * wrow[n];
+                    acc[n] = acc[n] + p;
+                    aacc[n] += fabs((double)a * (double)wrow[n]);
+                }
+            }
+            for (int j = 0; j < H; j++) {
+                float pre[4];
+                for (int q = 0; q < 4; q++) {
+                    pre[q] = acc[4 * j + q] + mpo_h2f(bias16[4 * j + q]);
+                    if (pre32) pre32[(size_t)b * N + 4 * j + q] = pre[q];
+                    if (absdot) absdot[(size_t)b * N + 4 * j + q] = aacc[4 * j + q];
+                }
+                float gi = mpo_sigmoid(pre[0]), gf = mpo_sigmoid(pre[1]), gg = tanhf(pre[2]), go = mpo_sigmoid(pre[3]);
+                uint16_t *arow = acts + (size_t)b * ldacts + 4 * j;
+                arow[0] = mpo_f2h(gi); arow[1] = mpo_f2h(gf); arow[2] = mpo_f2h(gg); arow[3] = mpo_f2h(go);
+                float cp = mpo_h2f(c_prev[(size_t)b * ldcp + j]);
+                float t1 = gf * cp;
+                float t2 = gi * gg;
+                float c = t1 + t2;
+                uint16_t c16 = mpo_f2h(c);
+                c_out[(size_t)b * ldco + j] = c16;
+                float tc = tanhf(mpo_h2f(c16));
+                float h = go * tc;
+                h_out[(size_t)b * ldh + j] = mpo_f2h(h);
+            }
+        }
+        free(acc);
+        free(aacc);
+    }
+    free(Wf);
+}
+
+/*
+ * Backward of the gate arithmetic for one time step, from stored FP16 values (the chain rule
+ * of the forward formulas; every operation one binary32 rounding, in the order written):
+ *   tc = tanh(h2f(c16));  dh, dc_next: scaled gradients wrt h_t and (from step t+1) wrt c_t
+ *   dc  = (dh*o)*(1 - tc*tc) + dc_next
+ *   dpre_o = (dh*tc) * (o*(1-o))
+ *   dpre_i = (dc*g)  * (i*(1-i))
+ *   dpre_f = (dc*cp) * (f*(1-f))
+ *   dpre_g = (dc*i)  * (1 - g*g)
+ *   dc_prev = dc*f
+ * dG[b,4j+q] = rn16(dpre_q), dc_prev16 = rn16(dc_prev).  dc_next may be NULL (last step: zero).
+ */
+void mpo_lstm_cell_bwd(int B, int H, const uint16_t *dh, int lddh, const uint16_t *dc_next, int lddc,
+                       const uint16_t *acts, int ldacts, const uint16_t *c_prev, int ldcp, const uint16_t *c16,
+                       int ldc, uint16_t *dG, int lddg, uint16_t *dc_prev, int lddcp)
+{
+#pragma omp parallel for schedule(static)
+    for (int b = 0; b < B; b++)
+        for (int j = 0; j < H; j++) {
+            const uint16_t *arow = acts + (size_t)b * ldacts + 4 * j;
+            float gi = mpo_h2f(arow[0]), gf = mpo_h2f(arow[1]), gg = mpo_h2f(arow[2]), go = mpo_h2f(arow[3]);
+            float cp = mpo_h2f(c_prev[(size_t)b * ldcp + j]);
+            float tc = tanhf(mpo_h2f(c16[(size_t)b * ldc + j]));
+            float dhv = mpo_h2f(dh[(size_t)b * lddh + j]);
+            float dcn = dc_next ? mpo_h2f(dc_next[(size_t)b * lddc + j]) : 0.0f;
+            float a1 = dhv * go;
+            float a2 = tc * tc;
+            float a3 = 1.0f - a2;
+            float a4 = a1 * a3;
+            float dc = a4 + dcn;
+            float o1 = dhv * tc;
+            float o2 = 1.0f - go;
+            float o3 = go * o2;
+            float dpo = o1 * o3;
+            float i1 = dc * gg;
+            float i2 = 1.0f - gi;
+            float i3 = gi * i2;
+            float dpi = i1 * i3;
+            float f1 = dc * cp;
+            float f2 = 1.0f - gf;
+            float f3 = gf * f2;
+            float dpf = f1 * f3;
+            float g1 = dc * gi;
+            float g2 = gg * gg;
+            float g3 = 1.0f - g2;
+            float dpg = g1 * g3;
+            float dcp = dc * gf;
+            uint16_t *drow = dG + (size_t)b * lddg + 4 * j;
+            drow[0] = mpo_f2h(dpi); drow[1] = mpo_f2h(dpf); drow[2] = mpo_f2h(dpg); drow[3] = mpo_f2h(dpo);
+            dc_prev[(size_t)b * lddcp + j] = mpo_f2h(dcp);
+        }
+}
+
+/* Bias gradient: column sums of the FP16 gate gradients over all rows, accumulated in binary32
+ * in ascending row order (section 3.3: reductions in FP32), rounded to FP16 on store. */
+void mpo_bias_grad(const uint16_t *dG, size_t rows, int cols, int ld, uint16_t *db16, float *db32)
+{
+#pragma omp parallel for schedule(static)
+    for (int n = 0; n < cols; n++) {
+        float s = 0.0f;
+        for (size_t r = 0; r < rows; r++) s = s + mpo_h2f(dG[r * (size_t)ld + n]);
+        if (db32) db32[n] = s;
+        db16[n] = mpo_f2h(s);
+    }
+}
+
+/* out = rn16(h2f(a) + h2f(b)) element-wise over a [rows, cols] block (gradient of a value that is
+ * consumed twice: by the layer above and by the next time step). */
+void mpo_add_f16(const uint16_t *a, int lda, const uint16_t *b, int ldb, uint16_t *out, int ldo, int rows, int cols)
+{
+    for (int r = 0; r < rows; r++)
+        for (int n = 0; n < cols; n++) {
+            float s = mpo_h2f(a[(size_t)r * lda + n]) + mpo_h2f(b[(size_t)r * ldb + n]);
+            out[(size_t)r * ldo + n] = mpo_f2h(s);
+        }
+}

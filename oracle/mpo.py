@@ -75,6 +75,17 @@ def lib() -> ctypes.CDLL:
         L.mpo_update_apply_clip.restype = None
         L.mpo_update_apply_clip.argtypes = [c.c_int, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p,
                                             c.c_size_t] + [c.c_float] * 9
+        L.mpo_lstm_cell_fwd.restype = None
+        L.mpo_lstm_cell_fwd.argtypes = [c.c_int, c.c_int, c.c_int, c.c_void_p, c.c_int, c.c_void_p, c.c_int, c.c_void_p,
+                                        c.c_void_p, c.c_int, c.c_void_p, c.c_int, c.c_void_p, c.c_int, c.c_void_p, c.c_int,
+                                        c.c_void_p, c.c_void_p]
+        L.mpo_lstm_cell_bwd.restype = None
+        L.mpo_lstm_cell_bwd.argtypes = [c.c_int, c.c_int, c.c_void_p, c.c_int, c.c_void_p, c.c_int, c.c_void_p, c.c_int,
+                                        c.c_void_p, c.c_int, c.c_void_p, c.c_int, c.c_void_p, c.c_int, c.c_void_p, c.c_int]
+        L.mpo_bias_grad.restype = None
+        L.mpo_bias_grad.argtypes = [c.c_void_p, c.c_size_t, c.c_int, c.c_int, c.c_void_p, c.c_void_p]
+        L.mpo_add_f16.restype = None
+        L.mpo_add_f16.argtypes = [c.c_void_p, c.c_int, c.c_void_p, c.c_int, c.c_void_p, c.c_int, c.c_int, c.c_int]
         _lib = L
     return _lib
 
@@ -239,3 +250,59 @@ def update_apply_clip(kind, g16, w32, s1, s2, w16, inv_S, coef, lr, mu, b2=0.0, 
     g = _u16(g16)
     lib().mpo_update_apply_clip(int(kind), _ptr(g), _ptr(w32), _ptr(s1), _ptr(s2), _ptr(w16), g.size, float(inv_S),
                                 float(coef), float(lr), float(mu), float(b2), float(eps), float(wd), float(bc1), float(bc2))
+
+
+def _ld(a):
+    """Row pitch in elements of a 2-D array whose rows are contiguous."""
+    assert a.ndim == 2 and a.strides[1] == a.itemsize
+    return a.strides[0] // a.itemsize if a.shape[0] > 1 else a.shape[1]
+
+
+def lstm_cell_fwd(xr, Wg, bias16, c_prev, want_pre=False):
+    """One time step of the LSTM cell (see mpo.c): xr [B,K], Wg [4H,K] gate-interleaved rows,
+    bias16 [4H], c_prev [B,H].  Returns (acts [B,4H], c [B,H], h [B,H]) as uint16 bit patterns,
+    plus (pre32 float32 [B,4H], absdot float64 [B,4H]) when want_pre."""
+    xr, Wg, bias16, c_prev = _u16(xr), _u16(Wg), np.ascontiguousarray(_u16(bias16)), _u16(c_prev)
+    B, K = xr.shape
+    N = Wg.shape[0]
+    H = N // 4
+    assert N == 4 * H and Wg.shape[1] == K and c_prev.shape == (B, H) and bias16.shape == (N,)
+    acts = np.zeros((B, N), dtype=np.uint16)
+    c = np.zeros((B, H), dtype=np.uint16)
+    h = np.zeros((B, H), dtype=np.uint16)
+    pre = np.zeros((B, N), dtype=np.float32) if want_pre else None
+    ab = np.zeros((B, N), dtype=np.float64) if want_pre else None
+    lib().mpo_lstm_cell_fwd(B, H, K, _ptr(xr), _ld(xr), _ptr(Wg), _ld(Wg), _ptr(bias16), _ptr(c_prev), _ld(c_prev),
+                            _ptr(acts), N, _ptr(c), H, _ptr(h), H, _ptr(pre), _ptr(ab))
+    if want_pre:
+        return acts, c, h, pre, ab
+    return acts, c, h
+
+
+def lstm_cell_bwd(dh, dc_next, acts, c_prev, c):
+    """Backward of the gate arithmetic of one time step: returns (dG [B,4H], dc_prev [B,H])."""
+    dh, acts, c_prev, c = _u16(dh), _u16(acts), _u16(c_prev), _u16(c)
+    B, H = dh.shape
+    dcn = None if dc_next is None else _u16(dc_next)
+    dG = np.zeros((B, 4 * H), dtype=np.uint16)
+    dcp = np.zeros((B, H), dtype=np.uint16)
+    lib().mpo_lstm_cell_bwd(B, H, _ptr(dh), _ld(dh), _ptr(dcn), _ld(dcn) if dcn is not None else 0, _ptr(acts), _ld(acts),
+                            _ptr(c_prev), _ld(c_prev), _ptr(c), _ld(c), _ptr(dG), 4 * H, _ptr(dcp), H)
+    return dG, dcp
+
+
+def bias_grad(dG):
+    """Column sums (binary32, ascending rows) of a [rows, cols] FP16 array: (db16, db32)."""
+    dG = _u16(dG)
+    rows, cols = dG.shape
+    db16 = np.zeros(cols, dtype=np.uint16)
+    db32 = np.zeros(cols, dtype=np.float32)
+    lib().mpo_bias_grad(_ptr(dG), rows, cols, _ld(dG), _ptr(db16), _ptr(db32))
+    return db16, db32
+
+
+def add_f16(a, b):
+    a, b = _u16(a), _u16(b)
+    out = np.zeros(a.shape, dtype=np.uint16)
+    lib().mpo_add_f16(_ptr(a), _ld(a), _ptr(b), _ld(b), _ptr(out), a.shape[1], a.shape[0], a.shape[1])
+    return out
