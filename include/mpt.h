@@ -335,6 +335,87 @@ int mpt_update_flat_opt(const mpt_optimizer *opt, const uint16_t *g16_dev, float
                         uint16_t *w16_dev, size_t n, float inv_S, float b1t, float b2t, int detect, uint32_t *flags_dev,
                         void *clip_scratch_dev, void *cuda_stream);
 
+/* ------------------------------------------------------------ LSTM layer with projection
+ *
+ * The recurrent layer of the paper's language model (section 4.6: 8192 cells projected to 1024)
+ * in the mixed-precision recipe: FP16 storage, recurrent products with FP32 accumulation
+ * (section 3.3), point-wise gate arithmetic in FP32 on the accumulators (section 3.3 leaves the
+ * precision of memory-bound point-wise work open), reductions in FP32.  Per time step t:
+ *   pre   = [x_t ; r_{t-1}] . Wg^T + bias         FP32 (never stored)
+ *   i, f, o = sigmoid(pre_0, pre_1, pre_3), g = tanh(pre_2);  sigmoid(x) = 1/(1+exp(-x))
+ *   c_t   = rn16(f*c_{t-1} + i*g)                 h_t = rn16(o * tanh(c_t as stored))
+ *   r_t   = rn16(h_t . Wp^T)
+ * Wg is [4H, I+P] with GATE-INTERLEAVED rows: row 4j+q is gate q of cell j (q: 0 input,
+ * 1 forget, 2 candidate, 3 output); bias16, acts, dG and dWg use the same order.  The gate
+ * arithmetic runs in the epilogue of the gate product: the pre-activations never reach memory.
+ * Backward (scaled gradients, section 3.2), t = T-1 .. 0:
+ *   drtot_t = rn16(dr_ext_t + recurrent part of dxr_{t+1})      dh_t = rn16(drtot_t . Wp)
+ *   dc  = (dh*o)*(1 - tanh(c_t)^2) + dc_next ;  dG_t = rn16 of
+ *         i: (dc*g)*(i*(1-i))  f: (dc*c_{t-1})*(f*(1-f))  g: (dc*i)*(1-g*g)  o: (dh*tanh(c_t))*(o*(1-o))
+ *   dc_prev = rn16(dc*f) ;  dxr_t = rn16(dG_t . Wg)
+ * and once, over all T*B rows (the sum over time is accumulated in FP32 inside one product):
+ *   dWg = rn16(dG^T . xr)   dWp = rn16(drtot^T . h)   dbias = rn16(FP32 column sums of dG)
+ * Every FP32 operation is rounded separately in the order written.
+ *
+ * All pointers are device memory owned by the caller; nothing is allocated.  Row-major, dense
+ * (pitch = row length).  I, H and P must be multiples of 8 (MPT_ERR_SHAPE otherwise); the
+ * tensor-core kernels are used when the product shapes allow, CUDA-core kernels otherwise. */
+typedef struct mpt_lstm_desc {
+    int32_t T, B;       /* time steps, rows per step (batch) */
+    int32_t I, H, P;    /* input width, cells, projection width */
+} mpt_lstm_desc;
+
+typedef struct mpt_lstm_tensors {
+    /* parameters (FP16 working copies) */
+    const uint16_t *Wg16;    /* [4H, I+P] */
+    const uint16_t *bias16;  /* [4H] */
+    const uint16_t *Wp16;    /* [P, H] */
+    /* forward: caller fills xr[t][:, :I] = x_t (t < T), xr[0][:, I:] = r_{-1}, c[0] = c_{-1};
+     * the forward pass writes xr[t+1][:, I:] = r_t, c[t+1], h[t], acts[t] */
+    uint16_t *xr;            /* [T+1, B, I+P] */
+    uint16_t *c;             /* [T+1, B, H] */
+    uint16_t *h;             /* [T, B, H] */
+    uint16_t *acts;          /* [T, B, 4H] gate activations kept for the backward pass */
+    /* backward */
+    const uint16_t *dr_ext;  /* [T, B, P] scaled gradient wrt r_t from the consumer of the layer */
+    uint16_t *dxr;           /* [T, B, I+P]: [:, :I] gradient wrt x_t, [:, I:] recurrent gradient wrt r_{t-1} */
+    uint16_t *drtot;         /* [T, B, P] */
+    uint16_t *dG;            /* [T, B, 4H] */
+    uint16_t *dh;            /* [B, H] scratch */
+    uint16_t *dc;            /* [2, B, H] scratch */
+    uint16_t *dWg16;         /* [4H, I+P] */
+    uint16_t *dWp16;         /* [P, H] */
+    uint16_t *dbias16;       /* [4H] */
+    float *bias_parts;       /* [8, 4H] FP32 scratch of the bias-gradient reduction */
+    uint32_t *nonfinite_flag; /* one word, OR-ed with 1 when a weight or bias gradient is inf/NaN (section 3.2);
+                                the caller zeroes it before mpt_lstm_backward */
+    uint32_t *status_dev;    /* MPT status block of >= 16 words (first device-side error at word 3) or null */
+} mpt_lstm_tensors;
+
+/* Forward over all T steps: 2T launches on the stream (gate product with fused gate epilogue,
+ * projection product).  Reads Wg16, bias16, Wp16, xr, c[0]; writes h, acts, c[1..T], xr[1..T][:, I:]. */
+int mpt_lstm_forward(const mpt_lstm_desc *desc, const mpt_lstm_tensors *t, void *cuda_stream);
+
+/* Backward over all T steps, then the weight and bias gradients.  Needs the tensors the forward
+ * pass wrote.  Writes dxr, drtot, dG, dWg16, dWp16, dbias16. */
+int mpt_lstm_backward(const mpt_lstm_desc *desc, const mpt_lstm_tensors *t, void *cuda_stream);
+
+/* The pieces on their own (same arithmetic).  mpt_lstm_cell_forward: one time step's gate product
+ * with the fused gate epilogue; xr [B, K] pitch ldxr, Wg [4H, K] pitch ldw, acts [B, 4H] pitch
+ * ldacts, c_prev/c_out/h_out [B, H] with their pitches.  mpt_lstm_cell_backward: dc_next may be
+ * null (last step).  mpt_bias_grad: parts = FP32 scratch [8, cols].  mpt_add_f16: out = rn16(a+b). */
+int mpt_lstm_cell_forward(int B, int H, int K, const uint16_t *xr, int ldxr, const uint16_t *Wg, int ldw,
+                          const uint16_t *bias16, const uint16_t *c_prev, int ldcp, uint16_t *acts, int ldacts,
+                          uint16_t *c_out, int ldco, uint16_t *h_out, int ldh, unsigned flags, uint32_t *status_dev,
+                          void *cuda_stream);
+int mpt_lstm_cell_backward(int B, int H, const uint16_t *dh, int lddh, const uint16_t *dc_next, int lddc,
+                           const uint16_t *acts, int ldacts, const uint16_t *c_prev, int ldcp, const uint16_t *c16, int ldc,
+                           uint16_t *dG, int lddg, uint16_t *dc_prev, int lddcp, void *cuda_stream);
+int mpt_bias_grad(const uint16_t *dG, size_t rows, int cols, int ld, float *parts, uint16_t *db16,
+                  uint32_t *nonfinite_flag, void *cuda_stream);
+int mpt_add_f16(const uint16_t *a, int lda, const uint16_t *b, int ldb, uint16_t *out, int ldo, int rows, int cols,
+                void *cuda_stream);
+
 /* Softmax cross-entropy forward and scaled backward (sections 3.2, 3.3), arithmetic
  * as in mpt_backward_scaled.  z_dev/dz_dev: FP16 [B, C] with pitches ldz/lddz
  * (the two must not overlap).  row_loss_dev: float [B] scratch; loss_dev: one float,

@@ -31,7 +31,9 @@ EXPORTS = ["mpt_workspace_bytes", "mpt_create", "mpt_workspace_bytes_opt", "mpt_
            "mpt_get_tensor", "mpt_set_grad", "mpt_set_momentum", "mpt_launch_count", "mpt_profile",
            "mpt_profile_read", "mpt_last_error",
            "mpt_destroy", "mpt_gemm_f16", "mpt_gemm_f16_ws", "mpt_gemm_workspace_bytes", "mpt_recast", "mpt_grad_nonfinite", "mpt_update_flat",
-           "mpt_softmax_ce", "mpt_softmax_ce_static", "mpt_version"]
+           "mpt_softmax_ce", "mpt_softmax_ce_static", "mpt_version",
+           "mpt_lstm_forward", "mpt_lstm_backward", "mpt_lstm_cell_forward", "mpt_lstm_cell_backward", "mpt_bias_grad",
+           "mpt_add_f16"]
 
 
 class MptError(RuntimeError):
@@ -48,6 +50,20 @@ class Optimizer(C.Structure):
     """mpt_optimizer: kind (OPT_*), lr, momentum (or Adam beta1), beta2, eps, weight_decay, clip_norm."""
     _fields_ = [("kind", C.c_int32), ("lr", C.c_float), ("momentum", C.c_float), ("beta2", C.c_float),
                 ("eps", C.c_float), ("weight_decay", C.c_float), ("clip_norm", C.c_float)]
+
+
+class LstmDesc(C.Structure):
+    """mpt_lstm_desc: T steps, B rows per step, input width I, H cells, projection width P."""
+    _fields_ = [("T", C.c_int32), ("B", C.c_int32), ("I", C.c_int32), ("H", C.c_int32), ("P", C.c_int32)]
+
+
+_LSTM_FIELDS = ["Wg16", "bias16", "Wp16", "xr", "c", "h", "acts", "dr_ext", "dxr", "drtot", "dG", "dh", "dc", "dWg16", "dWp16",
+                "dbias16", "bias_parts", "nonfinite_flag", "status_dev"]
+
+
+class LstmTensors(C.Structure):
+    """mpt_lstm_tensors: device pointers of every tensor of the layer (see include/mpt.h)."""
+    _fields_ = [(name, C.c_void_p) for name in _LSTM_FIELDS]
 
 
 _lib = None
@@ -101,6 +117,12 @@ def lib() -> C.CDLL:
     L.mpt_update_flat.argtypes = [vp, vp, vp, vp, sz, f32, f32, f32, i32, i32, vp, vp]
     L.mpt_softmax_ce.argtypes = [vp, i32, vp, i32, i32, f32, vp, i32, vp, vp, vp, vp]
     L.mpt_softmax_ce_static.argtypes = [vp, i32, vp, i32, i32, f32, vp, i32, vp, vp, vp]
+    L.mpt_lstm_forward.argtypes = [C.POINTER(LstmDesc), C.POINTER(LstmTensors), vp]
+    L.mpt_lstm_backward.argtypes = [C.POINTER(LstmDesc), C.POINTER(LstmTensors), vp]
+    L.mpt_lstm_cell_forward.argtypes = [i32, i32, i32, vp, i32, vp, i32, vp, vp, i32, vp, i32, vp, i32, vp, i32, u32, vp, vp]
+    L.mpt_lstm_cell_backward.argtypes = [i32, i32, vp, i32, vp, i32, vp, i32, vp, i32, vp, i32, vp, i32, vp, i32, vp]
+    L.mpt_bias_grad.argtypes = [vp, sz, i32, i32, vp, vp, vp, vp]
+    L.mpt_add_f16.argtypes = [vp, i32, vp, i32, vp, i32, i32, i32, vp]
     L.mpt_version.restype = C.c_char_p
     L.mpt_version.argtypes = []
     _lib = L
@@ -361,3 +383,56 @@ def mpt_softmax_ce_static(z, ldz, labels, B, Cn, S, dz, lddz, loss, bad_labels=N
 
 def mpt_version() -> str:
     return lib().mpt_version().decode()
+
+
+# ------------------------------------------------------------------ LSTM layer
+
+def mpt_lstm_cell_forward(B, H, K, xr, ldxr, Wg, ldw, bias16, c_prev, ldcp, acts, ldacts, c_out, ldco, h_out, ldh, flags=0,
+                          status=None, stream=None):
+    _check(lib().mpt_lstm_cell_forward(B, H, K, _dptr(xr), ldxr, _dptr(Wg), ldw, _dptr(bias16), _dptr(c_prev), ldcp,
+                                       _dptr(acts), ldacts, _dptr(c_out), ldco, _dptr(h_out), ldh, flags, _dptr(status),
+                                       _stream_ptr(stream)))
+
+
+def mpt_lstm_cell_backward(B, H, dh, lddh, dc_next, lddc, acts, ldacts, c_prev, ldcp, c16, ldc, dG, lddg, dc_prev, lddcp,
+                           stream=None):
+    _check(lib().mpt_lstm_cell_backward(B, H, _dptr(dh), lddh, _dptr(dc_next), lddc, _dptr(acts), ldacts, _dptr(c_prev), ldcp,
+                                        _dptr(c16), ldc, _dptr(dG), lddg, _dptr(dc_prev), lddcp, _stream_ptr(stream)))
+
+
+def mpt_bias_grad(dG, rows, cols, ld, parts, db16, nonfinite_flag=None, stream=None):
+    _check(lib().mpt_bias_grad(_dptr(dG), rows, cols, ld, _dptr(parts), _dptr(db16), _dptr(nonfinite_flag), _stream_ptr(stream)))
+
+
+def mpt_add_f16(a, lda, b, ldb, out, ldo, rows, cols, stream=None):
+    _check(lib().mpt_add_f16(_dptr(a), lda, _dptr(b), ldb, _dptr(out), ldo, rows, cols, _stream_ptr(stream)))
+
+
+class LstmLayer:
+    """Device buffers of one LSTM layer with projection plus the two calls that run it.  Holds
+    torch tensors (int16 views of FP16 bits) only to own the memory; all arithmetic happens in
+    mpt_lstm_forward / mpt_lstm_backward."""
+
+    def __init__(self, T, B, I, H, P):
+        import torch
+        self.desc = LstmDesc(T, B, I, H, P)
+        z16 = lambda *shape: torch.zeros(shape, dtype=torch.int16, device="cuda")  # noqa: E731
+        self.Wg16, self.bias16, self.Wp16 = z16(4 * H, I + P), z16(4 * H), z16(P, H)
+        self.xr, self.c, self.h, self.acts = z16(T + 1, B, I + P), z16(T + 1, B, H), z16(T, B, H), z16(T, B, 4 * H)
+        self.dr_ext, self.dxr, self.drtot, self.dG = z16(T, B, P), z16(T, B, I + P), z16(T, B, P), z16(T, B, 4 * H)
+        self.dh, self.dc = z16(B, H), z16(2, B, H)
+        self.dWg16, self.dWp16, self.dbias16 = z16(4 * H, I + P), z16(P, H), z16(4 * H)
+        self.bias_parts = torch.zeros((8, 4 * H), dtype=torch.float32, device="cuda")
+        self.status = torch.zeros(16, dtype=torch.int32, device="cuda")
+        self.nonfinite_flag = torch.zeros(1, dtype=torch.int32, device="cuda")
+        self.tensors = LstmTensors(*[getattr(self, n if n != "status_dev" else "status").data_ptr() for n in _LSTM_FIELDS])
+
+    def forward(self, stream=None):
+        _check(lib().mpt_lstm_forward(C.byref(self.desc), C.byref(self.tensors), _stream_ptr(stream)))
+
+    def backward(self, stream=None):
+        self.nonfinite_flag.zero_()
+        _check(lib().mpt_lstm_backward(C.byref(self.desc), C.byref(self.tensors), _stream_ptr(stream)))
+
+    def device_error(self) -> int:
+        return int(self.status[3].item())

@@ -64,6 +64,7 @@ struct TcParams {
     int split_k;
     float *partial;
     int ldp;
+    LstmEpi lstm;   // read only by the LSTM instantiations of the kernel
 };
 
 __device__ __forceinline__ void tile_coords(const TcParams &p, int tile, int &mb, int &nb)
@@ -85,7 +86,7 @@ __device__ __forceinline__ void report(const TcParams &p, volatile uint32_t *abo
     if (p.status) atomicCAS(p.status, 0u, code | ((uint32_t)blockIdx.x << 8));
 }
 
-template <bool A_MN, bool B_MN, int BLOCK_N>
+template <bool A_MN, bool B_MN, int BLOCK_N, bool LSTM = false>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcParams p)
 {
@@ -257,7 +258,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                                                  __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
                     }
                 } else if (row_ok && col0 < p.N) {
-                    epilogue_store32(r, crow, mrow, col0, p.N, p.relu != 0, bad);
+                    if constexpr (LSTM) epilogue_lstm32(r, crow, row, col0, p.lstm);
+                    else epilogue_store32(r, crow, mrow, col0, p.N, p.relu != 0, bad);
                 }
             }
             tc_fence_before();
@@ -359,13 +361,13 @@ bool tc_gemm_supported(int op, int M, int N, int K, const void *A, int lda, cons
     return true;
 }
 
-template <bool A_MN, bool B_MN, int BN>
+template <bool A_MN, bool B_MN, int BN, bool LSTM = false>
 static cudaError_t launch_variant(const CUtensorMap &ta, const CUtensorMap &tb, const TcParams &p, int grid,
                                   cudaStream_t st)
 {
     static bool configured[kMaxDevices] = {};
     constexpr int SMEM_BYTES = TileCfg<BN>::SMEM_BYTES;
-    auto kern = k_gemm_tc<A_MN, B_MN, BN>;
+    auto kern = k_gemm_tc<A_MN, B_MN, BN, LSTM>;
     const int dev = current_device_slot();
     if (dev < 0) return cudaErrorInvalidDevice;
     if (!configured[dev]) {
@@ -396,7 +398,8 @@ static cudaError_t launch_bn(int op, int M, int N, int K, const uint16_t *A, int
     int units = p.tiles_m * p.tiles_n * p.split_k;
     int grid = units < 148 ? units : 148;
     cudaError_t e;
-    if (op == MPT_OP_FWD) e = launch_variant<false, false, BN>(ta, tb, p, grid, st);
+    if (op == MPT_OP_FWD && p.lstm.c_out) e = launch_variant<false, false, BN, true>(ta, tb, p, grid, st);
+    else if (op == MPT_OP_FWD) e = launch_variant<false, false, BN>(ta, tb, p, grid, st);
     else if (op == MPT_OP_DGRAD) e = launch_variant<false, true, BN>(ta, tb, p, grid, st);
     else e = launch_variant<true, true, BN>(ta, tb, p, grid, st);
     if (e != cudaSuccess || p.split_k == 1) return e;
@@ -444,9 +447,15 @@ void tc_gemm_plan(int M, int N, int K, size_t ws_bytes, int *bn_out, int *split_
 
 cudaError_t launch_gemm_tc(int op, int M, int N, int K, const uint16_t *A, int lda, const uint16_t *B, int ldb,
                            uint16_t *C, int ldc, bool relu, const uint16_t *mask, int ldmask, uint32_t *nonfinite_flag,
-                           uint32_t *status, cudaStream_t st, float *splitk_ws, size_t splitk_ws_bytes)
+                           uint32_t *status, cudaStream_t st, float *splitk_ws, size_t splitk_ws_bytes, const LstmEpi *lstm)
 {
     TcParams p;
+    p.lstm = LstmEpi{};
+    if (lstm) {   // gate epilogue: forward products only, never split (the epilogue needs the whole sum)
+        if (op != MPT_OP_FWD || (N & 31) != 0) return cudaErrorInvalidValue;
+        p.lstm = *lstm;
+        splitk_ws = nullptr;
+    }
     p.M = M; p.N = N; p.K = K;
     p.C = C; p.ldc = ldc;
     p.mask = mask; p.ldmask = ldmask;

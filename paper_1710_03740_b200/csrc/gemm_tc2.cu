@@ -61,6 +61,7 @@ struct Params {
     uint32_t *status;
     int tiles_m, tiles_n, group_m;   // pair tiles (256 rows x 256 columns)
     int full_units, num_units;       // units [0, full_units) are whole tiles, the rest are half tiles
+    LstmEpi lstm;                    // read only by the LSTM instantiation of the kernel
 };
 
 struct Unit {
@@ -102,7 +103,7 @@ __device__ __forceinline__ void report(const Params &p, volatile uint32_t *abort
     if (p.status) atomicCAS(p.status, 0u, code | 0x80u | ((uint32_t)blockIdx.x << 8));
 }
 
-template <bool A_MN, bool B_MN>
+template <bool A_MN, bool B_MN, bool LSTM = false>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
            const __grid_constant__ CUtensorMap tmBh, const Params p)
@@ -260,7 +261,10 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
                 tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * TILE_N + c * 32), r);
                 tc_wait_ld();
                 const int col0 = w.nb * TILE_N + w.n_off + c * 32;
-                if (row_ok && col0 < p.N) epilogue_store32(r, crow, mrow, col0, p.N, p.relu != 0, bad);
+                if (row_ok && col0 < p.N) {
+                    if constexpr (LSTM) epilogue_lstm32(r, crow, row, col0, p.lstm);
+                    else epilogue_store32(r, crow, mrow, col0, p.N, p.relu != 0, bad);
+                }
             }
             tc_fence_before();
             __syncwarp();
@@ -280,12 +284,12 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
     }
 }
 
-template <bool A_MN, bool B_MN>
+template <bool A_MN, bool B_MN, bool LSTM = false>
 static cudaError_t launch_variant(const CUtensorMap &ta, const CUtensorMap &tb, const CUtensorMap &tbh, Params p,
                                   cudaStream_t st)
 {
     static int max_pairs_dev[kMaxDevices] = {};     // 0 = this device not configured yet
-    auto kern = k_gemm_tc2<A_MN, B_MN>;
+    auto kern = k_gemm_tc2<A_MN, B_MN, LSTM>;
     const int dev = current_device_slot();
     if (dev < 0) return cudaErrorInvalidDevice;
     cudaLaunchConfig_t cfg = {};
@@ -342,7 +346,7 @@ bool tc2_gemm_preferred(int M, int N, int K)
 
 cudaError_t launch_gemm_tc2(int op, int M, int N, int K, const uint16_t *A, int lda, const uint16_t *B, int ldb,
                             uint16_t *C, int ldc, bool relu, const uint16_t *mask, int ldmask, uint32_t *nonfinite_flag,
-                            uint32_t *status, cudaStream_t st)
+                            uint32_t *status, cudaStream_t st, const LstmEpi *lstm)
 {
     using namespace pair;
     CUtensorMap ta, tb, tbh;
@@ -369,6 +373,12 @@ cudaError_t launch_gemm_tc2(int op, int M, int N, int K, const uint16_t *A, int 
     p.tiles_n = (N + TILE_N - 1) / TILE_N;
     p.group_m = 8;
     p.full_units = p.num_units = 0;
+    p.lstm = LstmEpi{};
+    if (lstm) {
+        if (op != MPT_OP_FWD || (N & 31) != 0) return cudaErrorInvalidValue;
+        p.lstm = *lstm;
+        return launch_variant<false, false, true>(ta, tb, tbh, p, st);
+    }
     if (op == MPT_OP_FWD) return launch_variant<false, false>(ta, tb, tbh, p, st);
     if (op == MPT_OP_DGRAD) return launch_variant<false, true>(ta, tb, tbh, p, st);
     return launch_variant<true, true>(ta, tb, tbh, p, st);

@@ -1,0 +1,227 @@
+// LSTM layer pieces outside the tensor-core products (sections 3.3, 4.6 of the paper): the
+// backward of the gate arithmetic, the FP32 bias-gradient reduction, the FP16 add of two
+// gradient contributions, and a plain-CUDA-core forward cell for shapes the tensor-core
+// kernels do not take.  All of them are memory-bound streaming kernels on FP16 storage with
+// FP32 arithmetic; every FP32 operation is rounded separately, in the order the header documents.
+#include "mpt_common.cuh"
+#include "tc_ptx.cuh"
+
+namespace mpt {
+
+namespace {
+
+__device__ __forceinline__ float h2f_u(uint32_t h) { return __half2float(__ushort_as_half((unsigned short)h)); }
+__device__ __forceinline__ uint32_t f2h_u(float x) { return (uint32_t)__half_as_ushort(__float2half_rn(x)); }
+
+// ------------------------------------------------------------ forward cell, CUDA cores
+
+// One thread per (row, cell): four dot products in ascending k with FP32 accumulation, then the
+// same gate arithmetic as the fused tensor-core epilogue.  For small or unaligned shapes only.
+__global__ void __launch_bounds__(256) k_lstm_cell_simt(int B, int H, int K, const uint16_t *__restrict__ XR, int ldxr,
+                                                        const uint16_t *__restrict__ Wg, int ldw,
+                                                        uint16_t *__restrict__ acts, int ldacts, LstmEpi e)
+{
+    const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= (size_t)B * H) return;
+    const int b = (int)(idx / H), j = (int)(idx % H);
+    const uint16_t *x = XR + (size_t)b * ldxr;
+    float pre[4];
+#pragma unroll
+    for (int q = 0; q < 4; q++) {
+        const uint16_t *w = Wg + (size_t)(4 * j + q) * ldw;
+        float acc = 0.0f;
+        for (int k = 0; k < K; k++) acc = __fadd_rn(acc, __fmul_rn(h2f_u(x[k]), h2f_u(w[k])));
+        pre[q] = __fadd_rn(acc, h2f_u(e.bias[4 * j + q]));
+    }
+    uint32_t act[4], c16, h16;
+    lstm_cell_math(pre, h2f_u(e.c_prev[(size_t)b * e.ldcp + j]), act, c16, h16);
+#pragma unroll
+    for (int q = 0; q < 4; q++) acts[(size_t)b * ldacts + 4 * j + q] = (uint16_t)act[q];
+    e.c_out[(size_t)b * e.ldco + j] = (uint16_t)c16;
+    e.h_out[(size_t)b * e.ldh + j] = (uint16_t)h16;
+}
+
+// ------------------------------------------------------------ backward of the gate arithmetic
+
+struct CellGrad {
+    uint32_t dg[4];   // FP16 bits of the gradients wrt the four pre-activations
+    uint32_t dcp;     // FP16 bits of the gradient wrt c_{t-1}
+};
+
+__device__ __forceinline__ CellGrad cell_bwd(float gi, float gf, float gg, float go, float cp, float c, float dh, float dcn)
+{
+    const float tc = tanhf(c);
+    const float dc = __fadd_rn(__fmul_rn(__fmul_rn(dh, go), __fsub_rn(1.0f, __fmul_rn(tc, tc))), dcn);
+    const float dpo = __fmul_rn(__fmul_rn(dh, tc), __fmul_rn(go, __fsub_rn(1.0f, go)));
+    const float dpi = __fmul_rn(__fmul_rn(dc, gg), __fmul_rn(gi, __fsub_rn(1.0f, gi)));
+    const float dpf = __fmul_rn(__fmul_rn(dc, cp), __fmul_rn(gf, __fsub_rn(1.0f, gf)));
+    const float dpg = __fmul_rn(__fmul_rn(dc, gi), __fsub_rn(1.0f, __fmul_rn(gg, gg)));
+    CellGrad r;
+    r.dg[0] = f2h_u(dpi); r.dg[1] = f2h_u(dpf); r.dg[2] = f2h_u(dpg); r.dg[3] = f2h_u(dpo);
+    r.dcp = f2h_u(__fmul_rn(dc, gf));
+    return r;
+}
+
+// Two cells per thread: one 128-bit load of the activations, 32-bit loads of the per-cell values.
+// H is even and all pitches are even (checked by the launcher), so the 32-bit accesses are aligned.
+__global__ void __launch_bounds__(256) k_lstm_cell_bwd(int B, int H2, const uint16_t *__restrict__ dh, int lddh,
+                                                       const uint16_t *__restrict__ dc_next, int lddc,
+                                                       const uint16_t *__restrict__ acts, int ldacts,
+                                                       const uint16_t *__restrict__ c_prev, int ldcp,
+                                                       const uint16_t *__restrict__ c16, int ldc, uint16_t *__restrict__ dG,
+                                                       int lddg, uint16_t *__restrict__ dc_prev, int lddcp)
+{
+    const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= (size_t)B * H2) return;
+    const int b = (int)(idx / H2), j = 2 * (int)(idx % H2);
+    const uint4 av = *(const uint4 *)(acts + (size_t)b * ldacts + 4 * j);
+    const uint32_t cpw = *(const uint32_t *)(c_prev + (size_t)b * ldcp + j);
+    const uint32_t cw = *(const uint32_t *)(c16 + (size_t)b * ldc + j);
+    const uint32_t dhw = *(const uint32_t *)(dh + (size_t)b * lddh + j);
+    const uint32_t dcw = dc_next ? *(const uint32_t *)(dc_next + (size_t)b * lddc + j) : 0u;
+    const CellGrad g0 = cell_bwd(h2f_u(av.x & 0xFFFFu), h2f_u(av.x >> 16), h2f_u(av.y & 0xFFFFu), h2f_u(av.y >> 16),
+                                 h2f_u(cpw & 0xFFFFu), h2f_u(cw & 0xFFFFu), h2f_u(dhw & 0xFFFFu), h2f_u(dcw & 0xFFFFu));
+    const CellGrad g1 = cell_bwd(h2f_u(av.z & 0xFFFFu), h2f_u(av.z >> 16), h2f_u(av.w & 0xFFFFu), h2f_u(av.w >> 16),
+                                 h2f_u(cpw >> 16), h2f_u(cw >> 16), h2f_u(dhw >> 16), h2f_u(dcw >> 16));
+    *(uint4 *)(dG + (size_t)b * lddg + 4 * j) = make_uint4(g0.dg[0] | (g0.dg[1] << 16), g0.dg[2] | (g0.dg[3] << 16),
+                                                           g1.dg[0] | (g1.dg[1] << 16), g1.dg[2] | (g1.dg[3] << 16));
+    *(uint32_t *)(dc_prev + (size_t)b * lddcp + j) = g0.dcp | (g1.dcp << 16);
+}
+
+// scalar form for odd H or unaligned buffers
+__global__ void __launch_bounds__(256) k_lstm_cell_bwd_scalar(int B, int H, const uint16_t *__restrict__ dh, int lddh,
+                                                              const uint16_t *__restrict__ dc_next, int lddc,
+                                                              const uint16_t *__restrict__ acts, int ldacts,
+                                                              const uint16_t *__restrict__ c_prev, int ldcp,
+                                                              const uint16_t *__restrict__ c16, int ldc,
+                                                              uint16_t *__restrict__ dG, int lddg,
+                                                              uint16_t *__restrict__ dc_prev, int lddcp)
+{
+    const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= (size_t)B * H) return;
+    const int b = (int)(idx / H), j = (int)(idx % H);
+    const uint16_t *a = acts + (size_t)b * ldacts + 4 * j;
+    const CellGrad g = cell_bwd(h2f_u(a[0]), h2f_u(a[1]), h2f_u(a[2]), h2f_u(a[3]), h2f_u(c_prev[(size_t)b * ldcp + j]),
+                                h2f_u(c16[(size_t)b * ldc + j]), h2f_u(dh[(size_t)b * lddh + j]),
+                                dc_next ? h2f_u(dc_next[(size_t)b * lddc + j]) : 0.0f);
+    uint16_t *d = dG + (size_t)b * lddg + 4 * j;
+    d[0] = (uint16_t)g.dg[0]; d[1] = (uint16_t)g.dg[1]; d[2] = (uint16_t)g.dg[2]; d[3] = (uint16_t)g.dg[3];
+    dc_prev[(size_t)b * lddcp + j] = (uint16_t)g.dcp;
+}
+
+// ------------------------------------------------------------ bias gradient
+
+// Column sums in FP32 (section 3.3: reductions in FP32).  Fixed partition: the rows are cut into
+// kBiasRowParts contiguous ranges (blockIdx.y); inside a CTA warp w takes rows w, w+8, ... of
+// its range in ascending order, lane l the 8 columns 8l..8l+7 of the CTA's 256-column block; the
+// eight warps are combined in ascending order through shared memory into parts[range][column].
+__global__ void __launch_bounds__(256) k_bias_grad_partial(const uint16_t *__restrict__ dG, size_t rows, int cols, int ld,
+                                                           float *__restrict__ parts, bool vec)
+{
+    __shared__ float sh[8][256];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int col = blockIdx.x * 256 + lane * 8;
+    const size_t per = (rows + gridDim.y - 1) / gridDim.y;
+    const size_t r0 = (size_t)blockIdx.y * per;
+    const size_t r1 = r0 + per < rows ? r0 + per : rows;
+    float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    if (vec && col + 8 <= cols) {
+        for (size_t r = r0 + warp; r < r1; r += 8) {
+            const uint4 v = __ldcs((const uint4 *)(dG + r * (size_t)ld + col));
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int e = 0; e < 8; e++)
+                acc[e] = __fadd_rn(acc[e], h2f_u((e & 1) ? (w[e >> 1] >> 16) : (w[e >> 1] & 0xFFFFu)));
+        }
+    } else {
+        for (size_t r = r0 + warp; r < r1; r += 8)
+            for (int e = 0; e < 8 && col + e < cols; e++) acc[e] = __fadd_rn(acc[e], h2f_u(dG[r * (size_t)ld + col + e]));
+    }
+#pragma unroll
+    for (int e = 0; e < 8; e++) sh[warp][lane * 8 + e] = acc[e];
+    __syncthreads();
+    const int c = blockIdx.x * 256 + threadIdx.x;
+    if (c < cols) {
+        float s = 0.0f;
+#pragma unroll
+        for (int w = 0; w < 8; w++) s = __fadd_rn(s, sh[w][threadIdx.x]);
+        parts[(size_t)blockIdx.y * cols + c] = s;
+    }
+}
+
+__global__ void __launch_bounds__(256) k_bias_grad_final(const float *__restrict__ parts, int nparts, int cols,
+                                                         uint16_t *__restrict__ db16, uint32_t *nonfinite_flag)
+{
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    bool bad = false;
+    if (c < cols) {
+        float s = 0.0f;
+        for (int p = 0; p < nparts; p++) s = __fadd_rn(s, parts[(size_t)p * cols + c]);
+        const uint32_t h = f2h_u(s);
+        bad = half_bits_nonfinite(h);
+        db16[c] = (uint16_t)h;
+    }
+    if (nonfinite_flag && __any_sync(0xFFFFFFFFu, bad) && (threadIdx.x & 31) == 0) atomicOr(nonfinite_flag, 1u);
+}
+
+// ------------------------------------------------------------ FP16 add
+
+__global__ void __launch_bounds__(256) k_add_f16(const uint16_t *__restrict__ a, int lda, const uint16_t *__restrict__ b,
+                                                 int ldb, uint16_t *__restrict__ out, int ldo, int rows, int cols)
+{
+    const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= (size_t)rows * cols) return;
+    const int r = (int)(idx / cols), c = (int)(idx % cols);
+    out[(size_t)r * ldo + c] = (uint16_t)f2h_u(__fadd_rn(h2f_u(a[(size_t)r * lda + c]), h2f_u(b[(size_t)r * ldb + c])));
+}
+
+unsigned blocks_for(size_t n) { return (unsigned)((n + 255) / 256); }
+
+}  // namespace
+
+cudaError_t launch_lstm_cell_simt(int B, int H, int K, const uint16_t *XR, int ldxr, const uint16_t *Wg, int ldw,
+                                  uint16_t *acts, int ldacts, const LstmEpi &e, cudaStream_t st)
+{
+    if (B <= 0 || H <= 0) return cudaSuccess;
+    k_lstm_cell_simt<<<blocks_for((size_t)B * H), 256, 0, st>>>(B, H, K, XR, ldxr, Wg, ldw, acts, ldacts, e);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_lstm_cell_bwd(int B, int H, const uint16_t *dh, int lddh, const uint16_t *dc_next, int lddc,
+                                 const uint16_t *acts, int ldacts, const uint16_t *c_prev, int ldcp, const uint16_t *c16,
+                                 int ldc, uint16_t *dG, int lddg, uint16_t *dc_prev, int lddcp, cudaStream_t st)
+{
+    if (B <= 0 || H <= 0) return cudaSuccess;
+    const uintptr_t bits = (uintptr_t)acts | (uintptr_t)dG;
+    const uintptr_t bits4 = (uintptr_t)dh | (uintptr_t)dc_next | (uintptr_t)c_prev | (uintptr_t)c16 | (uintptr_t)dc_prev;
+    const bool vec = (H % 2) == 0 && (bits & 15) == 0 && (bits4 & 3) == 0 && (ldacts % 8) == 0 && (lddg % 8) == 0 &&
+                     ((lddh | lddc | ldcp | ldc | lddcp) % 2) == 0;
+    if (vec)
+        k_lstm_cell_bwd<<<blocks_for((size_t)B * (H / 2)), 256, 0, st>>>(B, H / 2, dh, lddh, dc_next, lddc, acts, ldacts, c_prev,
+                                                                         ldcp, c16, ldc, dG, lddg, dc_prev, lddcp);
+    else
+        k_lstm_cell_bwd_scalar<<<blocks_for((size_t)B * H), 256, 0, st>>>(B, H, dh, lddh, dc_next, lddc, acts, ldacts, c_prev,
+                                                                          ldcp, c16, ldc, dG, lddg, dc_prev, lddcp);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_bias_grad(const uint16_t *dG, size_t rows, int cols, int ld, float *parts, uint16_t *db16,
+                             uint32_t *nonfinite_flag, cudaStream_t st)
+{
+    if (cols <= 0) return cudaSuccess;
+    const bool vec = ((uintptr_t)dG & 15) == 0 && (ld % 8) == 0;
+    dim3 grid((unsigned)((cols + 255) / 256), (unsigned)kBiasRowParts);
+    k_bias_grad_partial<<<grid, 256, 0, st>>>(dG, rows, cols, ld, parts, vec);   // unaligned rows: element loads
+    k_bias_grad_final<<<blocks_for((size_t)cols), 256, 0, st>>>(parts, kBiasRowParts, cols, db16, nonfinite_flag);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_add_f16(const uint16_t *a, int lda, const uint16_t *b, int ldb, uint16_t *out, int ldo, int rows,
+                           int cols, cudaStream_t st)
+{
+    if (rows <= 0 || cols <= 0) return cudaSuccess;
+    k_add_f16<<<blocks_for((size_t)rows * cols), 256, 0, st>>>(a, lda, b, ldb, out, ldo, rows, cols);
+    return cudaGetLastError();
+}
+
+}  // namespace mpt

@@ -387,6 +387,40 @@ int finish_step(mpt_ctx *c, const uint32_t (&st)[ST_WORDS], int *overflow_host)
 
 }  // namespace
 
+namespace mpt {
+
+// Shape checks and kernel choice shared by the stateless product entry points and the LSTM layer:
+// CTA-pair kernel for large outputs, single-CTA kernel (with optional split-K scratch) for the
+// rest of what the tensor-core path takes, CUDA-core kernel otherwise.  lstm != null: forward
+// product with the fused gate epilogue (tensor-core kernels only; the caller checks that first).
+int dispatch_gemm(int op, int M, int N, int K, const uint16_t *A, int lda, const uint16_t *B, int ldb, uint16_t *C, int ldc,
+                  unsigned flags, const uint16_t *mask, int ldmask, uint32_t *nonfinite_flag, uint32_t *status_dev,
+                  void *splitk_ws_dev, size_t splitk_ws_bytes, cudaStream_t st, const LstmEpi *lstm)
+{
+    if (!A || !B || !C) return MPT_ERR_INVALID_ARG;
+    if (op != MPT_OP_FWD && op != MPT_OP_DGRAD && op != MPT_OP_WGRAD) return MPT_ERR_INVALID_ARG;
+    if (M < 0 || N < 0 || K < 0) return MPT_ERR_SHAPE;
+    if (M == 0 || N == 0) return MPT_OK;
+    const int a_cols = op == MPT_OP_WGRAD ? M : K, b_cols = op == MPT_OP_FWD ? K : N;
+    if (lda < a_cols || ldb < b_cols || ldc < N || (mask && ldmask < N)) return MPT_ERR_SHAPE;
+    const bool relu = (flags & MPT_GEMM_RELU) != 0;
+    bool tc_ok = K > 0 && tc_gemm_supported(op, M, N, K, A, lda, B, ldb, C, ldc, mask, ldmask);
+    if (((flags & (MPT_GEMM_FORCE_TC | MPT_GEMM_FORCE_PAIR)) || lstm) && !tc_ok) return MPT_ERR_SHAPE;
+    cudaError_t e;
+    if (tc_ok && !(flags & MPT_GEMM_FORCE_SIMT)) {
+        const bool pair = (flags & MPT_GEMM_FORCE_PAIR) || (!(flags & MPT_GEMM_FORCE_TC) && tc2_gemm_preferred(M, N, K));
+        if (pair)
+            e = launch_gemm_tc2(op, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite_flag, status_dev, st, lstm);
+        else
+            e = launch_gemm_tc(op, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite_flag, status_dev, st,
+                               (float *)splitk_ws_dev, splitk_ws_bytes, lstm);
+    } else
+        e = launch_gemm_simt(op, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite_flag, st);
+    return e == cudaSuccess ? MPT_OK : MPT_ERR_CUDA;
+}
+
+}  // namespace mpt
+
 extern "C" {
 
 const char *mpt_version(void) { return "mpt 0.1 sm_100a"; }
@@ -877,27 +911,8 @@ int mpt_gemm_f16_ws(int op, int M, int N, int K, const uint16_t *A, int lda, con
                     int ldc, unsigned flags, const uint16_t *mask, int ldmask, uint32_t *nonfinite_flag,
                     uint32_t *status_dev, void *splitk_ws_dev, size_t splitk_ws_bytes, void *cuda_stream)
 {
-    if (!A || !B || !C) return MPT_ERR_INVALID_ARG;
-    if (op != MPT_OP_FWD && op != MPT_OP_DGRAD && op != MPT_OP_WGRAD) return MPT_ERR_INVALID_ARG;
-    if (M < 0 || N < 0 || K < 0) return MPT_ERR_SHAPE;
-    if (M == 0 || N == 0) return MPT_OK;
-    const int a_cols = op == MPT_OP_WGRAD ? M : K, b_cols = op == MPT_OP_FWD ? K : N;
-    if (lda < a_cols || ldb < b_cols || ldc < N || (mask && ldmask < N)) return MPT_ERR_SHAPE;
-    cudaStream_t st = (cudaStream_t)cuda_stream;
-    const bool relu = (flags & MPT_GEMM_RELU) != 0;
-    bool tc_ok = K > 0 && tc_gemm_supported(op, M, N, K, A, lda, B, ldb, C, ldc, mask, ldmask);
-    if ((flags & (MPT_GEMM_FORCE_TC | MPT_GEMM_FORCE_PAIR)) && !tc_ok) return MPT_ERR_SHAPE;
-    cudaError_t e;
-    if (tc_ok && !(flags & MPT_GEMM_FORCE_SIMT)) {
-        const bool pair = (flags & MPT_GEMM_FORCE_PAIR) || (!(flags & MPT_GEMM_FORCE_TC) && tc2_gemm_preferred(M, N, K));
-        if (pair)
-            e = launch_gemm_tc2(op, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite_flag, status_dev, st);
-        else
-            e = launch_gemm_tc(op, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite_flag, status_dev, st,
-                               (float *)splitk_ws_dev, splitk_ws_bytes);
-    } else
-        e = launch_gemm_simt(op, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite_flag, st);
-    return e == cudaSuccess ? MPT_OK : MPT_ERR_CUDA;
+    return mpt::dispatch_gemm(op, M, N, K, A, lda, B, ldb, C, ldc, flags, mask, ldmask, nonfinite_flag, status_dev,
+                              splitk_ws_dev, splitk_ws_bytes, (cudaStream_t)cuda_stream, nullptr);
 }
 
 int mpt_recast(const float *w32_dev, uint16_t *w16_dev, size_t n, void *cuda_stream)

@@ -53,6 +53,21 @@ __device__ __forceinline__ bool f32_nonfinite(float x)
     return (__float_as_uint(x) & 0x7F800000u) == 0x7F800000u;
 }
 
+// Fused LSTM gate epilogue of a forward product whose output columns are gate-interleaved
+// (column 4j+q = gate q of cell j; q: 0 input, 1 forget, 2 candidate, 3 output): the FP32
+// accumulators plus bias go through the gate non-linearities, the product's own output receives
+// the FP16 gate activations, and the new cell state and hidden state are written beside it.
+// All pitches are multiples of 8 elements and all bases 16-byte aligned.
+struct LstmEpi {
+    const uint16_t *bias;     // [4H] FP16 working copy
+    const uint16_t *c_prev;   // [B, H], pitch ldcp
+    int ldcp;
+    uint16_t *c_out;          // [B, H], pitch ldco
+    int ldco;
+    uint16_t *h_out;          // [B, H], pitch ldh
+    int ldh;
+};
+
 // Launchers (each returns a cudaError_t from the launch; all asynchronous on `st`).
 cudaError_t launch_recast(const float *w32, uint16_t *w16, size_t n, cudaStream_t st);
 cudaError_t launch_grad_nonfinite(const uint16_t *g16, size_t n, float inv_S, uint32_t *flag,
@@ -104,13 +119,36 @@ bool tc_gemm_supported(int op, int M, int N, int K, const void *A, int lda, cons
 cudaError_t launch_gemm_tc(int op, int M, int N, int K, const uint16_t *A, int lda, const uint16_t *B,
                            int ldb, uint16_t *C, int ldc, bool relu, const uint16_t *mask, int ldmask,
                            uint32_t *nonfinite_flag, uint32_t *status, cudaStream_t st, float *splitk_ws = nullptr,
-                           size_t splitk_ws_bytes = 0);
+                           size_t splitk_ws_bytes = 0, const LstmEpi *lstm = nullptr);
 void tc_gemm_plan(int M, int N, int K, size_t ws_bytes, int *bn_out, int *split_out, size_t *ws_needed);
 
 // CTA-pair variant (tcgen05 cta_group::2, 256x256 tiles); same operand rules as launch_gemm_tc.
 bool tc2_gemm_preferred(int M, int N, int K);
 cudaError_t launch_gemm_tc2(int op, int M, int N, int K, const uint16_t *A, int lda, const uint16_t *B, int ldb,
                             uint16_t *C, int ldc, bool relu, const uint16_t *mask, int ldmask,
-                            uint32_t *nonfinite_flag, uint32_t *status, cudaStream_t st);
+                            uint32_t *nonfinite_flag, uint32_t *status, cudaStream_t st, const LstmEpi *lstm = nullptr);
+
+// Shape checks and kernel choice for one product (used by the stateless entry points and the LSTM
+// layer); returns an MPT_* code.
+int dispatch_gemm(int op, int M, int N, int K, const uint16_t *A, int lda, const uint16_t *B, int ldb, uint16_t *C, int ldc,
+                  unsigned flags, const uint16_t *mask, int ldmask, uint32_t *nonfinite_flag, uint32_t *status_dev,
+                  void *splitk_ws_dev, size_t splitk_ws_bytes, cudaStream_t st, const LstmEpi *lstm);
+
+// LSTM layer pieces outside the products (see mpt.h, mpt_lstm_*):
+// gate product + gate arithmetic for shapes the tensor-core kernels do not take (any size, slow)
+cudaError_t launch_lstm_cell_simt(int B, int H, int K, const uint16_t *XR, int ldxr, const uint16_t *Wg, int ldw,
+                                  uint16_t *acts, int ldacts, const LstmEpi &e, cudaStream_t st);
+// backward of the gate arithmetic of one time step (dc_next may be null: zero)
+cudaError_t launch_lstm_cell_bwd(int B, int H, const uint16_t *dh, int lddh, const uint16_t *dc_next, int lddc,
+                                 const uint16_t *acts, int ldacts, const uint16_t *c_prev, int ldcp, const uint16_t *c16,
+                                 int ldc, uint16_t *dG, int lddg, uint16_t *dc_prev, int lddcp, cudaStream_t st);
+// db16[n] = rn16(sum over rows of dG[r, n]) with FP32 accumulation over a fixed partition;
+// parts: FP32 scratch [kBiasRowParts][cols]
+static constexpr int kBiasRowParts = 8;
+cudaError_t launch_bias_grad(const uint16_t *dG, size_t rows, int cols, int ld, float *parts, uint16_t *db16,
+                             uint32_t *nonfinite_flag, cudaStream_t st);
+// out = rn16(f32(a) + f32(b)) over a [rows, cols] block with pitches
+cudaError_t launch_add_f16(const uint16_t *a, int lda, const uint16_t *b, int ldb, uint16_t *out, int ldo, int rows,
+                           int cols, cudaStream_t st);
 
 }  // namespace mpt

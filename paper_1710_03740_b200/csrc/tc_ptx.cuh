@@ -6,6 +6,8 @@
 #include <cuda_fp16.h>
 #include <stdint.h>
 
+#include "mpt_common.cuh"
+
 namespace mpt {
 
 static constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
@@ -187,6 +189,63 @@ __device__ __forceinline__ void epilogue_store32(const uint32_t (&r)[32], uint16
             }
         }
     }
+}
+
+// LSTM gate arithmetic on FP32 values (sections 3.3, 4.6): one cell from its four pre-activations
+// (bias already added).  Returns the FP16 bit patterns of the gate activations in act[4], the new
+// cell state and the hidden state; h uses the STORED (rounded) cell state.
+__device__ __forceinline__ float sigmoid_f32(float x) { return __fdiv_rn(1.0f, __fadd_rn(1.0f, expf(-x))); }
+__device__ __forceinline__ void lstm_cell_math(const float (&pre)[4], float c_prev, uint32_t (&act)[4], uint32_t &c16,
+                                               uint32_t &h16)
+{
+    const float gi = sigmoid_f32(pre[0]), gf = sigmoid_f32(pre[1]), gg = tanhf(pre[2]), go = sigmoid_f32(pre[3]);
+    act[0] = (uint32_t)__half_as_ushort(__float2half_rn(gi));
+    act[1] = (uint32_t)__half_as_ushort(__float2half_rn(gf));
+    act[2] = (uint32_t)__half_as_ushort(__float2half_rn(gg));
+    act[3] = (uint32_t)__half_as_ushort(__float2half_rn(go));
+    const float c = __fadd_rn(__fmul_rn(gf, c_prev), __fmul_rn(gi, gg));
+    const __half ch = __float2half_rn(c);
+    c16 = (uint32_t)__half_as_ushort(ch);
+    h16 = (uint32_t)__half_as_ushort(__float2half_rn(__fmul_rn(go, tanhf(__half2float(ch)))));
+}
+
+// Epilogue of one thread for 32 consecutive gate-interleaved accumulator columns (8 whole cells)
+// of its output row: bias add, gate arithmetic, 128-bit stores of the activations (4), the
+// cell state (1) and the hidden state (1).  col0 is a multiple of 32 and col0 + 32 <= 4H.
+__device__ __forceinline__ void epilogue_lstm32(const uint32_t (&r)[32], uint16_t *arow, int row, int col0, const LstmEpi &e)
+{
+    const int j0 = col0 >> 2;
+    const uint4 cpv = *(const uint4 *)(e.c_prev + (size_t)row * e.ldcp + j0);
+    const uint32_t cpw[4] = {cpv.x, cpv.y, cpv.z, cpv.w};
+    uint32_t cw[8], hw[8];
+#pragma unroll
+    for (int g8 = 0; g8 < 4; g8++) {
+        const uint4 bv = __ldg((const uint4 *)(e.bias + col0 + g8 * 8));
+        const uint32_t bw[4] = {bv.x, bv.y, bv.z, bv.w};
+        uint32_t a[8];
+#pragma unroll
+        for (int cell = 0; cell < 2; cell++) {
+            float pre[4];
+#pragma unroll
+            for (int q = 0; q < 4; q++) {
+                const int idx = cell * 4 + q;
+                const uint32_t bh = (idx & 1) ? (bw[idx >> 1] >> 16) : (bw[idx >> 1] & 0xFFFFu);
+                pre[q] = __fadd_rn(__uint_as_float(r[g8 * 8 + idx]), __half2float(__ushort_as_half((unsigned short)bh)));
+            }
+            const int jc = g8 * 2 + cell;
+            const uint32_t ch = (jc & 1) ? (cpw[jc >> 1] >> 16) : (cpw[jc >> 1] & 0xFFFFu);
+            uint32_t act[4];
+            lstm_cell_math(pre, __half2float(__ushort_as_half((unsigned short)ch)), act, cw[jc], hw[jc]);
+#pragma unroll
+            for (int q = 0; q < 4; q++) a[cell * 4 + q] = act[q];
+        }
+        *(uint4 *)(arow + col0 + g8 * 8) = make_uint4(a[0] | (a[1] << 16), a[2] | (a[3] << 16), a[4] | (a[5] << 16),
+                                                      a[6] | (a[7] << 16));
+    }
+    *(uint4 *)(e.c_out + (size_t)row * e.ldco + j0) = make_uint4(cw[0] | (cw[1] << 16), cw[2] | (cw[3] << 16),
+                                                                 cw[4] | (cw[5] << 16), cw[6] | (cw[7] << 16));
+    *(uint4 *)(e.h_out + (size_t)row * e.ldh + j0) = make_uint4(hw[0] | (hw[1] << 16), hw[2] | (hw[3] << 16),
+                                                                hw[4] | (hw[5] << 16), hw[6] | (hw[7] << 16));
 }
 
 // ------------------------------------------------------------ cluster / 2-CTA forms

@@ -144,3 +144,35 @@ def gemm_operands(op, M, N, K, seed=2, scale_a=None, scale_b=None, fast=False):
         return normal_f16_fast(seqs[0], shape_a, sa), normal_f16_fast(seqs[1], shape_b, sb)
     return (normal_f16(np.random.default_rng(seqs[0]), shape_a, sa),
             normal_f16(np.random.default_rng(seqs[1]), shape_b, sb))
+
+
+# LSTM layer with projection (the recurrent layer of the language model of section 4.6: 8192 cells
+# projected to 1024, input width 1024; the batch of 1024 there is spread over 4 GPUs with 20
+# unrolled steps).  "small" spans several tiles with ragged edges and finishes on the CPU in
+# seconds; "biglstm" is the paper's layer with 2048 rows per step.
+LSTM_CONFIGS = {
+    "small": dict(T=4, B=200, I=64, H=160, P=96, S=1024.0, seed=71),
+    "medium": dict(T=3, B=384, I=256, H=1024, P=256, S=1024.0, seed=72),
+    "biglstm": dict(T=20, B=2048, I=1024, H=8192, P=1024, S=1024.0, seed=73),
+}
+
+
+def lstm_tensors(cfg, fast=False):
+    """Seeded FP16 tensors of one LSTM layer: x [T,B,I] ~ N(0,1); Wg [4H,I+P] and Wp [P,H] ~
+    N(0, 1/fan_in) with gate-interleaved rows (row 4j+q: gate q of cell j); bias16 [4H] ~ N(0, 0.1)
+    with +1 on the forget gates (the usual initialisation); r0 [B,P], c0 [B,H] ~ N(0, 0.25);
+    dr_ext [T,B,P] ~ S * N(0, 1/B) (a mean-loss gradient scaled by the loss scale)."""
+    T, B, I, H, P, S = cfg["T"], cfg["B"], cfg["I"], cfg["H"], cfg["P"], cfg["S"]
+    ss = np.random.SeedSequence(cfg["seed"]).spawn(7)
+    gen = (lambda q, shape, scale: normal_f16_fast(ss[q], shape, scale)) if fast else \
+          (lambda q, shape, scale: normal_f16(np.random.default_rng(ss[q]), shape, scale))
+    x = gen(0, (T, B, I), 1.0)
+    Wg = gen(1, (4 * H, I + P), 1.0 / np.sqrt(I + P))
+    Wp = gen(2, (P, H), 1.0 / np.sqrt(H))
+    bias = gen(3, (4 * H,), 0.1).astype(np.float32)
+    bias[1::4] += 1.0
+    bias16 = bias.astype(np.float16)
+    r0 = gen(4, (B, P), 0.5)
+    c0 = gen(5, (B, H), 0.5)
+    dr_ext = gen(6, (T, B, P), S / B)
+    return dict(x=x, Wg=Wg, Wp=Wp, bias16=bias16, r0=r0, c0=c0, dr_ext=dr_ext)
