@@ -386,10 +386,13 @@ typedef struct mpt_lstm_tensors {
     uint16_t *dWg16;         /* [4H, I+P] */
     uint16_t *dWp16;         /* [P, H] */
     uint16_t *dbias16;       /* [4H] */
-    float *bias_parts;       /* [8, 4H] FP32 scratch of the bias-gradient reduction */
+    float *bias_parts;       /* [8, 4H] FP32 scratch: bias-gradient partial sums in the backward pass; the forward
+                              * pass keeps an FP32 copy of the bias in its first 4H entries (may be null there) */
     uint32_t *nonfinite_flag; /* one word, OR-ed with 1 when a weight or bias gradient is inf/NaN (section 3.2);
                                 the caller zeroes it before mpt_lstm_backward */
     uint32_t *status_dev;    /* MPT status block of >= 16 words (first device-side error at word 3) or null */
+    void *splitk_ws;         /* optional scratch that lets the projection product split its long contraction */
+    size_t splitk_ws_bytes;  /* (mpt_gemm_workspace_bytes(MPT_OP_FWD, B, P, H) bytes; null / 0: never split) */
 } mpt_lstm_tensors;
 
 /* Forward over all T steps: 2T launches on the stream (gate product with fused gate epilogue,

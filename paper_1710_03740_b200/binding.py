@@ -63,7 +63,7 @@ _LSTM_FIELDS = ["Wg16", "bias16", "Wp16", "xr", "c", "h", "acts", "dr_ext", "dxr
 
 class LstmTensors(C.Structure):
     """mpt_lstm_tensors: device pointers of every tensor of the layer (see include/mpt.h)."""
-    _fields_ = [(name, C.c_void_p) for name in _LSTM_FIELDS]
+    _fields_ = [(name, C.c_void_p) for name in _LSTM_FIELDS] + [("splitk_ws", C.c_void_p), ("splitk_ws_bytes", C.c_size_t)]
 
 
 _lib = None
@@ -425,7 +425,10 @@ class LstmLayer:
         self.bias_parts = torch.zeros((8, 4 * H), dtype=torch.float32, device="cuda")
         self.status = torch.zeros(16, dtype=torch.int32, device="cuda")
         self.nonfinite_flag = torch.zeros(1, dtype=torch.int32, device="cuda")
-        self.tensors = LstmTensors(*[getattr(self, n if n != "status_dev" else "status").data_ptr() for n in _LSTM_FIELDS])
+        ws_bytes = mpt_gemm_workspace_bytes(OP_FWD, B, P, H)
+        self.splitk_ws = torch.zeros(max(ws_bytes, 16) // 4, dtype=torch.float32, device="cuda")
+        self.tensors = LstmTensors(*([getattr(self, n if n != "status_dev" else "status").data_ptr() for n in _LSTM_FIELDS]
+                                     + [self.splitk_ws.data_ptr() if ws_bytes else None, ws_bytes]))
 
     def forward(self, stream=None):
         _check(lib().mpt_lstm_forward(C.byref(self.desc), C.byref(self.tensors), _stream_ptr(stream)))

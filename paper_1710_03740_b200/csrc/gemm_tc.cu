@@ -86,8 +86,16 @@ __device__ __forceinline__ void report(const TcParams &p, volatile uint32_t *abo
     if (p.status) atomicCAS(p.status, 0u, code | ((uint32_t)blockIdx.x << 8));
 }
 
+// The gate epilogue (LSTM) does far more arithmetic per element than the plain one: it runs on two
+// sets of four epilogue warps, each set taking half of the columns of a tile.
+template <bool LSTM>
+struct EpiCfg {
+    static constexpr int SETS = LSTM ? 2 : 1;
+    static constexpr int THREADS = 64 + 128 * SETS;
+};
+
 template <bool A_MN, bool B_MN, int BLOCK_N, bool LSTM = false>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+__global__ void __launch_bounds__(EpiCfg<LSTM>::THREADS, 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcParams p)
 {
     constexpr int STAGES = TileCfg<BLOCK_N>::STAGES;
@@ -116,7 +124,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; s++) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int b = 0; b < 2; b++) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), 4); }
+        for (int b = 0; b < 2; b++) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), 4 * EpiCfg<LSTM>::SETS); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -242,6 +250,12 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
             uint16_t *crow = p.C + (size_t)row * p.ldc;
             const uint16_t *mrow = p.mask ? p.mask + (size_t)row * p.ldmask : nullptr;
             bool bad = false;
+            if constexpr (LSTM) {
+                const int set = (warp - 2) >> 2;
+                constexpr int NCH = BLOCK_N / 64;                          // this set's half of the tile's columns
+                epilogue_lstm_tile(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BLOCK_N + set * NCH * 32), NCH,
+                                   nb * BLOCK_N + set * NCH * 32, p.N, row, row_ok, crow, p.lstm);
+            } else
 #pragma unroll 1
             for (int c = 0; c < BLOCK_N / 32; c++) {
                 uint32_t r[32];
@@ -258,8 +272,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                                                  __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
                     }
                 } else if (row_ok && col0 < p.N) {
-                    if constexpr (LSTM) epilogue_lstm32(r, crow, row, col0, p.lstm);
-                    else epilogue_store32(r, crow, mrow, col0, p.N, p.relu != 0, bad);
+                    epilogue_store32(r, crow, mrow, col0, p.N, p.relu != 0, bad);
                 }
             }
             tc_fence_before();
@@ -375,7 +388,7 @@ static cudaError_t launch_variant(const CUtensorMap &ta, const CUtensorMap &tb, 
         if (e != cudaSuccess) return e;
         configured[dev] = true;
     }
-    kern<<<grid, NUM_THREADS, SMEM_BYTES, st>>>(ta, tb, p);
+    kern<<<grid, EpiCfg<LSTM>::THREADS, SMEM_BYTES, st>>>(ta, tb, p);
     return cudaGetLastError();
 }
 

@@ -103,8 +103,16 @@ __device__ __forceinline__ void report(const Params &p, volatile uint32_t *abort
     if (p.status) atomicCAS(p.status, 0u, code | 0x80u | ((uint32_t)blockIdx.x << 8));
 }
 
+// The gate epilogue (LSTM) does far more arithmetic per element than the plain one: it runs on two
+// sets of four epilogue warps, each set taking half of the columns of a unit.
+template <bool LSTM>
+struct EpiCfg {
+    static constexpr int SETS = LSTM ? 2 : 1;
+    static constexpr int THREADS = 64 + 128 * SETS;
+};
+
 template <bool A_MN, bool B_MN, bool LSTM = false>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+__global__ void __launch_bounds__(EpiCfg<LSTM>::THREADS, 1)
 k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
            const __grid_constant__ CUtensorMap tmBh, const Params p)
 {
@@ -128,7 +136,7 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; s++) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int b = 0; b < 2; b++) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), 8); }
+        for (int b = 0; b < 2; b++) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), 8 * EpiCfg<LSTM>::SETS); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -255,16 +263,18 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
             uint16_t *crow = p.C + (size_t)row * p.ldc;
             const uint16_t *mrow = p.mask ? p.mask + (size_t)row * p.ldmask : nullptr;
             bool bad = false;
+            if constexpr (LSTM) {
+                const int set = (warp - 2) >> 2, nch = w.width / 64;       // this set's half of the unit's columns
+                epilogue_lstm_tile(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * TILE_N + set * nch * 32), nch,
+                                   w.nb * TILE_N + w.n_off + set * nch * 32, p.N, row, row_ok, crow, p.lstm);
+            } else
 #pragma unroll 1
             for (int c = 0; c < w.width / 32; c++) {
                 uint32_t r[32];
                 tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * TILE_N + c * 32), r);
                 tc_wait_ld();
                 const int col0 = w.nb * TILE_N + w.n_off + c * 32;
-                if (row_ok && col0 < p.N) {
-                    if constexpr (LSTM) epilogue_lstm32(r, crow, row, col0, p.lstm);
-                    else epilogue_store32(r, crow, mrow, col0, p.N, p.relu != 0, bad);
-                }
+                if (row_ok && col0 < p.N) epilogue_store32(r, crow, mrow, col0, p.N, p.relu != 0, bad);
             }
             tc_fence_before();
             __syncwarp();
@@ -298,7 +308,7 @@ static cudaError_t launch_variant(const CUtensorMap &ta, const CUtensorMap &tb, 
     attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
-    cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+    cfg.blockDim = dim3(EpiCfg<LSTM>::THREADS, 1, 1);
     cfg.dynamicSmemBytes = SMEM_BYTES;
     cfg.stream = st;
     cfg.attrs = attr;

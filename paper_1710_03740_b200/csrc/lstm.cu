@@ -175,6 +175,12 @@ __global__ void __launch_bounds__(256) k_add_f16(const uint16_t *__restrict__ a,
     out[(size_t)r * ldo + c] = (uint16_t)f2h_u(__fadd_rn(h2f_u(a[(size_t)r * lda + c]), h2f_u(b[(size_t)r * ldb + c])));
 }
 
+__global__ void __launch_bounds__(256) k_widen_f16(const uint16_t *__restrict__ in16, float *__restrict__ out32, size_t n)
+{
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) out32[i] = h2f_u(in16[i]);
+}
+
 unsigned blocks_for(size_t n) { return (unsigned)((n + 255) / 256); }
 
 }  // namespace
@@ -213,6 +219,13 @@ cudaError_t launch_bias_grad(const uint16_t *dG, size_t rows, int cols, int ld, 
     dim3 grid((unsigned)((cols + 255) / 256), (unsigned)kBiasRowParts);
     k_bias_grad_partial<<<grid, 256, 0, st>>>(dG, rows, cols, ld, parts, vec);   // unaligned rows: element loads
     k_bias_grad_final<<<blocks_for((size_t)cols), 256, 0, st>>>(parts, kBiasRowParts, cols, db16, nonfinite_flag);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_widen_f16(const uint16_t *in16, float *out32, size_t n, cudaStream_t st)
+{
+    if (n == 0) return cudaSuccess;
+    k_widen_f16<<<blocks_for(n), 256, 0, st>>>(in16, out32, n);
     return cudaGetLastError();
 }
 

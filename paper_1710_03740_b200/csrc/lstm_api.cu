@@ -46,7 +46,7 @@ int mpt_lstm_cell_forward(int B, int H, int K, const uint16_t *xr, int ldxr, con
     if (B < 0 || H < 0 || K < 0) return MPT_ERR_SHAPE;
     if (B == 0 || H == 0) return MPT_OK;
     if (ldxr < K || ldw < K || ldacts < 4 * H || ldcp < H || ldco < H || ldh < H) return MPT_ERR_SHAPE;
-    LstmEpi e{bias16, c_prev, ldcp, c_out, ldco, h_out, ldh};
+    LstmEpi e{bias16, nullptr, c_prev, ldcp, c_out, ldco, h_out, ldh};
     return cell_forward(B, H, K, xr, ldxr, Wg, ldw, acts, ldacts, e, flags, status_dev, (cudaStream_t)cuda_stream);
 }
 
@@ -91,13 +91,20 @@ int mpt_lstm_forward(const mpt_lstm_desc *d, const mpt_lstm_tensors *t, void *cu
     cudaStream_t st = (cudaStream_t)cuda_stream;
     const int B = d->B, I = d->I, H = d->H, P = d->P, K = I + P;
     const size_t xr_step = (size_t)B * K, c_step = (size_t)B * H, a_step = (size_t)B * 4 * H;
+    // the first 4H floats of the bias-gradient scratch hold an exact FP32 copy of the bias during
+    // the forward pass: the gate epilogue then needs no FP16->FP32 conversions for it
+    const float *bias32 = nullptr;
+    if (t->bias_parts && (((uintptr_t)t->bias_parts) & 15) == 0) {
+        if (launch_widen_f16(t->bias16, t->bias_parts, (size_t)4 * H, st) != cudaSuccess) return MPT_ERR_CUDA;
+        bias32 = t->bias_parts;
+    }
     for (int s = 0; s < d->T; s++) {
-        LstmEpi e{t->bias16, t->c + s * c_step, H, t->c + (s + 1) * c_step, H, t->h + s * c_step, H};
+        LstmEpi e{t->bias16, bias32, t->c + s * c_step, H, t->c + (s + 1) * c_step, H, t->h + s * c_step, H};
         int r = cell_forward(B, H, K, t->xr + s * xr_step, K, t->Wg16, K, t->acts + s * a_step, 4 * H, e, 0, t->status_dev, st);
         if (r != MPT_OK) return r;
         // r_s = h_s . Wp^T, written into the recurrent columns of the next step's input rows
         r = dispatch_gemm(MPT_OP_FWD, B, P, H, t->h + s * c_step, H, t->Wp16, H, t->xr + (s + 1) * xr_step + I, K, 0, nullptr, 0,
-                          nullptr, t->status_dev, nullptr, 0, st, nullptr);
+                          nullptr, t->status_dev, t->splitk_ws, t->splitk_ws ? t->splitk_ws_bytes : 0, st, nullptr);
         if (r != MPT_OK) return r;
     }
     return MPT_OK;

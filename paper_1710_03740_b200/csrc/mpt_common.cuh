@@ -60,6 +60,7 @@ __device__ __forceinline__ bool f32_nonfinite(float x)
 // All pitches are multiples of 8 elements and all bases 16-byte aligned.
 struct LstmEpi {
     const uint16_t *bias;     // [4H] FP16 working copy
+    const float *bias32;      // [4H] the same values converted to FP32 (exactly), or null
     const uint16_t *c_prev;   // [B, H], pitch ldcp
     int ldcp;
     uint16_t *c_out;          // [B, H], pitch ldco
@@ -147,6 +148,8 @@ cudaError_t launch_lstm_cell_bwd(int B, int H, const uint16_t *dh, int lddh, con
 static constexpr int kBiasRowParts = 8;
 cudaError_t launch_bias_grad(const uint16_t *dG, size_t rows, int cols, int ld, float *parts, uint16_t *db16,
                              uint32_t *nonfinite_flag, cudaStream_t st);
+// out32[i] = f32(in16[i]) (exact)
+cudaError_t launch_widen_f16(const uint16_t *in16, float *out32, size_t n, cudaStream_t st);
 // out = rn16(f32(a) + f32(b)) over a [rows, cols] block with pitches
 cudaError_t launch_add_f16(const uint16_t *a, int lda, const uint16_t *b, int ldb, uint16_t *out, int ldo, int rows,
                            int cols, cudaStream_t st);

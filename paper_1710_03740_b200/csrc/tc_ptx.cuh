@@ -194,58 +194,174 @@ __device__ __forceinline__ void epilogue_store32(const uint32_t (&r)[32], uint16
 // LSTM gate arithmetic on FP32 values (sections 3.3, 4.6): one cell from its four pre-activations
 // (bias already added).  Returns the FP16 bit patterns of the gate activations in act[4], the new
 // cell state and the hidden state; h uses the STORED (rounded) cell state.
-__device__ __forceinline__ float sigmoid_f32(float x) { return __fdiv_rn(1.0f, __fadd_rn(1.0f, expf(-x))); }
+// The gate functions are evaluated with the hardware exp2 and reciprocal approximations (about
+// 1e-6 relative error, three orders below the FP16 rounding of the stored result).  The epilogue
+// runs beside the MMA stream and must not outlast a tile's main loop; its scarce resource is the
+// special-function pipe (exp2, reciprocal and FP16<->FP32 conversions all issue there), so
+// reciprocals are shared (1/a and 1/b from one reciprocal of a*b) and conversions are packed.
+__device__ __forceinline__ float rcp_approx(float x)
+{
+    float r;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+    return r;
+}
+// tanh(x) for |x| below 1/16 (odd polynomial; the exp form cancels there), as a factor of |x|
+__device__ __forceinline__ float tanh_small(float ax, float x2)
+{
+    return ax * (1.0f + x2 * (-0.33333334f + x2 * (0.13333334f + x2 * -0.053968254f)));
+}
+// The four gate values of one cell from its pre-activations: sigmoid(x) = 1/(1+exp(-x)) for
+// i, f, o and tanh(x) = (1-e)/(1+e), e = exp(-2|x|), for g, with ONE reciprocal of the product of
+// the four denominators.  Arguments of the sigmoids are clamped at -20 (sigmoid(-20) = 2e-9 rounds
+// to zero in FP16 either way) so that the product stays below 2^127.
+__device__ __forceinline__ void lstm_gates(const float (&pre)[4], float &gi, float &gf, float &gg, float &go)
+{
+    const float di = 1.0f + __expf(-fmaxf(pre[0], -20.0f));
+    const float df = 1.0f + __expf(-fmaxf(pre[1], -20.0f));
+    const float dq = 1.0f + __expf(-fmaxf(pre[3], -20.0f));
+    const float ag = fabsf(pre[2]);
+    const float eg = __expf(-2.0f * ag);
+    const float dg = 1.0f + eg;
+    const float pif = di * df, pgo = dg * dq;
+    const float r = rcp_approx(pif * pgo);
+    const float rif = r * pgo, rgo = r * pif;          // 1/(di*df), 1/(dg*dq)
+    gi = rif * df;
+    gf = rif * di;
+    go = rgo * dg;
+    const float big = (1.0f - eg) * (rgo * dq);
+    gg = copysignf(ag < 0.0625f ? tanh_small(ag, ag * ag) : big, pre[2]);
+    // NaN pre-activations must stay NaN (fmaxf drops them)
+    if (pre[0] != pre[0]) gi = pre[0];
+    if (pre[1] != pre[1]) gf = pre[1];
+    if (pre[3] != pre[3]) go = pre[3];
+}
+__device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi)
+{
+    const __half2 v = __floats2half2_rn(lo, hi);
+    return *(const uint32_t *)&v;
+}
+// Two neighbouring cells at once: act[0..3] / act[4..7] are the FP16 gate activations of the two
+// cells packed in pairs (i|f, g|o), c2 and h2 the two new cell and hidden states packed.  The
+// hidden state uses the STORED (rounded) cell state.
+__device__ __forceinline__ void lstm_cell_pair_math(const float (&pre0)[4], const float (&pre1)[4], float cp0, float cp1,
+                                                    uint32_t (&act)[4], uint32_t &c2, uint32_t &h2)
+{
+    float gi0, gf0, gg0, go0, gi1, gf1, gg1, go1;
+    lstm_gates(pre0, gi0, gf0, gg0, go0);
+    lstm_gates(pre1, gi1, gf1, gg1, go1);
+    act[0] = pack_f16x2(gi0, gf0);
+    act[1] = pack_f16x2(gg0, go0);
+    act[2] = pack_f16x2(gi1, gf1);
+    act[3] = pack_f16x2(gg1, go1);
+    const float c0 = __fadd_rn(__fmul_rn(gf0, cp0), __fmul_rn(gi0, gg0));
+    const float c1 = __fadd_rn(__fmul_rn(gf1, cp1), __fmul_rn(gi1, gg1));
+    const __half2 ch = __floats2half2_rn(c0, c1);
+    c2 = *(const uint32_t *)&ch;
+    const float s0 = __low2float(ch), s1 = __high2float(ch);
+    const float a0 = fabsf(s0), a1 = fabsf(s1);
+    const float e0 = __expf(-2.0f * a0), e1 = __expf(-2.0f * a1);
+    const float d0 = 1.0f + e0, d1 = 1.0f + e1;
+    const float r = rcp_approx(d0 * d1);
+    float t0 = (1.0f - e0) * (r * d1), t1 = (1.0f - e1) * (r * d0);
+    t0 = copysignf(a0 < 0.0625f ? tanh_small(a0, a0 * a0) : t0, s0);
+    t1 = copysignf(a1 < 0.0625f ? tanh_small(a1, a1 * a1) : t1, s1);
+    h2 = pack_f16x2(__fmul_rn(go0, t0), __fmul_rn(go1, t1));
+}
+// One cell on its own (CUDA-core kernel): the same arithmetic with the second lane idle.
 __device__ __forceinline__ void lstm_cell_math(const float (&pre)[4], float c_prev, uint32_t (&act)[4], uint32_t &c16,
                                                uint32_t &h16)
 {
-    const float gi = sigmoid_f32(pre[0]), gf = sigmoid_f32(pre[1]), gg = tanhf(pre[2]), go = sigmoid_f32(pre[3]);
-    act[0] = (uint32_t)__half_as_ushort(__float2half_rn(gi));
-    act[1] = (uint32_t)__half_as_ushort(__float2half_rn(gf));
-    act[2] = (uint32_t)__half_as_ushort(__float2half_rn(gg));
-    act[3] = (uint32_t)__half_as_ushort(__float2half_rn(go));
-    const float c = __fadd_rn(__fmul_rn(gf, c_prev), __fmul_rn(gi, gg));
-    const __half ch = __float2half_rn(c);
-    c16 = (uint32_t)__half_as_ushort(ch);
-    h16 = (uint32_t)__half_as_ushort(__float2half_rn(__fmul_rn(go, tanhf(__half2float(ch)))));
+    uint32_t a[4], c2, h2;
+    lstm_cell_pair_math(pre, pre, c_prev, c_prev, a, c2, h2);
+    act[0] = a[0] & 0xFFFFu; act[1] = a[0] >> 16; act[2] = a[1] & 0xFFFFu; act[3] = a[1] >> 16;
+    c16 = c2 & 0xFFFFu;
+    h16 = h2 & 0xFFFFu;
+}
+
+// Operands of the gate epilogue for one chunk of 32 gate-interleaved columns (8 whole cells) of
+// one row: the bias values of the chunk (FP32 when the caller provides a converted copy, else
+// FP16 bits in the first four vectors) and the eight previous cell states.
+struct LstmChunkIn {
+    uint4 b[8];
+    uint4 cp;
+};
+__device__ __forceinline__ void lstm_fetch(LstmChunkIn &in, const LstmEpi &e, int row, int col0)
+{
+    in.cp = *(const uint4 *)(e.c_prev + (size_t)row * e.ldcp + (col0 >> 2));
+    if (e.bias32) {
+#pragma unroll
+        for (int v = 0; v < 8; v++) in.b[v] = __ldg((const uint4 *)(e.bias32 + col0 + v * 4));
+    } else {
+#pragma unroll
+        for (int g8 = 0; g8 < 4; g8++) in.b[g8] = __ldg((const uint4 *)(e.bias + col0 + g8 * 8));
+    }
 }
 
 // Epilogue of one thread for 32 consecutive gate-interleaved accumulator columns (8 whole cells)
 // of its output row: bias add, gate arithmetic, 128-bit stores of the activations (4), the
 // cell state (1) and the hidden state (1).  col0 is a multiple of 32 and col0 + 32 <= 4H.
-__device__ __forceinline__ void epilogue_lstm32(const uint32_t (&r)[32], uint16_t *arow, int row, int col0, const LstmEpi &e)
+__device__ __forceinline__ void epilogue_lstm32(const uint32_t (&r)[32], const LstmChunkIn &in, uint16_t *arow, int row, int col0,
+                                                const LstmEpi &e)
 {
     const int j0 = col0 >> 2;
-    const uint4 cpv = *(const uint4 *)(e.c_prev + (size_t)row * e.ldcp + j0);
-    const uint32_t cpw[4] = {cpv.x, cpv.y, cpv.z, cpv.w};
-    uint32_t cw[8], hw[8];
+    const uint32_t cpw[4] = {in.cp.x, in.cp.y, in.cp.z, in.cp.w};
+    uint32_t cw[4], hw[4];
+    const bool f32bias = e.bias32 != nullptr;
 #pragma unroll
-    for (int g8 = 0; g8 < 4; g8++) {
-        const uint4 bv = __ldg((const uint4 *)(e.bias + col0 + g8 * 8));
-        const uint32_t bw[4] = {bv.x, bv.y, bv.z, bv.w};
-        uint32_t a[8];
+    for (int g8 = 0; g8 < 4; g8++) {      // 8 columns = 2 cells
+        float bias[8];
+        if (f32bias) {
+            const uint4 lo = in.b[2 * g8], hi = in.b[2 * g8 + 1];
+            bias[0] = __uint_as_float(lo.x); bias[1] = __uint_as_float(lo.y); bias[2] = __uint_as_float(lo.z);
+            bias[3] = __uint_as_float(lo.w); bias[4] = __uint_as_float(hi.x); bias[5] = __uint_as_float(hi.y);
+            bias[6] = __uint_as_float(hi.z); bias[7] = __uint_as_float(hi.w);
+        } else {
+            const uint32_t bw[4] = {in.b[g8].x, in.b[g8].y, in.b[g8].z, in.b[g8].w};
 #pragma unroll
-        for (int cell = 0; cell < 2; cell++) {
-            float pre[4];
-#pragma unroll
-            for (int q = 0; q < 4; q++) {
-                const int idx = cell * 4 + q;
-                const uint32_t bh = (idx & 1) ? (bw[idx >> 1] >> 16) : (bw[idx >> 1] & 0xFFFFu);
-                pre[q] = __fadd_rn(__uint_as_float(r[g8 * 8 + idx]), __half2float(__ushort_as_half((unsigned short)bh)));
+            for (int v = 0; v < 4; v++) {
+                const float2 f = __half22float2(*(const __half2 *)&bw[v]);
+                bias[2 * v] = f.x; bias[2 * v + 1] = f.y;
             }
-            const int jc = g8 * 2 + cell;
-            const uint32_t ch = (jc & 1) ? (cpw[jc >> 1] >> 16) : (cpw[jc >> 1] & 0xFFFFu);
-            uint32_t act[4];
-            lstm_cell_math(pre, __half2float(__ushort_as_half((unsigned short)ch)), act, cw[jc], hw[jc]);
-#pragma unroll
-            for (int q = 0; q < 4; q++) a[cell * 4 + q] = act[q];
         }
-        *(uint4 *)(arow + col0 + g8 * 8) = make_uint4(a[0] | (a[1] << 16), a[2] | (a[3] << 16), a[4] | (a[5] << 16),
-                                                      a[6] | (a[7] << 16));
+        float pre0[4], pre1[4];
+#pragma unroll
+        for (int q = 0; q < 4; q++) {
+            pre0[q] = __fadd_rn(__uint_as_float(r[g8 * 8 + q]), bias[q]);
+            pre1[q] = __fadd_rn(__uint_as_float(r[g8 * 8 + 4 + q]), bias[4 + q]);
+        }
+        const float2 cp = __half22float2(*(const __half2 *)&cpw[g8]);
+        uint32_t act[4];
+        lstm_cell_pair_math(pre0, pre1, cp.x, cp.y, act, cw[g8], hw[g8]);
+        *(uint4 *)(arow + col0 + g8 * 8) = make_uint4(act[0], act[1], act[2], act[3]);
     }
-    *(uint4 *)(e.c_out + (size_t)row * e.ldco + j0) = make_uint4(cw[0] | (cw[1] << 16), cw[2] | (cw[3] << 16),
-                                                                 cw[4] | (cw[5] << 16), cw[6] | (cw[7] << 16));
-    *(uint4 *)(e.h_out + (size_t)row * e.ldh + j0) = make_uint4(hw[0] | (hw[1] << 16), hw[2] | (hw[3] << 16),
-                                                                hw[4] | (hw[5] << 16), hw[6] | (hw[7] << 16));
+    *(uint4 *)(e.c_out + (size_t)row * e.ldco + j0) = make_uint4(cw[0], cw[1], cw[2], cw[3]);
+    *(uint4 *)(e.h_out + (size_t)row * e.ldh + j0) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+}
+
+// The whole gate epilogue of one thread for `nchunks` chunks of 32 accumulator columns starting at
+// tensor-memory address taddr / output column col_base.  The global operands of chunk c+1 are
+// requested before the arithmetic of chunk c, so their latency is hidden behind it.  Every lane
+// runs the collective tensor-memory loads; only lanes whose row exists touch global memory.
+__device__ __forceinline__ void epilogue_lstm_tile(uint32_t taddr, int nchunks, int col_base, int N, int row, bool row_ok,
+                                                   uint16_t *arow, const LstmEpi &e)
+{
+    LstmChunkIn cur, nxt;
+    cur.cp = make_uint4(0, 0, 0, 0);
+#pragma unroll
+    for (int v = 0; v < 8; v++) cur.b[v] = make_uint4(0, 0, 0, 0);
+    nxt = cur;
+    if (row_ok && col_base < N) lstm_fetch(cur, e, row, col_base);
+#pragma unroll 1
+    for (int c = 0; c < nchunks; c++) {
+        uint32_t r[32];
+        tc_ld32(taddr + (uint32_t)(c * 32), r);
+        const int col0 = col_base + c * 32;
+        const bool more = c + 1 < nchunks && row_ok && col0 + 32 < N;
+        if (more) lstm_fetch(nxt, e, row, col0 + 32);
+        tc_wait_ld();
+        if (row_ok && col0 < N) epilogue_lstm32(r, cur, arow, row, col0, e);
+        cur = nxt;
+    }
 }
 
 // ------------------------------------------------------------ cluster / 2-CTA forms

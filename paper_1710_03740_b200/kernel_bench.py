@@ -188,6 +188,54 @@ def bench_update_opt(n, kind, wd, iters, clip=0.0):
             "sustained_gbs": bpp * n / sus / 1e6, "flags": flags.tolist()}
 
 
+def bench_lstm(name, iters, steps=None):
+    """LSTM layer with projection: the fused gate step against the bare gate product, the backward
+    gate kernel, the bias-gradient reduction, and the whole layer forward + backward."""
+    cfg = dict(inputs.LSTM_CONFIGS[name])
+    if steps:
+        cfg["T"] = steps
+    T, B, I, H, P = cfg["T"], cfg["B"], cfg["I"], cfg["H"], cfg["P"]
+    K = I + P
+    layer = mpt.LstmLayer(T, B, I, H, P)
+    g = torch.Generator(device="cuda").manual_seed(9)
+
+    def fill(t, scale):
+        t.copy_((torch.randn(t.shape, device="cuda", generator=g) * scale).half().view(torch.int16))
+
+    fill(layer.Wg16, K ** -0.5); fill(layer.Wp16, H ** -0.5); fill(layer.bias16, 0.1)
+    fill(layer.xr, 1.0); fill(layer.c[0], 0.5); fill(layer.dr_ext, 1024.0 / B)
+    out = {"kernel": "lstm", "config": name, "T": T, "B": B, "I": I, "H": H, "P": P}
+    # one step's gate product with and without the fused gate arithmetic
+    fused = lambda: mpt.mpt_lstm_cell_forward(B, H, K, layer.xr[0], K, layer.Wg16, K, layer.bias16, layer.c[0], H,  # noqa: E731
+                                              layer.acts[0], 4 * H, layer.c[1], H, layer.h[0], H, 0, layer.status)
+    bare = lambda: mpt.mpt_gemm_f16(0, B, 4 * H, K, layer.xr[0], K, layer.Wg16, K, layer.acts[0], 4 * H, 0, None, 0,  # noqa: E731
+                                    None, layer.status)
+    fl = 2.0 * B * 4 * H * K
+    for key, fn in (("gate_fused", fused), ("gate_bare", bare)):
+        best, sus = _time(fn, iters)
+        out[key + "_ms"] = sus
+        out[key + "_tflops"] = fl / sus / 1e9
+    # whole layer
+    layer.forward()
+    fwd_best, fwd = _time(layer.forward, max(3, iters // 4))
+    bwd_best, bwd = _time(layer.backward, max(3, iters // 4))
+    flops = 3.0 * T * (2.0 * B * 4 * H * K + 2.0 * B * P * H)
+    out.update({"forward_ms": fwd, "backward_ms": bwd, "layer_tflops": flops / (fwd + bwd) / 1e9,
+                "forward_tflops": flops / 3 / fwd / 1e9, "backward_tflops": flops * 2 / 3 / bwd / 1e9})
+    # pieces of the backward pass
+    cb = lambda: mpt.mpt_lstm_cell_backward(B, H, layer.dh, H, layer.dc[0], H, layer.acts[0], 4 * H, layer.c[0], H,  # noqa: E731
+                                            layer.c[1], H, layer.dG[0], 4 * H, layer.dc[1], H)
+    best, sus = _time(cb, iters)
+    out["cell_bwd_ms"] = sus
+    out["cell_bwd_gbs"] = 26.0 * B * H / sus / 1e6
+    bg = lambda: mpt.mpt_bias_grad(layer.dG, T * B, 4 * H, 4 * H, layer.bias_parts, layer.dbias16, layer.nonfinite_flag)  # noqa: E731
+    best, sus = _time(bg, iters)
+    out["bias_grad_ms"] = sus
+    out["bias_grad_gbs"] = 2.0 * T * B * 4 * H / sus / 1e6
+    out["device_error"] = layer.device_error()
+    return out
+
+
 def bench_softmax(B, Cn, iters):
     g = torch.Generator(device="cuda").manual_seed(4)
     z = (torch.randn((B, Cn), device="cuda", generator=g) * 3).half()
@@ -270,6 +318,10 @@ def main():
     s.add_argument("--rows", type=int, default=4096)
     s.add_argument("--classes", type=int, default=32000)
     s.add_argument("--iters", type=int, default=20)
+    ls = sub.add_parser("lstm")
+    ls.add_argument("--config", default="biglstm", choices=sorted(inputs.LSTM_CONFIGS))
+    ls.add_argument("--steps", type=int, default=0, help="override the number of time steps")
+    ls.add_argument("--iters", type=int, default=20)
     t = sub.add_parser("step")
     t.add_argument("--workload", default="tiny", choices=["tiny", "scale_sweep", "scale_sweep_twin", "large_twin"])
     t.add_argument("--iters", type=int, default=50)
@@ -285,6 +337,8 @@ def main():
                 res = bench_gemm(M, N, K, op, args.iters, args.compare_library, flags, not args.no_workspace, args.sustain)
                 res["kernel_choice"] = args.kernel
                 print(json.dumps(res), flush=True)
+    elif args.cmd == "lstm":
+        print(json.dumps(bench_lstm(args.config, args.iters, args.steps)), flush=True)
     elif args.cmd == "update":
         kind = ["sgd", "nesterov", "adagrad", "adam"].index(args.optimizer)
         if kind == 0 and args.weight_decay == 0.0 and args.clip_norm == 0.0:
