@@ -164,6 +164,30 @@ def oracle_sample(cfg, seconds_target=12.0, operands=None):
             "sample": "forward GEMM slab: %d of %d rows x N=%d x K=%d in %.1f s" % (rows, B, fout, fin, dt)}
 
 
+def oracle_streaming_samples():
+    """The oracle's master update (P = 150,994,944 parameters with momentum, 20 B each: the update
+    of the LSTM-shaped config) and softmax cross-entropy (4096 x 32000 logits, 4 B each), timed as
+    they stand on the host cores; GB/s on the same algorithmic bytes as the GPU figures."""
+    from oracle import mpo
+    n = 150994944
+    rng = np.random.default_rng(7)
+    g16 = inputs.normal_f16_fast(np.random.SeedSequence(7), (n // 4096, 4096), 37.0).reshape(-1)
+    w32 = np.ones(n, dtype=np.float32)
+    v = np.zeros(n, dtype=np.float32)
+    w16 = np.zeros(n, dtype=np.uint16)
+    t0 = time.perf_counter()
+    mpo.update_apply(g16, w32, v, w16, np.float32(1.0 / 512), np.float32(0.01), np.float32(0.9), True)
+    t_upd = time.perf_counter() - t0
+    B, Cn = 4096, 32000
+    z = inputs.normal_f16_fast(np.random.SeedSequence(8), (B, Cn), 3.0)
+    y = rng.integers(0, Cn, B).astype(np.int32)
+    t0 = time.perf_counter()
+    mpo.softmax_ce(z, y, 8192.0)
+    t_sm = time.perf_counter() - t0
+    return {"update_gbs": 20.0 * n / t_upd / 1e9, "update_sample": "P=%d with momentum in %.2f s" % (n, t_upd),
+            "softmax_gbs": 4.0 * B * Cn / t_sm / 1e9, "softmax_sample": "%dx%d in %.2f s" % (B, Cn, t_sm)}
+
+
 def run_reference(args, cfg, rank):
     """Reference arm: the CPU oracle on the host cores, bounded sample per step."""
     if rank != 0:
@@ -196,6 +220,7 @@ def main():
     ap.add_argument("--impl", default="mine", choices=["mine", "reference"])
     ap.add_argument("--workload", default="large", choices=sorted(inputs.MLP_CONFIGS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="skip the LSTM-layer timing appended to the JSON line")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "mine" else args.warmup
     cfg = inputs.MLP_CONFIGS[args.workload]
@@ -344,9 +369,23 @@ def main():
             "clocks": clocks,
             "last_loss": loss, "last_overflow": flag,
         }
+        if world == 1 and not args.no_extras:
+            # not part of the step metric: the LSTM layer of the paper's language model (section 4.6),
+            # forward + backward through time, timed with CUDA events after the step benchmark
+            try:
+                from paper_1710_03740_b200.kernel_bench import bench_lstm
+                r = bench_lstm("biglstm", 8)
+                out["lstm_layer"] = {"config": {k: r[k] for k in ("T", "B", "I", "H", "P")}, "forward_ms": r["forward_ms"],
+                                     "backward_ms": r["backward_ms"], "tflops": r["layer_tflops"],
+                                     "gate_step_fused_ms": r["gate_fused_ms"], "gate_product_alone_ms": r["gate_bare_ms"],
+                                     "cell_backward_gbs": r["cell_bwd_gbs"], "bias_grad_gbs": r["bias_grad_gbs"],
+                                     "device_error": r["device_error"]}
+            except Exception as ex:  # an extra; never fatal for the bench line
+                out["lstm_layer"] = {"error": repr(ex)}
         if not args.no_cpu_baseline:
             try:
                 out["cpu_baseline"] = oracle_sample(cfg)
+                out["cpu_baseline"].update(oracle_streaming_samples())
             except Exception as ex:  # the oracle is a reported baseline; never fatal for the bench line
                 out["cpu_baseline"] = {"value": None, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
                                        "sample": "failed: %r" % (ex,)}

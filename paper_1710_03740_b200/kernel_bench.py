@@ -86,25 +86,32 @@ def _time_graph(fn, iters):
     return e0.elapsed_time(e1) / iters
 
 
-def _time(fn, iters, warmup=3):
+def _time(fn, iters, warmup=5):
+    """(best single launch, mean of `iters` back-to-back launches) in ms after `warmup` calls; the
+    median of the individually timed launches is kept in _time.last_median."""
     for _ in range(warmup):
         fn()
     torch.cuda.synchronize()
-    best = float("inf")
-    for _ in range(min(iters, 5)):
+    singles = []
+    for _ in range(max(5, min(iters, 20))):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         fn()
         e1.record()
         torch.cuda.synchronize()
-        best = min(best, e0.elapsed_time(e1))
+        singles.append(e0.elapsed_time(e1))
+    singles.sort()
+    _time.last_median = singles[len(singles) // 2]
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(iters):
         fn()
     e1.record()
     torch.cuda.synchronize()
-    return best, e0.elapsed_time(e1) / iters
+    return singles[0], e0.elapsed_time(e1) / iters
+
+
+_time.last_median = None
 
 
 def bench_gemm(M, N, K, op, iters, compare=False, flags=mpt.GEMM_FORCE_TC, use_workspace=True, sustain_s=0.0):
@@ -125,7 +132,8 @@ def bench_gemm(M, N, K, op, iters, compare=False, flags=mpt.GEMM_FORCE_TC, use_w
         sus = min(sus, _time_graph(lambda: mpt.mpt_gemm_f16_ws(op, M, N, K, A, sa[1], B, sb[1], C, N, flags, None, 0, None,
                                                                 st, ws if nws else None, torch.cuda.current_stream()),
                                    iters))
-    out = {"kernel": "gemm", "op": OPS[op], "M": M, "N": N, "K": K, "best_ms": best, "sustained_ms": sus,
+    out = {"kernel": "gemm", "op": OPS[op], "M": M, "N": N, "K": K, "best_ms": best, "median_ms": _time.last_median,
+           "sustained_ms": sus,
            "best_tflops": fl / best / 1e9, "sustained_tflops": fl / sus / 1e9, "device_error": int(st[0]), "splitk_workspace_mb": nws / 1e6,
            "working_set_mb": (A.numel() + B.numel() + C.numel()) * 2 / 1e6}
     if sustain_s > 0:
@@ -151,7 +159,7 @@ def bench_gemm(M, N, K, op, iters, compare=False, flags=mpt.GEMM_FORCE_TC, use_w
     return out
 
 
-def bench_update(n, momentum, iters):
+def bench_update(n, momentum, iters, sustain_s=0.0):
     g = torch.Generator(device="cuda").manual_seed(3)
     g16 = (torch.randn(n, device="cuda", generator=g) * 37).half()
     w32 = torch.randn(n, device="cuda", generator=g)
@@ -161,9 +169,17 @@ def bench_update(n, momentum, iters):
     fn = lambda: mpt.mpt_update_flat(g16, w32, v, w16, n, 1.0 / 512, 1e-4, 0.9, momentum, False, flags)  # noqa: E731
     best, sus = _time(fn, iters)
     bpp = 20 if momentum else 12
-    return {"kernel": "update", "params": n, "momentum": bool(momentum), "bytes_per_param": bpp, "best_ms": best,
-            "sustained_ms": sus, "best_gbs": bpp * n / best / 1e6, "sustained_gbs": bpp * n / sus / 1e6,
-            "working_set_mb": bpp * n / 2e6, "flags": flags.tolist()}
+    out = {"kernel": "update", "params": n, "momentum": bool(momentum), "bytes_per_param": bpp, "best_ms": best,
+           "median_ms": _time.last_median, "sustained_ms": sus, "best_gbs": bpp * n / best / 1e6,
+           "median_gbs": bpp * n / _time.last_median / 1e6, "sustained_gbs": bpp * n / sus / 1e6,
+           "working_set_mb": bpp * n / 1e6, "flags": flags.tolist()}
+    if bpp * n < 256e6:
+        out["note"] = "working set below 256 MB: L2-resident, not an HBM claim"
+    if sustain_s > 0:
+        ms, clk = _sustained(fn, sustain_s)
+        out["sustained_%gs_gbs" % sustain_s] = bpp * n / ms / 1e6
+        out["sustained_clocks"] = clk
+    return out
 
 
 def bench_update_opt(n, kind, wd, iters, clip=0.0):
@@ -236,7 +252,7 @@ def bench_lstm(name, iters, steps=None):
     return out
 
 
-def bench_softmax(B, Cn, iters):
+def bench_softmax(B, Cn, iters, sustain_s=0.0):
     g = torch.Generator(device="cuda").manual_seed(4)
     z = (torch.randn((B, Cn), device="cuda", generator=g) * 3).half()
     y = torch.randint(0, Cn, (B,), device="cuda", generator=g, dtype=torch.int32)
@@ -246,8 +262,15 @@ def bench_softmax(B, Cn, iters):
     fn = lambda: mpt.mpt_softmax_ce(z, Cn, y, B, Cn, 8192.0, dz, Cn, rl, loss, None)  # noqa: E731
     best, sus = _time(fn, iters)
     by = 4.0 * B * Cn
-    return {"kernel": "softmax_ce", "rows": B, "classes": Cn, "best_ms": best, "sustained_ms": sus,
-            "best_gbs": by / best / 1e6, "sustained_gbs": by / sus / 1e6, "loss": float(loss.item())}
+    out = {"kernel": "softmax_ce", "rows": B, "classes": Cn, "best_ms": best, "median_ms": _time.last_median,
+           "sustained_ms": sus, "best_gbs": by / best / 1e6, "sustained_gbs": by / sus / 1e6, "loss": float(loss.item())}
+    if by < 256e6:
+        out["note"] = "working set below 256 MB: L2-resident, not an HBM claim"
+    if sustain_s > 0:
+        ms, clk = _sustained(fn, sustain_s)
+        out["sustained_%gs_gbs" % sustain_s] = by / ms / 1e6
+        out["sustained_clocks"] = clk
+    return out
 
 
 def bench_step(workload, iters):
@@ -313,11 +336,13 @@ def main():
     u.add_argument("--optimizer", default="sgd", choices=["sgd", "nesterov", "adagrad", "adam"])
     u.add_argument("--weight-decay", type=float, default=0.0)
     u.add_argument("--clip-norm", type=float, default=0.0)
+    u.add_argument("--sustain", type=float, default=0.0, help="also time SECONDS of back-to-back launches with clocks sampled")
     u.add_argument("--iters", type=int, default=20)
     s = sub.add_parser("softmax")
     s.add_argument("--rows", type=int, default=4096)
     s.add_argument("--classes", type=int, default=32000)
     s.add_argument("--iters", type=int, default=20)
+    s.add_argument("--sustain", type=float, default=0.0)
     ls = sub.add_parser("lstm")
     ls.add_argument("--config", default="biglstm", choices=sorted(inputs.LSTM_CONFIGS))
     ls.add_argument("--steps", type=int, default=0, help="override the number of time steps")
@@ -342,11 +367,11 @@ def main():
     elif args.cmd == "update":
         kind = ["sgd", "nesterov", "adagrad", "adam"].index(args.optimizer)
         if kind == 0 and args.weight_decay == 0.0 and args.clip_norm == 0.0:
-            print(json.dumps(bench_update(args.params, args.momentum, args.iters)), flush=True)
+            print(json.dumps(bench_update(args.params, args.momentum, args.iters, args.sustain)), flush=True)
         else:
             print(json.dumps(bench_update_opt(args.params, kind, args.weight_decay, args.iters, args.clip_norm)), flush=True)
     else:
-        print(json.dumps(bench_softmax(args.rows, args.classes, args.iters)), flush=True)
+        print(json.dumps(bench_softmax(args.rows, args.classes, args.iters, args.sustain)), flush=True)
 
 
 if __name__ == "__main__":
