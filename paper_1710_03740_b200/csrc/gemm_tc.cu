@@ -327,6 +327,17 @@ __global__ void __launch_bounds__(256) k_splitk_reduce(const float *__restrict__
     if (nonfinite_flag && __any_sync(0xFFFFFFFFu, bad) && (threadIdx.x & 31) == 0) atomicOr(nonfinite_flag, 1u);
 }
 
+cudaError_t launch_splitk_reduce(const float *partial, int split_k, int M, int N, int ldp, uint16_t *C, int ldc, bool relu,
+                                 const uint16_t *mask, int ldmask, uint32_t *nonfinite_flag, cudaStream_t st)
+{
+    const size_t work = (size_t)M * ((N + 7) / 8);
+    size_t blocks = (work + 255) / 256;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    k_splitk_reduce<<<(unsigned)blocks, 256, 0, st>>>(partial, split_k, M, N, ldp, C, ldc, relu ? 1 : 0, mask, ldmask,
+                                                      nonfinite_flag);
+    return cudaGetLastError();
+}
+
 // ------------------------------------------------------------------ host side
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
@@ -416,12 +427,7 @@ static cudaError_t launch_bn(int op, int M, int N, int K, const uint16_t *A, int
     else if (op == MPT_OP_DGRAD) e = launch_variant<false, true, BN>(ta, tb, p, grid, st);
     else e = launch_variant<true, true, BN>(ta, tb, p, grid, st);
     if (e != cudaSuccess || p.split_k == 1) return e;
-    const size_t work = (size_t)M * ((N + 7) / 8);
-    size_t blocks = (work + 255) / 256;
-    if (blocks > 148 * 16) blocks = 148 * 16;
-    k_splitk_reduce<<<(unsigned)blocks, 256, 0, st>>>(p.partial, p.split_k, M, N, p.ldp, p.C, p.ldc, p.relu, p.mask,
-                                                      p.ldmask, p.nonfinite_flag);
-    return cudaGetLastError();
+    return launch_splitk_reduce(p.partial, p.split_k, M, N, p.ldp, p.C, p.ldc, p.relu != 0, p.mask, p.ldmask, p.nonfinite_flag, st);
 }
 
 // Tile width and split factor for the single-CTA kernel.  Cost model in tensor-pipe cycles: a
@@ -433,7 +439,7 @@ static cudaError_t launch_bn(int op, int M, int N, int K, const uint16_t *A, int
 // stays in L2 (about 64 bytes per cycle and SM).  Calibrated with launches replayed from a CUDA
 // graph on 2048x1024x8192, 1024x1024x4096, 512x256x4096 and the tiny-MLP products.  The split
 // is only considered when a workspace is available.
-void tc_gemm_plan(int M, int N, int K, size_t ws_bytes, int *bn_out, int *split_out, size_t *ws_needed)
+void tc_gemm_plan(int M, int N, int K, size_t ws_bytes, int *bn_out, int *split_out, size_t *ws_needed, double *cost_out)
 {
     const long tm = (M + BLOCK_M - 1) / BLOCK_M;
     const int nkb = (K + BLOCK_K - 1) / BLOCK_K;
@@ -456,6 +462,26 @@ void tc_gemm_plan(int M, int N, int K, size_t ws_bytes, int *bn_out, int *split_
     *bn_out = best_bn;
     *split_out = best_s;
     if (ws_needed) *ws_needed = best_s > 1 ? (size_t)best_s * M * (((size_t)N + 31) / 32 * 32) * 4 : 0;
+    if (cost_out) *cost_out = best;
+}
+
+bool tc_choose_pair(int M, int N, int K, size_t ws_bytes, size_t *ws_needed)
+{
+    if (ws_needed) *ws_needed = 0;
+    if (tc2_gemm_preferred(M, N, K)) return true;
+    int bn, s1, s2;
+    size_t need1 = 0, need2 = 0;
+    double c1 = 0.0, c2 = 0.0;
+    tc_gemm_plan(M, N, K, ws_bytes, &bn, &s1, &need1, &c1);
+    if (M >= 256 && N >= 256) {
+        tc2_split_plan(M, N, K, ws_bytes, &s2, &need2, &c2);
+        if (s2 > 1 && c2 < c1) {
+            if (ws_needed) *ws_needed = need2;
+            return true;
+        }
+    }
+    if (ws_needed) *ws_needed = need1;
+    return false;
 }
 
 cudaError_t launch_gemm_tc(int op, int M, int N, int K, const uint16_t *A, int lda, const uint16_t *B, int ldb,

@@ -61,6 +61,12 @@ struct Params {
     uint32_t *status;
     int tiles_m, tiles_n, group_m;   // pair tiles (256 rows x 256 columns)
     int full_units, num_units;       // units [0, full_units) are whole tiles, the rest are half tiles
+    // split-K (few tiles, long contraction): every whole tile is cut into split_k units along K;
+    // a unit leaves its raw FP32 accumulator in partial[part][M][ldp] and a second kernel adds the
+    // parts in ascending order and applies the epilogue.  split_k == 1: off.
+    int split_k;
+    float *partial;
+    int ldp;
     LstmEpi lstm;                    // read only by the LSTM instantiation of the kernel
 };
 
@@ -68,6 +74,8 @@ struct Unit {
     int mb, nb;      // tile coordinates
     int n_off;       // first column of the unit inside its tile (0 or 128)
     int width;       // 256 (whole tile) or 128 (half)
+    int tile, part;  // tile index and K part (split-K)
+    int kb0, kb1;    // k-blocks [kb0, kb1) of the contraction
 };
 
 __device__ __forceinline__ void tile_coords(const Params &p, int tile, int &mb, int &nb)
@@ -81,18 +89,27 @@ __device__ __forceinline__ void tile_coords(const Params &p, int tile, int &mb, 
     nb = r / gsz;
 }
 
-__device__ __forceinline__ Unit unit_of(const Params &p, int u)
+__device__ __forceinline__ Unit unit_of(const Params &p, int u, int nkb)
 {
     Unit w;
     int tile = u;
     w.n_off = 0;
     w.width = TILE_N;
-    if (u >= p.full_units) {
+    w.part = 0;
+    w.kb0 = 0;
+    w.kb1 = nkb;
+    if (p.split_k > 1) {            // parts of one tile are neighbouring units: they run side by side
+        tile = u / p.split_k;
+        w.part = u - tile * p.split_k;
+        w.kb0 = (int)(((long long)nkb * w.part) / p.split_k);
+        w.kb1 = (int)(((long long)nkb * (w.part + 1)) / p.split_k);
+    } else if (u >= p.full_units) {
         const int h = u - p.full_units;
         tile = p.full_units + (h >> 1);
         w.n_off = (h & 1) * (TILE_N / 2);
         w.width = TILE_N / 2;
     }
+    w.tile = tile;
     tile_coords(p, tile, w.mb, w.nb);
     return w;
 }
@@ -159,12 +176,12 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
             uint32_t issued = 0, s = 0, ph = 0;
             bool ok = true;
             for (int u = pair_id; u < num_units && ok; u += num_pairs) {
-                const Unit w = unit_of(p, u);
+                const Unit w = unit_of(p, u, nkb);
                 const int cta_n = w.width >> 1;                            // columns of B this CTA loads
                 const int m0 = w.mb * (2 * CTA_M) + (int)rank * CTA_M;    // this CTA's rows of A
                 const int n0 = w.nb * TILE_N + w.n_off + (int)rank * cta_n;
                 const uint32_t tx_bytes = 2u * (uint32_t)(A_STAGE_BYTES + cta_n * BLOCK_K * 2);
-                for (int kb = 0; kb < nkb; kb++, issued++, s = (s + 1 == STAGES) ? 0 : s + 1, ph ^= (s == 0)) {
+                for (int kb = w.kb0; kb < w.kb1; kb++, issued++, s = (s + 1 == STAGES) ? 0 : s + 1, ph ^= (s == 0)) {
                     if (!mbar_try_wait(empty_bar(s), ph ^ 1u) && !mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) {
                         if (!*abort_flag) report(p, abort_flag, KERR_WAIT_EMPTY);
                         ok = false;
@@ -211,7 +228,8 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
             bool ok = true;
             int t = 0;
             for (int u = pair_id; u < num_units && ok; u += num_pairs, t++) {
-                const uint32_t idesc = idesc_base | ((uint32_t)((u < p.full_units ? TILE_N : TILE_N / 2) >> 3) << 17);
+                const Unit w = unit_of(p, u, nkb);
+                const uint32_t idesc = idesc_base | ((uint32_t)(w.width >> 3) << 17);
                 const int buf = t & 1;
                 const uint32_t acc_ph = (t >> 1) & 1u;
                 if (!mbar_try_wait(acce_bar(buf), acc_ph ^ 1u) && !mbar_wait(acce_bar(buf), acc_ph ^ 1u, abort_flag)) {
@@ -222,7 +240,7 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * TILE_N);
                 uint32_t acc = 0;                          // first MMA of a tile overwrites the accumulator
-                for (int kb = 0; kb < nkb; kb++) {
+                for (int kb = w.kb0; kb < w.kb1; kb++) {
                     if (!mbar_try_wait(full_bar(s), ph) && !mbar_wait(full_bar(s), ph, abort_flag)) {
                         if (!*abort_flag) report(p, abort_flag, KERR_WAIT_FULL);
                         ok = false;
@@ -248,7 +266,7 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
         bool ok = true;
         int t = 0;
         for (int u = pair_id; u < num_units && ok; u += num_pairs, t++) {
-            const Unit w = unit_of(p, u);
+            const Unit w = unit_of(p, u, nkb);
             const int buf = t & 1;
             const uint32_t acc_ph = (t >> 1) & 1u;
             const bool got = mbar_wait(accf_bar(buf), acc_ph, abort_flag);
@@ -267,6 +285,23 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
                 const int set = (warp - 2) >> 2, nch = w.width / 64;       // this set's half of the unit's columns
                 epilogue_lstm_tile(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * TILE_N + set * nch * 32), nch,
                                    w.nb * TILE_N + w.n_off + set * nch * 32, p.N, row, row_ok, crow, p.lstm);
+            } else if (p.split_k > 1) {
+                // raw FP32 partial sums of this unit; ldp is a multiple of 32, so a started chunk is whole
+                float *prow = p.partial + ((size_t)w.part * p.M + row) * p.ldp;
+#pragma unroll 1
+                for (int c = 0; c < TILE_N / 32; c++) {
+                    uint32_t r[32];
+                    tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * TILE_N + c * 32), r);
+                    tc_wait_ld();
+                    const int col0 = w.nb * TILE_N + c * 32;
+                    if (row_ok && col0 < p.ldp) {
+                        float4 *dst = (float4 *)(prow + col0);
+#pragma unroll
+                        for (int v = 0; v < 8; v++)
+                            __stcg(dst + v, make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
+                                                        __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3])));
+                    }
+                }
             } else
 #pragma unroll 1
             for (int c = 0; c < w.width / 32; c++) {
@@ -330,7 +365,10 @@ static cudaError_t launch_variant(const CUtensorMap &ta, const CUtensorMap &tb, 
     const int pairs = tiles < max_pairs ? tiles : max_pairs;
     int full = (tiles / pairs) * pairs, rest = tiles - full;
     if (2 * tiles <= max_pairs) { full = 0; rest = tiles; }   // too few tiles for the clusters: halves all the way
-    if (rest > 0 && 2 * rest <= max_pairs) {
+    if (p.split_k > 1) {
+        p.full_units = tiles * p.split_k;
+        p.num_units = tiles * p.split_k;
+    } else if (rest > 0 && 2 * rest <= max_pairs) {
         p.full_units = full;
         p.num_units = full + 2 * rest;
     } else {
@@ -354,9 +392,39 @@ bool tc2_gemm_preferred(int M, int N, int K)
     return M >= 256 && N >= 256 && tiles >= 48;
 }
 
+// Split factor for the pair kernel on outputs with few 256x256 tiles and a long contraction.
+// Cost model in tensor-pipe cycles, same units as tc_gemm_plan: 512 cycles per 64-deep k-block of a
+// pair tile, the exposed epilogue of the last unit, a launch, and for a split the reduce launch
+// and the FP32 parts going to L2 and back (about 64 bytes per cycle and SM).  A part keeps at
+// least 16 k-blocks; all units fit in one round of the 74 clusters.  Measured (graph replay):
+// 2048x1024x8192 39-40 us split in two against 45 us as 64 half tiles; level with the single-CTA
+// kernel's split there and a little behind it on 1024x1024x4096, hence the extra constant.  A
+// variant in which the unit of a tile that finishes last adds the parts itself (no second launch)
+// was slower: one warp per 32 rows cannot keep enough loads in flight (47-60 us).
+void tc2_split_plan(int M, int N, int K, size_t ws_bytes, int *split_out, size_t *ws_needed, double *cost_out)
+{
+    const long tiles = (long)((M + 255) / 256) * ((N + 255) / 256);
+    const int nkb = (K + pair::BLOCK_K - 1) / pair::BLOCK_K;
+    const size_t ldp = ((size_t)N + 31) / 32 * 32;
+    double best = 1e30;
+    int best_s = 1;
+    for (int s = 1; s <= 8; s++) {
+        if (s > 1 && (nkb / s < 16 || tiles * s > 74)) break;
+        const size_t need = s > 1 ? (size_t)s * M * ldp * 4 : 0;
+        if (need > ws_bytes) break;
+        const long rounds = (tiles * s + 73) / 74;
+        double cost = rounds * ((double)nkb / s) * 512.0 + 8 * 400.0 + 14000.0;
+        if (s > 1) cost += 8000.0 + (double)need * 2.0 / 148.0 / 64.0;    // cluster launch + second launch + partial traffic
+        if (cost < best * 0.99) { best = cost; best_s = s; }
+    }
+    *split_out = best_s;
+    if (ws_needed) *ws_needed = best_s > 1 ? (size_t)best_s * M * ldp * 4 : 0;
+    if (cost_out) *cost_out = best;
+}
+
 cudaError_t launch_gemm_tc2(int op, int M, int N, int K, const uint16_t *A, int lda, const uint16_t *B, int ldb,
                             uint16_t *C, int ldc, bool relu, const uint16_t *mask, int ldmask, uint32_t *nonfinite_flag,
-                            uint32_t *status, cudaStream_t st, const LstmEpi *lstm)
+                            uint32_t *status, cudaStream_t st, const LstmEpi *lstm, void *splitk_ws, size_t splitk_ws_bytes)
 {
     using namespace pair;
     CUtensorMap ta, tb, tbh;
@@ -383,15 +451,29 @@ cudaError_t launch_gemm_tc2(int op, int M, int N, int K, const uint16_t *A, int 
     p.tiles_n = (N + TILE_N - 1) / TILE_N;
     p.group_m = 8;
     p.full_units = p.num_units = 0;
+    p.split_k = 1;
+    p.partial = nullptr;
+    p.ldp = (N + 31) / 32 * 32;
+    if (!lstm && splitk_ws && (((uintptr_t)splitk_ws) & 15) == 0) {
+        int split = 1;
+        tc2_split_plan(M, N, K, splitk_ws_bytes, &split, nullptr, nullptr);
+        if (split > 1) {
+            p.split_k = split;
+            p.partial = (float *)splitk_ws;
+        }
+    }
     p.lstm = LstmEpi{};
     if (lstm) {
         if (op != MPT_OP_FWD || (N & 31) != 0) return cudaErrorInvalidValue;
         p.lstm = *lstm;
         return launch_variant<false, false, true>(ta, tb, tbh, p, st);
     }
-    if (op == MPT_OP_FWD) return launch_variant<false, false>(ta, tb, tbh, p, st);
-    if (op == MPT_OP_DGRAD) return launch_variant<false, true>(ta, tb, tbh, p, st);
-    return launch_variant<true, true>(ta, tb, tbh, p, st);
+    cudaError_t e;
+    if (op == MPT_OP_FWD) e = launch_variant<false, false>(ta, tb, tbh, p, st);
+    else if (op == MPT_OP_DGRAD) e = launch_variant<false, true>(ta, tb, tbh, p, st);
+    else e = launch_variant<true, true>(ta, tb, tbh, p, st);
+    if (e != cudaSuccess || p.split_k == 1) return e;
+    return launch_splitk_reduce(p.partial, p.split_k, M, N, p.ldp, C, ldc, relu, mask, ldmask, nonfinite_flag, st);
 }
 
 }  // namespace mpt

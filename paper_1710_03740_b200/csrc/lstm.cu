@@ -50,7 +50,7 @@ struct CellGrad {
 
 __device__ __forceinline__ CellGrad cell_bwd(float gi, float gf, float gg, float go, float cp, float c, float dh, float dcn)
 {
-    const float tc = tanhf(c);
+    const float tc = tanhf(c);   // accurate: 1 - tc*tc below cancels, so an approximate tanh would show in dc
     const float dc = __fadd_rn(__fmul_rn(__fmul_rn(dh, go), __fsub_rn(1.0f, __fmul_rn(tc, tc))), dcn);
     const float dpo = __fmul_rn(__fmul_rn(dh, tc), __fmul_rn(go, __fsub_rn(1.0f, go)));
     const float dpi = __fmul_rn(__fmul_rn(dc, gg), __fmul_rn(gi, __fsub_rn(1.0f, gi)));
@@ -62,9 +62,10 @@ __device__ __forceinline__ CellGrad cell_bwd(float gi, float gf, float gg, float
     return r;
 }
 
-// Two cells per thread: one 128-bit load of the activations, 32-bit loads of the per-cell values.
-// H is even and all pitches are even (checked by the launcher), so the 32-bit accesses are aligned.
-__global__ void __launch_bounds__(256) k_lstm_cell_bwd(int B, int H2, const uint16_t *__restrict__ dh, int lddh,
+// Four cells per thread: two 128-bit loads of the activations, 64-bit loads of the per-cell values
+// (streaming hints: nothing is read twice).  H is a multiple of 4 and all pitches are multiples of 4
+// (checked by the launcher), so the 64-bit accesses are aligned.
+__global__ void __launch_bounds__(256) k_lstm_cell_bwd(int B, int H4, const uint16_t *__restrict__ dh, int lddh,
                                                        const uint16_t *__restrict__ dc_next, int lddc,
                                                        const uint16_t *__restrict__ acts, int ldacts,
                                                        const uint16_t *__restrict__ c_prev, int ldcp,
@@ -72,20 +73,33 @@ __global__ void __launch_bounds__(256) k_lstm_cell_bwd(int B, int H2, const uint
                                                        int lddg, uint16_t *__restrict__ dc_prev, int lddcp)
 {
     const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (idx >= (size_t)B * H2) return;
-    const int b = (int)(idx / H2), j = 2 * (int)(idx % H2);
-    const uint4 av = *(const uint4 *)(acts + (size_t)b * ldacts + 4 * j);
-    const uint32_t cpw = *(const uint32_t *)(c_prev + (size_t)b * ldcp + j);
-    const uint32_t cw = *(const uint32_t *)(c16 + (size_t)b * ldc + j);
-    const uint32_t dhw = *(const uint32_t *)(dh + (size_t)b * lddh + j);
-    const uint32_t dcw = dc_next ? *(const uint32_t *)(dc_next + (size_t)b * lddc + j) : 0u;
-    const CellGrad g0 = cell_bwd(h2f_u(av.x & 0xFFFFu), h2f_u(av.x >> 16), h2f_u(av.y & 0xFFFFu), h2f_u(av.y >> 16),
-                                 h2f_u(cpw & 0xFFFFu), h2f_u(cw & 0xFFFFu), h2f_u(dhw & 0xFFFFu), h2f_u(dcw & 0xFFFFu));
-    const CellGrad g1 = cell_bwd(h2f_u(av.z & 0xFFFFu), h2f_u(av.z >> 16), h2f_u(av.w & 0xFFFFu), h2f_u(av.w >> 16),
-                                 h2f_u(cpw >> 16), h2f_u(cw >> 16), h2f_u(dhw >> 16), h2f_u(dcw >> 16));
-    *(uint4 *)(dG + (size_t)b * lddg + 4 * j) = make_uint4(g0.dg[0] | (g0.dg[1] << 16), g0.dg[2] | (g0.dg[3] << 16),
-                                                           g1.dg[0] | (g1.dg[1] << 16), g1.dg[2] | (g1.dg[3] << 16));
-    *(uint32_t *)(dc_prev + (size_t)b * lddcp + j) = g0.dcp | (g1.dcp << 16);
+    if (idx >= (size_t)B * H4) return;
+    const int b = (int)(idx / H4), j = 4 * (int)(idx % H4);
+    const uint4 *ap = (const uint4 *)(acts + (size_t)b * ldacts + 4 * j);
+    const uint4 a0 = __ldcs(ap), a1 = __ldcs(ap + 1);
+    const uint2 cpw = __ldcs((const uint2 *)(c_prev + (size_t)b * ldcp + j));
+    const uint2 cw = __ldcs((const uint2 *)(c16 + (size_t)b * ldc + j));
+    const uint2 dhw = __ldcs((const uint2 *)(dh + (size_t)b * lddh + j));
+    const uint2 dcw = dc_next ? __ldcs((const uint2 *)(dc_next + (size_t)b * lddc + j)) : make_uint2(0u, 0u);
+    const uint32_t aw[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+    const uint32_t cp2[2] = {cpw.x, cpw.y}, c2[2] = {cw.x, cw.y}, dh2[2] = {dhw.x, dhw.y}, dc2[2] = {dcw.x, dcw.y};
+    uint32_t outg[8], outc[2];
+#pragma unroll
+    for (int k = 0; k < 4; k++) {
+        const int sh = (k & 1) * 16;
+        const CellGrad g = cell_bwd(h2f_u(aw[2 * k] & 0xFFFFu), h2f_u(aw[2 * k] >> 16), h2f_u(aw[2 * k + 1] & 0xFFFFu),
+                                    h2f_u(aw[2 * k + 1] >> 16), h2f_u((cp2[k >> 1] >> sh) & 0xFFFFu),
+                                    h2f_u((c2[k >> 1] >> sh) & 0xFFFFu), h2f_u((dh2[k >> 1] >> sh) & 0xFFFFu),
+                                    h2f_u((dc2[k >> 1] >> sh) & 0xFFFFu));
+        outg[2 * k] = g.dg[0] | (g.dg[1] << 16);
+        outg[2 * k + 1] = g.dg[2] | (g.dg[3] << 16);
+        if (k & 1) outc[k >> 1] |= g.dcp << 16;
+        else outc[k >> 1] = g.dcp;
+    }
+    uint4 *gp = (uint4 *)(dG + (size_t)b * lddg + 4 * j);
+    __stcs(gp, make_uint4(outg[0], outg[1], outg[2], outg[3]));
+    __stcs(gp + 1, make_uint4(outg[4], outg[5], outg[6], outg[7]));
+    __stcs((uint2 *)(dc_prev + (size_t)b * lddcp + j), make_uint2(outc[0], outc[1]));
 }
 
 // scalar form for odd H or unaligned buffers
@@ -200,10 +214,10 @@ cudaError_t launch_lstm_cell_bwd(int B, int H, const uint16_t *dh, int lddh, con
     if (B <= 0 || H <= 0) return cudaSuccess;
     const uintptr_t bits = (uintptr_t)acts | (uintptr_t)dG;
     const uintptr_t bits4 = (uintptr_t)dh | (uintptr_t)dc_next | (uintptr_t)c_prev | (uintptr_t)c16 | (uintptr_t)dc_prev;
-    const bool vec = (H % 2) == 0 && (bits & 15) == 0 && (bits4 & 3) == 0 && (ldacts % 8) == 0 && (lddg % 8) == 0 &&
-                     ((lddh | lddc | ldcp | ldc | lddcp) % 2) == 0;
+    const bool vec = (H % 4) == 0 && (bits & 15) == 0 && (bits4 & 7) == 0 && (ldacts % 8) == 0 && (lddg % 8) == 0 &&
+                     ((lddh | lddc | ldcp | ldc | lddcp) % 4) == 0;
     if (vec)
-        k_lstm_cell_bwd<<<blocks_for((size_t)B * (H / 2)), 256, 0, st>>>(B, H / 2, dh, lddh, dc_next, lddc, acts, ldacts, c_prev,
+        k_lstm_cell_bwd<<<blocks_for((size_t)B * (H / 4)), 256, 0, st>>>(B, H / 4, dh, lddh, dc_next, lddc, acts, ldacts, c_prev,
                                                                          ldcp, c16, ldc, dG, lddg, dc_prev, lddcp);
     else
         k_lstm_cell_bwd_scalar<<<blocks_for((size_t)B * H), 256, 0, st>>>(B, H, dh, lddh, dc_next, lddc, acts, ldacts, c_prev,

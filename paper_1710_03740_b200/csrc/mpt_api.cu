@@ -112,10 +112,8 @@ void make_plan(const mpt_layer_desc *layers, int L, int max_batch, int n_states,
         const int shapes[3][3] = {{B, out, in}, {out, in, B}, {B, in, out}};   // forward, wgrad, dgrad as (M, N, K)
         for (int k = 0; k < 3; k++) {
             if (k == 2 && l == 0) continue;
-            if (tc2_gemm_preferred(shapes[k][0], shapes[k][1], shapes[k][2])) continue;
-            int bn, split;
             size_t need = 0;
-            tc_gemm_plan(shapes[k][0], shapes[k][1], shapes[k][2], (size_t)256 << 20, &bn, &split, &need);
+            tc_choose_pair(shapes[k][0], shapes[k][1], shapes[k][2], (size_t)256 << 20, &need);
             if (need > need_max) need_max = need;
         }
     }
@@ -256,9 +254,9 @@ int gemm(mpt_ctx *c, int op, int M, int N, int K, const uint16_t *A, int lda, co
     cudaError_t e;
     ProfSpan span(c, MPT_PROF_GEMM, 2.0 * M * N * K);
     if (!c->disable_tc && tc_gemm_supported(op, M, N, K, A, lda, B, ldb, C, ldc, mask, ldmask)) {
-        if (!c->disable_pair && tc2_gemm_preferred(M, N, K))
+        if (!c->disable_pair && tc_choose_pair(M, N, K, c->plan.splitk_bytes, nullptr))
             e = launch_gemm_tc2(op, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite,
-                                c->status + ST_KERNEL_ERR, c->stream);
+                                c->status + ST_KERNEL_ERR, c->stream, nullptr, c->splitk_ws, c->plan.splitk_bytes);
         else
             e = launch_gemm_tc(op, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite,
                                c->status + ST_KERNEL_ERR, c->stream, c->splitk_ws, c->plan.splitk_bytes);
@@ -408,9 +406,12 @@ int dispatch_gemm(int op, int M, int N, int K, const uint16_t *A, int lda, const
     if (((flags & (MPT_GEMM_FORCE_TC | MPT_GEMM_FORCE_PAIR)) || lstm) && !tc_ok) return MPT_ERR_SHAPE;
     cudaError_t e;
     if (tc_ok && !(flags & MPT_GEMM_FORCE_SIMT)) {
-        const bool pair = (flags & MPT_GEMM_FORCE_PAIR) || (!(flags & MPT_GEMM_FORCE_TC) && tc2_gemm_preferred(M, N, K));
+        const size_t ws_ok = (splitk_ws_dev && (((uintptr_t)splitk_ws_dev) & 15) == 0) ? splitk_ws_bytes : 0;
+        const bool pair = (flags & MPT_GEMM_FORCE_PAIR) ||
+                          (!(flags & MPT_GEMM_FORCE_TC) && (lstm ? tc2_gemm_preferred(M, N, K) : tc_choose_pair(M, N, K, ws_ok, nullptr)));
         if (pair)
-            e = launch_gemm_tc2(op, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite_flag, status_dev, st, lstm);
+            e = launch_gemm_tc2(op, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite_flag, status_dev, st, lstm,
+                                splitk_ws_dev, splitk_ws_bytes);
         else
             e = launch_gemm_tc(op, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite_flag, status_dev, st,
                                (float *)splitk_ws_dev, splitk_ws_bytes, lstm);
@@ -893,9 +894,8 @@ int mpt_gemm_workspace_bytes(int op, int M, int N, int K, size_t *bytes_out)
     if (op != MPT_OP_FWD && op != MPT_OP_DGRAD && op != MPT_OP_WGRAD) return MPT_ERR_INVALID_ARG;
     if (M < 0 || N < 0 || K < 0) return MPT_ERR_SHAPE;
     *bytes_out = 0;
-    if (M == 0 || N == 0 || K == 0 || tc2_gemm_preferred(M, N, K)) return MPT_OK;
-    int bn, split;
-    tc_gemm_plan(M, N, K, (size_t)256 << 20, &bn, &split, bytes_out);
+    if (M == 0 || N == 0 || K == 0) return MPT_OK;
+    tc_choose_pair(M, N, K, (size_t)256 << 20, bytes_out);
     return MPT_OK;
 }
 

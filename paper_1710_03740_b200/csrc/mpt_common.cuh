@@ -121,13 +121,25 @@ cudaError_t launch_gemm_tc(int op, int M, int N, int K, const uint16_t *A, int l
                            int ldb, uint16_t *C, int ldc, bool relu, const uint16_t *mask, int ldmask,
                            uint32_t *nonfinite_flag, uint32_t *status, cudaStream_t st, float *splitk_ws = nullptr,
                            size_t splitk_ws_bytes = 0, const LstmEpi *lstm = nullptr);
-void tc_gemm_plan(int M, int N, int K, size_t ws_bytes, int *bn_out, int *split_out, size_t *ws_needed);
+void tc_gemm_plan(int M, int N, int K, size_t ws_bytes, int *bn_out, int *split_out, size_t *ws_needed,
+                  double *cost_out = nullptr);
+// Kernel choice for a product the tensor-core path takes: true = CTA-pair kernel (possibly with a
+// split contraction), false = single-CTA kernel; ws_needed = scratch the choice would like.
+bool tc_choose_pair(int M, int N, int K, size_t ws_bytes, size_t *ws_needed);
 
 // CTA-pair variant (tcgen05 cta_group::2, 256x256 tiles); same operand rules as launch_gemm_tc.
 bool tc2_gemm_preferred(int M, int N, int K);
 cudaError_t launch_gemm_tc2(int op, int M, int N, int K, const uint16_t *A, int lda, const uint16_t *B, int ldb,
                             uint16_t *C, int ldc, bool relu, const uint16_t *mask, int ldmask,
-                            uint32_t *nonfinite_flag, uint32_t *status, cudaStream_t st, const LstmEpi *lstm = nullptr);
+                            uint32_t *nonfinite_flag, uint32_t *status, cudaStream_t st, const LstmEpi *lstm = nullptr,
+                            void *splitk_ws = nullptr, size_t splitk_ws_bytes = 0);
+// Second step of a split product: C = epilogue(partial[0] + partial[1] + ...), parts added in
+// ascending order with one rounding per add.
+cudaError_t launch_splitk_reduce(const float *partial, int split_k, int M, int N, int ldp, uint16_t *C, int ldc, bool relu,
+                                 const uint16_t *mask, int ldmask, uint32_t *nonfinite_flag, cudaStream_t st);
+// Split factor, scratch need (FP32 parts) and modelled cost
+// of the pair kernel for an output with few tiles and a long contraction; split 1 = no split.
+void tc2_split_plan(int M, int N, int K, size_t ws_bytes, int *split_out, size_t *ws_needed, double *cost_out);
 
 // Shape checks and kernel choice for one product (used by the stateless entry points and the LSTM
 // layer); returns an MPT_* code.

@@ -39,6 +39,8 @@ def run_gemm(op, A, B, M, N, K, flags=0, mask=None, pad=0, want_flag=False, work
         nbytes = b.mpt_gemm_workspace_bytes(op, M, N, K)
         if nbytes == 0:
             pytest.skip("the library does not split this shape")
+        # room for any split either kernel may choose (the need reported is that of the automatic choice)
+        nbytes = max(nbytes, 9 * M * ((N + 31) // 32 * 32) * 4)
         ws = torch.full((nbytes // 4,), float("nan"), dtype=torch.float32, device="cuda")
         b.mpt_gemm_f16_ws(op, M, N, K, Ad, lda, Bd, ldb, Cd, ldc, flags, md, ldc if mask is not None else 0,
                           flag if want_flag else None, status, ws)
@@ -90,7 +92,7 @@ def test_simt_gemm_relu_mask_flag():
 
 def _check_tc(op, M, N, K, flags=0, mask=None, seed=21, scale=None, want_flag=False, kernel="tc", workspace=False):
     from paper_1710_03740_b200 import binding as b
-    force = b.GEMM_FORCE_PAIR if kernel == "pair" else b.GEMM_FORCE_TC
+    force = {"pair": b.GEMM_FORCE_PAIR, "tc": b.GEMM_FORCE_TC, "auto": 0}[kernel]
     sa = sb = scale
     A, B = inputs.gemm_operands(op, M, N, K, seed=seed, scale_a=sa, scale_b=sb)
     ref, ex, ab = mpo.gemm_f16(op, A, B, relu=bool(flags & b.GEMM_RELU), mask=mask, want_exact=True)
@@ -171,6 +173,29 @@ def test_split_k_parity_and_determinism(op, M, N, K):
 
 
 @pytest.mark.parametrize("op", [0, 1, 2])
+@pytest.mark.parametrize("M,N,K", [(512, 512, 4096), (1024, 512, 8192), (264, 520, 2056), (2048, 1024, 8192)])
+def test_pair_kernel_split_k(op, M, N, K):
+    """Few 256x256 tiles and a long contraction on the CTA-pair kernel: the contraction is split over
+    clusters and the FP32 parts are added in ascending order by the reduce kernel.  Same acceptance
+    rule; identical bits on reruns; ReLU, mask and the overflow flag go through the reduce kernel; a
+    scratch full of NaN bits is fine."""
+    from paper_1710_03740_b200 import binding as b
+    assert b.mpt_gemm_workspace_bytes(op, M, N, K) > 0
+    big = (M, N, K) == (2048, 1024, 8192)
+    got, ref, _, _ = _check_tc(op, M, N, K, workspace=True, kernel="pair")
+    for _ in range(3):
+        again, _, _, _ = _check_tc(op, M, N, K, workspace=True, kernel="pair")
+        assert np.array_equal(got, again)
+    auto, _, _, _ = _check_tc(op, M, N, K, workspace=True, kernel="auto")
+    if not big:
+        _check_tc(op, M, N, K, flags=b.GEMM_RELU, workspace=True, kernel="pair")
+        mask = np.random.default_rng(8).standard_normal((M, N)).astype(np.float16)
+        _check_tc(op, M, N, K, mask=mask, workspace=True, kernel="pair")
+        _, ref, flag, _ = _check_tc(op, M, N, K, scale=30.0, want_flag=True, workspace=True, kernel="pair")
+        assert flag == int(((ref & 0x7FFF) >= 0x7C00).any()) == 1
+
+
+@pytest.mark.parametrize("op", [0, 1, 2])
 def test_random_ragged_shapes_all_kernels(op):
     """Seeded random shapes with ragged M, N, K (pitches are multiples of 8): every kernel choice the
     library can make (single CTA, pair, automatic with and without a split-K workspace)."""
@@ -181,7 +206,7 @@ def test_random_ragged_shapes_all_kernels(op):
         N = int(rng.integers(1, 90)) * 8
         K = int(rng.choice([8, 24, 64, 72, 200, 520, 1032, 2056, 4104]))
         relu = bool(rng.integers(0, 2))
-        for kernel, ws in (("tc", False), ("pair", False), ("tc", True)):
+        for kernel, ws in (("tc", False), ("pair", False), ("tc", True), ("pair", True), ("auto", True)):
             if ws and b.mpt_gemm_workspace_bytes(op, M, N, K) == 0:
                 continue
             _check_tc(op, M, N, K, flags=b.GEMM_RELU if relu else 0, seed=int(rng.integers(1 << 30)), kernel=kernel,
