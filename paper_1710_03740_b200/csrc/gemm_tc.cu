@@ -28,7 +28,6 @@ namespace mpt {
 static constexpr int BLOCK_M = 128, BLOCK_K = 64, UMMA_K = 16;
 static constexpr int A_STAGE_BYTES = BLOCK_M * BLOCK_K * 2;  // 16 KB
 static constexpr int MN_BOX_BYTES = 64 * BLOCK_K * 2;        // one 64(mn) x 64(k) box of an MN-major operand
-static constexpr int NUM_THREADS = 192;
 
 // Tile width BN is 256 (four 48 KB stages) or, for outputs with too few 128x256 tiles to fill
 // the SMs, 128 (six 32 KB stages).  The two accumulator buffers take 2 * BN tensor-memory columns.

@@ -41,7 +41,6 @@ static constexpr int B_STAGE_BYTES = CTA_N * BLOCK_K * 2;   // 16 KB
 static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
 static constexpr int MN_BOX_BYTES = 64 * BLOCK_K * 2;
 static constexpr int TMEM_COLS = 512;
-static constexpr int NUM_THREADS = 192;
 static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256;
 
 // instruction descriptor without the N field (N >> 3 goes to bits 17..22)

@@ -313,7 +313,7 @@ int do_backward(mpt_ctx *c, const int32_t *labels_dev)
         ProfSpan span(c, MPT_PROF_SOFTMAX, 4.0 * B * last.out);
         e = launch_softmax_ce(last.act, last.ld_out, labels_dev, B, last.out, c->S, last.dact, last.ld_out, c->row_loss,
                               (float *)(c->status + ST_LOSS), c->status + ST_BAD_LABELS, c->stream, &nl,
-                              (const float *)(c->status + ST_SCALE));
+                              (const float *)(c->status + ST_SCALE), c->status + ST_KERNEL_ERR);
     }
     c->launches += nl;
     if (e != cudaSuccess) return cuda_fail(c, e, "softmax launch");

@@ -80,7 +80,7 @@ cudaError_t launch_update(const uint16_t *g16, float *w32, float *v, uint16_t *w
                           const float *inv_S_dev = nullptr);
 cudaError_t launch_softmax_ce(const uint16_t *z, int ldz, const int32_t *labels, int B, int C, float S,
                               uint16_t *dz, int lddz, float *row_loss, float *loss, uint32_t *bad_labels,
-                              cudaStream_t st, int *n_launches, const float *S_dev = nullptr);
+                              cudaStream_t st, int *n_launches, const float *S_dev = nullptr, uint32_t *kerr = nullptr);
 // Optimizer steps other than SGD(+momentum), and weight decay (see mpt.h MPT_OPT_*).  s1 / s2:
 // FP32 state arrays (momentum or squared-gradient sum; Adam's second moment).  For Adam the
 // bias corrections are 1 - beta^t with beta^t either passed by value (b1t, b2t: the products

@@ -5,6 +5,7 @@
 // in registers (k_softmax_ce_reg); other rows go through shared memory or are re-read
 // (k_softmax_ce).
 #include "mpt_common.cuh"
+#include "tc_ptx.cuh"
 
 namespace mpt {
 
@@ -209,6 +210,168 @@ __global__ void __launch_bounds__(1024, VPT <= 4 ? 2 : 1) k_softmax_ce_reg(const
     }
 }
 
+
+// ---------------------------------------------------------------- rows staged by bulk copies
+//
+// Persistent form for rows whose bytes are a multiple of 16 and fit three times into shared
+// memory: one CTA per SM walks rows blockIdx.x, blockIdx.x + gridDim.x, ...  A row arrives by one
+// bulk asynchronous copy (cp.async.bulk, completion on an mbarrier), is turned into its gradient in
+// place, and leaves by one bulk store; with three row buffers the load of row k+1 and the store of
+// row k-1 are in flight while the threads work on row k, so the memory system always has work.
+// Arithmetic as in k_softmax_ce_reg.  The waits are bounded like those of the product kernels.
+static constexpr int kSmaxThreads = 1024;
+
+// Block-wide max or sum for exactly 32 warps: warp results go through shared memory, then every
+// warp combines the 32 of them with the same xor-butterfly (both partners of a step add the same
+// two numbers, so all lanes and all warps hold identical bits; the order is fixed).
+__device__ __forceinline__ float block_reduce32(float v, bool is_max, float *red)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float other = __shfl_xor_sync(0xFFFFFFFFu, v, o);
+        v = is_max ? fmaxf(v, other) : v + other;
+    }
+    if (lane == 0) red[warp] = v;   // the caller alternates between two arrays: no reuse hazard
+    __syncthreads();
+    float r = red[lane];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float other = __shfl_xor_sync(0xFFFFFFFFu, r, o);
+        r = is_max ? fmaxf(r, other) : r + other;
+    }
+    return r;
+}
+
+__device__ __forceinline__ void bulk_load_row(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
+{
+    mbar_arrive_expect_tx(bar, bytes);
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void bulk_store_row(void *dst, uint32_t src, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(bytes) : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}template <int VPT>
+__global__ void __launch_bounds__(kSmaxThreads, 1) k_softmax_ce_bulk(const uint16_t *__restrict__ z, int ldz,
+                                                                      const int32_t *__restrict__ labels, int B, int C, float c,
+                                                                      uint16_t *__restrict__ dz, int lddz,
+                                                                      float *__restrict__ row_loss, uint32_t *bad_labels,
+                                                                      const float *__restrict__ scale_dev, uint32_t *kerr)
+{
+    extern __shared__ __align__(128) uint8_t rows_smem[];
+    __shared__ float red[2][32];   // max and sum use different arrays; a row's last use is two barriers back
+    __shared__ __align__(8) uint64_t bars[3];
+    __shared__ uint32_t abort_word;
+    if (scale_dev) c = __fdiv_rn(*scale_dev, (float)B);
+    const int tid = threadIdx.x;
+    const uint32_t row_bytes = (uint32_t)C * 2u;
+    const uint32_t buf_stride = (row_bytes + 127u) & ~127u;
+    const int C8 = C >> 3;
+    if (tid == 0) {
+        for (int i = 0; i < 3; i++) mbar_init(smem_u32(&bars[i]), 1);
+        abort_word = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+    const int n_my = blockIdx.x < B ? (B - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+    const uint32_t smem0 = smem_u32(rows_smem);
+    if (tid == 0 && n_my > 0) bulk_load_row(smem0, z + (size_t)blockIdx.x * ldz, row_bytes, smem_u32(&bars[0]));
+    constexpr float LOG2E = 1.4426950408889634f;
+    for (int k = 0; k < n_my; k++) {
+        const int row = blockIdx.x + k * gridDim.x;
+        const int b = k % 3;
+        if (tid == 0 && k + 1 < n_my) {
+            // buffer (k+1)%3 last held row k-2: its store must have finished reading shared memory
+            asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+            bulk_load_row(smem0 + (uint32_t)((k + 1) % 3) * buf_stride, z + (size_t)(row + gridDim.x) * ldz, row_bytes,
+                          smem_u32(&bars[(k + 1) % 3]));
+        }
+        if (!mbar_wait(smem_u32(&bars[b]), (uint32_t)((k / 3) & 1), &abort_word)) {
+            abort_word = 1;
+            if (kerr && tid == 0) atomicCAS(kerr, 0u, (uint32_t)KERR_WAIT_FULL | 0x40u | ((uint32_t)blockIdx.x << 8));
+        }
+        __syncthreads();
+        if (abort_word) break;
+        uint4 *rowv = (uint4 *)(rows_smem + (size_t)b * buf_stride);
+        uint16_t *rowh = (uint16_t *)rowv;
+        const int y = labels[row];
+        const bool good = y >= 0 && y < C;
+        float zy = 0.0f;
+        if (tid == 0 && good) zy = hbits2f(rowh[y]);       // read long before the row is overwritten in place
+        // pass 1: the maximum, on packed FP16 values (max is exact in any precision; like fmaxf it
+        // drops NaN operands, which then surface through the exponentials)
+        __half2 mh = __half2half2(__ushort_as_half((unsigned short)0xFC00u));   // -inf
+#pragma unroll
+        for (int u = 0; u < VPT; u++) {
+            const int i = tid + u * kSmaxThreads;
+            if (i < C8) {
+                const uint4 x = rowv[i];
+                mh = __hmax2(mh, __hmax2(__hmax2(*(const __half2 *)&x.x, *(const __half2 *)&x.y),
+                                         __hmax2(*(const __half2 *)&x.z, *(const __half2 *)&x.w)));
+            }
+        }
+        float m = fmaxf(__low2float(mh), __high2float(mh));
+        m = block_reduce32(m, true, red[0]);
+        // pass 2: exponentials, kept in registers for pass 3 (conversions and exp2 share the
+        // special-function pipe, the scarce unit of this kernel), and their sum
+        float ev[VPT * 8];
+        float s = 0.0f;
+#pragma unroll
+        for (int u = 0; u < VPT; u++) {
+            const int i = tid + u * kSmaxThreads;
+            if (i < C8) {
+                const uint4 x = rowv[i];
+                const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+                for (int q = 0; q < 4; q++) {
+                    const float2 f = __half22float2(*(const __half2 *)&w[q]);
+                    ev[u * 8 + 2 * q] = exp2f((f.x - m) * LOG2E);
+                    ev[u * 8 + 2 * q + 1] = exp2f((f.y - m) * LOG2E);
+                    s += ev[u * 8 + 2 * q];
+                    s += ev[u * 8 + 2 * q + 1];
+                }
+            }
+        }
+        s = block_reduce32(s, false, red[1]);
+        const float inv_s = __fdiv_rn(1.0f, s);
+        const float kk = good ? inv_s * c : 0.0f;
+#pragma unroll
+        for (int u = 0; u < VPT; u++) {
+            const int i = tid + u * kSmaxThreads;
+            if (i < C8) {
+                uint32_t o[4];
+#pragma unroll
+                for (int q = 0; q < 4; q++) {
+                    const __half2 h = __floats2half2_rn(ev[u * 8 + 2 * q] * kk, ev[u * 8 + 2 * q + 1] * kk);
+                    o[q] = good ? *(const uint32_t *)&h : 0u;
+                }
+                rowv[i] = make_uint4(o[0], o[1], o[2], o[3]);
+            }
+        }
+        __syncthreads();   // the row's gradient is in place before the label element is patched
+        if (tid == 0) {
+            if (good) {    // d_y = (e_y / s - 1) * c, evaluated separately because of the cancellation
+                const float ey = exp2f((zy - m) * LOG2E);
+                rowh[y] = (uint16_t)f2hbits(__fmul_rn(__fsub_rn(ey * inv_s, 1.0f), c));
+                row_loss[row] = (m + logf(s)) - zy;
+            } else {       // a label outside [0, C) contributes neither loss nor gradient
+                row_loss[row] = 0.0f;
+                if (bad_labels) atomicAdd(bad_labels, 1u);
+            }
+        }
+        // every thread's shared-memory writes become visible to the bulk store
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncthreads();
+        if (tid == 0) bulk_store_row(dz + (size_t)row * lddz, smem0 + (uint32_t)b * buf_stride, row_bytes);
+    }
+    if (tid == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+}
+
+
+
 // loss = (float)( sum_i (double)row_loss[i] / B ), fixed reduction order.
 __global__ void __launch_bounds__(256) k_loss_mean(const float *__restrict__ row_loss, int B, float *loss)
 {
@@ -240,12 +403,40 @@ static cudaError_t launch_variant(const uint16_t *z, int ldz, const int32_t *lab
 
 cudaError_t launch_softmax_ce(const uint16_t *z, int ldz, const int32_t *labels, int B, int C, float S,
                               uint16_t *dz, int lddz, float *row_loss, float *loss, uint32_t *bad_labels,
-                              cudaStream_t st, int *n_launches, const float *S_dev)
+                              cudaStream_t st, int *n_launches, const float *S_dev, uint32_t *kerr)
 {
     if (n_launches) *n_launches = 0;
     if (B <= 0 || C <= 0) return cudaSuccess;
     const float c = S / (float)B;  // one FP32 division
     const bool vec = ((((uintptr_t)z | (uintptr_t)dz) & 15) == 0) && (ldz % 8 == 0) && (lddz % 8 == 0) && C >= 8;
+    // many long rows: persistent CTAs with rows staged through shared memory by bulk copies
+    if (vec && (C % 8) == 0 && C >= 16384 && C <= 32768 && B >= 2 * 148) {
+        static int sms_dev[kMaxDevices] = {};
+        const int dev = current_device_slot();
+        if (dev < 0) return cudaErrorInvalidDevice;
+        const size_t smem = 3 * (((size_t)C * 2 + 127) & ~(size_t)127);
+        const int vpt = (C >> 3) <= 2048 ? 2 : 4;
+        auto kern = vpt == 2 ? k_softmax_ce_bulk<2> : k_softmax_ce_bulk<4>;
+        if (sms_dev[dev] == 0) {
+            int n = 0;
+            cudaError_t e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+            if (e != cudaSuccess) return e;
+            e = cudaFuncSetAttribute(k_softmax_ce_bulk<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+            if (e == cudaSuccess) e = cudaFuncSetAttribute(k_softmax_ce_bulk<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+            if (e != cudaSuccess) return e;
+            sms_dev[dev] = n > 0 ? n : 148;
+        }
+        const int grid = B < sms_dev[dev] ? B : sms_dev[dev];
+        kern<<<grid, kSmaxThreads, smem, st>>>(z, ldz, labels, B, C, c, dz, lddz, row_loss, bad_labels, S_dev, kerr);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+        if (n_launches) *n_launches = 1;
+        if (loss) {
+            k_loss_mean<<<1, 256, 0, st>>>(row_loss, B, loss);
+            if (n_launches) *n_launches = 2;
+        }
+        return cudaGetLastError();
+    }
     if (vec && (C >> 3) <= 8 * 1024) {
         // register-resident rows: T threads x VPT vectors cover C / 8 vectors
         const int C8 = C >> 3;

@@ -84,3 +84,34 @@ def test_softmax_ce_bad_labels():
     assert np.array_equal(dz, dz_ref) or gemm_accept(dz, dz_ref)[0].all()
     assert not dz[1].any() and not dz[2].any()
     assert abs(loss - loss_ref) < 1e-6
+
+
+@pytest.mark.parametrize("B,C,ld", [(300, 16384, 16384), (457, 32000, 32008), (296, 20480, 20480), (1000, 32768, 32768)])
+def test_softmax_ce_bulk_staged_rows(B, C, ld):
+    """Many long rows take the persistent kernel whose rows travel through shared memory by bulk
+    copies (three buffers per CTA: several rows per CTA, ragged last round, pitched rows).  Edge
+    rows (NaN, inf, all-equal maxima, labels outside the range) are mixed in."""
+    rng = np.random.default_rng(B + C)
+    z = (rng.standard_normal((B, C)) * 4).astype(np.float16)
+    y = rng.integers(0, C, B)
+    z[3, 5] = np.nan
+    z[4, 0] = np.inf
+    z[5, :] = 65504.0
+    z[6, 17] = 40.0
+    y[7] = C            # outside the range
+    y[B - 1] = -1
+    y[8] = C - 1
+    S = 8192.0
+    dz_ref, rl_ref, loss_ref, bad_ref = mpo.softmax_ce(z, y, S)
+    dz, rl, loss, bad = _run(z, y, S, ld)
+    assert bad == bad_ref == 2
+    ok, stats = gemm_accept(dz, dz_ref)
+    assert ok.all(), stats
+    assert stats["max_ulp"] <= 2
+    assert not dz[7].any() and not dz[B - 1].any()
+    assert np.array_equal(np.isnan(rl), np.isnan(rl_ref))
+    fin = ~np.isnan(rl_ref)
+    assert np.allclose(rl[fin], rl_ref[fin], rtol=2e-6, atol=C * 2.0 ** -24 + 2e-6)
+    # identical bits on a second run
+    dz2, rl2, _, _ = _run(z, y, S, ld)
+    assert np.array_equal(dz, dz2) and np.array_equal(rl.view(np.uint32), rl2.view(np.uint32))
