@@ -85,16 +85,16 @@ __device__ __forceinline__ void report(const TcParams &p, volatile uint32_t *abo
     if (p.status) atomicCAS(p.status, 0u, code | ((uint32_t)blockIdx.x << 8));
 }
 
-// The gate epilogue (LSTM) does far more arithmetic per element than the plain one: it runs on two
-// sets of four epilogue warps, each set taking half of the columns of a tile.
-template <bool LSTM>
+// Epilogue width: one set of four warps, or two sets that each take half of the columns of a tile
+// (launch-bound products and the LSTM gate epilogue; see the CTA-pair kernel for the measurements).
+template <bool WIDE>
 struct EpiCfg {
-    static constexpr int SETS = LSTM ? 2 : 1;
+    static constexpr int SETS = WIDE ? 2 : 1;
     static constexpr int THREADS = 64 + 128 * SETS;
 };
 
-template <bool A_MN, bool B_MN, int BLOCK_N, bool LSTM = false>
-__global__ void __launch_bounds__(EpiCfg<LSTM>::THREADS, 1)
+template <bool A_MN, bool B_MN, int BLOCK_N, bool LSTM = false, bool WIDE = false>
+__global__ void __launch_bounds__(EpiCfg<LSTM || WIDE>::THREADS, 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcParams p)
 {
     constexpr int STAGES = TileCfg<BLOCK_N>::STAGES;
@@ -123,7 +123,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; s++) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int b = 0; b < 2; b++) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), 4 * EpiCfg<LSTM>::SETS); }
+        for (int b = 0; b < 2; b++) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), 4 * EpiCfg<LSTM || WIDE>::SETS); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -256,7 +256,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                                    nb * BLOCK_N + set * NCH * 32, p.N, row, row_ok, crow, p.lstm);
             } else
 #pragma unroll 1
-            for (int c = 0; c < BLOCK_N / 32; c++) {
+            for (int c = ((warp - 2) >> 2) * (BLOCK_N / 32 / EpiCfg<LSTM || WIDE>::SETS);
+                 c < (((warp - 2) >> 2) + 1) * (BLOCK_N / 32 / EpiCfg<LSTM || WIDE>::SETS); c++) {
                 uint32_t r[32];
                 tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BLOCK_N + c * 32), r);
                 tc_wait_ld();
@@ -384,13 +385,13 @@ bool tc_gemm_supported(int op, int M, int N, int K, const void *A, int lda, cons
     return true;
 }
 
-template <bool A_MN, bool B_MN, int BN, bool LSTM = false>
+template <bool A_MN, bool B_MN, int BN, bool LSTM = false, bool WIDE = false>
 static cudaError_t launch_variant(const CUtensorMap &ta, const CUtensorMap &tb, const TcParams &p, int grid,
                                   cudaStream_t st)
 {
     static bool configured[kMaxDevices] = {};
     constexpr int SMEM_BYTES = TileCfg<BN>::SMEM_BYTES;
-    auto kern = k_gemm_tc<A_MN, B_MN, BN, LSTM>;
+    auto kern = k_gemm_tc<A_MN, B_MN, BN, LSTM, WIDE>;
     const int dev = current_device_slot();
     if (dev < 0) return cudaErrorInvalidDevice;
     if (!configured[dev]) {
@@ -398,7 +399,7 @@ static cudaError_t launch_variant(const CUtensorMap &ta, const CUtensorMap &tb, 
         if (e != cudaSuccess) return e;
         configured[dev] = true;
     }
-    kern<<<grid, EpiCfg<LSTM>::THREADS, SMEM_BYTES, st>>>(ta, tb, p);
+    kern<<<grid, EpiCfg<LSTM || WIDE>::THREADS, SMEM_BYTES, st>>>(ta, tb, p);
     return cudaGetLastError();
 }
 
@@ -421,10 +422,13 @@ static cudaError_t launch_bn(int op, int M, int N, int K, const uint16_t *A, int
     int units = p.tiles_m * p.tiles_n * p.split_k;
     int grid = units < 148 ? units : 148;
     cudaError_t e;
+    // two epilogue warp sets when a CTA's whole main loop is short (see EpiCfg)
+    const long kblocks = ((long)(units + 147) / 148) * ((K + BLOCK_K - 1) / BLOCK_K / p.split_k);
+    const bool wide = kblocks <= 160;
     if (op == MPT_OP_FWD && p.lstm.c_out) e = launch_variant<false, false, BN, true>(ta, tb, p, grid, st);
-    else if (op == MPT_OP_FWD) e = launch_variant<false, false, BN>(ta, tb, p, grid, st);
-    else if (op == MPT_OP_DGRAD) e = launch_variant<false, true, BN>(ta, tb, p, grid, st);
-    else e = launch_variant<true, true, BN>(ta, tb, p, grid, st);
+    else if (op == MPT_OP_FWD) e = wide ? launch_variant<false, false, BN, false, true>(ta, tb, p, grid, st) : launch_variant<false, false, BN>(ta, tb, p, grid, st);
+    else if (op == MPT_OP_DGRAD) e = wide ? launch_variant<false, true, BN, false, true>(ta, tb, p, grid, st) : launch_variant<false, true, BN>(ta, tb, p, grid, st);
+    else e = wide ? launch_variant<true, true, BN, false, true>(ta, tb, p, grid, st) : launch_variant<true, true, BN>(ta, tb, p, grid, st);
     if (e != cudaSuccess || p.split_k == 1) return e;
     return launch_splitk_reduce(p.partial, p.split_k, M, N, p.ldp, p.C, p.ldc, p.relu != 0, p.mask, p.ldmask, p.nonfinite_flag, st);
 }

@@ -119,16 +119,19 @@ __device__ __forceinline__ void report(const Params &p, volatile uint32_t *abort
     if (p.status) atomicCAS(p.status, 0u, code | 0x80u | ((uint32_t)blockIdx.x << 8));
 }
 
-// The gate epilogue (LSTM) does far more arithmetic per element than the plain one: it runs on two
-// sets of four epilogue warps, each set taking half of the columns of a unit.
-template <bool LSTM>
+// Epilogue width.  One set of four warps drains an accumulator in about 2.4 us, which hides behind
+// the next tile's main loop when a CTA has many tiles.  With two sets, each taking half of the
+// columns of a unit, the exposed epilogue of the last tile halves: launch-bound products gain
+// (1024^3 -7 %, tiny-MLP step -12 %), long ones lose about 1.4 % (more warps polling under the power
+// cap).  The gate epilogue (LSTM) does far more arithmetic per element and always uses two sets.
+template <bool WIDE>
 struct EpiCfg {
-    static constexpr int SETS = LSTM ? 2 : 1;
+    static constexpr int SETS = WIDE ? 2 : 1;
     static constexpr int THREADS = 64 + 128 * SETS;
 };
 
-template <bool A_MN, bool B_MN, bool LSTM = false>
-__global__ void __launch_bounds__(EpiCfg<LSTM>::THREADS, 1)
+template <bool A_MN, bool B_MN, bool LSTM = false, bool WIDE = false>
+__global__ void __launch_bounds__(EpiCfg<LSTM || WIDE>::THREADS, 1)
 k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
            const __grid_constant__ CUtensorMap tmBh, const Params p)
 {
@@ -152,7 +155,7 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; s++) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int b = 0; b < 2; b++) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), 8 * EpiCfg<LSTM>::SETS); }
+        for (int b = 0; b < 2; b++) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), 8 * EpiCfg<LSTM || WIDE>::SETS); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -287,8 +290,10 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
             } else if (p.split_k > 1) {
                 // raw FP32 partial sums of this unit; ldp is a multiple of 32, so a started chunk is whole
                 float *prow = p.partial + ((size_t)w.part * p.M + row) * p.ldp;
+                constexpr int NCH = TILE_N / 32 / EpiCfg<LSTM || WIDE>::SETS;
+                const int set = (warp - 2) >> 2;
 #pragma unroll 1
-                for (int c = 0; c < TILE_N / 32; c++) {
+                for (int c = set * NCH; c < (set + 1) * NCH; c++) {
                     uint32_t r[32];
                     tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * TILE_N + c * 32), r);
                     tc_wait_ld();
@@ -301,14 +306,16 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
                                                         __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3])));
                     }
                 }
-            } else
+            } else {
+                const int set = (warp - 2) >> 2, nch = w.width / 32 / EpiCfg<LSTM || WIDE>::SETS;   // this set's share of the columns
 #pragma unroll 1
-            for (int c = 0; c < w.width / 32; c++) {
-                uint32_t r[32];
-                tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * TILE_N + c * 32), r);
-                tc_wait_ld();
-                const int col0 = w.nb * TILE_N + w.n_off + c * 32;
-                if (row_ok && col0 < p.N) epilogue_store32(r, crow, mrow, col0, p.N, p.relu != 0, bad);
+                for (int c = set * nch; c < (set + 1) * nch; c++) {
+                    uint32_t r[32];
+                    tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * TILE_N + c * 32), r);
+                    tc_wait_ld();
+                    const int col0 = w.nb * TILE_N + w.n_off + c * 32;
+                    if (row_ok && col0 < p.N) epilogue_store32(r, crow, mrow, col0, p.N, p.relu != 0, bad);
+                }
             }
             tc_fence_before();
             __syncwarp();
@@ -328,12 +335,12 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
     }
 }
 
-template <bool A_MN, bool B_MN, bool LSTM = false>
+template <bool A_MN, bool B_MN, bool LSTM = false, bool WIDE = false>
 static cudaError_t launch_variant(const CUtensorMap &ta, const CUtensorMap &tb, const CUtensorMap &tbh, Params p,
                                   cudaStream_t st)
 {
     static int max_pairs_dev[kMaxDevices] = {};     // 0 = this device not configured yet
-    auto kern = k_gemm_tc2<A_MN, B_MN, LSTM>;
+    auto kern = k_gemm_tc2<A_MN, B_MN, LSTM, WIDE>;
     const int dev = current_device_slot();
     if (dev < 0) return cudaErrorInvalidDevice;
     cudaLaunchConfig_t cfg = {};
@@ -342,7 +349,7 @@ static cudaError_t launch_variant(const CUtensorMap &ta, const CUtensorMap &tb, 
     attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
-    cfg.blockDim = dim3(EpiCfg<LSTM>::THREADS, 1, 1);
+    cfg.blockDim = dim3(EpiCfg<LSTM || WIDE>::THREADS, 1, 1);
     cfg.dynamicSmemBytes = SMEM_BYTES;
     cfg.stream = st;
     cfg.attrs = attr;
@@ -467,10 +474,14 @@ cudaError_t launch_gemm_tc2(int op, int M, int N, int K, const uint16_t *A, int 
         p.lstm = *lstm;
         return launch_variant<false, false, true>(ta, tb, tbh, p, st);
     }
+    // two epilogue warp sets when a cluster's whole main loop is short (see EpiCfg)
+    const long units = (long)p.tiles_m * p.tiles_n * p.split_k;
+    const long kblocks = ((units + 73) / 74) * ((K + BLOCK_K - 1) / BLOCK_K / p.split_k);
+    const bool wide = kblocks <= 160;
     cudaError_t e;
-    if (op == MPT_OP_FWD) e = launch_variant<false, false>(ta, tb, tbh, p, st);
-    else if (op == MPT_OP_DGRAD) e = launch_variant<false, true>(ta, tb, tbh, p, st);
-    else e = launch_variant<true, true>(ta, tb, tbh, p, st);
+    if (op == MPT_OP_FWD) e = wide ? launch_variant<false, false, false, true>(ta, tb, tbh, p, st) : launch_variant<false, false>(ta, tb, tbh, p, st);
+    else if (op == MPT_OP_DGRAD) e = wide ? launch_variant<false, true, false, true>(ta, tb, tbh, p, st) : launch_variant<false, true>(ta, tb, tbh, p, st);
+    else e = wide ? launch_variant<true, true, false, true>(ta, tb, tbh, p, st) : launch_variant<true, true>(ta, tb, tbh, p, st);
     if (e != cudaSuccess || p.split_k == 1) return e;
     return launch_splitk_reduce(p.partial, p.split_k, M, N, p.ldp, C, ldc, relu, mask, ldmask, nonfinite_flag, st);
 }
