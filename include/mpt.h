@@ -70,6 +70,10 @@ extern "C" {
                                   same alignment rules.  Without a FORCE flag the library picks the
                                   pair kernel when the output has at least 48 tiles of 256x256,
                                   else the single-CTA one */
+#define MPT_GEMM_FORCE_PAIR512 16u /* require the CTA-pair kernel with 256x512 tiles (two accumulators
+                                  fed by one stream of A, epilogue not overlapped); same alignment
+                                  rules.  Moves about a quarter fewer operand bytes and is not faster;
+                                  never picked automatically */
 
 /* mpt_get_tensor kinds */
 #define MPT_T_W16 0        /* FP16 working weights   [out, in]            */

@@ -403,9 +403,11 @@ int dispatch_gemm(int op, int M, int N, int K, const uint16_t *A, int lda, const
     if (lda < a_cols || ldb < b_cols || ldc < N || (mask && ldmask < N)) return MPT_ERR_SHAPE;
     const bool relu = (flags & MPT_GEMM_RELU) != 0;
     bool tc_ok = K > 0 && tc_gemm_supported(op, M, N, K, A, lda, B, ldb, C, ldc, mask, ldmask);
-    if (((flags & (MPT_GEMM_FORCE_TC | MPT_GEMM_FORCE_PAIR)) || lstm) && !tc_ok) return MPT_ERR_SHAPE;
+    if (((flags & (MPT_GEMM_FORCE_TC | MPT_GEMM_FORCE_PAIR | MPT_GEMM_FORCE_PAIR512)) || lstm) && !tc_ok) return MPT_ERR_SHAPE;
     cudaError_t e;
-    if (tc_ok && !(flags & MPT_GEMM_FORCE_SIMT)) {
+    if (tc_ok && !lstm && (flags & MPT_GEMM_FORCE_PAIR512)) {
+        e = launch_gemm_tc3(op, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite_flag, status_dev, st);
+    } else if (tc_ok && !(flags & MPT_GEMM_FORCE_SIMT)) {
         const size_t ws_ok = (splitk_ws_dev && (((uintptr_t)splitk_ws_dev) & 15) == 0) ? splitk_ws_bytes : 0;
         const bool pair = (flags & MPT_GEMM_FORCE_PAIR) ||
                           (!(flags & MPT_GEMM_FORCE_TC) && (lstm ? tc2_gemm_preferred(M, N, K) : tc_choose_pair(M, N, K, ws_ok, nullptr)));

@@ -137,6 +137,11 @@ cudaError_t launch_gemm_tc2(int op, int M, int N, int K, const uint16_t *A, int 
 // ascending order with one rounding per add.
 cudaError_t launch_splitk_reduce(const float *partial, int split_k, int M, int N, int ldp, uint16_t *C, int ldc, bool relu,
                                  const uint16_t *mask, int ldmask, uint32_t *nonfinite_flag, cudaStream_t st);
+// CTA-pair variant with 256x512 tiles (two accumulators fed by one stream of A; the epilogue is
+// not overlapped): less operand traffic, not faster; only on request (MPT_GEMM_FORCE_PAIR512).
+cudaError_t launch_gemm_tc3(int op, int M, int N, int K, const uint16_t *A, int lda, const uint16_t *B, int ldb,
+                            uint16_t *C, int ldc, bool relu, const uint16_t *mask, int ldmask,
+                            uint32_t *nonfinite_flag, uint32_t *status, cudaStream_t st);
 // Split factor, scratch need (FP32 parts) and modelled cost
 // of the pair kernel for an output with few tiles and a long contraction; split 1 = no split.
 void tc2_split_plan(int M, int N, int K, size_t ws_bytes, int *split_out, size_t *ws_needed, double *cost_out);

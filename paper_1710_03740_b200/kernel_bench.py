@@ -328,7 +328,7 @@ def main():
     g.add_argument("--no-workspace", action="store_true", help="do not offer a split-K scratch buffer")
     g.add_argument("--sustain", type=float, default=0.0, metavar="SECONDS",
                    help="also time a loop of at least this many seconds with clocks and power sampled")
-    g.add_argument("--kernel", default="auto", choices=["auto", "tc", "pair"],
+    g.add_argument("--kernel", default="auto", choices=["auto", "tc", "pair", "pair512"],
                    help="auto: the library's choice; tc: single-CTA 128x256 tiles; pair: cta_group::2 256x256 tiles")
     u = sub.add_parser("update")
     u.add_argument("--params", type=int, default=150994944)
@@ -358,7 +358,7 @@ def main():
                   else inputs.GEMM_SWEEP + [inputs.LSTM_GATE, inputs.LSTM_PROJ])
         for (M, N, K) in shapes:
             for op in args.op:
-                flags = {"auto": 0, "tc": mpt.GEMM_FORCE_TC, "pair": mpt.GEMM_FORCE_PAIR}[args.kernel]
+                flags = {"auto": 0, "tc": mpt.GEMM_FORCE_TC, "pair": mpt.GEMM_FORCE_PAIR, "pair512": mpt.GEMM_FORCE_PAIR512}[args.kernel]
                 res = bench_gemm(M, N, K, op, args.iters, args.compare_library, flags, not args.no_workspace, args.sustain)
                 res["kernel_choice"] = args.kernel
                 print(json.dumps(res), flush=True)

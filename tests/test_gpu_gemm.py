@@ -92,7 +92,7 @@ def test_simt_gemm_relu_mask_flag():
 
 def _check_tc(op, M, N, K, flags=0, mask=None, seed=21, scale=None, want_flag=False, kernel="tc", workspace=False):
     from paper_1710_03740_b200 import binding as b
-    force = {"pair": b.GEMM_FORCE_PAIR, "tc": b.GEMM_FORCE_TC, "auto": 0}[kernel]
+    force = {"pair": b.GEMM_FORCE_PAIR, "tc": b.GEMM_FORCE_TC, "auto": 0, "pair512": b.GEMM_FORCE_PAIR512}[kernel]
     sa = sb = scale
     A, B = inputs.gemm_operands(op, M, N, K, seed=seed, scale_a=sa, scale_b=sb)
     ref, ex, ab = mpo.gemm_f16(op, A, B, relu=bool(flags & b.GEMM_RELU), mask=mask, want_exact=True)
@@ -127,6 +127,38 @@ def test_tc_gemm_parity(op, M, N, K):
 @pytest.mark.parametrize("M,N,K", PAIR_SHAPES)
 def test_pair_gemm_parity(op, M, N, K):
     _check_tc(op, M, N, K, kernel="pair")
+
+
+PAIR512_SHAPES = [(256, 512, 64), (256, 512, 448), (512, 1536, 128), (256, 768, 72), (392, 1080, 136), (264, 264, 200),
+                  (64, 16, 512), (8, 8, 8), (1280, 2048, 1024), (256, 256, 320)]
+
+
+@pytest.mark.parametrize("op", [0, 1, 2])
+@pytest.mark.parametrize("M,N,K", PAIR512_SHAPES)
+def test_pair512_gemm_parity(op, M, N, K):
+    """CTA-pair kernel with 256x512 tiles: whole tiles, ragged right edges wider and narrower than
+    one accumulator, ragged M and K, and shapes smaller than a tile."""
+    _check_tc(op, M, N, K, kernel="pair512")
+
+
+@pytest.mark.parametrize("op", [0, 1, 2])
+def test_pair512_many_tiles_halves_relu_mask_flag(op):
+    """More tiles than clusters (the ring, the accumulator hand-over and the K direction all
+    alternate several times), a last round cut into 256-column halves, ReLU / mask / overflow flag
+    through the two epilogue sets, and identical bits on a rerun."""
+    from paper_1710_03740_b200 import binding as b
+    M, N, K = 2304, 5120 + 256, 136            # 9 x 11 tiles: 74 whole tiles, 25 cut into halves
+    got, _, _, _ = _check_tc(op, M, N, K, kernel="pair512")
+    again, _, _, _ = _check_tc(op, M, N, K, kernel="pair512")
+    assert np.array_equal(got, again)
+    M, N, K = 512, 1024, 320
+    _check_tc(op, M, N, K, flags=b.GEMM_RELU, kernel="pair512")
+    mask = np.random.default_rng(9).standard_normal((M, N)).astype(np.float16)
+    _check_tc(op, M, N, K, mask=mask, kernel="pair512")
+    _, ref, flag, _ = _check_tc(op, M, N, K, scale=40.0, want_flag=True, kernel="pair512")
+    assert flag == int(((ref & 0x7FFF) >= 0x7C00).any()) == 1
+    _, _, flag, _ = _check_tc(op, M, N, K, want_flag=True, kernel="pair512")
+    assert flag == 0
 
 
 @pytest.mark.parametrize("kernel", ["tc", "pair"])
@@ -206,7 +238,7 @@ def test_random_ragged_shapes_all_kernels(op):
         N = int(rng.integers(1, 90)) * 8
         K = int(rng.choice([8, 24, 64, 72, 200, 520, 1032, 2056, 4104]))
         relu = bool(rng.integers(0, 2))
-        for kernel, ws in (("tc", False), ("pair", False), ("tc", True), ("pair", True), ("auto", True)):
+        for kernel, ws in (("tc", False), ("pair", False), ("pair512", False), ("tc", True), ("pair", True), ("auto", True)):
             if ws and b.mpt_gemm_workspace_bytes(op, M, N, K) == 0:
                 continue
             _check_tc(op, M, N, K, flags=b.GEMM_RELU if relu else 0, seed=int(rng.integers(1 << 30)), kernel=kernel,
