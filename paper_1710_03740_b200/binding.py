@@ -199,7 +199,11 @@ class Context:
             lib().mpt_destroy(self._ctx)
             self._ctx = None
 
-    __del__ = close
+    def __del__(self):
+        try:                # at interpreter shutdown the module globals may already be gone
+            self.close()
+        except Exception:
+            pass
 
     def set_master(self, layer, w32):
         w = np.ascontiguousarray(w32, dtype=np.float32)
