@@ -73,7 +73,7 @@ struct Unit {
     int mb, nb;      // tile coordinates
     int n_off;       // first column of the unit inside its tile (0 or 128)
     int width;       // 256 (whole tile) or 128 (half)
-    int tile, part;  // tile index and K part (split-K)
+    int part;        // K part (split-K)
     int kb0, kb1;    // k-blocks [kb0, kb1) of the contraction
 };
 
@@ -108,7 +108,6 @@ __device__ __forceinline__ Unit unit_of(const Params &p, int u, int nkb)
         w.n_off = (h & 1) * (TILE_N / 2);
         w.width = TILE_N / 2;
     }
-    w.tile = tile;
     tile_coords(p, tile, w.mb, w.nb);
     return w;
 }

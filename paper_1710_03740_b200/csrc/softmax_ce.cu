@@ -58,7 +58,6 @@ __global__ void __launch_bounds__(1024) k_softmax_ce(const uint16_t *__restrict_
         }
         // pass 1: read the row once, keep it on chip, running max
         float m = -INFINITY;
-        bool first_nan = false;
         if (VEC) {
             const uint4 *zv = (const uint4 *)zr;
             for (int i = tid; i < C8; i += nt) {
@@ -77,7 +76,6 @@ __global__ void __launch_bounds__(1024) k_softmax_ce(const uint16_t *__restrict_
             if (CACHE) srow[j] = h;
             m = fmaxf(m, hbits2f(h));
         }
-        (void)first_nan;
         m = block_reduce(m, true, red);   // also orders the srow writes before the reads below
 
         // pass 2: sum of exponentials in FP32
