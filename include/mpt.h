@@ -300,7 +300,9 @@ int mpt_gemm_f16(int op, int M, int N, int K, const uint16_t *A_dev, int lda, co
 /* The same product with a caller-provided scratch buffer that allows the contraction to be
  * split (section 3.3 arithmetic unchanged except for the order of the FP32 additions: the
  * parts are added in ascending order by a second kernel, so results stay run-to-run
- * identical).  Outputs with few tiles and a long contraction (for instance 2048 x 1024 with
+ * identical).  Large products use the scratch too: the tiles left over for a last, partly
+ * filled round of the CTA-pair kernel are split along K so that the round takes a fraction of a
+ * tile's time.  Outputs with few tiles and a long contraction (for instance 2048 x 1024 with
  * K = 8192) otherwise leave most SMs idle.  mpt_gemm_workspace_bytes returns the scratch size
  * the library would like for a shape (0 when it would not split); a smaller or null buffer
  * simply disables or narrows the split.  splitk_ws_dev must be 16-byte aligned. */

@@ -327,6 +327,8 @@ __global__ void __launch_bounds__(256) k_splitk_reduce(const float *__restrict__
     if (nonfinite_flag && __any_sync(0xFFFFFFFFu, bad) && (threadIdx.x & 31) == 0) atomicOr(nonfinite_flag, 1u);
 }
 
+thread_local int g_last_gemm_launches = 1;
+
 cudaError_t launch_splitk_reduce(const float *partial, int split_k, int M, int N, int ldp, uint16_t *C, int ldc, bool relu,
                                  const uint16_t *mask, int ldmask, uint32_t *nonfinite_flag, cudaStream_t st)
 {
@@ -335,6 +337,7 @@ cudaError_t launch_splitk_reduce(const float *partial, int split_k, int M, int N
     if (blocks > 148 * 16) blocks = 148 * 16;
     k_splitk_reduce<<<(unsigned)blocks, 256, 0, st>>>(partial, split_k, M, N, ldp, C, ldc, relu ? 1 : 0, mask, ldmask,
                                                       nonfinite_flag);
+    g_last_gemm_launches = 2;
     return cudaGetLastError();
 }
 
@@ -471,7 +474,10 @@ void tc_gemm_plan(int M, int N, int K, size_t ws_bytes, int *bn_out, int *split_
 bool tc_choose_pair(int M, int N, int K, size_t ws_bytes, size_t *ws_needed)
 {
     if (ws_needed) *ws_needed = 0;
-    if (tc2_gemm_preferred(M, N, K)) return true;
+    if (tc2_gemm_preferred(M, N, K)) {
+        if (ws_needed) *ws_needed = tc2_tail_ws_bytes(M, N, K);     // scratch for the split tail of the last round
+        return true;
+    }
     int bn, s1, s2;
     size_t need1 = 0, need2 = 0;
     double c1 = 0.0, c2 = 0.0;
@@ -491,6 +497,7 @@ cudaError_t launch_gemm_tc(int op, int M, int N, int K, const uint16_t *A, int l
                            uint16_t *C, int ldc, bool relu, const uint16_t *mask, int ldmask, uint32_t *nonfinite_flag,
                            uint32_t *status, cudaStream_t st, float *splitk_ws, size_t splitk_ws_bytes, const LstmEpi *lstm)
 {
+    g_last_gemm_launches = 1;
     TcParams p;
     p.lstm = LstmEpi{};
     if (lstm) {   // gate epilogue: forward products only, never split (the epilogue needs the whole sum)

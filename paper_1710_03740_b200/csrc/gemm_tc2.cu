@@ -66,6 +66,12 @@ struct Params {
     int split_k;
     float *partial;
     int ldp;
+    // tail split: the tiles left over for a last, partly filled round are cut into tail_split units
+    // along K (full-width instructions, unlike the half-width units, which take as long as whole
+    // ones); unit h of the tail leaves its raw FP32 accumulator in tail_partial[h][256][256] and
+    // k_tail_reduce finishes those tiles.  tail_split == 1: off (half-width units instead).
+    int tail_split;
+    float *tail_partial;
     LstmEpi lstm;                    // read only by the LSTM instantiation of the kernel
 };
 
@@ -75,6 +81,7 @@ struct Unit {
     int width;       // 256 (whole tile) or 128 (half)
     int part;        // K part (split-K)
     int kb0, kb1;    // k-blocks [kb0, kb1) of the contraction
+    int tail_slot;   // >= 0: unit of the split tail, index of its 256x256 FP32 block; -1 otherwise
 };
 
 __device__ __forceinline__ void tile_coords(const Params &p, int tile, int &mb, int &nb)
@@ -97,11 +104,19 @@ __device__ __forceinline__ Unit unit_of(const Params &p, int u, int nkb)
     w.part = 0;
     w.kb0 = 0;
     w.kb1 = nkb;
+    w.tail_slot = -1;
     if (p.split_k > 1) {            // parts of one tile are neighbouring units: they run side by side
         tile = u / p.split_k;
         w.part = u - tile * p.split_k;
         w.kb0 = (int)(((long long)nkb * w.part) / p.split_k);
         w.kb1 = (int)(((long long)nkb * (w.part + 1)) / p.split_k);
+    } else if (u >= p.full_units && p.tail_split > 1) {
+        const int h = u - p.full_units;
+        tile = p.full_units + h / p.tail_split;
+        w.part = h - (tile - p.full_units) * p.tail_split;
+        w.kb0 = (int)(((long long)nkb * w.part) / p.tail_split);
+        w.kb1 = (int)(((long long)nkb * (w.part + 1)) / p.tail_split);
+        w.tail_slot = h;
     } else if (u >= p.full_units) {
         const int h = u - p.full_units;
         tile = p.full_units + (h >> 1);
@@ -292,6 +307,23 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
                 const int set = (warp - 2) >> 2, nch = w.width / 64;       // this set's half of the unit's columns
                 epilogue_lstm_tile(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * TILE_N + set * nch * 32), nch,
                                    w.nb * TILE_N + w.n_off + set * nch * 32, p.N, row, row_ok, crow, p.lstm);
+            } else if (w.tail_slot >= 0) {
+                // unit of the split tail: the raw 256x256 FP32 block of this part (all rows, all columns)
+                float *prow = p.tail_partial + (size_t)w.tail_slot * (2 * CTA_M * TILE_N) +
+                              (size_t)((int)rank * CTA_M + q * 32 + lane) * TILE_N;
+                constexpr int NCH = TILE_N / 32 / EpiCfg<LSTM || WIDE>::SETS;
+                const int set = (warp - 2) >> 2;
+#pragma unroll 1
+                for (int c = set * NCH; c < (set + 1) * NCH; c++) {
+                    uint32_t r[32];
+                    tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * TILE_N + c * 32), r);
+                    tc_wait_ld();
+                    float4 *dst = (float4 *)(prow + c * 32);
+#pragma unroll
+                    for (int v = 0; v < 8; v++)
+                        __stcg(dst + v, make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
+                                                    __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3])));
+                }
             } else if (p.split_k > 1) {
                 // raw FP32 partial sums of this unit; ldp is a multiple of 32, so a started chunk is whole
                 float *prow = p.partial + ((size_t)w.part * p.M + row) * p.ldp;
@@ -340,6 +372,45 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
     }
 }
 
+// Finishes the tiles of the split tail: C = epilogue(part 0 + part 1 + ...) with the parts added in
+// ascending order (one rounding per add), eight columns per thread.
+__global__ void __launch_bounds__(256) k_tail_reduce(const Params p, int first_tile, int n_tiles)
+{
+    constexpr int TILE_ELEMS = 2 * CTA_M * TILE_N;
+    const size_t total = (size_t)n_tiles * (2 * CTA_M) * (TILE_N / 8);
+    bool bad = false;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const int ti = (int)(i / ((2 * CTA_M) * (TILE_N / 8)));
+        const int rem = (int)(i - (size_t)ti * ((2 * CTA_M) * (TILE_N / 8)));
+        const int r = rem / (TILE_N / 8), g = rem - r * (TILE_N / 8);
+        int mb, nb;
+        tile_coords(p, first_tile + ti, mb, nb);
+        const int row = mb * (2 * CTA_M) + r, col = nb * TILE_N + g * 8;
+        if (row >= p.M || col >= p.N) continue;
+        const float *src = p.tail_partial + (size_t)ti * p.tail_split * TILE_ELEMS + (size_t)r * TILE_N + g * 8;
+        float4 a = __ldcg((const float4 *)src), b = __ldcg((const float4 *)(src + 4));
+        for (int sp = 1; sp < p.tail_split; sp++) {
+            const float *q = src + (size_t)sp * TILE_ELEMS;
+            const float4 c = __ldcg((const float4 *)q), d = __ldcg((const float4 *)(q + 4));
+            a.x = __fadd_rn(a.x, c.x); a.y = __fadd_rn(a.y, c.y); a.z = __fadd_rn(a.z, c.z); a.w = __fadd_rn(a.w, c.w);
+            b.x = __fadd_rn(b.x, d.x); b.y = __fadd_rn(b.y, d.y); b.z = __fadd_rn(b.z, d.z); b.w = __fadd_rn(b.w, d.w);
+        }
+        const float v[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+        for (int e = 0; e < 8 && col + e < p.N; e++) {
+            float s = v[e];
+            if (p.relu) s = (s > 0.0f || s != s) ? s : 0.0f;
+            uint32_t h = (uint32_t)__half_as_ushort(__float2half_rn(s));
+            if (p.mask) {
+                const uint32_t mh = p.mask[(size_t)row * p.ldmask + col + e];
+                if (!((mh & 0x8000u) == 0 && mh != 0 && mh <= 0x7C00u)) h = 0;
+            }
+            bad |= (h & 0x7C00u) == 0x7C00u;
+            p.C[(size_t)row * p.ldc + col + e] = (uint16_t)h;
+        }
+    }
+    if (p.nonfinite_flag && __any_sync(0xFFFFFFFFu, bad) && (threadIdx.x & 31) == 0) atomicOr(p.nonfinite_flag, 1u);
+}
+
 template <bool A_MN, bool B_MN, bool LSTM = false, bool WIDE = false>
 static cudaError_t launch_variant(const CUtensorMap &ta, const CUtensorMap &tb, const CUtensorMap &tbh, Params p,
                                   cudaStream_t st)
@@ -379,16 +450,39 @@ static cudaError_t launch_variant(const CUtensorMap &ta, const CUtensorMap &tb, 
     if (p.split_k > 1) {
         p.full_units = tiles * p.split_k;
         p.num_units = tiles * p.split_k;
+    } else if (p.tail_split > 1 && tiles > max_pairs && rest > 0 && 2 * rest <= max_pairs) {
+        // the launcher passed the scratch size in tail_split's place: units of 256x256 floats it holds
+        const int nkb = (p.K + BLOCK_K - 1) / BLOCK_K;
+        int split = max_pairs / rest;
+        if (split > 8) split = 8;
+        while (split > 1 && (nkb / split < 8 || (long)rest * split > (long)p.tail_split)) split--;
+        p.tail_split = split;
+        if (split > 1) {
+            p.full_units = full;
+            p.num_units = full + rest * split;
+        } else {
+            p.full_units = full;
+            p.num_units = full + 2 * rest;
+        }
     } else if (rest > 0 && 2 * rest <= max_pairs) {
+        p.tail_split = 1;
         p.full_units = full;
         p.num_units = full + 2 * rest;
     } else {
+        p.tail_split = 1;
         p.full_units = tiles;
         p.num_units = tiles;
     }
     const int grid_pairs = p.num_units < max_pairs ? p.num_units : max_pairs;
     cfg.gridDim = dim3(2 * grid_pairs, 1, 1);
-    return cudaLaunchKernelEx(&cfg, kern, ta, tb, tbh, p);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, ta, tb, tbh, p);
+    if (e != cudaSuccess || p.split_k > 1 || p.tail_split <= 1) return e;
+    const size_t work = (size_t)rest * (2 * CTA_M) * (TILE_N / 8);
+    size_t blocks = (work + 255) / 256;
+    if (blocks > 148 * 8) blocks = 148 * 8;
+    k_tail_reduce<<<(unsigned)blocks, 256, 0, st>>>(p, full, rest);
+    g_last_gemm_launches = 2;
+    return cudaGetLastError();
 }
 
 }  // namespace pair
@@ -401,6 +495,21 @@ bool tc2_gemm_preferred(int M, int N, int K)
     (void)K;
     const long tiles = (long)((M + 255) / 256) * ((N + 255) / 256);
     return M >= 256 && N >= 256 && tiles >= 48;
+}
+
+// Scratch the pair kernel would like for the split tail of a large product: one 256x256 FP32 block
+// per unit of the last round (at most 74), when the tiles do not fill the last round.
+size_t tc2_tail_ws_bytes(int M, int N, int K)
+{
+    const long tiles = (long)((M + 255) / 256) * ((N + 255) / 256);
+    const int nkb = (K + pair::BLOCK_K - 1) / pair::BLOCK_K;
+    if (tiles <= 74 || nkb < 16) return 0;
+    const long rest = tiles % 74;
+    if (rest == 0 || 2 * rest > 74) return 0;
+    long split = 74 / rest;
+    if (split > 8) split = 8;
+    while (split > 1 && nkb / split < 8) split--;
+    return split > 1 ? (size_t)(rest * split) * 256 * 256 * sizeof(float) : 0;
 }
 
 // Split factor for the pair kernel on outputs with few 256x256 tiles and a long contraction.
@@ -438,6 +547,7 @@ cudaError_t launch_gemm_tc2(int op, int M, int N, int K, const uint16_t *A, int 
                             uint32_t *status, cudaStream_t st, const LstmEpi *lstm, void *splitk_ws, size_t splitk_ws_bytes)
 {
     using namespace pair;
+    g_last_gemm_launches = 1;
     CUtensorMap ta, tb, tbh;
     bool ok;
     if (op == MPT_OP_WGRAD) ok = tc_encode_map(&ta, A, (uint64_t)K, (uint64_t)M, (uint64_t)lda, 64, BLOCK_K);
@@ -465,12 +575,21 @@ cudaError_t launch_gemm_tc2(int op, int M, int N, int K, const uint16_t *A, int 
     p.split_k = 1;
     p.partial = nullptr;
     p.ldp = (N + 31) / 32 * 32;
+    p.tail_split = 1;
+    p.tail_partial = nullptr;
     if (!lstm && splitk_ws && (((uintptr_t)splitk_ws) & 15) == 0) {
         int split = 1;
         tc2_split_plan(M, N, K, splitk_ws_bytes, &split, nullptr, nullptr);
         if (split > 1) {
             p.split_k = split;
             p.partial = (float *)splitk_ws;
+        } else {
+            // scratch for the split tail: launch_variant turns the capacity (in 256x256 FP32 blocks) into a split
+            const size_t blocks = splitk_ws_bytes / ((size_t)2 * CTA_M * TILE_N * sizeof(float));
+            if (blocks >= 2) {
+                p.tail_split = (int)(blocks > 1024 ? 1024 : blocks);
+                p.tail_partial = (float *)splitk_ws;
+            }
         }
     }
     p.lstm = LstmEpi{};

@@ -346,6 +346,7 @@ cudaError_t launch_gemm_tc3(int op, int M, int N, int K, const uint16_t *A, int 
                             uint32_t *status, cudaStream_t st)
 {
     using namespace pair512;
+    g_last_gemm_launches = 1;
     CUtensorMap ta, tb;
     bool ok;
     if (op == MPT_OP_WGRAD) ok = tc_encode_map(&ta, A, (uint64_t)K, (uint64_t)M, (uint64_t)lda, 64, BLOCK_K);

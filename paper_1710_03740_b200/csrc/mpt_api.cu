@@ -260,9 +260,11 @@ int gemm(mpt_ctx *c, int op, int M, int N, int K, const uint16_t *A, int lda, co
         else
             e = launch_gemm_tc(op, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite,
                                c->status + ST_KERNEL_ERR, c->stream, c->splitk_ws, c->plan.splitk_bytes);
-    } else
+        c->launches += g_last_gemm_launches;
+    } else {
         e = launch_gemm_simt(op, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite, c->stream);
-    c->launches++;
+        c->launches++;
+    }
     if (e != cudaSuccess) return cuda_fail(c, e, "gemm launch");
     return MPT_OK;
 }

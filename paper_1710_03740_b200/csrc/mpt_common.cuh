@@ -127,6 +127,10 @@ void tc_gemm_plan(int M, int N, int K, size_t ws_bytes, int *bn_out, int *split_
 // split contraction), false = single-CTA kernel; ws_needed = scratch the choice would like.
 bool tc_choose_pair(int M, int N, int K, size_t ws_bytes, size_t *ws_needed);
 
+// Number of kernels the last product launcher called on this host thread enqueued (the product
+// kernel plus, for a split contraction or a split tail, the reduce kernel): bookkeeping only.
+extern thread_local int g_last_gemm_launches;
+
 // CTA-pair variant (tcgen05 cta_group::2, 256x256 tiles); same operand rules as launch_gemm_tc.
 bool tc2_gemm_preferred(int M, int N, int K);
 cudaError_t launch_gemm_tc2(int op, int M, int N, int K, const uint16_t *A, int lda, const uint16_t *B, int ldb,
@@ -142,6 +146,7 @@ cudaError_t launch_splitk_reduce(const float *partial, int split_k, int M, int N
 cudaError_t launch_gemm_tc3(int op, int M, int N, int K, const uint16_t *A, int lda, const uint16_t *B, int ldb,
                             uint16_t *C, int ldc, bool relu, const uint16_t *mask, int ldmask,
                             uint32_t *nonfinite_flag, uint32_t *status, cudaStream_t st);
+size_t tc2_tail_ws_bytes(int M, int N, int K);
 // Split factor, scratch need (FP32 parts) and modelled cost
 // of the pair kernel for an output with few tiles and a long contraction; split 1 = no split.
 void tc2_split_plan(int M, int N, int K, size_t ws_bytes, int *split_out, size_t *ws_needed, double *cost_out);

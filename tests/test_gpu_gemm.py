@@ -90,12 +90,23 @@ def test_simt_gemm_relu_mask_flag():
     assert flag == 1 and (~np.isfinite(ref.view(np.float16).astype(np.float32))).any()
 
 
+_ORACLE_CACHE = {}
+
+
 def _check_tc(op, M, N, K, flags=0, mask=None, seed=21, scale=None, want_flag=False, kernel="tc", workspace=False):
     from paper_1710_03740_b200 import binding as b
     force = {"pair": b.GEMM_FORCE_PAIR, "tc": b.GEMM_FORCE_TC, "auto": 0, "pair512": b.GEMM_FORCE_PAIR512}[kernel]
     sa = sb = scale
-    A, B = inputs.gemm_operands(op, M, N, K, seed=seed, scale_a=sa, scale_b=sb)
-    ref, ex, ab = mpo.gemm_f16(op, A, B, relu=bool(flags & b.GEMM_RELU), mask=mask, want_exact=True)
+    key = (op, M, N, K, seed, scale, bool(flags & b.GEMM_RELU))
+    if mask is None and key in _ORACLE_CACHE:        # the oracle is slow: keep its answer for repeated inputs
+        A, B, ref, ex, ab = _ORACLE_CACHE[key]
+    else:
+        A, B = inputs.gemm_operands(op, M, N, K, seed=seed, scale_a=sa, scale_b=sb)
+        ref, ex, ab = mpo.gemm_f16(op, A, B, relu=bool(flags & b.GEMM_RELU), mask=mask, want_exact=True)
+        if mask is None:
+            if len(_ORACLE_CACHE) >= 4:
+                _ORACLE_CACHE.pop(next(iter(_ORACLE_CACHE)))
+            _ORACLE_CACHE[key] = (A, B, ref, ex, ab)
     got, flag = run_gemm(op, A, B, M, N, K, flags=flags | force, mask=mask,
                          pad=(8 if (M * N) % 3 == 0 else 0), want_flag=want_flag, workspace=workspace)
     ok, stats = gemm_accept(got, ref, K=K, absdot=ab)
@@ -220,6 +231,30 @@ def test_pair_kernel_split_k(op, M, N, K):
         assert np.array_equal(got, again)
     auto, _, _, _ = _check_tc(op, M, N, K, workspace=True, kernel="auto")
     if not big:
+        _check_tc(op, M, N, K, flags=b.GEMM_RELU, workspace=True, kernel="pair")
+        mask = np.random.default_rng(8).standard_normal((M, N)).astype(np.float16)
+        _check_tc(op, M, N, K, mask=mask, workspace=True, kernel="pair")
+        _, ref, flag, _ = _check_tc(op, M, N, K, scale=30.0, want_flag=True, workspace=True, kernel="pair")
+        assert flag == int(((ref & 0x7FFF) >= 0x7C00).any()) == 1
+
+
+@pytest.mark.parametrize("op", [0, 1, 2])
+@pytest.mark.parametrize("M,N,K,split", [(2304, 3072, 1024, 2), (1280, 4000, 4096, 8), (2304, 3000, 1160, 2)])
+def test_pair_kernel_split_tail(op, M, N, K, split):
+    """More 256x256 tiles than clusters with a partly filled last round: with a scratch buffer the
+    left-over tiles are cut along K (34 tiles in two parts, 6 tiles in eight parts, a ragged right
+    edge) and finished by the tail reduce kernel.  Same acceptance rule, identical bits on a rerun,
+    ReLU / mask / overflow flag through the tail reduce, and the automatic choice takes the same path."""
+    from paper_1710_03740_b200 import binding as b
+    assert b.mpt_gemm_workspace_bytes(op, M, N, K) >= split * 256 * 256 * 4
+    got, _, _, _ = _check_tc(op, M, N, K, workspace=True, kernel="pair")
+    again, _, _, _ = _check_tc(op, M, N, K, workspace=True, kernel="pair")
+    assert np.array_equal(got, again)
+    auto, _, _, _ = _check_tc(op, M, N, K, workspace=True, kernel="auto")
+    assert np.array_equal(got, auto)
+    nows, _, _, _ = _check_tc(op, M, N, K, workspace=False, kernel="pair")       # half-width units instead
+    assert (got != nows).mean() < 0.2                                            # same values up to summation order
+    if split == 2 and N == 3072:
         _check_tc(op, M, N, K, flags=b.GEMM_RELU, workspace=True, kernel="pair")
         mask = np.random.default_rng(8).standard_normal((M, N)).astype(np.float16)
         _check_tc(op, M, N, K, mask=mask, workspace=True, kernel="pair")
