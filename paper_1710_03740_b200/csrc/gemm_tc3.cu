@@ -235,15 +235,19 @@ k_gemm_tc3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
                     tc_fence_after();
                     const uint32_t alo = a_lo0 + s * (uint32_t)(STAGE_BYTES >> 4);
                     const uint32_t blo = b_lo0 + s * (uint32_t)(STAGE_BYTES >> 4);
+                    // the four k-steps of one accumulator back to back, then those of the other
 #pragma unroll
-                    for (int k = 0; k < BLOCK_K / UMMA_K; k++) {
-                        const uint64_t ad = desc_join(alo + k * KSTEP_A, a_hi);
-                        tc_mma_f16_pair(tmem_base, ad, desc_join(blo + k * KSTEP_B, b_hi), idesc, acc);
-                        if (two)
-                            tc_mma_f16_pair(tmem_base + ACC_N, ad, desc_join(blo + (uint32_t)(B_STAGE_BYTES >> 4) + k * KSTEP_B, b_hi),
-                                            idesc, acc);
-                        acc = 1;
+                    for (int k = 0; k < BLOCK_K / UMMA_K; k++)
+                        tc_mma_f16_pair(tmem_base, desc_join(alo + k * KSTEP_A, a_hi), desc_join(blo + k * KSTEP_B, b_hi), idesc,
+                                        k == 0 ? acc : 1u);
+                    if (two) {
+#pragma unroll
+                        for (int k = 0; k < BLOCK_K / UMMA_K; k++)
+                            tc_mma_f16_pair(tmem_base + ACC_N, desc_join(alo + k * KSTEP_A, a_hi),
+                                            desc_join(blo + (uint32_t)(B_STAGE_BYTES >> 4) + k * KSTEP_B, b_hi), idesc,
+                                            k == 0 ? acc : 1u);
                     }
+                    acc = 1;
                     tc_commit_pair(empty_bar(s), 3);        // both CTAs' producers may refill stage s
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
