@@ -252,6 +252,68 @@ def bench_lstm(name, iters, steps=None):
     return out
 
 
+def bench_steplike(steps, dense):
+    """The 26 products and the master update of the large-MLP step as stateless calls, alternating
+    like the training step, with this library's kernels and with torch.matmul (cuBLAS) on the same
+    operands: ReLU-like operands (half zeros) unless `dense`.  Context for the power-capped regime:
+    what a product leaves behind (clock state) shows in the update that follows it."""
+    B_, H, Cn = 4096, 12288, 32000
+    g = torch.Generator(device="cuda").manual_seed(5)
+    rnd = lambda *shape: torch.randn(shape, device="cuda", generator=g)  # noqa: E731
+    act = (lambda t: t) if dense else torch.relu
+    x = [act(rnd(B_, H)).half() for _ in range(9)]
+    W = [(rnd(H, H) * 0.01).half() for _ in range(8)] + [(rnd(Cn, H) * 0.01).half()]
+    keep = (lambda t: t) if dense else (lambda t: t * (torch.rand(t.shape, device="cuda", generator=g) > 0.5))
+    dz = [keep(rnd(B_, H)).half() for _ in range(8)] + [(rnd(B_, Cn) * 1e-3).half()]
+    n = sum(w.numel() for w in W)
+    g16 = rnd(n).half(); w32 = rnd(n); v = torch.zeros(n, device="cuda"); w16 = torch.empty(n, dtype=torch.half, device="cuda")
+    flags = torch.zeros(2, dtype=torch.int32, device="cuda")
+    st = torch.zeros(16, dtype=torch.int32, device="cuda")
+    ws = torch.zeros(20 * 1024 * 1024 // 4, device="cuda")
+    outs = {}
+
+    def out(kind, l, rows, cols):
+        return outs.setdefault((kind, l), torch.empty((rows, cols), dtype=torch.half, device="cuda"))
+
+    def ours():
+        for l in range(9):
+            N = W[l].shape[0]
+            mpt.mpt_gemm_f16_ws(0, B_, N, H, x[l], H, W[l], H, out("f", l, B_, N), N, 0, None, 0, None, st, ws)
+        for l in range(8, -1, -1):
+            N = W[l].shape[0]
+            mpt.mpt_gemm_f16_ws(2, N, H, B_, dz[l], N, x[l], H, out("w", l, N, H), H, 0, None, 0, None, st, ws)
+            if l > 0:
+                mpt.mpt_gemm_f16_ws(1, B_, H, N, dz[l], N, W[l], H, out("d", l, B_, H), H, 0, None, 0, None, st, ws)
+
+    def library():
+        for l in range(9):
+            torch.matmul(x[l], W[l].t())
+        for l in range(8, -1, -1):
+            torch.matmul(dz[l].t(), x[l])
+            if l > 0:
+                torch.matmul(dz[l], W[l])
+
+    upd = lambda: mpt.mpt_update_flat(g16, w32, v, w16, n, 1.0 / 512, 1e-4, 0.9, True, False, flags)  # noqa: E731
+
+    def run(products):
+        tg = tu = 0.0
+        for s_ in range(steps + 3):
+            e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+            e[0].record(); products(); e[1].record(); upd(); e[2].record()
+            torch.cuda.synchronize()
+            if s_ >= 3:
+                tg += e[0].elapsed_time(e[1]); tu += e[1].elapsed_time(e[2])
+        return tg / steps, tu / steps
+
+    res = {"kernel": "steplike", "operands": "dense" if dense else "relu-like (half zeros)", "steps": steps, "rounds": []}
+    for _ in range(2):
+        a, b = run(ours), run(library)
+        res["rounds"].append({"ours_products_ms": a[0], "ours_update_ms": a[1], "library_products_ms": b[0],
+                              "update_after_library_ms": b[1]})
+    res["device_error"] = int(st[0])
+    return res
+
+
 def bench_softmax(B, Cn, iters, sustain_s=0.0):
     g = torch.Generator(device="cuda").manual_seed(4)
     z = (torch.randn((B, Cn), device="cuda", generator=g) * 3).half()
@@ -343,6 +405,9 @@ def main():
     s.add_argument("--classes", type=int, default=32000)
     s.add_argument("--iters", type=int, default=20)
     s.add_argument("--sustain", type=float, default=0.0)
+    sl = sub.add_parser("steplike")
+    sl.add_argument("--steps", type=int, default=10)
+    sl.add_argument("--dense", action="store_true", help="dense normal operands instead of ReLU-like ones")
     ls = sub.add_parser("lstm")
     ls.add_argument("--config", default="biglstm", choices=sorted(inputs.LSTM_CONFIGS))
     ls.add_argument("--steps", type=int, default=0, help="override the number of time steps")
@@ -362,6 +427,8 @@ def main():
                 res = bench_gemm(M, N, K, op, args.iters, args.compare_library, flags, not args.no_workspace, args.sustain)
                 res["kernel_choice"] = args.kernel
                 print(json.dumps(res), flush=True)
+    elif args.cmd == "steplike":
+        print(json.dumps(bench_steplike(args.steps, args.dense)), flush=True)
     elif args.cmd == "lstm":
         print(json.dumps(bench_lstm(args.config, args.iters, args.steps)), flush=True)
     elif args.cmd == "update":
