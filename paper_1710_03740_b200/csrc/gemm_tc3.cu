@@ -11,10 +11,12 @@
 // four warps, one accumulator each).
 //
 // Measured on B200 (4096x12288x12288, 1000 W cap): DRAM traffic 1.06 GB per launch against 1.24 GB,
-// L2->SM traffic 7.3 GB against 9.7 GB, tensor pipe 90 % of active cycles against 98 %; burst rate
-// 1415 against 1435 TFLOP/s, seconds-long rate level (1211-1218 both); inside the training step,
-// where the products alternate with the update pass, 6 % slower (28.8 against 27.2 ms per step).
-// It is therefore never chosen automatically: MPT_GEMM_FORCE_PAIR512 selects it.
+// L2->SM traffic 7.3 GB against 9.7 GB, tensor pipe 90 % of active cycles against 98 %.  With the
+// stores of the epilogue coalesced through shared memory: burst rate level (1440 TFLOP/s),
+// seconds-long rate 1225-1234 against 1212-1216 for K = 12288, 1160-1165 against 1200-1207 for
+// K = 4096 (the exposed epilogue weighs more on short tiles); used for the long-K products of the
+// training step it changes the step time by less than the run-to-run spread.  It is therefore
+// never chosen automatically: MPT_GEMM_FORCE_PAIR512 selects it.
 //
 // Roles in each CTA (320 threads): warp 0 TMA producer, warp 1 MMA issuer (leader CTA only; both
 // CTAs' warp 1 take part in the paired tensor-memory allocation), warps 2-9 epilogue.  Barriers:
@@ -47,7 +49,8 @@ static constexpr int STAGE_BYTES = A_STAGE_BYTES + 2 * B_STAGE_BYTES;
 static constexpr int MN_BOX_BYTES = 64 * BLOCK_K * 2;
 static constexpr int TMEM_COLS = 512;
 static constexpr int NUM_THREADS = 320;
-static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256;
+static constexpr int EPI_STAGE_BYTES = 32 * kEpiStagePitch;                 // per epilogue warp
+static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256 + 8 * EPI_STAGE_BYTES;
 
 // instruction descriptor: FP32 accumulate, operand majors, N = 256, M = 256
 __host__ __device__ constexpr uint32_t make_idesc(bool a_mn, bool b_mn)
@@ -269,21 +272,20 @@ k_gemm_tc3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
                 break;
             }
             tc_fence_after();
-            const int row = w.mb * (2 * CTA_M) + (int)rank * CTA_M + q * 32 + lane;
-            const bool row_ok = row < p.M;
-            uint16_t *crow = p.C + (size_t)row * p.ldc;
-            const uint16_t *mrow = p.mask ? p.mask + (size_t)row * p.ldmask : nullptr;
             bool bad = false;
             // 512-wide unit: set s drains accumulator s (8 chunks of 32 columns); 256-wide: 4 chunks each
             const int nch = w.width == TILE_N ? ACC_N / 32 : ACC_N / 64;
             const int cbase = w.width == TILE_N ? set * ACC_N : set * (ACC_N / 2);
+            const int row0 = w.mb * (2 * CTA_M) + (int)rank * CTA_M + q * 32;
+            uint8_t *stage = base_ptr + STAGES * STAGE_BYTES + 256 + (warp - 2) * EPI_STAGE_BYTES;
 #pragma unroll 1
             for (int c = 0; c < nch; c++) {
                 uint32_t r[32];
                 tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(cbase + c * 32), r);
                 tc_wait_ld();
                 const int col0 = w.col0 + cbase + c * 32;
-                if (row_ok && col0 < p.N) epilogue_store32(r, crow, mrow, col0, p.N, p.relu != 0, bad);
+                if (col0 < p.N)      // warp-uniform
+                    epilogue_store32_coalesced(r, stage, p.C, p.ldc, p.mask, p.ldmask, row0, col0, p.M, p.N, p.relu != 0, bad);
             }
             tc_fence_before();
             __syncwarp();

@@ -191,6 +191,71 @@ __device__ __forceinline__ void epilogue_store32(const uint32_t (&r)[32], uint16
     }
 }
 
+// The same epilogue for 32 consecutive accumulator columns of the 32 rows a warp owns, with the
+// stores coalesced: each lane rounds its row's 32 values and parks them in a 32 x 32 FP16 block of
+// shared memory (pitch 80 bytes: conflict-free for 16-byte accesses), then the warp writes the
+// block out eight rows at a time, four lanes per row, 16 bytes per lane - 64 contiguous bytes per
+// row instead of one 16-byte piece per row and instruction (a quarter of the memory transactions).
+// The ReLU-derivative mask is read the same way.  stage: 32 * 80 bytes of shared memory owned by
+// this warp.  row0: first of the warp's 32 rows; col0: a multiple of 32.
+static constexpr int kEpiStagePitch = 80;
+__device__ __forceinline__ void epilogue_store32_coalesced(const uint32_t (&r)[32], uint8_t *stage, uint16_t *C, int ldc,
+                                                           const uint16_t *mask, int ldmask, int row0, int col0, int M, int N,
+                                                           bool relu, bool &bad)
+{
+    const int lane = threadIdx.x & 31;
+    uint4 *mine = (uint4 *)(stage + lane * kEpiStagePitch);
+#pragma unroll
+    for (int g8 = 0; g8 < 4; g8++) {
+        uint32_t h[8];
+#pragma unroll
+        for (int e = 0; e < 8; e++) {
+            float s = __uint_as_float(r[g8 * 8 + e]);
+            if (relu) s = (s > 0.0f || s != s) ? s : 0.0f;
+            h[e] = (uint32_t)__half_as_ushort(__float2half_rn(s));
+        }
+        mine[g8] = make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), h[4] | (h[5] << 16), h[6] | (h[7] << 16));
+    }
+    __syncwarp();
+    const int piece = lane & 3, col = col0 + piece * 8;
+#pragma unroll
+    for (int it = 0; it < 4; it++) {
+        const int rr = it * 8 + (lane >> 2), row = row0 + rr;
+        if (row < M && col < N) {
+            const uint4 v = *(const uint4 *)(stage + rr * kEpiStagePitch + piece * 16);
+            uint32_t w[4] = {v.x, v.y, v.z, v.w};
+            uint16_t *crow = C + (size_t)row * ldc;
+            if (col + 8 <= N) {
+                if (mask) {
+                    const uint4 mk = *(const uint4 *)(mask + (size_t)row * ldmask + col);
+                    const uint32_t mw[4] = {mk.x, mk.y, mk.z, mk.w};
+#pragma unroll
+                    for (int q = 0; q < 4; q++) {
+                        const uint32_t lo = mw[q] & 0xFFFFu, hi = mw[q] >> 16;
+                        // stored activation > 0  <=>  sign clear, non-zero, not NaN
+                        if (!((lo & 0x8000u) == 0 && lo != 0 && lo <= 0x7C00u)) w[q] &= 0xFFFF0000u;
+                        if (!((hi & 0x8000u) == 0 && hi != 0 && hi <= 0x7C00u)) w[q] &= 0x0000FFFFu;
+                    }
+                }
+#pragma unroll
+                for (int q = 0; q < 4; q++) bad |= ((w[q] & 0x7C00u) == 0x7C00u) || ((w[q] & 0x7C000000u) == 0x7C000000u);
+                *(uint4 *)(crow + col) = make_uint4(w[0], w[1], w[2], w[3]);
+            } else {
+                for (int e = 0; e < 8 && col + e < N; e++) {
+                    uint32_t x = (e & 1) ? (w[e >> 1] >> 16) : (w[e >> 1] & 0xFFFFu);
+                    if (mask) {
+                        const uint32_t mh = mask[(size_t)row * ldmask + col + e];
+                        if (!((mh & 0x8000u) == 0 && mh != 0 && mh <= 0x7C00u)) x = 0;
+                    }
+                    bad |= (x & 0x7C00u) == 0x7C00u;
+                    crow[col + e] = (uint16_t)x;
+                }
+            }
+        }
+    }
+    __syncwarp();    // the block may be overwritten by the next call
+}
+
 // LSTM gate arithmetic on FP32 values (sections 3.3, 4.6): one cell from its four pre-activations
 // (bias already added).  Returns the FP16 bit patterns of the gate activations in act[4], the new
 // cell state and the hidden state; h uses the STORED (rounded) cell state.
