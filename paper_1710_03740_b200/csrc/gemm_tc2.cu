@@ -456,6 +456,9 @@ static cudaError_t launch_variant(const CUtensorMap &ta, const CUtensorMap &tb, 
         int split = max_pairs / rest;
         if (split > 8) split = 8;
         while (split > 1 && (nkb / split < 8 || (long)rest * split > (long)p.tail_split)) split--;
+        // the reduce launch and the FP32 round trip cost about 10 us: worth it only when the split saves
+        // at least 96 k-blocks of main loop in the last round (4096^3 lost 5 % with it, K = 12288 gains)
+        if ((long)nkb * (split - 1) / split < 96) split = 1;
         p.tail_split = split;
         if (split > 1) {
             p.full_units = full;
@@ -509,6 +512,7 @@ size_t tc2_tail_ws_bytes(int M, int N, int K)
     long split = 74 / rest;
     if (split > 8) split = 8;
     while (split > 1 && nkb / split < 8) split--;
+    if ((long)nkb * (split - 1) / split < 96) split = 1;      // same rule as the launcher
     return split > 1 ? (size_t)(rest * split) * 256 * 256 * sizeof(float) : 0;
 }
 
