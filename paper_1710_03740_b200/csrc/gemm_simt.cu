@@ -19,6 +19,8 @@ __global__ void __launch_bounds__(256) k_gemm_simt(int M, int N, int K, const ui
                                                    int ldc, int relu, const uint16_t *__restrict__ mask, int ldmask,
                                                    uint32_t *nonfinite_flag)
 {
+    pdl_trigger();
+    pdl_wait();
     __shared__ float As[BK][BM + 4];
     __shared__ float Bs[BK][BN + 4];
     const int tid = threadIdx.x;
@@ -93,11 +95,11 @@ cudaError_t launch_gemm_simt(int op, int M, int N, int K, const uint16_t *A, int
     if (M <= 0 || N <= 0) return cudaSuccess;
     dim3 grid((N + BN - 1) / BN, (M + BM - 1) / BM);
     if (op == MPT_OP_FWD)
-        k_gemm_simt<false, false><<<grid, 256, 0, st>>>(M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite_flag);
+            { cudaError_t le_ = launch_pdl(k_gemm_simt<false, false>, dim3(grid), dim3(256), 0, st, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite_flag); if (le_ != cudaSuccess) return le_; }
     else if (op == MPT_OP_DGRAD)
-        k_gemm_simt<false, true><<<grid, 256, 0, st>>>(M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite_flag);
+            { cudaError_t le_ = launch_pdl(k_gemm_simt<false, true>, dim3(grid), dim3(256), 0, st, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite_flag); if (le_ != cudaSuccess) return le_; }
     else
-        k_gemm_simt<true, true><<<grid, 256, 0, st>>>(M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite_flag);
+            { cudaError_t le_ = launch_pdl(k_gemm_simt<true, true>, dim3(grid), dim3(256), 0, st, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite_flag); if (le_ != cudaSuccess) return le_; }
     return cudaGetLastError();
 }
 

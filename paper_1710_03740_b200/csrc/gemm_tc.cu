@@ -97,6 +97,7 @@ template <bool A_MN, bool B_MN, int BLOCK_N, bool LSTM = false, bool WIDE = fals
 __global__ void __launch_bounds__(EpiCfg<LSTM || WIDE>::THREADS, 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcParams p)
 {
+    pdl_trigger();
     constexpr int STAGES = TileCfg<BLOCK_N>::STAGES;
     constexpr int STAGE_BYTES = TileCfg<BLOCK_N>::STAGE_BYTES;
     constexpr int TMEM_COLS = TileCfg<BLOCK_N>::TMEM_COLS;
@@ -138,6 +139,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    pdl_wait();      // everything above ran beside the tail of the preceding kernel; global memory is touched below
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
@@ -298,6 +300,8 @@ __global__ void __launch_bounds__(256) k_splitk_reduce(const float *__restrict__
                                                        const uint16_t *__restrict__ mask, int ldmask,
                                                        uint32_t *nonfinite_flag)
 {
+    pdl_trigger();
+    pdl_wait();
     const int groups = (N + 7) / 8;
     const size_t total = (size_t)M * groups;
     bool bad = false;
@@ -335,8 +339,8 @@ cudaError_t launch_splitk_reduce(const float *partial, int split_k, int M, int N
     const size_t work = (size_t)M * ((N + 7) / 8);
     size_t blocks = (work + 255) / 256;
     if (blocks > 148 * 16) blocks = 148 * 16;
-    k_splitk_reduce<<<(unsigned)blocks, 256, 0, st>>>(partial, split_k, M, N, ldp, C, ldc, relu ? 1 : 0, mask, ldmask,
-                                                      nonfinite_flag);
+            { cudaError_t le_ = launch_pdl(k_splitk_reduce, dim3((unsigned)blocks), dim3(256), 0, st, partial, split_k, M, N, ldp, C, ldc, relu ? 1 : 0, mask, ldmask,
+                                                      nonfinite_flag); if (le_ != cudaSuccess) return le_; }
     g_last_gemm_launches = 2;
     return cudaGetLastError();
 }
@@ -402,7 +406,7 @@ static cudaError_t launch_variant(const CUtensorMap &ta, const CUtensorMap &tb, 
         if (e != cudaSuccess) return e;
         configured[dev] = true;
     }
-    kern<<<grid, EpiCfg<LSTM || WIDE>::THREADS, SMEM_BYTES, st>>>(ta, tb, p);
+            { cudaError_t le_ = launch_pdl(kern, dim3(grid), dim3(EpiCfg<LSTM || WIDE>::THREADS), SMEM_BYTES, st, ta, tb, p); if (le_ != cudaSuccess) return le_; }
     return cudaGetLastError();
 }
 

@@ -149,6 +149,7 @@ __global__ void __launch_bounds__(EpiCfg<LSTM || WIDE>::THREADS, 1)
 k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
            const __grid_constant__ CUtensorMap tmBh, const Params p)
 {
+    pdl_trigger();
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
@@ -185,6 +186,7 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
     cluster_sync_all();                            // the peer's barriers exist before anything signals them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    pdl_wait();      // everything above ran beside the tail of the preceding kernel; global memory is touched below
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer (both CTAs)
@@ -376,6 +378,8 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
 // ascending order (one rounding per add), eight columns per thread.
 __global__ void __launch_bounds__(256) k_tail_reduce(const Params p, int first_tile, int n_tiles)
 {
+    pdl_trigger();
+    pdl_wait();
     constexpr int TILE_ELEMS = 2 * CTA_M * TILE_N;
     const size_t total = (size_t)n_tiles * (2 * CTA_M) * (TILE_N / 8);
     bool bad = false;
@@ -420,11 +424,13 @@ static cudaError_t launch_variant(const CUtensorMap &ta, const CUtensorMap &tb, 
     const int dev = current_device_slot();
     if (dev < 0) return cudaErrorInvalidDevice;
     cudaLaunchConfig_t cfg = {};
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.blockDim = dim3(EpiCfg<LSTM || WIDE>::THREADS, 1, 1);
     cfg.dynamicSmemBytes = SMEM_BYTES;
     cfg.stream = st;
@@ -478,12 +484,13 @@ static cudaError_t launch_variant(const CUtensorMap &ta, const CUtensorMap &tb, 
     }
     const int grid_pairs = p.num_units < max_pairs ? p.num_units : max_pairs;
     cfg.gridDim = dim3(2 * grid_pairs, 1, 1);
+    cfg.numAttrs = 2;
     cudaError_t e = cudaLaunchKernelEx(&cfg, kern, ta, tb, tbh, p);
     if (e != cudaSuccess || p.split_k > 1 || p.tail_split <= 1) return e;
     const size_t work = (size_t)rest * (2 * CTA_M) * (TILE_N / 8);
     size_t blocks = (work + 255) / 256;
     if (blocks > 148 * 8) blocks = 148 * 8;
-    k_tail_reduce<<<(unsigned)blocks, 256, 0, st>>>(p, full, rest);
+            { cudaError_t le_ = launch_pdl(k_tail_reduce, dim3((unsigned)blocks), dim3(256), 0, st, p, full, rest); if (le_ != cudaSuccess) return le_; }
     g_last_gemm_launches = 2;
     return cudaGetLastError();
 }

@@ -117,6 +117,7 @@ template <bool A_MN, bool B_MN>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 k_gemm_tc3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const Params p)
 {
+    pdl_trigger();
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
@@ -153,6 +154,7 @@ k_gemm_tc3(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
     cluster_sync_all();                            // the peer's barriers exist before anything signals them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    pdl_wait();      // everything above ran beside the tail of the preceding kernel; global memory is touched below
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer (both CTAs)
@@ -313,11 +315,13 @@ static cudaError_t launch_variant(const CUtensorMap &ta, const CUtensorMap &tb, 
     const int dev = current_device_slot();
     if (dev < 0) return cudaErrorInvalidDevice;
     cudaLaunchConfig_t cfg = {};
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.blockDim = dim3(NUM_THREADS, 1, 1);
     cfg.dynamicSmemBytes = SMEM_BYTES;
     cfg.stream = st;
@@ -342,6 +346,7 @@ static cudaError_t launch_variant(const CUtensorMap &ta, const CUtensorMap &tb, 
     p.num_units = full + 2 * rest;
     const int grid_pairs = p.num_units < max_pairs ? p.num_units : max_pairs;
     cfg.gridDim = dim3(2 * grid_pairs, 1, 1);
+    cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, kern, ta, tb, p);
 }
 

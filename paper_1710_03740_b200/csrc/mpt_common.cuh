@@ -47,6 +47,33 @@ inline int current_device_slot()
     return d;
 }
 
+// Programmatic dependent launch.  Every kernel of the library starts with pdl_trigger() (its
+// dependents may be scheduled as soon as all of its CTAs have started) and executes pdl_wait()
+// before its first access to global memory (the wait returns when the preceding kernel in the
+// stream has completed and its writes are visible).  What runs before the wait - barrier set-up,
+// tensor-memory allocation, the launch itself - overlaps the tail of the preceding kernel.  In a
+// kernel launched without the attribute both are no-ops.
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// Launch with programmatic stream serialization (see above); kernels launched this way must call
+// pdl_wait() before touching global memory.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+
 __device__ __forceinline__ bool half_bits_nonfinite(uint32_t h) { return (h & 0x7C00u) == 0x7C00u; }
 __device__ __forceinline__ bool f32_nonfinite(float x)
 {

@@ -38,6 +38,8 @@ __global__ void __launch_bounds__(1024) k_softmax_ce(const uint16_t *__restrict_
                                                      uint16_t *dz, int lddz, float *__restrict__ row_loss,
                                                      uint32_t *bad_labels, const float *__restrict__ scale_dev)
 {
+    pdl_trigger();
+    pdl_wait();
     extern __shared__ __align__(16) uint16_t srow[];
     if (scale_dev) c = __fdiv_rn(*scale_dev, (float)B);
     __shared__ float red[32];
@@ -129,6 +131,8 @@ __global__ void __launch_bounds__(1024, VPT <= 4 ? 2 : 1) k_softmax_ce_reg(const
                                                          float *__restrict__ row_loss, uint32_t *bad_labels,
                                                          const float *__restrict__ scale_dev)
 {
+    pdl_trigger();
+    pdl_wait();
     __shared__ float red[32];
     if (scale_dev) c = __fdiv_rn(*scale_dev, (float)gridDim.x);   // one CTA per row: gridDim.x is the batch
     const int tid = threadIdx.x, nt = blockDim.x, row = blockIdx.x;
@@ -258,6 +262,8 @@ __global__ void __launch_bounds__(kSmaxThreads, 1) k_softmax_ce_bulk(const uint1
                                                                       float *__restrict__ row_loss, uint32_t *bad_labels,
                                                                       const float *__restrict__ scale_dev, uint32_t *kerr)
 {
+    pdl_trigger();
+    pdl_wait();
     extern __shared__ __align__(128) uint8_t rows_smem[];
     __shared__ float red[2][32];   // max and sum use different arrays; a row's last use is two barriers back
     __shared__ __align__(8) uint64_t bars[3];
@@ -373,6 +379,8 @@ __global__ void __launch_bounds__(kSmaxThreads, 1) k_softmax_ce_bulk(const uint1
 // loss = (float)( sum_i (double)row_loss[i] / B ), fixed reduction order.
 __global__ void __launch_bounds__(256) k_loss_mean(const float *__restrict__ row_loss, int B, float *loss)
 {
+    pdl_trigger();
+    pdl_wait();
     __shared__ double red[256];
     double acc = 0.0;
     for (int i = threadIdx.x; i < B; i += 256) acc += (double)row_loss[i];
@@ -395,7 +403,7 @@ static cudaError_t launch_variant(const uint16_t *z, int ldz, const int32_t *lab
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
     }
-    kern<<<grid, threads, smem, st>>>(z, ldz, labels, B, C, c, dz, lddz, row_loss, bad_labels, S_dev);
+            { cudaError_t le_ = launch_pdl(kern, dim3(grid), dim3(threads), smem, st, z, ldz, labels, B, C, c, dz, lddz, row_loss, bad_labels, S_dev); if (le_ != cudaSuccess) return le_; }
     return cudaGetLastError();
 }
 
@@ -425,12 +433,12 @@ cudaError_t launch_softmax_ce(const uint16_t *z, int ldz, const int32_t *labels,
             sms_dev[dev] = n > 0 ? n : 148;
         }
         const int grid = B < sms_dev[dev] ? B : sms_dev[dev];
-        kern<<<grid, kSmaxThreads, smem, st>>>(z, ldz, labels, B, C, c, dz, lddz, row_loss, bad_labels, S_dev, kerr);
+            { cudaError_t le_ = launch_pdl(kern, dim3(grid), dim3(kSmaxThreads), smem, st, z, ldz, labels, B, C, c, dz, lddz, row_loss, bad_labels, S_dev, kerr); if (le_ != cudaSuccess) return le_; }
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
         if (n_launches) *n_launches = 1;
         if (loss) {
-            k_loss_mean<<<1, 256, 0, st>>>(row_loss, B, loss);
+            { cudaError_t le_ = launch_pdl(k_loss_mean, dim3(1), dim3(256), 0, st, row_loss, B, loss); if (le_ != cudaSuccess) return le_; }
             if (n_launches) *n_launches = 2;
         }
         return cudaGetLastError();
@@ -444,16 +452,16 @@ cudaError_t launch_softmax_ce(const uint16_t *z, int ldz, const int32_t *labels,
         threads = ((threads + 31) / 32) * 32;
         if (threads < 32) threads = 32;
         switch (vpt) {
-            case 1: k_softmax_ce_reg<1><<<B, threads, 0, st>>>(z, ldz, labels, C, c, dz, lddz, row_loss, bad_labels, S_dev); break;
-            case 2: k_softmax_ce_reg<2><<<B, threads, 0, st>>>(z, ldz, labels, C, c, dz, lddz, row_loss, bad_labels, S_dev); break;
-            case 4: k_softmax_ce_reg<4><<<B, threads, 0, st>>>(z, ldz, labels, C, c, dz, lddz, row_loss, bad_labels, S_dev); break;
-            default: k_softmax_ce_reg<8><<<B, threads, 0, st>>>(z, ldz, labels, C, c, dz, lddz, row_loss, bad_labels, S_dev); break;
+            case 1: { cudaError_t le_ = launch_pdl(k_softmax_ce_reg<1>, dim3(B), dim3(threads), 0, st, z, ldz, labels, C, c, dz, lddz, row_loss, bad_labels, S_dev); if (le_ != cudaSuccess) return le_; } break;
+            case 2: { cudaError_t le_ = launch_pdl(k_softmax_ce_reg<2>, dim3(B), dim3(threads), 0, st, z, ldz, labels, C, c, dz, lddz, row_loss, bad_labels, S_dev); if (le_ != cudaSuccess) return le_; } break;
+            case 4: { cudaError_t le_ = launch_pdl(k_softmax_ce_reg<4>, dim3(B), dim3(threads), 0, st, z, ldz, labels, C, c, dz, lddz, row_loss, bad_labels, S_dev); if (le_ != cudaSuccess) return le_; } break;
+            default: { cudaError_t le_ = launch_pdl(k_softmax_ce_reg<8>, dim3(B), dim3(threads), 0, st, z, ldz, labels, C, c, dz, lddz, row_loss, bad_labels, S_dev); if (le_ != cudaSuccess) return le_; } break;
         }
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
         if (n_launches) *n_launches = 1;
         if (loss) {
-            k_loss_mean<<<1, 256, 0, st>>>(row_loss, B, loss);
+            { cudaError_t le_ = launch_pdl(k_loss_mean, dim3(1), dim3(256), 0, st, row_loss, B, loss); if (le_ != cudaSuccess) return le_; }
             if (n_launches) *n_launches = 2;
         }
         return cudaGetLastError();
@@ -474,7 +482,7 @@ cudaError_t launch_softmax_ce(const uint16_t *z, int ldz, const int32_t *labels,
     if (e != cudaSuccess) return e;
     if (n_launches) *n_launches = 1;
     if (loss) {
-        k_loss_mean<<<1, 256, 0, st>>>(row_loss, B, loss);
+            { cudaError_t le_ = launch_pdl(k_loss_mean, dim3(1), dim3(256), 0, st, row_loss, B, loss); if (le_ != cudaSuccess) return le_; }
         if (n_launches) *n_launches = 2;
     }
     return cudaGetLastError();

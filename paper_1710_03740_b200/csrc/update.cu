@@ -44,6 +44,8 @@ static inline unsigned vec_grid(size_t n8)
 __global__ void __launch_bounds__(kThreads) k_recast_vec(const float4 *__restrict__ w32, uint4 *__restrict__ w16,
                                                          size_t n8)
 {
+    pdl_trigger();
+    pdl_wait();
     const size_t base = (size_t)blockIdx.x * (kThreads * kVecPerThread) + threadIdx.x;
     float4 a[kVecPerThread], b[kVecPerThread];
 #pragma unroll
@@ -67,6 +69,8 @@ __global__ void __launch_bounds__(kThreads) k_recast_vec(const float4 *__restric
 
 __global__ void k_recast_scalar(const float *__restrict__ w32, uint16_t *__restrict__ w16, size_t begin, size_t n)
 {
+    pdl_trigger();
+    pdl_wait();
     size_t stride = (size_t)gridDim.x * blockDim.x;
     for (size_t i = begin + (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride)
         w16[i] = (uint16_t)f2h_bits(w32[i]);
@@ -77,8 +81,8 @@ cudaError_t launch_recast(const float *w32, uint16_t *w16, size_t n, cudaStream_
     if (n == 0) return cudaSuccess;
     bool aligned = (((uintptr_t)w32 | (uintptr_t)w16) & 15) == 0;
     size_t n8 = aligned ? n / 8 : 0;
-    if (n8) k_recast_vec<<<vec_grid(n8), kThreads, 0, st>>>((const float4 *)w32, (uint4 *)w16, n8);
-    if (n8 * 8 < n) k_recast_scalar<<<grid_for(n - n8 * 8), kThreads, 0, st>>>(w32, w16, n8 * 8, n);
+    if (n8){ cudaError_t le_ = launch_pdl(k_recast_vec, dim3(vec_grid(n8)), dim3(kThreads), 0, st, (const float4 *)w32, (uint4 *)w16, n8); if (le_ != cudaSuccess) return le_; }
+    if (n8 * 8 < n){ cudaError_t le_ = launch_pdl(k_recast_scalar, dim3(grid_for(n - n8 * 8)), dim3(kThreads), 0, st, w32, w16, n8 * 8, n); if (le_ != cudaSuccess) return le_; }
     return cudaGetLastError();
 }
 
@@ -93,6 +97,8 @@ __device__ __forceinline__ bool pair_nonfinite(uint32_t two_halfs, float inv)
 __global__ void __launch_bounds__(kThreads) k_nonfinite_vec(const uint4 *__restrict__ g, size_t n8, float inv,
                                                             uint32_t *flag)
 {
+    pdl_trigger();
+    pdl_wait();
     const size_t base = (size_t)blockIdx.x * (kThreads * kVecPerThread) + threadIdx.x;
     uint4 x[kVecPerThread];
 #pragma unroll
@@ -111,6 +117,8 @@ __global__ void __launch_bounds__(kThreads) k_nonfinite_vec(const uint4 *__restr
 
 __global__ void k_nonfinite_scalar(const uint16_t *__restrict__ g, size_t begin, size_t n, float inv, uint32_t *flag)
 {
+    pdl_trigger();
+    pdl_wait();
     size_t stride = (size_t)gridDim.x * blockDim.x;
     bool bad = false;
     for (size_t i = begin + (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride)
@@ -123,8 +131,8 @@ cudaError_t launch_grad_nonfinite(const uint16_t *g16, size_t n, float inv_S, ui
     if (n == 0) return cudaSuccess;
     bool aligned = ((uintptr_t)g16 & 15) == 0;
     size_t n8 = aligned ? n / 8 : 0;
-    if (n8) k_nonfinite_vec<<<vec_grid(n8), kThreads, 0, st>>>((const uint4 *)g16, n8, inv_S, flag);
-    if (n8 * 8 < n) k_nonfinite_scalar<<<grid_for(n - n8 * 8), kThreads, 0, st>>>(g16, n8 * 8, n, inv_S, flag);
+    if (n8){ cudaError_t le_ = launch_pdl(k_nonfinite_vec, dim3(vec_grid(n8)), dim3(kThreads), 0, st, (const uint4 *)g16, n8, inv_S, flag); if (le_ != cudaSuccess) return le_; }
+    if (n8 * 8 < n){ cudaError_t le_ = launch_pdl(k_nonfinite_scalar, dim3(grid_for(n - n8 * 8)), dim3(kThreads), 0, st, g16, n8 * 8, n, inv_S, flag); if (le_ != cudaSuccess) return le_; }
     return cudaGetLastError();
 }
 
@@ -174,6 +182,8 @@ __global__ void __launch_bounds__(kThreads) k_update_vec(const uint4 *__restrict
                                                          float inv, float lr, float mu, uint32_t *flags,
                                                          const float *__restrict__ inv_dev)
 {
+    pdl_trigger();
+    pdl_wait();
     if (*(volatile const uint32_t *)flags != 0u) return;
     if (inv_dev) inv = *inv_dev;
     const size_t base = (size_t)blockIdx.x * (kThreads * kVecPerThread) + threadIdx.x;
@@ -209,6 +219,8 @@ __global__ void k_update_scalar(const uint16_t *__restrict__ g16, float *__restr
                                 uint16_t *__restrict__ w16, size_t begin, size_t n, float inv, float lr, float mu,
                                 uint32_t *flags, const float *__restrict__ inv_dev)
 {
+    pdl_trigger();
+    pdl_wait();
     if (*(volatile const uint32_t *)flags != 0u) return;
     if (inv_dev) inv = *inv_dev;
     size_t stride = (size_t)gridDim.x * blockDim.x;
@@ -233,18 +245,18 @@ cudaError_t launch_update(const uint16_t *g16, float *w32, float *v, uint16_t *w
         const size_t per_cta = (size_t)kThreads * kVecPerThread;
         const unsigned grid = (unsigned)((n8 + per_cta - 1) / per_cta);
         if (use_momentum)
-            k_update_vec<true><<<grid, kThreads, 0, st>>>((const uint4 *)g16, (float4 *)w32, (float4 *)v, (uint4 *)w16,
-                                                          n8, inv_S, lr, mu, flags, inv_S_dev);
+            { cudaError_t le_ = launch_pdl(k_update_vec<true>, dim3(grid), dim3(kThreads), 0, st, (const uint4 *)g16, (float4 *)w32, (float4 *)v, (uint4 *)w16,
+                                                          n8, inv_S, lr, mu, flags, inv_S_dev); if (le_ != cudaSuccess) return le_; }
         else
-            k_update_vec<false><<<grid, kThreads, 0, st>>>((const uint4 *)g16, (float4 *)w32, nullptr, (uint4 *)w16, n8,
-                                                           inv_S, lr, mu, flags, inv_S_dev);
+            { cudaError_t le_ = launch_pdl(k_update_vec<false>, dim3(grid), dim3(kThreads), 0, st, (const uint4 *)g16, (float4 *)w32, nullptr, (uint4 *)w16, n8,
+                                                           inv_S, lr, mu, flags, inv_S_dev); if (le_ != cudaSuccess) return le_; }
     }
     if (n8 * 8 < n) {
         int grid = grid_for(n - n8 * 8);
         if (use_momentum)
-            k_update_scalar<true><<<grid, kThreads, 0, st>>>(g16, w32, v, w16, n8 * 8, n, inv_S, lr, mu, flags, inv_S_dev);
+            { cudaError_t le_ = launch_pdl(k_update_scalar<true>, dim3(grid), dim3(kThreads), 0, st, g16, w32, v, w16, n8 * 8, n, inv_S, lr, mu, flags, inv_S_dev); if (le_ != cudaSuccess) return le_; }
         else
-            k_update_scalar<false><<<grid, kThreads, 0, st>>>(g16, w32, nullptr, w16, n8 * 8, n, inv_S, lr, mu, flags, inv_S_dev);
+            { cudaError_t le_ = launch_pdl(k_update_scalar<false>, dim3(grid), dim3(kThreads), 0, st, g16, w32, nullptr, w16, n8 * 8, n, inv_S, lr, mu, flags, inv_S_dev); if (le_ != cudaSuccess) return le_; }
     }
     return cudaGetLastError();
 }
@@ -294,6 +306,8 @@ __global__ void __launch_bounds__(kThreads) k_update_opt(const uint4 *__restrict
                                                          const float *__restrict__ betat_dev,
                                                          const float *__restrict__ coef_dev)
 {
+    pdl_trigger();
+    pdl_wait();
     if (*(volatile const uint32_t *)flags != 0u) return;
     if (inv_dev) inv = *inv_dev;
     const float coef = coef_dev ? *coef_dev : 1.0f;
@@ -351,6 +365,8 @@ __global__ void k_update_opt_scalar(const uint16_t *__restrict__ g16, float *__r
                                     const float *__restrict__ inv_dev, const float *__restrict__ betat_dev,
                                     const float *__restrict__ coef_dev)
 {
+    pdl_trigger();
+    pdl_wait();
     if (*(volatile const uint32_t *)flags != 0u) return;
     if (inv_dev) inv = *inv_dev;
     const float coef = coef_dev ? *coef_dev : 1.0f;
@@ -381,13 +397,13 @@ static cudaError_t launch_opt_variant(const uint16_t *g16, float *w32, float *s1
     size_t n8 = (bits & 15) == 0 ? n / 8 : 0;
     if (n8) {
         const size_t per_cta = (size_t)kThreads * kOptVec;
-        k_update_opt<KIND, WD><<<(unsigned)((n8 + per_cta - 1) / per_cta), kThreads, 0, st>>>(
+            { cudaError_t le_ = launch_pdl(k_update_opt<KIND, WD>, dim3((unsigned)((n8 + per_cta - 1) / per_cta)), dim3(kThreads), 0, st, 
             (const uint4 *)g16, (float4 *)w32, (float4 *)s1, (float4 *)s2, (uint4 *)w16, n8, inv_S, lr, mu, b2, eps, wd, b1t, b2t,
-            flags, inv_dev, betat_dev, coef_dev);
+            flags, inv_dev, betat_dev, coef_dev); if (le_ != cudaSuccess) return le_; }
     }
     if (n8 * 8 < n)
-        k_update_opt_scalar<KIND, WD><<<grid_for(n - n8 * 8), kThreads, 0, st>>>(g16, w32, s1, s2, w16, n8 * 8, n, inv_S, lr, mu, b2,
-                                                                                eps, wd, b1t, b2t, flags, inv_dev, betat_dev, coef_dev);
+            { cudaError_t le_ = launch_pdl(k_update_opt_scalar<KIND, WD>, dim3(grid_for(n - n8 * 8)), dim3(kThreads), 0, st, g16, w32, s1, s2, w16, n8 * 8, n, inv_S, lr, mu, b2,
+                                                                                eps, wd, b1t, b2t, flags, inv_dev, betat_dev, coef_dev); if (le_ != cudaSuccess) return le_; }
     return cudaGetLastError();
 }
 
@@ -416,6 +432,8 @@ cudaError_t launch_update_opt(int kind, const uint16_t *g16, float *w32, float *
 __global__ void k_post_step(uint32_t *status, int interval, float backoff, float growth, float min_S, float max_S, int adam,
                             float b1, float b2)
 {
+    pdl_trigger();
+    pdl_wait();
     const bool overflow = status[ST_OVERFLOW] != 0u;
     if (adam && !overflow) {
         status[ST_B1T] = __float_as_uint(__fmul_rn(__uint_as_float(status[ST_B1T]), b1));
@@ -440,7 +458,7 @@ __global__ void k_post_step(uint32_t *status, int interval, float backoff, float
 cudaError_t launch_post_step(uint32_t *status, int interval, float backoff, float growth, float min_S, float max_S, int adam,
                              float b1, float b2, cudaStream_t st)
 {
-    k_post_step<<<1, 1, 0, st>>>(status, interval, backoff, growth, min_S, max_S, adam, b1, b2);
+            { cudaError_t le_ = launch_pdl(k_post_step, dim3(1), dim3(1), 0, st, status, interval, backoff, growth, min_S, max_S, adam, b1, b2); if (le_ != cudaSuccess) return le_; }
     return cudaGetLastError();
 }
 
@@ -452,6 +470,8 @@ cudaError_t launch_post_step(uint32_t *status, int interval, float backoff, floa
 // clamp to [min_S, max_S].  With power-of-two factors every scale stays a power of two.
 __global__ void k_scale_adjust(uint32_t *status, int interval, float backoff, float growth, float min_S, float max_S)
 {
+    pdl_trigger();
+    pdl_wait();
     float S = __uint_as_float(status[ST_SCALE]);
     uint32_t clean = status[ST_CLEAN_STEPS];
     if (status[ST_OVERFLOW] != 0u) {
@@ -469,7 +489,7 @@ __global__ void k_scale_adjust(uint32_t *status, int interval, float backoff, fl
 cudaError_t launch_scale_adjust(uint32_t *status, int interval, float backoff, float growth, float min_S, float max_S,
                                 cudaStream_t st)
 {
-    k_scale_adjust<<<1, 1, 0, st>>>(status, interval, backoff, growth, min_S, max_S);
+            { cudaError_t le_ = launch_pdl(k_scale_adjust, dim3(1), dim3(1), 0, st, status, interval, backoff, growth, min_S, max_S); if (le_ != cudaSuccess) return le_; }
     return cudaGetLastError();
 }
 
@@ -496,6 +516,8 @@ __device__ __forceinline__ double block_sum_fixed(double v, double *sh)
 __global__ void __launch_bounds__(kThreads) k_grad_sqnorm(const uint16_t *__restrict__ g16, size_t n, size_t n8, float inv,
                                                           const float *__restrict__ inv_dev, double *__restrict__ parts)
 {
+    pdl_trigger();
+    pdl_wait();
     __shared__ double sh[kThreads / 32];
     if (inv_dev) inv = *inv_dev;
     double acc = 0.0;
@@ -524,6 +546,8 @@ __global__ void __launch_bounds__(kThreads) k_grad_sqnorm(const uint16_t *__rest
 __global__ void __launch_bounds__(1024) k_clip_coef(const double *__restrict__ parts, int count, float clip,
                                                     float *__restrict__ out)
 {
+    pdl_trigger();
+    pdl_wait();
     __shared__ double sh[32];
     double acc = 0.0;
     for (int i = threadIdx.x; i < count; i += 1024) acc += parts[i];
@@ -541,8 +565,8 @@ cudaError_t launch_clip_coef(const uint16_t *g16, size_t n, float inv_S, const f
     const size_t n8 = ((uintptr_t)g16 & 15) == 0 ? n / 8 : 0;
     size_t want = (n8 + kThreads - 1) / kThreads;
     const int grid = (int)(want < 1 ? 1 : (want > (size_t)kNormParts ? (size_t)kNormParts : want));
-    k_grad_sqnorm<<<grid, kThreads, 0, st>>>(g16, n, n8, inv_S, inv_dev, parts);
-    k_clip_coef<<<1, 1024, 0, st>>>(parts, grid, clip, out2);
+            { cudaError_t le_ = launch_pdl(k_grad_sqnorm, dim3(grid), dim3(kThreads), 0, st, g16, n, n8, inv_S, inv_dev, parts); if (le_ != cudaSuccess) return le_; }
+            { cudaError_t le_ = launch_pdl(k_clip_coef, dim3(1), dim3(1024), 0, st, parts, grid, clip, out2); if (le_ != cudaSuccess) return le_; }
     return cudaGetLastError();
 }
 
