@@ -21,6 +21,8 @@ __global__ void __launch_bounds__(256) k_lstm_cell_simt(int B, int H, int K, con
                                                         const uint16_t *__restrict__ Wg, int ldw,
                                                         uint16_t *__restrict__ acts, int ldacts, LstmEpi e)
 {
+    pdl_trigger();
+    pdl_wait();
     const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= (size_t)B * H) return;
     const int b = (int)(idx / H), j = (int)(idx % H);
@@ -72,6 +74,8 @@ __global__ void __launch_bounds__(256) k_lstm_cell_bwd(int B, int H4, const uint
                                                        const uint16_t *__restrict__ c16, int ldc, uint16_t *__restrict__ dG,
                                                        int lddg, uint16_t *__restrict__ dc_prev, int lddcp)
 {
+    pdl_trigger();
+    pdl_wait();
     const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= (size_t)B * H4) return;
     const int b = (int)(idx / H4), j = 4 * (int)(idx % H4);
@@ -111,6 +115,8 @@ __global__ void __launch_bounds__(256) k_lstm_cell_bwd_scalar(int B, int H, cons
                                                               uint16_t *__restrict__ dG, int lddg,
                                                               uint16_t *__restrict__ dc_prev, int lddcp)
 {
+    pdl_trigger();
+    pdl_wait();
     const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= (size_t)B * H) return;
     const int b = (int)(idx / H), j = (int)(idx % H);
@@ -132,6 +138,8 @@ __global__ void __launch_bounds__(256) k_lstm_cell_bwd_scalar(int B, int H, cons
 __global__ void __launch_bounds__(256) k_bias_grad_partial(const uint16_t *__restrict__ dG, size_t rows, int cols, int ld,
                                                            float *__restrict__ parts, bool vec)
 {
+    pdl_trigger();
+    pdl_wait();
     __shared__ float sh[8][256];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int col = blockIdx.x * 256 + lane * 8;
@@ -166,6 +174,8 @@ __global__ void __launch_bounds__(256) k_bias_grad_partial(const uint16_t *__res
 __global__ void __launch_bounds__(256) k_bias_grad_final(const float *__restrict__ parts, int nparts, int cols,
                                                          uint16_t *__restrict__ db16, uint32_t *nonfinite_flag)
 {
+    pdl_trigger();
+    pdl_wait();
     const int c = blockIdx.x * blockDim.x + threadIdx.x;
     bool bad = false;
     if (c < cols) {
@@ -183,6 +193,8 @@ __global__ void __launch_bounds__(256) k_bias_grad_final(const float *__restrict
 __global__ void __launch_bounds__(256) k_add_f16(const uint16_t *__restrict__ a, int lda, const uint16_t *__restrict__ b,
                                                  int ldb, uint16_t *__restrict__ out, int ldo, int rows, int cols)
 {
+    pdl_trigger();
+    pdl_wait();
     const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= (size_t)rows * cols) return;
     const int r = (int)(idx / cols), c = (int)(idx % cols);
@@ -191,6 +203,8 @@ __global__ void __launch_bounds__(256) k_add_f16(const uint16_t *__restrict__ a,
 
 __global__ void __launch_bounds__(256) k_widen_f16(const uint16_t *__restrict__ in16, float *__restrict__ out32, size_t n)
 {
+    pdl_trigger();
+    pdl_wait();
     const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i < n) out32[i] = h2f_u(in16[i]);
 }
@@ -203,7 +217,7 @@ cudaError_t launch_lstm_cell_simt(int B, int H, int K, const uint16_t *XR, int l
                                   uint16_t *acts, int ldacts, const LstmEpi &e, cudaStream_t st)
 {
     if (B <= 0 || H <= 0) return cudaSuccess;
-    k_lstm_cell_simt<<<blocks_for((size_t)B * H), 256, 0, st>>>(B, H, K, XR, ldxr, Wg, ldw, acts, ldacts, e);
+    { cudaError_t le_ = launch_pdl(k_lstm_cell_simt, dim3(blocks_for((size_t)B * H)), dim3(256), 0, st, B, H, K, XR, ldxr, Wg, ldw, acts, ldacts, e); if (le_ != cudaSuccess) return le_; }
     return cudaGetLastError();
 }
 
@@ -217,11 +231,11 @@ cudaError_t launch_lstm_cell_bwd(int B, int H, const uint16_t *dh, int lddh, con
     const bool vec = (H % 4) == 0 && (bits & 15) == 0 && (bits4 & 7) == 0 && (ldacts % 8) == 0 && (lddg % 8) == 0 &&
                      ((lddh | lddc | ldcp | ldc | lddcp) % 4) == 0;
     if (vec)
-        k_lstm_cell_bwd<<<blocks_for((size_t)B * (H / 4)), 256, 0, st>>>(B, H / 4, dh, lddh, dc_next, lddc, acts, ldacts, c_prev,
-                                                                         ldcp, c16, ldc, dG, lddg, dc_prev, lddcp);
+    { cudaError_t le_ = launch_pdl(k_lstm_cell_bwd, dim3(blocks_for((size_t)B * (H / 4))), dim3(256), 0, st, B, H / 4, dh, lddh, dc_next, lddc, acts, ldacts, c_prev,
+                                                                         ldcp, c16, ldc, dG, lddg, dc_prev, lddcp); if (le_ != cudaSuccess) return le_; }
     else
-        k_lstm_cell_bwd_scalar<<<blocks_for((size_t)B * H), 256, 0, st>>>(B, H, dh, lddh, dc_next, lddc, acts, ldacts, c_prev,
-                                                                          ldcp, c16, ldc, dG, lddg, dc_prev, lddcp);
+    { cudaError_t le_ = launch_pdl(k_lstm_cell_bwd_scalar, dim3(blocks_for((size_t)B * H)), dim3(256), 0, st, B, H, dh, lddh, dc_next, lddc, acts, ldacts, c_prev,
+                                                                          ldcp, c16, ldc, dG, lddg, dc_prev, lddcp); if (le_ != cudaSuccess) return le_; }
     return cudaGetLastError();
 }
 
@@ -231,15 +245,15 @@ cudaError_t launch_bias_grad(const uint16_t *dG, size_t rows, int cols, int ld, 
     if (cols <= 0) return cudaSuccess;
     const bool vec = ((uintptr_t)dG & 15) == 0 && (ld % 8) == 0;
     dim3 grid((unsigned)((cols + 255) / 256), (unsigned)kBiasRowParts);
-    k_bias_grad_partial<<<grid, 256, 0, st>>>(dG, rows, cols, ld, parts, vec);   // unaligned rows: element loads
-    k_bias_grad_final<<<blocks_for((size_t)cols), 256, 0, st>>>(parts, kBiasRowParts, cols, db16, nonfinite_flag);
+    { cudaError_t le_ = launch_pdl(k_bias_grad_partial, dim3(grid), dim3(256), 0, st, dG, rows, cols, ld, parts, vec); if (le_ != cudaSuccess) return le_; }   // unaligned rows: element loads
+    { cudaError_t le_ = launch_pdl(k_bias_grad_final, dim3(blocks_for((size_t)cols)), dim3(256), 0, st, parts, kBiasRowParts, cols, db16, nonfinite_flag); if (le_ != cudaSuccess) return le_; }
     return cudaGetLastError();
 }
 
 cudaError_t launch_widen_f16(const uint16_t *in16, float *out32, size_t n, cudaStream_t st)
 {
     if (n == 0) return cudaSuccess;
-    k_widen_f16<<<blocks_for(n), 256, 0, st>>>(in16, out32, n);
+    { cudaError_t le_ = launch_pdl(k_widen_f16, dim3(blocks_for(n)), dim3(256), 0, st, in16, out32, n); if (le_ != cudaSuccess) return le_; }
     return cudaGetLastError();
 }
 
@@ -247,7 +261,7 @@ cudaError_t launch_add_f16(const uint16_t *a, int lda, const uint16_t *b, int ld
                            int cols, cudaStream_t st)
 {
     if (rows <= 0 || cols <= 0) return cudaSuccess;
-    k_add_f16<<<blocks_for((size_t)rows * cols), 256, 0, st>>>(a, lda, b, ldb, out, ldo, rows, cols);
+    { cudaError_t le_ = launch_pdl(k_add_f16, dim3(blocks_for((size_t)rows * cols)), dim3(256), 0, st, a, lda, b, ldb, out, ldo, rows, cols); if (le_ != cudaSuccess) return le_; }
     return cudaGetLastError();
 }
 
