@@ -95,11 +95,11 @@ cudaError_t launch_gemm_simt(int op, int M, int N, int K, const uint16_t *A, int
     if (M <= 0 || N <= 0) return cudaSuccess;
     dim3 grid((N + BN - 1) / BN, (M + BM - 1) / BM);
     if (op == MPT_OP_FWD)
-            { cudaError_t le_ = launch_pdl(k_gemm_simt<false, false>, dim3(grid), dim3(256), 0, st, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite_flag); if (le_ != cudaSuccess) return le_; }
+        MPT_LAUNCH(k_gemm_simt<false, false>, dim3(grid), dim3(256), 0, st, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite_flag);
     else if (op == MPT_OP_DGRAD)
-            { cudaError_t le_ = launch_pdl(k_gemm_simt<false, true>, dim3(grid), dim3(256), 0, st, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite_flag); if (le_ != cudaSuccess) return le_; }
+        MPT_LAUNCH(k_gemm_simt<false, true>, dim3(grid), dim3(256), 0, st, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite_flag);
     else
-            { cudaError_t le_ = launch_pdl(k_gemm_simt<true, true>, dim3(grid), dim3(256), 0, st, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite_flag); if (le_ != cudaSuccess) return le_; }
+        MPT_LAUNCH(k_gemm_simt<true, true>, dim3(grid), dim3(256), 0, st, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite_flag);
     return cudaGetLastError();
 }
 

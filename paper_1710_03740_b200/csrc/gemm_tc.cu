@@ -339,8 +339,8 @@ cudaError_t launch_splitk_reduce(const float *partial, int split_k, int M, int N
     const size_t work = (size_t)M * ((N + 7) / 8);
     size_t blocks = (work + 255) / 256;
     if (blocks > 148 * 16) blocks = 148 * 16;
-            { cudaError_t le_ = launch_pdl(k_splitk_reduce, dim3((unsigned)blocks), dim3(256), 0, st, partial, split_k, M, N, ldp, C, ldc, relu ? 1 : 0, mask, ldmask,
-                                                      nonfinite_flag); if (le_ != cudaSuccess) return le_; }
+    MPT_LAUNCH(k_splitk_reduce, dim3((unsigned)blocks), dim3(256), 0, st, partial, split_k, M, N, ldp, C, ldc, relu ? 1 : 0, mask, ldmask,
+               nonfinite_flag);
     g_last_gemm_launches = 2;
     return cudaGetLastError();
 }
@@ -406,7 +406,7 @@ static cudaError_t launch_variant(const CUtensorMap &ta, const CUtensorMap &tb, 
         if (e != cudaSuccess) return e;
         configured[dev] = true;
     }
-            { cudaError_t le_ = launch_pdl(kern, dim3(grid), dim3(EpiCfg<LSTM || WIDE>::THREADS), SMEM_BYTES, st, ta, tb, p); if (le_ != cudaSuccess) return le_; }
+    MPT_LAUNCH(kern, dim3(grid), dim3(EpiCfg<LSTM || WIDE>::THREADS), SMEM_BYTES, st, ta, tb, p);
     return cudaGetLastError();
 }
 

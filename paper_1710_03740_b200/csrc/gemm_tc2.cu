@@ -490,7 +490,7 @@ static cudaError_t launch_variant(const CUtensorMap &ta, const CUtensorMap &tb, 
     const size_t work = (size_t)rest * (2 * CTA_M) * (TILE_N / 8);
     size_t blocks = (work + 255) / 256;
     if (blocks > 148 * 8) blocks = 148 * 8;
-            { cudaError_t le_ = launch_pdl(k_tail_reduce, dim3((unsigned)blocks), dim3(256), 0, st, p, full, rest); if (le_ != cudaSuccess) return le_; }
+    MPT_LAUNCH(k_tail_reduce, dim3((unsigned)blocks), dim3(256), 0, st, p, full, rest);
     g_last_gemm_launches = 2;
     return cudaGetLastError();
 }

@@ -217,7 +217,7 @@ cudaError_t launch_lstm_cell_simt(int B, int H, int K, const uint16_t *XR, int l
                                   uint16_t *acts, int ldacts, const LstmEpi &e, cudaStream_t st)
 {
     if (B <= 0 || H <= 0) return cudaSuccess;
-    { cudaError_t le_ = launch_pdl(k_lstm_cell_simt, dim3(blocks_for((size_t)B * H)), dim3(256), 0, st, B, H, K, XR, ldxr, Wg, ldw, acts, ldacts, e); if (le_ != cudaSuccess) return le_; }
+    MPT_LAUNCH(k_lstm_cell_simt, dim3(blocks_for((size_t)B * H)), dim3(256), 0, st, B, H, K, XR, ldxr, Wg, ldw, acts, ldacts, e);
     return cudaGetLastError();
 }
 
@@ -231,11 +231,11 @@ cudaError_t launch_lstm_cell_bwd(int B, int H, const uint16_t *dh, int lddh, con
     const bool vec = (H % 4) == 0 && (bits & 15) == 0 && (bits4 & 7) == 0 && (ldacts % 8) == 0 && (lddg % 8) == 0 &&
                      ((lddh | lddc | ldcp | ldc | lddcp) % 4) == 0;
     if (vec)
-    { cudaError_t le_ = launch_pdl(k_lstm_cell_bwd, dim3(blocks_for((size_t)B * (H / 4))), dim3(256), 0, st, B, H / 4, dh, lddh, dc_next, lddc, acts, ldacts, c_prev,
-                                                                         ldcp, c16, ldc, dG, lddg, dc_prev, lddcp); if (le_ != cudaSuccess) return le_; }
+        MPT_LAUNCH(k_lstm_cell_bwd, dim3(blocks_for((size_t)B * (H / 4))), dim3(256), 0, st, B, H / 4, dh, lddh, dc_next, lddc, acts, ldacts, c_prev,
+                   ldcp, c16, ldc, dG, lddg, dc_prev, lddcp);
     else
-    { cudaError_t le_ = launch_pdl(k_lstm_cell_bwd_scalar, dim3(blocks_for((size_t)B * H)), dim3(256), 0, st, B, H, dh, lddh, dc_next, lddc, acts, ldacts, c_prev,
-                                                                          ldcp, c16, ldc, dG, lddg, dc_prev, lddcp); if (le_ != cudaSuccess) return le_; }
+        MPT_LAUNCH(k_lstm_cell_bwd_scalar, dim3(blocks_for((size_t)B * H)), dim3(256), 0, st, B, H, dh, lddh, dc_next, lddc, acts, ldacts, c_prev,
+                   ldcp, c16, ldc, dG, lddg, dc_prev, lddcp);
     return cudaGetLastError();
 }
 
@@ -245,15 +245,15 @@ cudaError_t launch_bias_grad(const uint16_t *dG, size_t rows, int cols, int ld, 
     if (cols <= 0) return cudaSuccess;
     const bool vec = ((uintptr_t)dG & 15) == 0 && (ld % 8) == 0;
     dim3 grid((unsigned)((cols + 255) / 256), (unsigned)kBiasRowParts);
-    { cudaError_t le_ = launch_pdl(k_bias_grad_partial, dim3(grid), dim3(256), 0, st, dG, rows, cols, ld, parts, vec); if (le_ != cudaSuccess) return le_; }   // unaligned rows: element loads
-    { cudaError_t le_ = launch_pdl(k_bias_grad_final, dim3(blocks_for((size_t)cols)), dim3(256), 0, st, parts, kBiasRowParts, cols, db16, nonfinite_flag); if (le_ != cudaSuccess) return le_; }
+    MPT_LAUNCH(k_bias_grad_partial, dim3(grid), dim3(256), 0, st, dG, rows, cols, ld, parts, vec);   // unaligned rows: element loads
+    MPT_LAUNCH(k_bias_grad_final, dim3(blocks_for((size_t)cols)), dim3(256), 0, st, parts, kBiasRowParts, cols, db16, nonfinite_flag);
     return cudaGetLastError();
 }
 
 cudaError_t launch_widen_f16(const uint16_t *in16, float *out32, size_t n, cudaStream_t st)
 {
     if (n == 0) return cudaSuccess;
-    { cudaError_t le_ = launch_pdl(k_widen_f16, dim3(blocks_for(n)), dim3(256), 0, st, in16, out32, n); if (le_ != cudaSuccess) return le_; }
+    MPT_LAUNCH(k_widen_f16, dim3(blocks_for(n)), dim3(256), 0, st, in16, out32, n);
     return cudaGetLastError();
 }
 
@@ -261,7 +261,7 @@ cudaError_t launch_add_f16(const uint16_t *a, int lda, const uint16_t *b, int ld
                            int cols, cudaStream_t st)
 {
     if (rows <= 0 || cols <= 0) return cudaSuccess;
-    { cudaError_t le_ = launch_pdl(k_add_f16, dim3(blocks_for((size_t)rows * cols)), dim3(256), 0, st, a, lda, b, ldb, out, ldo, rows, cols); if (le_ != cudaSuccess) return le_; }
+    MPT_LAUNCH(k_add_f16, dim3(blocks_for((size_t)rows * cols)), dim3(256), 0, st, a, lda, b, ldb, out, ldo, rows, cols);
     return cudaGetLastError();
 }
 

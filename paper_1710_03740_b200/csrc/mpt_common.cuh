@@ -74,6 +74,13 @@ inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, siz
     return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
 }
 
+// Launch through launch_pdl and return its error from the calling function if the launch failed.
+#define MPT_LAUNCH(...)                                      \
+    do {                                                     \
+        cudaError_t launch_err_ = launch_pdl(__VA_ARGS__);   \
+        if (launch_err_ != cudaSuccess) return launch_err_;  \
+    } while (0)
+
 __device__ __forceinline__ bool half_bits_nonfinite(uint32_t h) { return (h & 0x7C00u) == 0x7C00u; }
 __device__ __forceinline__ bool f32_nonfinite(float x)
 {

@@ -403,7 +403,7 @@ static cudaError_t launch_variant(const uint16_t *z, int ldz, const int32_t *lab
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
     }
-            { cudaError_t le_ = launch_pdl(kern, dim3(grid), dim3(threads), smem, st, z, ldz, labels, B, C, c, dz, lddz, row_loss, bad_labels, S_dev); if (le_ != cudaSuccess) return le_; }
+    MPT_LAUNCH(kern, dim3(grid), dim3(threads), smem, st, z, ldz, labels, B, C, c, dz, lddz, row_loss, bad_labels, S_dev);
     return cudaGetLastError();
 }
 
@@ -433,12 +433,12 @@ cudaError_t launch_softmax_ce(const uint16_t *z, int ldz, const int32_t *labels,
             sms_dev[dev] = n > 0 ? n : 148;
         }
         const int grid = B < sms_dev[dev] ? B : sms_dev[dev];
-            { cudaError_t le_ = launch_pdl(kern, dim3(grid), dim3(kSmaxThreads), smem, st, z, ldz, labels, B, C, c, dz, lddz, row_loss, bad_labels, S_dev, kerr); if (le_ != cudaSuccess) return le_; }
+        MPT_LAUNCH(kern, dim3(grid), dim3(kSmaxThreads), smem, st, z, ldz, labels, B, C, c, dz, lddz, row_loss, bad_labels, S_dev, kerr);
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
         if (n_launches) *n_launches = 1;
         if (loss) {
-            { cudaError_t le_ = launch_pdl(k_loss_mean, dim3(1), dim3(256), 0, st, row_loss, B, loss); if (le_ != cudaSuccess) return le_; }
+            MPT_LAUNCH(k_loss_mean, dim3(1), dim3(256), 0, st, row_loss, B, loss);
             if (n_launches) *n_launches = 2;
         }
         return cudaGetLastError();
@@ -452,16 +452,16 @@ cudaError_t launch_softmax_ce(const uint16_t *z, int ldz, const int32_t *labels,
         threads = ((threads + 31) / 32) * 32;
         if (threads < 32) threads = 32;
         switch (vpt) {
-            case 1: { cudaError_t le_ = launch_pdl(k_softmax_ce_reg<1>, dim3(B), dim3(threads), 0, st, z, ldz, labels, C, c, dz, lddz, row_loss, bad_labels, S_dev); if (le_ != cudaSuccess) return le_; } break;
-            case 2: { cudaError_t le_ = launch_pdl(k_softmax_ce_reg<2>, dim3(B), dim3(threads), 0, st, z, ldz, labels, C, c, dz, lddz, row_loss, bad_labels, S_dev); if (le_ != cudaSuccess) return le_; } break;
-            case 4: { cudaError_t le_ = launch_pdl(k_softmax_ce_reg<4>, dim3(B), dim3(threads), 0, st, z, ldz, labels, C, c, dz, lddz, row_loss, bad_labels, S_dev); if (le_ != cudaSuccess) return le_; } break;
-            default: { cudaError_t le_ = launch_pdl(k_softmax_ce_reg<8>, dim3(B), dim3(threads), 0, st, z, ldz, labels, C, c, dz, lddz, row_loss, bad_labels, S_dev); if (le_ != cudaSuccess) return le_; } break;
+            case 1: MPT_LAUNCH(k_softmax_ce_reg<1>, dim3(B), dim3(threads), 0, st, z, ldz, labels, C, c, dz, lddz, row_loss, bad_labels, S_dev); break;
+            case 2: MPT_LAUNCH(k_softmax_ce_reg<2>, dim3(B), dim3(threads), 0, st, z, ldz, labels, C, c, dz, lddz, row_loss, bad_labels, S_dev); break;
+            case 4: MPT_LAUNCH(k_softmax_ce_reg<4>, dim3(B), dim3(threads), 0, st, z, ldz, labels, C, c, dz, lddz, row_loss, bad_labels, S_dev); break;
+            default: MPT_LAUNCH(k_softmax_ce_reg<8>, dim3(B), dim3(threads), 0, st, z, ldz, labels, C, c, dz, lddz, row_loss, bad_labels, S_dev); break;
         }
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
         if (n_launches) *n_launches = 1;
         if (loss) {
-            { cudaError_t le_ = launch_pdl(k_loss_mean, dim3(1), dim3(256), 0, st, row_loss, B, loss); if (le_ != cudaSuccess) return le_; }
+            MPT_LAUNCH(k_loss_mean, dim3(1), dim3(256), 0, st, row_loss, B, loss);
             if (n_launches) *n_launches = 2;
         }
         return cudaGetLastError();
@@ -482,7 +482,7 @@ cudaError_t launch_softmax_ce(const uint16_t *z, int ldz, const int32_t *labels,
     if (e != cudaSuccess) return e;
     if (n_launches) *n_launches = 1;
     if (loss) {
-            { cudaError_t le_ = launch_pdl(k_loss_mean, dim3(1), dim3(256), 0, st, row_loss, B, loss); if (le_ != cudaSuccess) return le_; }
+        MPT_LAUNCH(k_loss_mean, dim3(1), dim3(256), 0, st, row_loss, B, loss);
         if (n_launches) *n_launches = 2;
     }
     return cudaGetLastError();

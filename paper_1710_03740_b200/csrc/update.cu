@@ -81,8 +81,8 @@ cudaError_t launch_recast(const float *w32, uint16_t *w16, size_t n, cudaStream_
     if (n == 0) return cudaSuccess;
     bool aligned = (((uintptr_t)w32 | (uintptr_t)w16) & 15) == 0;
     size_t n8 = aligned ? n / 8 : 0;
-    if (n8){ cudaError_t le_ = launch_pdl(k_recast_vec, dim3(vec_grid(n8)), dim3(kThreads), 0, st, (const float4 *)w32, (uint4 *)w16, n8); if (le_ != cudaSuccess) return le_; }
-    if (n8 * 8 < n){ cudaError_t le_ = launch_pdl(k_recast_scalar, dim3(grid_for(n - n8 * 8)), dim3(kThreads), 0, st, w32, w16, n8 * 8, n); if (le_ != cudaSuccess) return le_; }
+    if (n8) MPT_LAUNCH(k_recast_vec, dim3(vec_grid(n8)), dim3(kThreads), 0, st, (const float4 *)w32, (uint4 *)w16, n8);
+    if (n8 * 8 < n) MPT_LAUNCH(k_recast_scalar, dim3(grid_for(n - n8 * 8)), dim3(kThreads), 0, st, w32, w16, n8 * 8, n);
     return cudaGetLastError();
 }
 
@@ -131,8 +131,8 @@ cudaError_t launch_grad_nonfinite(const uint16_t *g16, size_t n, float inv_S, ui
     if (n == 0) return cudaSuccess;
     bool aligned = ((uintptr_t)g16 & 15) == 0;
     size_t n8 = aligned ? n / 8 : 0;
-    if (n8){ cudaError_t le_ = launch_pdl(k_nonfinite_vec, dim3(vec_grid(n8)), dim3(kThreads), 0, st, (const uint4 *)g16, n8, inv_S, flag); if (le_ != cudaSuccess) return le_; }
-    if (n8 * 8 < n){ cudaError_t le_ = launch_pdl(k_nonfinite_scalar, dim3(grid_for(n - n8 * 8)), dim3(kThreads), 0, st, g16, n8 * 8, n, inv_S, flag); if (le_ != cudaSuccess) return le_; }
+    if (n8) MPT_LAUNCH(k_nonfinite_vec, dim3(vec_grid(n8)), dim3(kThreads), 0, st, (const uint4 *)g16, n8, inv_S, flag);
+    if (n8 * 8 < n) MPT_LAUNCH(k_nonfinite_scalar, dim3(grid_for(n - n8 * 8)), dim3(kThreads), 0, st, g16, n8 * 8, n, inv_S, flag);
     return cudaGetLastError();
 }
 
@@ -245,18 +245,18 @@ cudaError_t launch_update(const uint16_t *g16, float *w32, float *v, uint16_t *w
         const size_t per_cta = (size_t)kThreads * kVecPerThread;
         const unsigned grid = (unsigned)((n8 + per_cta - 1) / per_cta);
         if (use_momentum)
-            { cudaError_t le_ = launch_pdl(k_update_vec<true>, dim3(grid), dim3(kThreads), 0, st, (const uint4 *)g16, (float4 *)w32, (float4 *)v, (uint4 *)w16,
-                                                          n8, inv_S, lr, mu, flags, inv_S_dev); if (le_ != cudaSuccess) return le_; }
+            MPT_LAUNCH(k_update_vec<true>, dim3(grid), dim3(kThreads), 0, st, (const uint4 *)g16, (float4 *)w32, (float4 *)v, (uint4 *)w16,
+                       n8, inv_S, lr, mu, flags, inv_S_dev);
         else
-            { cudaError_t le_ = launch_pdl(k_update_vec<false>, dim3(grid), dim3(kThreads), 0, st, (const uint4 *)g16, (float4 *)w32, nullptr, (uint4 *)w16, n8,
-                                                           inv_S, lr, mu, flags, inv_S_dev); if (le_ != cudaSuccess) return le_; }
+            MPT_LAUNCH(k_update_vec<false>, dim3(grid), dim3(kThreads), 0, st, (const uint4 *)g16, (float4 *)w32, nullptr, (uint4 *)w16, n8,
+                       inv_S, lr, mu, flags, inv_S_dev);
     }
     if (n8 * 8 < n) {
         int grid = grid_for(n - n8 * 8);
         if (use_momentum)
-            { cudaError_t le_ = launch_pdl(k_update_scalar<true>, dim3(grid), dim3(kThreads), 0, st, g16, w32, v, w16, n8 * 8, n, inv_S, lr, mu, flags, inv_S_dev); if (le_ != cudaSuccess) return le_; }
+            MPT_LAUNCH(k_update_scalar<true>, dim3(grid), dim3(kThreads), 0, st, g16, w32, v, w16, n8 * 8, n, inv_S, lr, mu, flags, inv_S_dev);
         else
-            { cudaError_t le_ = launch_pdl(k_update_scalar<false>, dim3(grid), dim3(kThreads), 0, st, g16, w32, nullptr, w16, n8 * 8, n, inv_S, lr, mu, flags, inv_S_dev); if (le_ != cudaSuccess) return le_; }
+            MPT_LAUNCH(k_update_scalar<false>, dim3(grid), dim3(kThreads), 0, st, g16, w32, nullptr, w16, n8 * 8, n, inv_S, lr, mu, flags, inv_S_dev);
     }
     return cudaGetLastError();
 }
@@ -397,13 +397,13 @@ static cudaError_t launch_opt_variant(const uint16_t *g16, float *w32, float *s1
     size_t n8 = (bits & 15) == 0 ? n / 8 : 0;
     if (n8) {
         const size_t per_cta = (size_t)kThreads * kOptVec;
-            { cudaError_t le_ = launch_pdl(k_update_opt<KIND, WD>, dim3((unsigned)((n8 + per_cta - 1) / per_cta)), dim3(kThreads), 0, st, 
-            (const uint4 *)g16, (float4 *)w32, (float4 *)s1, (float4 *)s2, (uint4 *)w16, n8, inv_S, lr, mu, b2, eps, wd, b1t, b2t,
-            flags, inv_dev, betat_dev, coef_dev); if (le_ != cudaSuccess) return le_; }
+        MPT_LAUNCH(k_update_opt<KIND, WD>, dim3((unsigned)((n8 + per_cta - 1) / per_cta)), dim3(kThreads), 0, st,
+                   (const uint4 *)g16, (float4 *)w32, (float4 *)s1, (float4 *)s2, (uint4 *)w16, n8, inv_S, lr, mu, b2, eps, wd, b1t, b2t,
+                   flags, inv_dev, betat_dev, coef_dev);
     }
     if (n8 * 8 < n)
-            { cudaError_t le_ = launch_pdl(k_update_opt_scalar<KIND, WD>, dim3(grid_for(n - n8 * 8)), dim3(kThreads), 0, st, g16, w32, s1, s2, w16, n8 * 8, n, inv_S, lr, mu, b2,
-                                                                                eps, wd, b1t, b2t, flags, inv_dev, betat_dev, coef_dev); if (le_ != cudaSuccess) return le_; }
+        MPT_LAUNCH(k_update_opt_scalar<KIND, WD>, dim3(grid_for(n - n8 * 8)), dim3(kThreads), 0, st, g16, w32, s1, s2, w16, n8 * 8, n, inv_S, lr, mu, b2,
+                   eps, wd, b1t, b2t, flags, inv_dev, betat_dev, coef_dev);
     return cudaGetLastError();
 }
 
@@ -458,7 +458,7 @@ __global__ void k_post_step(uint32_t *status, int interval, float backoff, float
 cudaError_t launch_post_step(uint32_t *status, int interval, float backoff, float growth, float min_S, float max_S, int adam,
                              float b1, float b2, cudaStream_t st)
 {
-            { cudaError_t le_ = launch_pdl(k_post_step, dim3(1), dim3(1), 0, st, status, interval, backoff, growth, min_S, max_S, adam, b1, b2); if (le_ != cudaSuccess) return le_; }
+    MPT_LAUNCH(k_post_step, dim3(1), dim3(1), 0, st, status, interval, backoff, growth, min_S, max_S, adam, b1, b2);
     return cudaGetLastError();
 }
 
@@ -489,7 +489,7 @@ __global__ void k_scale_adjust(uint32_t *status, int interval, float backoff, fl
 cudaError_t launch_scale_adjust(uint32_t *status, int interval, float backoff, float growth, float min_S, float max_S,
                                 cudaStream_t st)
 {
-            { cudaError_t le_ = launch_pdl(k_scale_adjust, dim3(1), dim3(1), 0, st, status, interval, backoff, growth, min_S, max_S); if (le_ != cudaSuccess) return le_; }
+    MPT_LAUNCH(k_scale_adjust, dim3(1), dim3(1), 0, st, status, interval, backoff, growth, min_S, max_S);
     return cudaGetLastError();
 }
 
@@ -565,8 +565,8 @@ cudaError_t launch_clip_coef(const uint16_t *g16, size_t n, float inv_S, const f
     const size_t n8 = ((uintptr_t)g16 & 15) == 0 ? n / 8 : 0;
     size_t want = (n8 + kThreads - 1) / kThreads;
     const int grid = (int)(want < 1 ? 1 : (want > (size_t)kNormParts ? (size_t)kNormParts : want));
-            { cudaError_t le_ = launch_pdl(k_grad_sqnorm, dim3(grid), dim3(kThreads), 0, st, g16, n, n8, inv_S, inv_dev, parts); if (le_ != cudaSuccess) return le_; }
-            { cudaError_t le_ = launch_pdl(k_clip_coef, dim3(1), dim3(1024), 0, st, parts, grid, clip, out2); if (le_ != cudaSuccess) return le_; }
+    MPT_LAUNCH(k_grad_sqnorm, dim3(grid), dim3(kThreads), 0, st, g16, n, n8, inv_S, inv_dev, parts);
+    MPT_LAUNCH(k_clip_coef, dim3(1), dim3(1024), 0, st, parts, grid, clip, out2);
     return cudaGetLastError();
 }
 
