@@ -606,3 +606,39 @@ void mpo_add_f16(const uint16_t *a, int lda, const uint16_t *b, int ldb, uint16_
             out[(size_t)r * ldo + n] = mpo_f2h(s);
         }
 }
+
+/*
+ * One data-parallel step over R replicas of the model (section 4.5 trains with a batch aggregated
+ * over 4 GPUs; the paper gives no formulas for the exchange, so the plain definition is used: the
+ * gradient of the mean loss over the aggregated batch is the mean of the replicas' gradients).
+ * Every replica holds a loss-scaled binary16 gradient g_q; per element, each line one separately
+ * rounded binary32 operation:
+ *   s = h2f(g_0[e]) ; for q = 1 .. R-1 in ascending order: s = s + h2f(g_q[e])
+ *   g = s * inv_SR                    inv_SR = 1 / (S * R), formed by the caller in binary32
+ *   then the momentum / plain lines of mpo_update_apply:  v, w32, w16 = rn16(w32)
+ * The sum stays in binary32 (it is never stored as binary16), so it cannot overflow when its
+ * terms are finite.  The caller decides the skip: this function must only be called when
+ * mpo_grad_nonfinite returned 0 for EVERY replica's gradient.
+ */
+void mpo_dp_update_apply(const uint16_t *const *g16, int R, float *w32, float *v, uint16_t *w16,
+                         size_t n, float inv_SR, float lr, float mu, int use_momentum)
+{
+#pragma omp parallel for schedule(static)
+    for (size_t e = 0; e < n; e++) {
+        float s = mpo_h2f(g16[0][e]);
+        for (int q = 1; q < R; q++) s = s + mpo_h2f(g16[q][e]);
+        float g = s * inv_SR;
+        float u;
+        if (use_momentum) {
+            float t = mu * v[e];
+            float nv = t + g;
+            v[e] = nv;
+            u = lr * nv;
+        } else {
+            u = lr * g;
+        }
+        float w = w32[e] - u;
+        w32[e] = w;
+        w16[e] = mpo_f2h(w);
+    }
+}

@@ -86,6 +86,9 @@ def lib() -> ctypes.CDLL:
         L.mpo_bias_grad.argtypes = [c.c_void_p, c.c_size_t, c.c_int, c.c_int, c.c_void_p, c.c_void_p]
         L.mpo_add_f16.restype = None
         L.mpo_add_f16.argtypes = [c.c_void_p, c.c_int, c.c_void_p, c.c_int, c.c_void_p, c.c_int, c.c_int, c.c_int]
+        L.mpo_dp_update_apply.restype = None
+        L.mpo_dp_update_apply.argtypes = [c.c_void_p, c.c_int, c.c_void_p, c.c_void_p, c.c_void_p, c.c_size_t,
+                                          c.c_float, c.c_float, c.c_float, c.c_int]
         _lib = L
     return _lib
 
@@ -306,3 +309,22 @@ def add_f16(a, b):
     out = np.zeros(a.shape, dtype=np.uint16)
     lib().mpo_add_f16(_ptr(a), _ld(a), _ptr(b), _ld(b), _ptr(out), a.shape[1], a.shape[0], a.shape[1])
     return out
+
+
+def dp_inv_scale(S, R) -> np.float32:
+    """1 / (S * R) in binary32: one multiplication, one division."""
+    return np.float32(1.0) / (np.float32(S) * np.float32(R))
+
+
+def dp_update_apply(g16_list, w32, v, w16, S, lr, mu, use_momentum) -> None:
+    """In-place data-parallel master update (see mpo.c): g16_list holds one contiguous gradient
+    array per replica, in replica order.  The caller has checked every replica's overflow flag."""
+    gs = [np.ascontiguousarray(_u16(g)).reshape(-1) for g in g16_list]
+    R = len(gs)
+    assert R >= 1 and all(g.size == gs[0].size for g in gs)
+    for a in (w32, w16) + ((v,) if v is not None else ()):
+        assert a.flags["C_CONTIGUOUS"]
+    assert w32.dtype == np.float32 and w16.dtype == np.uint16 and w32.size == gs[0].size
+    table = (ctypes.c_void_p * R)(*[g.ctypes.data for g in gs])
+    lib().mpo_dp_update_apply(table, R, _ptr(w32), _ptr(v) if use_momentum else None, _ptr(w16), gs[0].size,
+                              float(dp_inv_scale(S, R)), float(lr), float(mu), int(bool(use_momentum)))

@@ -1,0 +1,93 @@
+"""Pins for the oracle's data-parallel step (section 4.5: a batch aggregated over several GPUs):
+cases whose result is fixed by arithmetic that can be done by hand or by an already pinned routine."""
+import numpy as np
+
+from oracle import mpo
+from paper_1710_03740_b200 import inputs
+
+
+def _state(n, seed):
+    rng = np.random.default_rng(seed)
+    w32 = rng.standard_normal(n).astype(np.float32)
+    v = (0.1 * rng.standard_normal(n)).astype(np.float32)
+    return w32, v
+
+
+def test_one_replica_is_the_plain_update():
+    # R = 1: the sum has one term and 1/(S*1) = 1/S, so the step is the single-GPU update
+    n = 4099
+    g = inputs.loguniform_grads(n, 1024.0, seed=11).view(np.uint16)
+    w32, v = _state(n, 1)
+    wa, va, ha = w32.copy(), v.copy(), np.zeros(n, np.uint16)
+    wb, vb, hb = w32.copy(), v.copy(), np.zeros(n, np.uint16)
+    S = 1024.0
+    mpo.dp_update_apply([g], wa, va, ha, S, 0.05, 0.9, True)
+    mpo.update_apply(g, wb, vb, hb, np.float32(1.0) / np.float32(S), 0.05, 0.9, True)
+    assert np.array_equal(wa.view(np.uint32), wb.view(np.uint32))
+    assert np.array_equal(va.view(np.uint32), vb.view(np.uint32))
+    assert np.array_equal(ha, hb)
+
+
+def test_identical_replicas_power_of_two_equal_single_replica():
+    # R = 4 copies of the same gradient, S a power of two: the binary32 sum is exactly 4*g and
+    # 1/(4*S) is exact, so s * inv_SR == g * (1/S) exactly and the step equals the one-replica step
+    n = 2048 + 5
+    g = inputs.loguniform_grads(n, 256.0, seed=5).view(np.uint16)
+    w32, v = _state(n, 2)
+    wa, va, ha = w32.copy(), v.copy(), np.zeros(n, np.uint16)
+    wb, vb, hb = w32.copy(), v.copy(), np.zeros(n, np.uint16)
+    mpo.dp_update_apply([g, g.copy(), g.copy(), g.copy()], wa, va, ha, 256.0, 0.01, 0.5, True)
+    mpo.update_apply(g, wb, vb, hb, np.float32(1.0 / 256.0), 0.01, 0.5, True)
+    assert np.array_equal(wa.view(np.uint32), wb.view(np.uint32))
+    assert np.array_equal(va.view(np.uint32), vb.view(np.uint32))
+    assert np.array_equal(ha, hb)
+
+
+def test_mean_of_small_integers_is_exact():
+    # integer gradients, S = 1, R = 4, lr = 1, no momentum: every operation is exact, so
+    # w - mean(g) must come out exactly (computed here in float64)
+    rng = np.random.default_rng(3)
+    n, R = 1000, 4
+    gs = [rng.integers(-64, 65, n).astype(np.float16) for _ in range(R)]
+    w0 = rng.integers(-1000, 1000, n).astype(np.float32)
+    w, h = w0.copy(), np.zeros(n, np.uint16)
+    mpo.dp_update_apply([g.view(np.uint16) for g in gs], w, None, h, 1.0, 1.0, 0.0, False)
+    want = w0.astype(np.float64) - sum(g.astype(np.float64) for g in gs) / R
+    assert np.array_equal(w.astype(np.float64), want)
+    assert np.array_equal(h, want.astype(np.float16).view(np.uint16))
+
+
+def test_sum_runs_in_ascending_replica_order_in_binary32():
+    # replicas hold (65504, 2^-24, -65504): in ascending order the tiny term is absorbed by the
+    # first addition (2^-24 is far below half an ulp of 65504 in binary32) and the sum is exactly 0;
+    # any order that adds the two large terms first would leave 2^-24.  With S = 1, lr = 3 (so that
+    # lr * g / 3 is visible), w0 = 0: ascending order leaves w = 0, another order gives -2^-24.
+    big = np.array([65504.0], np.float16).view(np.uint16)
+    tiny = np.array([0x0001], np.uint16)
+    neg = np.array([-65504.0], np.float16).view(np.uint16)
+    w, h = np.zeros(1, np.float32), np.zeros(1, np.uint16)
+    mpo.dp_update_apply([big, tiny, neg], w, None, h, 1.0, 3.0, 0.0, False)
+    assert w[0] == 0.0 and h[0] == 0
+    w2, h2 = np.zeros(1, np.float32), np.zeros(1, np.uint16)
+    mpo.dp_update_apply([big, neg, tiny], w2, None, h2, 1.0, 3.0, 0.0, False)
+    # 1/(1*3) in binary32 times 2^-24 times 3 rounds back to 2^-24 (one ulp of slack allowed)
+    assert abs(float(w2[0]) + 2.0 ** -24) <= 2.0 ** -47
+
+
+def test_sum_is_not_rounded_to_binary16():
+    # two replicas with 40000 each: the sum 80000 exceeds the binary16 range but is a legal binary32
+    # intermediate; with S = 2 the unscaled mean is 20000 and w = 0 - 1 * 20000
+    g = np.array([40000.0], np.float16).view(np.uint16)
+    gval = float(g.view(np.float16)[0])     # 40000 is representable exactly in binary16
+    assert gval == 40000.0
+    w, h = np.zeros(1, np.float32), np.zeros(1, np.uint16)
+    mpo.dp_update_apply([g, g.copy()], w, None, h, 2.0, 1.0, 0.0, False)
+    assert w[0] == -20000.0
+    assert h[0] == np.array([-20000.0], np.float16).view(np.uint16)[0]
+
+
+def test_inverse_scale_is_one_division_of_the_binary32_product():
+    assert mpo.dp_inv_scale(128.0, 4) == np.float32(1.0 / 512.0)
+    # 3 replicas: 1/(S*3) is not exact; the value is the binary32 quotient, not a double rounded twice
+    x = mpo.dp_inv_scale(1.0, 3)
+    assert x == np.float32(1.0) / np.float32(3.0)
