@@ -370,7 +370,7 @@ def main():
             "last_loss": loss, "last_overflow": flag,
         }
         if world == 1 and not args.no_extras:
-            # not part of the step metric: the LSTM layer of the paper's language model (section 4.6),
+            # not part of the step metric: the LSTM layer of the paper's language model (section 4.5),
             # forward + backward through time, timed with CUDA events after the step benchmark
             try:
                 from paper_1710_03740_b200.kernel_bench import bench_lstm

@@ -344,7 +344,7 @@ int mpt_update_flat_opt(const mpt_optimizer *opt, const uint16_t *g16_dev, float
 
 /* ------------------------------------------------------------ LSTM layer with projection
  *
- * The recurrent layer of the paper's language model (section 4.6: 8192 cells projected to 1024)
+ * The recurrent layer of the paper's language model (section 4.5: 8192 cells projected to 1024)
  * in the mixed-precision recipe: FP16 storage, recurrent products with FP32 accumulation
  * (section 3.3), point-wise gate arithmetic in FP32 on the accumulators (section 3.3 leaves the
  * precision of memory-bound point-wise work open), reductions in FP32.  Per time step t:
@@ -463,6 +463,61 @@ int mpt_softmax_ce(const uint16_t *z_dev, int ldz, const int32_t *labels_dev, in
 int mpt_softmax_ce_static(const uint16_t *z_dev, int ldz, const int32_t *labels_dev, int B, int C, float S,
                           uint16_t *dz_dev, int lddz, float *loss_dev, uint32_t *bad_labels_dev,
                           void *cuda_stream);
+
+/* ------------------------------------------------------------ data-parallel step
+ *
+ * The paper's language model aggregates its batch over 4 GPUs (section 4.5); it gives no formulas
+ * for the exchange.  Here R replicas hold identical FP16 weights, each runs forward and scaled
+ * backward on its part of the batch, and ONE kernel per replica then does the gradient exchange,
+ * the master-weight pass and the weight broadcast for that replica's shard of the parameters:
+ *
+ *   shard:   mpt_dp_shard(n, R, q) = elements [lo, hi) owned by replica q; per-replica length is
+ *            ceil(ceil(n/8)/R)*8 (a multiple of 8, so every shard starts 16-byte aligned within
+ *            16-byte aligned arrays), the last shards may be short or empty
+ *   skip:    if ANY replica's overflow word is non-zero, nothing is written except flags_dev[0] = 1
+ *            (section 3.2: the step is skipped everywhere); the per-replica words are what the
+ *            weight-gradient epilogues (or mpt_grad_nonfinite) produced on each replica
+ *   element e of the shard, each line one separately rounded FP32 operation:
+ *            s = f32(g_0[e]) ; s = s + f32(g_q[e]) for q = 1 .. R-1 in ascending order
+ *            g = s * inv_SR          inv_SR = 1 / (S * R): one FP32 multiplication, one division
+ *            v = mu * v + g ; w32 = w32 - lr * v      (mu == 0 and v null: w32 = w32 - lr * g)
+ *            h = rn16(w32) ; w16_q[e] = h for every replica q (its own copy included)
+ *   The sum stays in FP32, so finite terms cannot overflow it.  Only the shard owner holds FP32
+ *   state for its shard: w32_shard / v_shard point at element lo (a replica may allocate the shard
+ *   alone, 8 instead of 8*R bytes per parameter across the job).
+ *
+ * g16_peers / flag_peers / w16_peers are HOST arrays of R DEVICE pointers in replica order; entry
+ * `rank` is this replica's own buffer, the others are peer mappings of the other replicas' buffers
+ * (all replicas use the same layout, n elements each).  Each gradient element crosses the link
+ * once (read by its owner), each FP16 weight once per peer (written by its owner); the kernel
+ * never waits on another replica.  Ordering is the caller's job: every replica's gradients and
+ * overflow word must be complete before any replica calls this, and every replica's call must
+ * have completed before any replica reads its weights or clears its overflow word (a stream-
+ * ordered barrier across the replicas on both sides).  flags_dev: device uint32[2] of this
+ * replica; [0] receives the OR of all replicas' words, [1] the kernel's own inspection of the
+ * unscaled mean gradients it formed (must have been zeroed by the caller).  flags_dev may be the
+ * same memory as flag_peers[rank]: the kernel only ever sets bits there.
+ * Errors: MPT_ERR_INVALID_ARG for R outside [1, MPT_DP_MAX_REPLICAS], rank outside [0, R), a null or
+ * misaligned (16 bytes) pointer; MPT_ERR_CUDA if the launch fails. */
+#define MPT_DP_MAX_REPLICAS 16
+int mpt_dp_shard(size_t n, int R, int rank, size_t *lo_out, size_t *hi_out);
+int mpt_dp_step_flat(const uint16_t *const *g16_peers, const uint32_t *const *flag_peers, uint16_t *const *w16_peers,
+                     float *w32_shard_dev, float *v_shard_dev, size_t n, int R, int rank, float S, float lr, float mu,
+                     uint32_t *flags_dev, void *cuda_stream);
+
+/* Device memory that other processes can map (the buffers the replicas exchange).  mpt_dp_alloc
+ * returns memory from the driver's allocator (not from a framework's pool, whose blocks cannot be
+ * exported); mpt_dp_export writes an opaque MPT_DP_HANDLE_BYTES handle for the allocation that
+ * contains dev_ptr - dev_ptr must be the pointer mpt_dp_alloc returned; mpt_dp_open maps another
+ * PROCESS's allocation (on this or another GPU with peer access) and returns a device pointer
+ * valid in the calling process; mpt_dp_close unmaps it.  The owner frees with mpt_dp_free only
+ * after every peer has closed its mapping.  Errors: MPT_ERR_INVALID_ARG, MPT_ERR_CUDA. */
+#define MPT_DP_HANDLE_BYTES 64
+int mpt_dp_alloc(size_t bytes, void **dev_ptr_out);
+int mpt_dp_free(void *dev_ptr);
+int mpt_dp_export(const void *dev_ptr, uint8_t *handle_out);
+int mpt_dp_open(const uint8_t *handle, void **dev_ptr_out);
+int mpt_dp_close(void *dev_ptr);
 
 /* Library build identification, e.g. "mpt 0.1 sm_100a". */
 const char *mpt_version(void);

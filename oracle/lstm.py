@@ -1,7 +1,7 @@
 """One LSTM layer with a projection, unrolled over time, in the mixed-precision recipe, on the CPU.
 
 TEST INFRASTRUCTURE ONLY (see mpo.c).  The layer is the recurrent layer of the paper's language
-model (section 4.6: 8192 cells projected to 1024): per time step
+model (section 4.5: 8192 cells projected to 1024): per time step
 
   [x_t ; r_{t-1}] . Wg^T + b  ->  gates  ->  c_t, h_t          (mpo_lstm_cell_fwd)
   r_t = rn16(h_t . Wp^T)                                          (FP32 accumulate, FP16 store)

@@ -458,7 +458,7 @@ void mpo_update_apply_clip(int kind, const uint16_t *g16, float *w32, float *s1,
 }
 
 /* ------------------------------------------------------------------------
- * LSTM cell with fused gate arithmetic (sections 3.3 and 4.6: recurrent matrix products on
+ * LSTM cell with fused gate arithmetic (sections 3.3 and 4.5: recurrent matrix products on
  * FP16 inputs with FP32 accumulation; point-wise gate arithmetic is memory-bound and may run
  * in either precision - here FP32 arithmetic on FP16 storage).
  *

@@ -33,7 +33,8 @@ EXPORTS = ["mpt_workspace_bytes", "mpt_create", "mpt_workspace_bytes_opt", "mpt_
            "mpt_destroy", "mpt_gemm_f16", "mpt_gemm_f16_ws", "mpt_gemm_workspace_bytes", "mpt_recast", "mpt_grad_nonfinite", "mpt_update_flat",
            "mpt_softmax_ce", "mpt_softmax_ce_static", "mpt_version",
            "mpt_lstm_forward", "mpt_lstm_backward", "mpt_lstm_cell_forward", "mpt_lstm_cell_backward", "mpt_bias_grad",
-           "mpt_add_f16"]
+           "mpt_add_f16",
+           "mpt_dp_shard", "mpt_dp_step_flat", "mpt_dp_alloc", "mpt_dp_free", "mpt_dp_export", "mpt_dp_open", "mpt_dp_close"]
 
 
 class MptError(RuntimeError):
@@ -123,6 +124,13 @@ def lib() -> C.CDLL:
     L.mpt_lstm_cell_backward.argtypes = [i32, i32, vp, i32, vp, i32, vp, i32, vp, i32, vp, i32, vp, i32, vp, i32, vp]
     L.mpt_bias_grad.argtypes = [vp, sz, i32, i32, vp, vp, vp, vp]
     L.mpt_add_f16.argtypes = [vp, i32, vp, i32, vp, i32, i32, i32, vp]
+    L.mpt_dp_shard.argtypes = [sz, i32, i32, C.POINTER(sz), C.POINTER(sz)]
+    L.mpt_dp_step_flat.argtypes = [vp, vp, vp, vp, vp, sz, i32, i32, f32, f32, f32, vp, vp]
+    L.mpt_dp_alloc.argtypes = [sz, C.POINTER(vp)]
+    L.mpt_dp_free.argtypes = [vp]
+    L.mpt_dp_export.argtypes = [vp, vp]
+    L.mpt_dp_open.argtypes = [vp, C.POINTER(vp)]
+    L.mpt_dp_close.argtypes = [vp]
     L.mpt_version.restype = C.c_char_p
     L.mpt_version.argtypes = []
     _lib = L
@@ -443,3 +451,150 @@ class LstmLayer:
 
     def device_error(self) -> int:
         return int(self.status[3].item())
+
+
+# ------------------------------------------------------------------ data-parallel step
+
+DP_MAX_REPLICAS = 16
+DP_HANDLE_BYTES = 64
+
+
+def mpt_dp_shard(n, R, rank):
+    """Elements [lo, hi) of the flat parameter array that replica `rank` of R owns (host only)."""
+    lo, hi = C.c_size_t(0), C.c_size_t(0)
+    _check(lib().mpt_dp_shard(int(n), int(R), int(rank), C.byref(lo), C.byref(hi)))
+    return int(lo.value), int(hi.value)
+
+
+def _addr(x):
+    """Device address of a tensor, a DeviceBuffer or a plain integer."""
+    if isinstance(x, int):
+        return x
+    if isinstance(x, DeviceBuffer):
+        return x.ptr
+    return x.data_ptr()
+
+
+def mpt_dp_step_flat(g16_peers, flag_peers, w16_peers, w32_shard, v_shard, n, R, rank, S, lr, mu, flags, stream=None):
+    """One replica's part of the data-parallel step: the *_peers arguments are sequences of R device
+    buffers (tensors, DeviceBuffers or addresses) in replica order, entry `rank` being this replica's."""
+    assert len(g16_peers) == R and len(flag_peers) == R and len(w16_peers) == R
+    tab = lambda xs: (C.c_void_p * R)(*[_addr(x) for x in xs])
+    _check(lib().mpt_dp_step_flat(tab(g16_peers), tab(flag_peers), tab(w16_peers),
+                                  None if w32_shard is None else C.c_void_p(_addr(w32_shard)),
+                                  None if v_shard is None else C.c_void_p(_addr(v_shard)),
+                                  int(n), int(R), int(rank), float(S), float(lr), float(mu), C.c_void_p(_addr(flags)),
+                                  _stream_ptr(stream)))
+
+
+class DeviceBuffer:
+    """Device memory that other processes can map: either this process's own allocation (made by
+    the library from the driver's allocator) or a mapping of a peer's, opened from its handle.
+    `tensor(dtype)` views it as a torch tensor without copying."""
+
+    def __init__(self, nbytes=None, handle=None):
+        p = C.c_void_p(0)
+        if handle is None:
+            _check(lib().mpt_dp_alloc(int(nbytes), C.byref(p)))
+            self.owned = True
+        else:
+            assert len(handle) == DP_HANDLE_BYTES
+            buf = (C.c_uint8 * DP_HANDLE_BYTES).from_buffer_copy(handle)
+            _check(lib().mpt_dp_open(buf, C.byref(p)))
+            self.owned = False
+        self.ptr = int(p.value)
+        self.nbytes = nbytes
+
+    def export(self) -> bytes:
+        assert self.owned
+        buf = (C.c_uint8 * DP_HANDLE_BYTES)()
+        _check(lib().mpt_dp_export(C.c_void_p(self.ptr), buf))
+        return bytes(buf)
+
+    def tensor(self, dtype, count=None):
+        import torch
+        item = torch.empty((), dtype=dtype).element_size()
+        n = self.nbytes // item if count is None else int(count)
+        typestr = {torch.uint8: "|u1", torch.int16: "<i2", torch.float16: "<f2", torch.float32: "<f4",
+                   torch.int32: "<i4", torch.uint16: "<u2"}[dtype]
+
+        class _View:
+            __cuda_array_interface__ = dict(shape=(n,), typestr=typestr, data=(self.ptr, False), version=2)
+
+        return torch.as_tensor(_View(), device="cuda")
+
+    def close(self):
+        if self.ptr:
+            if self.owned:
+                _check(lib().mpt_dp_free(C.c_void_p(self.ptr)))
+            else:
+                _check(lib().mpt_dp_close(C.c_void_p(self.ptr)))
+            self.ptr = 0
+
+
+def dp_exchange_handles(handles: dict, group=None):
+    """All-gather of each replica's {name: handle bytes} through torch.distributed (any backend):
+    returns a list over replicas of such dicts, in rank order."""
+    import torch.distributed as dist
+    out = [None] * dist.get_world_size(group)
+    dist.all_gather_object(out, handles, group=group)
+    return out
+
+
+class DataParallelFlat:
+    """Replica `rank` of R for a flat parameter array of n elements: owns the exchange buffers
+    (scaled FP16 gradient, FP16 weights, overflow words), maps the peers' buffers, holds the FP32
+    master and momentum of its own shard only, and runs the one-kernel step.  Replicas are
+    processes of a torch.distributed group (one per GPU); the group's barrier orders them around
+    the step (host-synchronous: the stream is drained first)."""
+
+    def __init__(self, n, S, lr, mu, group=None):
+        import torch
+        import torch.distributed as dist
+        self.group = group
+        self.R, self.rank = dist.get_world_size(group), dist.get_rank(group)
+        self.n, self.S, self.lr, self.mu = int(n), float(S), float(lr), float(mu)
+        self.lo, self.hi = mpt_dp_shard(n, self.R, self.rank)
+        pad = (self.n + 7) // 8 * 16
+        self._own = dict(g16=DeviceBuffer(pad), w16=DeviceBuffer(pad), flags=DeviceBuffer(256))
+        self.g16 = self._own["g16"].tensor(torch.int16, self.n)
+        self.w16 = self._own["w16"].tensor(torch.int16, self.n)
+        self.flags = self._own["flags"].tensor(torch.int32, 2)
+        self.flags.zero_()
+        cnt = max(self.hi - self.lo, 1)
+        self.w32 = torch.zeros(cnt, dtype=torch.float32, device="cuda")
+        self.v = torch.zeros(cnt, dtype=torch.float32, device="cuda") if self.mu != 0.0 else None
+        table = dp_exchange_handles({k: b.export() for k, b in self._own.items()}, group)
+        self._peers = []
+        for q in range(self.R):
+            self._peers.append(self._own if q == self.rank else {k: DeviceBuffer(handle=h) for k, h in table[q].items()})
+
+    def _barrier(self):
+        import torch
+        import torch.distributed as dist
+        torch.cuda.current_stream().synchronize()
+        dist.barrier(group=self.group)
+
+    def step(self):
+        """Gradients (self.g16) and overflow word (self.flags[0]) of every replica must have been
+        produced on the current stream.  Returns True when the step was skipped everywhere."""
+        self._barrier()
+        mpt_dp_step_flat([p["g16"] for p in self._peers], [p["flags"] for p in self._peers],
+                         [p["w16"] for p in self._peers], self.w32, self.v, self.n, self.R, self.rank, self.S,
+                         self.lr, self.mu, self._own["flags"])
+        self._barrier()
+        # every replica's kernel has finished: nobody reads this word again before the next step's
+        # first barrier, which also drains the stream the clear is queued on
+        skipped = bool(int(self.flags[0].item()) != 0)
+        self.flags.zero_()
+        return skipped
+
+    def close(self):
+        self._barrier()
+        for q, p in enumerate(self._peers):
+            if q != self.rank:
+                for b in p.values():
+                    b.close()
+        self._barrier()
+        for b in self._own.values():
+            b.close()

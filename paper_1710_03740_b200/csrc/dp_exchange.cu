@@ -1,0 +1,252 @@
+// Data-parallel step (the paper's language model aggregates its batch over 4 GPUs, section 4.5):
+// gradient exchange, master-weight pass and weight broadcast for one replica's shard of the
+// parameters in ONE kernel over peer memory.  The owner of a shard pulls that shard of every
+// replica's FP16 gradient (each element crosses the link once), adds them in FP32 in replica order,
+// applies the update of sections 3.1 / 3.2 to its FP32 master shard, and pushes the re-rounded FP16
+// weights into every replica's working copy.  Plain loads and stores on peer pointers only: no
+// waits on other replicas inside the kernel (the caller orders the replicas around the call), no
+// multicast.  Arithmetic contract: include/mpt.h (mpt_dp_step_flat).
+#include <string.h>
+
+#include "mpt_common.cuh"
+
+namespace mpt {
+
+namespace {
+
+constexpr int kDpThreads = 256;
+
+struct DpPeers {
+    const uint16_t *g[MPT_DP_MAX_REPLICAS];
+    const uint32_t *flag[MPT_DP_MAX_REPLICAS];
+    uint16_t *w[MPT_DP_MAX_REPLICAS];
+};
+
+__device__ __forceinline__ float h2f_bits_dp(uint32_t h) { return __half2float(__ushort_as_half((unsigned short)h)); }
+__device__ __forceinline__ uint32_t f2h_bits_dp(float x) { return (uint32_t)__half_as_ushort(__float2half_rn(x)); }
+
+// one element: s is the FP32 sum of the replicas' scaled gradients
+template <bool MOM>
+__device__ __forceinline__ void dp_elem(float s, float inv, float lr, float mu, float &w, float &v, bool &bad)
+{
+    const float g = __fmul_rn(s, inv);
+    bad |= f32_nonfinite(g);
+    float u;
+    if (MOM) {
+        v = __fadd_rn(__fmul_rn(mu, v), g);
+        u = __fmul_rn(lr, v);
+    } else {
+        u = __fmul_rn(lr, g);
+    }
+    w = __fsub_rn(w, u);
+}
+
+__device__ __forceinline__ bool any_replica_overflowed(const DpPeers &pp, int R)
+{
+    uint32_t any = 0;
+    for (int q = 0; q < R; q++) any |= *(volatile const uint32_t *)pp.flag[q];
+    return any != 0;
+}
+
+// RT: replica count known at compile time (the loads of all replicas are then issued before the
+// first addition), 0: any count.  `first` is the index of the shard's first element in the
+// replicas' full-length arrays; w32 / v point at that element of the owner's state.
+template <int RT, bool MOM>
+__global__ void __launch_bounds__(kDpThreads) k_dp_step(const DpPeers pp, int R_dyn, float4 *__restrict__ w32,
+                                                        float4 *__restrict__ v, size_t first, size_t n8, float inv,
+                                                        float lr, float mu, uint32_t *flags)
+{
+    pdl_trigger();
+    pdl_wait();
+    const int R = RT ? RT : R_dyn;
+    if (any_replica_overflowed(pp, R)) {
+        if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(flags, 1u);
+        return;
+    }
+    const size_t j = (size_t)blockIdx.x * kDpThreads + threadIdx.x;
+    if (j >= n8) return;
+    const size_t vec = first / 8 + j;          // `first` is a multiple of 8
+    float s[8];
+    if (RT) {
+        uint4 g[RT ? RT : 1];
+#pragma unroll
+        for (int q = 0; q < RT; q++) g[q] = __ldcs((const uint4 *)pp.g[q] + vec);
+#pragma unroll
+        for (int q = 0; q < RT; q++) {
+            const uint32_t gw[4] = {g[q].x, g[q].y, g[q].z, g[q].w};
+#pragma unroll
+            for (int e = 0; e < 8; e++) {
+                const float x = h2f_bits_dp((e & 1) ? (gw[e >> 1] >> 16) : (gw[e >> 1] & 0xFFFFu));
+                s[e] = q == 0 ? x : __fadd_rn(s[e], x);
+            }
+        }
+    } else {
+        for (int q = 0; q < R; q++) {
+            const uint4 g = __ldcs((const uint4 *)pp.g[q] + vec);
+            const uint32_t gw[4] = {g.x, g.y, g.z, g.w};
+#pragma unroll
+            for (int e = 0; e < 8; e++) {
+                const float x = h2f_bits_dp((e & 1) ? (gw[e >> 1] >> 16) : (gw[e >> 1] & 0xFFFFu));
+                s[e] = q == 0 ? x : __fadd_rn(s[e], x);
+            }
+        }
+    }
+    float4 w0 = __ldcs(w32 + 2 * j), w1 = __ldcs(w32 + 2 * j + 1);
+    float4 v0 = make_float4(0, 0, 0, 0), v1 = v0;
+    if (MOM) { v0 = __ldcs(v + 2 * j); v1 = __ldcs(v + 2 * j + 1); }
+    bool bad = false;
+    float *wf[2] = {&w0.x, &w1.x}, *vf[2] = {&v0.x, &v1.x};
+#pragma unroll
+    for (int e = 0; e < 8; e++) dp_elem<MOM>(s[e], inv, lr, mu, wf[e >> 2][e & 3], vf[e >> 2][e & 3], bad);
+    uint4 h;
+    h.x = f2h_bits_dp(w0.x) | (f2h_bits_dp(w0.y) << 16);
+    h.y = f2h_bits_dp(w0.z) | (f2h_bits_dp(w0.w) << 16);
+    h.z = f2h_bits_dp(w1.x) | (f2h_bits_dp(w1.y) << 16);
+    h.w = f2h_bits_dp(w1.z) | (f2h_bits_dp(w1.w) << 16);
+    __stcs(w32 + 2 * j, w0);
+    __stcs(w32 + 2 * j + 1, w1);
+    if (MOM) { __stcs(v + 2 * j, v0); __stcs(v + 2 * j + 1, v1); }
+    if (RT) {
+#pragma unroll
+        for (int q = 0; q < RT; q++) __stcs((uint4 *)pp.w[q] + vec, h);
+    } else {
+        for (int q = 0; q < R; q++) __stcs((uint4 *)pp.w[q] + vec, h);
+    }
+    if (__any_sync(__activemask(), bad) && (threadIdx.x & 31) == 0) atomicOr(flags + 1, 1u);
+}
+
+// the up to seven elements after the last whole vector of a shard (one warp)
+template <bool MOM>
+__global__ void k_dp_step_tail(const DpPeers pp, int R, float *__restrict__ w32, float *__restrict__ v, size_t first,
+                               size_t begin, size_t count, float inv, float lr, float mu, uint32_t *flags)
+{
+    pdl_trigger();
+    pdl_wait();
+    if (any_replica_overflowed(pp, R)) {
+        if (threadIdx.x == 0) atomicOr(flags, 1u);
+        return;
+    }
+    bool bad = false;
+    for (size_t i = begin + threadIdx.x; i < count; i += blockDim.x) {
+        float s = h2f_bits_dp(pp.g[0][first + i]);
+        for (int q = 1; q < R; q++) s = __fadd_rn(s, h2f_bits_dp(pp.g[q][first + i]));
+        float w = w32[i], m = MOM ? v[i] : 0.0f;
+        dp_elem<MOM>(s, inv, lr, mu, w, m, bad);
+        w32[i] = w;
+        if (MOM) v[i] = m;
+        const uint16_t h = (uint16_t)f2h_bits_dp(w);
+        for (int q = 0; q < R; q++) pp.w[q][first + i] = h;
+    }
+    if (bad) atomicOr(flags + 1, 1u);
+}
+
+template <bool MOM>
+cudaError_t launch_dp(const DpPeers &pp, int R, float *w32, float *v, size_t first, size_t count, float inv, float lr,
+                      float mu, uint32_t *flags, cudaStream_t st)
+{
+    const size_t n8 = count / 8;
+    if (n8) {
+        const dim3 grid((unsigned)((n8 + kDpThreads - 1) / kDpThreads)), block(kDpThreads);
+        switch (R) {
+            case 2: MPT_LAUNCH(k_dp_step<2, MOM>, grid, block, 0, st, pp, R, (float4 *)w32, (float4 *)v, first, n8, inv, lr, mu, flags); break;
+            case 4: MPT_LAUNCH(k_dp_step<4, MOM>, grid, block, 0, st, pp, R, (float4 *)w32, (float4 *)v, first, n8, inv, lr, mu, flags); break;
+            case 8: MPT_LAUNCH(k_dp_step<8, MOM>, grid, block, 0, st, pp, R, (float4 *)w32, (float4 *)v, first, n8, inv, lr, mu, flags); break;
+            default: MPT_LAUNCH(k_dp_step<0, MOM>, grid, block, 0, st, pp, R, (float4 *)w32, (float4 *)v, first, n8, inv, lr, mu, flags); break;
+        }
+    }
+    // also for an empty shard: the launch then only publishes the skip decision in this replica's flags
+    if (n8 * 8 < count || count == 0)
+        MPT_LAUNCH(k_dp_step_tail<MOM>, dim3(1), dim3(32), 0, st, pp, R, w32, v, first, n8 * 8, count, inv, lr, mu, flags);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+}  // namespace mpt
+
+using namespace mpt;
+
+extern "C" {
+
+int mpt_dp_shard(size_t n, int R, int rank, size_t *lo_out, size_t *hi_out)
+{
+    if (R < 1 || R > MPT_DP_MAX_REPLICAS || rank < 0 || rank >= R || !lo_out || !hi_out) return MPT_ERR_INVALID_ARG;
+    const size_t vecs = (n + 7) / 8;
+    const size_t per = ((vecs + (size_t)R - 1) / (size_t)R) * 8;
+    size_t lo = per * (size_t)rank, hi = lo + per;
+    if (lo > n) lo = n;
+    if (hi > n) hi = n;
+    *lo_out = lo;
+    *hi_out = hi;
+    return MPT_OK;
+}
+
+int mpt_dp_step_flat(const uint16_t *const *g16_peers, const uint32_t *const *flag_peers, uint16_t *const *w16_peers,
+                     float *w32_shard_dev, float *v_shard_dev, size_t n, int R, int rank, float S, float lr, float mu,
+                     uint32_t *flags_dev, void *cuda_stream)
+{
+    if (!g16_peers || !flag_peers || !w16_peers || !flags_dev) return MPT_ERR_INVALID_ARG;
+    size_t lo = 0, hi = 0;
+    if (mpt_dp_shard(n, R, rank, &lo, &hi) != MPT_OK) return MPT_ERR_INVALID_ARG;
+    if (!(S > 0.0f) || !(lr == lr) || !(mu == mu)) return MPT_ERR_INVALID_ARG;
+    const bool mom = mu != 0.0f;
+    DpPeers pp = {};
+    for (int q = 0; q < R; q++) {
+        if (!g16_peers[q] || !flag_peers[q] || !w16_peers[q]) return MPT_ERR_INVALID_ARG;
+        if ((((uintptr_t)g16_peers[q] | (uintptr_t)w16_peers[q]) & 15) != 0 || ((uintptr_t)flag_peers[q] & 3) != 0)
+            return MPT_ERR_INVALID_ARG;
+        pp.g[q] = g16_peers[q];
+        pp.flag[q] = flag_peers[q];
+        pp.w[q] = w16_peers[q];
+    }
+    const size_t count = hi - lo;
+    if (count && (!w32_shard_dev || (mom && !v_shard_dev))) return MPT_ERR_INVALID_ARG;
+    if (count && (((uintptr_t)w32_shard_dev | (uintptr_t)v_shard_dev) & 15) != 0) return MPT_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    cudaError_t e = cudaMemsetAsync(flags_dev + 1, 0, sizeof(uint32_t), st);
+    if (e != cudaSuccess) return MPT_ERR_CUDA;
+    const float inv = 1.0f / (S * (float)R);
+    e = mom ? launch_dp<true>(pp, R, w32_shard_dev, v_shard_dev, lo, count, inv, lr, mu, flags_dev, st)
+            : launch_dp<false>(pp, R, w32_shard_dev, nullptr, lo, count, inv, lr, mu, flags_dev, st);
+    return e == cudaSuccess ? MPT_OK : MPT_ERR_CUDA;
+}
+
+int mpt_dp_alloc(size_t bytes, void **dev_ptr_out)
+{
+    if (!dev_ptr_out || bytes == 0) return MPT_ERR_INVALID_ARG;
+    *dev_ptr_out = nullptr;
+    return cudaMalloc(dev_ptr_out, bytes) == cudaSuccess ? MPT_OK : MPT_ERR_CUDA;
+}
+
+int mpt_dp_free(void *dev_ptr)
+{
+    if (!dev_ptr) return MPT_ERR_INVALID_ARG;
+    return cudaFree(dev_ptr) == cudaSuccess ? MPT_OK : MPT_ERR_CUDA;
+}
+
+int mpt_dp_export(const void *dev_ptr, uint8_t *handle_out)
+{
+    static_assert(sizeof(cudaIpcMemHandle_t) == MPT_DP_HANDLE_BYTES, "handle size");
+    if (!dev_ptr || !handle_out) return MPT_ERR_INVALID_ARG;
+    cudaIpcMemHandle_t h;
+    if (cudaIpcGetMemHandle(&h, const_cast<void *>(dev_ptr)) != cudaSuccess) return MPT_ERR_CUDA;
+    memcpy(handle_out, &h, sizeof(h));
+    return MPT_OK;
+}
+
+int mpt_dp_open(const uint8_t *handle, void **dev_ptr_out)
+{
+    if (!handle || !dev_ptr_out) return MPT_ERR_INVALID_ARG;
+    cudaIpcMemHandle_t h;
+    memcpy(&h, handle, sizeof(h));
+    *dev_ptr_out = nullptr;
+    return cudaIpcOpenMemHandle(dev_ptr_out, h, cudaIpcMemLazyEnablePeerAccess) == cudaSuccess ? MPT_OK : MPT_ERR_CUDA;
+}
+
+int mpt_dp_close(void *dev_ptr)
+{
+    if (!dev_ptr) return MPT_ERR_INVALID_ARG;
+    return cudaIpcCloseMemHandle(dev_ptr) == cudaSuccess ? MPT_OK : MPT_ERR_CUDA;
+}
+
+}  // extern "C"

@@ -1,4 +1,4 @@
-// LSTM layer pieces outside the tensor-core products (sections 3.3, 4.6 of the paper): the
+// LSTM layer pieces outside the tensor-core products (sections 3.3, 4.5 of the paper): the
 // backward of the gate arithmetic, the FP32 bias-gradient reduction, the FP16 add of two
 // gradient contributions, and a plain-CUDA-core forward cell for shapes the tensor-core
 // kernels do not take.  All of them are memory-bound streaming kernels on FP16 storage with

@@ -256,7 +256,7 @@ __device__ __forceinline__ void epilogue_store32_coalesced(const uint32_t (&r)[3
     __syncwarp();    // the block may be overwritten by the next call
 }
 
-// LSTM gate arithmetic on FP32 values (sections 3.3, 4.6): one cell from its four pre-activations
+// LSTM gate arithmetic on FP32 values (sections 3.3, 4.5): one cell from its four pre-activations
 // (bias already added).  Returns the FP16 bit patterns of the gate activations in act[4], the new
 // cell state and the hidden state; h uses the STORED (rounded) cell state.
 // The gate functions are evaluated with the hardware exp2 and reciprocal approximations (about

@@ -146,7 +146,7 @@ def gemm_operands(op, M, N, K, seed=2, scale_a=None, scale_b=None, fast=False):
             normal_f16(np.random.default_rng(seqs[1]), shape_b, sb))
 
 
-# LSTM layer with projection (the recurrent layer of the language model of section 4.6: 8192 cells
+# LSTM layer with projection (the recurrent layer of the language model of section 4.5: 8192 cells
 # projected to 1024, input width 1024; the batch of 1024 there is spread over 4 GPUs with 20
 # unrolled steps).  "small" spans several tiles with ragged edges and finishes on the CPU in
 # seconds; "biglstm" is the paper's layer with 2048 rows per step.

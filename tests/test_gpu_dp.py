@@ -1,0 +1,207 @@
+"""Data-parallel step (section 4.5: a batch aggregated over several GPUs) against the oracle,
+bit for bit.  With one GPU the replicas are emulated: every replica's buffers live on the same
+device and the per-replica calls run one after another (the kernel never waits on a peer, so the
+order of the calls does not matter).  A second test runs two replicas as two PROCESSES that map
+each other's buffers."""
+import os
+import socket
+
+import numpy as np
+import pytest
+
+from oracle import mpo
+from gpu_util import dev, host_u16, require_gpu, torch
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _gpu():
+    require_gpu()
+
+
+def _binding():
+    from paper_1710_03740_b200 import binding
+    return binding
+
+
+def _inputs(n, R, seed):
+    rng = np.random.default_rng(seed)
+    gs = []
+    for q in range(R):
+        mag = np.exp2(rng.uniform(-20.0, 4.0, n))
+        gs.append((mag * rng.choice([-1.0, 1.0], n)).astype(np.float32).astype(np.float16))
+    w = rng.standard_normal(n).astype(np.float32)
+    v = (0.1 * rng.standard_normal(n)).astype(np.float32)
+    return gs, w, v
+
+
+def _emulate(n, R, S, lr, mu, gs, w, v, flag_words=None, order=None):
+    """Run the R per-replica calls on one device.  Returns (w32, v, [w16 per replica], [flags per replica])."""
+    b = _binding()
+    npad = n + 8
+    g_dev = [torch.zeros(npad, dtype=torch.int16, device="cuda") for _ in range(R)]
+    h_dev = [torch.full((npad,), 0x1234, dtype=torch.int16, device="cuda") for _ in range(R)]
+    f_dev = [torch.zeros(2, dtype=torch.int32, device="cuda") for _ in range(R)]
+    for q in range(R):
+        if n:
+            g_dev[q][:n] = dev(gs[q].view(np.uint16))
+        if flag_words is not None:
+            f_dev[q][0] = int(flag_words[q])
+    w_full = torch.zeros(npad, dtype=torch.float32, device="cuda")
+    v_full = torch.zeros(npad, dtype=torch.float32, device="cuda")
+    if n:
+        w_full[:n] = dev(w)
+        v_full[:n] = dev(v)
+    for q in (order if order is not None else range(R)):
+        lo, hi = b.mpt_dp_shard(n, R, q)
+        # the shard owner's state: here a slice of one array; lo is a multiple of 8, so it stays aligned
+        b.mpt_dp_step_flat(g_dev, f_dev, h_dev, w_full[lo:], v_full[lo:] if mu != 0.0 else None, n, R, q, S, lr, mu, f_dev[q])
+    torch.cuda.synchronize()
+    return (w_full[:n].cpu().numpy(), v_full[:n].cpu().numpy(), [host_u16(h[:n]) for h in h_dev],
+            [f.cpu().numpy() for f in f_dev], [host_u16(h[n:]) for h in h_dev])
+
+
+def _oracle(n, R, S, lr, mu, gs, w, v):
+    w32, vv, w16 = w.copy(), v.copy(), np.zeros(n, np.uint16)
+    mpo.dp_update_apply([g.view(np.uint16) for g in gs], w32, vv if mu != 0.0 else None, w16, S, lr, mu, mu != 0.0)
+    return w32, vv, w16
+
+
+@pytest.mark.parametrize("mu", [0.0, 0.9])
+@pytest.mark.parametrize("R", [1, 2, 3, 4, 8, 16])
+@pytest.mark.parametrize("n", [5, 8 * 256 * 2 + 3, (1 << 20) + 13])
+def test_dp_step_bit_exact(n, R, mu):
+    S, lr = 1024.0, 0.05
+    gs, w, v = _inputs(n, R, seed=n + 31 * R)
+    w32, vv, w16s, flags, guard = _emulate(n, R, S, lr, mu, gs, w, v)
+    rw, rv, rh = _oracle(n, R, S, lr, mu, gs, w, v)
+    assert np.array_equal(w32.view(np.uint32), rw.view(np.uint32))
+    if mu != 0.0:
+        assert np.array_equal(vv.view(np.uint32), rv.view(np.uint32))
+    else:
+        assert np.array_equal(vv.view(np.uint32), v.view(np.uint32))       # untouched
+    for q in range(R):
+        assert np.array_equal(w16s[q], rh), "replica %d's FP16 weights" % q
+        assert np.all(guard[q] == 0x1234)                                   # nothing written past n
+        assert flags[q][0] == 0 and flags[q][1] == 0
+
+
+def test_dp_order_of_calls_does_not_matter():
+    n, R, S, lr, mu = 4099, 4, 256.0, 0.01, 0.5
+    gs, w, v = _inputs(n, R, seed=9)
+    a = _emulate(n, R, S, lr, mu, gs, w, v)
+    b = _emulate(n, R, S, lr, mu, gs, w, v, order=[3, 1, 0, 2])
+    assert np.array_equal(a[0].view(np.uint32), b[0].view(np.uint32))
+    assert all(np.array_equal(x, y) for x, y in zip(a[2], b[2]))
+
+
+@pytest.mark.parametrize("bad_replica", [0, 2])
+def test_dp_skip_when_any_replica_overflowed(bad_replica):
+    # section 3.2: an overflow anywhere skips the update everywhere; nothing but the flags changes
+    n, R, S, lr, mu = 3000, 3, 1024.0, 0.05, 0.9
+    gs, w, v = _inputs(n, R, seed=4)
+    gs[bad_replica][17] = np.float16(np.inf)
+    words = [0] * R
+    words[bad_replica] = 1          # what that replica's weight-gradient epilogue reported
+    w32, vv, w16s, flags, _ = _emulate(n, R, S, lr, mu, gs, w, v, flag_words=words)
+    assert np.array_equal(w32.view(np.uint32), w.view(np.uint32))
+    assert np.array_equal(vv.view(np.uint32), v.view(np.uint32))
+    for q in range(R):
+        assert np.all(w16s[q] == 0x1234)
+        assert flags[q][0] != 0
+
+
+def test_dp_kernel_reports_a_nonfinite_mean_it_meets():
+    # a non-finite gradient that no replica flagged: the owner of that element sees it in flags[1]
+    n, R = 2048, 2
+    gs, w, v = _inputs(n, R, seed=6)
+    gs[1][1500] = np.float16(np.nan)
+    b = _binding()
+    owner = [q for q in range(R) if b.mpt_dp_shard(n, R, q)[0] <= 1500 < b.mpt_dp_shard(n, R, q)[1]][0]
+    _, _, _, flags, _ = _emulate(n, R, 8.0, 0.1, 0.0, gs, w, v)
+    for q in range(R):
+        assert flags[q][0] == 0
+        assert (flags[q][1] != 0) == (q == owner)
+
+
+def test_dp_empty_problem_and_bad_arguments():
+    b = _binding()
+    gs, w, v = _inputs(0, 2, seed=1)
+    _emulate(0, 2, 4.0, 0.1, 0.9, gs, w, v)           # n = 0: launches only publish the (clear) decision
+    t = torch.zeros(64, dtype=torch.int16, device="cuda")
+    f = torch.zeros(2, dtype=torch.int32, device="cuda")
+    w32 = torch.zeros(64, dtype=torch.float32, device="cuda")
+    with pytest.raises(b.MptError):
+        b.mpt_dp_step_flat([t, t], [f, f], [t, t], w32, None, 64, 2, 2, 1.0, 0.1, 0.0, f)      # rank out of range
+    with pytest.raises(b.MptError):
+        b.mpt_dp_step_flat([t[1:], t], [f, f], [t, t], w32, None, 32, 2, 0, 1.0, 0.1, 0.0, f)  # misaligned gradient
+    with pytest.raises(b.MptError):
+        b.mpt_dp_step_flat([t, t], [f, f], [t, t], w32, None, 64, 2, 0, 0.0, 0.1, 0.0, f)      # S must be positive
+    with pytest.raises(b.MptError):
+        b.mpt_dp_step_flat([t, t], [f, f], [t, t], w32, None, 64, 2, 0, 1.0, 0.1, 0.9, f)      # momentum without state
+
+
+# ---------------------------------------------------------------- two processes, mapped buffers
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _replica_main(rank, R, port, n, S, lr, mu, steps, out_dir):
+    import datetime
+    import torch as th
+    import torch.distributed as dist
+    from paper_1710_03740_b200 import binding as b
+    th.cuda.set_device(0)
+    dist.init_process_group("gloo", init_method="tcp://127.0.0.1:%d" % port, rank=rank, world_size=R,
+                            timeout=datetime.timedelta(seconds=90))
+    try:
+        dp = b.DataParallelFlat(n, S, lr, mu)
+        gs0, w, v = _inputs(n, R, seed=77)
+        lo, hi = dp.lo, dp.hi
+        if hi > lo:
+            dp.w32[:hi - lo] = th.from_numpy(w[lo:hi]).cuda()
+            dp.v[:hi - lo] = th.from_numpy(v[lo:hi]).cuda()
+        skipped = []
+        for t in range(steps):
+            gs, _, _ = _inputs(n, R, seed=100 + t)
+            dp.g16[:] = th.from_numpy(gs[rank].view(np.int16)).cuda()
+            if t == 1 and rank == 1:
+                dp.flags[0] = 1                     # this replica's backward overflowed in step 1
+            skipped.append(dp.step())
+        th.cuda.synchronize()
+        np.savez(os.path.join(out_dir, "r%d.npz" % rank), w32=dp.w32[:max(hi - lo, 0)].cpu().numpy(),
+                 v=dp.v[:max(hi - lo, 0)].cpu().numpy(), w16=dp.w16.cpu().numpy().view(np.uint16),
+                 skipped=np.array(skipped), lo=lo, hi=hi)
+        dp.close()
+    finally:
+        dist.destroy_process_group()
+
+
+@pytest.mark.timeout(300)
+def test_dp_two_processes_mapped_buffers(tmp_path):
+    """Two replicas as two processes on this GPU: each maps the other's gradient, weight and flag
+    buffers through exported handles and runs its shard's kernel between host barriers.  Three
+    steps, the second one skipped because one replica reported an overflow."""
+    import torch.multiprocessing as mp
+    R, n, S, lr, mu, steps = 2, 100003, 512.0, 0.05, 0.9, 3
+    port = _free_port()
+    mp.spawn(_replica_main, args=(R, port, n, S, lr, mu, steps, str(tmp_path)), nprocs=R, join=True)
+    _, w, v = _inputs(n, R, seed=77)
+    w16 = np.zeros(n, np.uint16)
+    for t in range(steps):
+        gs, _, _ = _inputs(n, R, seed=100 + t)
+        if t == 1:
+            continue
+        mpo.dp_update_apply([g.view(np.uint16) for g in gs], w, v, w16, S, lr, mu, True)
+    for q in range(R):
+        z = np.load(os.path.join(str(tmp_path), "r%d.npz" % q))
+        lo, hi = int(z["lo"]), int(z["hi"])
+        assert list(z["skipped"]) == [False, True, False]
+        assert np.array_equal(z["w32"].view(np.uint32), w[lo:hi].view(np.uint32))
+        assert np.array_equal(z["v"].view(np.uint32), v[lo:hi].view(np.uint32))
+        assert np.array_equal(z["w16"], w16), "replica %d holds all shards' FP16 weights" % q
