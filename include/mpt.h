@@ -494,9 +494,9 @@ int mpt_softmax_ce_static(const uint16_t *z_dev, int ldz, const int32_t *labels_
  * overflow word must be complete before any replica calls this, and every replica's call must
  * have completed before any replica reads its weights or clears its overflow word (a stream-
  * ordered barrier across the replicas on both sides).  flags_dev: device uint32[2] of this
- * replica; [0] receives the OR of all replicas' words, [1] the kernel's own inspection of the
- * unscaled mean gradients it formed (must have been zeroed by the caller).  flags_dev may be the
- * same memory as flag_peers[rank]: the kernel only ever sets bits there.
+ * replica; [0] receives the OR of all replicas' words, [1] (zeroed by the call) the kernel's own
+ * inspection of the unscaled mean gradients it formed.  flags_dev may be the same memory as
+ * flag_peers[rank]: the kernel only ever sets bits there.
  * Errors: MPT_ERR_INVALID_ARG for R outside [1, MPT_DP_MAX_REPLICAS], rank outside [0, R), a null or
  * misaligned (16 bytes) pointer; MPT_ERR_CUDA if the launch fails. */
 #define MPT_DP_MAX_REPLICAS 16
@@ -504,6 +504,30 @@ int mpt_dp_shard(size_t n, int R, int rank, size_t *lo_out, size_t *hi_out);
 int mpt_dp_step_flat(const uint16_t *const *g16_peers, const uint32_t *const *flag_peers, uint16_t *const *w16_peers,
                      float *w32_shard_dev, float *v_shard_dev, size_t n, int R, int rank, float S, float lr, float mu,
                      uint32_t *flags_dev, void *cuda_stream);
+
+/* Data-parallel training of an mpt_ctx.  mpt_dp_layout_of reports where, inside the context's
+ * workspace, the buffers live that the replicas exchange: byte offsets from the workspace base of
+ * the scaled FP16 gradient arena, the FP16 weight arena and the overflow word (followed by the
+ * word that receives the kernel's own inspection), and n, the arenas' length in elements.
+ * Contexts created from the same description have the same layout, so a replica that has mapped a
+ * peer's workspace forms that peer's pointers as mapped base + offset.
+ * mpt_dp_attach: from now on mpt_step runs the kernel of mpt_dp_step_flat over the arenas instead
+ * of the single-GPU master pass.  Entry `rank` of each array must be this context's own buffer.
+ * The FP32 master weights and momentum are then current only inside this replica's shard
+ * (mpt_get_master returns stale values outside it); the FP16 weights are complete on every
+ * replica.  SGD with or without momentum only: MPT_ERR_STATE from mpt_step for other kinds, weight
+ * decay or clipping.  Dynamic loss scaling works unchanged: every replica sees the same OR-ed
+ * overflow word and moves its scale identically; the kernel reads S from device memory.  The
+ * caller orders the replicas around mpt_step as described for mpt_dp_step_flat (before: every
+ * replica's mpt_backward_scaled has completed; after: every replica's mpt_step has completed
+ * before any replica's next mpt_forward).  R == 1 detaches (the arrays may then be null). */
+typedef struct mpt_dp_layout {
+    size_t g16_offset, w16_offset, flags_offset; /* bytes from the workspace base */
+    size_t n;                                    /* elements in each arena */
+} mpt_dp_layout;
+int mpt_dp_layout_of(mpt_ctx *ctx, mpt_dp_layout *out);
+int mpt_dp_attach(mpt_ctx *ctx, int R, int rank, const uint16_t *const *g16_peers, const uint32_t *const *flag_peers,
+                  uint16_t *const *w16_peers);
 
 /* Device memory that other processes can map (the buffers the replicas exchange).  mpt_dp_alloc
  * returns memory from the driver's allocator (not from a framework's pool, whose blocks cannot be

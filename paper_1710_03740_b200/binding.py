@@ -34,7 +34,8 @@ EXPORTS = ["mpt_workspace_bytes", "mpt_create", "mpt_workspace_bytes_opt", "mpt_
            "mpt_softmax_ce", "mpt_softmax_ce_static", "mpt_version",
            "mpt_lstm_forward", "mpt_lstm_backward", "mpt_lstm_cell_forward", "mpt_lstm_cell_backward", "mpt_bias_grad",
            "mpt_add_f16",
-           "mpt_dp_shard", "mpt_dp_step_flat", "mpt_dp_alloc", "mpt_dp_free", "mpt_dp_export", "mpt_dp_open", "mpt_dp_close"]
+           "mpt_dp_shard", "mpt_dp_step_flat", "mpt_dp_alloc", "mpt_dp_free", "mpt_dp_export", "mpt_dp_open", "mpt_dp_close",
+           "mpt_dp_layout_of", "mpt_dp_attach"]
 
 
 class MptError(RuntimeError):
@@ -68,6 +69,10 @@ class LstmTensors(C.Structure):
 
 
 _lib = None
+
+
+class DpLayout(C.Structure):
+    _fields_ = [("g16_offset", C.c_size_t), ("w16_offset", C.c_size_t), ("flags_offset", C.c_size_t), ("n", C.c_size_t)]
 
 
 def lib() -> C.CDLL:
@@ -131,6 +136,8 @@ def lib() -> C.CDLL:
     L.mpt_dp_export.argtypes = [vp, vp]
     L.mpt_dp_open.argtypes = [vp, C.POINTER(vp)]
     L.mpt_dp_close.argtypes = [vp]
+    L.mpt_dp_layout_of.argtypes = [vp, C.POINTER(DpLayout)]
+    L.mpt_dp_attach.argtypes = [vp, i32, i32, vp, vp, vp]
     L.mpt_version.restype = C.c_char_p
     L.mpt_version.argtypes = []
     _lib = L
@@ -179,8 +186,11 @@ def mpt_workspace_bytes(layers, max_batch, use_momentum) -> int:
 class Context:
     """One mpt_ctx over a torch-allocated workspace.  Method names follow the C calls."""
 
-    def __init__(self, layers, S, lr, momentum=0.0, max_batch=1, device="cuda:0", stream=None, optimizer=None):
-        """optimizer: an Optimizer struct; default SGD with the given lr and momentum."""
+    def __init__(self, layers, S, lr, momentum=0.0, max_batch=1, device="cuda:0", stream=None, optimizer=None,
+                 shareable=False):
+        """optimizer: an Optimizer struct; default SGD with the given lr and momentum.  shareable: take
+        the workspace from the driver's allocator (a DeviceBuffer other processes can map) instead of
+        torch's pool."""
         import torch
         self.layers = [(int(i), int(o), int(r)) for (i, o, r) in layers]
         self.device = torch.device(device)
@@ -192,8 +202,13 @@ class Context:
                                              C.byref(out)))
         nbytes = int(out.value)
         with torch.cuda.device(self.device):
-            self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
-            base = self.workspace.data_ptr()
+            if shareable:
+                self.workspace = DeviceBuffer(nbytes + 256)
+                base = self.workspace.ptr
+                torch.cuda.synchronize()
+            else:
+                self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
+                base = self.workspace.data_ptr()
             self._ws_ptr = (base + 255) // 256 * 256
             self._ctx = C.c_void_p()
             _check(lib().mpt_create_opt(_layer_array(self.layers), len(self.layers), float(S), C.byref(opt),
@@ -206,6 +221,17 @@ class Context:
         if getattr(self, "_ctx", None):
             lib().mpt_destroy(self._ctx)
             self._ctx = None
+            if isinstance(self.workspace, DeviceBuffer):
+                self.workspace.close()
+
+    def dp_layout(self):
+        out = DpLayout()
+        _check(lib().mpt_dp_layout_of(self._ctx, C.byref(out)), self._ctx)
+        return out
+
+    def dp_attach(self, R, rank, g16_peers, flag_peers, w16_peers):
+        tab = lambda xs: (C.c_void_p * R)(*[_addr(x) for x in xs])
+        _check(lib().mpt_dp_attach(self._ctx, int(R), int(rank), tab(g16_peers), tab(flag_peers), tab(w16_peers)), self._ctx)
 
     def __del__(self):
         try:                # at interpreter shutdown the module globals may already be gone
@@ -598,3 +624,55 @@ class DataParallelFlat:
         self._barrier()
         for b in self._own.values():
             b.close()
+
+
+class DataParallelMLP:
+    """Replica `rank` of R of an MLP context in a torch.distributed group (one process per GPU):
+    the context's workspace is shareable, the replicas map each other's workspaces, and step() runs
+    the one-kernel data-parallel step between two barriers.  Every replica feeds its own part of
+    the batch (equal sizes) through forward() / backward_scaled() of `ctx`."""
+
+    def __init__(self, layers, S, lr, momentum=0.0, max_batch=1, group=None):
+        import torch.distributed as dist
+        self.group = group
+        self.R, self.rank = dist.get_world_size(group), dist.get_rank(group)
+        self.ctx = Context(layers, S, lr, momentum, max_batch, shareable=True)
+        lay = self.ctx.dp_layout()
+        own = self.ctx.workspace
+        table = dp_exchange_handles({"ws": own.export(), "skew": self.ctx._ws_ptr - own.ptr}, group)
+        self._maps = []
+        g, f, w = [], [], []
+        for q in range(self.R):
+            if q == self.rank:
+                base = self.ctx._ws_ptr
+            else:
+                m = DeviceBuffer(handle=table[q]["ws"])
+                self._maps.append(m)
+                base = m.ptr + table[q]["skew"]
+            g.append(base + lay.g16_offset)
+            w.append(base + lay.w16_offset)
+            f.append(base + lay.flags_offset)
+        if self.R > 1:
+            self.ctx.dp_attach(self.R, self.rank, g, f, w)
+        self.shard = mpt_dp_shard(lay.n, self.R, self.rank)
+
+    def _barrier(self):
+        import torch
+        import torch.distributed as dist
+        torch.cuda.current_stream().synchronize()
+        dist.barrier(group=self.group)
+
+    def step(self):
+        """All replicas call this after their backward_scaled(); returns True if the step was skipped."""
+        self._barrier()
+        overflow = self.ctx.step()
+        self._barrier()
+        return bool(overflow)
+
+    def close(self):
+        self._barrier()
+        for m in self._maps:
+            m.close()
+        self._maps = []
+        self._barrier()
+        self.ctx.close()

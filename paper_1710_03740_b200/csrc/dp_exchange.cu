@@ -54,11 +54,13 @@ __device__ __forceinline__ bool any_replica_overflowed(const DpPeers &pp, int R)
 template <int RT, bool MOM>
 __global__ void __launch_bounds__(kDpThreads) k_dp_step(const DpPeers pp, int R_dyn, float4 *__restrict__ w32,
                                                         float4 *__restrict__ v, size_t first, size_t n8, float inv,
-                                                        float lr, float mu, uint32_t *flags)
+                                                        const float *__restrict__ S_dev, float lr, float mu,
+                                                        uint32_t *flags)
 {
     pdl_trigger();
     pdl_wait();
     const int R = RT ? RT : R_dyn;
+    if (S_dev) inv = __fdiv_rn(1.0f, __fmul_rn(*S_dev, (float)R));
     if (any_replica_overflowed(pp, R)) {
         if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(flags, 1u);
         return;
@@ -118,10 +120,12 @@ __global__ void __launch_bounds__(kDpThreads) k_dp_step(const DpPeers pp, int R_
 // the up to seven elements after the last whole vector of a shard (one warp)
 template <bool MOM>
 __global__ void k_dp_step_tail(const DpPeers pp, int R, float *__restrict__ w32, float *__restrict__ v, size_t first,
-                               size_t begin, size_t count, float inv, float lr, float mu, uint32_t *flags)
+                               size_t begin, size_t count, float inv, const float *__restrict__ S_dev, float lr, float mu,
+                               uint32_t *flags)
 {
     pdl_trigger();
     pdl_wait();
+    if (S_dev) inv = __fdiv_rn(1.0f, __fmul_rn(*S_dev, (float)R));
     if (any_replica_overflowed(pp, R)) {
         if (threadIdx.x == 0) atomicOr(flags, 1u);
         return;
@@ -141,26 +145,41 @@ __global__ void k_dp_step_tail(const DpPeers pp, int R, float *__restrict__ w32,
 }
 
 template <bool MOM>
-cudaError_t launch_dp(const DpPeers &pp, int R, float *w32, float *v, size_t first, size_t count, float inv, float lr,
-                      float mu, uint32_t *flags, cudaStream_t st)
+cudaError_t launch_dp(const DpPeers &pp, int R, float *w32, float *v, size_t first, size_t count, float inv,
+                      const float *S_dev, float lr, float mu, uint32_t *flags, cudaStream_t st, int *n_launches)
 {
+    if (n_launches) *n_launches = (count / 8 ? 1 : 0) + ((count / 8) * 8 < count || count == 0 ? 1 : 0);
     const size_t n8 = count / 8;
     if (n8) {
         const dim3 grid((unsigned)((n8 + kDpThreads - 1) / kDpThreads)), block(kDpThreads);
         switch (R) {
-            case 2: MPT_LAUNCH(k_dp_step<2, MOM>, grid, block, 0, st, pp, R, (float4 *)w32, (float4 *)v, first, n8, inv, lr, mu, flags); break;
-            case 4: MPT_LAUNCH(k_dp_step<4, MOM>, grid, block, 0, st, pp, R, (float4 *)w32, (float4 *)v, first, n8, inv, lr, mu, flags); break;
-            case 8: MPT_LAUNCH(k_dp_step<8, MOM>, grid, block, 0, st, pp, R, (float4 *)w32, (float4 *)v, first, n8, inv, lr, mu, flags); break;
-            default: MPT_LAUNCH(k_dp_step<0, MOM>, grid, block, 0, st, pp, R, (float4 *)w32, (float4 *)v, first, n8, inv, lr, mu, flags); break;
+            case 2: MPT_LAUNCH(k_dp_step<2, MOM>, grid, block, 0, st, pp, R, (float4 *)w32, (float4 *)v, first, n8, inv, S_dev, lr, mu, flags); break;
+            case 4: MPT_LAUNCH(k_dp_step<4, MOM>, grid, block, 0, st, pp, R, (float4 *)w32, (float4 *)v, first, n8, inv, S_dev, lr, mu, flags); break;
+            case 8: MPT_LAUNCH(k_dp_step<8, MOM>, grid, block, 0, st, pp, R, (float4 *)w32, (float4 *)v, first, n8, inv, S_dev, lr, mu, flags); break;
+            default: MPT_LAUNCH(k_dp_step<0, MOM>, grid, block, 0, st, pp, R, (float4 *)w32, (float4 *)v, first, n8, inv, S_dev, lr, mu, flags); break;
         }
     }
     // also for an empty shard: the launch then only publishes the skip decision in this replica's flags
     if (n8 * 8 < count || count == 0)
-        MPT_LAUNCH(k_dp_step_tail<MOM>, dim3(1), dim3(32), 0, st, pp, R, w32, v, first, n8 * 8, count, inv, lr, mu, flags);
+        MPT_LAUNCH(k_dp_step_tail<MOM>, dim3(1), dim3(32), 0, st, pp, R, w32, v, first, n8 * 8, count, inv, S_dev, lr, mu, flags);
     return cudaGetLastError();
 }
 
 }  // namespace
+
+cudaError_t launch_dp_step(const uint16_t *const *g16, const uint32_t *const *flag, uint16_t *const *w16, int R,
+                           float *w32_shard, float *v_shard, size_t first, size_t count, float inv_SR, const float *S_dev,
+                           float lr, float mu, uint32_t *flags, cudaStream_t st, int *n_launches)
+{
+    DpPeers pp = {};
+    for (int q = 0; q < R; q++) {
+        pp.g[q] = g16[q];
+        pp.flag[q] = flag[q];
+        pp.w[q] = w16[q];
+    }
+    return mu != 0.0f ? launch_dp<true>(pp, R, w32_shard, v_shard, first, count, inv_SR, S_dev, lr, mu, flags, st, n_launches)
+                      : launch_dp<false>(pp, R, w32_shard, nullptr, first, count, inv_SR, S_dev, lr, mu, flags, st, n_launches);
+}
 
 }  // namespace mpt
 
@@ -190,14 +209,10 @@ int mpt_dp_step_flat(const uint16_t *const *g16_peers, const uint32_t *const *fl
     if (mpt_dp_shard(n, R, rank, &lo, &hi) != MPT_OK) return MPT_ERR_INVALID_ARG;
     if (!(S > 0.0f) || !(lr == lr) || !(mu == mu)) return MPT_ERR_INVALID_ARG;
     const bool mom = mu != 0.0f;
-    DpPeers pp = {};
     for (int q = 0; q < R; q++) {
         if (!g16_peers[q] || !flag_peers[q] || !w16_peers[q]) return MPT_ERR_INVALID_ARG;
         if ((((uintptr_t)g16_peers[q] | (uintptr_t)w16_peers[q]) & 15) != 0 || ((uintptr_t)flag_peers[q] & 3) != 0)
             return MPT_ERR_INVALID_ARG;
-        pp.g[q] = g16_peers[q];
-        pp.flag[q] = flag_peers[q];
-        pp.w[q] = w16_peers[q];
     }
     const size_t count = hi - lo;
     if (count && (!w32_shard_dev || (mom && !v_shard_dev))) return MPT_ERR_INVALID_ARG;
@@ -206,8 +221,8 @@ int mpt_dp_step_flat(const uint16_t *const *g16_peers, const uint32_t *const *fl
     cudaError_t e = cudaMemsetAsync(flags_dev + 1, 0, sizeof(uint32_t), st);
     if (e != cudaSuccess) return MPT_ERR_CUDA;
     const float inv = 1.0f / (S * (float)R);
-    e = mom ? launch_dp<true>(pp, R, w32_shard_dev, v_shard_dev, lo, count, inv, lr, mu, flags_dev, st)
-            : launch_dp<false>(pp, R, w32_shard_dev, nullptr, lo, count, inv, lr, mu, flags_dev, st);
+    e = launch_dp_step(g16_peers, flag_peers, w16_peers, R, w32_shard_dev, v_shard_dev, lo, count, inv, nullptr, lr, mu, flags_dev,
+                       st, nullptr);
     return e == cudaSuccess ? MPT_OK : MPT_ERR_CUDA;
 }
 

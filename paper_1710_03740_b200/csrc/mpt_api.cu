@@ -156,6 +156,11 @@ struct mpt_ctx {
     bool dynamic_scale = false;
     int growth_interval = 2000;
     float scale_backoff = 0.5f, scale_growth = 2.0f, scale_min = 0x1p-100f, scale_max = 0x1p120f;
+    // data-parallel step (mpt_dp_attach): replica count (0 or 1: off), this replica, peer tables
+    int dp_R = 0, dp_rank = 0;
+    const uint16_t *dp_g16[MPT_DP_MAX_REPLICAS] = {};
+    const uint32_t *dp_flag[MPT_DP_MAX_REPLICAS] = {};
+    uint16_t *dp_w16[MPT_DP_MAX_REPLICAS] = {};
     std::string err;
     // optional per-kernel timing with CUDA events (mpt_profile)
     bool profiling = false;
@@ -344,7 +349,23 @@ int do_step(mpt_ctx *c)
     const float inv = 1.0f / c->S;
     CK(cudaMemsetAsync(c->status + ST_OVERFLOW_SEEN, 0, sizeof(uint32_t), c->stream), "status clear");
     cudaError_t e;
-    {
+    if (c->dp_R > 1) {
+        if (c->opt_kind != MPT_OPT_SGD || c->wd != 0.0f || c->clip > 0.0f)
+            return fail(c, MPT_ERR_STATE, "the data-parallel step supports SGD with or without momentum only");
+        size_t lo = 0, hi = 0;
+        mpt_dp_shard(c->plan.P_pad, c->dp_R, c->dp_rank, &lo, &hi);
+        int nl = 0;
+        {
+            // bytes through this GPU's memory system: R gradients read, the shard's state, R weight copies written
+            const double per_elem = 2.0 * c->dp_R + 8.0 + (c->use_momentum ? 8.0 : 0.0) + 2.0 * c->dp_R;
+            ProfSpan span(c, MPT_PROF_UPDATE, per_elem * (double)(hi - lo));
+            e = launch_dp_step(c->dp_g16, c->dp_flag, c->dp_w16, c->dp_R, c->master + lo, c->use_momentum ? c->mom + lo : nullptr,
+                               lo, hi - lo, 1.0f / (c->S * (float)c->dp_R), (const float *)(c->status + ST_SCALE), c->lr,
+                               c->use_momentum ? c->mu : 0.0f, c->status + ST_OVERFLOW, c->stream, &nl);
+        }
+        c->launches += nl;
+        if (e != cudaSuccess) return cuda_fail(c, e, "data-parallel step launch");
+    } else {
         const double bytes_per_param = 12.0 + 8.0 * (c->use_momentum ? 1 : 0) + 8.0 * (c->state2 ? 1 : 0) + (c->clip > 0.0f ? 2.0 : 0.0);
         ProfSpan span(c, MPT_PROF_UPDATE, bytes_per_param * (double)c->plan.P_pad);
         if (c->clip > 0.0f) {
@@ -363,9 +384,9 @@ int do_step(mpt_ctx *c)
                                   (const float *)(c->status + ST_INV_SCALE),
                                   c->opt_kind == MPT_OPT_ADAM ? (const float *)(c->status + ST_B1T) : nullptr,
                                   c->clip > 0.0f ? (const float *)(c->status + ST_CLIP_COEF) : nullptr);
+        c->launches++;
+        if (e != cudaSuccess) return cuda_fail(c, e, "update launch");
     }
-    c->launches++;
-    if (e != cudaSuccess) return cuda_fail(c, e, "update launch");
     if (c->dynamic_scale || c->opt_kind == MPT_OPT_ADAM) {
         // end-of-step bookkeeping on the device: loss scale and Adam's beta^t move only on applied steps
         ProfSpan span(c, MPT_PROF_OTHER, 0.0);
@@ -879,6 +900,46 @@ int mpt_get_grad_norm(mpt_ctx *c, float *norm_out, float *coef_out)
     if (r != MPT_OK) return r;
     memcpy(norm_out, &st[ST_GRAD_NORM], 4);
     memcpy(coef_out, &st[ST_CLIP_COEF], 4);
+    return MPT_OK;
+}
+
+int mpt_dp_layout_of(mpt_ctx *c, mpt_dp_layout *out)
+{
+    int r = usable(c);
+    if (r != MPT_OK) return r;
+    if (!out) return fail(c, MPT_ERR_INVALID_ARG, "null output");
+    out->g16_offset = (size_t)((const uint8_t *)c->g16 - c->ws);
+    out->w16_offset = (size_t)((const uint8_t *)c->w16 - c->ws);
+    out->flags_offset = (size_t)((const uint8_t *)(c->status + ST_OVERFLOW) - c->ws);
+    out->n = c->plan.P_pad;
+    return MPT_OK;
+}
+
+int mpt_dp_attach(mpt_ctx *c, int R, int rank, const uint16_t *const *g16_peers, const uint32_t *const *flag_peers,
+                  uint16_t *const *w16_peers)
+{
+    int r = usable(c);
+    if (r != MPT_OK) return r;
+    if (R == 1) {
+        c->dp_R = 0;
+        return MPT_OK;
+    }
+    if (R < 2 || R > MPT_DP_MAX_REPLICAS || rank < 0 || rank >= R) return fail(c, MPT_ERR_INVALID_ARG, "replica count or rank");
+    if (!g16_peers || !flag_peers || !w16_peers) return fail(c, MPT_ERR_INVALID_ARG, "null peer table");
+    for (int q = 0; q < R; q++) {
+        if (!g16_peers[q] || !flag_peers[q] || !w16_peers[q]) return fail(c, MPT_ERR_INVALID_ARG, "null peer pointer");
+        if ((((uintptr_t)g16_peers[q] | (uintptr_t)w16_peers[q]) & 15) != 0 || ((uintptr_t)flag_peers[q] & 3) != 0)
+            return fail(c, MPT_ERR_INVALID_ARG, "misaligned peer pointer");
+    }
+    if (g16_peers[rank] != c->g16 || w16_peers[rank] != c->w16 || flag_peers[rank] != c->status + ST_OVERFLOW)
+        return fail(c, MPT_ERR_INVALID_ARG, "this replica's entries must be the context's own buffers");
+    for (int q = 0; q < R; q++) {
+        c->dp_g16[q] = g16_peers[q];
+        c->dp_flag[q] = flag_peers[q];
+        c->dp_w16[q] = w16_peers[q];
+    }
+    c->dp_R = R;
+    c->dp_rank = rank;
     return MPT_OK;
 }
 

@@ -130,6 +130,13 @@ cudaError_t launch_update_opt(int kind, const uint16_t *g16, float *w32, float *
 static constexpr int kNormParts = 1184;
 cudaError_t launch_clip_coef(const uint16_t *g16, size_t n, float inv_S, const float *inv_S_dev, float clip, double *parts,
                              float *out2, cudaStream_t st);
+// Data-parallel step for one replica's shard (see mpt.h, mpt_dp_step_flat): g16 / flag / w16 are
+// host arrays of R device pointers; w32_shard / v_shard point at element `first` of the owner's
+// state, `count` elements.  S_dev (may be null): the loss scale is read from device memory and
+// 1/(S*R) formed in the kernel (one multiplication, one division) instead of taking inv_SR.
+cudaError_t launch_dp_step(const uint16_t *const *g16, const uint32_t *const *flag, uint16_t *const *w16, int R,
+                           float *w32_shard, float *v_shard, size_t first, size_t count, float inv_SR, const float *S_dev,
+                           float lr, float mu, uint32_t *flags, cudaStream_t st, int *n_launches);
 // End-of-step bookkeeping on the device (one thread): dynamic loss scale (if interval > 0) and
 // Adam's running products beta^t (if adam != 0); both only move on a step that was applied.
 cudaError_t launch_post_step(uint32_t *status, int interval, float backoff, float growth, float min_S, float max_S,

@@ -205,3 +205,117 @@ def test_dp_two_processes_mapped_buffers(tmp_path):
         assert np.array_equal(z["w32"].view(np.uint32), w[lo:hi].view(np.uint32))
         assert np.array_equal(z["v"].view(np.uint32), v[lo:hi].view(np.uint32))
         assert np.array_equal(z["w16"], w16), "replica %d holds all shards' FP16 weights" % q
+
+
+# ---------------------------------------------------------------- MLP contexts as replicas
+
+_MLP_LAYERS = [(64, 96, 1), (96, 10, 0)]
+_MLP = dict(S=256.0, lr=0.05, mu=0.9, batch=32, inj_steps=3, e2e_steps=3)
+
+
+def _mlp_masters():
+    rng = np.random.default_rng(5)
+    return [(rng.standard_normal((o, i)) * i ** -0.5).astype(np.float16).astype(np.float32) for (i, o, _) in _MLP_LAYERS]
+
+
+def _mlp_injected_grad(t, q, l):
+    i, o, _ = _MLP_LAYERS[l]
+    rng = np.random.default_rng([t, q, l, 41])
+    g = (rng.standard_normal((o, i)) * 8.0).astype(np.float16)
+    if t == 1 and q == 1 and l == 0:
+        g[3, 7] = np.float16(np.inf)            # replica 1 overflows in step 1: everybody skips
+    return g
+
+
+def _mlp_batch(t, q):
+    rng = np.random.default_rng([t, q, 43])
+    x = rng.standard_normal((_MLP["batch"], _MLP_LAYERS[0][0])).astype(np.float16)
+    y = rng.integers(0, _MLP_LAYERS[-1][1], _MLP["batch"]).astype(np.int32)
+    return x, y
+
+
+def _mlp_replica_main(rank, R, port, out_dir):
+    import datetime
+    import torch as th
+    import torch.distributed as dist
+    from paper_1710_03740_b200 import binding as b
+    th.cuda.set_device(0)
+    dist.init_process_group("gloo", init_method="tcp://127.0.0.1:%d" % port, rank=rank, world_size=R,
+                            timeout=datetime.timedelta(seconds=90))
+    try:
+        dp = b.DataParallelMLP(_MLP_LAYERS, _MLP["S"], _MLP["lr"], _MLP["mu"], max_batch=_MLP["batch"])
+        L = len(_MLP_LAYERS)
+        for l, w in enumerate(_mlp_masters()):
+            dp.ctx.set_master(l, w)
+        rec = {}
+        for t in range(_MLP["inj_steps"]):
+            for l in range(L):
+                dp.ctx.set_grad(l, _mlp_injected_grad(t, rank, l).view(np.uint16))
+            rec["inj_skip_%d" % t] = np.array(dp.step())
+            for l in range(L):
+                rec["inj_w16_%d_%d" % (t, l)] = dp.ctx.get_tensor(b.T_W16, l)
+                rec["inj_w32_%d_%d" % (t, l)] = dp.ctx.get_master(l)
+                rec["inj_v_%d_%d" % (t, l)] = dp.ctx.get_tensor(b.T_MOMENTUM32, l)
+        for t in range(_MLP["e2e_steps"]):
+            x, y = _mlp_batch(t, rank)
+            dp.ctx.forward(th.from_numpy(x.view(np.int16)).cuda())
+            rec["e2e_loss_%d" % t] = np.array(dp.ctx.backward_scaled(th.from_numpy(y).cuda()))
+            for l in range(L):
+                rec["e2e_g16_%d_%d" % (t, l)] = dp.ctx.get_tensor(b.T_GRAD16, l)
+            rec["e2e_skip_%d" % t] = np.array(dp.step())
+            for l in range(L):
+                rec["e2e_w16_%d_%d" % (t, l)] = dp.ctx.get_tensor(b.T_W16, l)
+        rec["launches"] = np.array(dp.ctx.launch_count())
+        np.savez(os.path.join(out_dir, "m%d.npz" % rank), **rec)
+        dp.close()
+    finally:
+        dist.destroy_process_group()
+
+
+@pytest.mark.timeout(300)
+def test_dp_mlp_two_processes(tmp_path):
+    """Two MLP contexts as two processes on this GPU, attached to each other's workspaces.
+    Injected (seeded) gradients: FP16 weights of every replica, and the FP32 state inside each
+    replica's shard, equal the oracle's data-parallel step bit for bit, including a skipped step.
+    Then whole iterations: losses against the oracle's replicas, and the step against the oracle
+    applied to the gradients each replica's backward produced."""
+    import torch.multiprocessing as mp
+    from oracle.dp import OracleDataParallelMLP
+    R = 2
+    mp.spawn(_mlp_replica_main, args=(R, _free_port(), str(tmp_path)), nprocs=R, join=True)
+    rec = [np.load(os.path.join(str(tmp_path), "m%d.npz" % q)) for q in range(R)]
+    L = len(_MLP_LAYERS)
+    ora = OracleDataParallelMLP(_MLP_LAYERS, _MLP["S"], _MLP["lr"], _MLP["mu"], R)
+    for l, w in enumerate(_mlp_masters()):
+        ora.set_master(l, w)
+    for t in range(_MLP["inj_steps"]):
+        for q in range(R):
+            for l in range(L):
+                ora.set_grad(q, l, _mlp_injected_grad(t, q, l).view(np.uint16))
+        skipped = ora.step()
+        assert skipped == (1 if t == 1 else 0)
+        for l in range(L):
+            want16, want32, wantv = ora.replicas[0].w16[l], ora.replicas[0].w32[l], ora.replicas[0].v[l]
+            owned = np.zeros(want32.shape, bool)
+            for q in range(R):
+                assert bool(rec[q]["inj_skip_%d" % t]) == bool(skipped)
+                assert np.array_equal(rec[q]["inj_w16_%d_%d" % (t, l)].reshape(want16.shape), want16), (t, l, q)
+                m = rec[q]["inj_w32_%d_%d" % (t, l)].reshape(want32.shape).view(np.uint32) == want32.view(np.uint32)
+                m &= rec[q]["inj_v_%d_%d" % (t, l)].reshape(wantv.shape).view(np.uint32) == wantv.view(np.uint32)
+                owned |= m
+            assert owned.all(), "every element's FP32 state is current on the replica that owns it"
+    for t in range(_MLP["e2e_steps"]):
+        xs, ys = zip(*[_mlp_batch(t, q) for q in range(R)])
+        losses = ora.forward_backward(list(xs), list(ys))
+        for q in range(R):
+            got = float(rec[q]["e2e_loss_%d" % t])
+            assert abs(got - losses[q]) <= 1e-3 * abs(losses[q]), (t, q, got, losses[q])
+            for l in range(L):
+                ora.set_grad(q, l, rec[q]["e2e_g16_%d_%d" % (t, l)])       # the step is checked on the gradients it read
+        skipped = ora.step()
+        for q in range(R):
+            assert bool(rec[q]["e2e_skip_%d" % t]) == bool(skipped)
+            for l in range(L):
+                want16 = ora.replicas[0].w16[l]
+                assert np.array_equal(rec[q]["e2e_w16_%d_%d" % (t, l)].reshape(want16.shape), want16), (t, l, q)
+    assert all(int(r["launches"]) > 0 for r in rec)

@@ -91,3 +91,90 @@ def test_inverse_scale_is_one_division_of_the_binary32_product():
     # 3 replicas: 1/(S*3) is not exact; the value is the binary32 quotient, not a double rounded twice
     x = mpo.dp_inv_scale(1.0, 3)
     assert x == np.float32(1.0) / np.float32(3.0)
+
+
+# ---- the replicated MLP iteration
+
+
+def _mlp_setup(R, layers, S=128.0, lr=0.1, mu=0.9, seed=0):
+    from oracle.dp import OracleDataParallelMLP
+    from oracle.mlp import OracleMLP
+    rng = np.random.default_rng(seed)
+    dp, one = OracleDataParallelMLP(layers, S, lr, mu, R), OracleMLP(layers, S, lr, mu)
+    for l, (i, o, _) in enumerate(layers):
+        w = (rng.standard_normal((o, i)) * i ** -0.5).astype(np.float32)
+        dp.set_master(l, w)
+        one.set_master(l, w)
+    return dp, one, rng
+
+
+def test_mlp_one_replica_is_the_single_gpu_iteration():
+    layers = [(16, 32, 1), (32, 10, 0)]
+    dp, one, rng = _mlp_setup(1, layers)
+    for t in range(3):
+        x = rng.standard_normal((8, 16)).astype(np.float16)
+        y = rng.integers(0, 10, 8).astype(np.int32)
+        la = dp.forward_backward([x], [y])[0]
+        one.forward(x)
+        lb = one.backward_scaled(y)
+        assert la == lb and dp.step() == one.step()
+        for l in range(2):
+            assert np.array_equal(dp.replicas[0].w32[l].view(np.uint32), one.w32[l].view(np.uint32))
+            assert np.array_equal(dp.replicas[0].w16[l], one.w16[l])
+
+
+def test_mlp_replicas_fed_the_same_batch_equal_one_replica():
+    # R = 2 replicas see the same rows: both gradients are identical, their FP32 sum is exactly 2g,
+    # and 1/(2S) is exact for S a power of two, so the run equals the single replica bit for bit
+    layers = [(16, 24, 1), (24, 5, 0)]
+    dp, one, rng = _mlp_setup(2, layers, S=64.0)
+    for t in range(3):
+        x = rng.standard_normal((8, 16)).astype(np.float16)
+        y = rng.integers(0, 5, 8).astype(np.int32)
+        dp.forward_backward([x, x.copy()], [y, y.copy()])
+        one.forward(x)
+        one.backward_scaled(y)
+        assert dp.step() == one.step() == 0
+        for q in range(2):
+            for l in range(2):
+                assert np.array_equal(dp.replicas[q].w32[l].view(np.uint32), one.w32[l].view(np.uint32))
+                assert np.array_equal(dp.replicas[q].w16[l], one.w16[l])
+
+
+def test_mlp_two_halves_approximate_the_full_batch_step():
+    # mean of the half-batch mean gradients = full-batch mean gradient in exact arithmetic; with FP16
+    # gradient storage the two runs differ by rounding only (a "sum instead of mean" mistake would
+    # double the step, a dropped replica would change it by tens of percent)
+    layers = [(32, 48, 1), (48, 10, 0)]
+    dp, one, rng = _mlp_setup(2, layers, S=256.0, lr=0.5, mu=0.0)
+    x = rng.standard_normal((64, 32)).astype(np.float16)
+    y = rng.integers(0, 10, 64).astype(np.int32)
+    w_before = [w.copy() for w in one.w32]
+    dp.forward_backward([x[:32], x[32:]], [y[:32], y[32:]])
+    one.forward(x)
+    one.backward_scaled(y)
+    assert dp.step() == one.step() == 0
+    for l in range(2):
+        da = dp.replicas[0].w32[l].astype(np.float64) - w_before[l]
+        db = one.w32[l].astype(np.float64) - w_before[l]
+        assert np.linalg.norm(da - db) <= 2e-2 * np.linalg.norm(db)
+        assert np.array_equal(dp.replicas[0].w16[l], dp.replicas[1].w16[l])
+
+
+def test_mlp_overflow_on_one_replica_skips_all_and_halves_every_scale():
+    layers = [(8, 8, 0)]
+    dp, _, rng = _mlp_setup(2, layers, S=1024.0)
+    for r in dp.replicas:
+        r.set_dynamic_scale(2, 1.0, 65536.0)
+    before = [r.w32[0].copy() for r in dp.replicas]
+    g = (rng.standard_normal((8, 8))).astype(np.float16)
+    bad = g.copy()
+    bad[2, 3] = np.float16(np.inf)
+    dp.set_grad(0, 0, g.view(np.uint16))
+    dp.set_grad(1, 0, bad.view(np.uint16))
+    assert dp.step() == 1
+    for q, r in enumerate(dp.replicas):
+        assert np.array_equal(r.w32[0], before[q]) and r.S == np.float32(512.0)
+    dp.set_grad(1, 0, g.view(np.uint16))
+    assert dp.step() == 0 and dp.step() == 0        # two clean steps: the scale doubles again
+    assert all(r.S == np.float32(1024.0) for r in dp.replicas)
