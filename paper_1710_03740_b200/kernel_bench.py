@@ -204,6 +204,26 @@ def bench_update_opt(n, kind, wd, iters, clip=0.0):
             "sustained_gbs": bpp * n / sus / 1e6, "flags": flags.tolist()}
 
 
+def bench_dp(n, R, momentum, iters):
+    """Data-parallel step of ONE replica (rank 0 of R) with every replica's buffers on this GPU: the
+    kernel's own memory-system rate with local "peers".  Says nothing about NVLink."""
+    g = torch.Generator(device="cuda").manual_seed(3)
+    gs = [(torch.randn(n, device="cuda", generator=g) * 37).half() for _ in range(R)]
+    ws = [torch.empty(n, dtype=torch.half, device="cuda") for _ in range(R)]
+    fl = [torch.zeros(2, dtype=torch.int32, device="cuda") for _ in range(R)]
+    lo, hi = mpt.mpt_dp_shard(n, R, 0)
+    w32 = torch.randn(hi - lo, device="cuda", generator=g)
+    v = torch.zeros(hi - lo, device="cuda") if momentum else None
+    fn = lambda: mpt.mpt_dp_step_flat(gs, fl, ws, w32, v, n, R, 0, 512.0, 1e-4, 0.9 if momentum else 0.0, fl[0])  # noqa: E731
+    best, sus = _time(fn, iters)
+    per_elem = 2 * R + 8 + (8 if momentum else 0) + 2 * R       # R gradients in, state in and out, R weight copies out
+    nbytes = per_elem * (hi - lo)
+    return {"kernel": "dp_step", "params": n, "replicas": R, "shard": hi - lo, "momentum": bool(momentum),
+            "bytes_per_shard_element": per_elem, "best_ms": best, "median_ms": _time.last_median, "sustained_ms": sus,
+            "best_gbs": nbytes / best / 1e6, "median_gbs": nbytes / _time.last_median / 1e6,
+            "link_bytes_each_way_if_remote": 2 * (hi - lo) * (R - 1), "peers": "local (one GPU)", "flags": fl[0].tolist()}
+
+
 def bench_lstm(name, iters, steps=None):
     """LSTM layer with projection: the fused gate step against the bare gate product, the backward
     gate kernel, the bias-gradient reduction, and the whole layer forward + backward."""
@@ -412,6 +432,11 @@ def main():
     ls.add_argument("--config", default="biglstm", choices=sorted(inputs.LSTM_CONFIGS))
     ls.add_argument("--steps", type=int, default=0, help="override the number of time steps")
     ls.add_argument("--iters", type=int, default=20)
+    d = sub.add_parser("dp")
+    d.add_argument("--params", type=int, default=150994944)
+    d.add_argument("--replicas", type=int, default=8)
+    d.add_argument("--momentum", type=int, default=1)
+    d.add_argument("--iters", type=int, default=20)
     t = sub.add_parser("step")
     t.add_argument("--workload", default="tiny", choices=["tiny", "scale_sweep", "scale_sweep_twin", "large_twin"])
     t.add_argument("--iters", type=int, default=50)
@@ -427,6 +452,8 @@ def main():
                 res = bench_gemm(M, N, K, op, args.iters, args.compare_library, flags, not args.no_workspace, args.sustain)
                 res["kernel_choice"] = args.kernel
                 print(json.dumps(res), flush=True)
+    elif args.cmd == "dp":
+        print(json.dumps(bench_dp(args.params, args.replicas, args.momentum, args.iters)), flush=True)
     elif args.cmd == "steplike":
         print(json.dumps(bench_steplike(args.steps, args.dense)), flush=True)
     elif args.cmd == "lstm":
