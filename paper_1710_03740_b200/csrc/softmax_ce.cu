@@ -226,7 +226,8 @@ static constexpr int kSmaxThreads = 1024;
 // Block-wide max or sum for exactly 32 warps: warp results go through shared memory, then every
 // warp combines the 32 of them with the same xor-butterfly (both partners of a step add the same
 // two numbers, so all lanes and all warps hold identical bits; the order is fixed).
-__device__ __forceinline__ float block_reduce32(float v, bool is_max, float *red)
+// any_out (may be null): receives the OR of `pred` over the block, carried by the reduction's barrier.
+__device__ __forceinline__ float block_reduce32(float v, bool is_max, float *red, bool pred = false, int *any_out = nullptr)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 #pragma unroll
@@ -235,7 +236,8 @@ __device__ __forceinline__ float block_reduce32(float v, bool is_max, float *red
         v = is_max ? fmaxf(v, other) : v + other;
     }
     if (lane == 0) red[warp] = v;   // the caller alternates between two arrays: no reuse hazard
-    __syncthreads();
+    if (any_out) *any_out = __syncthreads_or(pred ? 1 : 0);
+    else __syncthreads();
     float r = red[lane];
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
@@ -255,7 +257,18 @@ __device__ __forceinline__ void bulk_store_row(void *dst, uint32_t src, uint32_t
 {
     asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(bytes) : "memory");
     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-}template <int VPT>
+}
+
+// 2^x on the special-function unit, one instruction: results below 2^-126 flush to zero (such a
+// term is 10^-38 of a sum that is at least 1), NaN and the infinities behave as in exp2f.
+__device__ __forceinline__ float ex2_ftz(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+template <int VPT>
 __global__ void __launch_bounds__(kSmaxThreads, 1) k_softmax_ce_bulk(const uint16_t *__restrict__ z, int ldz,
                                                                       const int32_t *__restrict__ labels, int B, int C, float c,
                                                                       uint16_t *__restrict__ dz, int lddz,
@@ -293,18 +306,18 @@ __global__ void __launch_bounds__(kSmaxThreads, 1) k_softmax_ce_bulk(const uint1
             bulk_load_row(smem0 + (uint32_t)((k + 1) % 3) * buf_stride, z + (size_t)(row + gridDim.x) * ldz, row_bytes,
                           smem_u32(&bars[(k + 1) % 3]));
         }
-        if (!mbar_wait(smem_u32(&bars[b]), (uint32_t)((k / 3) & 1), &abort_word)) {
-            abort_word = 1;
-            if (kerr && tid == 0) atomicCAS(kerr, 0u, (uint32_t)KERR_WAIT_FULL | 0x40u | ((uint32_t)blockIdx.x << 8));
-        }
-        __syncthreads();
-        if (abort_word) break;
+        // every thread waits for the row itself; whether any of them gave up is learnt on the barrier
+        // of the first reduction (a thread that gave up scans stale data until then, harmlessly)
+        const bool arrived = mbar_wait(smem_u32(&bars[b]), (uint32_t)((k / 3) & 1), &abort_word);
+        if (!arrived) abort_word = 1;
         uint4 *rowv = (uint4 *)(rows_smem + (size_t)b * buf_stride);
         uint16_t *rowh = (uint16_t *)rowv;
         const int y = labels[row];
         const bool good = y >= 0 && y < C;
+        // the thread that will write the vector holding the label's element also patches it
+        const bool owner = good && tid == ((y >> 3) & (kSmaxThreads - 1));
         float zy = 0.0f;
-        if (tid == 0 && good) zy = hbits2f(rowh[y]);       // read long before the row is overwritten in place
+        if (owner) zy = hbits2f(rowh[y]);                  // read long before the row is overwritten in place
         // pass 1: the maximum, on packed FP16 values (max is exact in any precision; like fmaxf it
         // drops NaN operands, which then surface through the exponentials)
         __half2 mh = __half2half2(__ushort_as_half((unsigned short)0xFC00u));   // -inf
@@ -318,9 +331,18 @@ __global__ void __launch_bounds__(kSmaxThreads, 1) k_softmax_ce_bulk(const uint1
             }
         }
         float m = fmaxf(__low2float(mh), __high2float(mh));
-        m = block_reduce32(m, true, red[0]);
-        // pass 2: exponentials, kept in registers for pass 3 (conversions and exp2 share the
-        // special-function pipe, the scarce unit of this kernel), and their sum
+        int gave_up = 0;
+        m = block_reduce32(m, true, red[0], !arrived, &gave_up);
+        if (gave_up) {
+            if (kerr && tid == 0) atomicCAS(kerr, 0u, (uint32_t)KERR_WAIT_FULL | 0x40u | ((uint32_t)blockIdx.x << 8));
+            break;
+        }
+        // pass 2: exponentials, kept in registers for pass 3, and their sum.  One FMA and one
+        // special-function instruction per logit: 2^(z*log2e - mL) with mL = rn(m*log2e).  Rounding mL
+        // scales every exponential of the row by the same 2^delta (delta = m*log2e - mL, obtained
+        // exactly by an FMA): it cancels in e/s and is taken out of log(s) below.
+        const float mL = __fmul_rn(m, LOG2E);
+        const float delta = fmaf(m, LOG2E, -mL);
         float ev[VPT * 8];
         float s = 0.0f;
 #pragma unroll
@@ -332,8 +354,8 @@ __global__ void __launch_bounds__(kSmaxThreads, 1) k_softmax_ce_bulk(const uint1
 #pragma unroll
                 for (int q = 0; q < 4; q++) {
                     const float2 f = __half22float2(*(const __half2 *)&w[q]);
-                    ev[u * 8 + 2 * q] = exp2f((f.x - m) * LOG2E);
-                    ev[u * 8 + 2 * q + 1] = exp2f((f.y - m) * LOG2E);
+                    ev[u * 8 + 2 * q] = ex2_ftz(fmaf(f.x, LOG2E, -mL));
+                    ev[u * 8 + 2 * q + 1] = ex2_ftz(fmaf(f.y, LOG2E, -mL));
                     s += ev[u * 8 + 2 * q];
                     s += ev[u * 8 + 2 * q + 1];
                 }
@@ -341,30 +363,39 @@ __global__ void __launch_bounds__(kSmaxThreads, 1) k_softmax_ce_bulk(const uint1
         }
         s = block_reduce32(s, false, red[1]);
         const float inv_s = __fdiv_rn(1.0f, s);
-        const float kk = good ? inv_s * c : 0.0f;
+        const float kk = inv_s * c;
+        if (good) {
 #pragma unroll
-        for (int u = 0; u < VPT; u++) {
-            const int i = tid + u * kSmaxThreads;
-            if (i < C8) {
-                uint32_t o[4];
+            for (int u = 0; u < VPT; u++) {
+                const int i = tid + u * kSmaxThreads;
+                if (i < C8) {
+                    uint32_t o[4];
 #pragma unroll
-                for (int q = 0; q < 4; q++) {
-                    const __half2 h = __floats2half2_rn(ev[u * 8 + 2 * q] * kk, ev[u * 8 + 2 * q + 1] * kk);
-                    o[q] = good ? *(const uint32_t *)&h : 0u;
+                    for (int q = 0; q < 4; q++) {
+                        const __half2 h = __floats2half2_rn(ev[u * 8 + 2 * q] * kk, ev[u * 8 + 2 * q + 1] * kk);
+                        o[q] = *(const uint32_t *)&h;
+                    }
+                    rowv[i] = make_uint4(o[0], o[1], o[2], o[3]);
                 }
-                rowv[i] = make_uint4(o[0], o[1], o[2], o[3]);
+            }
+        } else {           // a label outside [0, C): the whole gradient row is zero
+#pragma unroll
+            for (int u = 0; u < VPT; u++) {
+                const int i = tid + u * kSmaxThreads;
+                if (i < C8) rowv[i] = make_uint4(0u, 0u, 0u, 0u);
             }
         }
-        __syncthreads();   // the row's gradient is in place before the label element is patched
-        if (tid == 0) {
-            if (good) {    // d_y = (e_y / s - 1) * c, evaluated separately because of the cancellation
-                const float ey = exp2f((zy - m) * LOG2E);
-                rowh[y] = (uint16_t)f2hbits(__fmul_rn(__fsub_rn(ey * inv_s, 1.0f), c));
-                row_loss[row] = (m + logf(s)) - zy;
-            } else {       // a label outside [0, C) contributes neither loss nor gradient
-                row_loss[row] = 0.0f;
-                if (bad_labels) atomicAdd(bad_labels, 1u);
-            }
+        // the label's element: d_y = (e_y / s - 1) * c, evaluated separately because of the
+        // cancellation; its owner wrote the vector around it just above, so no block barrier is needed
+        // (the warp-level one keeps the two stores, made through different pointer types, in order)
+        __syncwarp();
+        if (owner) {
+            const float ey = ex2_ftz(fmaf(zy, LOG2E, -mL));
+            rowh[y] = (uint16_t)f2hbits(__fmul_rn(__fsub_rn(ey * inv_s, 1.0f), c));
+            row_loss[row] = (m + (logf(s) - delta * 0.69314718055994531f)) - zy;
+        } else if (!good && tid == 0) {   // a label outside [0, C) contributes neither loss nor gradient
+            row_loss[row] = 0.0f;
+            if (bad_labels) atomicAdd(bad_labels, 1u);
         }
         // every thread's shared-memory writes become visible to the bulk store
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
