@@ -14,6 +14,15 @@ static constexpr int kMaxSmemRowBytes = 200 * 1024;
 __device__ __forceinline__ float hbits2f(uint32_t h) { return __half2float(__ushort_as_half((unsigned short)h)); }
 __device__ __forceinline__ uint32_t f2hbits(float x) { return (uint32_t)__half_as_ushort(__float2half_rn(x)); }
 
+// 2^x on the special-function unit, one instruction: results below 2^-126 flush to zero (such a
+// term is 10^-38 of a sum that is at least 1), NaN and the infinities behave as in exp2f.
+__device__ __forceinline__ float ex2_ftz(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
 __device__ __forceinline__ float block_reduce(float v, bool is_max, float *red)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
@@ -171,6 +180,11 @@ __global__ void __launch_bounds__(1024, VPT <= 4 ? 2 : 1) k_softmax_ce_reg(const
     if (has_tail) m = fmaxf(m, tv);
     m = block_reduce(m, true, red);
 
+    // one FMA and one special-function instruction per logit: 2^(z*log2e - mL), mL = rn(m*log2e);
+    // the factor 2^delta this puts on every exponential of the row (delta = m*log2e - mL, exact by
+    // an FMA) cancels in e/s and is taken out of log(s)
+    const float mL = __fmul_rn(m, LOG2E);
+    const float delta = fmaf(m, LOG2E, -mL);
     float s = 0.0f;
 #pragma unroll
     for (int u = 0; u < VPT; u++) {
@@ -178,16 +192,17 @@ __global__ void __launch_bounds__(1024, VPT <= 4 ? 2 : 1) k_softmax_ce_reg(const
             const uint32_t w[4] = {x[u].x, x[u].y, x[u].z, x[u].w};
 #pragma unroll
             for (int q = 0; q < 4; q++) {
-                s += exp2f((hbits2f(w[q] & 0xFFFFu) - m) * LOG2E);
-                s += exp2f((hbits2f(w[q] >> 16) - m) * LOG2E);
+                const float2 f = __half22float2(*(const __half2 *)&w[q]);
+                s += ex2_ftz(fmaf(f.x, LOG2E, -mL));
+                s += ex2_ftz(fmaf(f.y, LOG2E, -mL));
             }
         }
     }
-    if (has_tail) s += exp2f((tv - m) * LOG2E);
+    if (has_tail) s += ex2_ftz(fmaf(tv, LOG2E, -mL));
     s = block_reduce(s, false, red);
     const float inv_s = __fdiv_rn(1.0f, s);
     const float k = inv_s * c;
-    if (tid == 0) row_loss[row] = (m + logf(s)) - hbits2f(zr[y]);
+    if (tid == 0) row_loss[row] = (m + (logf(s) - delta * 0.69314718055994531f)) - hbits2f(zr[y]);
 
 #pragma unroll
     for (int u = 0; u < VPT; u++) {
@@ -197,17 +212,17 @@ __global__ void __launch_bounds__(1024, VPT <= 4 ? 2 : 1) k_softmax_ce_reg(const
             uint32_t o[4];
 #pragma unroll
             for (int q = 0; q < 4; q++) {
-                const float d0 = exp2f((hbits2f(w[q] & 0xFFFFu) - m) * LOG2E) * k;
-                const float d1 = exp2f((hbits2f(w[q] >> 16) - m) * LOG2E) * k;
-                o[q] = f2hbits(d0) | (f2hbits(d1) << 16);
+                const float2 f = __half22float2(*(const __half2 *)&w[q]);
+                const __half2 h = __floats2half2_rn(ex2_ftz(fmaf(f.x, LOG2E, -mL)) * k, ex2_ftz(fmaf(f.y, LOG2E, -mL)) * k);
+                o[q] = *(const uint32_t *)&h;
             }
             __stcs((uint4 *)dr + i, make_uint4(o[0], o[1], o[2], o[3]));
         }
     }
-    if (has_tail) dr[C8 * 8 + tid] = (uint16_t)f2hbits(exp2f((tv - m) * LOG2E) * k);
+    if (has_tail) dr[C8 * 8 + tid] = (uint16_t)f2hbits(ex2_ftz(fmaf(tv, LOG2E, -mL)) * k);
     __syncthreads();  // the row's stores are done before the label element is patched
     if (tid == 0) {
-        const float ey = exp2f((hbits2f(zr[y]) - m) * LOG2E);
+        const float ey = ex2_ftz(fmaf(hbits2f(zr[y]), LOG2E, -mL));
         dr[y] = (uint16_t)f2hbits(__fmul_rn(__fsub_rn(ey * inv_s, 1.0f), c));
     }
 }
@@ -257,15 +272,6 @@ __device__ __forceinline__ void bulk_store_row(void *dst, uint32_t src, uint32_t
 {
     asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(bytes) : "memory");
     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-}
-
-// 2^x on the special-function unit, one instruction: results below 2^-126 flush to zero (such a
-// term is 10^-38 of a sum that is at least 1), NaN and the infinities behave as in exp2f.
-__device__ __forceinline__ float ex2_ftz(float x)
-{
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
 }
 
 template <int VPT>
