@@ -234,7 +234,7 @@ def _mlp_batch(t, q):
     return x, y
 
 
-def _mlp_replica_main(rank, R, port, out_dir):
+def _mlp_replica_main(rank, R, port, out_dir, dynamic=False):
     import datetime
     import torch as th
     import torch.distributed as dist
@@ -247,11 +247,14 @@ def _mlp_replica_main(rank, R, port, out_dir):
         L = len(_MLP_LAYERS)
         for l, w in enumerate(_mlp_masters()):
             dp.ctx.set_master(l, w)
+        if dynamic:
+            dp.ctx.set_dynamic_scale(True, growth_interval=2, min_scale=1.0, max_scale=65536.0)
         rec = {}
         for t in range(_MLP["inj_steps"]):
             for l in range(L):
                 dp.ctx.set_grad(l, _mlp_injected_grad(t, rank, l).view(np.uint16))
             rec["inj_skip_%d" % t] = np.array(dp.step())
+            rec["inj_scale_%d" % t] = np.array(dp.ctx.get_scale())
             for l in range(L):
                 rec["inj_w16_%d_%d" % (t, l)] = dp.ctx.get_tensor(b.T_W16, l)
                 rec["inj_w32_%d_%d" % (t, l)] = dp.ctx.get_master(l)
@@ -319,3 +322,49 @@ def test_dp_mlp_two_processes(tmp_path):
                 want16 = ora.replicas[0].w16[l]
                 assert np.array_equal(rec[q]["e2e_w16_%d_%d" % (t, l)].reshape(want16.shape), want16), (t, l, q)
     assert all(int(r["launches"]) > 0 for r in rec)
+
+
+@pytest.mark.timeout(300)
+def test_dp_mlp_two_processes_dynamic_scale(tmp_path):
+    """The same two attached contexts with dynamic loss scaling: the kernel reads S from device
+    memory, every replica sees the OR-ed overflow word, so both halve S after the skipped step and
+    double it after two clean ones - the oracle's replicas do the same, bit for bit."""
+    import torch.multiprocessing as mp
+    from oracle.dp import OracleDataParallelMLP
+    R = 2
+    mp.spawn(_mlp_replica_main, args=(R, _free_port(), str(tmp_path), True), nprocs=R, join=True)
+    rec = [np.load(os.path.join(str(tmp_path), "m%d.npz" % q)) for q in range(R)]
+    L = len(_MLP_LAYERS)
+    ora = OracleDataParallelMLP(_MLP_LAYERS, _MLP["S"], _MLP["lr"], _MLP["mu"], R)
+    for l, w in enumerate(_mlp_masters()):
+        ora.set_master(l, w)
+    for r in ora.replicas:
+        r.set_dynamic_scale(2, 1.0, 65536.0)
+    scales = []
+    for t in range(_MLP["inj_steps"]):
+        for q in range(R):
+            for l in range(L):
+                ora.set_grad(q, l, _mlp_injected_grad(t, q, l).view(np.uint16))
+        skipped = ora.step()
+        scales.append(float(ora.replicas[0].S))
+        for q in range(R):
+            assert bool(rec[q]["inj_skip_%d" % t]) == bool(skipped)
+            assert float(rec[q]["inj_scale_%d" % t]) == float(ora.replicas[q].S), (t, q)
+            for l in range(L):
+                want16 = ora.replicas[0].w16[l]
+                assert np.array_equal(rec[q]["inj_w16_%d_%d" % (t, l)].reshape(want16.shape), want16), (t, l, q)
+    assert scales[1] == _MLP["S"] / 2          # the skipped step halved the scale everywhere
+    for t in range(_MLP["e2e_steps"]):
+        xs, ys = zip(*[_mlp_batch(t, q) for q in range(R)])
+        losses = ora.forward_backward(list(xs), list(ys))
+        for q in range(R):
+            got = float(rec[q]["e2e_loss_%d" % t])
+            assert abs(got - losses[q]) <= 1e-3 * abs(losses[q]), (t, q, got, losses[q])
+            for l in range(L):
+                ora.set_grad(q, l, rec[q]["e2e_g16_%d_%d" % (t, l)])
+        skipped = ora.step()
+        for q in range(R):
+            assert bool(rec[q]["e2e_skip_%d" % t]) == bool(skipped)
+            for l in range(L):
+                want16 = ora.replicas[0].w16[l]
+                assert np.array_equal(rec[q]["e2e_w16_%d_%d" % (t, l)].reshape(want16.shape), want16), (t, l, q)
