@@ -35,6 +35,12 @@ class OracleDataParallelMLP:
     def set_grad(self, q, l, g16):
         self.replicas[q].set_grad(l, g16)
 
+    def set_optimizer(self, kind, lr, mu=0.0, b2=0.0, eps=0.0, wd=0.0):
+        """Any kind of mlp.OracleMLP.set_optimizer except clipping (its norm would have to be taken
+        over the mean gradient of all replicas; not part of this step)."""
+        for r in self.replicas:
+            r.set_optimizer(kind, lr, mu, b2, eps, wd, clip=0.0)
+
     def step(self):
         lead = self.replicas[0]
         inv = np.float32(1.0) / lead.S
@@ -43,12 +49,27 @@ class OracleDataParallelMLP:
             for g in r.g16:
                 overflow |= mpo.grad_nonfinite(g, inv)
         if not overflow:
+            kind = lead.opt["kind"]
+            plain = kind == mpo.OPT_SGD and float(lead.opt["wd"]) == 0.0
+            if kind == mpo.OPT_ADAM:       # bias corrections use the products including this step
+                for r in self.replicas:
+                    r.b1t = np.float32(r.b1t * r.mu)
+                    r.b2t = np.float32(r.b2t * r.opt["b2"])
+            bc1 = np.float32(1.0) - lead.b1t
+            bc2 = np.float32(1.0) - lead.b2t
             for l in range(len(lead.layers)):
-                mpo.dp_update_apply([r.g16[l] for r in self.replicas], lead.w32[l], lead.v[l], lead.w16[l], lead.S,
-                                    lead.lr, lead.mu, lead.use_momentum)
+                gs = [r.g16[l] for r in self.replicas]
+                if plain:
+                    mpo.dp_update_apply(gs, lead.w32[l], lead.v[l], lead.w16[l], lead.S, lead.lr, lead.mu, lead.use_momentum)
+                else:
+                    s1 = lead.v[l] if (kind != mpo.OPT_SGD or lead.use_momentum) else None
+                    s2 = lead.s2[l] if kind == mpo.OPT_ADAM else None
+                    mpo.dp_update_apply_opt(kind, gs, lead.w32[l], s1, s2, lead.w16[l], lead.S, lead.lr, lead.mu,
+                                            lead.opt["b2"], lead.opt["eps"], lead.opt["wd"], bc1, bc2)
                 for r in self.replicas[1:]:
                     r.w32[l][...] = lead.w32[l]
                     r.v[l][...] = lead.v[l]
+                    r.s2[l][...] = lead.s2[l]
                     r.w16[l][...] = lead.w16[l]
         if lead.dynamic is not None:
             interval, backoff, growth, smin, smax = lead.dynamic

@@ -348,6 +348,54 @@ void mpo_update_apply(const uint16_t *g16, float *w32, float *v, uint16_t *w16,
  *   w = w - u ; w16 = rn16(w)
  * mu doubles as b1.  s1 / s2 may be NULL when the kind does not use them.
  */
+/* One element of the steps listed above: g is the UNSCALED gradient; returns the new w. */
+static inline float mpo_opt_elem(int kind, float g, float w, float *s1, float *s2, size_t i, float lr, float mu,
+                                 float b2, float eps, float wd, float omb1, float omb2, float bc1, float bc2)
+{
+    if (wd != 0.0f) { float t = wd * w; g = g + t; }
+    float u;
+    if (kind == 1) {
+        float a = mu * s1[i];
+        float v = a + g;
+        s1[i] = v;
+        float b = mu * v;
+        float c = g + b;
+        u = lr * c;
+    } else if (kind == 2) {
+        float q = g * g;
+        float h = s1[i] + q;
+        s1[i] = h;
+        float r = sqrtf(h);
+        float d = r + eps;
+        float c = g / d;
+        u = lr * c;
+    } else if (kind == 3) {
+        float a = mu * s1[i];
+        float b = omb1 * g;
+        float m = a + b;
+        s1[i] = m;
+        float q = g * g;
+        float c = b2 * s2[i];
+        float d = omb2 * q;
+        float v = c + d;
+        s2[i] = v;
+        float mh = m / bc1;
+        float vh = v / bc2;
+        float r = sqrtf(vh);
+        float e = r + eps;
+        float f = mh / e;
+        u = lr * f;
+    } else if (s1) {
+        float a = mu * s1[i];
+        float v = a + g;
+        s1[i] = v;
+        u = lr * v;
+    } else {
+        u = lr * g;
+    }
+    return w - u;
+}
+
 void mpo_update_apply_opt(int kind, const uint16_t *g16, float *w32, float *s1, float *s2, uint16_t *w16,
                           size_t n, float inv_S, float lr, float mu, float b2, float eps, float wd,
                           float bc1, float bc2)
@@ -355,50 +403,29 @@ void mpo_update_apply_opt(int kind, const uint16_t *g16, float *w32, float *s1, 
     const float omb1 = 1.0f - mu, omb2 = 1.0f - b2;
 #pragma omp parallel for schedule(static)
     for (size_t i = 0; i < n; i++) {
-        float w = w32[i];
         float g = mpo_h2f(g16[i]) * inv_S;
-        if (wd != 0.0f) { float t = wd * w; g = g + t; }
-        float u;
-        if (kind == 1) {
-            float a = mu * s1[i];
-            float v = a + g;
-            s1[i] = v;
-            float b = mu * v;
-            float c = g + b;
-            u = lr * c;
-        } else if (kind == 2) {
-            float q = g * g;
-            float h = s1[i] + q;
-            s1[i] = h;
-            float r = sqrtf(h);
-            float d = r + eps;
-            float c = g / d;
-            u = lr * c;
-        } else if (kind == 3) {
-            float a = mu * s1[i];
-            float b = omb1 * g;
-            float m = a + b;
-            s1[i] = m;
-            float q = g * g;
-            float c = b2 * s2[i];
-            float d = omb2 * q;
-            float v = c + d;
-            s2[i] = v;
-            float mh = m / bc1;
-            float vh = v / bc2;
-            float r = sqrtf(vh);
-            float e = r + eps;
-            float f = mh / e;
-            u = lr * f;
-        } else if (s1) {
-            float a = mu * s1[i];
-            float v = a + g;
-            s1[i] = v;
-            u = lr * v;
-        } else {
-            u = lr * g;
-        }
-        w = w - u;
+        float w = mpo_opt_elem(kind, g, w32[i], s1, s2, i, lr, mu, b2, eps, wd, omb1, omb2, bc1, bc2);
+        w32[i] = w;
+        w16[i] = mpo_f2h(w);
+    }
+}
+
+/*
+ * The same steps in the data-parallel setting of mpo_dp_update_apply (declared further down):
+ * g = (h2f(g_0[i]) + h2f(g_1[i]) + ... in ascending replica order, binary32) * inv_SR, then the
+ * lines above unchanged.  (Section 4.5: the language model trained over 4 GPUs uses Adagrad.)
+ */
+void mpo_dp_update_apply_opt(int kind, const uint16_t *const *g16, int R, float *w32, float *s1, float *s2,
+                             uint16_t *w16, size_t n, float inv_SR, float lr, float mu, float b2, float eps,
+                             float wd, float bc1, float bc2)
+{
+    const float omb1 = 1.0f - mu, omb2 = 1.0f - b2;
+#pragma omp parallel for schedule(static)
+    for (size_t i = 0; i < n; i++) {
+        float s = mpo_h2f(g16[0][i]);
+        for (int q = 1; q < R; q++) s = s + mpo_h2f(g16[q][i]);
+        float g = s * inv_SR;
+        float w = mpo_opt_elem(kind, g, w32[i], s1, s2, i, lr, mu, b2, eps, wd, omb1, omb2, bc1, bc2);
         w32[i] = w;
         w16[i] = mpo_f2h(w);
     }

@@ -178,3 +178,77 @@ def test_mlp_overflow_on_one_replica_skips_all_and_halves_every_scale():
     dp.set_grad(1, 0, g.view(np.uint16))
     assert dp.step() == 0 and dp.step() == 0        # two clean steps: the scale doubles again
     assert all(r.S == np.float32(1024.0) for r in dp.replicas)
+
+
+# ---- other optimizers in the data-parallel step
+
+
+import pytest
+
+
+@pytest.mark.parametrize("kind", [mpo.OPT_SGD, mpo.OPT_NESTEROV, mpo.OPT_ADAGRAD, mpo.OPT_ADAM])
+@pytest.mark.parametrize("wd", [0.0, 0.01])
+def test_opt_one_replica_is_the_single_gpu_step(kind, wd):
+    # R = 1: the sum has one term and 1/(S*1) = 1/S: the step is update_apply_opt (pinned elsewhere)
+    n, S = 3001, 512.0
+    g = inputs.loguniform_grads(n, S, seed=21).view(np.uint16)
+    rng = np.random.default_rng(kind)
+    w = rng.standard_normal(n).astype(np.float32)
+    s1 = np.abs(0.1 * rng.standard_normal(n)).astype(np.float32)
+    s2 = np.abs(0.01 * rng.standard_normal(n)).astype(np.float32)
+    a = [w.copy(), s1.copy(), s2.copy(), np.zeros(n, np.uint16)]
+    b = [w.copy(), s1.copy(), s2.copy(), np.zeros(n, np.uint16)]
+    args = dict(b2=0.999, eps=1e-8, wd=wd, bc1=0.19, bc2=0.002)
+    mpo.dp_update_apply_opt(kind, [g], a[0], a[1], a[2], a[3], S, 0.01, 0.9, **args)
+    mpo.update_apply_opt(kind, g, b[0], b[1], b[2], b[3], np.float32(1.0) / np.float32(S), 0.01, 0.9, **args)
+    for x, y in zip(a, b):
+        assert np.array_equal(x.view(np.uint8), y.view(np.uint8))
+
+
+@pytest.mark.parametrize("kind", [mpo.OPT_NESTEROV, mpo.OPT_ADAGRAD, mpo.OPT_ADAM])
+def test_opt_identical_replicas_power_of_two_equal_single_replica(kind):
+    # four copies of one gradient, S a power of two: s * 1/(4S) == g * 1/S exactly
+    n, S = 2053, 128.0
+    g = inputs.loguniform_grads(n, S, seed=22).view(np.uint16)
+    rng = np.random.default_rng(kind + 10)
+    w = rng.standard_normal(n).astype(np.float32)
+    s1 = np.abs(0.1 * rng.standard_normal(n)).astype(np.float32)
+    s2 = np.abs(0.01 * rng.standard_normal(n)).astype(np.float32)
+    a = [w.copy(), s1.copy(), s2.copy(), np.zeros(n, np.uint16)]
+    b = [w.copy(), s1.copy(), s2.copy(), np.zeros(n, np.uint16)]
+    args = dict(b2=0.99, eps=1e-6, wd=0.0, bc1=0.1, bc2=0.01)
+    mpo.dp_update_apply_opt(kind, [g, g.copy(), g.copy(), g.copy()], a[0], a[1], a[2], a[3], S, 0.02, 0.9, **args)
+    mpo.update_apply_opt(kind, g, b[0], b[1], b[2], b[3], np.float32(1.0 / S), 0.02, 0.9, **args)
+    for x, y in zip(a, b):
+        assert np.array_equal(x.view(np.uint8), y.view(np.uint8))
+
+
+def test_opt_adagrad_mean_of_integers_by_hand():
+    # two replicas, gradients 3 and 5 (mean 4), S = 1, accumulator 9 -> 25, sqrt 5, eps 0:
+    # w = 10 - 2 * 4 / 5 = 8.4 (rounded to binary32 as the oracle's operations do)
+    g0 = np.array([3.0], np.float16).view(np.uint16)
+    g1 = np.array([5.0], np.float16).view(np.uint16)
+    w, s1, h = np.array([10.0], np.float32), np.array([9.0], np.float32), np.zeros(1, np.uint16)
+    mpo.dp_update_apply_opt(mpo.OPT_ADAGRAD, [g0, g1], w, s1, None, h, 1.0, 2.0, 0.0, eps=0.0)
+    assert s1[0] == 25.0
+    assert w[0] == np.float32(10.0) - np.float32(2.0) * (np.float32(4.0) / np.float32(5.0))
+    assert abs(float(w[0]) - 8.4) < 1e-6
+
+
+@pytest.mark.parametrize("kind", [mpo.OPT_NESTEROV, mpo.OPT_ADAGRAD, mpo.OPT_ADAM])
+def test_mlp_optimizer_replicas_fed_the_same_batch_equal_one_replica(kind):
+    layers = [(16, 24, 1), (24, 5, 0)]
+    dp, one, rng = _mlp_setup(2, layers, S=64.0)
+    dp.set_optimizer(kind, 0.01, 0.9, b2=0.999, eps=1e-8, wd=0.001)
+    one.set_optimizer(kind, 0.01, 0.9, b2=0.999, eps=1e-8, wd=0.001)
+    for t in range(3):
+        x = rng.standard_normal((8, 16)).astype(np.float16)
+        y = rng.integers(0, 5, 8).astype(np.int32)
+        dp.forward_backward([x, x.copy()], [y, y.copy()])
+        one.forward(x)
+        one.backward_scaled(y)
+        assert dp.step() == one.step() == 0
+        for q in range(2):
+            for l in range(2):
+                assert np.array_equal(dp.replicas[q].w32[l].view(np.uint32), one.w32[l].view(np.uint32))
+                assert np.array_equal(dp.replicas[q].w16[l], one.w16[l])
