@@ -505,6 +505,16 @@ int mpt_dp_step_flat(const uint16_t *const *g16_peers, const uint32_t *const *fl
                      float *w32_shard_dev, float *v_shard_dev, size_t n, int R, int rank, float S, float lr, float mu,
                      uint32_t *flags_dev, void *cuda_stream);
 
+/* The same step with any optimizer of mpt_optimizer on the mean gradient (weight decay, Nesterov,
+ * Adagrad, Adam; op order as in mpt_update_flat_opt with g = s * inv_SR).  s1_shard / s2_shard:
+ * the FP32 states of this replica's shard (null when the kind does not use them); b1t / b2t as in
+ * mpt_update_flat_opt.  Global-norm clipping is not available here (its norm would have to be
+ * taken over the mean gradient of all shards before any shard is updated): opt->clip_norm must be
+ * 0, else MPT_ERR_INVALID_ARG. */
+int mpt_dp_step_flat_opt(const mpt_optimizer *opt, const uint16_t *const *g16_peers, const uint32_t *const *flag_peers,
+                         uint16_t *const *w16_peers, float *w32_shard_dev, float *s1_shard_dev, float *s2_shard_dev, size_t n,
+                         int R, int rank, float S, float b1t, float b2t, uint32_t *flags_dev, void *cuda_stream);
+
 /* Data-parallel training of an mpt_ctx.  mpt_dp_layout_of reports where, inside the context's
  * workspace, the buffers live that the replicas exchange: byte offsets from the workspace base of
  * the scaled FP16 gradient arena, the FP16 weight arena and the overflow word (followed by the
@@ -515,8 +525,8 @@ int mpt_dp_step_flat(const uint16_t *const *g16_peers, const uint32_t *const *fl
  * of the single-GPU master pass.  Entry `rank` of each array must be this context's own buffer.
  * The FP32 master weights and momentum are then current only inside this replica's shard
  * (mpt_get_master returns stale values outside it); the FP16 weights are complete on every
- * replica.  SGD with or without momentum only: MPT_ERR_STATE from mpt_step for other kinds, weight
- * decay or clipping.  Dynamic loss scaling works unchanged: every replica sees the same OR-ed
+ * replica.  Every optimizer kind and weight decay are supported; global-norm clipping is not
+ * (MPT_ERR_STATE from mpt_step).  Dynamic loss scaling works unchanged: every replica sees the same OR-ed
  * overflow word and moves its scale identically; the kernel reads S from device memory.  The
  * caller orders the replicas around mpt_step as described for mpt_dp_step_flat (before: every
  * replica's mpt_backward_scaled has completed; after: every replica's mpt_step has completed

@@ -35,7 +35,7 @@ EXPORTS = ["mpt_workspace_bytes", "mpt_create", "mpt_workspace_bytes_opt", "mpt_
            "mpt_lstm_forward", "mpt_lstm_backward", "mpt_lstm_cell_forward", "mpt_lstm_cell_backward", "mpt_bias_grad",
            "mpt_add_f16",
            "mpt_dp_shard", "mpt_dp_step_flat", "mpt_dp_alloc", "mpt_dp_free", "mpt_dp_export", "mpt_dp_open", "mpt_dp_close",
-           "mpt_dp_layout_of", "mpt_dp_attach"]
+           "mpt_dp_layout_of", "mpt_dp_attach", "mpt_dp_step_flat_opt"]
 
 
 class MptError(RuntimeError):
@@ -131,6 +131,7 @@ def lib() -> C.CDLL:
     L.mpt_add_f16.argtypes = [vp, i32, vp, i32, vp, i32, i32, i32, vp]
     L.mpt_dp_shard.argtypes = [sz, i32, i32, C.POINTER(sz), C.POINTER(sz)]
     L.mpt_dp_step_flat.argtypes = [vp, vp, vp, vp, vp, sz, i32, i32, f32, f32, f32, vp, vp]
+    L.mpt_dp_step_flat_opt.argtypes = [C.POINTER(Optimizer), vp, vp, vp, vp, vp, vp, sz, i32, i32, f32, f32, f32, vp, vp]
     L.mpt_dp_alloc.argtypes = [sz, C.POINTER(vp)]
     L.mpt_dp_free.argtypes = [vp]
     L.mpt_dp_export.argtypes = [vp, vp]
@@ -513,6 +514,17 @@ def mpt_dp_step_flat(g16_peers, flag_peers, w16_peers, w32_shard, v_shard, n, R,
                                   _stream_ptr(stream)))
 
 
+def mpt_dp_step_flat_opt(opt, g16_peers, flag_peers, w16_peers, w32_shard, s1_shard, s2_shard, n, R, rank, S, b1t, b2t,
+                         flags, stream=None):
+    """mpt_dp_step_flat with any optimizer kind and weight decay (no clipping)."""
+    assert len(g16_peers) == R and len(flag_peers) == R and len(w16_peers) == R
+    tab = lambda xs: (C.c_void_p * R)(*[_addr(x) for x in xs])
+    ptr = lambda x: None if x is None else C.c_void_p(_addr(x))
+    _check(lib().mpt_dp_step_flat_opt(C.byref(opt), tab(g16_peers), tab(flag_peers), tab(w16_peers), ptr(w32_shard),
+                                      ptr(s1_shard), ptr(s2_shard), int(n), int(R), int(rank), float(S), float(b1t), float(b2t),
+                                      C.c_void_p(_addr(flags)), _stream_ptr(stream)))
+
+
 class DeviceBuffer:
     """Device memory that other processes can map: either this process's own allocation (made by
     the library from the driver's allocator) or a mapping of a peer's, opened from its handle.
@@ -632,11 +644,11 @@ class DataParallelMLP:
     the one-kernel data-parallel step between two barriers.  Every replica feeds its own part of
     the batch (equal sizes) through forward() / backward_scaled() of `ctx`."""
 
-    def __init__(self, layers, S, lr, momentum=0.0, max_batch=1, group=None):
+    def __init__(self, layers, S, lr, momentum=0.0, max_batch=1, group=None, optimizer=None):
         import torch.distributed as dist
         self.group = group
         self.R, self.rank = dist.get_world_size(group), dist.get_rank(group)
-        self.ctx = Context(layers, S, lr, momentum, max_batch, shareable=True)
+        self.ctx = Context(layers, S, lr, momentum, max_batch, shareable=True, optimizer=optimizer)
         lay = self.ctx.dp_layout()
         own = self.ctx.workspace
         table = dp_exchange_handles({"ws": own.export(), "skew": self.ctx._ws_ptr - own.ptr}, group)

@@ -9,6 +9,7 @@
 #include <string.h>
 
 #include "mpt_common.cuh"
+#include "update_math.cuh"
 
 namespace mpt {
 
@@ -144,6 +145,113 @@ __global__ void k_dp_step_tail(const DpPeers pp, int R, float *__restrict__ w32,
     if (bad) atomicOr(flags + 1, 1u);
 }
 
+// The same exchange with the other optimizer steps (weight decay, Nesterov, Adagrad, Adam) on the
+// mean gradient: replica count at run time, states s1 / s2 of the shard (s2: Adam only).
+template <int KIND, bool WD>
+__global__ void __launch_bounds__(kDpThreads) k_dp_step_opt(const DpPeers pp, int R, float4 *__restrict__ w32,
+                                                            float4 *__restrict__ s1p, float4 *__restrict__ s2p, size_t first,
+                                                            size_t n8, float inv, const float *__restrict__ S_dev, float lr,
+                                                            float mu, float b2, float eps, float wd, float b1t, float b2t,
+                                                            const float *__restrict__ betat_dev, uint32_t *flags)
+{
+    pdl_trigger();
+    pdl_wait();
+    if (S_dev) inv = __fdiv_rn(1.0f, __fmul_rn(*S_dev, (float)R));
+    if (any_replica_overflowed(pp, R)) {
+        if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(flags, 1u);
+        return;
+    }
+    const size_t j = (size_t)blockIdx.x * kDpThreads + threadIdx.x;
+    if (j >= n8) return;
+    if (betat_dev) { b1t = __fmul_rn(betat_dev[0], mu); b2t = __fmul_rn(betat_dev[1], b2); }
+    const float bc1 = __fsub_rn(1.0f, b1t), bc2 = __fsub_rn(1.0f, b2t);
+    const float omb1 = __fsub_rn(1.0f, mu), omb2 = __fsub_rn(1.0f, b2);
+    const bool use_s1 = KIND != MPT_OPT_SGD || mu != 0.0f;
+    constexpr bool S2 = KIND == MPT_OPT_ADAM;
+    const size_t vec = first / 8 + j;
+    float s[8];
+#pragma unroll 4
+    for (int q = 0; q < R; q++) {
+        const uint4 g = __ldcs((const uint4 *)pp.g[q] + vec);
+        const uint32_t gw[4] = {g.x, g.y, g.z, g.w};
+#pragma unroll
+        for (int e = 0; e < 8; e++) {
+            const float x = h2f_bits_dp((e & 1) ? (gw[e >> 1] >> 16) : (gw[e >> 1] & 0xFFFFu));
+            s[e] = q == 0 ? x : __fadd_rn(s[e], x);
+        }
+    }
+    float4 w0 = __ldcs(w32 + 2 * j), w1 = __ldcs(w32 + 2 * j + 1);
+    float4 a0 = make_float4(0, 0, 0, 0), a1 = a0, b0 = a0, b1 = a0;
+    if (use_s1) { a0 = __ldcs(s1p + 2 * j); a1 = __ldcs(s1p + 2 * j + 1); }
+    if (S2) { b0 = __ldcs(s2p + 2 * j); b1 = __ldcs(s2p + 2 * j + 1); }
+    bool bad = false;
+    float *wf[2] = {&w0.x, &w1.x}, *af[2] = {&a0.x, &a1.x}, *bf[2] = {&b0.x, &b1.x};
+#pragma unroll
+    for (int e = 0; e < 8; e++)
+        opt1<KIND, WD>(s[e], wf[e >> 2][e & 3], af[e >> 2][e & 3], bf[e >> 2][e & 3], inv, lr, mu, b2, omb1, omb2, eps, wd,
+                       bc1, bc2, 1.0f, bad);
+    uint4 h;
+    h.x = f2h_bits_dp(w0.x) | (f2h_bits_dp(w0.y) << 16);
+    h.y = f2h_bits_dp(w0.z) | (f2h_bits_dp(w0.w) << 16);
+    h.z = f2h_bits_dp(w1.x) | (f2h_bits_dp(w1.y) << 16);
+    h.w = f2h_bits_dp(w1.z) | (f2h_bits_dp(w1.w) << 16);
+    __stcs(w32 + 2 * j, w0);
+    __stcs(w32 + 2 * j + 1, w1);
+    if (use_s1) { __stcs(s1p + 2 * j, a0); __stcs(s1p + 2 * j + 1, a1); }
+    if (S2) { __stcs(s2p + 2 * j, b0); __stcs(s2p + 2 * j + 1, b1); }
+    for (int q = 0; q < R; q++) __stcs((uint4 *)pp.w[q] + vec, h);
+    if (__any_sync(__activemask(), bad) && (threadIdx.x & 31) == 0) atomicOr(flags + 1, 1u);
+}
+
+template <int KIND, bool WD>
+__global__ void k_dp_step_opt_tail(const DpPeers pp, int R, float *__restrict__ w32, float *__restrict__ s1p,
+                                   float *__restrict__ s2p, size_t first, size_t begin, size_t count, float inv,
+                                   const float *__restrict__ S_dev, float lr, float mu, float b2, float eps, float wd,
+                                   float b1t, float b2t, const float *__restrict__ betat_dev, uint32_t *flags)
+{
+    pdl_trigger();
+    pdl_wait();
+    if (S_dev) inv = __fdiv_rn(1.0f, __fmul_rn(*S_dev, (float)R));
+    if (any_replica_overflowed(pp, R)) {
+        if (threadIdx.x == 0) atomicOr(flags, 1u);
+        return;
+    }
+    if (betat_dev) { b1t = __fmul_rn(betat_dev[0], mu); b2t = __fmul_rn(betat_dev[1], b2); }
+    const float bc1 = __fsub_rn(1.0f, b1t), bc2 = __fsub_rn(1.0f, b2t);
+    const float omb1 = __fsub_rn(1.0f, mu), omb2 = __fsub_rn(1.0f, b2);
+    const bool use_s1 = KIND != MPT_OPT_SGD || mu != 0.0f;
+    bool bad = false;
+    for (size_t i = begin + threadIdx.x; i < count; i += blockDim.x) {
+        float s = h2f_bits_dp(pp.g[0][first + i]);
+        for (int q = 1; q < R; q++) s = __fadd_rn(s, h2f_bits_dp(pp.g[q][first + i]));
+        float w = w32[i], a = use_s1 ? s1p[i] : 0.0f, b = KIND == MPT_OPT_ADAM ? s2p[i] : 0.0f;
+        opt1<KIND, WD>(s, w, a, b, inv, lr, mu, b2, omb1, omb2, eps, wd, bc1, bc2, 1.0f, bad);
+        w32[i] = w;
+        if (use_s1) s1p[i] = a;
+        if (KIND == MPT_OPT_ADAM) s2p[i] = b;
+        const uint16_t h = (uint16_t)f2h_bits_dp(w);
+        for (int q = 0; q < R; q++) pp.w[q][first + i] = h;
+    }
+    if (bad) atomicOr(flags + 1, 1u);
+}
+
+template <int KIND, bool WD>
+cudaError_t launch_dp_opt(const DpPeers &pp, int R, float *w32, float *s1, float *s2, size_t first, size_t count, float inv,
+                          const float *S_dev, float lr, float mu, float b2, float eps, float wd, float b1t, float b2t,
+                          const float *betat_dev, uint32_t *flags, cudaStream_t st, int *n_launches)
+{
+    const size_t n8 = count / 8;
+    if (n_launches) *n_launches = (n8 ? 1 : 0) + (n8 * 8 < count || count == 0 ? 1 : 0);
+    if (n8)
+        MPT_LAUNCH(k_dp_step_opt<KIND, WD>, dim3((unsigned)((n8 + kDpThreads - 1) / kDpThreads)), dim3(kDpThreads), 0, st, pp, R,
+                   (float4 *)w32, (float4 *)s1, (float4 *)s2, first, n8, inv, S_dev, lr, mu, b2, eps, wd, b1t, b2t, betat_dev,
+                   flags);
+    if (n8 * 8 < count || count == 0)
+        MPT_LAUNCH(k_dp_step_opt_tail<KIND, WD>, dim3(1), dim3(32), 0, st, pp, R, w32, s1, s2, first, n8 * 8, count, inv, S_dev,
+                   lr, mu, b2, eps, wd, b1t, b2t, betat_dev, flags);
+    return cudaGetLastError();
+}
+
 template <bool MOM>
 cudaError_t launch_dp(const DpPeers &pp, int R, float *w32, float *v, size_t first, size_t count, float inv,
                       const float *S_dev, float lr, float mu, uint32_t *flags, cudaStream_t st, int *n_launches)
@@ -179,6 +287,32 @@ cudaError_t launch_dp_step(const uint16_t *const *g16, const uint32_t *const *fl
     }
     return mu != 0.0f ? launch_dp<true>(pp, R, w32_shard, v_shard, first, count, inv_SR, S_dev, lr, mu, flags, st, n_launches)
                       : launch_dp<false>(pp, R, w32_shard, nullptr, first, count, inv_SR, S_dev, lr, mu, flags, st, n_launches);
+}
+
+cudaError_t launch_dp_step_opt(int kind, const uint16_t *const *g16, const uint32_t *const *flag, uint16_t *const *w16, int R,
+                               float *w32_shard, float *s1_shard, float *s2_shard, size_t first, size_t count, float inv_SR,
+                               const float *S_dev, float lr, float mu, float b2, float eps, float wd, float b1t, float b2t,
+                               const float *betat_dev, uint32_t *flags, cudaStream_t st, int *n_launches)
+{
+    DpPeers pp = {};
+    for (int q = 0; q < R; q++) {
+        pp.g[q] = g16[q];
+        pp.flag[q] = flag[q];
+        pp.w[q] = w16[q];
+    }
+#define MPT_DP_OPT(KIND)                                                                                                    \
+    (wd != 0.0f ? launch_dp_opt<KIND, true>(pp, R, w32_shard, s1_shard, s2_shard, first, count, inv_SR, S_dev, lr, mu, b2, eps, \
+                                            wd, b1t, b2t, betat_dev, flags, st, n_launches)                                  \
+                : launch_dp_opt<KIND, false>(pp, R, w32_shard, s1_shard, s2_shard, first, count, inv_SR, S_dev, lr, mu, b2,   \
+                                             eps, wd, b1t, b2t, betat_dev, flags, st, n_launches))
+    switch (kind) {
+        case MPT_OPT_SGD: return MPT_DP_OPT(MPT_OPT_SGD);
+        case MPT_OPT_NESTEROV: return MPT_DP_OPT(MPT_OPT_NESTEROV);
+        case MPT_OPT_ADAGRAD: return MPT_DP_OPT(MPT_OPT_ADAGRAD);
+        case MPT_OPT_ADAM: return MPT_DP_OPT(MPT_OPT_ADAM);
+        default: return cudaErrorInvalidValue;
+    }
+#undef MPT_DP_OPT
 }
 
 }  // namespace mpt
@@ -223,6 +357,34 @@ int mpt_dp_step_flat(const uint16_t *const *g16_peers, const uint32_t *const *fl
     const float inv = 1.0f / (S * (float)R);
     e = launch_dp_step(g16_peers, flag_peers, w16_peers, R, w32_shard_dev, v_shard_dev, lo, count, inv, nullptr, lr, mu, flags_dev,
                        st, nullptr);
+    return e == cudaSuccess ? MPT_OK : MPT_ERR_CUDA;
+}
+
+int mpt_dp_step_flat_opt(const mpt_optimizer *opt, const uint16_t *const *g16_peers, const uint32_t *const *flag_peers,
+                         uint16_t *const *w16_peers, float *w32_shard_dev, float *s1_shard_dev, float *s2_shard_dev, size_t n,
+                         int R, int rank, float S, float b1t, float b2t, uint32_t *flags_dev, void *cuda_stream)
+{
+    if (!opt || !g16_peers || !flag_peers || !w16_peers || !flags_dev) return MPT_ERR_INVALID_ARG;
+    if (opt->kind < MPT_OPT_SGD || opt->kind > MPT_OPT_ADAM || opt->clip_norm != 0.0f) return MPT_ERR_INVALID_ARG;
+    size_t lo = 0, hi = 0;
+    if (mpt_dp_shard(n, R, rank, &lo, &hi) != MPT_OK) return MPT_ERR_INVALID_ARG;
+    if (!(S > 0.0f) || !(opt->lr == opt->lr)) return MPT_ERR_INVALID_ARG;
+    for (int q = 0; q < R; q++) {
+        if (!g16_peers[q] || !flag_peers[q] || !w16_peers[q]) return MPT_ERR_INVALID_ARG;
+        if ((((uintptr_t)g16_peers[q] | (uintptr_t)w16_peers[q]) & 15) != 0 || ((uintptr_t)flag_peers[q] & 3) != 0)
+            return MPT_ERR_INVALID_ARG;
+    }
+    const size_t count = hi - lo;
+    const bool need1 = opt->kind != MPT_OPT_SGD || opt->momentum != 0.0f, need2 = opt->kind == MPT_OPT_ADAM;
+    if (count && (!w32_shard_dev || (need1 && !s1_shard_dev) || (need2 && !s2_shard_dev))) return MPT_ERR_INVALID_ARG;
+    if (count && (((uintptr_t)w32_shard_dev | (uintptr_t)s1_shard_dev | (uintptr_t)s2_shard_dev) & 15) != 0) return MPT_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    cudaError_t e = cudaMemsetAsync(flags_dev + 1, 0, sizeof(uint32_t), st);
+    if (e != cudaSuccess) return MPT_ERR_CUDA;
+    const float inv = 1.0f / (S * (float)R);
+    e = launch_dp_step_opt(opt->kind, g16_peers, flag_peers, w16_peers, R, w32_shard_dev, s1_shard_dev, s2_shard_dev, lo, count, inv,
+                           nullptr, opt->lr, opt->momentum, opt->beta2, opt->eps, opt->weight_decay, b1t, b2t, nullptr, flags_dev, st,
+                           nullptr);
     return e == cudaSuccess ? MPT_OK : MPT_ERR_CUDA;
 }
 

@@ -350,18 +350,26 @@ int do_step(mpt_ctx *c)
     CK(cudaMemsetAsync(c->status + ST_OVERFLOW_SEEN, 0, sizeof(uint32_t), c->stream), "status clear");
     cudaError_t e;
     if (c->dp_R > 1) {
-        if (c->opt_kind != MPT_OPT_SGD || c->wd != 0.0f || c->clip > 0.0f)
-            return fail(c, MPT_ERR_STATE, "the data-parallel step supports SGD with or without momentum only");
+        if (c->clip > 0.0f) return fail(c, MPT_ERR_STATE, "the data-parallel step does not support global-norm clipping");
         size_t lo = 0, hi = 0;
         mpt_dp_shard(c->plan.P_pad, c->dp_R, c->dp_rank, &lo, &hi);
         int nl = 0;
         {
             // bytes through this GPU's memory system: R gradients read, the shard's state, R weight copies written
-            const double per_elem = 2.0 * c->dp_R + 8.0 + (c->use_momentum ? 8.0 : 0.0) + 2.0 * c->dp_R;
+            const double per_elem = 2.0 * c->dp_R + 8.0 + (c->use_momentum ? 8.0 : 0.0) + (c->state2 ? 8.0 : 0.0) + 2.0 * c->dp_R;
             ProfSpan span(c, MPT_PROF_UPDATE, per_elem * (double)(hi - lo));
-            e = launch_dp_step(c->dp_g16, c->dp_flag, c->dp_w16, c->dp_R, c->master + lo, c->use_momentum ? c->mom + lo : nullptr,
-                               lo, hi - lo, 1.0f / (c->S * (float)c->dp_R), (const float *)(c->status + ST_SCALE), c->lr,
-                               c->use_momentum ? c->mu : 0.0f, c->status + ST_OVERFLOW, c->stream, &nl);
+            const float inv_SR = 1.0f / (c->S * (float)c->dp_R);
+            const float *S_dev = (const float *)(c->status + ST_SCALE);
+            if (c->opt_kind == MPT_OPT_SGD && c->wd == 0.0f)
+                e = launch_dp_step(c->dp_g16, c->dp_flag, c->dp_w16, c->dp_R, c->master + lo, c->use_momentum ? c->mom + lo : nullptr,
+                                   lo, hi - lo, inv_SR, S_dev, c->lr, c->use_momentum ? c->mu : 0.0f, c->status + ST_OVERFLOW,
+                                   c->stream, &nl);
+            else
+                e = launch_dp_step_opt(c->opt_kind, c->dp_g16, c->dp_flag, c->dp_w16, c->dp_R, c->master + lo,
+                                       c->mom ? c->mom + lo : nullptr, c->state2 ? c->state2 + lo : nullptr, lo, hi - lo, inv_SR,
+                                       S_dev, c->lr, c->mu, c->beta2, c->eps, c->wd, 1.0f, 1.0f,
+                                       c->opt_kind == MPT_OPT_ADAM ? (const float *)(c->status + ST_B1T) : nullptr,
+                                       c->status + ST_OVERFLOW, c->stream, &nl);
         }
         c->launches += nl;
         if (e != cudaSuccess) return cuda_fail(c, e, "data-parallel step launch");

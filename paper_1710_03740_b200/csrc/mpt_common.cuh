@@ -137,6 +137,11 @@ cudaError_t launch_clip_coef(const uint16_t *g16, size_t n, float inv_S, const f
 cudaError_t launch_dp_step(const uint16_t *const *g16, const uint32_t *const *flag, uint16_t *const *w16, int R,
                            float *w32_shard, float *v_shard, size_t first, size_t count, float inv_SR, const float *S_dev,
                            float lr, float mu, uint32_t *flags, cudaStream_t st, int *n_launches);
+// The same with the optimizer steps of launch_update_opt on the mean gradient (no clipping).
+cudaError_t launch_dp_step_opt(int kind, const uint16_t *const *g16, const uint32_t *const *flag, uint16_t *const *w16, int R,
+                               float *w32_shard, float *s1_shard, float *s2_shard, size_t first, size_t count, float inv_SR,
+                               const float *S_dev, float lr, float mu, float b2, float eps, float wd, float b1t, float b2t,
+                               const float *betat_dev, uint32_t *flags, cudaStream_t st, int *n_launches);
 // End-of-step bookkeeping on the device (one thread): dynamic loss scale (if interval > 0) and
 // Adam's running products beta^t (if adam != 0); both only move on a step that was applied.
 cudaError_t launch_post_step(uint32_t *status, int interval, float backoff, float growth, float min_S, float max_S,

@@ -12,6 +12,7 @@
 // Bit-exactness contract: every FP32 operation is rounded separately (the __f*_rn
 // intrinsics are never contracted into a fused multiply-add), no flush-to-zero.
 #include "mpt_common.cuh"
+#include "update_math.cuh"
 
 namespace mpt {
 
@@ -263,38 +264,6 @@ cudaError_t launch_update(const uint16_t *g16, float *w32, float *v, uint16_t *w
 
 // ------------------------------------------- other optimizer steps, weight decay
 
-// One element; every operation rounded separately, in the order documented in mpt.h.
-template <int KIND, bool WD>
-__device__ __forceinline__ void opt1(uint32_t gh, float &w, float &s1, float &s2, float inv, float lr, float mu, float b2,
-                                     float omb1, float omb2, float eps, float wd, float bc1, float bc2, float coef, bool &bad)
-{
-    float g = __fmul_rn(h2f_bits(gh), inv);
-    bad |= f32_nonfinite(g);
-    g = __fmul_rn(g, coef);     // global-norm clipping coefficient (exactly 1.0f when clipping is off)
-    if (WD) g = __fadd_rn(g, __fmul_rn(wd, w));
-    float u;
-    if (KIND == MPT_OPT_NESTEROV) {
-        s1 = __fadd_rn(__fmul_rn(mu, s1), g);
-        u = __fmul_rn(lr, __fadd_rn(g, __fmul_rn(mu, s1)));
-    } else if (KIND == MPT_OPT_ADAGRAD) {
-        s1 = __fadd_rn(s1, __fmul_rn(g, g));
-        u = __fmul_rn(lr, __fdiv_rn(g, __fadd_rn(__fsqrt_rn(s1), eps)));
-    } else if (KIND == MPT_OPT_ADAM) {
-        s1 = __fadd_rn(__fmul_rn(mu, s1), __fmul_rn(omb1, g));
-        s2 = __fadd_rn(__fmul_rn(b2, s2), __fmul_rn(omb2, __fmul_rn(g, g)));
-        const float mh = __fdiv_rn(s1, bc1), vh = __fdiv_rn(s2, bc2);
-        u = __fmul_rn(lr, __fdiv_rn(mh, __fadd_rn(__fsqrt_rn(vh), eps)));
-    } else {  // SGD with weight decay: momentum iff s1 is in use (mu != 0)
-        if (mu != 0.0f) {
-            s1 = __fadd_rn(__fmul_rn(mu, s1), g);
-            u = __fmul_rn(lr, s1);
-        } else {
-            u = __fmul_rn(lr, g);
-        }
-    }
-    w = __fsub_rn(w, u);
-}
-
 static constexpr int kOptVec = 2;   // vectors per thread (up to 72 bytes of loads each)
 
 template <int KIND, bool WD>
@@ -341,7 +310,7 @@ __global__ void __launch_bounds__(kThreads) k_update_opt(const uint4 *__restrict
 #pragma unroll
             for (int e = 0; e < 8; e++) {
                 const uint32_t gh = (e & 1) ? (gw[e >> 1] >> 16) : (gw[e >> 1] & 0xFFFFu);
-                opt1<KIND, WD>(gh, wf[e >> 2][e & 3], af[e >> 2][e & 3], bf[e >> 2][e & 3], inv, lr, mu, b2, omb1, omb2, eps,
+                opt1<KIND, WD>(h2f_bits(gh), wf[e >> 2][e & 3], af[e >> 2][e & 3], bf[e >> 2][e & 3], inv, lr, mu, b2, omb1, omb2, eps,
                                wd, bc1, bc2, coef, bad);
             }
             uint4 h;
@@ -378,7 +347,7 @@ __global__ void k_update_opt_scalar(const uint16_t *__restrict__ g16, float *__r
     bool bad = false;
     for (size_t i = begin + (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
         float w = w32[i], a = use_s1 ? s1p[i] : 0.0f, b = KIND == MPT_OPT_ADAM ? s2p[i] : 0.0f;
-        opt1<KIND, WD>(g16[i], w, a, b, inv, lr, mu, b2, omb1, omb2, eps, wd, bc1, bc2, coef, bad);
+        opt1<KIND, WD>(h2f_bits(g16[i]), w, a, b, inv, lr, mu, b2, omb1, omb2, eps, wd, bc1, bc2, coef, bad);
         w32[i] = w;
         if (use_s1) s1p[i] = a;
         if (KIND == MPT_OPT_ADAM) s2p[i] = b;

@@ -142,6 +142,59 @@ def test_dp_empty_problem_and_bad_arguments():
         b.mpt_dp_step_flat([t, t], [f, f], [t, t], w32, None, 64, 2, 0, 1.0, 0.1, 0.9, f)      # momentum without state
 
 
+@pytest.mark.parametrize("wd", [0.0, 0.01])
+@pytest.mark.parametrize("kind", [0, 1, 2, 3])
+@pytest.mark.parametrize("R,n", [(2, 8 * 256 + 5), (3, 4099), (8, (1 << 18) + 3)])
+def test_dp_step_other_optimizers_bit_exact(R, n, kind, wd):
+    """Weight decay, Nesterov, Adagrad, Adam on the mean gradient (section 4.5 trains its
+    multi-GPU language model with Adagrad), emulated replicas, against the oracle."""
+    if kind == 0 and wd == 0.0:
+        pytest.skip("plain SGD(+momentum) is covered above")
+    b = _binding()
+    S, lr, mu, b2, eps = 512.0, 0.01, 0.9, 0.999, 1e-8
+    gs, w, _ = _inputs(n, R, seed=n + kind)
+    rng = np.random.default_rng(kind + 7)
+    s1 = np.abs(0.1 * rng.standard_normal(n)).astype(np.float32)
+    s2 = np.abs(0.01 * rng.standard_normal(n)).astype(np.float32)
+    b1t, b2t = np.float32(0.81), np.float32(0.998)
+    opt = b.Optimizer(kind, lr, mu, b2, eps, wd, 0.0)
+    npad = n + 8
+    g_dev = [torch.zeros(npad, dtype=torch.int16, device="cuda") for _ in range(R)]
+    h_dev = [torch.full((npad,), 0x1234, dtype=torch.int16, device="cuda") for _ in range(R)]
+    f_dev = [torch.zeros(2, dtype=torch.int32, device="cuda") for _ in range(R)]
+    for q in range(R):
+        g_dev[q][:n] = dev(gs[q].view(np.uint16))
+    full = [torch.zeros(npad, dtype=torch.float32, device="cuda") for _ in range(3)]
+    for t, a in zip(full, (w, s1, s2)):
+        t[:n] = dev(a)
+    for q in range(R):
+        lo, hi = b.mpt_dp_shard(n, R, q)
+        b.mpt_dp_step_flat_opt(opt, g_dev, f_dev, h_dev, full[0][lo:], full[1][lo:], full[2][lo:] if kind == 3 else None,
+                               n, R, q, S, float(b1t), float(b2t), f_dev[q])
+    torch.cuda.synchronize()
+    rw, r1, r2, rh = w.copy(), s1.copy(), s2.copy(), np.zeros(n, np.uint16)
+    use_s1 = kind != 0 or mu != 0.0
+    mpo.dp_update_apply_opt(kind, [g.view(np.uint16) for g in gs], rw, r1 if use_s1 else None, r2 if kind == 3 else None, rh,
+                            S, lr, mu, b2, eps, wd, np.float32(1.0) - b1t, np.float32(1.0) - b2t)
+    assert np.array_equal(full[0][:n].cpu().numpy().view(np.uint32), rw.view(np.uint32))
+    assert np.array_equal(full[1][:n].cpu().numpy().view(np.uint32), r1.view(np.uint32))
+    assert np.array_equal(full[2][:n].cpu().numpy().view(np.uint32), (r2 if kind == 3 else s2).view(np.uint32))
+    for q in range(R):
+        assert np.array_equal(host_u16(h_dev[q][:n]), rh)
+        assert np.all(host_u16(h_dev[q][n:]) == 0x1234)
+        assert f_dev[q].cpu().numpy().tolist() == [0, 0]
+
+
+def test_dp_step_opt_rejects_clipping():
+    b = _binding()
+    t = torch.zeros(64, dtype=torch.int16, device="cuda")
+    f = torch.zeros(2, dtype=torch.int32, device="cuda")
+    w32 = torch.zeros(64, dtype=torch.float32, device="cuda")
+    with pytest.raises(b.MptError):
+        b.mpt_dp_step_flat_opt(b.Optimizer(2, 0.1, 0.0, 0.0, 1e-8, 0.0, 1.0), [t, t], [f, f], [t, t], w32, w32, None, 64, 2, 0,
+                               1.0, 1.0, 1.0, f)
+
+
 # ---------------------------------------------------------------- two processes, mapped buffers
 
 
@@ -234,7 +287,7 @@ def _mlp_batch(t, q):
     return x, y
 
 
-def _mlp_replica_main(rank, R, port, out_dir, dynamic=False):
+def _mlp_replica_main(rank, R, port, out_dir, dynamic=False, opt_kind=0):
     import datetime
     import torch as th
     import torch.distributed as dist
@@ -243,7 +296,8 @@ def _mlp_replica_main(rank, R, port, out_dir, dynamic=False):
     dist.init_process_group("gloo", init_method="tcp://127.0.0.1:%d" % port, rank=rank, world_size=R,
                             timeout=datetime.timedelta(seconds=90))
     try:
-        dp = b.DataParallelMLP(_MLP_LAYERS, _MLP["S"], _MLP["lr"], _MLP["mu"], max_batch=_MLP["batch"])
+        opt = b.Optimizer(opt_kind, _MLP["lr"], _MLP["mu"], 0.999, 1e-8, 0.001, 0.0) if opt_kind else None
+        dp = b.DataParallelMLP(_MLP_LAYERS, _MLP["S"], _MLP["lr"], _MLP["mu"], max_batch=_MLP["batch"], optimizer=opt)
         L = len(_MLP_LAYERS)
         for l, w in enumerate(_mlp_masters()):
             dp.ctx.set_master(l, w)
@@ -354,6 +408,49 @@ def test_dp_mlp_two_processes_dynamic_scale(tmp_path):
                 want16 = ora.replicas[0].w16[l]
                 assert np.array_equal(rec[q]["inj_w16_%d_%d" % (t, l)].reshape(want16.shape), want16), (t, l, q)
     assert scales[1] == _MLP["S"] / 2          # the skipped step halved the scale everywhere
+    for t in range(_MLP["e2e_steps"]):
+        xs, ys = zip(*[_mlp_batch(t, q) for q in range(R)])
+        losses = ora.forward_backward(list(xs), list(ys))
+        for q in range(R):
+            got = float(rec[q]["e2e_loss_%d" % t])
+            assert abs(got - losses[q]) <= 1e-3 * abs(losses[q]), (t, q, got, losses[q])
+            for l in range(L):
+                ora.set_grad(q, l, rec[q]["e2e_g16_%d_%d" % (t, l)])
+        skipped = ora.step()
+        for q in range(R):
+            assert bool(rec[q]["e2e_skip_%d" % t]) == bool(skipped)
+            for l in range(L):
+                want16 = ora.replicas[0].w16[l]
+                assert np.array_equal(rec[q]["e2e_w16_%d_%d" % (t, l)].reshape(want16.shape), want16), (t, l, q)
+
+
+@pytest.mark.timeout(300)
+@pytest.mark.parametrize("kind", [2, 3])
+def test_dp_mlp_two_processes_adagrad_adam(tmp_path, kind):
+    """Two attached contexts stepping with Adagrad (the optimizer of the paper's multi-GPU language
+    model, section 4.5) or Adam, with weight decay: FP16 weights of both replicas bit-exact against
+    the oracle's replicas through a skipped step; Adam's running beta products stay in step."""
+    import torch.multiprocessing as mp
+    from oracle.dp import OracleDataParallelMLP
+    R = 2
+    mp.spawn(_mlp_replica_main, args=(R, _free_port(), str(tmp_path), False, kind), nprocs=R, join=True)
+    rec = [np.load(os.path.join(str(tmp_path), "m%d.npz" % q)) for q in range(R)]
+    L = len(_MLP_LAYERS)
+    ora = OracleDataParallelMLP(_MLP_LAYERS, _MLP["S"], _MLP["lr"], _MLP["mu"], R)
+    ora.set_optimizer(kind, _MLP["lr"], _MLP["mu"], b2=0.999, eps=1e-8, wd=0.001)
+    for l, w in enumerate(_mlp_masters()):
+        ora.set_master(l, w)
+    for t in range(_MLP["inj_steps"]):
+        for q in range(R):
+            for l in range(L):
+                ora.set_grad(q, l, _mlp_injected_grad(t, q, l).view(np.uint16))
+        skipped = ora.step()
+        assert skipped == (1 if t == 1 else 0)
+        for q in range(R):
+            assert bool(rec[q]["inj_skip_%d" % t]) == bool(skipped)
+            for l in range(L):
+                want16 = ora.replicas[0].w16[l]
+                assert np.array_equal(rec[q]["inj_w16_%d_%d" % (t, l)].reshape(want16.shape), want16), (t, l, q)
     for t in range(_MLP["e2e_steps"]):
         xs, ys = zip(*[_mlp_batch(t, q) for q in range(R)])
         losses = ora.forward_backward(list(xs), list(ys))
