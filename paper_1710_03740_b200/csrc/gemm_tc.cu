@@ -30,12 +30,12 @@ static constexpr int A_STAGE_BYTES = BLOCK_M * BLOCK_K * 2;  // 16 KB
 static constexpr int MN_BOX_BYTES = 64 * BLOCK_K * 2;        // one 64(mn) x 64(k) box of an MN-major operand
 
 // Tile width BN is 256 (four 48 KB stages) or, for outputs with too few 128x256 tiles to fill
-// the SMs, 128 (six 32 KB stages).  The two accumulator buffers take 2 * BN tensor-memory columns.
+// the SMs, 128 (six 32 KB stages) or 64 (eight 24 KB stages).  The two accumulator buffers take 2 * BN tensor-memory columns.
 template <int BN>
 struct TileCfg {
     static constexpr int B_STAGE_BYTES = BN * BLOCK_K * 2;
     static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
-    static constexpr int STAGES = BN == 256 ? 4 : 6;
+    static constexpr int STAGES = BN == 256 ? 4 : (BN == 128 ? 6 : 8);
     static constexpr int TMEM_COLS = 2 * BN;
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
@@ -443,7 +443,9 @@ static cudaError_t launch_bn(int op, int M, int N, int K, const uint16_t *A, int
 // Tile width and split factor for the single-CTA kernel.  Cost model in tensor-pipe cycles: a
 // 128x256 tile needs 512 cycles per 64-deep k-block; a 128x128 tile needs 256 but runs at about
 // 0.6 of that rate (operand reads from shared memory bound it); measured per k-block: about 600
-// and 437 cycles.  The epilogue of a tile costs about 400 cycles per 32 columns and is exposed
+// and 437 cycles; a 128x64 tile takes as long as a 128x128 one per k-block (about 450: the A
+// operand's shared-memory reads do not shrink with the tile), so it only pays when it fills more
+// SMs or saves the second launch of a split.  The epilogue of a tile costs about 400 cycles per 32 columns and is exposed
 // for the last tile of a CTA; a launch costs about 14000 cycles; a split adds a second, mostly
 // overlapped launch (about 4000) and one FP32 write and read of the output per part, which
 // stays in L2 (about 64 bytes per cycle and SM).  Calibrated with launches replayed from a CUDA
@@ -455,10 +457,10 @@ void tc_gemm_plan(int M, int N, int K, size_t ws_bytes, int *bn_out, int *split_
     const int nkb = (K + BLOCK_K - 1) / BLOCK_K;
     double best = 1e30;
     int best_bn = 256, best_s = 1;
-    for (int bn : {256, 128}) {
-        if (bn == 128 && N <= 128) continue;
+    for (int bn : {256, 128, 64}) {
+        if (bn < 256 && N <= bn) continue;
         const long tiles = tm * ((N + bn - 1) / bn);
-        const double cyc = bn == 256 ? 600.0 : 437.0;
+        const double cyc = bn == 256 ? 600.0 : (bn == 128 ? 437.0 : 450.0);
         for (int s = 1; s <= 8; s++) {
             if (s > 1 && (nkb / s < 8)) break;
             const size_t need = s > 1 ? (size_t)s * M * (((size_t)N + 31) / 32 * 32) * 4 : 0;
@@ -520,7 +522,8 @@ cudaError_t launch_gemm_tc(int op, int M, int N, int K, const uint16_t *A, int l
     p.split_k = split;
     p.partial = splitk_ws;
     p.ldp = (N + 31) / 32 * 32;
-    if (bn == 128) return launch_bn<128>(op, M, N, K, A, lda, B, ldb, p, st);
+    if (bn == 64 && !lstm) return launch_bn<64>(op, M, N, K, A, lda, B, ldb, p, st);
+    if (bn <= 128) return launch_bn<128>(op, M, N, K, A, lda, B, ldb, p, st);
     return launch_bn<256>(op, M, N, K, A, lda, B, ldb, p, st);
 }
 

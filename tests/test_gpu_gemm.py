@@ -122,7 +122,8 @@ def _check_tc(op, M, N, K, flags=0, mask=None, seed=21, scale=None, want_flag=Fa
 
 
 TC_SHAPES = [(128, 256, 64), (128, 256, 256), (256, 512, 128), (128, 256, 72), (200, 304, 136),
-             (64, 16, 512), (8, 8, 8), (384, 768, 1024), (1024, 1024, 1024)]
+             (64, 16, 512), (8, 8, 8), (384, 768, 1024), (1024, 1024, 1024),
+             (1000, 1016, 1032)]      # the last two take 128x64 tiles (ragged in every dimension here)
 
 
 PAIR_SHAPES = [(256, 256, 64), (256, 256, 448), (512, 768, 128), (256, 512, 72), (392, 560, 136),
