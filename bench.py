@@ -382,6 +382,17 @@ def main():
                                      "device_error": r["device_error"]}
             except Exception as ex:  # an extra; never fatal for the bench line
                 out["lstm_layer"] = {"error": repr(ex)}
+            # not part of the step metric either: the data-parallel step of one replica of 8 for a
+            # 151 M parameter model, with all eight replicas' buffers on this GPU (the kernel's own
+            # rate; nothing here crosses NVLink)
+            try:
+                from paper_1710_03740_b200.kernel_bench import bench_dp
+                r = bench_dp(150994944, 8, 1, 10)
+                out["dp_step"] = {"replicas": r["replicas"], "params": r["params"], "shard": r["shard"], "ms": r["median_ms"],
+                                  "gbs": r["median_gbs"], "bytes_per_shard_element": r["bytes_per_shard_element"],
+                                  "peers": r["peers"], "link_bytes_each_way_if_remote": r["link_bytes_each_way_if_remote"]}
+            except Exception as ex:
+                out["dp_step"] = {"error": repr(ex)}
         if not args.no_cpu_baseline:
             try:
                 out["cpu_baseline"] = oracle_sample(cfg)
