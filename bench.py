@@ -8,9 +8,11 @@ One "step" is one pass of the whole hot path over one batch: mpt_forward,
 mpt_backward_scaled, mpt_step.  The default workload "large" is the large-MLP
 configuration (8 x 12288^2 ReLU layers + 12288 -> 32000 head, batch 4096, S = 8192,
 SGD momentum 0.9); "large_twin" and "tiny" are small cases.  Prints ONE JSON line on
-rank 0.  With N > 1 (launched by torch.distributed.run) every rank runs an independent
-replica of the step on its own GPU (the path has no exchange step); the time is the
-maximum over ranks and the value the sum of all ranks' work over that time.
+rank 0.  With N > 1 every rank runs an independent replica of the step on its own GPU (the
+path has no exchange step); the time is the maximum over ranks and the value the sum of all
+ranks' work over that time.  `--gpus N` run plainly (no WORLD_SIZE in the environment) starts
+its own N ranks under torch.distributed.run on 127.0.0.1; launched by torch.distributed.run it
+takes rank and world size from the environment, and the two must agree.
 """
 from __future__ import annotations
 
@@ -19,6 +21,7 @@ import json
 import os
 import subprocess
 import sys
+import tempfile
 import threading
 import time
 
@@ -34,6 +37,85 @@ UNIT = "TFLOP/s"
 NOMINAL_FP16_TFLOPS = 2250.0
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def spawn_ranks(n, argv):
+    """Re-runs this script as n ranks of one node under torch.distributed.run (rendezvous on
+    127.0.0.1, a free port) and returns its exit code.  Rank 0's JSON line goes to stdout."""
+    import socket
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(n),
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
+    return subprocess.call(cmd)
+
+
+def rank_check(args, rank, world):
+    """The rank plumbing of the N > 1 path without a GPU: gloo ranks, a made-up per-rank time,
+    maximum over ranks, whole-job value, one line from rank 0.  Used by the CPU tests."""
+    import torch.distributed as dist
+    if world > 1:
+        dist.init_process_group("gloo")
+    ms = max_over_ranks([10.0 + rank])[0]
+    if rank == 0:
+        print(json.dumps({"rank_check": True, "n_gpus": world, "gpus_arg": args.gpus, "ms_per_step": ms,
+                          "value": job_tflops(1e12, world, ms), "scaling": "weak"}), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def bench_config(args, cfg):
+    """The `config` object of the JSON line; both arms print the same one."""
+    return {"workload": args.workload, "layers": len(cfg["layers"]), "batch": cfg["batch"], "params": n_params(cfg),
+            "S": cfg["S"], "momentum": cfg["momentum"], "parallelism": "replicas only",
+            "l2": "inputs larger than L2 (weights %.1f GB per pass)" % (n_params(cfg) * 2 / 1e9),
+            "flop_per_step": step_flops(cfg)}
+
+
+def dp_step_over_peers(n, iters, dev):
+    """The data-parallel step (one kernel per replica: gradient reduce-scatter over peer loads,
+    master pass on the owned shard, FP16 weight all-gather over peer stores) across the N GPUs of
+    this job: every rank owns exchange buffers the others map.  Times the kernel with CUDA events
+    between process-group barriers; returns the slowest rank's median and the bytes each GPU pulls
+    and pushes over NVLink per step.  An extra: not part of the step metric."""
+    import torch
+    import torch.distributed as dist
+    from paper_1710_03740_b200 import binding as mpt
+    dp, err = None, None
+    try:
+        dp = mpt.DataParallelFlat(n, 512.0, 1e-4, 0.9)
+    except Exception as ex:       # e.g. no peer access between two of the GPUs
+        err = repr(ex)
+    # every rank must agree to go on: the timing loop below is full of barriers
+    ok = torch.tensor([0 if dp is None else 1], dtype=torch.int32, device=dev)
+    dist.all_reduce(ok, op=dist.ReduceOp.MIN)
+    if int(ok.item()) == 0:
+        return {"error": err or "set-up failed on another rank"}
+    g = torch.Generator(device=dev).manual_seed(3 + dp.rank)
+    dp.g16.copy_((torch.randn(n, device=dev, generator=g) * 37).half().view(torch.int16))
+    times = []
+    for it in range(iters + 2):
+        dp._barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        mpt.mpt_dp_step_flat([p["g16"] for p in dp._peers], [p["flags"] for p in dp._peers], [p["w16"] for p in dp._peers],
+                             dp.w32, dp.v, dp.n, dp.R, dp.rank, dp.S, dp.lr, dp.mu, dp._own["flags"])
+        e1.record()
+        dp._barrier()
+        if it >= 2:
+            times.append(e0.elapsed_time(e1))
+    times.sort()
+    med = max_over_ranks([times[len(times) // 2]], dev)[0]
+    shard = dp.hi - dp.lo
+    link = 2 * shard * (dp.R - 1)
+    res = {"replicas": dp.R, "params": n, "shard": shard, "ms": med, "peers": "remote (one GPU per replica)",
+           "link_bytes_each_way": link, "link_gbs_each_way": link / med / 1e6,
+           "hbm_bytes": (2 + 16 + 2) * shard}
+    dp.close()
+    return res
 
 
 def step_flops(cfg):
@@ -205,7 +287,8 @@ def run_reference(args, cfg, rank):
     out = {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
            "vs_baseline": None, "dtype": "f16", "data": "synthetic",
-           "config": {"workload": args.workload, "note": "CPU oracle, bounded sample per step, extrapolated"},
+           "config": bench_config(args, cfg),
+           "note": "CPU oracle, bounded sample per step, extrapolated to a whole step",
            "cpu_baseline": {"value": v, "unit": UNIT, "cores": vals[-1]["cores"], "kind": "oracle", "sample": sample},
            "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
            "gpu_launches": 0}
@@ -221,14 +304,24 @@ def main():
     ap.add_argument("--workload", default="large", choices=sorted(inputs.MLP_CONFIGS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the LSTM-layer timing appended to the JSON line")
+    ap.add_argument("--rank-check", action="store_true", help="run only the rank plumbing on CPU (gloo); for tests")
     args = ap.parse_args()
+    if args.gpus < 1:
+        raise SystemExit("--gpus must be >= 1")
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not (args.impl == "reference"):
+        sys.exit(spawn_ranks(args.gpus, sys.argv[1:]))
     args.warmup = max(args.warmup, 3) if args.impl == "mine" else args.warmup
     cfg = inputs.MLP_CONFIGS[args.workload]
 
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "mine" and world != args.gpus:
+        raise SystemExit("--gpus %d but WORLD_SIZE=%d: launch with --nproc-per-node equal to --gpus" % (args.gpus, world))
 
+    if args.rank_check:
+        rank_check(args, rank, world)
+        return
     if args.impl == "reference":
         run_reference(args, cfg, rank)
         return
@@ -241,7 +334,12 @@ def main():
         raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
+    nccl_log = None
     if world > 1:
+        # keep NCCL's communicator log (transport, NVLS or not) but out of stdout, where the one JSON line goes
+        os.environ.setdefault("NCCL_DEBUG", "INFO")
+        os.environ.setdefault("NCCL_DEBUG_FILE", os.path.join(tempfile.gettempdir(), "mpt_bench_nccl_%h_%p.log"))
+        nccl_log = os.environ["NCCL_DEBUG_FILE"]
         dist.init_process_group("nccl", device_id=dev)
 
     # ---- synthetic inputs (seeded; rank r uses seed + 100 r so replicas differ)
@@ -325,6 +423,11 @@ def main():
 
     ms_total, ms_e2e = max_over_ranks([ms_total, ms_e2e], dev)
 
+    dp_peers = None
+    if world > 1 and not args.no_extras:
+        # every rank takes part; rank 0 reports.  Not part of the step metric.
+        dp_peers = dp_step_over_peers(150994944, 10, dev)
+
     if rank == 0:
         peaks, peak_src = measured_peaks()
         fl = step_flops(cfg)
@@ -344,15 +447,15 @@ def main():
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f16", "data": "synthetic",
-            "config": {"workload": args.workload, "layers": L, "batch": cfg["batch"], "params": n_params(cfg),
-                       "S": cfg["S"], "momentum": cfg["momentum"], "parallelism": "replicas only",
-                       "l2": "inputs larger than L2 (weights %.1f GB per pass)" % (n_params(cfg) * 2 / 1e9),
-                       "flop_per_step": fl},
+            "config": bench_config(args, cfg),
             "frac_of_nominal_fp16_peak": value / world / NOMINAL_FP16_TFLOPS,
             "roofline": {"bound": "tensor", "kernel": "pair::k_gemm_tc2 (all GEMM launches of the step)",
                          "achieved": gemm_tflops, "peak": peak_t, "peak_source": peak_src + " (sustained bf16 GEMM; fp16 has the same nominal rate)",
                          "unit": "TFLOP/s", "frac": (gemm_tflops / peak_t) if gemm_tflops else None,
                          "frac_of_nominal": (gemm_tflops / NOMINAL_FP16_TFLOPS) if gemm_tflops else None,
+                         "frac_of_clock_ceiling": (gemm_tflops * 1e12 / (148 * 8192 * clocks["sm_mhz"] * 1e6))
+                         if gemm_tflops and clocks and clocks.get("sm_mhz") else None,
+                         "clock_ceiling_note": "148 SMs x 8192 dense FP16 flop per clock x median sampled SM clock",
                          "launches": g_n, "avg_launch_ms": g_ms / g_n if g_n else None, "traffic": traffic,
                          "traffic_note": ("ncu dram bytes of one %s launch; algorithmic minimum %.3e"
                                           % (tr["launch"], tr["algorithmic_bytes"])) if tr else None},
@@ -393,6 +496,10 @@ def main():
                                   "peers": r["peers"], "link_bytes_each_way_if_remote": r["link_bytes_each_way_if_remote"]}
             except Exception as ex:
                 out["dp_step"] = {"error": repr(ex)}
+        if dp_peers is not None:
+            out["dp_step"] = dp_peers
+        if nccl_log:
+            out["nccl_log"] = nccl_log
         if not args.no_cpu_baseline:
             try:
                 out["cpu_baseline"] = oracle_sample(cfg)

@@ -20,10 +20,16 @@
  *     is round-to-nearest-even with gradual underflow everywhere.
  *   - "_dev" pointers are CUDA device pointers, "_host" pointers are host
  *     pointers (pageable or pinned).  Nothing in a signature is a torch type.
- *   - The library never allocates or frees device memory, never creates a
- *     stream, and keeps no global state.  The caller owns the workspace, the
- *     inputs, the stream and all host buffers; the library owns only its
- *     host-side context object.
+ *   - The model-level calls (mpt_create ... mpt_destroy) and the stateless launchers never
+ *     allocate or free device memory and never create a stream.  The caller owns the
+ *     workspace, the inputs, the stream and all host buffers; the library owns only its
+ *     host-side context object.  Exceptions, each documented at its declaration:
+ *     mpt_dp_alloc / mpt_dp_free obtain and release device memory from the driver;
+ *     mpt_softmax_ce_static uses a fixed device array inside the library that all calls on a
+ *     GPU share; and the launchers keep small per-device host-side caches that are filled on
+ *     first use (SM count, opt-in shared-memory sizes, cluster occupancy, the address of that
+ *     array).  Because of those caches the FIRST call of each kernel on a device makes CUDA
+ *     runtime queries and must come before any stream capture.
  *   - Every call returns MPT_OK (0) or a negative MPT_ERR_* code and never
  *     throws.  A null context or a null required pointer gives
  *     MPT_ERR_INVALID_ARG with nothing dereferenced.  Calls are asynchronous on
@@ -222,9 +228,9 @@ int mpt_train_step_staged(mpt_ctx *ctx, float *loss_host, int *overflow_host);
 int mpt_set_scale(mpt_ctx *ctx, float S);
 int mpt_set_lr(mpt_ctx *ctx, float lr);
 
-/* Dynamic loss scaling (the paper's closing section: the scale "could be dynamically increased
- * or decreased by inspecting the weight gradients for overflow, skipping weight updates when
- * an overflow is detected"; no schedule is given there).  The schedule taken here: after a
+/* Dynamic loss scaling (section 5 proposes adjusting S up or down from the overflow history of
+ * the weight gradients, with overflowing steps skipped; it gives no schedule).  The schedule
+ * taken here: after a
  * step that overflowed (and was skipped) S <- max(S/2, min_scale); after growth_interval
  * consecutive steps without overflow S <- min(2*S, max_scale); either event restarts the
  * count.  S stays a power of two if it starts as one, so scaling remains exact.  The scale
@@ -430,10 +436,12 @@ int mpt_add_f16(const uint16_t *a, int lda, const uint16_t *b, int ldb, uint16_t
  * as in mpt_backward_scaled.  z_dev/dz_dev: FP16 [B, C] with pitches ldz/lddz
  * (the two must not overlap).  row_loss_dev: float [B] scratch; loss_dev: one float,
  * receives the unscaled mean; bad_labels_dev: one uint32, receives the number of
- * labels outside [0, C) (may be null). */
+ * labels outside [0, C) (may be null).  status_dev (may be null): one uint32 the caller has
+ * zeroed; the kernel that stages rows with asynchronous bulk copies writes a non-zero
+ * time-out code there if one of its bounded waits runs out (rows are then left unwritten). */
 int mpt_softmax_ce(const uint16_t *z_dev, int ldz, const int32_t *labels_dev, int B, int C, float S,
                    uint16_t *dz_dev, int lddz, float *row_loss_dev, float *loss_dev,
-                   uint32_t *bad_labels_dev, void *cuda_stream);
+                   uint32_t *bad_labels_dev, uint32_t *status_dev, void *cuda_stream);
 
 /* mpt_softmax_ce without the caller-provided scratch.  (The paper has no counterpart:
  * this entry point exists for the sake of callers, not of the method.)
@@ -452,7 +460,9 @@ int mpt_softmax_ce(const uint16_t *z_dev, int ldz, const int32_t *labels_dev, in
  *     MPT_ERR_SHAPE and launches nothing; use mpt_softmax_ce for such batches.
  *   - The first call made on a device looks up the array's device address (a host-side
  *     runtime query, done once per device with that device current).  Make that first
- *     call during set-up, before any stream capture.
+ *     call during set-up, before any stream capture.  The stream must belong to the
+ *     current device (the address looked up is the current device's): a stream of another
+ *     device returns MPT_ERR_INVALID_ARG.
  *   - All calls on a GPU share the one array.  Two calls whose kernels overlap on the
  *     GPU (different streams, or different threads) race on it and may return wrong
  *     losses; calls on one stream are ordered and safe.  The array keeps the previous
@@ -462,7 +472,25 @@ int mpt_softmax_ce(const uint16_t *z_dev, int ldz, const int32_t *labels_dev, in
 #define MPT_SOFTMAX_STATIC_MAX_ROWS 65536
 int mpt_softmax_ce_static(const uint16_t *z_dev, int ldz, const int32_t *labels_dev, int B, int C, float S,
                           uint16_t *dz_dev, int lddz, float *loss_dev, uint32_t *bad_labels_dev,
-                          void *cuda_stream);
+                          uint32_t *status_dev, void *cuda_stream);
+
+/* Self-test of the bounded device-side waits (no counterpart in the paper: its only failure is
+ * the gradient overflow of section 3.2).  Every pipeline kernel of this library waits on its
+ * barriers for a limited time (2 s), then records a code in a status word and returns, so that
+ * a fault in a copy or a peer can never hang the GPU.  These two calls make exactly that
+ * happen on purpose, harmlessly: one CTA waits limit_us microseconds (1 .. 2,000,000) on a
+ * barrier that nothing signals, gives up, writes its code and exits; the CUDA context stays
+ * usable.
+ *   mpt_selftest_wait_timeout      stateless.  status_dev: one uint32 the caller has zeroed.
+ *                                  Synchronises the stream and returns MPT_ERR_TIMEOUT when the
+ *                                  kernel reported the expiry (the expected outcome; the word is
+ *                                  left set), MPT_OK if the word stayed zero.
+ *   mpt_selftest_wait_timeout_ctx  the same through a context: the code lands in the context's
+ *                                  status block, the call returns MPT_ERR_TIMEOUT and the context
+ *                                  is poisoned exactly as after a real expiry (only
+ *                                  mpt_last_error and mpt_destroy succeed afterwards). */
+int mpt_selftest_wait_timeout(unsigned limit_us, uint32_t *status_dev, void *cuda_stream);
+int mpt_selftest_wait_timeout_ctx(mpt_ctx *ctx, unsigned limit_us);
 
 /* ------------------------------------------------------------ data-parallel step
  *

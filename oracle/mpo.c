@@ -454,31 +454,12 @@ void mpo_update_apply_clip(int kind, const uint16_t *g16, float *w32, float *s1,
                            size_t n, float inv_S, float coef, float lr, float mu, float b2, float eps, float wd,
                            float bc1, float bc2)
 {
-    /* scale the gradient through a temporary binary32 copy, then reuse the step with inv = 1:
-     * h2f(g)*inv*coef has to be formed before the step, which takes binary16 input, so the
-     * step is restated here on binary32 gradients */
     const float omb1 = 1.0f - mu, omb2 = 1.0f - b2;
 #pragma omp parallel for schedule(static)
     for (size_t i = 0; i < n; i++) {
-        float w = w32[i];
         float g = mpo_h2f(g16[i]) * inv_S;
         g = g * coef;
-        if (wd != 0.0f) { float t = wd * w; g = g + t; }
-        float u;
-        if (kind == 1) {
-            float a = mu * s1[i]; float v = a + g; s1[i] = v; float b = mu * v; float c = g + b; u = lr * c;
-        } else if (kind == 2) {
-            float q = g * g; float h = s1[i] + q; s1[i] = h; float r = sqrtf(h); float d = r + eps; float c = g / d; u = lr * c;
-        } else if (kind == 3) {
-            float a = mu * s1[i]; float b = omb1 * g; float m = a + b; s1[i] = m;
-            float q = g * g; float c = b2 * s2[i]; float d = omb2 * q; float v = c + d; s2[i] = v;
-            float mh = m / bc1; float vh = v / bc2; float r = sqrtf(vh); float e = r + eps; float f = mh / e; u = lr * f;
-        } else if (s1) {
-            float a = mu * s1[i]; float v = a + g; s1[i] = v; u = lr * v;
-        } else {
-            u = lr * g;
-        }
-        w = w - u;
+        float w = mpo_opt_elem(kind, g, w32[i], s1, s2, i, lr, mu, b2, eps, wd, omb1, omb2, bc1, bc2);
         w32[i] = w;
         w16[i] = mpo_f2h(w);
     }

@@ -32,6 +32,7 @@ EXPORTS = ["mpt_workspace_bytes", "mpt_create", "mpt_workspace_bytes_opt", "mpt_
            "mpt_profile_read", "mpt_last_error",
            "mpt_destroy", "mpt_gemm_f16", "mpt_gemm_f16_ws", "mpt_gemm_workspace_bytes", "mpt_recast", "mpt_grad_nonfinite", "mpt_update_flat",
            "mpt_softmax_ce", "mpt_softmax_ce_static", "mpt_version",
+           "mpt_selftest_wait_timeout", "mpt_selftest_wait_timeout_ctx",
            "mpt_lstm_forward", "mpt_lstm_backward", "mpt_lstm_cell_forward", "mpt_lstm_cell_backward", "mpt_bias_grad",
            "mpt_add_f16",
            "mpt_dp_shard", "mpt_dp_step_flat", "mpt_dp_alloc", "mpt_dp_free", "mpt_dp_export", "mpt_dp_open", "mpt_dp_close",
@@ -121,8 +122,10 @@ def lib() -> C.CDLL:
     L.mpt_recast.argtypes = [vp, vp, sz, vp]
     L.mpt_grad_nonfinite.argtypes = [vp, sz, f32, vp, vp]
     L.mpt_update_flat.argtypes = [vp, vp, vp, vp, sz, f32, f32, f32, i32, i32, vp, vp]
-    L.mpt_softmax_ce.argtypes = [vp, i32, vp, i32, i32, f32, vp, i32, vp, vp, vp, vp]
-    L.mpt_softmax_ce_static.argtypes = [vp, i32, vp, i32, i32, f32, vp, i32, vp, vp, vp]
+    L.mpt_softmax_ce.argtypes = [vp, i32, vp, i32, i32, f32, vp, i32, vp, vp, vp, vp, vp]
+    L.mpt_softmax_ce_static.argtypes = [vp, i32, vp, i32, i32, f32, vp, i32, vp, vp, vp, vp]
+    L.mpt_selftest_wait_timeout.argtypes = [u32, vp, vp]
+    L.mpt_selftest_wait_timeout_ctx.argtypes = [vp, u32]
     L.mpt_lstm_forward.argtypes = [C.POINTER(LstmDesc), C.POINTER(LstmTensors), vp]
     L.mpt_lstm_backward.argtypes = [C.POINTER(LstmDesc), C.POINTER(LstmTensors), vp]
     L.mpt_lstm_cell_forward.argtypes = [i32, i32, i32, vp, i32, vp, i32, vp, vp, i32, vp, i32, vp, i32, vp, i32, u32, vp, vp]
@@ -357,6 +360,14 @@ class Context:
     def set_adam_products(self, b1t, b2t):
         _check(lib().mpt_set_adam_products(self._ctx, float(b1t), float(b2t)), self._ctx)
 
+    def selftest_wait_timeout(self):
+        """Makes a bounded device-side wait run out inside this context (1 ms limit): raises
+        MptError(MPT_ERR_TIMEOUT) and leaves the context poisoned, as a real expiry would."""
+        _check(lib().mpt_selftest_wait_timeout_ctx(self._ctx, 1000), self._ctx)
+
+    def last_error(self) -> str:
+        return lib().mpt_last_error(self._ctx).decode()
+
     def launch_count(self):
         n = C.c_longlong(0)
         _check(lib().mpt_launch_count(self._ctx, C.byref(n)), self._ctx)
@@ -408,16 +419,22 @@ def mpt_update_flat_opt(opt, g16, w32, s1, s2, w16, n, inv_S, b1t, b2t, detect, 
                                      _dptr(clip_scratch), _stream_ptr(stream)))
 
 
-def mpt_softmax_ce(z, ldz, labels, B, Cn, S, dz, lddz, row_loss, loss, bad_labels=None, stream=None):
+def mpt_softmax_ce(z, ldz, labels, B, Cn, S, dz, lddz, row_loss, loss, bad_labels=None, stream=None, status=None):
     _check(lib().mpt_softmax_ce(_dptr(z), ldz, _dptr(labels), B, Cn, float(S), _dptr(dz), lddz, _dptr(row_loss),
-                                _dptr(loss), _dptr(bad_labels), _stream_ptr(stream)))
+                                _dptr(loss), _dptr(bad_labels), _dptr(status), _stream_ptr(stream)))
 
 
-def mpt_softmax_ce_static(z, ldz, labels, B, Cn, S, dz, lddz, loss, bad_labels=None, stream=None):
+def mpt_softmax_ce_static(z, ldz, labels, B, Cn, S, dz, lddz, loss, bad_labels=None, stream=None, status=None):
     """mpt_softmax_ce for callers that cannot provide the float[B] scratch: the per-row losses
     live in a fixed array inside the library (B <= 65536; calls that overlap on the GPU race)."""
     _check(lib().mpt_softmax_ce_static(_dptr(z), ldz, _dptr(labels), B, Cn, float(S), _dptr(dz), lddz, _dptr(loss),
-                                       _dptr(bad_labels), _stream_ptr(stream)))
+                                       _dptr(bad_labels), _dptr(status), _stream_ptr(stream)))
+
+
+def mpt_selftest_wait_timeout(limit_us, status, stream=None) -> int:
+    """Makes one bounded device-side wait run out on purpose; returns the library's code
+    (MPT_ERR_TIMEOUT = -6 is the expected outcome) instead of raising."""
+    return int(lib().mpt_selftest_wait_timeout(int(limit_us), _dptr(status), _stream_ptr(stream)))
 
 
 def mpt_version() -> str:

@@ -1049,7 +1049,8 @@ int mpt_update_flat_opt(const mpt_optimizer *opt, const uint16_t *g16_dev, float
 }
 
 int mpt_softmax_ce(const uint16_t *z_dev, int ldz, const int32_t *labels_dev, int B, int C, float S, uint16_t *dz_dev,
-                   int lddz, float *row_loss_dev, float *loss_dev, uint32_t *bad_labels_dev, void *cuda_stream)
+                   int lddz, float *row_loss_dev, float *loss_dev, uint32_t *bad_labels_dev, uint32_t *status_dev,
+                   void *cuda_stream)
 {
     if (!z_dev || !labels_dev || !dz_dev || !row_loss_dev || !loss_dev) return MPT_ERR_INVALID_ARG;
     if (B < 0 || C < 0 || ldz < C || lddz < C) return MPT_ERR_SHAPE;
@@ -1058,8 +1059,32 @@ int mpt_softmax_ce(const uint16_t *z_dev, int ldz, const int32_t *labels_dev, in
     cudaError_t e = cudaSuccess;
     if (bad_labels_dev) e = cudaMemsetAsync(bad_labels_dev, 0, sizeof(uint32_t), st);
     if (e == cudaSuccess)
-        e = launch_softmax_ce(z_dev, ldz, labels_dev, B, C, S, dz_dev, lddz, row_loss_dev, loss_dev, bad_labels_dev, st, nullptr);
+        e = launch_softmax_ce(z_dev, ldz, labels_dev, B, C, S, dz_dev, lddz, row_loss_dev, loss_dev, bad_labels_dev, st, nullptr,
+                              nullptr, status_dev);
     return e == cudaSuccess ? MPT_OK : MPT_ERR_CUDA;
+}
+
+int mpt_selftest_wait_timeout(unsigned limit_us, uint32_t *status_dev, void *cuda_stream)
+{
+    if (!status_dev) return MPT_ERR_INVALID_ARG;
+    if (limit_us < 1 || limit_us > 2000000u) return MPT_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (launch_wait_selftest(limit_us, status_dev, st) != cudaSuccess) return MPT_ERR_CUDA;
+    uint32_t word = 0;
+    if (cudaMemcpyAsync(&word, status_dev, sizeof word, cudaMemcpyDeviceToHost, st) != cudaSuccess) return MPT_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return MPT_ERR_CUDA;
+    return word != 0 ? MPT_ERR_TIMEOUT : MPT_OK;
+}
+
+int mpt_selftest_wait_timeout_ctx(mpt_ctx *c, unsigned limit_us)
+{
+    int r = usable(c);
+    if (r != MPT_OK) return r;
+    if (limit_us < 1 || limit_us > 2000000u) return fail(c, MPT_ERR_INVALID_ARG, "limit outside [1, 2000000] microseconds");
+    CK(launch_wait_selftest(limit_us, c->status + ST_KERNEL_ERR, c->stream), "self-test launch");
+    c->launches++;
+    uint32_t st[ST_WORDS];
+    return read_status(c, st);       // MPT_ERR_TIMEOUT, and the context is poisoned from here on
 }
 
 }  // extern "C"

@@ -34,7 +34,8 @@ enum KernelErr : uint32_t {
     KERR_WAIT_EMPTY = 2,  // producer gave up waiting for a free stage
     KERR_WAIT_ACC = 3,    // epilogue gave up waiting for the accumulator
     KERR_WAIT_ACC_FREE = 4, // MMA issuer gave up waiting for a drained accumulator
-    KERR_TMEM_ALLOC = 5
+    KERR_TMEM_ALLOC = 5,
+    KERR_WAIT_SELFTEST = 6  // the self-test's wait on a barrier nobody signals ran out, as intended
 };
 
 // Kernel attributes (opt-in shared memory size, cluster occupancy) are per device: launchers
@@ -115,6 +116,9 @@ cudaError_t launch_update(const uint16_t *g16, float *w32, float *v, uint16_t *w
 cudaError_t launch_softmax_ce(const uint16_t *z, int ldz, const int32_t *labels, int B, int C, float S,
                               uint16_t *dz, int lddz, float *row_loss, float *loss, uint32_t *bad_labels,
                               cudaStream_t st, int *n_launches, const float *S_dev = nullptr, uint32_t *kerr = nullptr);
+// One CTA waits, for at most limit_us, on a barrier nothing arrives on; on expiry it records
+// KERR_WAIT_SELFTEST in *status (wait_selftest.cu).
+cudaError_t launch_wait_selftest(unsigned limit_us, uint32_t *status, cudaStream_t st);
 // Optimizer steps other than SGD(+momentum), and weight decay (see mpt.h MPT_OPT_*).  s1 / s2:
 // FP32 state arrays (momentum or squared-gradient sum; Adam's second moment).  For Adam the
 // bias corrections are 1 - beta^t with beta^t either passed by value (b1t, b2t: the products

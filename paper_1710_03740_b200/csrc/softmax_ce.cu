@@ -544,7 +544,7 @@ float *g_static_ptr[mpt::kMaxDevices];   // per device, filled on the first call
 
 extern "C" int mpt_softmax_ce_static(const uint16_t *z_dev, int ldz, const int32_t *labels_dev, int B, int C, float S,
                                      uint16_t *dz_dev, int lddz, float *loss_dev, uint32_t *bad_labels_dev,
-                                     void *cuda_stream)
+                                     uint32_t *status_dev, void *cuda_stream)
 {
     if (!z_dev || !labels_dev || !dz_dev || !loss_dev) return MPT_ERR_INVALID_ARG;
     if (B < 0 || C < 0 || ldz < C || lddz < C) return MPT_ERR_SHAPE;
@@ -553,18 +553,23 @@ extern "C" int mpt_softmax_ce_static(const uint16_t *z_dev, int ldz, const int32
     int device = -1;
     if (cudaGetDevice(&device) != cudaSuccess) return MPT_ERR_CUDA;
     if (device < 0 || device >= mpt::kMaxDevices) return MPT_ERR_INTERNAL;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    // The array's address belongs to the CURRENT device; a stream of another device would hand its
+    // kernels a pointer into the wrong GPU's copy of the array.
+    int stream_device = device;
+    if (cudaStreamGetDevice(st, &stream_device) != cudaSuccess) return MPT_ERR_CUDA;
+    if (stream_device != device) return MPT_ERR_INVALID_ARG;
     if (!g_static_ptr[device]) {
         float *p = nullptr;
         if (cudaGetSymbolAddress((void **)&p, g_static_row_loss) != cudaSuccess || !p) return MPT_ERR_CUDA;
         g_static_ptr[device] = p;
     }
-    cudaStream_t st = (cudaStream_t)cuda_stream;
     cudaError_t e = cudaSuccess;
     if (bad_labels_dev) e = cudaMemsetAsync(bad_labels_dev, 0, sizeof(uint32_t), st);
     // Nothing in the scratch has to start at zero: rows 0..B-1 are each written by the row
     // kernel before the mean kernel reads exactly those rows; older contents are never read.
     if (e == cudaSuccess)
         e = mpt::launch_softmax_ce(z_dev, ldz, labels_dev, B, C, S, dz_dev, lddz, g_static_ptr[device], loss_dev,
-                                   bad_labels_dev, st, nullptr);
+                                   bad_labels_dev, st, nullptr, nullptr, status_dev);
     return e == cudaSuccess ? MPT_OK : MPT_ERR_CUDA;
 }

@@ -52,8 +52,10 @@ __device__ __forceinline__ unsigned long long global_ns()
     return t;
 }
 
-// Bounded wait.  Returns false when the CTA is aborting or the time limit expired.
-static __device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag)
+// Bounded wait.  Returns false when the CTA is aborting or the time limit expired.  The limit is
+// an argument (default 2 s) so that a self-test can make a wait run out within a millisecond.
+static __device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag,
+                                              unsigned long long limit_ns = WAIT_LIMIT_NS)
 {
     unsigned long long t0 = 0;
     for (uint32_t it = 0;; ++it) {
@@ -62,7 +64,7 @@ static __device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, vol
             if (*abort_flag) return false;
             unsigned long long now = global_ns();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > WAIT_LIMIT_NS) return false;
+            else if (now - t0 > limit_ns) return false;
         }
     }
 }

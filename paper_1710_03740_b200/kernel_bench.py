@@ -6,16 +6,16 @@ sweep, the bigLSTM-shaped products, the master-update pass and the softmax cross
     python -m paper_1710_03740_b200.kernel_bench softmax [--rows B] [--classes C] [--iters 20]
     python -m paper_1710_03740_b200.kernel_bench step    [--workload tiny|scale_sweep|large_twin] [--iters 50]
 
+    python -m paper_1710_03740_b200.kernel_bench lstm    [--config biglstm] [--iters 20]
+    python -m paper_1710_03740_b200.kernel_bench dp      [--params N] [--replicas R]
+
 Prints one JSON line per case: best-of and back-to-back ("sustained") rates.  Working sets
 are larger than the 126 MB L2 unless the shape itself is smaller; small cases say so.
-`--compare-library` adds torch.matmul (cuBLAS) on the same operands as context.
 """
 from __future__ import annotations
 
 import argparse
 import json
-import subprocess
-import time
 
 import torch
 
@@ -23,46 +23,6 @@ from . import binding as mpt
 from . import inputs
 
 OPS = {0: "fwd", 1: "dgrad", 2: "wgrad"}
-
-
-def _sustained(fn, seconds):
-    """Rate over a loop of at least `seconds` of back-to-back launches, with the SM clock and power
-    sampled by nvidia-smi every 100 ms meanwhile (the GPU settles under its power cap)."""
-    q = "clocks.sm,power.draw,clocks_event_reasons.sw_power_cap,clocks_event_reasons.hw_slowdown,clocks_event_reasons.sw_thermal_slowdown"
-    try:
-        smi = subprocess.Popen(["nvidia-smi", "-i", str(torch.cuda.current_device()), "--query-gpu=" + q,
-                                "--format=csv,noheader,nounits", "-lms", "100"], stdout=subprocess.PIPE, text=True)
-    except OSError:
-        smi = None
-    for _ in range(3):
-        fn()
-    torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    n, t0 = 0, time.time()
-    e0.record()
-    while time.time() - t0 < seconds:
-        for _ in range(50):
-            fn()
-        n += 50
-        torch.cuda.synchronize()
-    e1.record()
-    torch.cuda.synchronize()
-    ms = e0.elapsed_time(e1) / n
-    clocks, power, reasons = [], [], set()
-    if smi is not None:
-        smi.terminate()
-        for line in smi.stdout.read().strip().splitlines()[3:]:
-            f = [x.strip() for x in line.split(",")]
-            try:
-                clocks.append(float(f[0])); power.append(float(f[1]))
-            except (ValueError, IndexError):
-                continue
-            for name, v in zip(("sw_power_cap", "hw_slowdown", "sw_thermal_slowdown"), f[2:5]):
-                if v.lower().startswith("active"):
-                    reasons.add(name)
-    clocks.sort(); power.sort()
-    return ms, {"sm_mhz_median": clocks[len(clocks) // 2] if clocks else None,
-                "power_w_median": power[len(power) // 2] if power else None, "reasons": sorted(reasons)}
 
 
 def _time_graph(fn, iters):
@@ -114,7 +74,7 @@ def _time(fn, iters, warmup=5):
 _time.last_median = None
 
 
-def bench_gemm(M, N, K, op, iters, compare=False, flags=mpt.GEMM_FORCE_TC, use_workspace=True, sustain_s=0.0):
+def bench_gemm(M, N, K, op, iters, flags=mpt.GEMM_FORCE_TC, use_workspace=True):
     sa = (K, M) if op == 2 else (M, K)
     sb = (N, K) if op == 0 else (K, N)
     g = torch.Generator(device="cuda").manual_seed(2)
@@ -136,30 +96,10 @@ def bench_gemm(M, N, K, op, iters, compare=False, flags=mpt.GEMM_FORCE_TC, use_w
            "sustained_ms": sus,
            "best_tflops": fl / best / 1e9, "sustained_tflops": fl / sus / 1e9, "device_error": int(st[0]), "splitk_workspace_mb": nws / 1e6,
            "working_set_mb": (A.numel() + B.numel() + C.numel()) * 2 / 1e6}
-    if sustain_s > 0:
-        ms, clk = _sustained(fn, sustain_s)
-        out["sustained_%gs_tflops" % sustain_s] = fl / ms / 1e9
-        out["sustained_clocks"] = clk
-    if compare:
-        if op == 0:
-            ref = lambda: torch.matmul(A, B.t())  # noqa: E731
-        elif op == 1:
-            ref = lambda: torch.matmul(A, B)  # noqa: E731
-        else:
-            ref = lambda: torch.matmul(A.t(), B)  # noqa: E731
-        rb, rs = _time(ref, iters)
-        if rs < 0.2:
-            rs = min(rs, _time_graph(ref, iters))
-        out["library_best_tflops"] = fl / rb / 1e9
-        out["library_sustained_tflops"] = fl / rs / 1e9
-        if sustain_s > 0:
-            ms, clk = _sustained(ref, sustain_s)
-            out["library_sustained_%gs_tflops" % sustain_s] = fl / ms / 1e9
-            out["library_sustained_clocks"] = clk
     return out
 
 
-def bench_update(n, momentum, iters, sustain_s=0.0):
+def bench_update(n, momentum, iters):
     g = torch.Generator(device="cuda").manual_seed(3)
     g16 = (torch.randn(n, device="cuda", generator=g) * 37).half()
     w32 = torch.randn(n, device="cuda", generator=g)
@@ -175,10 +115,6 @@ def bench_update(n, momentum, iters, sustain_s=0.0):
            "working_set_mb": bpp * n / 1e6, "flags": flags.tolist()}
     if bpp * n < 256e6:
         out["note"] = "working set below 256 MB: L2-resident, not an HBM claim"
-    if sustain_s > 0:
-        ms, clk = _sustained(fn, sustain_s)
-        out["sustained_%gs_gbs" % sustain_s] = bpp * n / ms / 1e6
-        out["sustained_clocks"] = clk
     return out
 
 
@@ -272,69 +208,7 @@ def bench_lstm(name, iters, steps=None):
     return out
 
 
-def bench_steplike(steps, dense):
-    """The 26 products and the master update of the large-MLP step as stateless calls, alternating
-    like the training step, with this library's kernels and with torch.matmul (cuBLAS) on the same
-    operands: ReLU-like operands (half zeros) unless `dense`.  Context for the power-capped regime:
-    what a product leaves behind (clock state) shows in the update that follows it."""
-    B_, H, Cn = 4096, 12288, 32000
-    g = torch.Generator(device="cuda").manual_seed(5)
-    rnd = lambda *shape: torch.randn(shape, device="cuda", generator=g)  # noqa: E731
-    act = (lambda t: t) if dense else torch.relu
-    x = [act(rnd(B_, H)).half() for _ in range(9)]
-    W = [(rnd(H, H) * 0.01).half() for _ in range(8)] + [(rnd(Cn, H) * 0.01).half()]
-    keep = (lambda t: t) if dense else (lambda t: t * (torch.rand(t.shape, device="cuda", generator=g) > 0.5))
-    dz = [keep(rnd(B_, H)).half() for _ in range(8)] + [(rnd(B_, Cn) * 1e-3).half()]
-    n = sum(w.numel() for w in W)
-    g16 = rnd(n).half(); w32 = rnd(n); v = torch.zeros(n, device="cuda"); w16 = torch.empty(n, dtype=torch.half, device="cuda")
-    flags = torch.zeros(2, dtype=torch.int32, device="cuda")
-    st = torch.zeros(16, dtype=torch.int32, device="cuda")
-    ws = torch.zeros(20 * 1024 * 1024 // 4, device="cuda")
-    outs = {}
-
-    def out(kind, l, rows, cols):
-        return outs.setdefault((kind, l), torch.empty((rows, cols), dtype=torch.half, device="cuda"))
-
-    def ours():
-        for l in range(9):
-            N = W[l].shape[0]
-            mpt.mpt_gemm_f16_ws(0, B_, N, H, x[l], H, W[l], H, out("f", l, B_, N), N, 0, None, 0, None, st, ws)
-        for l in range(8, -1, -1):
-            N = W[l].shape[0]
-            mpt.mpt_gemm_f16_ws(2, N, H, B_, dz[l], N, x[l], H, out("w", l, N, H), H, 0, None, 0, None, st, ws)
-            if l > 0:
-                mpt.mpt_gemm_f16_ws(1, B_, H, N, dz[l], N, W[l], H, out("d", l, B_, H), H, 0, None, 0, None, st, ws)
-
-    def library():
-        for l in range(9):
-            torch.matmul(x[l], W[l].t())
-        for l in range(8, -1, -1):
-            torch.matmul(dz[l].t(), x[l])
-            if l > 0:
-                torch.matmul(dz[l], W[l])
-
-    upd = lambda: mpt.mpt_update_flat(g16, w32, v, w16, n, 1.0 / 512, 1e-4, 0.9, True, False, flags)  # noqa: E731
-
-    def run(products):
-        tg = tu = 0.0
-        for s_ in range(steps + 3):
-            e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
-            e[0].record(); products(); e[1].record(); upd(); e[2].record()
-            torch.cuda.synchronize()
-            if s_ >= 3:
-                tg += e[0].elapsed_time(e[1]); tu += e[1].elapsed_time(e[2])
-        return tg / steps, tu / steps
-
-    res = {"kernel": "steplike", "operands": "dense" if dense else "relu-like (half zeros)", "steps": steps, "rounds": []}
-    for _ in range(2):
-        a, b = run(ours), run(library)
-        res["rounds"].append({"ours_products_ms": a[0], "ours_update_ms": a[1], "library_products_ms": b[0],
-                              "update_after_library_ms": b[1]})
-    res["device_error"] = int(st[0])
-    return res
-
-
-def bench_softmax(B, Cn, iters, sustain_s=0.0):
+def bench_softmax(B, Cn, iters):
     g = torch.Generator(device="cuda").manual_seed(4)
     z = (torch.randn((B, Cn), device="cuda", generator=g) * 3).half()
     y = torch.randint(0, Cn, (B,), device="cuda", generator=g, dtype=torch.int32)
@@ -348,10 +222,6 @@ def bench_softmax(B, Cn, iters, sustain_s=0.0):
            "sustained_ms": sus, "best_gbs": by / best / 1e6, "sustained_gbs": by / sus / 1e6, "loss": float(loss.item())}
     if by < 256e6:
         out["note"] = "working set below 256 MB: L2-resident, not an HBM claim"
-    if sustain_s > 0:
-        ms, clk = _sustained(fn, sustain_s)
-        out["sustained_%gs_gbs" % sustain_s] = by / ms / 1e6
-        out["sustained_clocks"] = clk
     return out
 
 
@@ -406,10 +276,7 @@ def main():
     g.add_argument("--shape", nargs="*", default=None, help="MxNxK; default: the sweep and the bigLSTM shapes")
     g.add_argument("--op", nargs="*", type=int, default=[0, 1, 2])
     g.add_argument("--iters", type=int, default=20)
-    g.add_argument("--compare-library", action="store_true")
     g.add_argument("--no-workspace", action="store_true", help="do not offer a split-K scratch buffer")
-    g.add_argument("--sustain", type=float, default=0.0, metavar="SECONDS",
-                   help="also time a loop of at least this many seconds with clocks and power sampled")
     g.add_argument("--kernel", default="auto", choices=["auto", "tc", "pair", "pair512"],
                    help="auto: the library's choice; tc: single-CTA 128x256 tiles; pair: cta_group::2 256x256 tiles")
     u = sub.add_parser("update")
@@ -418,16 +285,11 @@ def main():
     u.add_argument("--optimizer", default="sgd", choices=["sgd", "nesterov", "adagrad", "adam"])
     u.add_argument("--weight-decay", type=float, default=0.0)
     u.add_argument("--clip-norm", type=float, default=0.0)
-    u.add_argument("--sustain", type=float, default=0.0, help="also time SECONDS of back-to-back launches with clocks sampled")
     u.add_argument("--iters", type=int, default=20)
     s = sub.add_parser("softmax")
     s.add_argument("--rows", type=int, default=4096)
     s.add_argument("--classes", type=int, default=32000)
     s.add_argument("--iters", type=int, default=20)
-    s.add_argument("--sustain", type=float, default=0.0)
-    sl = sub.add_parser("steplike")
-    sl.add_argument("--steps", type=int, default=10)
-    sl.add_argument("--dense", action="store_true", help="dense normal operands instead of ReLU-like ones")
     ls = sub.add_parser("lstm")
     ls.add_argument("--config", default="biglstm", choices=sorted(inputs.LSTM_CONFIGS))
     ls.add_argument("--steps", type=int, default=0, help="override the number of time steps")
@@ -449,23 +311,21 @@ def main():
         for (M, N, K) in shapes:
             for op in args.op:
                 flags = {"auto": 0, "tc": mpt.GEMM_FORCE_TC, "pair": mpt.GEMM_FORCE_PAIR, "pair512": mpt.GEMM_FORCE_PAIR512}[args.kernel]
-                res = bench_gemm(M, N, K, op, args.iters, args.compare_library, flags, not args.no_workspace, args.sustain)
+                res = bench_gemm(M, N, K, op, args.iters, flags, not args.no_workspace)
                 res["kernel_choice"] = args.kernel
                 print(json.dumps(res), flush=True)
     elif args.cmd == "dp":
         print(json.dumps(bench_dp(args.params, args.replicas, args.momentum, args.iters)), flush=True)
-    elif args.cmd == "steplike":
-        print(json.dumps(bench_steplike(args.steps, args.dense)), flush=True)
     elif args.cmd == "lstm":
         print(json.dumps(bench_lstm(args.config, args.iters, args.steps)), flush=True)
     elif args.cmd == "update":
         kind = ["sgd", "nesterov", "adagrad", "adam"].index(args.optimizer)
         if kind == 0 and args.weight_decay == 0.0 and args.clip_norm == 0.0:
-            print(json.dumps(bench_update(args.params, args.momentum, args.iters, args.sustain)), flush=True)
+            print(json.dumps(bench_update(args.params, args.momentum, args.iters)), flush=True)
         else:
             print(json.dumps(bench_update_opt(args.params, kind, args.weight_decay, args.iters, args.clip_norm)), flush=True)
     else:
-        print(json.dumps(bench_softmax(args.rows, args.classes, args.iters, args.sustain)), flush=True)
+        print(json.dumps(bench_softmax(args.rows, args.classes, args.iters)), flush=True)
 
 
 if __name__ == "__main__":

@@ -109,14 +109,14 @@ def _check_tc(op, M, N, K, flags=0, mask=None, seed=21, scale=None, want_flag=Fa
             _ORACLE_CACHE[key] = (A, B, ref, ex, ab)
     got, flag = run_gemm(op, A, B, M, N, K, flags=flags | force, mask=mask,
                          pad=(8 if (M * N) % 3 == 0 else 0), want_flag=want_flag, workspace=workspace)
-    ok, stats = gemm_accept(got, ref, K=K, absdot=ab)
+    ok, stats = gemm_accept(got, ref, K=K, absdot=ab, exact=ex)
     assert ok.all(), (op, M, N, K, stats, np.argwhere(~ok)[:8].tolist())
     assert stats["by_abs_only"] <= max(2, stats["n"] // 1000), stats
     # both sides within the summation bound of the exactly rounded sum
     if not flags and mask is None:
         with np.errstate(over="ignore"):      # sums beyond the FP16 range become inf, as intended
             exact16 = ex.astype(np.float32).astype(np.float16).view(np.uint16)
-        ok2, st2 = gemm_accept(got, exact16, K=K, absdot=ab)
+        ok2, st2 = gemm_accept(got, exact16, K=K, absdot=ab, exact=ex)
         assert ok2.all(), st2
     return got, ref, flag, stats
 
@@ -140,6 +140,24 @@ def test_tc_gemm_parity(op, M, N, K):
 @pytest.mark.parametrize("M,N,K", PAIR_SHAPES)
 def test_pair_gemm_parity(op, M, N, K):
     _check_tc(op, M, N, K, kernel="pair")
+
+
+@pytest.mark.parametrize("op", [0, 1, 2])
+def test_sweep_2048_cubed_in_full_every_kernel(op):
+    """2048^3 of the isolated-GEMM sweep (seed and operand distribution of that sweep), every
+    output element against the oracle: under the library's own kernel choice with and without a
+    scratch buffer, and with each tensor-core kernel forced.  This is the size at which the
+    automatic choice passes from the single-CTA kernel to the CTA pair."""
+    from paper_1710_03740_b200 import binding as b
+    M = N = K = 2048
+    assert (M, N, K) in inputs.GEMM_SWEEP
+    auto, _, _, _ = _check_tc(op, M, N, K, seed=2, kernel="auto")
+    again, _, _, _ = _check_tc(op, M, N, K, seed=2, kernel="auto")
+    assert np.array_equal(auto, again)
+    for kernel in ("tc", "pair", "pair512"):
+        _check_tc(op, M, N, K, seed=2, kernel=kernel)
+    if b.mpt_gemm_workspace_bytes(op, M, N, K):
+        _check_tc(op, M, N, K, seed=2, kernel="auto", workspace=True)
 
 
 PAIR512_SHAPES = [(256, 512, 64), (256, 512, 448), (512, 1536, 128), (256, 768, 72), (392, 1080, 136), (264, 264, 200),

@@ -561,6 +561,20 @@ def test_global_norm_clipping_closed_forms():
         assert float(net.w32[0][0, 0]) == float(f(1.0) - f(0.5) * (f(3.0) * coef))
         assert float(net.w32[0][0, 1]) == 2.0
         assert float(net.w32[1][0, 0]) == float(f(3.0) - f(0.5) * (f(4.0) * coef))
+    # a bound that binary32 cannot hold (0.3): the optimizer's parameter is a binary32 number, so the
+    # quotient is formed from float32(0.3); with the 3-4-5 gradient the two readings give different
+    # binary32 coefficients (0x3D75C28D from the rounded bound, one code lower from the double 0.3)
+    net = OracleMLP([(2, 1, 0)], 1.0, 0.5, 0.0)
+    net.set_master(0, np.zeros((1, 2), dtype=np.float32))
+    net.set_optimizer(0, 0.5, clip=0.3)
+    net.set_grad(0, np.array([[3.0, 4.0]], dtype=np.float16))
+    net.step()
+    want = f(float(f(0.3)) / (5.0 + 1e-6))
+    other = f(0.3 / (5.0 + 1e-6))
+    assert want.view(np.uint32) == 0x3D75C28D and other.view(np.uint32) == 0x3D75C28C
+    assert np.float32(net.last_coef).view(np.uint32) == 0x3D75C28D
+    assert np.float32(mpo.clip_coef(25.0, 0.3)).view(np.uint32) == 0x3D75C28D
+    assert float(net.w32[0][0, 0]) == float(f(0.0) - f(0.5) * (f(3.0) * want))
     # a norm under the bound leaves the gradient alone (coefficient exactly 1)
     net = OracleMLP([(2, 1, 0)], 1.0, 0.5, 0.0)
     net.set_master(0, np.zeros((1, 2), dtype=np.float32))

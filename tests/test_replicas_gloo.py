@@ -70,3 +70,27 @@ def test_step_flops_counts_every_gemm_of_an_iteration():
     big = inputs.MLP_CONFIGS["large"]
     assert abs(bench.step_flops(big) - 3.8113539784704e13) < 1e6
     assert bench.n_params(big) == 8 * 12288 * 12288 + 12288 * 32000
+
+
+def test_bench_gpus_2_starts_its_own_two_ranks():
+    """`python bench.py --gpus 2` run plainly starts two ranks by itself (torch.distributed.run on
+    127.0.0.1) and reports n_gpus = 2; here with the CPU-only rank check (gloo) in place of the
+    GPU step."""
+    import json
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_ADDR", "MASTER_PORT")}
+    p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--rank-check"], env=env,
+                       stdout=subprocess.PIPE, stderr=subprocess.PIPE, text=True, timeout=300)
+    assert p.returncode == 0, p.stderr[-2000:]
+    lines = [ln for ln in p.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1, p.stdout
+    out = json.loads(lines[0])
+    assert out["n_gpus"] == 2 and out["gpus_arg"] == 2
+    assert out["ms_per_step"] == 11.0                       # maximum over the ranks' 10 and 11 ms
+    assert abs(out["value"] - 2e12 / 11e-3 / 1e12) < 1e-9   # both ranks' work over that time
+
+
+def test_bench_refuses_a_world_size_that_contradicts_gpus():
+    env = dict(os.environ, RANK="0", LOCAL_RANK="0", WORLD_SIZE="1", MASTER_ADDR="127.0.0.1", MASTER_PORT="29999")
+    p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--rank-check"], env=env,
+                       stdout=subprocess.PIPE, stderr=subprocess.PIPE, text=True, timeout=120)
+    assert p.returncode != 0 and "WORLD_SIZE" in p.stderr
