@@ -432,6 +432,60 @@ int mpt_bias_grad(const uint16_t *dG, size_t rows, int cols, int ld, float *part
 int mpt_add_f16(const uint16_t *a, int lda, const uint16_t *b, int ldb, uint16_t *out, int ldo, int rows, int cols,
                 void *cuda_stream);
 
+/* ------------------------------------------------------------ the LSTM layer, trained
+ *
+ * The layer above with everything section 3 asks of a trained layer: FP32 master copies of Wg,
+ * Wp and the bias with FP16 working copies re-rounded after every applied step (section 3.1), a
+ * loss multiplied by S before back-propagation, weight gradients unscaled and inspected for
+ * inf/NaN with the step skipped on overflow (section 3.2; the paper's language model, section
+ * 4.5, is its loss-scaling showcase: S = 128, Adagrad), optionally the dynamic scale schedule of
+ * mpt_set_dynamic_scale.  One call runs one iteration on a batch of T*B rows:
+ *   1. x_t into the step rows, r_{-1} = 0, c_{-1} = 0, then mpt_lstm_forward
+ *   2. softmax cross-entropy over the projected outputs r_t taken as logits over P classes, one
+ *      label per (t, b) row, mean over all T*B rows; dr_ext = rn16((p - onehot) * S / (T*B))
+ *      (the arithmetic of mpt_softmax_ce)
+ *   3. mpt_lstm_backward; the overflow word is OR-ed by the epilogues of dWg, dWp and dbias
+ *   4. the optimizer step of mpt_update_flat_opt over the flat arena [Wg | Wp | bias] (one launch;
+ *      every mpt_optimizer kind, weight decay, global-norm clipping), then the scale schedule
+ * The workspace (mpt_lstm_workspace_bytes, 256-byte aligned, caller-owned) holds all parameters,
+ * optimizer state, activations and gradients; nothing is allocated.  Asynchronous on the stream
+ * unless loss_host / overflow_host is non-null (then the stream is synchronised and the unscaled
+ * mean loss / the 0-1 skip flag of this iteration are written).  Error codes and the poisoned
+ * state after MPT_ERR_CUDA / MPT_ERR_TIMEOUT are those of mpt_ctx; labels outside [0, P) contribute
+ * nothing and are reported as MPT_ERR_INVALID_ARG by a synchronising call, after the step ran.
+ * mpt_lstm_get_tensor kinds: masters (FP32), working copies, gradients of the last iteration
+ * (FP16, scaled by S), first optimizer state (FP32), the step rows xr [T+1, B, I+P] whose right
+ * columns hold r_t, and dr_ext [T, B, P]; the byte count must match exactly. */
+typedef struct mpt_lstm_ctx mpt_lstm_ctx;
+#define MPT_LSTM_T_WG32 0
+#define MPT_LSTM_T_WP32 1
+#define MPT_LSTM_T_BIAS32 2
+#define MPT_LSTM_T_WG16 3
+#define MPT_LSTM_T_WP16 4
+#define MPT_LSTM_T_BIAS16 5
+#define MPT_LSTM_T_DWG16 6
+#define MPT_LSTM_T_DWP16 7
+#define MPT_LSTM_T_DBIAS16 8
+#define MPT_LSTM_T_S1_WG32 9
+#define MPT_LSTM_T_S1_WP32 10
+#define MPT_LSTM_T_S1_BIAS32 11
+#define MPT_LSTM_T_XR16 12
+#define MPT_LSTM_T_DREXT16 13
+int mpt_lstm_workspace_bytes(const mpt_lstm_desc *desc, const mpt_optimizer *opt, size_t *bytes_out);
+int mpt_lstm_create(const mpt_lstm_desc *desc, float S, const mpt_optimizer *opt, void *workspace_dev,
+                    size_t workspace_bytes, void *cuda_stream, mpt_lstm_ctx **out);
+/* Masters from HOST arrays Wg [4H, I+P] (gate-interleaved rows), bias [4H], Wp [P, H]; rounds the
+ * working copies and zeroes the optimizer state.  Synchronous. */
+int mpt_lstm_set_params(mpt_lstm_ctx *ctx, const float *Wg_host, const float *bias_host, const float *Wp_host);
+/* x_dev: FP16 [T, B, I] dense; labels_dev: int32 [T*B], row t*B + b. */
+int mpt_lstm_train_step(mpt_lstm_ctx *ctx, const uint16_t *x_dev, const int32_t *labels_dev, float *loss_host,
+                        int *overflow_host);
+int mpt_lstm_get_tensor(mpt_lstm_ctx *ctx, int kind, void *dst_host, size_t bytes);
+int mpt_lstm_set_dynamic_scale(mpt_lstm_ctx *ctx, int enable, int growth_interval, float min_scale, float max_scale);
+int mpt_lstm_get_scale(mpt_lstm_ctx *ctx, float *S_out);
+const char *mpt_lstm_last_error(mpt_lstm_ctx *ctx);
+void mpt_lstm_destroy(mpt_lstm_ctx *ctx);
+
 /* Softmax cross-entropy forward and scaled backward (sections 3.2, 3.3), arithmetic
  * as in mpt_backward_scaled.  z_dev/dz_dev: FP16 [B, C] with pitches ldz/lddz
  * (the two must not overlap).  row_loss_dev: float [B] scratch; loss_dev: one float,
@@ -580,6 +634,13 @@ int mpt_dp_free(void *dev_ptr);
 int mpt_dp_export(const void *dev_ptr, uint8_t *handle_out);
 int mpt_dp_open(const uint8_t *handle, void **dev_ptr_out);
 int mpt_dp_close(void *dev_ptr);
+
+/* Measurement aid (no counterpart in the paper): a one-warp kernel that measures the clock its SM
+ * runs at, in MHz, by counting SM cycles over window_us (1 .. 100000) microseconds of the global
+ * timer, and writes it to *mhz_dev (one float).  Asynchronous on the stream.  Enqueued before and
+ * after a kernel it shows the clock that kernel ran at, which under a power cap changes from one
+ * kernel of a training step to the next, far below the sampling period of nvidia-smi. */
+int mpt_sm_clock_probe(unsigned window_us, float *mhz_dev, void *cuda_stream);
 
 /* Library build identification, e.g. "mpt 0.1 sm_100a". */
 const char *mpt_version(void);

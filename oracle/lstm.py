@@ -69,3 +69,99 @@ class OracleLSTM:
         self.dWp = mpo.gemm_f16(mpo.OP_WGRAD, self.drtot.reshape(T * B, P), self.h.reshape(T * B, H))
         self.db16, self.db32 = mpo.bias_grad(self.dG.reshape(T * B, 4 * H))
         return self.dxr[:, :, :I]
+
+
+class OracleLSTMTrainer:
+    """The LSTM layer trained in the mixed-precision recipe (sections 3.1, 3.2; the paper's
+    language model, section 4.5, uses S = 128 and Adagrad): FP32 masters of Wg, Wp and the bias,
+    FP16 working copies, and per iteration
+
+      forward from zero state -> softmax cross-entropy over r_t as logits (mean over all T*B rows,
+      logit gradient times S) -> backward through time -> inspect the unscaled weight and bias
+      gradients for inf/NaN -> skip, or the optimizer step on the masters and re-round the copies
+      -> optional dynamic scale (same schedule as OracleMLP).
+
+    Readings where the paper is silent: the layer's projected output is used directly as the
+    logits of the loss; recurrent input and cell state start at zero every iteration; the three
+    parameter tensors share one optimizer (one clipping norm over all of them)."""
+
+    def __init__(self, T, B, I, H, P, S, kind, lr, mu=0.0, b2=0.0, eps=0.0, wd=0.0, clip=0.0):
+        self.net = OracleLSTM(T, B, I, H, P)
+        self.T, self.B, self.I, self.H, self.P = T, B, I, H, P
+        self.S = np.float32(S)
+        self.kind, self.lr, self.mu = int(kind), np.float32(lr), np.float32(mu)
+        self.b2, self.eps, self.wd, self.clip = np.float32(b2), np.float32(eps), np.float32(wd), float(clip)
+        self.b1t, self.b2t = np.float32(1.0), np.float32(1.0)
+        self.dynamic = None
+        self.clean_steps = 0
+        self.last_coef = np.float32(1.0)
+        self.names = ("Wg", "Wp", "bias")
+
+    def set_params(self, Wg, bias, Wp):
+        K = self.I + self.P
+        self.w32 = dict(Wg=np.array(Wg, dtype=np.float32).reshape(4 * self.H, K).copy(),
+                        Wp=np.array(Wp, dtype=np.float32).reshape(self.P, self.H).copy(),
+                        bias=np.array(bias, dtype=np.float32).reshape(4 * self.H).copy())
+        self.w16 = {k: mpo.f2h(v) for k, v in self.w32.items()}
+        self.s1 = {k: np.zeros_like(v) for k, v in self.w32.items()}
+        self.s2 = {k: np.zeros_like(v) for k, v in self.w32.items()}
+        self.g16 = {k: np.zeros(v.shape, dtype=np.uint16) for k, v in self.w32.items()}
+
+    def set_dynamic_scale(self, growth_interval, min_scale, max_scale, backoff=0.5, growth=2.0):
+        self.dynamic = (int(growth_interval), np.float32(backoff), np.float32(growth), np.float32(min_scale),
+                        np.float32(max_scale))
+        self.clean_steps = 0
+        self.S = np.float32(min(max(self.S, np.float32(min_scale)), np.float32(max_scale)))
+
+    def forward_backward(self, x16, labels):
+        T, B, P, H = self.T, self.B, self.P, self.H
+        r = self.net.forward(x16, np.zeros((B, P), dtype=np.uint16), np.zeros((B, H), dtype=np.uint16),
+                             self.w16["Wg"], self.w16["bias"], self.w16["Wp"])
+        self.logits = np.ascontiguousarray(r).reshape(T * B, P)
+        dz, _, loss, bad = mpo.softmax_ce(self.logits, labels, self.S)
+        self.dr_ext = dz.reshape(T, B, P)
+        self.net.backward(self.dr_ext)
+        self.g16 = dict(Wg=self.net.dWg, Wp=self.net.dWp, bias=self.net.db16)
+        self.loss = loss
+        return loss
+
+    def step(self):
+        inv = np.float32(1.0) / self.S
+        overflow = 0
+        for k in self.names:
+            overflow |= mpo.grad_nonfinite(self.g16[k], inv)
+        if not overflow:
+            if self.clip > 0.0:
+                total = sum(mpo.grad_sqnorm(self.g16[k], inv) for k in self.names)
+                self.last_coef = mpo.clip_coef(total, self.clip)
+            if self.kind == mpo.OPT_ADAM:
+                self.b1t = np.float32(self.b1t * self.mu)
+                self.b2t = np.float32(self.b2t * self.b2)
+            bc1, bc2 = np.float32(1.0) - self.b1t, np.float32(1.0) - self.b2t
+            for k in self.names:
+                g = np.ascontiguousarray(self.g16[k]).reshape(-1)
+                w, h = self.w32[k].reshape(-1), self.w16[k].reshape(-1)
+                use_s1 = self.kind != mpo.OPT_SGD or float(self.mu) != 0.0
+                s1 = self.s1[k].reshape(-1) if use_s1 else None
+                s2 = self.s2[k].reshape(-1) if self.kind == mpo.OPT_ADAM else None
+                if self.clip > 0.0:
+                    mpo.update_apply_clip(self.kind, g, w, s1, s2, h, inv, self.last_coef, self.lr, self.mu, self.b2,
+                                          self.eps, self.wd, bc1, bc2)
+                else:
+                    mpo.update_apply_opt(self.kind, g, w, s1, s2, h, inv, self.lr, self.mu, self.b2, self.eps, self.wd,
+                                         bc1, bc2)
+        if self.dynamic is not None:
+            interval, backoff, growth, smin, smax = self.dynamic
+            if overflow:
+                self.S = np.float32(max(np.float32(self.S * backoff), smin))
+                self.clean_steps = 0
+            else:
+                self.clean_steps += 1
+                if self.clean_steps >= interval:
+                    self.S = np.float32(min(np.float32(self.S * growth), smax))
+                    self.clean_steps = 0
+        return 1 if overflow else 0
+
+    def train_step(self, x16, labels):
+        loss = self.forward_backward(x16, labels)
+        return loss, self.step()

@@ -32,7 +32,9 @@ EXPORTS = ["mpt_workspace_bytes", "mpt_create", "mpt_workspace_bytes_opt", "mpt_
            "mpt_profile_read", "mpt_last_error",
            "mpt_destroy", "mpt_gemm_f16", "mpt_gemm_f16_ws", "mpt_gemm_workspace_bytes", "mpt_recast", "mpt_grad_nonfinite", "mpt_update_flat",
            "mpt_softmax_ce", "mpt_softmax_ce_static", "mpt_version",
-           "mpt_selftest_wait_timeout", "mpt_selftest_wait_timeout_ctx",
+           "mpt_selftest_wait_timeout", "mpt_selftest_wait_timeout_ctx", "mpt_sm_clock_probe",
+           "mpt_lstm_workspace_bytes", "mpt_lstm_create", "mpt_lstm_set_params", "mpt_lstm_train_step", "mpt_lstm_get_tensor",
+           "mpt_lstm_set_dynamic_scale", "mpt_lstm_get_scale", "mpt_lstm_last_error", "mpt_lstm_destroy",
            "mpt_lstm_forward", "mpt_lstm_backward", "mpt_lstm_cell_forward", "mpt_lstm_cell_backward", "mpt_bias_grad",
            "mpt_add_f16",
            "mpt_dp_shard", "mpt_dp_step_flat", "mpt_dp_alloc", "mpt_dp_free", "mpt_dp_export", "mpt_dp_open", "mpt_dp_close",
@@ -124,6 +126,18 @@ def lib() -> C.CDLL:
     L.mpt_update_flat.argtypes = [vp, vp, vp, vp, sz, f32, f32, f32, i32, i32, vp, vp]
     L.mpt_softmax_ce.argtypes = [vp, i32, vp, i32, i32, f32, vp, i32, vp, vp, vp, vp, vp]
     L.mpt_softmax_ce_static.argtypes = [vp, i32, vp, i32, i32, f32, vp, i32, vp, vp, vp, vp]
+    L.mpt_sm_clock_probe.argtypes = [u32, vp, vp]
+    L.mpt_lstm_workspace_bytes.argtypes = [C.POINTER(LstmDesc), C.POINTER(Optimizer), C.POINTER(sz)]
+    L.mpt_lstm_create.argtypes = [C.POINTER(LstmDesc), f32, C.POINTER(Optimizer), vp, sz, vp, C.POINTER(vp)]
+    L.mpt_lstm_set_params.argtypes = [vp, vp, vp, vp]
+    L.mpt_lstm_train_step.argtypes = [vp, vp, vp, C.POINTER(f32), C.POINTER(i32)]
+    L.mpt_lstm_get_tensor.argtypes = [vp, i32, vp, sz]
+    L.mpt_lstm_set_dynamic_scale.argtypes = [vp, i32, i32, f32, f32]
+    L.mpt_lstm_get_scale.argtypes = [vp, C.POINTER(f32)]
+    L.mpt_lstm_last_error.argtypes = [vp]
+    L.mpt_lstm_last_error.restype = C.c_char_p
+    L.mpt_lstm_destroy.argtypes = [vp]
+    L.mpt_lstm_destroy.restype = None
     L.mpt_selftest_wait_timeout.argtypes = [u32, vp, vp]
     L.mpt_selftest_wait_timeout_ctx.argtypes = [vp, u32]
     L.mpt_lstm_forward.argtypes = [C.POINTER(LstmDesc), C.POINTER(LstmTensors), vp]
@@ -431,6 +445,11 @@ def mpt_softmax_ce_static(z, ldz, labels, B, Cn, S, dz, lddz, loss, bad_labels=N
                                        _dptr(bad_labels), _dptr(status), _stream_ptr(stream)))
 
 
+def mpt_sm_clock_probe(window_us, mhz, stream=None):
+    """Enqueues the one-warp clock probe: mhz (a float32 CUDA tensor element) receives the SM clock in MHz."""
+    _check(lib().mpt_sm_clock_probe(int(window_us), _dptr(mhz), _stream_ptr(stream)))
+
+
 def mpt_selftest_wait_timeout(limit_us, status, stream=None) -> int:
     """Makes one bounded device-side wait run out on purpose; returns the library's code
     (MPT_ERR_TIMEOUT = -6 is the expected outcome) instead of raising."""
@@ -495,6 +514,87 @@ class LstmLayer:
 
     def device_error(self) -> int:
         return int(self.status[3].item())
+
+
+LSTM_T = dict(Wg32=0, Wp32=1, bias32=2, Wg16=3, Wp16=4, bias16=5, dWg16=6, dWp16=7, dbias16=8, s1_Wg32=9, s1_Wp32=10,
+              s1_bias32=11, xr16=12, dr_ext16=13)
+
+
+class LstmTrainer:
+    """One mpt_lstm_ctx over a torch-allocated workspace: the LSTM layer with projection trained
+    with loss scaling (mpt_lstm_train_step).  Argument marshalling only."""
+
+    def __init__(self, T, B, I, H, P, S, optimizer, device="cuda:0", stream=None):
+        import torch
+        self.desc = LstmDesc(T, B, I, H, P)
+        self.T, self.B, self.I, self.H, self.P = T, B, I, H, P
+        self.optimizer = optimizer
+        self.stream = stream
+        out = C.c_size_t(0)
+        _check(lib().mpt_lstm_workspace_bytes(C.byref(self.desc), C.byref(optimizer), C.byref(out)))
+        nbytes = int(out.value)
+        with torch.cuda.device(torch.device(device)):
+            self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=device)
+            base = (self.workspace.data_ptr() + 255) // 256 * 256
+            self._ctx = C.c_void_p()
+            _check(lib().mpt_lstm_create(C.byref(self.desc), float(S), C.byref(optimizer), C.c_void_p(base), nbytes,
+                                         _stream_ptr(stream), C.byref(self._ctx)))
+        self.workspace_bytes = nbytes
+
+    def _ck(self, code):
+        if code != OK:
+            raise MptError(code, lib().mpt_lstm_last_error(self._ctx).decode())
+
+    def set_params(self, Wg, bias, Wp):
+        Wg = np.ascontiguousarray(Wg, dtype=np.float32)
+        bias = np.ascontiguousarray(bias, dtype=np.float32)
+        Wp = np.ascontiguousarray(Wp, dtype=np.float32)
+        assert Wg.shape == (4 * self.H, self.I + self.P) and bias.shape == (4 * self.H,) and Wp.shape == (self.P, self.H)
+        self._ck(lib().mpt_lstm_set_params(self._ctx, _hptr(Wg), _hptr(bias), _hptr(Wp)))
+
+    def train_step(self, x_dev, labels_dev, want=True):
+        """x_dev: FP16 bits [T, B, I]; labels_dev: int32 [T*B].  Returns (loss, overflow) when `want`."""
+        if not want:
+            self._ck(lib().mpt_lstm_train_step(self._ctx, _dptr(x_dev), _dptr(labels_dev), None, None))
+            return None
+        loss, flag = C.c_float(0.0), C.c_int(0)
+        self._ck(lib().mpt_lstm_train_step(self._ctx, _dptr(x_dev), _dptr(labels_dev), C.byref(loss), C.byref(flag)))
+        return float(loss.value), int(flag.value)
+
+    def get_tensor(self, name):
+        T, B, I, H, P = self.T, self.B, self.I, self.H, self.P
+        K = I + P
+        by_param = dict(Wg=(4 * H, K), Wp=(P, H), bias=(4 * H,))
+        if name == "xr16":
+            shape = (T + 1, B, K)
+        elif name == "dr_ext16":
+            shape = (T, B, P)
+        else:
+            shape = next(v for k, v in by_param.items() if k in name)
+        dt = np.float32 if name.endswith("32") else np.uint16
+        out = np.empty(shape, dtype=dt)
+        self._ck(lib().mpt_lstm_get_tensor(self._ctx, LSTM_T[name], _hptr(out), out.nbytes))
+        return out
+
+    def set_dynamic_scale(self, enable, growth_interval=2000, min_scale=2.0 ** -100, max_scale=2.0 ** 120):
+        self._ck(lib().mpt_lstm_set_dynamic_scale(self._ctx, int(bool(enable)), int(growth_interval), float(min_scale),
+                                                  float(max_scale)))
+
+    def get_scale(self):
+        s = C.c_float(0.0)
+        self._ck(lib().mpt_lstm_get_scale(self._ctx, C.byref(s)))
+        return float(s.value)
+
+    def close(self):
+        if getattr(self, "_ctx", None):
+            lib().mpt_lstm_destroy(self._ctx)
+            self._ctx = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
 
 
 # ------------------------------------------------------------------ data-parallel step

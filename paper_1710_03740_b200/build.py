@@ -16,7 +16,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmpt.so")
-SOURCES = ["update.cu", "softmax_ce.cu", "gemm_simt.cu", "gemm_tc.cu", "gemm_tc2.cu", "gemm_tc3.cu", "lstm.cu", "lstm_api.cu", "dp_exchange.cu", "wait_selftest.cu", "mpt_api.cu"]
+SOURCES = ["update.cu", "softmax_ce.cu", "gemm_simt.cu", "gemm_tc.cu", "gemm_tc2.cu", "gemm_tc3.cu", "lstm.cu", "lstm_api.cu", "lstm_train.cu", "dp_exchange.cu", "wait_selftest.cu", "clock_probe.cu", "mpt_api.cu"]
 HEADERS = [os.path.join(CSRC, "mpt_common.cuh"), os.path.join(CSRC, "tc_ptx.cuh"), os.path.join(CSRC, "update_math.cuh"),
            os.path.join(ROOT, "include", "mpt.h")]
 

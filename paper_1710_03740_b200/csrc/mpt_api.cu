@@ -1064,6 +1064,13 @@ int mpt_softmax_ce(const uint16_t *z_dev, int ldz, const int32_t *labels_dev, in
     return e == cudaSuccess ? MPT_OK : MPT_ERR_CUDA;
 }
 
+int mpt_sm_clock_probe(unsigned window_us, float *mhz_dev, void *cuda_stream)
+{
+    if (!mhz_dev) return MPT_ERR_INVALID_ARG;
+    if (window_us < 1 || window_us > 100000u) return MPT_ERR_INVALID_ARG;
+    return launch_clock_probe(window_us, mhz_dev, (cudaStream_t)cuda_stream) == cudaSuccess ? MPT_OK : MPT_ERR_CUDA;
+}
+
 int mpt_selftest_wait_timeout(unsigned limit_us, uint32_t *status_dev, void *cuda_stream)
 {
     if (!status_dev) return MPT_ERR_INVALID_ARG;

@@ -116,6 +116,8 @@ cudaError_t launch_update(const uint16_t *g16, float *w32, float *v, uint16_t *w
 cudaError_t launch_softmax_ce(const uint16_t *z, int ldz, const int32_t *labels, int B, int C, float S,
                               uint16_t *dz, int lddz, float *row_loss, float *loss, uint32_t *bad_labels,
                               cudaStream_t st, int *n_launches, const float *S_dev = nullptr, uint32_t *kerr = nullptr);
+// One warp measures its SM's clock over window_us of wall time and writes MHz to *mhz_out (clock_probe.cu).
+cudaError_t launch_clock_probe(unsigned window_us, float *mhz_out, cudaStream_t st);
 // One CTA waits, for at most limit_us, on a barrier nothing arrives on; on expiry it records
 // KERR_WAIT_SELFTEST in *status (wait_selftest.cu).
 cudaError_t launch_wait_selftest(unsigned limit_us, uint32_t *status, cudaStream_t st);

@@ -91,3 +91,15 @@ def test_softmax_status_word_stays_clear_on_the_bulk_kernel():
     b.mpt_softmax_ce_static(z, C, y, B, C, 128.0, dz, C, loss, None, status=status)
     torch.cuda.synchronize()
     assert int(status.item()) == 0 and np.isfinite(float(loss.item()))
+
+
+def test_sm_clock_probe_reports_a_plausible_clock():
+    from paper_1710_03740_b200 import binding as b
+    mhz = torch.zeros(2, dtype=torch.float32, device="cuda")
+    b.mpt_sm_clock_probe(50, mhz[0:1])
+    b.mpt_sm_clock_probe(200, mhz[1:2])
+    torch.cuda.synchronize()
+    a, c = mhz.tolist()
+    assert 100.0 < a < 2500.0 and 100.0 < c < 2500.0
+    with pytest.raises(b.MptError):
+        b.mpt_sm_clock_probe(0, mhz)

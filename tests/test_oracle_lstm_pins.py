@@ -149,3 +149,81 @@ def test_weight_gradient_sums_over_time_before_rounding():
     ref = sum(net.dG[t].view(np.float16).astype(np.float64).T @ net.xr[t].view(np.float16).astype(np.float64) for t in range(T))
     got = net.dWg.view(np.float16).astype(np.float64)
     assert np.abs(got - ref).max() <= 2.0 ** -10 * np.abs(ref).max() + 1e-7
+
+
+def _trainer_case(seed=21, T=4, B=5, I=8, H=16, P=8):
+    rng = np.random.default_rng(seed)
+    x = _rand16(rng, T, B, I, scale=1.0)
+    Wg, b, Wp = _rand16(rng, 4 * H, I + P), _rand16(rng, 4 * H), _rand16(rng, P, H, scale=0.8)
+    y = rng.integers(0, P, T * B).astype(np.int32)
+    return (T, B, I, H, P), x, Wg, b, Wp, y
+
+
+def test_trainer_loss_and_gradients_against_torch_float64_and_adagrad_first_step():
+    """The trained layer (forward from zero state, cross-entropy over r_t as logits, BPTT, unscale,
+    Adagrad on the masters) against torch float64: nn.LSTM with a projection, F.cross_entropy (mean),
+    autograd.  The first Adagrad step from zero state is w - lr*g/(|g| + eps) in closed form."""
+    from oracle.lstm import OracleLSTMTrainer
+    (T, B, I, H, P), x, Wg, b, Wp, y = _trainer_case()
+    S, lr, eps = 128.0, 0.05, 1e-6
+    tr = OracleLSTMTrainer(T, B, I, H, P, S, mpo.OPT_ADAGRAD, lr, eps=eps)
+    tr.set_params(Wg.astype(np.float32), b.astype(np.float32), Wp.astype(np.float32))
+    w0 = {k: v.copy() for k, v in tr.w32.items()}
+    loss = tr.forward_backward(x, y)
+    lstm, xt, out = _torch_lstm(T, B, I, H, P, x, np.zeros((B, P), np.float16), np.zeros((B, H), np.float16), Wg, b, Wp)
+    ref = torch.nn.functional.cross_entropy(out.reshape(T * B, P), torch.from_numpy(y.astype(np.int64)))
+    assert abs(loss - ref.item()) < 2e-3 * ref.item()
+    ref.backward()
+    dWg_ref = np.zeros((4 * H, I + P))
+    db_ref = np.zeros(4 * H)
+    for q in range(4):
+        dWg_ref[q::4, :I] = lstm.weight_ih_l0.grad.numpy()[q * H:(q + 1) * H]
+        dWg_ref[q::4, I:] = lstm.weight_hh_l0.grad.numpy()[q * H:(q + 1) * H]
+        db_ref[q::4] = lstm.bias_ih_l0.grad.numpy()[q * H:(q + 1) * H]
+    refs = dict(Wg=dWg_ref, Wp=lstm.weight_hr_l0.grad.numpy(), bias=db_ref)
+    unscaled = {k: tr.g16[k].view(np.float16).astype(np.float64) / S for k in tr.names}
+    for k in tr.names:
+        scale = np.abs(refs[k]).max()
+        assert scale > 0 and np.abs(unscaled[k] - refs[k].reshape(unscaled[k].shape)).max() < 0.03 * scale, k
+    assert tr.step() == 0
+    for k in tr.names:
+        g = tr.g16[k].view(np.float16).astype(np.float32) * np.float32(1.0 / S)
+        want = w0[k].astype(np.float64) - lr * g.astype(np.float64) / (np.abs(g.astype(np.float64)) + eps)
+        assert np.allclose(tr.w32[k], want.reshape(tr.w32[k].shape), rtol=0, atol=2e-6), k
+        assert np.array_equal(tr.w16[k], mpo.f2h(tr.w32[k]))
+        # Adagrad's state after one step is the squared unscaled gradient, bit for bit
+        assert np.array_equal(tr.s1[k].reshape(-1), (g * g).reshape(-1))
+
+
+def test_trainer_loss_falls_and_overflow_skips_and_dynamic_scale_recovers():
+    from oracle.lstm import OracleLSTMTrainer
+    (T, B, I, H, P), x, Wg, b, Wp, y = _trainer_case(seed=22)
+    tr = OracleLSTMTrainer(T, B, I, H, P, 128.0, mpo.OPT_ADAGRAD, 0.05, eps=1e-6)
+    tr.set_params(Wg.astype(np.float32), b.astype(np.float32), Wp.astype(np.float32))
+    losses = [tr.train_step(x, y)[0] for _ in range(8)]
+    assert losses[-1] < 0.8 * losses[0]                      # the same batch repeated: the loss must fall
+    # a scale far too large overflows the weight gradients: every tensor untouched, flag 1
+    big = OracleLSTMTrainer(T, B, I, H, P, 2.0 ** 24, mpo.OPT_ADAGRAD, 0.05, eps=1e-6)
+    big.set_params(Wg.astype(np.float32), b.astype(np.float32), Wp.astype(np.float32))
+    before = {k: v.copy() for k, v in big.w32.items()}
+    loss, flag = big.train_step(x, y)
+    assert flag == 1 and all(np.array_equal(before[k], big.w32[k]) for k in big.names)
+    assert not any(big.s1[k].any() for k in big.names)
+    # with the dynamic schedule the scale halves until the step applies, then stays
+    big.set_dynamic_scale(1000, 1.0, 2.0 ** 24)
+    flags, scales = [], []
+    for _ in range(12):
+        flags.append(big.train_step(x, y)[1])
+        scales.append(float(big.S))
+    assert flags[0] == 1 and flags[-1] == 0 and 0 in flags
+    first_ok = flags.index(0)
+    assert all(f == 1 for f in flags[:first_ok]) and all(f == 0 for f in flags[first_ok:])
+    assert scales[first_ok] == scales[-1] == 2.0 ** 24 / 2 ** first_ok
+    # the settled run equals a constant-scale run started at that scale, bit for bit (scaling by a
+    # power of two is exact as long as nothing leaves the FP16 range)
+    ref = OracleLSTMTrainer(T, B, I, H, P, scales[-1], mpo.OPT_ADAGRAD, 0.05, eps=1e-6)
+    ref.set_params(Wg.astype(np.float32), b.astype(np.float32), Wp.astype(np.float32))
+    for _ in range(12 - first_ok):
+        ref.train_step(x, y)
+    for k in ref.names:
+        assert np.array_equal(ref.w32[k], big.w32[k]), k
