@@ -1,6 +1,9 @@
 """Builds the CUDA shared library in-tree with nvcc for sm_100a.
 
-    python -m paper_1710_03740_b200.build [--force] [--verbose]
+    python -m paper_1710_03740_b200.build [--force] [--verbose] [--trace]
+
+--trace additionally builds libmpt_trace.so: the same library with the CTA-pair product kernel
+instrumented (per-cluster timestamps and cycle counts; see kernel_bench gemm --trace).
 
 Output: paper_1710_03740_b200/libmpt.so (cudart linked statically, so the library
 loads on a machine without a GPU; the driver entry point for tensor-map encoding is
@@ -57,5 +60,20 @@ def build(force=False, verbose=False):
     return LIB
 
 
+def build_trace():
+    """libmpt_trace.so: every object of the normal build except gemm_tc2, which is recompiled with
+    -DMPT_GEMM_TRACE."""
+    build()
+    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    o = os.path.join(CSRC, "gemm_tc2_trace.o")
+    subprocess.run([nvcc] + NVCC_FLAGS + ["-DMPT_GEMM_TRACE", "-c", os.path.join(CSRC, "gemm_tc2.cu"), "-o", o], check=True)
+    objs = [os.path.join(CSRC, s.replace(".cu", ".o")) for s in SOURCES if s != "gemm_tc2.cu"] + [o]
+    lib = os.path.join(HERE, "libmpt_trace.so")
+    subprocess.run([nvcc, "-shared", "-cudart", "static", "-gencode", "arch=compute_100a,code=sm_100a", "-o", lib] + objs, check=True)
+    return lib
+
+
 if __name__ == "__main__":
     print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
+    if "--trace" in sys.argv:
+        print(build_trace())

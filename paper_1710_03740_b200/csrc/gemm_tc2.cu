@@ -251,6 +251,15 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
             uint32_t s = 0, ph = 0;
             bool ok = true;
             int t = 0;
+#ifdef MPT_GEMM_TRACE
+            // Trace build only (python -m paper_1710_03740_b200.build --trace): the issuing thread of every
+            // cluster records when it started, how many SM cycles its main loops took and how many
+            // k-blocks it issued, into words [64 + 8 * cluster ...] of the status array, which the
+            // caller must then size at 1024 words.
+            const unsigned long long tr_t0 = global_ns();
+            const long long tr_c0 = clock64();
+            unsigned tr_kb = 0;
+#endif
             for (int u = pair_id; u < num_units && ok; u += num_pairs, t++) {
                 const Unit w = unit_of(p, u, nkb);
                 const uint32_t idesc = idesc_base | ((uint32_t)(w.width >> 3) << 17);
@@ -280,9 +289,22 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
                     }
                     tc_commit_pair(empty_bar(s), 3);        // both CTAs' producers may refill stage s
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
+#ifdef MPT_GEMM_TRACE
+                    tr_kb++;
+#endif
                 }
                 if (ok) tc_commit_pair(accf_bar(buf), 3);   // both CTAs' epilogues may read the accumulator
             }
+#ifdef MPT_GEMM_TRACE
+            if (p.status) {
+                uint32_t *tr = p.status + 64 + 8 * pair_id;
+                tr[0] = (uint32_t)tr_t0;
+                tr[1] = (uint32_t)global_ns();
+                tr[2] = (uint32_t)(clock64() - tr_c0);
+                tr[3] = tr_kb;
+                tr[4] = (uint32_t)t;
+            }
+#endif
         }
     } else {
         // ---------------------------------------------------------------- epilogue (both CTAs)

@@ -99,6 +99,40 @@ def bench_gemm(M, N, K, op, iters, flags=mpt.GEMM_FORCE_TC, use_workspace=True):
     return out
 
 
+def trace_gemm(M, N, K, op):
+    """One launch of the CTA-pair kernel from the trace build (build.py --trace) after 30 warm-up
+    launches: per cluster, the main loops' SM cycles per issued k-block (512 = the tensor pipe's
+    full rate for a 256x256x64 block), the SM clock they ran at, and when the clusters finished."""
+    import numpy as np
+    sa = (K, M) if op == 2 else (M, K)
+    sb = (N, K) if op == 0 else (K, N)
+    g = torch.Generator(device="cuda").manual_seed(2)
+    A = (torch.randn(sa, device="cuda", generator=g) * K ** -0.5).half()
+    B = (torch.randn(sb, device="cuda", generator=g) * K ** -0.5).half()
+    C = torch.empty((M, N), dtype=torch.half, device="cuda")
+    st = torch.zeros(1024, dtype=torch.int32, device="cuda")
+    nws = mpt.mpt_gemm_workspace_bytes(op, M, N, K)
+    ws = torch.empty(max(nws, 16) // 4, dtype=torch.float32, device="cuda")
+    run = lambda: mpt.mpt_gemm_f16_ws(op, M, N, K, A, sa[1], B, sb[1], C, N, mpt.GEMM_FORCE_PAIR, None, 0, None, st,  # noqa: E731
+                                      ws if nws else None)
+    for _ in range(30):
+        run()
+    torch.cuda.synchronize()
+    st.zero_()
+    run()
+    torch.cuda.synchronize()
+    t = st.cpu().numpy().view(np.uint32)[64:64 + 8 * 74].reshape(74, 8).astype(np.int64)
+    t = t[t[:, 3] > 0]
+    us = ((t[:, 1] - t[:, 0]) % (1 << 32)) / 1e3
+    end = ((t[:, 1] - t[:, 0].min()) % (1 << 32)) / 1e3
+    cyc, kb = t[:, 2], t[:, 3]
+    return {"kernel": "gemm_trace", "op": OPS[op], "M": M, "N": N, "K": K, "clusters": int(len(t)),
+            "units_per_cluster": [int(t[:, 4].min()), int(t[:, 4].max())],
+            "cycles_per_kblock_median": float(np.median(cyc / kb)), "cycles_per_kblock_max": float((cyc / kb).max()),
+            "sm_mhz_median": float(np.median(cyc / us)), "last_issue_us": [float(end.min()), float(end.max())],
+            "device_error": int(st[0])}
+
+
 def bench_update(n, momentum, iters):
     g = torch.Generator(device="cuda").manual_seed(3)
     g16 = (torch.randn(n, device="cuda", generator=g) * 37).half()
@@ -277,6 +311,8 @@ def main():
     g.add_argument("--op", nargs="*", type=int, default=[0, 1, 2])
     g.add_argument("--iters", type=int, default=20)
     g.add_argument("--no-workspace", action="store_true", help="do not offer a split-K scratch buffer")
+    g.add_argument("--trace", action="store_true",
+                   help="per-cluster main-loop cycles from the instrumented build (python -m paper_1710_03740_b200.build --trace)")
     g.add_argument("--kernel", default="auto", choices=["auto", "tc", "pair", "pair512"],
                    help="auto: the library's choice; tc: single-CTA 128x256 tiles; pair: cta_group::2 256x256 tiles")
     u = sub.add_parser("update")
@@ -305,6 +341,13 @@ def main():
     args = ap.parse_args()
     if args.cmd == "step":
         print(json.dumps(bench_step(args.workload, args.iters)), flush=True)
+    elif args.cmd == "gemm" and args.trace:
+        import os
+        mpt.LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libmpt_trace.so")
+        for t in args.shape or ["4096x12288x12288"]:
+            M, N, K = (int(x) for x in t.split("x"))
+            for op in args.op:
+                print(json.dumps(trace_gemm(M, N, K, op)), flush=True)
     elif args.cmd == "gemm":
         shapes = ([tuple(int(x) for x in t.split("x")) for t in args.shape] if args.shape
                   else inputs.GEMM_SWEEP + [inputs.LSTM_GATE, inputs.LSTM_PROJ])
