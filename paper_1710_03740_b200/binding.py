@@ -13,7 +13,8 @@ import os
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libmpt.so")
+# MPT_LIB: another build of the library to load instead (comparing two builds in one session)
+LIB_PATH = os.environ.get("MPT_LIB") or os.path.join(_HERE, "libmpt.so")
 
 OK = 0
 ERR = {-1: "MPT_ERR_INVALID_ARG", -2: "MPT_ERR_SHAPE", -3: "MPT_ERR_STATE", -4: "MPT_ERR_WORKSPACE",
