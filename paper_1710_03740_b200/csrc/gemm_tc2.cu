@@ -603,7 +603,12 @@ cudaError_t launch_gemm_tc2(int op, int M, int N, int K, const uint16_t *A, int 
     p.status = status;
     p.tiles_m = (M + 2 * CTA_M - 1) / (2 * CTA_M);
     p.tiles_n = (N + TILE_N - 1) / TILE_N;
-    p.group_m = 8;
+    // Row blocks per group of the tile order.  Consecutive waves of a group share its A panels; whether
+    // those survive in L2 between waves depends on their size: with the short panels of a weight-gradient
+    // product (K = batch = 4096: 2 MB each) 16 of them do, and DRAM reads of 12288x12288x4096 fall from
+    // 1.01 GB (groups of 8) to 0.66 GB (0.77 / 0.82 / 1.00 / 1.57 GB with 12 / 24 / 32 / 4); with 6.3 MB
+    // panels (K = 12288) nothing survives either way and 8 keeps the wave's own footprint smallest.
+    p.group_m = K <= 6144 ? 16 : 8;
     p.full_units = p.num_units = 0;
     p.split_k = 1;
     p.partial = nullptr;
