@@ -81,41 +81,50 @@ def dp_step_over_peers(n, iters, dev):
     this job: every rank owns exchange buffers the others map.  Times the kernel with CUDA events
     between process-group barriers; returns the slowest rank's median and the bytes each GPU pulls
     and pushes over NVLink per step.  An extra: not part of the step metric."""
+    import datetime
     import torch
     import torch.distributed as dist
     from paper_1710_03740_b200 import binding as mpt
-    dp, err = None, None
+    # Every collective of this extra runs on its own gloo group with a short time limit: a rank that
+    # fails (no peer access, a launch error) must end this measurement on all ranks within a minute,
+    # never hang the benchmark whose line is still to be printed.
+    grp = dist.new_group(backend="gloo", timeout=datetime.timedelta(seconds=60))
+    dp = None
     try:
-        dp = mpt.DataParallelFlat(n, 512.0, 1e-4, 0.9)
-    except Exception as ex:       # e.g. no peer access between two of the GPUs
-        err = repr(ex)
-    # every rank must agree to go on: the timing loop below is full of barriers
-    ok = torch.tensor([0 if dp is None else 1], dtype=torch.int32, device=dev)
-    dist.all_reduce(ok, op=dist.ReduceOp.MIN)
-    if int(ok.item()) == 0:
-        return {"error": err or "set-up failed on another rank"}
-    g = torch.Generator(device=dev).manual_seed(3 + dp.rank)
-    dp.g16.copy_((torch.randn(n, device=dev, generator=g) * 37).half().view(torch.int16))
-    times = []
-    for it in range(iters + 2):
-        dp._barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        mpt.mpt_dp_step_flat([p["g16"] for p in dp._peers], [p["flags"] for p in dp._peers], [p["w16"] for p in dp._peers],
-                             dp.w32, dp.v, dp.n, dp.R, dp.rank, dp.S, dp.lr, dp.mu, dp._own["flags"])
-        e1.record()
-        dp._barrier()
-        if it >= 2:
-            times.append(e0.elapsed_time(e1))
-    times.sort()
-    med = max_over_ranks([times[len(times) // 2]], dev)[0]
-    shard = dp.hi - dp.lo
-    link = 2 * shard * (dp.R - 1)
-    res = {"replicas": dp.R, "params": n, "shard": shard, "ms": med, "peers": "remote (one GPU per replica)",
-           "link_bytes_each_way": link, "link_gbs_each_way": link / med / 1e6,
-           "hbm_bytes": (2 + 16 + 2) * shard}
-    dp.close()
-    return res
+        err = None
+        try:
+            dp = mpt.DataParallelFlat(n, 512.0, 1e-4, 0.9, group=grp)
+        except Exception as ex:       # e.g. no peer access between two of the GPUs
+            err = repr(ex)
+        ok = torch.tensor([0 if dp is None else 1], dtype=torch.int32)
+        dist.all_reduce(ok, op=dist.ReduceOp.MIN, group=grp)
+        if int(ok.item()) == 0:
+            return {"error": err or "set-up failed on another rank"}
+        g = torch.Generator(device=dev).manual_seed(3 + dp.rank)
+        dp.g16.copy_((torch.randn(n, device=dev, generator=g) * 37).half().view(torch.int16))
+        times = []
+        for it in range(iters + 2):
+            dp._barrier()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            mpt.mpt_dp_step_flat([p["g16"] for p in dp._peers], [p["flags"] for p in dp._peers], [p["w16"] for p in dp._peers],
+                                 dp.w32, dp.v, dp.n, dp.R, dp.rank, dp.S, dp.lr, dp.mu, dp._own["flags"])
+            e1.record()
+            dp._barrier()
+            if it >= 2:
+                times.append(e0.elapsed_time(e1))
+        times.sort()
+        t = torch.tensor([times[len(times) // 2]], dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX, group=grp)
+        med = float(t.item())
+        shard = dp.hi - dp.lo
+        link = 2 * shard * (dp.R - 1)
+        res = {"replicas": dp.R, "params": n, "shard": shard, "ms": med, "peers": "remote (one GPU per replica)",
+               "link_bytes_each_way": link, "link_gbs_each_way": link / med / 1e6, "hbm_bytes": (2 + 16 + 2) * shard}
+        dp.close()
+        return res
+    except BaseException as ex:       # an extra: whatever goes wrong here is reported, not raised
+        return {"error": repr(ex)}
 
 
 def step_flops(cfg):
