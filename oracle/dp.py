@@ -35,11 +35,12 @@ class OracleDataParallelMLP:
     def set_grad(self, q, l, g16):
         self.replicas[q].set_grad(l, g16)
 
-    def set_optimizer(self, kind, lr, mu=0.0, b2=0.0, eps=0.0, wd=0.0):
-        """Any kind of mlp.OracleMLP.set_optimizer except clipping (its norm would have to be taken
-        over the mean gradient of all replicas; not part of this step)."""
+    def set_optimizer(self, kind, lr, mu=0.0, b2=0.0, eps=0.0, wd=0.0, clip=0.0):
+        """Any kind of mlp.OracleMLP.set_optimizer.  Clipping (section 3.2) bounds the global norm of
+        the MEAN unscaled gradient over all layers - the gradient of the aggregated batch - so every
+        replica applies the same coefficient."""
         for r in self.replicas:
-            r.set_optimizer(kind, lr, mu, b2, eps, wd, clip=0.0)
+            r.set_optimizer(kind, lr, mu, b2, eps, wd, clip=clip)
 
     def step(self):
         lead = self.replicas[0]
@@ -50,7 +51,13 @@ class OracleDataParallelMLP:
                 overflow |= mpo.grad_nonfinite(g, inv)
         if not overflow:
             kind = lead.opt["kind"]
-            plain = kind == mpo.OPT_SGD and float(lead.opt["wd"]) == 0.0
+            clip = lead.opt["clip"]
+            plain = kind == mpo.OPT_SGD and float(lead.opt["wd"]) == 0.0 and clip <= 0.0
+            if clip > 0.0:
+                total = sum(mpo.dp_grad_sqnorm([r.g16[l] for r in self.replicas], lead.S) for l in range(len(lead.layers)))
+                coef = mpo.clip_coef(total, clip)
+                for r in self.replicas:
+                    r.last_coef = coef
             if kind == mpo.OPT_ADAM:       # bias corrections use the products including this step
                 for r in self.replicas:
                     r.b1t = np.float32(r.b1t * r.mu)
@@ -61,6 +68,11 @@ class OracleDataParallelMLP:
                 gs = [r.g16[l] for r in self.replicas]
                 if plain:
                     mpo.dp_update_apply(gs, lead.w32[l], lead.v[l], lead.w16[l], lead.S, lead.lr, lead.mu, lead.use_momentum)
+                elif clip > 0.0:
+                    s1 = lead.v[l] if (kind != mpo.OPT_SGD or lead.use_momentum) else None
+                    s2 = lead.s2[l] if kind == mpo.OPT_ADAM else None
+                    mpo.dp_update_apply_clip(kind, gs, lead.w32[l], s1, s2, lead.w16[l], lead.S, lead.last_coef, lead.lr,
+                                             lead.mu, lead.opt["b2"], lead.opt["eps"], lead.opt["wd"], bc1, bc2)
                 else:
                     s1 = lead.v[l] if (kind != mpo.OPT_SGD or lead.use_momentum) else None
                     s2 = lead.s2[l] if kind == mpo.OPT_ADAM else None

@@ -432,6 +432,43 @@ void mpo_dp_update_apply_opt(int kind, const uint16_t *const *g16, int R, float 
 }
 
 /*
+ * Global-norm clipping in the data-parallel setting (section 3.2 puts clipping after unscaling;
+ * section 4.5 aggregates the batch over several GPUs): the norm is that of the MEAN gradient the
+ * update uses, g = (h2f(g_0[i]) + ... + h2f(g_{R-1}[i])) * inv_SR in binary32 as above, squares and
+ * their sum in double; the update multiplies g by coef right after forming it, then the lines of
+ * mpo_opt_elem unchanged.
+ */
+double mpo_dp_grad_sqnorm(const uint16_t *const *g16, int R, size_t n, float inv_SR)
+{
+    double total = 0.0;
+#pragma omp parallel for schedule(static) reduction(+ : total)
+    for (size_t i = 0; i < n; i++) {
+        float s = mpo_h2f(g16[0][i]);
+        for (int q = 1; q < R; q++) s = s + mpo_h2f(g16[q][i]);
+        float g = s * inv_SR;
+        total += (double)g * (double)g;
+    }
+    return total;
+}
+
+void mpo_dp_update_apply_clip(int kind, const uint16_t *const *g16, int R, float *w32, float *s1, float *s2,
+                              uint16_t *w16, size_t n, float inv_SR, float coef, float lr, float mu, float b2,
+                              float eps, float wd, float bc1, float bc2)
+{
+    const float omb1 = 1.0f - mu, omb2 = 1.0f - b2;
+#pragma omp parallel for schedule(static)
+    for (size_t i = 0; i < n; i++) {
+        float s = mpo_h2f(g16[0][i]);
+        for (int q = 1; q < R; q++) s = s + mpo_h2f(g16[q][i]);
+        float g = s * inv_SR;
+        g = g * coef;
+        float w = mpo_opt_elem(kind, g, w32[i], s1, s2, i, lr, mu, b2, eps, wd, omb1, omb2, bc1, bc2);
+        w32[i] = w;
+        w16[i] = mpo_f2h(w);
+    }
+}
+
+/*
  * Sum of squares of the unscaled weight gradients, accumulated in double (section 3.2: gradient
  * clipping acts on the unscaled gradients; section 3.3: reductions are carried out in higher
  * precision than the stored values).  Global-norm clipping then multiplies every unscaled

@@ -90,6 +90,12 @@ def lib() -> ctypes.CDLL:
         L.mpo_dp_update_apply_opt.argtypes = [c.c_int, c.c_void_p, c.c_int, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p,
                                               c.c_size_t, c.c_float, c.c_float, c.c_float, c.c_float, c.c_float, c.c_float,
                                               c.c_float, c.c_float]
+        L.mpo_dp_grad_sqnorm.restype = c.c_double
+        L.mpo_dp_grad_sqnorm.argtypes = [c.c_void_p, c.c_int, c.c_size_t, c.c_float]
+        L.mpo_dp_update_apply_clip.restype = None
+        L.mpo_dp_update_apply_clip.argtypes = [c.c_int, c.c_void_p, c.c_int, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p,
+                                               c.c_size_t, c.c_float, c.c_float, c.c_float, c.c_float, c.c_float, c.c_float,
+                                               c.c_float, c.c_float, c.c_float]
         L.mpo_dp_update_apply.restype = None
         L.mpo_dp_update_apply.argtypes = [c.c_void_p, c.c_int, c.c_void_p, c.c_void_p, c.c_void_p, c.c_size_t,
                                           c.c_float, c.c_float, c.c_float, c.c_int]
@@ -332,6 +338,25 @@ def dp_update_apply(g16_list, w32, v, w16, S, lr, mu, use_momentum) -> None:
     table = (ctypes.c_void_p * R)(*[g.ctypes.data for g in gs])
     lib().mpo_dp_update_apply(table, R, _ptr(w32), _ptr(v) if use_momentum else None, _ptr(w16), gs[0].size,
                               float(dp_inv_scale(S, R)), float(lr), float(mu), int(bool(use_momentum)))
+
+
+def dp_grad_sqnorm(g16_list, S) -> float:
+    """Sum of squares (double) of the mean unscaled gradient of the replicas (see mpo.c)."""
+    gs = [np.ascontiguousarray(_u16(g)).reshape(-1) for g in g16_list]
+    R = len(gs)
+    table = (ctypes.c_void_p * R)(*[g.ctypes.data for g in gs])
+    return float(lib().mpo_dp_grad_sqnorm(table, R, gs[0].size, float(dp_inv_scale(S, R))))
+
+
+def dp_update_apply_clip(kind, g16_list, w32, s1, s2, w16, S, coef, lr, mu, b2=0.0, eps=0.0, wd=0.0, bc1=1.0, bc2=1.0) -> None:
+    """dp_update_apply_opt with the clipping coefficient applied to the mean gradient."""
+    gs = [np.ascontiguousarray(_u16(g)).reshape(-1) for g in g16_list]
+    R = len(gs)
+    assert R >= 1 and all(g.size == gs[0].size for g in gs)
+    table = (ctypes.c_void_p * R)(*[g.ctypes.data for g in gs])
+    lib().mpo_dp_update_apply_clip(int(kind), table, R, _ptr(w32), _ptr(s1), _ptr(s2), _ptr(w16), gs[0].size,
+                                   float(dp_inv_scale(S, R)), float(coef), float(lr), float(mu), float(b2), float(eps),
+                                   float(wd), float(bc1), float(bc2))
 
 
 def dp_update_apply_opt(kind, g16_list, w32, s1, s2, w16, S, lr, mu, b2=0.0, eps=0.0, wd=0.0, bc1=1.0, bc2=1.0) -> None:

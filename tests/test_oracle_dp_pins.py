@@ -252,3 +252,60 @@ def test_mlp_optimizer_replicas_fed_the_same_batch_equal_one_replica(kind):
             for l in range(2):
                 assert np.array_equal(dp.replicas[q].w32[l].view(np.uint32), one.w32[l].view(np.uint32))
                 assert np.array_equal(dp.replicas[q].w16[l], one.w16[l])
+
+
+def test_clip_one_replica_is_the_single_gpu_clip_and_identical_replicas_too():
+    # R = 1: norm and update are those of the pinned single-GPU clipping; four identical replicas with
+    # a power-of-two S have the same mean gradient bit for bit, hence the same norm and the same step
+    n, S = 4099, 256.0
+    g = inputs.loguniform_grads(n, S, seed=31).view(np.uint16)
+    inv = np.float32(1.0) / np.float32(S)
+    assert mpo.dp_grad_sqnorm([g], S) == mpo.grad_sqnorm(g, inv)
+    assert mpo.dp_grad_sqnorm([g, g.copy(), g.copy(), g.copy()], S) == mpo.grad_sqnorm(g, inv)
+    coef = mpo.clip_coef(mpo.grad_sqnorm(g, inv), 1e-4)
+    assert 0.0 < float(coef) < 1.0
+    rng = np.random.default_rng(3)
+    w = rng.standard_normal(n).astype(np.float32)
+    s1 = np.abs(0.1 * rng.standard_normal(n)).astype(np.float32)
+    a = [w.copy(), s1.copy(), np.zeros(n, np.uint16)]
+    b = [w.copy(), s1.copy(), np.zeros(n, np.uint16)]
+    c = [w.copy(), s1.copy(), np.zeros(n, np.uint16)]
+    mpo.dp_update_apply_clip(mpo.OPT_ADAGRAD, [g], a[0], a[1], None, a[2], S, coef, 0.05, 0.0, eps=1e-6)
+    mpo.update_apply_clip(mpo.OPT_ADAGRAD, g, b[0], b[1], None, b[2], inv, coef, 0.05, 0.0, eps=1e-6)
+    mpo.dp_update_apply_clip(mpo.OPT_ADAGRAD, [g, g.copy(), g.copy(), g.copy()], c[0], c[1], None, c[2], S, coef, 0.05, 0.0, eps=1e-6)
+    for x, y, z in zip(a, b, c):
+        assert np.array_equal(x.view(np.uint8), y.view(np.uint8)) and np.array_equal(x.view(np.uint8), z.view(np.uint8))
+
+
+def test_clip_norm_is_taken_over_the_mean_gradient_by_hand():
+    # two replicas with gradients (6, 0) and (0, 8), S = 1: the mean is (3, 4), norm 5 - not the
+    # norm of either replica's gradient (6, 8) nor of their sum (10); bound 2.5 halves the step
+    g0 = np.array([6.0, 0.0], np.float16).view(np.uint16)
+    g1 = np.array([0.0, 8.0], np.float16).view(np.uint16)
+    assert mpo.dp_grad_sqnorm([g0, g1], 1.0) == 25.0
+    coef = mpo.clip_coef(25.0, 2.5)
+    assert float(coef) == float(np.float32(2.5 / (5.0 + 1e-6)))
+    w, h = np.zeros(2, np.float32), np.zeros(2, np.uint16)
+    mpo.dp_update_apply_clip(mpo.OPT_SGD, [g0, g1], w, None, None, h, 1.0, coef, 1.0, 0.0)
+    assert w[0] == -(np.float32(3.0) * coef) and w[1] == -(np.float32(4.0) * coef)
+
+
+def test_mlp_clipped_replicas_fed_the_same_batch_equal_one_clipped_replica():
+    layers = [(16, 24, 1), (24, 5, 0)]
+    dp, one, rng = _mlp_setup(2, layers, S=64.0)
+    dp.set_optimizer(mpo.OPT_SGD, 0.05, 0.9, clip=0.05)
+    one.set_optimizer(mpo.OPT_SGD, 0.05, 0.9, clip=0.05)
+    clipped = False
+    for t in range(3):
+        x = rng.standard_normal((8, 16)).astype(np.float16)
+        y = rng.integers(0, 5, 8).astype(np.int32)
+        dp.forward_backward([x, x.copy()], [y, y.copy()])
+        one.forward(x)
+        one.backward_scaled(y)
+        assert dp.step() == one.step() == 0
+        assert float(dp.replicas[0].last_coef) == float(one.last_coef)
+        clipped |= float(one.last_coef) < 1.0
+        for q in range(2):
+            for l in range(2):
+                assert np.array_equal(dp.replicas[q].w32[l].view(np.uint32), one.w32[l].view(np.uint32))
+    assert clipped
