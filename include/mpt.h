@@ -590,12 +590,25 @@ int mpt_dp_step_flat(const uint16_t *const *g16_peers, const uint32_t *const *fl
 /* The same step with any optimizer of mpt_optimizer on the mean gradient (weight decay, Nesterov,
  * Adagrad, Adam; op order as in mpt_update_flat_opt with g = s * inv_SR).  s1_shard / s2_shard:
  * the FP32 states of this replica's shard (null when the kind does not use them); b1t / b2t as in
- * mpt_update_flat_opt.  Global-norm clipping is not available here (its norm would have to be
- * taken over the mean gradient of all shards before any shard is updated): opt->clip_norm must be
- * 0, else MPT_ERR_INVALID_ARG. */
+ * mpt_update_flat_opt.
+ * Global-norm clipping (section 3.2: after unscaling) bounds the norm of the MEAN gradient over all
+ * n elements, which no single replica sees, so it takes two calls with the replicas ordered in
+ * between: (1) every replica calls mpt_dp_norm_flat, which adds, in double over a fixed partition,
+ * the squares of g = s * inv_SR over its own shard and stores the sum in *norm_slot_dev (a double in
+ * memory the other replicas can map); scratch_dev: MPT_DP_NORM_SCRATCH_BYTES of this replica's own
+ * memory, 8-byte aligned; (2) once every replica's call has completed, mpt_dp_step_flat_opt with
+ * opt->clip_norm > 0 reads all R slots through norm_peers (HOST array of R DEVICE pointers, replica
+ * order), adds them in ascending order, forms coef = min(1, clip_norm / (sqrt(total) + 1e-6)) rounded
+ * to FP32 - the same bits on every replica - writes coef and the norm to clip_out_dev[0..1] (this
+ * replica's memory) and multiplies every g by coef before weight decay and the step.  With
+ * opt->clip_norm == 0 norm_peers and clip_out_dev are ignored (may be null). */
+#define MPT_DP_NORM_SCRATCH_BYTES 8192
+int mpt_dp_norm_flat(const uint16_t *const *g16_peers, size_t n, int R, int rank, float S, void *scratch_dev,
+                     double *norm_slot_dev, void *cuda_stream);
 int mpt_dp_step_flat_opt(const mpt_optimizer *opt, const uint16_t *const *g16_peers, const uint32_t *const *flag_peers,
                          uint16_t *const *w16_peers, float *w32_shard_dev, float *s1_shard_dev, float *s2_shard_dev, size_t n,
-                         int R, int rank, float S, float b1t, float b2t, uint32_t *flags_dev, void *cuda_stream);
+                         int R, int rank, float S, float b1t, float b2t, uint32_t *flags_dev,
+                         const double *const *norm_peers, float *clip_out_dev, void *cuda_stream);
 
 /* Data-parallel training of an mpt_ctx.  mpt_dp_layout_of reports where, inside the context's
  * workspace, the buffers live that the replicas exchange: byte offsets from the workspace base of
@@ -607,8 +620,13 @@ int mpt_dp_step_flat_opt(const mpt_optimizer *opt, const uint16_t *const *g16_pe
  * of the single-GPU master pass.  Entry `rank` of each array must be this context's own buffer.
  * The FP32 master weights and momentum are then current only inside this replica's shard
  * (mpt_get_master returns stale values outside it); the FP16 weights are complete on every
- * replica.  Every optimizer kind and weight decay are supported; global-norm clipping is not
- * (MPT_ERR_STATE from mpt_step).  Dynamic loss scaling works unchanged: every replica sees the same OR-ed
+ * replica.  Every optimizer kind and weight decay are supported.  Global-norm clipping (contexts
+ * created with clip_norm > 0) needs one more call and one more ordering point per iteration: after
+ * mpt_backward_scaled every replica calls mpt_dp_norm (its shard of the squared norm of the mean
+ * gradient, published in its status block next to the overflow word, so no further pointer table is
+ * needed); when every replica's mpt_dp_norm has completed, mpt_step forms the common coefficient
+ * from all replicas' values (mpt_step without that call: MPT_ERR_STATE); mpt_get_grad_norm then
+ * returns the norm of the mean gradient.  Dynamic loss scaling works unchanged: every replica sees the same OR-ed
  * overflow word and moves its scale identically; the kernel reads S from device memory.  The
  * caller orders the replicas around mpt_step as described for mpt_dp_step_flat (before: every
  * replica's mpt_backward_scaled has completed; after: every replica's mpt_step has completed
@@ -620,6 +638,7 @@ typedef struct mpt_dp_layout {
 int mpt_dp_layout_of(mpt_ctx *ctx, mpt_dp_layout *out);
 int mpt_dp_attach(mpt_ctx *ctx, int R, int rank, const uint16_t *const *g16_peers, const uint32_t *const *flag_peers,
                   uint16_t *const *w16_peers);
+int mpt_dp_norm(mpt_ctx *ctx);
 
 /* Device memory that other processes can map (the buffers the replicas exchange).  mpt_dp_alloc
  * returns memory from the driver's allocator (not from a framework's pool, whose blocks cannot be

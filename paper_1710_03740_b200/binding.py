@@ -39,7 +39,7 @@ EXPORTS = ["mpt_workspace_bytes", "mpt_create", "mpt_workspace_bytes_opt", "mpt_
            "mpt_lstm_forward", "mpt_lstm_backward", "mpt_lstm_cell_forward", "mpt_lstm_cell_backward", "mpt_bias_grad",
            "mpt_add_f16",
            "mpt_dp_shard", "mpt_dp_step_flat", "mpt_dp_alloc", "mpt_dp_free", "mpt_dp_export", "mpt_dp_open", "mpt_dp_close",
-           "mpt_dp_layout_of", "mpt_dp_attach", "mpt_dp_step_flat_opt"]
+           "mpt_dp_layout_of", "mpt_dp_attach", "mpt_dp_step_flat_opt", "mpt_dp_norm_flat", "mpt_dp_norm"]
 
 
 class MptError(RuntimeError):
@@ -149,7 +149,9 @@ def lib() -> C.CDLL:
     L.mpt_add_f16.argtypes = [vp, i32, vp, i32, vp, i32, i32, i32, vp]
     L.mpt_dp_shard.argtypes = [sz, i32, i32, C.POINTER(sz), C.POINTER(sz)]
     L.mpt_dp_step_flat.argtypes = [vp, vp, vp, vp, vp, sz, i32, i32, f32, f32, f32, vp, vp]
-    L.mpt_dp_step_flat_opt.argtypes = [C.POINTER(Optimizer), vp, vp, vp, vp, vp, vp, sz, i32, i32, f32, f32, f32, vp, vp]
+    L.mpt_dp_step_flat_opt.argtypes = [C.POINTER(Optimizer), vp, vp, vp, vp, vp, vp, sz, i32, i32, f32, f32, f32, vp, vp, vp, vp]
+    L.mpt_dp_norm_flat.argtypes = [vp, sz, i32, i32, f32, vp, vp, vp]
+    L.mpt_dp_norm.argtypes = [vp]
     L.mpt_dp_alloc.argtypes = [sz, C.POINTER(vp)]
     L.mpt_dp_free.argtypes = [vp]
     L.mpt_dp_export.argtypes = [vp, vp]
@@ -247,6 +249,11 @@ class Context:
         out = DpLayout()
         _check(lib().mpt_dp_layout_of(self._ctx, C.byref(out)), self._ctx)
         return out
+
+    def dp_norm(self):
+        """Clipping in data-parallel mode: publish this replica's shard of the squared norm of the
+        mean gradient (call on every replica after backward_scaled, order the replicas, then step)."""
+        _check(lib().mpt_dp_norm(self._ctx), self._ctx)
 
     def dp_attach(self, R, rank, g16_peers, flag_peers, w16_peers):
         tab = lambda xs: (C.c_void_p * R)(*[_addr(x) for x in xs])
@@ -632,15 +639,30 @@ def mpt_dp_step_flat(g16_peers, flag_peers, w16_peers, w32_shard, v_shard, n, R,
                                   _stream_ptr(stream)))
 
 
+DP_NORM_SCRATCH_BYTES = 8192
+
+
+def mpt_dp_norm_flat(g16_peers, n, R, rank, S, scratch, norm_slot, stream=None):
+    """First half of clipping in data-parallel mode: this replica's shard of the squared norm of the
+    mean unscaled gradient, as a double in norm_slot (memory the other replicas can map)."""
+    assert len(g16_peers) == R
+    tab = (C.c_void_p * R)(*[_addr(x) for x in g16_peers])
+    _check(lib().mpt_dp_norm_flat(tab, int(n), int(R), int(rank), float(S), C.c_void_p(_addr(scratch)),
+                                  C.c_void_p(_addr(norm_slot)), _stream_ptr(stream)))
+
+
 def mpt_dp_step_flat_opt(opt, g16_peers, flag_peers, w16_peers, w32_shard, s1_shard, s2_shard, n, R, rank, S, b1t, b2t,
-                         flags, stream=None):
-    """mpt_dp_step_flat with any optimizer kind and weight decay (no clipping)."""
+                         flags, stream=None, norm_peers=None, clip_out=None):
+    """mpt_dp_step_flat with any optimizer kind and weight decay; with opt.clip_norm > 0 also
+    norm_peers (the R replicas' norm slots, after mpt_dp_norm_flat on every replica) and clip_out
+    (two floats of this replica: coefficient, norm)."""
     assert len(g16_peers) == R and len(flag_peers) == R and len(w16_peers) == R
     tab = lambda xs: (C.c_void_p * R)(*[_addr(x) for x in xs])
     ptr = lambda x: None if x is None else C.c_void_p(_addr(x))
     _check(lib().mpt_dp_step_flat_opt(C.byref(opt), tab(g16_peers), tab(flag_peers), tab(w16_peers), ptr(w32_shard),
                                       ptr(s1_shard), ptr(s2_shard), int(n), int(R), int(rank), float(S), float(b1t), float(b2t),
-                                      C.c_void_p(_addr(flags)), _stream_ptr(stream)))
+                                      C.c_void_p(_addr(flags)), None if norm_peers is None else tab(norm_peers), ptr(clip_out),
+                                      _stream_ptr(stream)))
 
 
 class DeviceBuffer:
@@ -795,6 +817,9 @@ class DataParallelMLP:
     def step(self):
         """All replicas call this after their backward_scaled(); returns True if the step was skipped."""
         self._barrier()
+        if self.R > 1 and self.ctx.optimizer.clip_norm > 0.0:
+            self.ctx.dp_norm()          # every replica's part of the norm, then all of them visible to all
+            self._barrier()
         overflow = self.ctx.step()
         self._barrier()
         return bool(overflow)

@@ -152,7 +152,8 @@ __global__ void __launch_bounds__(kDpThreads) k_dp_step_opt(const DpPeers pp, in
                                                             float4 *__restrict__ s1p, float4 *__restrict__ s2p, size_t first,
                                                             size_t n8, float inv, const float *__restrict__ S_dev, float lr,
                                                             float mu, float b2, float eps, float wd, float b1t, float b2t,
-                                                            const float *__restrict__ betat_dev, uint32_t *flags)
+                                                            const float *__restrict__ betat_dev, uint32_t *flags,
+                                                            const float *__restrict__ coef_dev)
 {
     pdl_trigger();
     pdl_wait();
@@ -161,6 +162,7 @@ __global__ void __launch_bounds__(kDpThreads) k_dp_step_opt(const DpPeers pp, in
         if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(flags, 1u);
         return;
     }
+    const float coef = coef_dev ? *coef_dev : 1.0f;      // global-norm clipping of the mean gradient (1 = off)
     const size_t j = (size_t)blockIdx.x * kDpThreads + threadIdx.x;
     if (j >= n8) return;
     if (betat_dev) { b1t = __fmul_rn(betat_dev[0], mu); b2t = __fmul_rn(betat_dev[1], b2); }
@@ -189,7 +191,7 @@ __global__ void __launch_bounds__(kDpThreads) k_dp_step_opt(const DpPeers pp, in
 #pragma unroll
     for (int e = 0; e < 8; e++)
         opt1<KIND, WD>(s[e], wf[e >> 2][e & 3], af[e >> 2][e & 3], bf[e >> 2][e & 3], inv, lr, mu, b2, omb1, omb2, eps, wd,
-                       bc1, bc2, 1.0f, bad);
+                       bc1, bc2, coef, bad);
     uint4 h;
     h.x = f2h_bits_dp(w0.x) | (f2h_bits_dp(w0.y) << 16);
     h.y = f2h_bits_dp(w0.z) | (f2h_bits_dp(w0.w) << 16);
@@ -207,7 +209,8 @@ template <int KIND, bool WD>
 __global__ void k_dp_step_opt_tail(const DpPeers pp, int R, float *__restrict__ w32, float *__restrict__ s1p,
                                    float *__restrict__ s2p, size_t first, size_t begin, size_t count, float inv,
                                    const float *__restrict__ S_dev, float lr, float mu, float b2, float eps, float wd,
-                                   float b1t, float b2t, const float *__restrict__ betat_dev, uint32_t *flags)
+                                   float b1t, float b2t, const float *__restrict__ betat_dev, uint32_t *flags,
+                                   const float *__restrict__ coef_dev)
 {
     pdl_trigger();
     pdl_wait();
@@ -216,6 +219,7 @@ __global__ void k_dp_step_opt_tail(const DpPeers pp, int R, float *__restrict__ 
         if (threadIdx.x == 0) atomicOr(flags, 1u);
         return;
     }
+    const float coef = coef_dev ? *coef_dev : 1.0f;
     if (betat_dev) { b1t = __fmul_rn(betat_dev[0], mu); b2t = __fmul_rn(betat_dev[1], b2); }
     const float bc1 = __fsub_rn(1.0f, b1t), bc2 = __fsub_rn(1.0f, b2t);
     const float omb1 = __fsub_rn(1.0f, mu), omb2 = __fsub_rn(1.0f, b2);
@@ -225,7 +229,7 @@ __global__ void k_dp_step_opt_tail(const DpPeers pp, int R, float *__restrict__ 
         float s = h2f_bits_dp(pp.g[0][first + i]);
         for (int q = 1; q < R; q++) s = __fadd_rn(s, h2f_bits_dp(pp.g[q][first + i]));
         float w = w32[i], a = use_s1 ? s1p[i] : 0.0f, b = KIND == MPT_OPT_ADAM ? s2p[i] : 0.0f;
-        opt1<KIND, WD>(s, w, a, b, inv, lr, mu, b2, omb1, omb2, eps, wd, bc1, bc2, 1.0f, bad);
+        opt1<KIND, WD>(s, w, a, b, inv, lr, mu, b2, omb1, omb2, eps, wd, bc1, bc2, coef, bad);
         w32[i] = w;
         if (use_s1) s1p[i] = a;
         if (KIND == MPT_OPT_ADAM) s2p[i] = b;
@@ -238,18 +242,103 @@ __global__ void k_dp_step_opt_tail(const DpPeers pp, int R, float *__restrict__ 
 template <int KIND, bool WD>
 cudaError_t launch_dp_opt(const DpPeers &pp, int R, float *w32, float *s1, float *s2, size_t first, size_t count, float inv,
                           const float *S_dev, float lr, float mu, float b2, float eps, float wd, float b1t, float b2t,
-                          const float *betat_dev, uint32_t *flags, cudaStream_t st, int *n_launches)
+                          const float *betat_dev, uint32_t *flags, cudaStream_t st, int *n_launches, const float *coef_dev)
 {
     const size_t n8 = count / 8;
     if (n_launches) *n_launches = (n8 ? 1 : 0) + (n8 * 8 < count || count == 0 ? 1 : 0);
     if (n8)
         MPT_LAUNCH(k_dp_step_opt<KIND, WD>, dim3((unsigned)((n8 + kDpThreads - 1) / kDpThreads)), dim3(kDpThreads), 0, st, pp, R,
                    (float4 *)w32, (float4 *)s1, (float4 *)s2, first, n8, inv, S_dev, lr, mu, b2, eps, wd, b1t, b2t, betat_dev,
-                   flags);
+                   flags, coef_dev);
     if (n8 * 8 < count || count == 0)
         MPT_LAUNCH(k_dp_step_opt_tail<KIND, WD>, dim3(1), dim3(32), 0, st, pp, R, w32, s1, s2, first, n8 * 8, count, inv, S_dev,
-                   lr, mu, b2, eps, wd, b1t, b2t, betat_dev, flags);
+                   lr, mu, b2, eps, wd, b1t, b2t, betat_dev, flags, coef_dev);
     return cudaGetLastError();
+}
+
+// ---- global-norm clipping of the mean gradient (section 3.2): sum of squares of this replica's shard
+// of the mean unscaled gradient in double over a fixed partition (same tree as the single-GPU norm),
+// combined into one double that the replica publishes; then every replica adds all replicas' doubles
+// in ascending replica order and forms the same coefficient.
+constexpr int kDpNormParts = 592;
+
+__device__ __forceinline__ double dp_block_sum_fixed(double v, double *sh)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    const int warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    if ((threadIdx.x & 31) == 0) sh[warp] = v;
+    __syncthreads();
+    double total = 0.0;
+    if (threadIdx.x == 0)
+        for (int w = 0; w < nwarps; w++) total += sh[w];
+    return total;   // valid in thread 0
+}
+
+__global__ void __launch_bounds__(kDpThreads) k_dp_sqnorm(const DpPeers pp, int R, size_t first, size_t count, float inv,
+                                                          const float *__restrict__ S_dev, double *__restrict__ parts)
+{
+    pdl_trigger();
+    pdl_wait();
+    __shared__ double sh[kDpThreads / 32];
+    if (S_dev) inv = __fdiv_rn(1.0f, __fmul_rn(*S_dev, (float)R));
+    double acc = 0.0;
+    const size_t n8 = count / 8, stride = (size_t)gridDim.x * kDpThreads;
+    for (size_t j = (size_t)blockIdx.x * kDpThreads + threadIdx.x; j < n8; j += stride) {
+        const size_t vec = first / 8 + j;
+        float s[8];
+        for (int q = 0; q < R; q++) {
+            const uint4 g = __ldcs((const uint4 *)pp.g[q] + vec);
+            const uint32_t gw[4] = {g.x, g.y, g.z, g.w};
+#pragma unroll
+            for (int e = 0; e < 8; e++) {
+                const float x = h2f_bits_dp((e & 1) ? (gw[e >> 1] >> 16) : (gw[e >> 1] & 0xFFFFu));
+                s[e] = q == 0 ? x : __fadd_rn(s[e], x);
+            }
+        }
+#pragma unroll
+        for (int e = 0; e < 8; e++) {
+            const double v = (double)__fmul_rn(s[e], inv);
+            acc += v * v;
+        }
+    }
+    if (blockIdx.x == 0)      // the up to seven elements after the shard's last whole vector
+        for (size_t i = n8 * 8 + threadIdx.x; i < count; i += kDpThreads) {
+            float s = h2f_bits_dp(pp.g[0][first + i]);
+            for (int q = 1; q < R; q++) s = __fadd_rn(s, h2f_bits_dp(pp.g[q][first + i]));
+            const double v = (double)__fmul_rn(s, inv);
+            acc += v * v;
+        }
+    const double total = dp_block_sum_fixed(acc, sh);
+    if (threadIdx.x == 0) parts[blockIdx.x] = total;
+}
+
+__global__ void __launch_bounds__(1024) k_dp_norm_publish(const double *__restrict__ parts, int nparts, double *slot)
+{
+    pdl_trigger();
+    pdl_wait();
+    __shared__ double sh[32];
+    double acc = 0.0;
+    for (int i = threadIdx.x; i < nparts; i += 1024) acc += parts[i];
+    const double total = dp_block_sum_fixed(acc, sh);
+    if (threadIdx.x == 0) *slot = total;
+}
+
+struct DpNormPeers {
+    const double *slot[MPT_DP_MAX_REPLICAS];
+};
+
+// out[0] = coef = min(1, clip / (sqrt(total) + 1e-6)) rounded to FP32, out[1] = norm (FP32);
+// total = the replicas' shard sums added in ascending replica order.
+__global__ void k_dp_clip_coef(const DpNormPeers np, int R, float clip, float *out)
+{
+    pdl_trigger();
+    pdl_wait();
+    double total = 0.0;
+    for (int q = 0; q < R; q++) total += *(volatile const double *)np.slot[q];
+    const double norm = sqrt(total);
+    out[0] = (float)fmin(1.0, (double)clip / (norm + 1e-6));
+    out[1] = (float)norm;
 }
 
 template <bool MOM>
@@ -292,7 +381,8 @@ cudaError_t launch_dp_step(const uint16_t *const *g16, const uint32_t *const *fl
 cudaError_t launch_dp_step_opt(int kind, const uint16_t *const *g16, const uint32_t *const *flag, uint16_t *const *w16, int R,
                                float *w32_shard, float *s1_shard, float *s2_shard, size_t first, size_t count, float inv_SR,
                                const float *S_dev, float lr, float mu, float b2, float eps, float wd, float b1t, float b2t,
-                               const float *betat_dev, uint32_t *flags, cudaStream_t st, int *n_launches)
+                               const float *betat_dev, uint32_t *flags, cudaStream_t st, int *n_launches,
+                               const float *coef_dev)
 {
     DpPeers pp = {};
     for (int q = 0; q < R; q++) {
@@ -302,9 +392,9 @@ cudaError_t launch_dp_step_opt(int kind, const uint16_t *const *g16, const uint3
     }
 #define MPT_DP_OPT(KIND)                                                                                                    \
     (wd != 0.0f ? launch_dp_opt<KIND, true>(pp, R, w32_shard, s1_shard, s2_shard, first, count, inv_SR, S_dev, lr, mu, b2, eps, \
-                                            wd, b1t, b2t, betat_dev, flags, st, n_launches)                                  \
+                                            wd, b1t, b2t, betat_dev, flags, st, n_launches, coef_dev)                        \
                 : launch_dp_opt<KIND, false>(pp, R, w32_shard, s1_shard, s2_shard, first, count, inv_SR, S_dev, lr, mu, b2,   \
-                                             eps, wd, b1t, b2t, betat_dev, flags, st, n_launches))
+                                             eps, wd, b1t, b2t, betat_dev, flags, st, n_launches, coef_dev))
     switch (kind) {
         case MPT_OPT_SGD: return MPT_DP_OPT(MPT_OPT_SGD);
         case MPT_OPT_NESTEROV: return MPT_DP_OPT(MPT_OPT_NESTEROV);
@@ -313,6 +403,26 @@ cudaError_t launch_dp_step_opt(int kind, const uint16_t *const *g16, const uint3
         default: return cudaErrorInvalidValue;
     }
 #undef MPT_DP_OPT
+}
+
+cudaError_t launch_dp_sqnorm(const uint16_t *const *g16, int R, size_t first, size_t count, float inv_SR, const float *S_dev,
+                             double *parts, double *slot, cudaStream_t st)
+{
+    DpPeers pp = {};
+    for (int q = 0; q < R; q++) pp.g[q] = g16[q];
+    size_t want = (count / 8 + kDpThreads - 1) / kDpThreads;
+    const int grid = (int)(want < 1 ? 1 : (want > (size_t)kDpNormParts ? (size_t)kDpNormParts : want));
+    MPT_LAUNCH(k_dp_sqnorm, dim3(grid), dim3(kDpThreads), 0, st, pp, R, first, count, inv_SR, S_dev, parts);
+    MPT_LAUNCH(k_dp_norm_publish, dim3(1), dim3(1024), 0, st, (const double *)parts, grid, slot);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_dp_clip_coef(const double *const *slots, int R, float clip, float *out2, cudaStream_t st)
+{
+    DpNormPeers np = {};
+    for (int q = 0; q < R; q++) np.slot[q] = slots[q];
+    MPT_LAUNCH(k_dp_clip_coef, dim3(1), dim3(1), 0, st, np, R, clip, out2);
+    return cudaGetLastError();
 }
 
 }  // namespace mpt
@@ -360,12 +470,36 @@ int mpt_dp_step_flat(const uint16_t *const *g16_peers, const uint32_t *const *fl
     return e == cudaSuccess ? MPT_OK : MPT_ERR_CUDA;
 }
 
+int mpt_dp_norm_flat(const uint16_t *const *g16_peers, size_t n, int R, int rank, float S, void *scratch_dev,
+                     double *norm_slot_dev, void *cuda_stream)
+{
+    if (!g16_peers || !scratch_dev || !norm_slot_dev) return MPT_ERR_INVALID_ARG;
+    size_t lo = 0, hi = 0;
+    if (mpt_dp_shard(n, R, rank, &lo, &hi) != MPT_OK) return MPT_ERR_INVALID_ARG;
+    if (!(S > 0.0f)) return MPT_ERR_INVALID_ARG;
+    for (int q = 0; q < R; q++)
+        if (!g16_peers[q] || ((uintptr_t)g16_peers[q] & 15) != 0) return MPT_ERR_INVALID_ARG;
+    if ((((uintptr_t)scratch_dev | (uintptr_t)norm_slot_dev) & 7) != 0) return MPT_ERR_INVALID_ARG;
+    const float inv = 1.0f / (S * (float)R);
+    return launch_dp_sqnorm(g16_peers, R, lo, hi - lo, inv, nullptr, (double *)scratch_dev, norm_slot_dev,
+                            (cudaStream_t)cuda_stream) == cudaSuccess
+               ? MPT_OK
+               : MPT_ERR_CUDA;
+}
+
 int mpt_dp_step_flat_opt(const mpt_optimizer *opt, const uint16_t *const *g16_peers, const uint32_t *const *flag_peers,
                          uint16_t *const *w16_peers, float *w32_shard_dev, float *s1_shard_dev, float *s2_shard_dev, size_t n,
-                         int R, int rank, float S, float b1t, float b2t, uint32_t *flags_dev, void *cuda_stream)
+                         int R, int rank, float S, float b1t, float b2t, uint32_t *flags_dev, const double *const *norm_peers,
+                         float *clip_out_dev, void *cuda_stream)
 {
     if (!opt || !g16_peers || !flag_peers || !w16_peers || !flags_dev) return MPT_ERR_INVALID_ARG;
-    if (opt->kind < MPT_OPT_SGD || opt->kind > MPT_OPT_ADAM || opt->clip_norm != 0.0f) return MPT_ERR_INVALID_ARG;
+    if (opt->kind < MPT_OPT_SGD || opt->kind > MPT_OPT_ADAM || !(opt->clip_norm >= 0.0f)) return MPT_ERR_INVALID_ARG;
+    const bool clip = opt->clip_norm > 0.0f;
+    if (clip) {
+        if (!norm_peers || !clip_out_dev || R < 1 || R > MPT_DP_MAX_REPLICAS) return MPT_ERR_INVALID_ARG;
+        for (int q = 0; q < R; q++)
+            if (!norm_peers[q] || ((uintptr_t)norm_peers[q] & 7) != 0) return MPT_ERR_INVALID_ARG;
+    }
     size_t lo = 0, hi = 0;
     if (mpt_dp_shard(n, R, rank, &lo, &hi) != MPT_OK) return MPT_ERR_INVALID_ARG;
     if (!(S > 0.0f) || !(opt->lr == opt->lr)) return MPT_ERR_INVALID_ARG;
@@ -382,9 +516,10 @@ int mpt_dp_step_flat_opt(const mpt_optimizer *opt, const uint16_t *const *g16_pe
     cudaError_t e = cudaMemsetAsync(flags_dev + 1, 0, sizeof(uint32_t), st);
     if (e != cudaSuccess) return MPT_ERR_CUDA;
     const float inv = 1.0f / (S * (float)R);
+    if (clip && launch_dp_clip_coef(norm_peers, R, opt->clip_norm, clip_out_dev, st) != cudaSuccess) return MPT_ERR_CUDA;
     e = launch_dp_step_opt(opt->kind, g16_peers, flag_peers, w16_peers, R, w32_shard_dev, s1_shard_dev, s2_shard_dev, lo, count, inv,
                            nullptr, opt->lr, opt->momentum, opt->beta2, opt->eps, opt->weight_decay, b1t, b2t, nullptr, flags_dev, st,
-                           nullptr);
+                           nullptr, clip ? clip_out_dev : nullptr);
     return e == cudaSuccess ? MPT_OK : MPT_ERR_CUDA;
 }
 

@@ -158,6 +158,7 @@ struct mpt_ctx {
     float scale_backoff = 0.5f, scale_growth = 2.0f, scale_min = 0x1p-100f, scale_max = 0x1p120f;
     // data-parallel step (mpt_dp_attach): replica count (0 or 1: off), this replica, peer tables
     int dp_R = 0, dp_rank = 0;
+    bool dp_norm_done = false;   // mpt_dp_norm has run since the last backward pass (clipping in data-parallel mode)
     const uint16_t *dp_g16[MPT_DP_MAX_REPLICAS] = {};
     const uint32_t *dp_flag[MPT_DP_MAX_REPLICAS] = {};
     uint16_t *dp_w16[MPT_DP_MAX_REPLICAS] = {};
@@ -350,17 +351,27 @@ int do_step(mpt_ctx *c)
     CK(cudaMemsetAsync(c->status + ST_OVERFLOW_SEEN, 0, sizeof(uint32_t), c->stream), "status clear");
     cudaError_t e;
     if (c->dp_R > 1) {
-        if (c->clip > 0.0f) return fail(c, MPT_ERR_STATE, "the data-parallel step does not support global-norm clipping");
         size_t lo = 0, hi = 0;
         mpt_dp_shard(c->plan.P_pad, c->dp_R, c->dp_rank, &lo, &hi);
         int nl = 0;
+        if (c->clip > 0.0f) {
+            // every replica adds all replicas' published shard sums in replica order: same coefficient everywhere
+            if (!c->dp_norm_done)
+                return fail(c, MPT_ERR_STATE, "clipping in data-parallel mode: call mpt_dp_norm on every replica (then order the replicas) before mpt_step");
+            const double *slots[MPT_DP_MAX_REPLICAS];
+            for (int q = 0; q < c->dp_R; q++) slots[q] = (const double *)(c->dp_flag[q] + (ST_DP_NORM - ST_OVERFLOW));
+            e = launch_dp_clip_coef(slots, c->dp_R, c->clip, (float *)(c->status + ST_CLIP_COEF), c->stream);
+            c->launches++;
+            if (e != cudaSuccess) return cuda_fail(c, e, "clip launch");
+            c->dp_norm_done = false;
+        }
         {
             // bytes through this GPU's memory system: R gradients read, the shard's state, R weight copies written
             const double per_elem = 2.0 * c->dp_R + 8.0 + (c->use_momentum ? 8.0 : 0.0) + (c->state2 ? 8.0 : 0.0) + 2.0 * c->dp_R;
             ProfSpan span(c, MPT_PROF_UPDATE, per_elem * (double)(hi - lo));
             const float inv_SR = 1.0f / (c->S * (float)c->dp_R);
             const float *S_dev = (const float *)(c->status + ST_SCALE);
-            if (c->opt_kind == MPT_OPT_SGD && c->wd == 0.0f)
+            if (c->opt_kind == MPT_OPT_SGD && c->wd == 0.0f && c->clip <= 0.0f)
                 e = launch_dp_step(c->dp_g16, c->dp_flag, c->dp_w16, c->dp_R, c->master + lo, c->use_momentum ? c->mom + lo : nullptr,
                                    lo, hi - lo, inv_SR, S_dev, c->lr, c->use_momentum ? c->mu : 0.0f, c->status + ST_OVERFLOW,
                                    c->stream, &nl);
@@ -369,7 +380,8 @@ int do_step(mpt_ctx *c)
                                        c->mom ? c->mom + lo : nullptr, c->state2 ? c->state2 + lo : nullptr, lo, hi - lo, inv_SR,
                                        S_dev, c->lr, c->mu, c->beta2, c->eps, c->wd, 1.0f, 1.0f,
                                        c->opt_kind == MPT_OPT_ADAM ? (const float *)(c->status + ST_B1T) : nullptr,
-                                       c->status + ST_OVERFLOW, c->stream, &nl);
+                                       c->status + ST_OVERFLOW, c->stream, &nl,
+                                       c->clip > 0.0f ? (const float *)(c->status + ST_CLIP_COEF) : nullptr);
         }
         c->launches += nl;
         if (e != cudaSuccess) return cuda_fail(c, e, "data-parallel step launch");
@@ -948,6 +960,24 @@ int mpt_dp_attach(mpt_ctx *c, int R, int rank, const uint16_t *const *g16_peers,
     }
     c->dp_R = R;
     c->dp_rank = rank;
+    return MPT_OK;
+}
+
+int mpt_dp_norm(mpt_ctx *c)
+{
+    int r = usable(c);
+    if (r != MPT_OK) return r;
+    if (c->dp_R < 2) return fail(c, MPT_ERR_STATE, "mpt_dp_norm needs an attached data-parallel context");
+    if (c->clip <= 0.0f) return fail(c, MPT_ERR_STATE, "the context was created without gradient clipping");
+    if (!c->have_grads) return fail(c, MPT_ERR_STATE, "mpt_dp_norm needs gradients (mpt_backward_scaled or mpt_set_grad)");
+    size_t lo = 0, hi = 0;
+    mpt_dp_shard(c->plan.P_pad, c->dp_R, c->dp_rank, &lo, &hi);
+    const float inv_SR = 1.0f / (c->S * (float)c->dp_R);
+    cudaError_t e = launch_dp_sqnorm(c->dp_g16, c->dp_R, lo, hi - lo, inv_SR, (const float *)(c->status + ST_SCALE), c->norm_parts,
+                                     (double *)(c->status + ST_DP_NORM), c->stream);
+    c->launches += 2;
+    if (e != cudaSuccess) return cuda_fail(c, e, "data-parallel norm launch");
+    c->dp_norm_done = true;
     return MPT_OK;
 }
 

@@ -24,6 +24,7 @@ enum StatusWord : int {
     ST_B2T = 9,           // float: beta2^t
     ST_CLIP_COEF = 10,    // float: clipping coefficient of the last step (global-norm clipping)
     ST_GRAD_NORM = 11,    // float: norm of the unscaled gradients of the last step
+    ST_DP_NORM = 12,      // double (words 12, 13): this replica's shard of the squared norm of the mean gradient
     ST_WORDS = 16
 };
 
@@ -147,7 +148,15 @@ cudaError_t launch_dp_step(const uint16_t *const *g16, const uint32_t *const *fl
 cudaError_t launch_dp_step_opt(int kind, const uint16_t *const *g16, const uint32_t *const *flag, uint16_t *const *w16, int R,
                                float *w32_shard, float *s1_shard, float *s2_shard, size_t first, size_t count, float inv_SR,
                                const float *S_dev, float lr, float mu, float b2, float eps, float wd, float b1t, float b2t,
-                               const float *betat_dev, uint32_t *flags, cudaStream_t st, int *n_launches);
+                               const float *betat_dev, uint32_t *flags, cudaStream_t st, int *n_launches,
+                               const float *coef_dev = nullptr);
+// Clipping in the data-parallel step: this replica's shard of the sum of squares of the mean unscaled
+// gradient (double) into *slot (parts: scratch of kDpNormScratch doubles); then, once every replica
+// has published its slot, out2[0] = coefficient, out2[1] = norm from all R slots in replica order.
+static constexpr int kDpNormScratch = 592;
+cudaError_t launch_dp_sqnorm(const uint16_t *const *g16, int R, size_t first, size_t count, float inv_SR, const float *S_dev,
+                             double *parts, double *slot, cudaStream_t st);
+cudaError_t launch_dp_clip_coef(const double *const *slots, int R, float clip, float *out2, cudaStream_t st);
 // End-of-step bookkeeping on the device (one thread): dynamic loss scale (if interval > 0) and
 // Adam's running products beta^t (if adam != 0); both only move on a step that was applied.
 cudaError_t launch_post_step(uint32_t *status, int interval, float backoff, float growth, float min_S, float max_S,

@@ -185,12 +185,68 @@ def test_dp_step_other_optimizers_bit_exact(R, n, kind, wd):
         assert f_dev[q].cpu().numpy().tolist() == [0, 0]
 
 
-def test_dp_step_opt_rejects_clipping():
+@pytest.mark.parametrize("kind,R,n", [(0, 2, 4099), (2, 4, (1 << 18) + 5), (3, 3, 70001), (1, 8, 12345)])
+def test_dp_clipped_step_bit_exact(kind, R, n):
+    """Global-norm clipping of the mean gradient: every emulated replica publishes its shard's sum
+    of squares, then each forms the coefficient from all of them.  Norm within 1e-12 of the
+    oracle's sequential double sum, coefficient the same FP32 bits on every replica and equal to
+    the oracle's, update bit for bit."""
+    b = _binding()
+    S, lr, mu, b2, eps, wd, clip = 256.0, 0.01, 0.9, 0.999, 1e-8, 1e-3, 0.01
+    opt = b.Optimizer(kind, lr, mu, b2, eps, wd, clip)
+    gs, w, _ = _inputs(n, R, seed=n + R)
+    rng = np.random.default_rng(kind)
+    s1 = np.abs(0.1 * rng.standard_normal(n)).astype(np.float32)
+    s2 = np.abs(0.01 * rng.standard_normal(n)).astype(np.float32)
+    b1t, b2t = np.float32(0.81), np.float32(0.998)
+    npad = n + 8
+    g_dev = [torch.zeros(npad, dtype=torch.int16, device="cuda") for _ in range(R)]
+    h_dev = [torch.full((npad,), 0x1234, dtype=torch.int16, device="cuda") for _ in range(R)]
+    f_dev = [torch.zeros(2, dtype=torch.int32, device="cuda") for _ in range(R)]
+    slots = [torch.full((1,), -1.0, dtype=torch.float64, device="cuda") for _ in range(R)]
+    outs = [torch.zeros(2, dtype=torch.float32, device="cuda") for _ in range(R)]
+    scratch = torch.zeros(b.DP_NORM_SCRATCH_BYTES // 8, dtype=torch.float64, device="cuda")
+    for q in range(R):
+        g_dev[q][:n] = dev(gs[q].view(np.uint16))
+    full = [torch.zeros(npad, dtype=torch.float32, device="cuda") for _ in range(3)]
+    for t, a_ in zip(full, (w, s1, s2)):
+        t[:n] = dev(a_)
+    for q in range(R):                                   # phase 1 on every replica
+        b.mpt_dp_norm_flat(g_dev, n, R, q, S, scratch, slots[q])
+    torch.cuda.synchronize()                             # "order the replicas"
+    for q in range(R):                                   # phase 2
+        lo, hi = b.mpt_dp_shard(n, R, q)
+        b.mpt_dp_step_flat_opt(opt, g_dev, f_dev, h_dev, full[0][lo:], full[1][lo:], full[2][lo:] if kind == 3 else None,
+                               n, R, q, S, float(b1t), float(b2t), f_dev[q], norm_peers=slots, clip_out=outs[q])
+    torch.cuda.synchronize()
+    glist = [g.view(np.uint16) for g in gs]
+    total_ref = mpo.dp_grad_sqnorm(glist, S)
+    total_dev = float(sum(float(x.item()) for x in slots))
+    assert abs(total_dev - total_ref) <= 1e-12 * total_ref
+    coef_ref = mpo.clip_coef(total_ref, clip)
+    assert 0.0 < float(coef_ref) < 1.0                   # the bound bites in this test
+    for q in range(R):
+        c, nrm = outs[q].cpu().numpy()
+        assert np.float32(c).view(np.uint32) == np.float32(coef_ref).view(np.uint32)
+        assert abs(float(nrm) - np.sqrt(total_ref)) <= 1e-6 * np.sqrt(total_ref)
+    rw, r1, r2, rh = w.copy(), s1.copy(), s2.copy(), np.zeros(n, np.uint16)
+    use_s1 = kind != 0 or mu != 0.0
+    mpo.dp_update_apply_clip(kind, glist, rw, r1 if use_s1 else None, r2 if kind == 3 else None, rh, S, coef_ref, lr, mu, b2, eps,
+                             wd, np.float32(1.0) - b1t, np.float32(1.0) - b2t)
+    assert np.array_equal(full[0][:n].cpu().numpy().view(np.uint32), rw.view(np.uint32))
+    assert np.array_equal(full[1][:n].cpu().numpy().view(np.uint32), r1.view(np.uint32))
+    assert np.array_equal(full[2][:n].cpu().numpy().view(np.uint32), (r2 if kind == 3 else s2).view(np.uint32))
+    for q in range(R):
+        assert np.array_equal(host_u16(h_dev[q][:n]), rh)
+        assert np.all(host_u16(h_dev[q][n:]) == 0x1234)
+
+
+def test_dp_step_opt_clipping_needs_the_norm_slots():
     b = _binding()
     t = torch.zeros(64, dtype=torch.int16, device="cuda")
     f = torch.zeros(2, dtype=torch.int32, device="cuda")
     w32 = torch.zeros(64, dtype=torch.float32, device="cuda")
-    with pytest.raises(b.MptError):
+    with pytest.raises(b.MptError):                      # clip_norm > 0 without norm_peers / clip_out
         b.mpt_dp_step_flat_opt(b.Optimizer(2, 0.1, 0.0, 0.0, 1e-8, 0.0, 1.0), [t, t], [f, f], [t, t], w32, w32, None, 64, 2, 0,
                                1.0, 1.0, 1.0, f)
 
@@ -287,7 +343,7 @@ def _mlp_batch(t, q):
     return x, y
 
 
-def _mlp_replica_main(rank, R, port, out_dir, dynamic=False, opt_kind=0):
+def _mlp_replica_main(rank, R, port, out_dir, dynamic=False, opt_kind=0, clip=0.0):
     import datetime
     import torch as th
     import torch.distributed as dist
@@ -296,7 +352,7 @@ def _mlp_replica_main(rank, R, port, out_dir, dynamic=False, opt_kind=0):
     dist.init_process_group("gloo", init_method="tcp://127.0.0.1:%d" % port, rank=rank, world_size=R,
                             timeout=datetime.timedelta(seconds=90))
     try:
-        opt = b.Optimizer(opt_kind, _MLP["lr"], _MLP["mu"], 0.999, 1e-8, 0.001, 0.0) if opt_kind else None
+        opt = b.Optimizer(opt_kind, _MLP["lr"], _MLP["mu"], 0.999, 1e-8, 0.001, clip) if (opt_kind or clip) else None
         dp = b.DataParallelMLP(_MLP_LAYERS, _MLP["S"], _MLP["lr"], _MLP["mu"], max_batch=_MLP["batch"], optimizer=opt)
         L = len(_MLP_LAYERS)
         for l, w in enumerate(_mlp_masters()):
@@ -320,6 +376,8 @@ def _mlp_replica_main(rank, R, port, out_dir, dynamic=False, opt_kind=0):
             for l in range(L):
                 rec["e2e_g16_%d_%d" % (t, l)] = dp.ctx.get_tensor(b.T_GRAD16, l)
             rec["e2e_skip_%d" % t] = np.array(dp.step())
+            if clip > 0.0:
+                rec["e2e_norm_coef_%d" % t] = np.array(dp.ctx.get_grad_norm(), dtype=np.float32)
             for l in range(L):
                 rec["e2e_w16_%d_%d" % (t, l)] = dp.ctx.get_tensor(b.T_W16, l)
         rec["launches"] = np.array(dp.ctx.launch_count())
@@ -465,3 +523,50 @@ def test_dp_mlp_two_processes_adagrad_adam(tmp_path, kind):
             for l in range(L):
                 want16 = ora.replicas[0].w16[l]
                 assert np.array_equal(rec[q]["e2e_w16_%d_%d" % (t, l)].reshape(want16.shape), want16), (t, l, q)
+
+
+@pytest.mark.timeout(300)
+def test_dp_mlp_two_processes_clipped(tmp_path):
+    """Two attached contexts with global-norm clipping (section 3.2) of the mean gradient: every
+    replica publishes its shard's part of the norm (mpt_dp_norm), the replicas are ordered, every
+    replica forms the same coefficient in mpt_step.  Coefficient bits and FP16 weights of both
+    replicas against the oracle's replicas, through a skipped step; and mpt_step without the norm
+    call is refused."""
+    import torch.multiprocessing as mp
+    from oracle.dp import OracleDataParallelMLP
+    R, kind, clip = 2, 2, 0.02
+    mp.spawn(_mlp_replica_main, args=(R, _free_port(), str(tmp_path), False, kind, clip), nprocs=R, join=True)
+    rec = [np.load(os.path.join(str(tmp_path), "m%d.npz" % q)) for q in range(R)]
+    L = len(_MLP_LAYERS)
+    ora = OracleDataParallelMLP(_MLP_LAYERS, _MLP["S"], _MLP["lr"], _MLP["mu"], R)
+    ora.set_optimizer(kind, _MLP["lr"], _MLP["mu"], b2=0.999, eps=1e-8, wd=0.001, clip=clip)
+    for l, w in enumerate(_mlp_masters()):
+        ora.set_master(l, w)
+    for t in range(_MLP["inj_steps"]):
+        for q in range(R):
+            for l in range(L):
+                ora.set_grad(q, l, _mlp_injected_grad(t, q, l).view(np.uint16))
+        skipped = ora.step()
+        assert skipped == (1 if t == 1 else 0)
+        for q in range(R):
+            assert bool(rec[q]["inj_skip_%d" % t]) == bool(skipped)
+            for l in range(L):
+                want16 = ora.replicas[0].w16[l]
+                assert np.array_equal(rec[q]["inj_w16_%d_%d" % (t, l)].reshape(want16.shape), want16), (t, l, q)
+    bit = False
+    for t in range(_MLP["e2e_steps"]):
+        xs, ys = zip(*[_mlp_batch(t, q) for q in range(R)])
+        ora.forward_backward(list(xs), list(ys))
+        for q in range(R):
+            for l in range(L):
+                ora.set_grad(q, l, rec[q]["e2e_g16_%d_%d" % (t, l)])
+        skipped = ora.step()
+        coef = np.float32(ora.replicas[0].last_coef)
+        bit |= float(coef) < 1.0
+        for q in range(R):
+            assert bool(rec[q]["e2e_skip_%d" % t]) == bool(skipped)
+            assert np.float32(rec[q]["e2e_norm_coef_%d" % t][1]).view(np.uint32) == coef.view(np.uint32), (t, q)
+            for l in range(L):
+                want16 = ora.replicas[0].w16[l]
+                assert np.array_equal(rec[q]["e2e_w16_%d_%d" % (t, l)].reshape(want16.shape), want16), (t, l, q)
+    assert bit                                           # the bound was active in at least one iteration
