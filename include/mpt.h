@@ -80,6 +80,15 @@ extern "C" {
                                   fed by one stream of A, epilogue not overlapped); same alignment
                                   rules.  Moves about a quarter fewer operand bytes and is not faster;
                                   never picked automatically */
+#define MPT_GEMM_FORCE_SPLIT2 32u /* require the in-cluster split kernel: a cluster of two CTA pairs per
+                                  256x256 tile, each pair running half of the contraction, the two FP32
+                                  accumulators added through distributed shared memory (parts in ascending
+                                  order, one rounding per add) before the one rounding to FP16.  Same
+                                  alignment rules; K >= 128.  Picked automatically for outputs of at most
+                                  32 tiles with K >= 2048 (section 4.5's projection product) */
+#define MPT_GEMM_FORCE_SPLIT4 64u /* the same with four CTA pairs per tile (a cluster of eight CTAs), each
+                                  running a quarter of the contraction; K >= 256.  Picked automatically
+                                  for outputs of at most 12 tiles with K >= 4096 */
 
 /* mpt_get_tensor kinds */
 #define MPT_T_W16 0        /* FP16 working weights   [out, in]            */

@@ -21,6 +21,7 @@ ERR = {-1: "MPT_ERR_INVALID_ARG", -2: "MPT_ERR_SHAPE", -3: "MPT_ERR_STATE", -4: 
        -5: "MPT_ERR_CUDA", -6: "MPT_ERR_TIMEOUT", -7: "MPT_ERR_INTERNAL"}
 OP_FWD, OP_DGRAD, OP_WGRAD = 0, 1, 2
 GEMM_RELU, GEMM_FORCE_SIMT, GEMM_FORCE_TC, GEMM_FORCE_PAIR, GEMM_FORCE_PAIR512 = 1, 2, 4, 8, 16
+GEMM_FORCE_SPLIT2, GEMM_FORCE_SPLIT4 = 32, 64
 T_W16, T_GRAD16, T_ACT16, T_DACT16, T_MOMENTUM32, T_MASTER32, T_STATE2_32 = range(7)
 OPT_SGD, OPT_NESTEROV, OPT_ADAGRAD, OPT_ADAM = 0, 1, 2, 3
 

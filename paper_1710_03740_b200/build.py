@@ -19,7 +19,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmpt.so")
-SOURCES = ["update.cu", "softmax_ce.cu", "gemm_simt.cu", "gemm_tc.cu", "gemm_tc2.cu", "gemm_tc3.cu", "lstm.cu", "lstm_api.cu", "lstm_train.cu", "dp_exchange.cu", "wait_selftest.cu", "clock_probe.cu", "mpt_api.cu"]
+SOURCES = ["update.cu", "softmax_ce.cu", "gemm_simt.cu", "gemm_tc.cu", "gemm_tc2.cu", "gemm_tc3.cu", "gemm_tc4.cu", "lstm.cu", "lstm_api.cu", "lstm_train.cu", "dp_exchange.cu", "wait_selftest.cu", "clock_probe.cu", "mpt_api.cu"]
 HEADERS = [os.path.join(CSRC, "mpt_common.cuh"), os.path.join(CSRC, "tc_ptx.cuh"), os.path.join(CSRC, "update_math.cuh"),
            os.path.join(ROOT, "include", "mpt.h")]
 
@@ -61,13 +61,16 @@ def build(force=False, verbose=False):
 
 
 def build_trace():
-    """libmpt_trace.so: every object of the normal build except gemm_tc2, which is recompiled with
+    """libmpt_trace.so: every object of the normal build except gemm_tc2 and gemm_tc4, which are recompiled with
     -DMPT_GEMM_TRACE."""
     build()
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    o = os.path.join(CSRC, "gemm_tc2_trace.o")
-    subprocess.run([nvcc] + NVCC_FLAGS + ["-DMPT_GEMM_TRACE", "-c", os.path.join(CSRC, "gemm_tc2.cu"), "-o", o], check=True)
-    objs = [os.path.join(CSRC, s.replace(".cu", ".o")) for s in SOURCES if s != "gemm_tc2.cu"] + [o]
+    traced = ["gemm_tc2.cu", "gemm_tc4.cu"]
+    objs = [os.path.join(CSRC, s.replace(".cu", ".o")) for s in SOURCES if s not in traced]
+    for src in traced:
+        o = os.path.join(CSRC, src.replace(".cu", "_trace.o"))
+        subprocess.run([nvcc] + NVCC_FLAGS + ["-DMPT_GEMM_TRACE", "-c", os.path.join(CSRC, src), "-o", o], check=True)
+        objs.append(o)
     lib = os.path.join(HERE, "libmpt_trace.so")
     subprocess.run([nvcc, "-shared", "-cudart", "static", "-gencode", "arch=compute_100a,code=sm_100a", "-o", lib] + objs, check=True)
     return lib

@@ -260,7 +260,11 @@ int gemm(mpt_ctx *c, int op, int M, int N, int K, const uint16_t *A, int lda, co
     cudaError_t e;
     ProfSpan span(c, MPT_PROF_GEMM, 2.0 * M * N * K);
     if (!c->disable_tc && tc_gemm_supported(op, M, N, K, A, lda, B, ldb, C, ldc, mask, ldmask)) {
-        if (!c->disable_pair && tc_choose_pair(M, N, K, c->plan.splitk_bytes, nullptr))
+        const int split = c->disable_pair ? 0 : tc4_split_for(M, N, K);
+        if (split)
+            e = launch_gemm_tc4(op, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite, c->status + ST_KERNEL_ERR,
+                                c->stream, split);
+        else if (!c->disable_pair && tc_choose_pair(M, N, K, c->plan.splitk_bytes, nullptr))
             e = launch_gemm_tc2(op, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite,
                                 c->status + ST_KERNEL_ERR, c->stream, nullptr, c->splitk_ws, c->plan.splitk_bytes);
         else
@@ -446,9 +450,17 @@ int dispatch_gemm(int op, int M, int N, int K, const uint16_t *A, int lda, const
     if (lda < a_cols || ldb < b_cols || ldc < N || (mask && ldmask < N)) return MPT_ERR_SHAPE;
     const bool relu = (flags & MPT_GEMM_RELU) != 0;
     bool tc_ok = K > 0 && tc_gemm_supported(op, M, N, K, A, lda, B, ldb, C, ldc, mask, ldmask);
-    if (((flags & (MPT_GEMM_FORCE_TC | MPT_GEMM_FORCE_PAIR | MPT_GEMM_FORCE_PAIR512)) || lstm) && !tc_ok) return MPT_ERR_SHAPE;
+    constexpr unsigned kForceSplit = MPT_GEMM_FORCE_SPLIT2 | MPT_GEMM_FORCE_SPLIT4;
+    if (((flags & (MPT_GEMM_FORCE_TC | MPT_GEMM_FORCE_PAIR | MPT_GEMM_FORCE_PAIR512 | kForceSplit)) || lstm) && !tc_ok)
+        return MPT_ERR_SHAPE;
+    if ((flags & kForceSplit) && (lstm || K < ((flags & MPT_GEMM_FORCE_SPLIT4) ? 256 : 128))) return MPT_ERR_SHAPE;
+    const unsigned forced = flags & (MPT_GEMM_FORCE_SIMT | MPT_GEMM_FORCE_TC | MPT_GEMM_FORCE_PAIR | MPT_GEMM_FORCE_PAIR512 | kForceSplit);
+    const int auto_split = (tc_ok && !lstm && !forced) ? tc4_split_for(M, N, K) : 0;
     cudaError_t e;
-    if (tc_ok && !lstm && (flags & MPT_GEMM_FORCE_PAIR512)) {
+    if (tc_ok && ((flags & kForceSplit) || auto_split)) {
+        const int split = (flags & MPT_GEMM_FORCE_SPLIT4) ? 4 : ((flags & MPT_GEMM_FORCE_SPLIT2) ? 2 : auto_split);
+        e = launch_gemm_tc4(op, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite_flag, status_dev, st, split);
+    } else if (tc_ok && !lstm && (flags & MPT_GEMM_FORCE_PAIR512)) {
         e = launch_gemm_tc3(op, M, N, K, A, lda, B, ldb, C, ldc, relu, mask, ldmask, nonfinite_flag, status_dev, st);
     } else if (tc_ok && !(flags & MPT_GEMM_FORCE_SIMT)) {
         const size_t ws_ok = (splitk_ws_dev && (((uintptr_t)splitk_ws_dev) & 15) == 0) ? splitk_ws_bytes : 0;
@@ -998,6 +1010,7 @@ int mpt_gemm_workspace_bytes(int op, int M, int N, int K, size_t *bytes_out)
     if (M < 0 || N < 0 || K < 0) return MPT_ERR_SHAPE;
     *bytes_out = 0;
     if (M == 0 || N == 0 || K == 0) return MPT_OK;
+    if (tc4_split_for(M, N, K)) return MPT_OK;       // the in-cluster split needs no scratch
     tc_choose_pair(M, N, K, (size_t)256 << 20, bytes_out);
     return MPT_OK;
 }

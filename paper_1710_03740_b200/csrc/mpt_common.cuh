@@ -36,7 +36,8 @@ enum KernelErr : uint32_t {
     KERR_WAIT_ACC = 3,    // epilogue gave up waiting for the accumulator
     KERR_WAIT_ACC_FREE = 4, // MMA issuer gave up waiting for a drained accumulator
     KERR_TMEM_ALLOC = 5,
-    KERR_WAIT_SELFTEST = 6  // the self-test's wait on a barrier nobody signals ran out, as intended
+    KERR_WAIT_SELFTEST = 6, // the self-test's wait on a barrier nobody signals ran out, as intended
+    KERR_WAIT_PARTIAL = 7   // a warp gave up waiting for another CTA pair's part of a split contraction
 };
 
 // Kernel attributes (opt-in shared memory size, cluster occupancy) are per device: launchers
@@ -207,6 +208,13 @@ cudaError_t launch_splitk_reduce(const float *partial, int split_k, int M, int N
 cudaError_t launch_gemm_tc3(int op, int M, int N, int K, const uint16_t *A, int lda, const uint16_t *B, int ldb,
                             uint16_t *C, int ldc, bool relu, const uint16_t *mask, int ldmask,
                             uint32_t *nonfinite_flag, uint32_t *status, cudaStream_t st);
+// In-cluster split (gemm_tc4.cu): a cluster of `split` CTA pairs (2 or 4) per 256x256 tile, each pair
+// running 1/split of the contraction, parts added through distributed shared memory; no scratch, one
+// launch.  tc4_split_for: the split this kernel would use for a shape, 0 when it is not the kernel for it.
+int tc4_split_for(int M, int N, int K);
+cudaError_t launch_gemm_tc4(int op, int M, int N, int K, const uint16_t *A, int lda, const uint16_t *B, int ldb,
+                            uint16_t *C, int ldc, bool relu, const uint16_t *mask, int ldmask,
+                            uint32_t *nonfinite_flag, uint32_t *status, cudaStream_t st, int split);
 size_t tc2_tail_ws_bytes(int M, int N, int K);
 // Split factor, scratch need (FP32 parts) and modelled cost
 // of the pair kernel for an output with few tiles and a long contraction; split 1 = no split.

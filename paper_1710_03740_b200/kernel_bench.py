@@ -313,7 +313,7 @@ def main():
     g.add_argument("--no-workspace", action="store_true", help="do not offer a split-K scratch buffer")
     g.add_argument("--trace", action="store_true",
                    help="per-cluster main-loop cycles from the instrumented build (python -m paper_1710_03740_b200.build --trace)")
-    g.add_argument("--kernel", default="auto", choices=["auto", "tc", "pair", "pair512"],
+    g.add_argument("--kernel", default="auto", choices=["auto", "tc", "pair", "pair512", "split2", "split4"],
                    help="auto: the library's choice; tc: single-CTA 128x256 tiles; pair: cta_group::2 256x256 tiles")
     u = sub.add_parser("update")
     u.add_argument("--params", type=int, default=150994944)
@@ -353,7 +353,8 @@ def main():
                   else inputs.GEMM_SWEEP + [inputs.LSTM_GATE, inputs.LSTM_PROJ])
         for (M, N, K) in shapes:
             for op in args.op:
-                flags = {"auto": 0, "tc": mpt.GEMM_FORCE_TC, "pair": mpt.GEMM_FORCE_PAIR, "pair512": mpt.GEMM_FORCE_PAIR512}[args.kernel]
+                flags = {"auto": 0, "tc": mpt.GEMM_FORCE_TC, "pair": mpt.GEMM_FORCE_PAIR, "pair512": mpt.GEMM_FORCE_PAIR512,
+                         "split2": mpt.GEMM_FORCE_SPLIT2, "split4": mpt.GEMM_FORCE_SPLIT4}[args.kernel]
                 res = bench_gemm(M, N, K, op, args.iters, flags, not args.no_workspace)
                 res["kernel_choice"] = args.kernel
                 print(json.dumps(res), flush=True)

@@ -37,8 +37,8 @@ def run_gemm(op, A, B, M, N, K, flags=0, mask=None, pad=0, want_flag=False, work
     status = torch.zeros(4, dtype=torch.int32, device="cuda")
     if workspace:
         nbytes = b.mpt_gemm_workspace_bytes(op, M, N, K)
-        if nbytes == 0:
-            pytest.skip("the library does not split this shape")
+        if nbytes == 0 and not flags & (b.GEMM_FORCE_TC | b.GEMM_FORCE_PAIR):
+            pytest.skip("the library's own choice needs no scratch for this shape")
         # room for any split either kernel may choose (the need reported is that of the automatic choice)
         nbytes = max(nbytes, 9 * M * ((N + 31) // 32 * 32) * 4)
         ws = torch.full((nbytes // 4,), float("nan"), dtype=torch.float32, device="cuda")
@@ -95,7 +95,8 @@ _ORACLE_CACHE = {}
 
 def _check_tc(op, M, N, K, flags=0, mask=None, seed=21, scale=None, want_flag=False, kernel="tc", workspace=False):
     from paper_1710_03740_b200 import binding as b
-    force = {"pair": b.GEMM_FORCE_PAIR, "tc": b.GEMM_FORCE_TC, "auto": 0, "pair512": b.GEMM_FORCE_PAIR512}[kernel]
+    force = {"pair": b.GEMM_FORCE_PAIR, "tc": b.GEMM_FORCE_TC, "auto": 0, "pair512": b.GEMM_FORCE_PAIR512,
+             "split2": b.GEMM_FORCE_SPLIT2, "split4": b.GEMM_FORCE_SPLIT4}[kernel]
     sa = sb = scale
     key = (op, M, N, K, seed, scale, bool(flags & b.GEMM_RELU))
     if mask is None and key in _ORACLE_CACHE:        # the oracle is slow: keep its answer for repeated inputs
@@ -192,6 +193,50 @@ def test_pair512_many_tiles_halves_relu_mask_flag(op):
     assert flag == 0
 
 
+CLUSTER_SPLIT_SHAPES = [(256, 256, 256), (256, 256, 448), (512, 768, 1024), (392, 560, 328), (264, 264, 2056),
+                        (64, 16, 512), (8, 8, 256), (1024, 1024, 4096)]
+
+
+@pytest.mark.parametrize("kernel", ["split2", "split4"])
+@pytest.mark.parametrize("op", [0, 1, 2])
+@pytest.mark.parametrize("M,N,K", CLUSTER_SPLIT_SHAPES)
+def test_cluster_split_gemm_parity(op, M, N, K, kernel):
+    """In-cluster split of the contraction (2 or 4 CTA pairs per tile, parts added through distributed
+    shared memory): one tile and several, parts of unequal length (7, 6, 33 k-blocks), ragged M, N and
+    K, shapes smaller than a tile, and more clusters than the GPU holds at once (16 tiles of 8 CTAs)."""
+    _check_tc(op, M, N, K, kernel=kernel)
+
+
+@pytest.mark.parametrize("kernel", ["split2", "split4"])
+@pytest.mark.parametrize("op", [0, 1, 2])
+def test_cluster_split_relu_mask_flag_and_rerun(op, kernel):
+    from paper_1710_03740_b200 import binding as b
+    M, N, K = 520, 776, 1352
+    got, _, _, _ = _check_tc(op, M, N, K, kernel=kernel)
+    again, _, _, _ = _check_tc(op, M, N, K, kernel=kernel)
+    assert np.array_equal(got, again)
+    _check_tc(op, M, N, K, flags=b.GEMM_RELU, kernel=kernel)
+    mask = np.random.default_rng(10).standard_normal((M, N)).astype(np.float16)
+    _check_tc(op, M, N, K, mask=mask, kernel=kernel)
+    _, ref, flag, _ = _check_tc(op, M, N, K, scale=30.0, want_flag=True, kernel=kernel)
+    assert flag == int(((ref & 0x7FFF) >= 0x7C00).any()) == 1
+    _, _, flag, _ = _check_tc(op, M, N, K, want_flag=True, kernel=kernel)
+    assert flag == 0
+
+
+def test_cluster_split_is_the_automatic_choice_for_the_projection_shape():
+    """Section 4.5's projection product (2048 x 1024 x 8192: 32 tiles, 128 k-blocks): the library picks
+    the in-cluster split by itself, needs no scratch for it, and gives the bits of the forced kernel."""
+    from paper_1710_03740_b200 import binding as b
+    M, N, K = 2048, 1024, 8192
+    assert b.mpt_gemm_workspace_bytes(0, M, N, K) == 0
+    auto, _, _, _ = _check_tc(0, M, N, K, seed=5, kernel="auto")
+    forced, _, _, _ = _check_tc(0, M, N, K, seed=5, kernel="split2")
+    assert np.array_equal(auto, forced)
+    with pytest.raises(b.MptError):          # a part must have at least one k-block
+        _check_tc(0, 256, 256, 64, kernel="split2")
+
+
 @pytest.mark.parametrize("kernel", ["tc", "pair"])
 @pytest.mark.parametrize("op", [0, 1, 2])
 def test_tc_gemm_run_to_run_identical(op, kernel):
@@ -223,8 +268,8 @@ def test_split_k_parity_and_determinism(op, M, N, K):
     added in a fixed order by a second kernel.  Same acceptance rule; identical bits on a rerun;
     ReLU, mask and the overflow flag go through the reduce kernel."""
     from paper_1710_03740_b200 import binding as b
-    if (M, N, K) == (512, 256, 4096):
-        assert b.mpt_gemm_workspace_bytes(op, M, N, K) > 0      # the canonical few-tiles / long-K case must split
+    if (M, N, K) == (136, 96, 8192):
+        assert b.mpt_gemm_workspace_bytes(op, M, N, K) > 0      # few tiles, long K, too small for a CTA pair: must split
     got, ref, _, _ = _check_tc(op, M, N, K, workspace=True)
     again, _, _, _ = _check_tc(op, M, N, K, workspace=True)
     assert np.array_equal(got, again)
@@ -243,13 +288,12 @@ def test_pair_kernel_split_k(op, M, N, K):
     rule; identical bits on reruns; ReLU, mask and the overflow flag go through the reduce kernel; a
     scratch full of NaN bits is fine."""
     from paper_1710_03740_b200 import binding as b
-    assert b.mpt_gemm_workspace_bytes(op, M, N, K) > 0
     big = (M, N, K) == (2048, 1024, 8192)
     got, ref, _, _ = _check_tc(op, M, N, K, workspace=True, kernel="pair")
     for _ in range(3):
         again, _, _, _ = _check_tc(op, M, N, K, workspace=True, kernel="pair")
         assert np.array_equal(got, again)
-    auto, _, _, _ = _check_tc(op, M, N, K, workspace=True, kernel="auto")
+    _check_tc(op, M, N, K, kernel="auto")        # the library's own choice here is the in-cluster split: no scratch
     if not big:
         _check_tc(op, M, N, K, flags=b.GEMM_RELU, workspace=True, kernel="pair")
         mask = np.random.default_rng(8).standard_normal((M, N)).astype(np.float16)
