@@ -74,8 +74,9 @@ extern "C" {
                                   MPT_ERR_SHAPE if the operands do not meet its alignment rules */
 #define MPT_GEMM_FORCE_PAIR 8u /* require the CTA-pair tcgen05 kernel (cta_group::2, 256x256 tiles);
                                   same alignment rules.  Without a FORCE flag the library picks the
-                                  pair kernel when the output has at least 48 tiles of 256x256,
-                                  else the single-CTA one */
+                                  pair kernel when the output has more 256x256 tiles than the 74 CTA
+                                  pairs run at once (or at least 48 with K >= 16384), the in-cluster
+                                  split for few tiles and a long K (below), else the single-CTA one */
 #define MPT_GEMM_FORCE_PAIR512 16u /* require the CTA-pair kernel with 256x512 tiles (two accumulators
                                   fed by one stream of A, epilogue not overlapped); same alignment
                                   rules.  Moves about a quarter fewer operand bytes and is not faster;

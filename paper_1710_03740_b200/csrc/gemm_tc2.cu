@@ -521,12 +521,15 @@ static cudaError_t launch_variant(const CUtensorMap &ta, const CUtensorMap &tb, 
 
 bool tc2_gemm_preferred(int M, int N, int K)
 {
-    // measured on B200 with launches replayed from a CUDA graph: from about 48 tiles of 256x256
-    // (two thirds of the 74 clusters) the pair kernel wins; below that the single-CTA kernel
-    // with narrower tiles or a split contraction has more parallelism
-    (void)K;
+    // Measured on B200 with launches replayed from a CUDA graph.  When all tiles run in one round either
+    // way (at most 74 tiles of 256x256 = 148 of 128x256) both kernels spend the same time per k-block
+    // (0.32 us) and the single-CTA kernel starts and ends about 1.7 us sooner (no cluster to place, no
+    // paired allocation): 2048^3 16.4 against 18.2 us, 2048x2048x4096 26.7 against 28.3, 72 tiles with
+    // K = 2048 18.8 against 19.3.  With more tiles than that the pair kernel wins (4096^3 100 against
+    // 116 us: a third fewer operand bytes from L2, epilogues hidden behind the next tile).
     const long tiles = (long)((M + 255) / 256) * ((N + 255) / 256);
-    return M >= 256 && N >= 256 && tiles >= 48;
+    const long nkb = (K + 63) / 64;
+    return M >= 256 && N >= 256 && (tiles > 74 || (tiles >= 48 && nkb >= 256));
 }
 
 // Scratch the pair kernel would like for the split tail of a large product: one 256x256 FP32 block

@@ -145,6 +145,36 @@ __device__ __forceinline__ uint64_t desc_join(uint32_t lo, uint32_t hi)
     return d;
 }
 
+// Rounds 32 FP32 sums to 16 words of two FP16 values each (element 2i in the low half), with the
+// optional ReLU fused into the conversion: cvt.rn.relu turns a negative result into +0 and keeps NaN,
+// which equals x > 0 ? x : +0 on the FP32 sum followed by the rounding (rounding is monotonic and
+// keeps the sign).  One instruction per two elements.
+__device__ __forceinline__ void round_pack32(const uint32_t (&r)[32], bool relu, uint32_t (&w)[16])
+{
+    if (relu) {
+#pragma unroll
+        for (int i = 0; i < 16; i++)
+            asm("cvt.rn.relu.f16x2.f32 %0, %1, %2;" : "=r"(w[i]) : "f"(__uint_as_float(r[2 * i + 1])), "f"(__uint_as_float(r[2 * i])));
+    } else {
+#pragma unroll
+        for (int i = 0; i < 16; i++)
+            asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(w[i]) : "f"(__uint_as_float(r[2 * i + 1])), "f"(__uint_as_float(r[2 * i])));
+    }
+}
+// ReLU-derivative mask on a word of two FP16 results: keep a half where the stored FP16 activation
+// in the same half of mw is > 0 (sign clear, non-zero, not NaN).
+__device__ __forceinline__ uint32_t mask_pair(uint32_t w, uint32_t mw)
+{
+    const uint32_t lo = mw & 0xFFFFu, hi = mw >> 16;
+    if (!(lo != 0 && lo <= 0x7C00u)) w &= 0xFFFF0000u;
+    if (!(hi != 0 && hi <= 0x7C00u)) w &= 0x0000FFFFu;
+    return w;
+}
+// inf/NaN vote on words of two FP16 values: adding 0x0400 to an exponent field carries into bit 15
+// of its half exactly when the field is all ones; acc collects the carries (test acc & 0x80008000).
+__device__ __forceinline__ void nonfinite_acc(uint32_t w, uint32_t &acc) { acc |= (w & 0x7C007C00u) + 0x04000400u; }
+__device__ __forceinline__ bool nonfinite_any(uint32_t acc) { return (acc & 0x80008000u) != 0; }
+
 // Epilogue of one thread for 32 consecutive accumulator columns of its output row:
 // optional ReLU on the FP32 sum, round to FP16, optional ReLU-derivative mask taken from a
 // stored FP16 activation (keep where it is > 0), inf/NaN vote, 128-bit stores where the
@@ -152,45 +182,35 @@ __device__ __forceinline__ uint64_t desc_join(uint32_t lo, uint32_t hi)
 __device__ __forceinline__ void epilogue_store32(const uint32_t (&r)[32], uint16_t *crow, const uint16_t *mrow, int col0,
                                                  int N, bool relu, bool &bad)
 {
+    uint32_t w[16], acc = 0;
+    round_pack32(r, relu, w);
 #pragma unroll
     for (int g8 = 0; g8 < 4; g8++) {
         const int col = col0 + g8 * 8;
-        uint32_t h[8];
-#pragma unroll
-        for (int e = 0; e < 8; e++) {
-            float s = __uint_as_float(r[g8 * 8 + e]);
-            if (relu) s = (s > 0.0f || s != s) ? s : 0.0f;
-            h[e] = (uint32_t)__half_as_ushort(__float2half_rn(s));
-        }
         if (col + 8 <= N) {
             if (mrow) {
-                uint4 mk = *(const uint4 *)(mrow + col);
-                uint32_t mw[4] = {mk.x, mk.y, mk.z, mk.w};
-#pragma unroll
-                for (int e = 0; e < 8; e++) {
-                    uint32_t mh = (e & 1) ? (mw[e >> 1] >> 16) : (mw[e >> 1] & 0xFFFFu);
-                    // stored activation > 0  <=>  sign clear, non-zero, not NaN
-                    bool keep = (mh & 0x8000u) == 0 && mh != 0 && mh <= 0x7C00u;
-                    if (!keep) h[e] = 0;
-                }
+                const uint4 mk = *(const uint4 *)(mrow + col);
+                w[4 * g8] = mask_pair(w[4 * g8], mk.x);
+                w[4 * g8 + 1] = mask_pair(w[4 * g8 + 1], mk.y);
+                w[4 * g8 + 2] = mask_pair(w[4 * g8 + 2], mk.z);
+                w[4 * g8 + 3] = mask_pair(w[4 * g8 + 3], mk.w);
             }
 #pragma unroll
-            for (int e = 0; e < 8; e++) bad |= (h[e] & 0x7C00u) == 0x7C00u;
-            *(uint4 *)(crow + col) = make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), h[4] | (h[5] << 16),
-                                                h[6] | (h[7] << 16));
+            for (int e = 0; e < 4; e++) nonfinite_acc(w[4 * g8 + e], acc);
+            *(uint4 *)(crow + col) = make_uint4(w[4 * g8], w[4 * g8 + 1], w[4 * g8 + 2], w[4 * g8 + 3]);
         } else {
             for (int e = 0; e < 8 && col + e < N; e++) {
-                uint32_t v = h[e];
+                uint32_t v = (e & 1) ? (w[4 * g8 + (e >> 1)] >> 16) : (w[4 * g8 + (e >> 1)] & 0xFFFFu);
                 if (mrow) {
-                    uint32_t mh = mrow[col + e];
-                    bool keep = (mh & 0x8000u) == 0 && mh != 0 && mh <= 0x7C00u;
-                    if (!keep) v = 0;
+                    const uint32_t mh = mrow[col + e];
+                    if (!(mh != 0 && mh <= 0x7C00u)) v = 0;
                 }
-                bad |= (v & 0x7C00u) == 0x7C00u;
+                nonfinite_acc(v, acc);
                 crow[col + e] = (uint16_t)v;
             }
         }
     }
+    bad |= nonfinite_any(acc);
 }
 
 // The same epilogue for 32 consecutive accumulator columns of the 32 rows a warp owns, with the
@@ -207,19 +227,15 @@ __device__ __forceinline__ void epilogue_store32_coalesced(const uint32_t (&r)[3
 {
     const int lane = threadIdx.x & 31;
     uint4 *mine = (uint4 *)(stage + lane * kEpiStagePitch);
+    {
+        uint32_t w[16];
+        round_pack32(r, relu, w);
 #pragma unroll
-    for (int g8 = 0; g8 < 4; g8++) {
-        uint32_t h[8];
-#pragma unroll
-        for (int e = 0; e < 8; e++) {
-            float s = __uint_as_float(r[g8 * 8 + e]);
-            if (relu) s = (s > 0.0f || s != s) ? s : 0.0f;
-            h[e] = (uint32_t)__half_as_ushort(__float2half_rn(s));
-        }
-        mine[g8] = make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), h[4] | (h[5] << 16), h[6] | (h[7] << 16));
+        for (int g8 = 0; g8 < 4; g8++) mine[g8] = make_uint4(w[4 * g8], w[4 * g8 + 1], w[4 * g8 + 2], w[4 * g8 + 3]);
     }
     __syncwarp();
     const int piece = lane & 3, col = col0 + piece * 8;
+    uint32_t acc = 0;
 #pragma unroll
     for (int it = 0; it < 4; it++) {
         const int rr = it * 8 + (lane >> 2), row = row0 + rr;
@@ -230,31 +246,28 @@ __device__ __forceinline__ void epilogue_store32_coalesced(const uint32_t (&r)[3
             if (col + 8 <= N) {
                 if (mask) {
                     const uint4 mk = *(const uint4 *)(mask + (size_t)row * ldmask + col);
-                    const uint32_t mw[4] = {mk.x, mk.y, mk.z, mk.w};
-#pragma unroll
-                    for (int q = 0; q < 4; q++) {
-                        const uint32_t lo = mw[q] & 0xFFFFu, hi = mw[q] >> 16;
-                        // stored activation > 0  <=>  sign clear, non-zero, not NaN
-                        if (!((lo & 0x8000u) == 0 && lo != 0 && lo <= 0x7C00u)) w[q] &= 0xFFFF0000u;
-                        if (!((hi & 0x8000u) == 0 && hi != 0 && hi <= 0x7C00u)) w[q] &= 0x0000FFFFu;
-                    }
+                    w[0] = mask_pair(w[0], mk.x);
+                    w[1] = mask_pair(w[1], mk.y);
+                    w[2] = mask_pair(w[2], mk.z);
+                    w[3] = mask_pair(w[3], mk.w);
                 }
 #pragma unroll
-                for (int q = 0; q < 4; q++) bad |= ((w[q] & 0x7C00u) == 0x7C00u) || ((w[q] & 0x7C000000u) == 0x7C000000u);
+                for (int q = 0; q < 4; q++) nonfinite_acc(w[q], acc);
                 *(uint4 *)(crow + col) = make_uint4(w[0], w[1], w[2], w[3]);
             } else {
                 for (int e = 0; e < 8 && col + e < N; e++) {
                     uint32_t x = (e & 1) ? (w[e >> 1] >> 16) : (w[e >> 1] & 0xFFFFu);
                     if (mask) {
                         const uint32_t mh = mask[(size_t)row * ldmask + col + e];
-                        if (!((mh & 0x8000u) == 0 && mh != 0 && mh <= 0x7C00u)) x = 0;
+                        if (!(mh != 0 && mh <= 0x7C00u)) x = 0;
                     }
-                    bad |= (x & 0x7C00u) == 0x7C00u;
+                    nonfinite_acc(x, acc);
                     crow[col + e] = (uint16_t)x;
                 }
             }
         }
     }
+    bad |= nonfinite_any(acc);
     __syncwarp();    // the block may be overwritten by the next call
 }
 

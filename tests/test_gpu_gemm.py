@@ -147,8 +147,8 @@ def test_pair_gemm_parity(op, M, N, K):
 def test_sweep_2048_cubed_in_full_every_kernel(op):
     """2048^3 of the isolated-GEMM sweep (seed and operand distribution of that sweep), every
     output element against the oracle: under the library's own kernel choice with and without a
-    scratch buffer, and with each tensor-core kernel forced.  This is the size at which the
-    automatic choice passes from the single-CTA kernel to the CTA pair."""
+    scratch buffer, and with each tensor-core kernel forced.  The automatic choice changes hands
+    near this size (64 tiles of 256x256: the last shape of the sweep the single-CTA kernel takes)."""
     from paper_1710_03740_b200 import binding as b
     M = N = K = 2048
     assert (M, N, K) in inputs.GEMM_SWEEP
