@@ -22,6 +22,7 @@
 // pipeline with 64 columns of B per CTA and N = 128 instructions.
 // No TMA multicast is used.  Every mbarrier wait is bounded (see tc_ptx.cuh).
 #include <cuda.h>
+#include <stdlib.h>
 
 #include "mpt_common.cuh"
 #include "tc_ptx.cuh"
@@ -72,6 +73,7 @@ struct Params {
     // k_tail_reduce finishes those tiles.  tail_split == 1: off (half-width units instead).
     int tail_split;
     float *tail_partial;
+    int hint_a, hint_b;              // L2 eviction priority of the operand loads (0 normal, 1 last, 2 first)
     LstmEpi lstm;                    // read only by the LSTM instantiation of the kernel
 };
 
@@ -194,6 +196,7 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
             uint32_t issued = 0, s = 0, ph = 0;
             bool ok = true;
             int tt = 0;
+            const uint64_t pol_a = l2_policy(p.hint_a), pol_b = l2_policy(p.hint_b);
             for (int u = pair_id; u < num_units && ok; u += num_pairs, tt++) {
                 const Unit w = unit_of(p, u, nkb);
                 // Every other unit of a cluster walks its k-blocks downwards: the operand panels a wave of
@@ -217,15 +220,15 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
                     const int k0 = (down ? (w.kb0 + w.kb1 - 1 - kb) : kb) * BLOCK_K;
                     if (A_MN) {
 #pragma unroll
-                        for (int j = 0; j < CTA_M / 64; j++) tma_load_2d_pair(sa + j * MN_BOX_BYTES, &tmA, m0 + 64 * j, k0, lead_full);
+                        for (int j = 0; j < CTA_M / 64; j++) tma_load_2d_pair_hint(sa + j * MN_BOX_BYTES, &tmA, m0 + 64 * j, k0, lead_full, pol_a);
                     } else {
-                        tma_load_2d_pair(sa, &tmA, k0, m0, lead_full);
+                        tma_load_2d_pair_hint(sa, &tmA, k0, m0, lead_full, pol_a);
                     }
                     if (B_MN) {
-                        tma_load_2d_pair(sb, &tmB, n0, k0, lead_full);
-                        if (cta_n == CTA_N) tma_load_2d_pair(sb + MN_BOX_BYTES, &tmB, n0 + 64, k0, lead_full);
+                        tma_load_2d_pair_hint(sb, &tmB, n0, k0, lead_full, pol_b);
+                        if (cta_n == CTA_N) tma_load_2d_pair_hint(sb + MN_BOX_BYTES, &tmB, n0 + 64, k0, lead_full, pol_b);
                     } else {
-                        tma_load_2d_pair(sb, cta_n == CTA_N ? &tmB : &tmBh, k0, n0, lead_full);
+                        tma_load_2d_pair_hint(sb, cta_n == CTA_N ? &tmB : &tmBh, k0, n0, lead_full, pol_b);
                     }
                 }
             }
@@ -612,6 +615,13 @@ cudaError_t launch_gemm_tc2(int op, int M, int N, int K, const uint16_t *A, int 
     // 1.01 GB (groups of 8) to 0.66 GB (0.77 / 0.82 / 1.00 / 1.57 GB with 12 / 24 / 32 / 4); with 6.3 MB
     // panels (K = 12288) nothing survives either way and 8 keeps the wave's own footprint smallest.
     p.group_m = K <= 6144 ? 16 : 8;
+    {
+        // both operands "evict last" (see tma_load_2d_pair_hint); MPT_L2_HINT=<A digit><B digit> overrides for
+        // comparisons: 0 normal, 1 evict last, 2 evict first
+        const char *e = getenv("MPT_L2_HINT");
+        p.hint_a = e && e[0] ? e[0] - '0' : 1;
+        p.hint_b = e && e[0] && e[1] ? e[1] - '0' : 1;
+    }
     p.full_units = p.num_units = 0;
     p.split_k = 1;
     p.partial = nullptr;
