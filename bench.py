@@ -468,7 +468,7 @@ def main():
                          "launches": g_n, "avg_launch_ms": g_ms / g_n if g_n else None, "traffic": traffic,
                          "traffic_note": ("ncu dram bytes of one %s launch; algorithmic minimum %.3e"
                                           % (tr["launch"], tr["algorithmic_bytes"])) if tr else None},
-            "update": {"bound": "hbm", "kernel": "k_update_vec", "achieved": upd_gbs, "peak": peaks["hbm_gbs"],
+            "update": {"bound": "hbm", "kernel": "k_update_quad", "achieved": upd_gbs, "peak": peaks["hbm_gbs"],
                        "peak_source": peak_src, "unit": "GB/s", "frac": (upd_gbs / peaks["hbm_gbs"]) if upd_gbs else None,
                        "frac_of_nominal": (upd_gbs / NOMINAL_HBM_GBS) if upd_gbs else None,
                        "bytes_per_param": 20 if cfg["momentum"] else 12, "avg_launch_ms": u_ms / u_n if u_n else None},

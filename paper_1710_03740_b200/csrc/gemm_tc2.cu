@@ -612,9 +612,12 @@ cudaError_t launch_gemm_tc2(int op, int M, int N, int K, const uint16_t *A, int 
     // Row blocks per group of the tile order.  Consecutive waves of a group share its A panels; whether
     // those survive in L2 between waves depends on their size: with the short panels of a weight-gradient
     // product (K = batch = 4096: 2 MB each) 16 of them do, and DRAM reads of 12288x12288x4096 fall from
-    // 1.01 GB (groups of 8) to 0.66 GB (0.77 / 0.82 / 1.00 / 1.57 GB with 12 / 24 / 32 / 4); with 6.3 MB
-    // panels (K = 12288) nothing survives either way and 8 keeps the wave's own footprint smallest.
-    p.group_m = K <= 6144 ? 16 : 8;
+    // 1.01 GB (groups of 8) to 0.66 GB (0.77 / 0.82 / 1.00 / 1.57 GB with 12 / 24 / 32 / 4).  With long
+    // panels nothing survives a wave, and 8 keeps the wave's own footprint smallest - unless the output has
+    // no more than 16 row blocks: one group then spans all of M and no B panel is ever asked for twice
+    // (4096x32000x12288: 5.6 -> 4.5 GB and 2.45 -> 2.30 ms; 4096x12288x32000: 6.5 -> 5.7 GB; the
+    // large-MLP step 0.6 % faster).
+    p.group_m = (K <= 6144 || p.tiles_m <= 16) ? 16 : 8;
     {
         // both operands "evict last" (see tma_load_2d_pair_hint); MPT_L2_HINT=<A digit><B digit> overrides for
         // comparisons: 0 normal, 1 evict last, 2 evict first
