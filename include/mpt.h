@@ -650,6 +650,29 @@ int mpt_dp_attach(mpt_ctx *ctx, int R, int rank, const uint16_t *const *g16_peer
                   uint16_t *const *w16_peers);
 int mpt_dp_norm(mpt_ctx *ctx);
 
+/* A context that keeps FP32 state for its own shard only (sections 3.1 and 4.5: the master copy costs 4
+ * bytes per parameter and every optimizer state another 4; with R replicas each needs them for 1/R of
+ * the parameters, because a replica updates only its shard).  mpt_workspace_bytes_dp / mpt_create_dp are
+ * mpt_workspace_bytes_opt / mpt_create_opt for replica `rank` of `replicas` (2 <= replicas <=
+ * MPT_DP_MAX_REPLICAS): the FP32 master array and the optimizer-state arrays hold the elements
+ * [lo, hi) of mpt_dp_shard(n, replicas, rank) of the flat parameter array (n from mpt_dp_layout_of) and
+ * nothing else; all replicas' workspaces have the same size and layout.  Such a context
+ *   - steps only while attached by mpt_dp_attach with the same replicas and rank (mpt_step otherwise:
+ *     MPT_ERR_STATE; mpt_dp_attach with other values: MPT_ERR_INVALID_ARG);
+ *   - mpt_set_master: rounds the whole layer into the FP16 weights (every replica must be given the
+ *     same values) and keeps the FP32 values that fall inside the shard; it uses the gradient array as
+ *     scratch, so gradients present are discarded;
+ *   - mpt_set_momentum / mpt_set_state2 keep, and mpt_get_master / mpt_get_tensor(MASTER32, MOMENTUM32,
+ *     STATE2_32) write, only the part of the layer inside the shard: elements [first, first + count) of
+ *     the layer as mpt_state_range reports (count may be 0); the rest of the host buffer is not touched.
+ *     Gathering a layer for a checkpoint is therefore one such call per replica into the same buffer.
+ * mpt_state_range works on every context (first = 0, count = out*in for an ordinary one). */
+int mpt_workspace_bytes_dp(const mpt_layer_desc *layers, int n_layers, int max_batch, const mpt_optimizer *opt, int replicas,
+                           int rank, size_t *bytes_out);
+int mpt_create_dp(const mpt_layer_desc *layers, int n_layers, float S, const mpt_optimizer *opt, int max_batch, int replicas,
+                  int rank, void *workspace_dev, size_t workspace_bytes, void *cuda_stream, mpt_ctx **out);
+int mpt_state_range(mpt_ctx *ctx, int layer, size_t *first_out, size_t *count_out);
+
 /* Device memory that other processes can map (the buffers the replicas exchange).  mpt_dp_alloc
  * returns memory from the driver's allocator (not from a framework's pool, whose blocks cannot be
  * exported); mpt_dp_export writes an opaque MPT_DP_HANDLE_BYTES handle for the allocation that

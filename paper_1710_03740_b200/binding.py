@@ -40,7 +40,8 @@ EXPORTS = ["mpt_workspace_bytes", "mpt_create", "mpt_workspace_bytes_opt", "mpt_
            "mpt_lstm_forward", "mpt_lstm_backward", "mpt_lstm_cell_forward", "mpt_lstm_cell_backward", "mpt_bias_grad",
            "mpt_add_f16",
            "mpt_dp_shard", "mpt_dp_step_flat", "mpt_dp_alloc", "mpt_dp_free", "mpt_dp_export", "mpt_dp_open", "mpt_dp_close",
-           "mpt_dp_layout_of", "mpt_dp_attach", "mpt_dp_step_flat_opt", "mpt_dp_norm_flat", "mpt_dp_norm"]
+           "mpt_dp_layout_of", "mpt_dp_attach", "mpt_dp_step_flat_opt", "mpt_dp_norm_flat", "mpt_dp_norm",
+           "mpt_workspace_bytes_dp", "mpt_create_dp", "mpt_state_range"]
 
 
 class MptError(RuntimeError):
@@ -93,6 +94,9 @@ def lib() -> C.CDLL:
     L.mpt_create.argtypes = [C.POINTER(LayerDesc), i32, f32, f32, f32, i32, vp, sz, vp, C.POINTER(vp)]
     L.mpt_workspace_bytes_opt.argtypes = [C.POINTER(LayerDesc), i32, i32, C.POINTER(Optimizer), C.POINTER(sz)]
     L.mpt_create_opt.argtypes = [C.POINTER(LayerDesc), i32, f32, C.POINTER(Optimizer), i32, vp, sz, vp, C.POINTER(vp)]
+    L.mpt_workspace_bytes_dp.argtypes = [C.POINTER(LayerDesc), i32, i32, C.POINTER(Optimizer), i32, i32, C.POINTER(sz)]
+    L.mpt_create_dp.argtypes = [C.POINTER(LayerDesc), i32, f32, C.POINTER(Optimizer), i32, i32, i32, vp, sz, vp, C.POINTER(vp)]
+    L.mpt_state_range.argtypes = [vp, i32, C.POINTER(sz), C.POINTER(sz)]
     L.mpt_set_state2.argtypes = [vp, i32, vp, sz]
     L.mpt_get_adam_products.argtypes = [vp, C.POINTER(f32), C.POINTER(f32)]
     L.mpt_set_adam_products.argtypes = [vp, f32, f32]
@@ -209,10 +213,10 @@ class Context:
     """One mpt_ctx over a torch-allocated workspace.  Method names follow the C calls."""
 
     def __init__(self, layers, S, lr, momentum=0.0, max_batch=1, device="cuda:0", stream=None, optimizer=None,
-                 shareable=False):
+                 shareable=False, shard=None):
         """optimizer: an Optimizer struct; default SGD with the given lr and momentum.  shareable: take
         the workspace from the driver's allocator (a DeviceBuffer other processes can map) instead of
-        torch's pool."""
+        torch's pool.  shard: (replicas, rank) - mpt_create_dp: FP32 state for that replica's shard only."""
         import torch
         self.layers = [(int(i), int(o), int(r)) for (i, o, r) in layers]
         self.device = torch.device(device)
@@ -220,8 +224,13 @@ class Context:
         opt = optimizer if optimizer is not None else Optimizer(OPT_SGD, float(lr), float(momentum), 0.0, 0.0, 0.0)
         self.optimizer = opt
         out = C.c_size_t(0)
-        _check(lib().mpt_workspace_bytes_opt(_layer_array(self.layers), len(self.layers), int(max_batch), C.byref(opt),
-                                             C.byref(out)))
+        self.shard = (int(shard[0]), int(shard[1])) if shard else None
+        if self.shard:
+            _check(lib().mpt_workspace_bytes_dp(_layer_array(self.layers), len(self.layers), int(max_batch), C.byref(opt),
+                                                self.shard[0], self.shard[1], C.byref(out)))
+        else:
+            _check(lib().mpt_workspace_bytes_opt(_layer_array(self.layers), len(self.layers), int(max_batch), C.byref(opt),
+                                                 C.byref(out)))
         nbytes = int(out.value)
         with torch.cuda.device(self.device):
             if shareable:
@@ -233,9 +242,14 @@ class Context:
                 base = self.workspace.data_ptr()
             self._ws_ptr = (base + 255) // 256 * 256
             self._ctx = C.c_void_p()
-            _check(lib().mpt_create_opt(_layer_array(self.layers), len(self.layers), float(S), C.byref(opt),
-                                        int(max_batch), C.c_void_p(self._ws_ptr), nbytes, _stream_ptr(stream),
-                                        C.byref(self._ctx)))
+            if self.shard:
+                _check(lib().mpt_create_dp(_layer_array(self.layers), len(self.layers), float(S), C.byref(opt),
+                                           int(max_batch), self.shard[0], self.shard[1], C.c_void_p(self._ws_ptr), nbytes,
+                                           _stream_ptr(stream), C.byref(self._ctx)))
+            else:
+                _check(lib().mpt_create_opt(_layer_array(self.layers), len(self.layers), float(S), C.byref(opt),
+                                            int(max_batch), C.c_void_p(self._ws_ptr), nbytes, _stream_ptr(stream),
+                                            C.byref(self._ctx)))
         self.workspace_bytes = nbytes
         self.batch = 0
 
@@ -245,6 +259,12 @@ class Context:
             self._ctx = None
             if isinstance(self.workspace, DeviceBuffer):
                 self.workspace.close()
+
+    def state_range(self, layer):
+        """(first, count): the elements of the layer whose FP32 master and optimizer state live here."""
+        first, count = C.c_size_t(0), C.c_size_t(0)
+        _check(lib().mpt_state_range(self._ctx, int(layer), C.byref(first), C.byref(count)), self._ctx)
+        return int(first.value), int(count.value)
 
     def dp_layout(self):
         out = DpLayout()
@@ -272,7 +292,8 @@ class Context:
 
     def get_master(self, layer):
         i, o, _ = self.layers[layer]
-        out = np.empty((o, i), dtype=np.float32)
+        # a context with FP32 state for its shard only fills in just that part (state_range): NaN elsewhere
+        out = np.full((o, i), np.nan, dtype=np.float32) if self.shard else np.empty((o, i), dtype=np.float32)
         _check(lib().mpt_get_master(self._ctx, layer, _hptr(out), out.size), self._ctx)
         return out
 
@@ -338,7 +359,7 @@ class Context:
         if kind in (T_W16, T_GRAD16):
             out = np.empty((o, i), dtype=np.uint16)
         elif kind in (T_MOMENTUM32, T_MASTER32, T_STATE2_32):
-            out = np.empty((o, i), dtype=np.float32)
+            out = np.full((o, i), np.nan, dtype=np.float32) if self.shard else np.empty((o, i), dtype=np.float32)
         else:
             out = np.empty((self.batch, o), dtype=np.uint16)
         _check(lib().mpt_get_tensor(self._ctx, kind, layer, _hptr(out), out.nbytes), self._ctx)
@@ -785,11 +806,13 @@ class DataParallelMLP:
     the one-kernel data-parallel step between two barriers.  Every replica feeds its own part of
     the batch (equal sizes) through forward() / backward_scaled() of `ctx`."""
 
-    def __init__(self, layers, S, lr, momentum=0.0, max_batch=1, group=None, optimizer=None):
+    def __init__(self, layers, S, lr, momentum=0.0, max_batch=1, group=None, optimizer=None, shard_state=False):
+        """shard_state: keep FP32 master and optimizer state for this replica's shard only (mpt_create_dp)."""
         import torch.distributed as dist
         self.group = group
         self.R, self.rank = dist.get_world_size(group), dist.get_rank(group)
-        self.ctx = Context(layers, S, lr, momentum, max_batch, shareable=True, optimizer=optimizer)
+        self.ctx = Context(layers, S, lr, momentum, max_batch, shareable=True, optimizer=optimizer,
+                           shard=(self.R, self.rank) if shard_state and self.R > 1 else None)
         lay = self.ctx.dp_layout()
         own = self.ctx.workspace
         table = dp_exchange_handles({"ws": own.export(), "skew": self.ctx._ws_ptr - own.ptr}, group)

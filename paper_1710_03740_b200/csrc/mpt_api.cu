@@ -28,6 +28,7 @@ struct Layer {
 
 struct Plan {
     size_t total = 0, P_pad = 0;
+    size_t st_lo = 0, st_n = 0;      // elements [st_lo, st_lo + st_n) of the flat parameter array have FP32 state here
     size_t off_status = 0, off_master = 0, off_mom = 0, off_state2 = 0, off_w16 = 0, off_g16 = 0, off_x[2] = {0, 0},
            off_labels[2] = {0, 0}, off_rowloss = 0, off_norm = 0, off_splitk = 0, splitk_bytes = 0;
     std::vector<size_t> off_act, off_dact, lay_off;
@@ -75,7 +76,7 @@ int validate_layers(const mpt_layer_desc *layers, int n_layers, int max_batch)
     return MPT_OK;
 }
 
-void make_plan(const mpt_layer_desc *layers, int L, int max_batch, int n_states, Plan &pl)
+void make_plan(const mpt_layer_desc *layers, int L, int max_batch, int n_states, Plan &pl, int replicas = 1, int rank = 0)
 {
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
@@ -87,9 +88,24 @@ void make_plan(const mpt_layer_desc *layers, int L, int max_batch, int n_states,
         P += align_up((size_t)layers[l].in_features * layers[l].out_features, 128);
     }
     pl.P_pad = P;
-    pl.off_master = take(P * 4);
-    pl.off_mom = n_states >= 1 ? take(P * 4) : 0;
-    pl.off_state2 = n_states >= 2 ? take(P * 4) : 0;
+    pl.st_lo = 0;
+    pl.st_n = P;
+    if (replicas > 1) {   // FP32 state of this replica's shard only
+        size_t lo = 0, hi = 0;
+        mpt_dp_shard(P, replicas, rank, &lo, &hi);
+        pl.st_lo = lo;
+        pl.st_n = hi - lo;
+    }
+    size_t state_elems = P;
+    if (replicas > 1) {   // every replica reserves the size of the largest shard, so that all layouts are the same
+        size_t lo0 = 0, hi0 = 0;
+        mpt_dp_shard(P, replicas, 0, &lo0, &hi0);
+        state_elems = hi0 - lo0;
+    }
+    const size_t state_bytes = (state_elems ? state_elems : 1) * 4;
+    pl.off_master = take(state_bytes);
+    pl.off_mom = n_states >= 1 ? take(state_bytes) : 0;
+    pl.off_state2 = n_states >= 2 ? take(state_bytes) : 0;
     pl.off_w16 = take(P * 2);
     pl.off_g16 = take(P * 2);
     pl.off_act.resize(L); pl.off_dact.resize(L); pl.ld_out.resize(L);
@@ -158,6 +174,9 @@ struct mpt_ctx {
     float scale_backoff = 0.5f, scale_growth = 2.0f, scale_min = 0x1p-100f, scale_max = 0x1p120f;
     // data-parallel step (mpt_dp_attach): replica count (0 or 1: off), this replica, peer tables
     int dp_R = 0, dp_rank = 0;
+    // mpt_create_dp: FP32 master and optimizer state exist for this replica's shard only; master / mom /
+    // state2 are then bases such that element i of the flat array is at [i] for i inside the shard
+    int shard_R = 0, shard_rank = 0;
     bool dp_norm_done = false;   // mpt_dp_norm has run since the last backward pass (clipping in data-parallel mode)
     const uint16_t *dp_g16[MPT_DP_MAX_REPLICAS] = {};
     const uint32_t *dp_flag[MPT_DP_MAX_REPLICAS] = {};
@@ -351,6 +370,8 @@ int do_backward(mpt_ctx *c, const int32_t *labels_dev)
 int do_step(mpt_ctx *c)
 {
     if (!c->have_grads) return fail(c, MPT_ERR_STATE, "mpt_step needs gradients (mpt_backward_scaled or mpt_set_grad)");
+    if (c->shard_R > 1 && (c->dp_R != c->shard_R || c->dp_rank != c->shard_rank))
+        return fail(c, MPT_ERR_STATE, "a context created by mpt_create_dp steps only while attached (mpt_dp_attach) as that replica");
     const float inv = 1.0f / c->S;
     CK(cudaMemsetAsync(c->status + ST_OVERFLOW_SEEN, 0, sizeof(uint32_t), c->stream), "status clear");
     cudaError_t e;
@@ -477,6 +498,17 @@ int dispatch_gemm(int op, int M, int N, int K, const uint16_t *A, int lda, const
     return e == cudaSuccess ? MPT_OK : MPT_ERR_CUDA;
 }
 
+// Part of a layer's parameters whose FP32 state this context holds: all of it, or, for a context made
+// by mpt_create_dp, the part inside the replica's shard.  first is relative to the layer.
+void state_part(const mpt_ctx *c, const Layer &ly, size_t *first, size_t *count)
+{
+    const size_t a = ly.off > c->plan.st_lo ? ly.off : c->plan.st_lo;
+    const size_t e1 = ly.off + ly.n, e2 = c->plan.st_lo + c->plan.st_n;
+    const size_t b = e1 < e2 ? e1 : e2;
+    *first = a < b ? a - ly.off : 0;
+    *count = a < b ? b - a : 0;
+}
+
 }  // namespace mpt
 
 extern "C" {
@@ -514,8 +546,41 @@ int mpt_create(const mpt_layer_desc *layers, int n_layers, float S, float lr, fl
     return mpt_create_opt(layers, n_layers, S, &opt, max_batch, workspace_dev, workspace_bytes, cuda_stream, out);
 }
 
+static int create_impl(const mpt_layer_desc *layers, int n_layers, float S, const mpt_optimizer *opt, int max_batch,
+                       int replicas, int rank, void *workspace_dev, size_t workspace_bytes, void *cuda_stream, mpt_ctx **out);
+
 int mpt_create_opt(const mpt_layer_desc *layers, int n_layers, float S, const mpt_optimizer *opt, int max_batch,
                    void *workspace_dev, size_t workspace_bytes, void *cuda_stream, mpt_ctx **out)
+{
+    return create_impl(layers, n_layers, S, opt, max_batch, 1, 0, workspace_dev, workspace_bytes, cuda_stream, out);
+}
+
+int mpt_workspace_bytes_dp(const mpt_layer_desc *layers, int n_layers, int max_batch, const mpt_optimizer *opt, int replicas,
+                           int rank, size_t *bytes_out)
+{
+    if (!bytes_out || !opt) return MPT_ERR_INVALID_ARG;
+    int r = validate_layers(layers, n_layers, max_batch);
+    if (r != MPT_OK) return r;
+    if (!valid_optimizer(opt)) return MPT_ERR_INVALID_ARG;
+    if (replicas < 2 || replicas > MPT_DP_MAX_REPLICAS || rank < 0 || rank >= replicas) return MPT_ERR_INVALID_ARG;
+    Plan pl;
+    make_plan(layers, n_layers, max_batch, opt_states(*opt), pl, replicas, rank);
+    *bytes_out = pl.total;
+    return MPT_OK;
+}
+
+int mpt_create_dp(const mpt_layer_desc *layers, int n_layers, float S, const mpt_optimizer *opt, int max_batch, int replicas,
+                  int rank, void *workspace_dev, size_t workspace_bytes, void *cuda_stream, mpt_ctx **out)
+{
+    if (replicas < 2 || replicas > MPT_DP_MAX_REPLICAS || rank < 0 || rank >= replicas) {
+        if (out) *out = nullptr;
+        return MPT_ERR_INVALID_ARG;
+    }
+    return create_impl(layers, n_layers, S, opt, max_batch, replicas, rank, workspace_dev, workspace_bytes, cuda_stream, out);
+}
+
+static int create_impl(const mpt_layer_desc *layers, int n_layers, float S, const mpt_optimizer *opt, int max_batch,
+                       int replicas, int rank, void *workspace_dev, size_t workspace_bytes, void *cuda_stream, mpt_ctx **out)
 {
     if (!out) return MPT_ERR_INVALID_ARG;
     *out = nullptr;
@@ -529,17 +594,18 @@ int mpt_create_opt(const mpt_layer_desc *layers, int n_layers, float S, const mp
     const int n_states = opt_states(*opt);
     c->use_momentum = n_states >= 1;
     c->opt_kind = opt->kind; c->beta2 = opt->beta2; c->eps = opt->eps; c->wd = opt->weight_decay; c->clip = opt->clip_norm;
-    make_plan(layers, n_layers, max_batch, n_states, c->plan);
+    make_plan(layers, n_layers, max_batch, n_states, c->plan, replicas, rank);
     if (workspace_bytes < c->plan.total) { delete c; return MPT_ERR_WORKSPACE; }
+    if (replicas > 1) { c->shard_R = replicas; c->shard_rank = rank; }
     const float lr = opt->lr, momentum = opt->momentum;
     c->S = S; c->lr = lr; c->mu = momentum; c->max_batch = max_batch;
     c->stream = (cudaStream_t)cuda_stream;
     c->ws = (uint8_t *)workspace_dev;
     const Plan &pl = c->plan;
     c->status = (uint32_t *)(c->ws + pl.off_status);
-    c->master = (float *)(c->ws + pl.off_master);
-    c->mom = c->use_momentum ? (float *)(c->ws + pl.off_mom) : nullptr;
-    c->state2 = n_states >= 2 ? (float *)(c->ws + pl.off_state2) : nullptr;
+    c->master = (float *)(c->ws + pl.off_master) - pl.st_lo;
+    c->mom = c->use_momentum ? (float *)(c->ws + pl.off_mom) - pl.st_lo : nullptr;
+    c->state2 = n_states >= 2 ? (float *)(c->ws + pl.off_state2) - pl.st_lo : nullptr;
     c->w16 = (uint16_t *)(c->ws + pl.off_w16);
     c->g16 = (uint16_t *)(c->ws + pl.off_g16);
     for (int k = 0; k < 2; k++) {
@@ -693,11 +759,41 @@ int mpt_set_master(mpt_ctx *c, int layer, const float *src_host, size_t n)
     if (layer < 0 || layer >= (int)c->layers.size()) return fail(c, MPT_ERR_INVALID_ARG, "layer index");
     Layer &ly = c->layers[layer];
     if (n != ly.n) return fail(c, MPT_ERR_SHAPE, "n must equal out*in");
+    if (c->shard_R > 1) {
+        // FP32 values of the whole layer pass through the gradient array (as scratch, in pieces) to be
+        // rounded into the FP16 weights; the part inside the shard is kept as the master copy
+        float *scratch = (float *)c->g16;
+        const size_t cap = c->plan.P_pad / 2;
+        c->have_grads = false;
+        for (size_t at = 0; at < n; at += cap) {
+            const size_t m = n - at < cap ? n - at : cap;
+            CK(cudaMemcpyAsync(scratch, src_host + at, m * 4, cudaMemcpyHostToDevice, c->stream), "master upload");
+            cudaError_t e = launch_recast(scratch, c->w16 + ly.off + at, m, c->stream);
+            c->launches++;
+            if (e != cudaSuccess) return cuda_fail(c, e, "recast launch");
+        }
+        CK(cudaMemsetAsync(c->g16, 0, c->plan.P_pad * 2, c->stream), "gradient clear");
+        size_t first = 0, count = 0;
+        state_part(c, ly, &first, &count);
+        if (count) CK(cudaMemcpyAsync(c->master + ly.off + first, src_host + first, count * 4, cudaMemcpyHostToDevice, c->stream), "master upload");
+        CK(cudaStreamSynchronize(c->stream), "stream synchronize");
+        return MPT_OK;
+    }
     CK(cudaMemcpyAsync(c->master + ly.off, src_host, n * 4, cudaMemcpyHostToDevice, c->stream), "master upload");
     cudaError_t e = launch_recast(c->master + ly.off, c->w16 + ly.off, n, c->stream);
     c->launches++;
     if (e != cudaSuccess) return cuda_fail(c, e, "recast launch");
     CK(cudaStreamSynchronize(c->stream), "stream synchronize");
+    return MPT_OK;
+}
+
+int mpt_state_range(mpt_ctx *c, int layer, size_t *first_out, size_t *count_out)
+{
+    int r = usable(c);
+    if (r != MPT_OK) return r;
+    if (!first_out || !count_out) return fail(c, MPT_ERR_INVALID_ARG, "null output");
+    if (layer < 0 || layer >= (int)c->layers.size()) return fail(c, MPT_ERR_INVALID_ARG, "layer index");
+    state_part(c, c->layers[layer], first_out, count_out);
     return MPT_OK;
 }
 
@@ -709,7 +805,9 @@ int mpt_get_master(mpt_ctx *c, int layer, float *dst_host, size_t n)
     if (layer < 0 || layer >= (int)c->layers.size()) return fail(c, MPT_ERR_INVALID_ARG, "layer index");
     Layer &ly = c->layers[layer];
     if (n != ly.n) return fail(c, MPT_ERR_SHAPE, "n must equal out*in");
-    CK(cudaMemcpyAsync(dst_host, c->master + ly.off, n * 4, cudaMemcpyDeviceToHost, c->stream), "master download");
+    size_t first = 0, count = 0;
+    state_part(c, ly, &first, &count);
+    if (count) CK(cudaMemcpyAsync(dst_host + first, c->master + ly.off + first, count * 4, cudaMemcpyDeviceToHost, c->stream), "master download");
     CK(cudaStreamSynchronize(c->stream), "stream synchronize");
     return MPT_OK;
 }
@@ -856,6 +954,14 @@ int mpt_get_tensor(mpt_ctx *c, int kind, int layer, void *dst_host, size_t bytes
         default: return fail(c, MPT_ERR_INVALID_ARG, "tensor kind");
     }
     if (bytes != rows * row_bytes) return fail(c, MPT_ERR_SHAPE, "byte count does not match the tensor");
+    if (c->shard_R > 1 && (kind == MPT_T_MASTER32 || kind == MPT_T_MOMENTUM32 || kind == MPT_T_STATE2_32)) {
+        // only the part inside this replica's shard exists (mpt_state_range); the rest of dst_host is left alone
+        size_t first = 0, count = 0;
+        state_part(c, ly, &first, &count);
+        if (count) CK(cudaMemcpyAsync((float *)dst_host + first, (const float *)src + first, count * 4, cudaMemcpyDeviceToHost, c->stream), "tensor download");
+        CK(cudaStreamSynchronize(c->stream), "stream synchronize");
+        return MPT_OK;
+    }
     CK(cudaMemcpy2DAsync(dst_host, row_bytes, src, pitch, row_bytes, rows, cudaMemcpyDeviceToHost, c->stream), "tensor download");
     CK(cudaStreamSynchronize(c->stream), "stream synchronize");
     return MPT_OK;
@@ -889,7 +995,9 @@ int mpt_set_momentum(mpt_ctx *c, int layer, const float *src_host, size_t n)
     if (!c->use_momentum) return fail(c, MPT_ERR_STATE, "context has no momentum buffer");
     Layer &ly = c->layers[layer];
     if (n != ly.n) return fail(c, MPT_ERR_SHAPE, "n must equal out*in");
-    CK(cudaMemcpyAsync(c->mom + ly.off, src_host, n * 4, cudaMemcpyHostToDevice, c->stream), "momentum upload");
+    size_t first = 0, count = 0;
+    state_part(c, ly, &first, &count);
+    if (count) CK(cudaMemcpyAsync(c->mom + ly.off + first, src_host + first, count * 4, cudaMemcpyHostToDevice, c->stream), "momentum upload");
     CK(cudaStreamSynchronize(c->stream), "stream synchronize");
     return MPT_OK;
 }
@@ -903,7 +1011,9 @@ int mpt_set_state2(mpt_ctx *c, int layer, const float *src_host, size_t n)
     if (!c->state2) return fail(c, MPT_ERR_STATE, "context has no second optimizer state");
     Layer &ly = c->layers[layer];
     if (n != ly.n) return fail(c, MPT_ERR_SHAPE, "n must equal out*in");
-    CK(cudaMemcpyAsync(c->state2 + ly.off, src_host, n * 4, cudaMemcpyHostToDevice, c->stream), "state upload");
+    size_t first = 0, count = 0;
+    state_part(c, ly, &first, &count);
+    if (count) CK(cudaMemcpyAsync(c->state2 + ly.off + first, src_host + first, count * 4, cudaMemcpyHostToDevice, c->stream), "state upload");
     CK(cudaStreamSynchronize(c->stream), "stream synchronize");
     return MPT_OK;
 }
@@ -957,6 +1067,8 @@ int mpt_dp_attach(mpt_ctx *c, int R, int rank, const uint16_t *const *g16_peers,
         return MPT_OK;
     }
     if (R < 2 || R > MPT_DP_MAX_REPLICAS || rank < 0 || rank >= R) return fail(c, MPT_ERR_INVALID_ARG, "replica count or rank");
+    if (c->shard_R > 1 && (R != c->shard_R || rank != c->shard_rank))
+        return fail(c, MPT_ERR_INVALID_ARG, "the context was created by mpt_create_dp for another replica count or rank");
     if (!g16_peers || !flag_peers || !w16_peers) return fail(c, MPT_ERR_INVALID_ARG, "null peer table");
     for (int q = 0; q < R; q++) {
         if (!g16_peers[q] || !flag_peers[q] || !w16_peers[q]) return fail(c, MPT_ERR_INVALID_ARG, "null peer pointer");

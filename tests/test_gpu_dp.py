@@ -343,7 +343,7 @@ def _mlp_batch(t, q):
     return x, y
 
 
-def _mlp_replica_main(rank, R, port, out_dir, dynamic=False, opt_kind=0, clip=0.0):
+def _mlp_replica_main(rank, R, port, out_dir, dynamic=False, opt_kind=0, clip=0.0, shard_state=False):
     import datetime
     import torch as th
     import torch.distributed as dist
@@ -353,7 +353,8 @@ def _mlp_replica_main(rank, R, port, out_dir, dynamic=False, opt_kind=0, clip=0.
                             timeout=datetime.timedelta(seconds=90))
     try:
         opt = b.Optimizer(opt_kind, _MLP["lr"], _MLP["mu"], 0.999, 1e-8, 0.001, clip) if (opt_kind or clip) else None
-        dp = b.DataParallelMLP(_MLP_LAYERS, _MLP["S"], _MLP["lr"], _MLP["mu"], max_batch=_MLP["batch"], optimizer=opt)
+        dp = b.DataParallelMLP(_MLP_LAYERS, _MLP["S"], _MLP["lr"], _MLP["mu"], max_batch=_MLP["batch"], optimizer=opt,
+                               shard_state=shard_state)
         L = len(_MLP_LAYERS)
         for l, w in enumerate(_mlp_masters()):
             dp.ctx.set_master(l, w)
@@ -381,6 +382,11 @@ def _mlp_replica_main(rank, R, port, out_dir, dynamic=False, opt_kind=0, clip=0.
             for l in range(L):
                 rec["e2e_w16_%d_%d" % (t, l)] = dp.ctx.get_tensor(b.T_W16, l)
         rec["launches"] = np.array(dp.ctx.launch_count())
+        rec["workspace_bytes"] = np.array(dp.ctx.workspace_bytes)
+        rec["state_ranges"] = np.array([dp.ctx.state_range(l) for l in range(L)], dtype=np.int64)
+        if opt_kind == 3:
+            for l in range(L):
+                rec["end_state2_%d" % l] = dp.ctx.get_tensor(b.T_STATE2_32, l)
         np.savez(os.path.join(out_dir, "m%d.npz" % rank), **rec)
         dp.close()
     finally:
@@ -434,6 +440,115 @@ def test_dp_mlp_two_processes(tmp_path):
                 want16 = ora.replicas[0].w16[l]
                 assert np.array_equal(rec[q]["e2e_w16_%d_%d" % (t, l)].reshape(want16.shape), want16), (t, l, q)
     assert all(int(r["launches"]) > 0 for r in rec)
+
+
+@pytest.mark.timeout(300)
+@pytest.mark.parametrize("kind", [0, 3])
+def test_dp_mlp_two_processes_shard_only_state(tmp_path, kind):
+    """The same two processes with contexts that keep FP32 master and optimizer state for their own
+    shard only (mpt_create_dp; sections 3.1 and 4.5: 4 bytes per parameter and state, needed on one
+    replica each).  FP16 weights of both replicas stay bit-exact with the oracle's replicas through the
+    injected steps (one of them skipped) and whole iterations; each replica returns FP32 state for exactly
+    its shard (NaN fill elsewhere), bit-exact there, and the shards cover every element; the workspace
+    is smaller than an ordinary context's by the FP32 state of the other shard."""
+    import torch.multiprocessing as mp
+    from oracle.dp import OracleDataParallelMLP
+    from paper_1710_03740_b200 import binding as b
+    R = 2
+    mp.spawn(_mlp_replica_main, args=(R, _free_port(), str(tmp_path), False, kind, 0.0, True), nprocs=R, join=True)
+    rec = [np.load(os.path.join(str(tmp_path), "m%d.npz" % q)) for q in range(R)]
+    L = len(_MLP_LAYERS)
+    ora = OracleDataParallelMLP(_MLP_LAYERS, _MLP["S"], _MLP["lr"], _MLP["mu"], R)
+    if kind:
+        ora.set_optimizer(kind, _MLP["lr"], _MLP["mu"], 0.999, 1e-8, 0.001)
+    for l, w in enumerate(_mlp_masters()):
+        ora.set_master(l, w)
+    for t in range(_MLP["inj_steps"]):
+        for q in range(R):
+            for l in range(L):
+                ora.set_grad(q, l, _mlp_injected_grad(t, q, l).view(np.uint16))
+        skipped = ora.step()
+        assert skipped == (1 if t == 1 else 0)
+        for l in range(L):
+            want16, want32 = ora.replicas[0].w16[l], ora.replicas[0].w32[l]
+            wantv = ora.replicas[0].v[l]
+            covered = np.zeros(want32.size, np.int32)
+            for q in range(R):
+                assert bool(rec[q]["inj_skip_%d" % t]) == bool(skipped)
+                assert np.array_equal(rec[q]["inj_w16_%d_%d" % (t, l)].reshape(want16.shape), want16), (t, l, q)
+                first, count = (int(x) for x in rec[q]["state_ranges"][l])
+                for name, want in (("inj_w32_%d_%d", want32), ("inj_v_%d_%d", wantv)):
+                    got = rec[q][name % (t, l)].reshape(-1)
+                    inside = np.zeros(got.size, bool)
+                    inside[first:first + count] = True
+                    assert np.isnan(got[~inside]).all(), "nothing is reported outside the shard"
+                    assert np.array_equal(got[inside].view(np.uint32), want.reshape(-1)[inside].view(np.uint32)), (t, l, q, name)
+                covered[first:first + count] += 1
+            assert (covered == 1).all(), "every element's FP32 state lives on exactly one replica"
+    for t in range(_MLP["e2e_steps"]):
+        xs, ys = zip(*[_mlp_batch(t, q) for q in range(R)])
+        losses = ora.forward_backward(list(xs), list(ys))
+        for q in range(R):
+            got = float(rec[q]["e2e_loss_%d" % t])
+            assert abs(got - losses[q]) <= 1e-3 * abs(losses[q]), (t, q, got, losses[q])
+            for l in range(L):
+                ora.set_grad(q, l, rec[q]["e2e_g16_%d_%d" % (t, l)])
+        skipped = ora.step()
+        for q in range(R):
+            assert bool(rec[q]["e2e_skip_%d" % t]) == bool(skipped)
+            for l in range(L):
+                want16 = ora.replicas[0].w16[l]
+                assert np.array_equal(rec[q]["e2e_w16_%d_%d" % (t, l)].reshape(want16.shape), want16), (t, l, q)
+    if kind == 3:
+        for l in range(L):
+            want = ora.replicas[0].s2[l].reshape(-1)
+            for q in range(R):
+                first, count = (int(x) for x in rec[q]["state_ranges"][l])
+                got = rec[q]["end_state2_%d" % l].reshape(-1)
+                assert np.array_equal(got[first:first + count].view(np.uint32), want[first:first + count].view(np.uint32))
+    # the workspace: same size on both replicas, smaller than an ordinary context's by the other shard's FP32 state
+    opt = b.Optimizer(kind, _MLP["lr"], _MLP["mu"], 0.999, 1e-8, 0.001, 0.0) if kind else None
+    full = b.Context(_MLP_LAYERS, _MLP["S"], _MLP["lr"], _MLP["mu"], max_batch=_MLP["batch"], optimizer=opt)
+    n = full.dp_layout().n
+    n_states = 1 + (2 if kind == 3 else 1)
+    assert int(rec[0]["workspace_bytes"]) == int(rec[1]["workspace_bytes"])
+    saved = full.workspace_bytes - int(rec[0]["workspace_bytes"])
+    assert abs(saved - n_states * 4 * (n - n // R)) <= n_states * (256 + 32 * R), (saved, n, n_states)
+    full.close()
+
+
+def test_shard_only_context_refuses_what_it_cannot_do():
+    """A context made by mpt_create_dp has no FP32 state outside its shard: it steps only while attached
+    as that replica, and cannot be attached as another."""
+    require_gpu()
+    from paper_1710_03740_b200 import binding as b
+    ctx = b.Context(_MLP_LAYERS, _MLP["S"], _MLP["lr"], _MLP["mu"], max_batch=_MLP["batch"], shard=(2, 1))
+    L = len(_MLP_LAYERS)
+    for l, w in enumerate(_mlp_masters()):
+        ctx.set_master(l, w)
+        got = ctx.get_master(l).reshape(-1)
+        first, count = ctx.state_range(l)
+        assert np.array_equal(got[first:first + count], w.reshape(-1)[first:first + count])
+        assert np.isnan(got[:first]).all() and np.isnan(got[first + count:]).all()
+        with np.errstate(over="ignore"):
+            assert np.array_equal(ctx.get_tensor(b.T_W16, l).reshape(-1), w.astype(np.float16).view(np.uint16).reshape(-1))
+    total = sum(ctx.state_range(l)[1] for l in range(L))
+    lo, hi = b.mpt_dp_shard(ctx.dp_layout().n, 2, 1)
+    assert 0 < total <= hi - lo
+    for l in range(L):
+        ctx.set_grad(l, _mlp_injected_grad(0, 0, l).view(np.uint16))
+    with pytest.raises(b.MptError) as e:
+        ctx.step()
+    assert e.value.code == -3          # MPT_ERR_STATE
+    lay = ctx.dp_layout()
+    base = ctx._ws_ptr
+    tabs = [[base + off] * 2 for off in (lay.g16_offset, lay.flags_offset, lay.w16_offset)]
+    with pytest.raises(b.MptError) as e:
+        ctx.dp_attach(2, 0, *tabs)
+    assert e.value.code == -1          # MPT_ERR_INVALID_ARG
+    ctx.close()
+    with pytest.raises(b.MptError):
+        b.Context(_MLP_LAYERS, _MLP["S"], _MLP["lr"], _MLP["mu"], max_batch=_MLP["batch"], shard=(1, 0))
 
 
 @pytest.mark.timeout(300)
