@@ -98,6 +98,7 @@ __global__ void __launch_bounds__(EpiCfg<LSTM || WIDE>::THREADS, 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcParams p)
 {
     pdl_trigger();
+    if (threadIdx.x == 32) { prefetch_tensormap(&tmA); prefetch_tensormap(&tmB); }
     constexpr int STAGES = TileCfg<BLOCK_N>::STAGES;
     constexpr int STAGE_BYTES = TileCfg<BLOCK_N>::STAGE_BYTES;
     constexpr int TMEM_COLS = TileCfg<BLOCK_N>::TMEM_COLS;

@@ -113,6 +113,7 @@ k_gemm_tc4(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
     static_assert(RECV_BYTES + SEND_BYTES + EPI_WARPS * EPI_STAGE_BYTES <= STAGES * STAGE_BYTES, "the blocks of the exchange must fit the ring");
 
     pdl_trigger();
+    if (threadIdx.x == 32) { prefetch_tensormap(&tmA); prefetch_tensormap(&tmB); }
     if (threadIdx.x == 0) TC4_STAMP(0);
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;

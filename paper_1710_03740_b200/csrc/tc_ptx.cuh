@@ -69,6 +69,15 @@ static __device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, vol
     }
 }
 
+// Starts the fetch of a tensor map (a kernel parameter) into the TMA unit's descriptor cache, so that the
+// first tensor load does not wait for it.
+__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap *map)
+{
+#ifndef MPT_NO_TMAP_PREFETCH
+    asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+#endif
+}
+
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar)
 {
     asm volatile(
