@@ -41,7 +41,8 @@ EXPORTS = ["mpt_workspace_bytes", "mpt_create", "mpt_workspace_bytes_opt", "mpt_
            "mpt_add_f16",
            "mpt_dp_shard", "mpt_dp_step_flat", "mpt_dp_alloc", "mpt_dp_free", "mpt_dp_export", "mpt_dp_open", "mpt_dp_close",
            "mpt_dp_layout_of", "mpt_dp_attach", "mpt_dp_step_flat_opt", "mpt_dp_norm_flat", "mpt_dp_norm",
-           "mpt_workspace_bytes_dp", "mpt_create_dp", "mpt_state_range"]
+           "mpt_workspace_bytes_dp", "mpt_create_dp", "mpt_state_range", "mpt_dp_overlap_events", "mpt_dp_overlap_attach",
+           "mpt_dp_reduce_async"]
 
 
 class MptError(RuntimeError):
@@ -97,6 +98,9 @@ def lib() -> C.CDLL:
     L.mpt_workspace_bytes_dp.argtypes = [C.POINTER(LayerDesc), i32, i32, C.POINTER(Optimizer), i32, i32, C.POINTER(sz)]
     L.mpt_create_dp.argtypes = [C.POINTER(LayerDesc), i32, f32, C.POINTER(Optimizer), i32, i32, i32, vp, sz, vp, C.POINTER(vp)]
     L.mpt_state_range.argtypes = [vp, i32, C.POINTER(sz), C.POINTER(sz)]
+    L.mpt_dp_overlap_events.argtypes = [vp, vp]
+    L.mpt_dp_overlap_attach.argtypes = [vp, vp, vp, sz]
+    L.mpt_dp_reduce_async.argtypes = [vp]
     L.mpt_set_state2.argtypes = [vp, i32, vp, sz]
     L.mpt_get_adam_products.argtypes = [vp, C.POINTER(f32), C.POINTER(f32)]
     L.mpt_set_adam_products.argtypes = [vp, f32, f32]
@@ -265,6 +269,25 @@ class Context:
         first, count = C.c_size_t(0), C.c_size_t(0)
         _check(lib().mpt_state_range(self._ctx, int(layer), C.byref(first), C.byref(count)), self._ctx)
         return int(first.value), int(count.value)
+
+    def dp_overlap_events(self):
+        """Handles of this context's per-layer events (bytes) for the other replicas."""
+        buf = (C.c_uint8 * (len(self.layers) * DP_HANDLE_BYTES))()
+        _check(lib().mpt_dp_overlap_events(self._ctx, buf), self._ctx)
+        return bytes(buf)
+
+    def dp_overlap_attach(self, peer_handles, rank):
+        """peer_handles: list of R byte strings from dp_overlap_events (entry `rank` ignored)."""
+        import torch
+        R = len(peer_handles)
+        lo, hi = mpt_dp_shard(self.dp_layout().n, R, rank)
+        self._sum32 = torch.empty(max(hi - lo, 4), dtype=torch.float32, device=self.device)
+        keep = [C.create_string_buffer(h, len(h)) if q != rank else None for q, h in enumerate(peer_handles)]
+        tab = (C.c_void_p * R)(*[C.cast(k, C.c_void_p) if k is not None else None for k in keep])
+        _check(lib().mpt_dp_overlap_attach(self._ctx, tab, _dptr(self._sum32), self._sum32.numel() * 4), self._ctx)
+
+    def dp_reduce_async(self):
+        _check(lib().mpt_dp_reduce_async(self._ctx), self._ctx)
 
     def dp_layout(self):
         out = DpLayout()
@@ -806,8 +829,11 @@ class DataParallelMLP:
     the one-kernel data-parallel step between two barriers.  Every replica feeds its own part of
     the batch (equal sizes) through forward() / backward_scaled() of `ctx`."""
 
-    def __init__(self, layers, S, lr, momentum=0.0, max_batch=1, group=None, optimizer=None, shard_state=False):
-        """shard_state: keep FP32 master and optimizer state for this replica's shard only (mpt_create_dp)."""
+    def __init__(self, layers, S, lr, momentum=0.0, max_batch=1, group=None, optimizer=None, shard_state=False,
+                 overlap=False):
+        """shard_state: keep FP32 master and optimizer state for this replica's shard only (mpt_create_dp).
+        overlap: pull and add the replicas' gradients layer by layer beside the backward pass (interprocess
+        events; call ctx.backward_scaled(labels, want_loss=False) so that the pass is only enqueued)."""
         import torch.distributed as dist
         self.group = group
         self.R, self.rank = dist.get_world_size(group), dist.get_rank(group)
@@ -830,6 +856,12 @@ class DataParallelMLP:
             f.append(base + lay.flags_offset)
         if self.R > 1:
             self.ctx.dp_attach(self.R, self.rank, g, f, w)
+        self.overlap = bool(overlap) and self.R > 1
+        if self.overlap:
+            mine = self.ctx.dp_overlap_events()
+            handles = [None] * self.R
+            dist.all_gather_object(handles, mine, group=group)
+            self.ctx.dp_overlap_attach(handles, self.rank)
         self.shard = mpt_dp_shard(lay.n, self.R, self.rank)
 
     def _barrier(self):
@@ -840,6 +872,13 @@ class DataParallelMLP:
 
     def step(self):
         """All replicas call this after their backward_scaled(); returns True if the step was skipped."""
+        if self.overlap:
+            import torch.distributed as dist
+            dist.barrier(group=self.group)      # every replica has ENQUEUED its backward pass; nobody waits for a GPU here
+            self.ctx.dp_reduce_async()
+            overflow = self.ctx.step()          # waits on the streams for the sums and for every replica's pass
+            self._barrier()
+            return bool(overflow)
         self._barrier()
         if self.R > 1 and self.ctx.optimizer.clip_norm > 0.0:
             self.ctx.dp_norm()          # every replica's part of the norm, then all of them visible to all

@@ -153,7 +153,8 @@ __global__ void __launch_bounds__(kDpThreads) k_dp_step_opt(const DpPeers pp, in
                                                             size_t n8, float inv, const float *__restrict__ S_dev, float lr,
                                                             float mu, float b2, float eps, float wd, float b1t, float b2t,
                                                             const float *__restrict__ betat_dev, uint32_t *flags,
-                                                            const float *__restrict__ coef_dev)
+                                                            const float *__restrict__ coef_dev,
+                                                            const float4 *__restrict__ sum32)
 {
     pdl_trigger();
     pdl_wait();
@@ -172,14 +173,19 @@ __global__ void __launch_bounds__(kDpThreads) k_dp_step_opt(const DpPeers pp, in
     constexpr bool S2 = KIND == MPT_OPT_ADAM;
     const size_t vec = first / 8 + j;
     float s[8];
+    if (sum32) {      // the FP32 sums over the replicas were formed earlier (k_dp_reduce), in the same order
+        const float4 x0 = __ldcs(sum32 + 2 * j), x1 = __ldcs(sum32 + 2 * j + 1);
+        s[0] = x0.x; s[1] = x0.y; s[2] = x0.z; s[3] = x0.w; s[4] = x1.x; s[5] = x1.y; s[6] = x1.z; s[7] = x1.w;
+    } else {
 #pragma unroll 4
-    for (int q = 0; q < R; q++) {
-        const uint4 g = __ldcs((const uint4 *)pp.g[q] + vec);
-        const uint32_t gw[4] = {g.x, g.y, g.z, g.w};
+        for (int q = 0; q < R; q++) {
+            const uint4 g = __ldcs((const uint4 *)pp.g[q] + vec);
+            const uint32_t gw[4] = {g.x, g.y, g.z, g.w};
 #pragma unroll
-        for (int e = 0; e < 8; e++) {
-            const float x = h2f_bits_dp((e & 1) ? (gw[e >> 1] >> 16) : (gw[e >> 1] & 0xFFFFu));
-            s[e] = q == 0 ? x : __fadd_rn(s[e], x);
+            for (int e = 0; e < 8; e++) {
+                const float x = h2f_bits_dp((e & 1) ? (gw[e >> 1] >> 16) : (gw[e >> 1] & 0xFFFFu));
+                s[e] = q == 0 ? x : __fadd_rn(s[e], x);
+            }
         }
     }
     float4 w0 = __ldcs(w32 + 2 * j), w1 = __ldcs(w32 + 2 * j + 1);
@@ -210,7 +216,7 @@ __global__ void k_dp_step_opt_tail(const DpPeers pp, int R, float *__restrict__ 
                                    float *__restrict__ s2p, size_t first, size_t begin, size_t count, float inv,
                                    const float *__restrict__ S_dev, float lr, float mu, float b2, float eps, float wd,
                                    float b1t, float b2t, const float *__restrict__ betat_dev, uint32_t *flags,
-                                   const float *__restrict__ coef_dev)
+                                   const float *__restrict__ coef_dev, const float *__restrict__ sum32)
 {
     pdl_trigger();
     pdl_wait();
@@ -226,8 +232,13 @@ __global__ void k_dp_step_opt_tail(const DpPeers pp, int R, float *__restrict__ 
     const bool use_s1 = KIND != MPT_OPT_SGD || mu != 0.0f;
     bool bad = false;
     for (size_t i = begin + threadIdx.x; i < count; i += blockDim.x) {
-        float s = h2f_bits_dp(pp.g[0][first + i]);
-        for (int q = 1; q < R; q++) s = __fadd_rn(s, h2f_bits_dp(pp.g[q][first + i]));
+        float s;
+        if (sum32) {
+            s = sum32[i];
+        } else {
+            s = h2f_bits_dp(pp.g[0][first + i]);
+            for (int q = 1; q < R; q++) s = __fadd_rn(s, h2f_bits_dp(pp.g[q][first + i]));
+        }
         float w = w32[i], a = use_s1 ? s1p[i] : 0.0f, b = KIND == MPT_OPT_ADAM ? s2p[i] : 0.0f;
         opt1<KIND, WD>(s, w, a, b, inv, lr, mu, b2, omb1, omb2, eps, wd, bc1, bc2, coef, bad);
         w32[i] = w;
@@ -242,18 +253,45 @@ __global__ void k_dp_step_opt_tail(const DpPeers pp, int R, float *__restrict__ 
 template <int KIND, bool WD>
 cudaError_t launch_dp_opt(const DpPeers &pp, int R, float *w32, float *s1, float *s2, size_t first, size_t count, float inv,
                           const float *S_dev, float lr, float mu, float b2, float eps, float wd, float b1t, float b2t,
-                          const float *betat_dev, uint32_t *flags, cudaStream_t st, int *n_launches, const float *coef_dev)
+                          const float *betat_dev, uint32_t *flags, cudaStream_t st, int *n_launches, const float *coef_dev,
+                          const float *sum32)
 {
     const size_t n8 = count / 8;
     if (n_launches) *n_launches = (n8 ? 1 : 0) + (n8 * 8 < count || count == 0 ? 1 : 0);
     if (n8)
         MPT_LAUNCH(k_dp_step_opt<KIND, WD>, dim3((unsigned)((n8 + kDpThreads - 1) / kDpThreads)), dim3(kDpThreads), 0, st, pp, R,
                    (float4 *)w32, (float4 *)s1, (float4 *)s2, first, n8, inv, S_dev, lr, mu, b2, eps, wd, b1t, b2t, betat_dev,
-                   flags, coef_dev);
+                   flags, coef_dev, (const float4 *)sum32);
     if (n8 * 8 < count || count == 0)
         MPT_LAUNCH(k_dp_step_opt_tail<KIND, WD>, dim3(1), dim3(32), 0, st, pp, R, w32, s1, s2, first, n8 * 8, count, inv, S_dev,
-                   lr, mu, b2, eps, wd, b1t, b2t, betat_dev, flags, coef_dev);
+                   lr, mu, b2, eps, wd, b1t, b2t, betat_dev, flags, coef_dev, sum32);
     return cudaGetLastError();
+}
+
+// First half of the exchange by itself: the FP32 sum over the replicas, in replica order, of the elements
+// [first, first + count) of their FP16 gradient arrays (first and count multiples of 8), stored raw.  The
+// step kernels take such sums in place of the gradients (their sum32 argument), so the pull over the link
+// can run per layer beside the rest of the backward pass and the update after the overflow is known.
+__global__ void __launch_bounds__(kDpThreads) k_dp_reduce(const DpPeers pp, int R, size_t first, size_t n8, float4 *__restrict__ out)
+{
+    pdl_trigger();
+    pdl_wait();
+    const size_t j = (size_t)blockIdx.x * kDpThreads + threadIdx.x;
+    if (j >= n8) return;
+    const size_t vec = first / 8 + j;
+    float s[8];
+#pragma unroll 4
+    for (int q = 0; q < R; q++) {
+        const uint4 g = __ldcs((const uint4 *)pp.g[q] + vec);
+        const uint32_t gw[4] = {g.x, g.y, g.z, g.w};
+#pragma unroll
+        for (int e = 0; e < 8; e++) {
+            const float x = h2f_bits_dp((e & 1) ? (gw[e >> 1] >> 16) : (gw[e >> 1] & 0xFFFFu));
+            s[e] = q == 0 ? x : __fadd_rn(s[e], x);
+        }
+    }
+    out[2 * j] = make_float4(s[0], s[1], s[2], s[3]);
+    out[2 * j + 1] = make_float4(s[4], s[5], s[6], s[7]);
 }
 
 // ---- global-norm clipping of the mean gradient (section 3.2): sum of squares of this replica's shard
@@ -382,7 +420,7 @@ cudaError_t launch_dp_step_opt(int kind, const uint16_t *const *g16, const uint3
                                float *w32_shard, float *s1_shard, float *s2_shard, size_t first, size_t count, float inv_SR,
                                const float *S_dev, float lr, float mu, float b2, float eps, float wd, float b1t, float b2t,
                                const float *betat_dev, uint32_t *flags, cudaStream_t st, int *n_launches,
-                               const float *coef_dev)
+                               const float *coef_dev, const float *sum32)
 {
     DpPeers pp = {};
     for (int q = 0; q < R; q++) {
@@ -392,9 +430,9 @@ cudaError_t launch_dp_step_opt(int kind, const uint16_t *const *g16, const uint3
     }
 #define MPT_DP_OPT(KIND)                                                                                                    \
     (wd != 0.0f ? launch_dp_opt<KIND, true>(pp, R, w32_shard, s1_shard, s2_shard, first, count, inv_SR, S_dev, lr, mu, b2, eps, \
-                                            wd, b1t, b2t, betat_dev, flags, st, n_launches, coef_dev)                        \
+                                            wd, b1t, b2t, betat_dev, flags, st, n_launches, coef_dev, sum32)                 \
                 : launch_dp_opt<KIND, false>(pp, R, w32_shard, s1_shard, s2_shard, first, count, inv_SR, S_dev, lr, mu, b2,   \
-                                             eps, wd, b1t, b2t, betat_dev, flags, st, n_launches, coef_dev))
+                                             eps, wd, b1t, b2t, betat_dev, flags, st, n_launches, coef_dev, sum32))
     switch (kind) {
         case MPT_OPT_SGD: return MPT_DP_OPT(MPT_OPT_SGD);
         case MPT_OPT_NESTEROV: return MPT_DP_OPT(MPT_OPT_NESTEROV);
@@ -403,6 +441,18 @@ cudaError_t launch_dp_step_opt(int kind, const uint16_t *const *g16, const uint3
         default: return cudaErrorInvalidValue;
     }
 #undef MPT_DP_OPT
+}
+
+cudaError_t launch_dp_reduce(const uint16_t *const *g16, int R, size_t first, size_t count, float *sum32_out, cudaStream_t st)
+{
+    if ((first | count) & 7) return cudaErrorInvalidValue;
+    if (count == 0) return cudaSuccess;
+    DpPeers pp = {};
+    for (int q = 0; q < R; q++) pp.g[q] = g16[q];
+    const size_t n8 = count / 8;
+    MPT_LAUNCH(k_dp_reduce, dim3((unsigned)((n8 + kDpThreads - 1) / kDpThreads)), dim3(kDpThreads), 0, st, pp, R, first, n8,
+               (float4 *)sum32_out);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_dp_sqnorm(const uint16_t *const *g16, int R, size_t first, size_t count, float inv_SR, const float *S_dev,

@@ -177,6 +177,14 @@ struct mpt_ctx {
     // mpt_create_dp: FP32 master and optimizer state exist for this replica's shard only; master / mom /
     // state2 are then bases such that element i of the flat array is at [i] for i inside the shard
     int shard_R = 0, shard_rank = 0;
+    // overlapped exchange (mpt_dp_overlap_attach): the pull-and-sum of each layer's gradients runs on dp_stream
+    // as soon as that layer's weight gradient is complete on every replica (interprocess events)
+    bool dp_overlap = false, dp_reduced = false;
+    cudaStream_t dp_stream = nullptr;
+    std::vector<cudaEvent_t> ev_own;                      // per layer: this replica's weight gradient is complete
+    std::vector<cudaEvent_t> ev_peer[MPT_DP_MAX_REPLICAS]; // the same events of the other replicas, opened here
+    cudaEvent_t ev_reduced = nullptr;
+    float *sum32 = nullptr;                               // FP32 sums over the replicas, this replica's shard
     bool dp_norm_done = false;   // mpt_dp_norm has run since the last backward pass (clipping in data-parallel mode)
     const uint16_t *dp_g16[MPT_DP_MAX_REPLICAS] = {};
     const uint32_t *dp_flag[MPT_DP_MAX_REPLICAS] = {};
@@ -355,6 +363,7 @@ int do_backward(mpt_ctx *c, const int32_t *labels_dev)
         int r = gemm(c, MPT_OP_WGRAD, ly.out, ly.in, B, ly.dact, ly.ld_out, a_prev, ld_prev, c->g16 + ly.off, ly.in, false,
                      nullptr, 0, c->status + ST_OVERFLOW);
         if (r != MPT_OK) return r;
+        if (c->dp_overlap) CK(cudaEventRecord(c->ev_own[l], c->stream), "event record");
         if (l > 0) {
             Layer &pv = c->layers[l - 1];
             r = gemm(c, MPT_OP_DGRAD, B, ly.in, ly.out, ly.dact, ly.ld_out, c->w16 + ly.off, ly.in, pv.dact, pv.ld_out, false,
@@ -390,13 +399,24 @@ int do_step(mpt_ctx *c)
             if (e != cudaSuccess) return cuda_fail(c, e, "clip launch");
             c->dp_norm_done = false;
         }
+        const float *sums = nullptr;
+        if (c->dp_overlap) {
+            // the sums were formed on dp_stream (mpt_dp_reduce_async); the new weights may be written into a
+            // replica only when its whole backward pass is complete (its last event)
+            if (!c->dp_reduced) return fail(c, MPT_ERR_STATE, "overlapped exchange: call mpt_dp_reduce_async before mpt_step");
+            CK(cudaStreamWaitEvent(c->stream, c->ev_reduced, 0), "event wait");
+            for (int q = 0; q < c->dp_R; q++)
+                if (q != c->dp_rank) CK(cudaStreamWaitEvent(c->stream, c->ev_peer[q][0], 0), "event wait");
+            c->dp_reduced = false;
+            sums = c->sum32;
+        }
         {
             // bytes through this GPU's memory system: R gradients read, the shard's state, R weight copies written
             const double per_elem = 2.0 * c->dp_R + 8.0 + (c->use_momentum ? 8.0 : 0.0) + (c->state2 ? 8.0 : 0.0) + 2.0 * c->dp_R;
             ProfSpan span(c, MPT_PROF_UPDATE, per_elem * (double)(hi - lo));
             const float inv_SR = 1.0f / (c->S * (float)c->dp_R);
             const float *S_dev = (const float *)(c->status + ST_SCALE);
-            if (c->opt_kind == MPT_OPT_SGD && c->wd == 0.0f && c->clip <= 0.0f)
+            if (!sums && c->opt_kind == MPT_OPT_SGD && c->wd == 0.0f && c->clip <= 0.0f)
                 e = launch_dp_step(c->dp_g16, c->dp_flag, c->dp_w16, c->dp_R, c->master + lo, c->use_momentum ? c->mom + lo : nullptr,
                                    lo, hi - lo, inv_SR, S_dev, c->lr, c->use_momentum ? c->mu : 0.0f, c->status + ST_OVERFLOW,
                                    c->stream, &nl);
@@ -406,7 +426,7 @@ int do_step(mpt_ctx *c)
                                        S_dev, c->lr, c->mu, c->beta2, c->eps, c->wd, 1.0f, 1.0f,
                                        c->opt_kind == MPT_OPT_ADAM ? (const float *)(c->status + ST_B1T) : nullptr,
                                        c->status + ST_OVERFLOW, c->stream, &nl,
-                                       c->clip > 0.0f ? (const float *)(c->status + ST_CLIP_COEF) : nullptr);
+                                       c->clip > 0.0f ? (const float *)(c->status + ST_CLIP_COEF) : nullptr, sums);
         }
         c->launches += nl;
         if (e != cudaSuccess) return cuda_fail(c, e, "data-parallel step launch");
@@ -646,6 +666,10 @@ static int create_impl(const mpt_layer_desc *layers, int n_layers, float S, cons
 void mpt_destroy(mpt_ctx *c)
 {
     if (!c) return;
+    for (auto e : c->ev_own) if (e) cudaEventDestroy(e);
+    for (auto &v : c->ev_peer) for (auto e : v) if (e) cudaEventDestroy(e);
+    if (c->ev_reduced) cudaEventDestroy(c->ev_reduced);
+    if (c->dp_stream) cudaStreamDestroy(c->dp_stream);
     for (auto &sp : c->spans) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
     for (auto &sp : c->pool) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
     for (int k = 0; k < 2; k++) {
@@ -1102,6 +1126,81 @@ int mpt_dp_norm(mpt_ctx *c)
     c->launches += 2;
     if (e != cudaSuccess) return cuda_fail(c, e, "data-parallel norm launch");
     c->dp_norm_done = true;
+    return MPT_OK;
+}
+
+int mpt_dp_overlap_events(mpt_ctx *c, uint8_t *handles_out)
+{
+    static_assert(sizeof(cudaIpcEventHandle_t) == MPT_DP_HANDLE_BYTES, "handle size");
+    int r = usable(c);
+    if (r != MPT_OK) return r;
+    if (!handles_out) return fail(c, MPT_ERR_INVALID_ARG, "null output");
+    const size_t L = c->layers.size();
+    if (c->ev_own.empty()) {
+        c->ev_own.resize(L, nullptr);
+        for (size_t l = 0; l < L; l++)
+            CK(cudaEventCreateWithFlags(&c->ev_own[l], cudaEventDisableTiming | cudaEventInterprocess), "event create");
+    }
+    for (size_t l = 0; l < L; l++) {
+        cudaIpcEventHandle_t h;
+        CK(cudaIpcGetEventHandle(&h, c->ev_own[l]), "event export");
+        memcpy(handles_out + l * MPT_DP_HANDLE_BYTES, &h, MPT_DP_HANDLE_BYTES);
+    }
+    return MPT_OK;
+}
+
+int mpt_dp_overlap_attach(mpt_ctx *c, const uint8_t *const *peer_handles, float *sum32_dev, size_t sum32_bytes)
+{
+    int r = usable(c);
+    if (r != MPT_OK) return r;
+    if (c->dp_R < 2) return fail(c, MPT_ERR_STATE, "mpt_dp_overlap_attach needs an attached data-parallel context");
+    if (c->ev_own.empty()) return fail(c, MPT_ERR_STATE, "call mpt_dp_overlap_events first");
+    if (c->dp_overlap) return fail(c, MPT_ERR_STATE, "already attached");
+    if (c->clip > 0.0f) return fail(c, MPT_ERR_STATE, "global-norm clipping is not available with the overlapped exchange");
+    if (!peer_handles || !sum32_dev) return fail(c, MPT_ERR_INVALID_ARG, "null argument");
+    size_t lo = 0, hi = 0;
+    mpt_dp_shard(c->plan.P_pad, c->dp_R, c->dp_rank, &lo, &hi);
+    if (sum32_bytes < (hi - lo) * 4 || ((uintptr_t)sum32_dev & 15)) return fail(c, MPT_ERR_WORKSPACE, "scratch for the sums too small or misaligned");
+    const size_t L = c->layers.size();
+    for (int q = 0; q < c->dp_R; q++) {
+        if (q == c->dp_rank) continue;
+        if (!peer_handles[q]) return fail(c, MPT_ERR_INVALID_ARG, "null peer handles");
+        c->ev_peer[q].assign(L, nullptr);
+        for (size_t l = 0; l < L; l++) {
+            cudaIpcEventHandle_t h;
+            memcpy(&h, peer_handles[q] + l * MPT_DP_HANDLE_BYTES, MPT_DP_HANDLE_BYTES);
+            CK(cudaIpcOpenEventHandle(&c->ev_peer[q][l], h), "event open");
+        }
+    }
+    CK(cudaStreamCreateWithFlags(&c->dp_stream, cudaStreamNonBlocking), "stream create");
+    CK(cudaEventCreateWithFlags(&c->ev_reduced, cudaEventDisableTiming), "event create");
+    c->sum32 = sum32_dev;
+    c->dp_overlap = true;
+    c->dp_reduced = false;
+    return MPT_OK;
+}
+
+int mpt_dp_reduce_async(mpt_ctx *c)
+{
+    int r = usable(c);
+    if (r != MPT_OK) return r;
+    if (!c->dp_overlap) return fail(c, MPT_ERR_STATE, "mpt_dp_reduce_async needs mpt_dp_overlap_attach");
+    if (!c->have_grads) return fail(c, MPT_ERR_STATE, "mpt_dp_reduce_async needs gradients (mpt_backward_scaled or mpt_set_grad)");
+    size_t lo = 0, hi = 0;
+    mpt_dp_shard(c->plan.P_pad, c->dp_R, c->dp_rank, &lo, &hi);
+    const int L = (int)c->layers.size();
+    for (int l = L - 1; l >= 0; l--) {      // the order in which the backward pass completes the layers
+        const size_t a0 = c->layers[l].off, b0 = l + 1 < L ? c->layers[l + 1].off : c->plan.P_pad;   // with the padding after it
+        const size_t a = a0 > lo ? a0 : lo, b = b0 < hi ? b0 : hi;
+        if (a >= b) continue;
+        for (int q = 0; q < c->dp_R; q++)
+            CK(cudaStreamWaitEvent(c->dp_stream, q == c->dp_rank ? c->ev_own[l] : c->ev_peer[q][l], 0), "event wait");
+        cudaError_t e = launch_dp_reduce(c->dp_g16, c->dp_R, a, b - a, c->sum32 + (a - lo), c->dp_stream);
+        c->launches++;
+        if (e != cudaSuccess) return cuda_fail(c, e, "reduce launch");
+    }
+    CK(cudaEventRecord(c->ev_reduced, c->dp_stream), "event record");
+    c->dp_reduced = true;
     return MPT_OK;
 }
 

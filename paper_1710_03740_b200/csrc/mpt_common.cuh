@@ -150,7 +150,11 @@ cudaError_t launch_dp_step_opt(int kind, const uint16_t *const *g16, const uint3
                                float *w32_shard, float *s1_shard, float *s2_shard, size_t first, size_t count, float inv_SR,
                                const float *S_dev, float lr, float mu, float b2, float eps, float wd, float b1t, float b2t,
                                const float *betat_dev, uint32_t *flags, cudaStream_t st, int *n_launches,
-                               const float *coef_dev = nullptr);
+                               const float *coef_dev = nullptr, const float *sum32 = nullptr);
+// The FP32 sums over the replicas of elements [first, first + count) of their gradient arrays (multiples of
+// 8), stored at sum32_out[0 .. count); launch_dp_step_opt takes them through its sum32 argument (indexed
+// like w32_shard) in place of the gradients.
+cudaError_t launch_dp_reduce(const uint16_t *const *g16, int R, size_t first, size_t count, float *sum32_out, cudaStream_t st);
 // Clipping in the data-parallel step: this replica's shard of the sum of squares of the mean unscaled
 // gradient (double) into *slot (parts: scratch of kDpNormScratch doubles); then, once every replica
 // has published its slot, out2[0] = coefficient, out2[1] = norm from all R slots in replica order.

@@ -343,7 +343,7 @@ def _mlp_batch(t, q):
     return x, y
 
 
-def _mlp_replica_main(rank, R, port, out_dir, dynamic=False, opt_kind=0, clip=0.0, shard_state=False):
+def _mlp_replica_main(rank, R, port, out_dir, dynamic=False, opt_kind=0, clip=0.0, shard_state=False, overlap=False):
     import datetime
     import torch as th
     import torch.distributed as dist
@@ -354,7 +354,7 @@ def _mlp_replica_main(rank, R, port, out_dir, dynamic=False, opt_kind=0, clip=0.
     try:
         opt = b.Optimizer(opt_kind, _MLP["lr"], _MLP["mu"], 0.999, 1e-8, 0.001, clip) if (opt_kind or clip) else None
         dp = b.DataParallelMLP(_MLP_LAYERS, _MLP["S"], _MLP["lr"], _MLP["mu"], max_batch=_MLP["batch"], optimizer=opt,
-                               shard_state=shard_state)
+                               shard_state=shard_state, overlap=overlap)
         L = len(_MLP_LAYERS)
         for l, w in enumerate(_mlp_masters()):
             dp.ctx.set_master(l, w)
@@ -373,10 +373,20 @@ def _mlp_replica_main(rank, R, port, out_dir, dynamic=False, opt_kind=0, clip=0.
         for t in range(_MLP["e2e_steps"]):
             x, y = _mlp_batch(t, rank)
             dp.ctx.forward(th.from_numpy(x.view(np.int16)).cuda())
-            rec["e2e_loss_%d" % t] = np.array(dp.ctx.backward_scaled(th.from_numpy(y).cuda()))
-            for l in range(L):
-                rec["e2e_g16_%d_%d" % (t, l)] = dp.ctx.get_tensor(b.T_GRAD16, l)
-            rec["e2e_skip_%d" % t] = np.array(dp.step())
+            if overlap and t % 2 == 0:
+                # the pass is only enqueued: the exchange of the last layers runs while the first are still being
+                # differentiated; the gradients are read back after the step (the step does not change them)
+                yd = th.from_numpy(y).cuda()
+                dp.ctx.backward_scaled(yd, want_loss=False)
+                rec["e2e_skip_%d" % t] = np.array(dp.step())
+                rec["e2e_loss_%d" % t] = np.array(np.nan)
+                for l in range(L):
+                    rec["e2e_g16_%d_%d" % (t, l)] = dp.ctx.get_tensor(b.T_GRAD16, l)
+            else:
+                rec["e2e_loss_%d" % t] = np.array(dp.ctx.backward_scaled(th.from_numpy(y).cuda()))
+                for l in range(L):
+                    rec["e2e_g16_%d_%d" % (t, l)] = dp.ctx.get_tensor(b.T_GRAD16, l)
+                rec["e2e_skip_%d" % t] = np.array(dp.step())
             if clip > 0.0:
                 rec["e2e_norm_coef_%d" % t] = np.array(dp.ctx.get_grad_norm(), dtype=np.float32)
             for l in range(L):
@@ -515,6 +525,80 @@ def test_dp_mlp_two_processes_shard_only_state(tmp_path, kind):
     saved = full.workspace_bytes - int(rec[0]["workspace_bytes"])
     assert abs(saved - n_states * 4 * (n - n // R)) <= n_states * (256 + 32 * R), (saved, n, n_states)
     full.close()
+
+
+@pytest.mark.timeout(300)
+@pytest.mark.parametrize("kind,shard_state", [(0, False), (2, True)])
+def test_dp_mlp_two_processes_overlapped_exchange(tmp_path, kind, shard_state):
+    """The exchange overlapped with the backward pass: per-layer interprocess events, the sums of each
+    layer's gradients formed on a second stream as soon as that layer is complete on both replicas, the
+    step from the sums once both passes are complete.  Same bits as the one-kernel exchange: FP16 weights
+    of both replicas against the oracle's replicas through injected steps (one skipped) and whole
+    iterations, half of them with the backward pass only enqueued when the exchange is issued."""
+    import torch.multiprocessing as mp
+    from oracle.dp import OracleDataParallelMLP
+    R = 2
+    mp.spawn(_mlp_replica_main, args=(R, _free_port(), str(tmp_path), False, kind, 0.0, shard_state, True), nprocs=R, join=True)
+    rec = [np.load(os.path.join(str(tmp_path), "m%d.npz" % q)) for q in range(R)]
+    L = len(_MLP_LAYERS)
+    ora = OracleDataParallelMLP(_MLP_LAYERS, _MLP["S"], _MLP["lr"], _MLP["mu"], R)
+    if kind:
+        ora.set_optimizer(kind, _MLP["lr"], _MLP["mu"], 0.999, 1e-8, 0.001)
+    for l, w in enumerate(_mlp_masters()):
+        ora.set_master(l, w)
+    for t in range(_MLP["inj_steps"]):
+        for q in range(R):
+            for l in range(L):
+                ora.set_grad(q, l, _mlp_injected_grad(t, q, l).view(np.uint16))
+        skipped = ora.step()
+        assert skipped == (1 if t == 1 else 0)
+        for l in range(L):
+            want16, want32 = ora.replicas[0].w16[l], ora.replicas[0].w32[l]
+            for q in range(R):
+                assert bool(rec[q]["inj_skip_%d" % t]) == bool(skipped)
+                assert np.array_equal(rec[q]["inj_w16_%d_%d" % (t, l)].reshape(want16.shape), want16), (t, l, q)
+                first, count = (int(x) for x in rec[q]["state_ranges"][l])
+                if shard_state:
+                    got = rec[q]["inj_w32_%d_%d" % (t, l)].reshape(-1)[first:first + count]
+                    assert np.array_equal(got.view(np.uint32), want32.reshape(-1)[first:first + count].view(np.uint32))
+    for t in range(_MLP["e2e_steps"]):
+        xs, ys = zip(*[_mlp_batch(t, q) for q in range(R)])
+        losses = ora.forward_backward(list(xs), list(ys))
+        for q in range(R):
+            got = float(rec[q]["e2e_loss_%d" % t])
+            assert np.isnan(got) == (t % 2 == 0)
+            if not np.isnan(got):
+                assert abs(got - losses[q]) <= 1e-3 * abs(losses[q]), (t, q, got, losses[q])
+            for l in range(L):
+                ora.set_grad(q, l, rec[q]["e2e_g16_%d_%d" % (t, l)])
+        skipped = ora.step()
+        for q in range(R):
+            assert bool(rec[q]["e2e_skip_%d" % t]) == bool(skipped)
+            for l in range(L):
+                want16 = ora.replicas[0].w16[l]
+                assert np.array_equal(rec[q]["e2e_w16_%d_%d" % (t, l)].reshape(want16.shape), want16), (t, l, q)
+
+
+def test_overlapped_exchange_error_paths():
+    """The overlapped exchange needs an attached context, its events before the attach, and a call of
+    mpt_dp_reduce_async; a context that is none of that says so and stays usable."""
+    require_gpu()
+    from paper_1710_03740_b200 import binding as b
+    ctx = b.Context(_MLP_LAYERS, _MLP["S"], _MLP["lr"], _MLP["mu"], max_batch=_MLP["batch"])
+    with pytest.raises(b.MptError) as e:
+        ctx.dp_reduce_async()
+    assert e.value.code == -3
+    handles = ctx.dp_overlap_events()
+    assert len(handles) == len(_MLP_LAYERS) * b.DP_HANDLE_BYTES and handles == ctx.dp_overlap_events()
+    with pytest.raises(b.MptError) as e:
+        ctx.dp_overlap_attach([handles, handles], 0)        # not attached to any replica
+    assert e.value.code == -3
+    for l, w in enumerate(_mlp_masters()):
+        ctx.set_master(l, w)
+    for l in range(len(_MLP_LAYERS)):
+        ctx.set_grad(l, _mlp_injected_grad(0, 0, l).view(np.uint16))
+    assert ctx.step() == 0                                   # the ordinary single-GPU step still works
+    ctx.close()
 
 
 def test_shard_only_context_refuses_what_it_cannot_do():
