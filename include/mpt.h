@@ -25,6 +25,8 @@
  *     workspace, the inputs, the stream and all host buffers; the library owns only its
  *     host-side context object.  Exceptions, each documented at its declaration:
  *     mpt_dp_alloc / mpt_dp_free obtain and release device memory from the driver;
+ *     mpt_dp_overlap_events / mpt_dp_overlap_attach create events and one more stream, which
+ *     mpt_destroy releases;
  *     mpt_softmax_ce_static uses a fixed device array inside the library that all calls on a
  *     GPU share; and the launchers keep small per-device host-side caches that are filled on
  *     first use (SM count, opt-in shared-memory sizes, cluster occupancy, the address of that

@@ -5,7 +5,9 @@
 // applies the update of sections 3.1 / 3.2 to its FP32 master shard, and pushes the re-rounded FP16
 // weights into every replica's working copy.  Plain loads and stores on peer pointers only: no
 // waits on other replicas inside the kernel (the caller orders the replicas around the call), no
-// multicast.  Arithmetic contract: include/mpt.h (mpt_dp_step_flat).
+// multicast.  Arithmetic contract: include/mpt.h (mpt_dp_step_flat).  k_dp_reduce is the first half (pull
+// and sum) by itself, for running it layer by layer beside the backward pass; the step kernels then take
+// the sums in place of the gradients.
 #include <string.h>
 
 #include "mpt_common.cuh"
