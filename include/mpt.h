@@ -682,20 +682,24 @@ int mpt_state_range(mpt_ctx *ctx, int layer, size_t *first_out, size_t *count_ou
  * the master pass and the weight broadcast once the whole pass - and with it the overflow decision of
  * section 3.2 - is complete on every replica.  The arithmetic is that of mpt_dp_step_flat_opt (FP32 sum in
  * replica order, then the step), so the results are the same bits as without the overlap.
- *   mpt_dp_overlap_events: creates, once, one interprocess event per layer on this context and writes
- *     their handles (n_layers x MPT_DP_HANDLE_BYTES, HOST) for the other replicas; mpt_backward_scaled then
+ *   mpt_dp_overlap_events: creates, once, one interprocess event per layer (and one more, see below) on this
+ *     context and writes their handles ((n_layers + 1) x MPT_DP_HANDLE_BYTES, HOST) for the other replicas; mpt_backward_scaled then
  *     records event l on the context's stream after layer l's weight-gradient product.
  *   mpt_dp_overlap_attach: peer_handles = HOST array of R pointers to the other replicas' handle blocks
  *     (entry `rank` ignored); sum32_dev = DEVICE scratch of at least 4 bytes per element of this replica's
  *     shard (16-byte aligned, owned by the caller, must outlive the context's use of it).  Creates a second
- *     stream.  Not with global-norm clipping (MPT_ERR_STATE).
+ *     stream.  The handle blocks have n_layers + 1 entries: the last event marks the publication of this
+ *     replica's part of the gradient norm (global-norm clipping).
  *   mpt_dp_reduce_async: enqueues, on the second stream, for each layer from the last to the first: waits
  *     on that layer's event of every replica, then the sum of the part of the layer inside this replica's
  *     shard.  Call it after mpt_backward_scaled has RETURNED on every replica (a host-side ordering point
  *     that need not wait for the GPUs: pass loss_host_or_null = NULL to mpt_backward_scaled so that it does
  *     not synchronise) - an event wait refers to the latest record enqueued before it.
- *   mpt_step then waits (on the stream) for the sums and for every replica's last event, and runs the step
- *     from the sums.  MPT_ERR_STATE if mpt_dp_reduce_async has not been called since the last step.
+ *     With global-norm clipping it also forms, from the sums, this replica's part of the squared norm of
+ *     the mean gradient (as mpt_dp_norm does), publishes it and records the extra event; mpt_step must then be
+ *     called after mpt_dp_reduce_async has RETURNED on every replica (one more host-side ordering point).
+ *   mpt_step then waits (on the stream) for the sums and for every replica's last event (and norm event), and
+ *     runs the step from the sums.  MPT_ERR_STATE if mpt_dp_reduce_async has not been called since the last step.
  * After mpt_step the replicas are ordered as for mpt_dp_attach.  Works with ordinary contexts and with
  * those of mpt_create_dp. */
 int mpt_dp_overlap_events(mpt_ctx *ctx, uint8_t *handles_out);

@@ -272,7 +272,7 @@ class Context:
 
     def dp_overlap_events(self):
         """Handles of this context's per-layer events (bytes) for the other replicas."""
-        buf = (C.c_uint8 * (len(self.layers) * DP_HANDLE_BYTES))()
+        buf = (C.c_uint8 * ((len(self.layers) + 1) * DP_HANDLE_BYTES))()
         _check(lib().mpt_dp_overlap_events(self._ctx, buf), self._ctx)
         return bytes(buf)
 
@@ -876,6 +876,8 @@ class DataParallelMLP:
             import torch.distributed as dist
             dist.barrier(group=self.group)      # every replica has ENQUEUED its backward pass; nobody waits for a GPU here
             self.ctx.dp_reduce_async()
+            if self.ctx.optimizer.clip_norm > 0.0:
+                dist.barrier(group=self.group)  # every replica has enqueued the publication of its part of the norm
             overflow = self.ctx.step()          # waits on the streams for the sums and for every replica's pass
             self._barrier()
             return bool(overflow)

@@ -316,7 +316,8 @@ __device__ __forceinline__ double dp_block_sum_fixed(double v, double *sh)
 }
 
 __global__ void __launch_bounds__(kDpThreads) k_dp_sqnorm(const DpPeers pp, int R, size_t first, size_t count, float inv,
-                                                          const float *__restrict__ S_dev, double *__restrict__ parts)
+                                                          const float *__restrict__ S_dev, double *__restrict__ parts,
+                                                          const float *__restrict__ sum32)
 {
     pdl_trigger();
     pdl_wait();
@@ -327,13 +328,18 @@ __global__ void __launch_bounds__(kDpThreads) k_dp_sqnorm(const DpPeers pp, int 
     for (size_t j = (size_t)blockIdx.x * kDpThreads + threadIdx.x; j < n8; j += stride) {
         const size_t vec = first / 8 + j;
         float s[8];
-        for (int q = 0; q < R; q++) {
-            const uint4 g = __ldcs((const uint4 *)pp.g[q] + vec);
-            const uint32_t gw[4] = {g.x, g.y, g.z, g.w};
+        if (sum32) {      // sums formed earlier by k_dp_reduce
+            const float4 x0 = __ldcs((const float4 *)sum32 + 2 * j), x1 = __ldcs((const float4 *)sum32 + 2 * j + 1);
+            s[0] = x0.x; s[1] = x0.y; s[2] = x0.z; s[3] = x0.w; s[4] = x1.x; s[5] = x1.y; s[6] = x1.z; s[7] = x1.w;
+        } else {
+            for (int q = 0; q < R; q++) {
+                const uint4 g = __ldcs((const uint4 *)pp.g[q] + vec);
+                const uint32_t gw[4] = {g.x, g.y, g.z, g.w};
 #pragma unroll
-            for (int e = 0; e < 8; e++) {
-                const float x = h2f_bits_dp((e & 1) ? (gw[e >> 1] >> 16) : (gw[e >> 1] & 0xFFFFu));
-                s[e] = q == 0 ? x : __fadd_rn(s[e], x);
+                for (int e = 0; e < 8; e++) {
+                    const float x = h2f_bits_dp((e & 1) ? (gw[e >> 1] >> 16) : (gw[e >> 1] & 0xFFFFu));
+                    s[e] = q == 0 ? x : __fadd_rn(s[e], x);
+                }
             }
         }
 #pragma unroll
@@ -344,8 +350,13 @@ __global__ void __launch_bounds__(kDpThreads) k_dp_sqnorm(const DpPeers pp, int 
     }
     if (blockIdx.x == 0)      // the up to seven elements after the shard's last whole vector
         for (size_t i = n8 * 8 + threadIdx.x; i < count; i += kDpThreads) {
-            float s = h2f_bits_dp(pp.g[0][first + i]);
-            for (int q = 1; q < R; q++) s = __fadd_rn(s, h2f_bits_dp(pp.g[q][first + i]));
+            float s;
+            if (sum32) {
+                s = sum32[i];
+            } else {
+                s = h2f_bits_dp(pp.g[0][first + i]);
+                for (int q = 1; q < R; q++) s = __fadd_rn(s, h2f_bits_dp(pp.g[q][first + i]));
+            }
             const double v = (double)__fmul_rn(s, inv);
             acc += v * v;
         }
@@ -458,13 +469,13 @@ cudaError_t launch_dp_reduce(const uint16_t *const *g16, int R, size_t first, si
 }
 
 cudaError_t launch_dp_sqnorm(const uint16_t *const *g16, int R, size_t first, size_t count, float inv_SR, const float *S_dev,
-                             double *parts, double *slot, cudaStream_t st)
+                             double *parts, double *slot, cudaStream_t st, const float *sum32)
 {
     DpPeers pp = {};
     for (int q = 0; q < R; q++) pp.g[q] = g16[q];
     size_t want = (count / 8 + kDpThreads - 1) / kDpThreads;
     const int grid = (int)(want < 1 ? 1 : (want > (size_t)kDpNormParts ? (size_t)kDpNormParts : want));
-    MPT_LAUNCH(k_dp_sqnorm, dim3(grid), dim3(kDpThreads), 0, st, pp, R, first, count, inv_SR, S_dev, parts);
+    MPT_LAUNCH(k_dp_sqnorm, dim3(grid), dim3(kDpThreads), 0, st, pp, R, first, count, inv_SR, S_dev, parts, sum32);
     MPT_LAUNCH(k_dp_norm_publish, dim3(1), dim3(1024), 0, st, (const double *)parts, grid, slot);
     return cudaGetLastError();
 }

@@ -388,6 +388,20 @@ int do_step(mpt_ctx *c)
         size_t lo = 0, hi = 0;
         mpt_dp_shard(c->plan.P_pad, c->dp_R, c->dp_rank, &lo, &hi);
         int nl = 0;
+        const float *sums = nullptr;
+        if (c->dp_overlap) {
+            // the sums were formed on dp_stream (mpt_dp_reduce_async); the new weights may be written into a
+            // replica only when its whole backward pass is complete (its last event)
+            if (!c->dp_reduced) return fail(c, MPT_ERR_STATE, "overlapped exchange: call mpt_dp_reduce_async before mpt_step");
+            CK(cudaStreamWaitEvent(c->stream, c->ev_reduced, 0), "event wait");
+            for (int q = 0; q < c->dp_R; q++)
+                if (q != c->dp_rank) CK(cudaStreamWaitEvent(c->stream, c->ev_peer[q][0], 0), "event wait");
+            if (c->clip > 0.0f)      // every replica's part of the norm is published
+                for (int q = 0; q < c->dp_R; q++)
+                    if (q != c->dp_rank) CK(cudaStreamWaitEvent(c->stream, c->ev_peer[q][c->layers.size()], 0), "event wait");
+            c->dp_reduced = false;
+            sums = c->sum32;
+        }
         if (c->clip > 0.0f) {
             // every replica adds all replicas' published shard sums in replica order: same coefficient everywhere
             if (!c->dp_norm_done)
@@ -398,17 +412,6 @@ int do_step(mpt_ctx *c)
             c->launches++;
             if (e != cudaSuccess) return cuda_fail(c, e, "clip launch");
             c->dp_norm_done = false;
-        }
-        const float *sums = nullptr;
-        if (c->dp_overlap) {
-            // the sums were formed on dp_stream (mpt_dp_reduce_async); the new weights may be written into a
-            // replica only when its whole backward pass is complete (its last event)
-            if (!c->dp_reduced) return fail(c, MPT_ERR_STATE, "overlapped exchange: call mpt_dp_reduce_async before mpt_step");
-            CK(cudaStreamWaitEvent(c->stream, c->ev_reduced, 0), "event wait");
-            for (int q = 0; q < c->dp_R; q++)
-                if (q != c->dp_rank) CK(cudaStreamWaitEvent(c->stream, c->ev_peer[q][0], 0), "event wait");
-            c->dp_reduced = false;
-            sums = c->sum32;
         }
         {
             // bytes through this GPU's memory system: R gradients read, the shard's state, R weight copies written
@@ -1135,7 +1138,7 @@ int mpt_dp_overlap_events(mpt_ctx *c, uint8_t *handles_out)
     int r = usable(c);
     if (r != MPT_OK) return r;
     if (!handles_out) return fail(c, MPT_ERR_INVALID_ARG, "null output");
-    const size_t L = c->layers.size();
+    const size_t L = c->layers.size() + 1;      // one per layer and one for the published norm (clipping)
     if (c->ev_own.empty()) {
         c->ev_own.resize(L, nullptr);
         for (size_t l = 0; l < L; l++)
@@ -1156,12 +1159,11 @@ int mpt_dp_overlap_attach(mpt_ctx *c, const uint8_t *const *peer_handles, float 
     if (c->dp_R < 2) return fail(c, MPT_ERR_STATE, "mpt_dp_overlap_attach needs an attached data-parallel context");
     if (c->ev_own.empty()) return fail(c, MPT_ERR_STATE, "call mpt_dp_overlap_events first");
     if (c->dp_overlap) return fail(c, MPT_ERR_STATE, "already attached");
-    if (c->clip > 0.0f) return fail(c, MPT_ERR_STATE, "global-norm clipping is not available with the overlapped exchange");
     if (!peer_handles || !sum32_dev) return fail(c, MPT_ERR_INVALID_ARG, "null argument");
     size_t lo = 0, hi = 0;
     mpt_dp_shard(c->plan.P_pad, c->dp_R, c->dp_rank, &lo, &hi);
     if (sum32_bytes < (hi - lo) * 4 || ((uintptr_t)sum32_dev & 15)) return fail(c, MPT_ERR_WORKSPACE, "scratch for the sums too small or misaligned");
-    const size_t L = c->layers.size();
+    const size_t L = c->layers.size() + 1;
     for (int q = 0; q < c->dp_R; q++) {
         if (q == c->dp_rank) continue;
         if (!peer_handles[q]) return fail(c, MPT_ERR_INVALID_ARG, "null peer handles");
@@ -1198,6 +1200,17 @@ int mpt_dp_reduce_async(mpt_ctx *c)
         cudaError_t e = launch_dp_reduce(c->dp_g16, c->dp_R, a, b - a, c->sum32 + (a - lo), c->dp_stream);
         c->launches++;
         if (e != cudaSuccess) return cuda_fail(c, e, "reduce launch");
+    }
+    if (c->clip > 0.0f) {
+        // this replica's part of the squared norm of the mean gradient, from the sums, published next to its
+        // overflow word; the event tells the other replicas when it is there
+        const float inv_SR = 1.0f / (c->S * (float)c->dp_R);
+        cudaError_t e = launch_dp_sqnorm(c->dp_g16, c->dp_R, lo, hi - lo, inv_SR, (const float *)(c->status + ST_SCALE), c->norm_parts,
+                                         (double *)(c->status + ST_DP_NORM), c->dp_stream, c->sum32);
+        c->launches += 2;
+        if (e != cudaSuccess) return cuda_fail(c, e, "norm launch");
+        CK(cudaEventRecord(c->ev_own[L], c->dp_stream), "event record");
+        c->dp_norm_done = true;
     }
     CK(cudaEventRecord(c->ev_reduced, c->dp_stream), "event record");
     c->dp_reduced = true;

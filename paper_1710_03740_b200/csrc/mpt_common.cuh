@@ -160,7 +160,7 @@ cudaError_t launch_dp_reduce(const uint16_t *const *g16, int R, size_t first, si
 // has published its slot, out2[0] = coefficient, out2[1] = norm from all R slots in replica order.
 static constexpr int kDpNormScratch = 592;
 cudaError_t launch_dp_sqnorm(const uint16_t *const *g16, int R, size_t first, size_t count, float inv_SR, const float *S_dev,
-                             double *parts, double *slot, cudaStream_t st);
+                             double *parts, double *slot, cudaStream_t st, const float *sum32 = nullptr);
 cudaError_t launch_dp_clip_coef(const double *const *slots, int R, float clip, float *out2, cudaStream_t st);
 // End-of-step bookkeeping on the device (one thread): dynamic loss scale (if interval > 0) and
 // Adam's running products beta^t (if adam != 0); both only move on a step that was applied.

@@ -528,22 +528,23 @@ def test_dp_mlp_two_processes_shard_only_state(tmp_path, kind):
 
 
 @pytest.mark.timeout(300)
-@pytest.mark.parametrize("kind,shard_state", [(0, False), (2, True)])
-def test_dp_mlp_two_processes_overlapped_exchange(tmp_path, kind, shard_state):
+@pytest.mark.parametrize("kind,shard_state,clip", [(0, False, 0.0), (2, True, 0.0), (2, False, 0.02)])
+def test_dp_mlp_two_processes_overlapped_exchange(tmp_path, kind, shard_state, clip):
     """The exchange overlapped with the backward pass: per-layer interprocess events, the sums of each
     layer's gradients formed on a second stream as soon as that layer is complete on both replicas, the
     step from the sums once both passes are complete.  Same bits as the one-kernel exchange: FP16 weights
     of both replicas against the oracle's replicas through injected steps (one skipped) and whole
-    iterations, half of them with the backward pass only enqueued when the exchange is issued."""
+    iterations, half of them with the backward pass only enqueued when the exchange is issued.  With
+    global-norm clipping the parts of the norm come from the sums and the coefficient has the oracle's bits."""
     import torch.multiprocessing as mp
     from oracle.dp import OracleDataParallelMLP
     R = 2
-    mp.spawn(_mlp_replica_main, args=(R, _free_port(), str(tmp_path), False, kind, 0.0, shard_state, True), nprocs=R, join=True)
+    mp.spawn(_mlp_replica_main, args=(R, _free_port(), str(tmp_path), False, kind, clip, shard_state, True), nprocs=R, join=True)
     rec = [np.load(os.path.join(str(tmp_path), "m%d.npz" % q)) for q in range(R)]
     L = len(_MLP_LAYERS)
     ora = OracleDataParallelMLP(_MLP_LAYERS, _MLP["S"], _MLP["lr"], _MLP["mu"], R)
     if kind:
-        ora.set_optimizer(kind, _MLP["lr"], _MLP["mu"], 0.999, 1e-8, 0.001)
+        ora.set_optimizer(kind, _MLP["lr"], _MLP["mu"], 0.999, 1e-8, 0.001, clip)
     for l, w in enumerate(_mlp_masters()):
         ora.set_master(l, w)
     for t in range(_MLP["inj_steps"]):
@@ -574,6 +575,9 @@ def test_dp_mlp_two_processes_overlapped_exchange(tmp_path, kind, shard_state):
         skipped = ora.step()
         for q in range(R):
             assert bool(rec[q]["e2e_skip_%d" % t]) == bool(skipped)
+            if clip > 0.0:
+                coef = np.float32(ora.replicas[0].last_coef)
+                assert np.float32(rec[q]["e2e_norm_coef_%d" % t][1]).view(np.uint32) == coef.view(np.uint32), (t, q)
             for l in range(L):
                 want16 = ora.replicas[0].w16[l]
                 assert np.array_equal(rec[q]["e2e_w16_%d_%d" % (t, l)].reshape(want16.shape), want16), (t, l, q)
@@ -589,7 +593,7 @@ def test_overlapped_exchange_error_paths():
         ctx.dp_reduce_async()
     assert e.value.code == -3
     handles = ctx.dp_overlap_events()
-    assert len(handles) == len(_MLP_LAYERS) * b.DP_HANDLE_BYTES and handles == ctx.dp_overlap_events()
+    assert len(handles) == (len(_MLP_LAYERS) + 1) * b.DP_HANDLE_BYTES and handles == ctx.dp_overlap_events()
     with pytest.raises(b.MptError) as e:
         ctx.dp_overlap_attach([handles, handles], 0)        # not attached to any replica
     assert e.value.code == -3
