@@ -257,25 +257,39 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                 constexpr int NCH = BLOCK_N / 64;                          // this set's half of the tile's columns
                 epilogue_lstm_tile(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BLOCK_N + set * NCH * 32), NCH,
                                    nb * BLOCK_N + set * NCH * 32, p.N, row, row_ok, crow, p.lstm);
-            } else
-#pragma unroll 1
-            for (int c = ((warp - 2) >> 2) * (BLOCK_N / 32 / EpiCfg<LSTM || WIDE>::SETS);
-                 c < (((warp - 2) >> 2) + 1) * (BLOCK_N / 32 / EpiCfg<LSTM || WIDE>::SETS); c++) {
-                uint32_t r[32];
-                tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BLOCK_N + c * 32), r);
-                tc_wait_ld();
-                const int col0 = nb * BLOCK_N + c * 32;
-                if (p.split_k > 1) {
-                    // raw FP32 partial sums; ldp is a multiple of 32, so a started chunk is always whole
-                    if (row_ok && col0 < p.ldp) {
-                        float4 *dst = (float4 *)(p.partial + ((size_t)part * p.M + row) * p.ldp + col0);
+            } else {
+                // two register sets: the tensor-memory load of the next 32 columns is in flight while the
+                // current ones are rounded and stored
+                constexpr int NCHW = BLOCK_N / 32 / EpiCfg<LSTM || WIDE>::SETS;
+                const int c_begin = ((warp - 2) >> 2) * NCHW, c_end = c_begin + NCHW;
+                const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BLOCK_N);
+                auto finish = [&](const uint32_t (&r)[32], int c) {
+                    const int col0 = nb * BLOCK_N + c * 32;
+                    if (p.split_k > 1) {
+                        // raw FP32 partial sums; ldp is a multiple of 32, so a started chunk is always whole
+                        if (row_ok && col0 < p.ldp) {
+                            float4 *dst = (float4 *)(p.partial + ((size_t)part * p.M + row) * p.ldp + col0);
 #pragma unroll
-                        for (int v = 0; v < 8; v++)
-                            dst[v] = make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
-                                                 __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
+                            for (int v = 0; v < 8; v++)
+                                dst[v] = make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
+                                                     __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
+                        }
+                    } else if (row_ok && col0 < p.N) {
+                        epilogue_store32(r, crow, mrow, col0, p.N, p.relu != 0, bad);
                     }
-                } else if (row_ok && col0 < p.N) {
-                    epilogue_store32(r, crow, mrow, col0, p.N, p.relu != 0, bad);
+                };
+                uint32_t ra[32], rb[32];
+                tc_ld32(t_row + (uint32_t)(c_begin * 32), ra);
+#pragma unroll 1
+                for (int c = c_begin; c < c_end; c += 2) {
+                    tc_wait_ld();
+                    if (c + 1 < c_end) tc_ld32(t_row + (uint32_t)((c + 1) * 32), rb);
+                    finish(ra, c);
+                    if (c + 1 < c_end) {
+                        tc_wait_ld();
+                        if (c + 2 < c_end) tc_ld32(t_row + (uint32_t)((c + 2) * 32), ra);
+                        finish(rb, c + 1);
+                    }
                 }
             }
             tc_fence_before();
