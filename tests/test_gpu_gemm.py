@@ -237,6 +237,22 @@ def test_cluster_split_is_the_automatic_choice_for_the_projection_shape():
         _check_tc(0, 256, 256, 64, kernel="split2")
 
 
+@pytest.mark.parametrize("M,N,K,same_as", [(1024, 768, 4096, "split4"), (1024, 1024, 4096, "split2"),
+                                            (512, 512, 2048, "split2"), (512, 512, 1984, "tc"), (2048, 1280, 2048, "tc")])
+def test_automatic_kernel_choice_around_the_split_thresholds(M, N, K, same_as):
+    """Which kernel the library picks by itself, shown by the bits: 12 tiles with K = 4096 take four
+    parts, 16 tiles two parts, 4 tiles with 32 k-blocks two parts, one k-block fewer or 40 tiles none
+    (single-CTA kernel) - each result equal to that kernel forced, and all within the acceptance rule."""
+    from paper_1710_03740_b200 import binding as b
+    assert b.mpt_gemm_workspace_bytes(0, M, N, K) == 0 or same_as == "tc"
+    auto, _, _, _ = _check_tc(0, M, N, K, seed=7, kernel="auto")
+    forced, _, _, _ = _check_tc(0, M, N, K, seed=7, kernel=same_as)
+    assert np.array_equal(auto, forced)
+    if same_as != "tc":
+        other, _, _, _ = _check_tc(0, M, N, K, seed=7, kernel="tc")
+        assert not np.array_equal(auto, other)          # a split sum rounds differently somewhere
+
+
 @pytest.mark.parametrize("kernel", ["tc", "pair"])
 @pytest.mark.parametrize("op", [0, 1, 2])
 def test_tc_gemm_run_to_run_identical(op, kernel):
