@@ -36,13 +36,15 @@ static constexpr int CTA_M = 128;          // rows per CTA (256 per pair)
 static constexpr int TILE_N = 256;         // columns per pair tile
 static constexpr int CTA_N = 128;          // columns of B each CTA loads
 static constexpr int BLOCK_K = 64, UMMA_K = 16;
-static constexpr int STAGES = 7;
+static constexpr int STAGES = 6;             // 7 stages are not faster inside the step; the seventh's 32 KB stage the output
+static constexpr int EPI_BOX_BYTES = 32 * 64 * 2;          // one box of the output: 32 rows x 64 columns of FP16
+static constexpr int EPI_BYTES = 8 * EPI_BOX_BYTES;        // two boxes for each of four epilogue warps
 static constexpr int A_STAGE_BYTES = CTA_M * BLOCK_K * 2;   // 16 KB
 static constexpr int B_STAGE_BYTES = CTA_N * BLOCK_K * 2;   // 16 KB
 static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
 static constexpr int MN_BOX_BYTES = 64 * BLOCK_K * 2;
 static constexpr int TMEM_COLS = 512;
-static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256;
+static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BYTES + 1024 + 256;
 
 // instruction descriptor without the N field (N >> 3 goes to bits 17..22)
 __host__ __device__ constexpr uint32_t make_idesc(bool a_mn, bool b_mn)
@@ -73,6 +75,7 @@ struct Params {
     // k_tail_reduce finishes those tiles.  tail_split == 1: off (half-width units instead).
     int tail_split;
     float *tail_partial;
+    int tma_store;                   // output of whole and half tiles through shared memory and tensor stores
     int hint_a, hint_b;              // L2 eviction priority of the operand loads (0 normal, 1 last, 2 first)
     LstmEpi lstm;                    // read only by the LSTM instantiation of the kernel
 };
@@ -149,19 +152,20 @@ struct EpiCfg {
 template <bool A_MN, bool B_MN, bool LSTM = false, bool WIDE = false>
 __global__ void __launch_bounds__(EpiCfg<LSTM || WIDE>::THREADS, 1)
 k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-           const __grid_constant__ CUtensorMap tmBh, const Params p)
+           const __grid_constant__ CUtensorMap tmBh, const __grid_constant__ CUtensorMap tmC, const Params p)
 {
     pdl_trigger();
-    if (threadIdx.x == 32) { prefetch_tensormap(&tmA); prefetch_tensormap(&tmB); prefetch_tensormap(&tmBh); }
+    if (threadIdx.x == 32) { prefetch_tensormap(&tmA); prefetch_tensormap(&tmB); prefetch_tensormap(&tmBh); prefetch_tensormap(&tmC); }
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
-    const uint32_t bars = base + STAGES * STAGE_BYTES;
+    const uint32_t epi_stage = base + STAGES * STAGE_BYTES;        // 1024-byte aligned boxes for the output stores
+    const uint32_t bars = epi_stage + EPI_BYTES;
     auto full_bar = [&](int s) { return bars + 8u * s; };
     auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
     auto accf_bar = [&](int b) { return bars + 8u * (2 * STAGES + b); };
     auto acce_bar = [&](int b) { return bars + 8u * (2 * STAGES + 2 + b); };
-    volatile uint32_t *tmem_slot = (volatile uint32_t *)(base_ptr + STAGES * STAGE_BYTES + 8 * (2 * STAGES + 4));
+    volatile uint32_t *tmem_slot = (volatile uint32_t *)(base_ptr + STAGES * STAGE_BYTES + EPI_BYTES + 8 * (2 * STAGES + 4));
     volatile uint32_t *abort_flag = tmem_slot + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -315,6 +319,7 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
         const int q = warp & 3;
         bool ok = true;
         int t = 0;
+        int boxes_sent = 0;          // tensor stores this warp has issued (lane 0 tracks their bulk groups)
         for (int u = pair_id; u < num_units && ok; u += num_pairs, t++) {
             const Unit w = unit_of(p, u, nkb);
             const int buf = t & 1;
@@ -371,6 +376,60 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
                                                         __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3])));
                     }
                 }
+            } else if (!(LSTM || WIDE) && p.tma_store) {
+                // Output through shared memory and tensor stores: each lane rounds its row's 64 values of a box
+                // (32 rows x 64 columns) into the swizzled layout the tensor map expects, one lane sends the box
+                // with one bulk tensor store - whole 128-byte lines instead of 16-byte pieces of 32 different
+                // rows per instruction.  Two boxes per warp: the store of one is read out while the next fills.
+                const int nbox = w.width / 64;
+                const int row0 = w.mb * (2 * CTA_M) + (int)rank * CTA_M + q * 32;
+                uint32_t acc_bits = 0;
+#pragma unroll 1
+                for (int bx = 0; bx < nbox; bx++, boxes_sent++) {
+                    const uint32_t box = epi_stage + (uint32_t)(((warp - 2) * 2 + (boxes_sent & 1)) * EPI_BOX_BYTES);
+                    if (lane == 0 && boxes_sent >= 2) bulk_wait_group_read<1>();     // the store before last has left this box
+                    __syncwarp();
+                    const int colb = w.nb * TILE_N + w.n_off + bx * 64;
+#pragma unroll
+                    for (int h = 0; h < 2; h++) {
+                        uint32_t r[32], hw[16];
+                        tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * TILE_N + bx * 64 + h * 32), r);
+                        tc_wait_ld();
+                        round_pack32(r, p.relu != 0, hw);
+                        const int col0 = colb + h * 32;
+                        if (mrow && row_ok) {
+#pragma unroll
+                            for (int g8 = 0; g8 < 4; g8++) {
+                                if (col0 + g8 * 8 + 8 <= p.N) {
+                                    const uint4 mk = *(const uint4 *)(mrow + col0 + g8 * 8);
+                                    hw[4 * g8] = mask_pair(hw[4 * g8], mk.x);
+                                    hw[4 * g8 + 1] = mask_pair(hw[4 * g8 + 1], mk.y);
+                                    hw[4 * g8 + 2] = mask_pair(hw[4 * g8 + 2], mk.z);
+                                    hw[4 * g8 + 3] = mask_pair(hw[4 * g8 + 3], mk.w);
+                                }
+                            }
+                        }
+#pragma unroll
+                        for (int g8 = 0; g8 < 4; g8++) {
+                            // values outside the matrix are not stored (the tensor store clips) and must not vote
+                            if (row_ok && col0 + g8 * 8 + 8 <= p.N) {
+#pragma unroll
+                                for (int e = 0; e < 4; e++) nonfinite_acc(hw[4 * g8 + e], acc_bits);
+                            }
+                            const uint32_t piece = (uint32_t)((h * 4 + g8) ^ (lane & 7));      // 128-byte swizzle
+                            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(box + (uint32_t)(lane * 128) + (piece << 4)),
+                                         "r"(hw[4 * g8]), "r"(hw[4 * g8 + 1]), "r"(hw[4 * g8 + 2]), "r"(hw[4 * g8 + 3])
+                                         : "memory");
+                        }
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the tensor store reads what the lanes wrote
+                    __syncwarp();
+                    if (lane == 0) {      // a group per box, also when the box lies outside the matrix: the wait above counts groups
+                        if (row0 < p.M && colb < p.N) tma_store_2d(&tmC, box, colb, row0);
+                        bulk_commit_group();
+                    }
+                }
+                bad |= nonfinite_any(acc_bits);
             } else {
                 const int set = (warp - 2) >> 2, nch = w.width / 32 / EpiCfg<LSTM || WIDE>::SETS;   // this set's share of the columns
 #pragma unroll 1
@@ -387,6 +446,7 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
             if (lane == 0) mbar_arrive_cluster(mapa_u32(acce_bar(buf), 0));
             if (p.nonfinite_flag && __any_sync(0xFFFFFFFFu, bad) && lane == 0) atomicOr(p.nonfinite_flag, 1u);
         }
+        if (lane == 0) bulk_wait_group_read<0>();      // shared memory must outlive the tensor stores that read it
     }
 
     // common exit: all waits above are bounded, so both CTAs of the pair arrive here; neither
@@ -442,8 +502,8 @@ __global__ void __launch_bounds__(256) k_tail_reduce(const Params p, int first_t
 }
 
 template <bool A_MN, bool B_MN, bool LSTM = false, bool WIDE = false>
-static cudaError_t launch_variant(const CUtensorMap &ta, const CUtensorMap &tb, const CUtensorMap &tbh, Params p,
-                                  cudaStream_t st)
+static cudaError_t launch_variant(const CUtensorMap &ta, const CUtensorMap &tb, const CUtensorMap &tbh, const CUtensorMap &tc,
+                                  Params p, cudaStream_t st)
 {
     static int max_pairs_dev[kMaxDevices] = {};     // 0 = this device not configured yet
     auto kern = k_gemm_tc2<A_MN, B_MN, LSTM, WIDE>;
@@ -511,7 +571,7 @@ static cudaError_t launch_variant(const CUtensorMap &ta, const CUtensorMap &tb, 
     const int grid_pairs = p.num_units < max_pairs ? p.num_units : max_pairs;
     cfg.gridDim = dim3(2 * grid_pairs, 1, 1);
     cfg.numAttrs = 2;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, ta, tb, tbh, p);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, ta, tb, tbh, tc, p);
     if (e != cudaSuccess || p.split_k > 1 || p.tail_split <= 1) return e;
     const size_t work = (size_t)rest * (2 * CTA_M) * (TILE_N / 8);
     size_t blocks = (work + 255) / 256;
@@ -600,10 +660,15 @@ cudaError_t launch_gemm_tc2(int op, int M, int N, int K, const uint16_t *A, int 
         ok = ok && tc_encode_map(&tb, B, (uint64_t)K, (uint64_t)N, (uint64_t)ldb, 64, BLOCK_K);
         tbh = tb;
     }
+    CUtensorMap tcm;      // the output, in boxes of 32 rows x 64 columns
+    ok = ok && tc_encode_map(&tcm, C, (uint64_t)M, (uint64_t)N, (uint64_t)ldc, 64, 32);
     if (!ok) return cudaErrorInvalidValue;
     Params p;
     p.M = M; p.N = N; p.K = K;
     p.C = C; p.ldc = ldc;
+    // tensor stores of the output: whole groups of 8 columns only (the mask and the inf/NaN vote work on such groups);
+    // MPT_TMA_STORE=0 selects the per-lane 16-byte stores for comparisons
+    { const char *x = getenv("MPT_TMA_STORE"); p.tma_store = (N % 8 == 0) && (x ? atoi(x) != 0 : true); }
     p.mask = mask; p.ldmask = ldmask;
     p.relu = relu ? 1 : 0;
     p.nonfinite_flag = nonfinite_flag;
@@ -651,16 +716,16 @@ cudaError_t launch_gemm_tc2(int op, int M, int N, int K, const uint16_t *A, int 
     if (lstm) {
         if (op != MPT_OP_FWD || (N & 31) != 0) return cudaErrorInvalidValue;
         p.lstm = *lstm;
-        return launch_variant<false, false, true>(ta, tb, tbh, p, st);
+        return launch_variant<false, false, true>(ta, tb, tbh, tcm, p, st);
     }
     // two epilogue warp sets when a cluster's whole main loop is short (see EpiCfg)
     const long units = (long)p.tiles_m * p.tiles_n * p.split_k;
     const long kblocks = ((units + 73) / 74) * ((K + BLOCK_K - 1) / BLOCK_K / p.split_k);
     const bool wide = kblocks <= 160;
     cudaError_t e;
-    if (op == MPT_OP_FWD) e = wide ? launch_variant<false, false, false, true>(ta, tb, tbh, p, st) : launch_variant<false, false>(ta, tb, tbh, p, st);
-    else if (op == MPT_OP_DGRAD) e = wide ? launch_variant<false, true, false, true>(ta, tb, tbh, p, st) : launch_variant<false, true>(ta, tb, tbh, p, st);
-    else e = wide ? launch_variant<true, true, false, true>(ta, tb, tbh, p, st) : launch_variant<true, true>(ta, tb, tbh, p, st);
+    if (op == MPT_OP_FWD) e = wide ? launch_variant<false, false, false, true>(ta, tb, tbh, tcm, p, st) : launch_variant<false, false>(ta, tb, tbh, tcm, p, st);
+    else if (op == MPT_OP_DGRAD) e = wide ? launch_variant<false, true, false, true>(ta, tb, tbh, tcm, p, st) : launch_variant<false, true>(ta, tb, tbh, tcm, p, st);
+    else e = wide ? launch_variant<true, true, false, true>(ta, tb, tbh, tcm, p, st) : launch_variant<true, true>(ta, tb, tbh, tcm, p, st);
     if (e != cudaSuccess || p.split_k == 1) return e;
     return launch_splitk_reduce(p.partial, p.split_k, M, N, p.ldp, C, ldc, relu, mask, ldmask, nonfinite_flag, st);
 }

@@ -532,6 +532,22 @@ __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap
         ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(cluster_bar)
         : "memory");
 }
+// Tensor store of one box from this CTA's shared memory (layout as the tensor map's swizzle mode says) to
+// global memory; parts of the box outside the tensor are not written.  x (the inner coordinate) times the
+// element size must be a multiple of 16 bytes, and no coordinate may be negative.  Completion is tracked by
+// the issuing thread's bulk groups.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, uint32_t src, int x, int y)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];" ::"l"(map), "r"(x), "r"(y), "r"(src)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// waits until all but the N most recent bulk groups of this thread have finished READING shared memory
+template <int N>
+__device__ __forceinline__ void bulk_wait_group_read()
+{
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
 // The same load with an L2 eviction-priority hint (policy from l2_policy()).  Operand lines marked
 // "evict last" outlive the output stores and the other kernels' streams in L2: inside the large-MLP step
 // the products run 2-2.5 % faster with both operands marked (an operand one product has just read, or

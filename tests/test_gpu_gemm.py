@@ -270,6 +270,32 @@ def test_pair_kernel_runs_many_tiles_per_cluster():
 
 
 @pytest.mark.parametrize("op", [0, 1, 2])
+def test_pair_kernel_tensor_store_epilogue(op):
+    """Long main loops take the epilogue that stages 32 x 64 boxes in shared memory and writes them with
+    tensor stores: ragged M and N (boxes cut by the matrix edge, boxes wholly outside), ReLU, the ReLU mask,
+    the overflow flag, identical bits on a rerun and identical bits to the per-lane stores."""
+    import os
+    from paper_1710_03740_b200 import binding as b
+    M, N, K = 520, 776, 10304            # 161 k-blocks: one epilogue warp set; 3 x 4 tiles, the last ones ragged
+    got, _, _, _ = _check_tc(op, M, N, K, kernel="pair")
+    again, _, _, _ = _check_tc(op, M, N, K, kernel="pair")
+    assert np.array_equal(got, again)
+    os.environ["MPT_TMA_STORE"] = "0"
+    try:
+        plain, _, _, _ = _check_tc(op, M, N, K, kernel="pair")
+    finally:
+        del os.environ["MPT_TMA_STORE"]
+    assert np.array_equal(got, plain)
+    _check_tc(op, M, N, K, flags=b.GEMM_RELU, kernel="pair")
+    mask = np.random.default_rng(11).standard_normal((M, N)).astype(np.float16)
+    _check_tc(op, M, N, K, mask=mask, kernel="pair")
+    _, ref, flag, _ = _check_tc(op, M, N, K, scale=30.0, want_flag=True, kernel="pair")
+    assert flag == int(((ref & 0x7FFF) >= 0x7C00).any()) == 1
+    _, _, flag, _ = _check_tc(op, M, N, K, want_flag=True, kernel="pair")
+    assert flag == 0
+
+
+@pytest.mark.parametrize("op", [0, 1, 2])
 @pytest.mark.parametrize("M,N,K", [(1280, 4000, 136), (1280, 3944, 72), (2304, 3072, 200)])
 def test_pair_kernel_half_width_tail_units(op, M, N, K):
     """A few more tiles than clusters: the left-over tiles run as two 256x128 halves, including
