@@ -6,11 +6,13 @@
 // own 128 rows of A and its own 128 columns of B (64 k per stage, 32 KB per stage and CTA),
 // the tensor core reads both CTAs' shared memory, and each CTA's tensor memory receives the
 // 128 x 256 accumulator block of its rows.  Compared with one CTA per 128x256 tile this
-// moves a third fewer operand bytes from L2 to the SMs and leaves room for a 7-stage ring.
+// moves a third fewer operand bytes from L2 to the SMs and leaves room for a 6-stage ring plus
+// 32 KB in which the epilogue stages the output for bulk tensor stores.
 //
 // Roles in each CTA (192 threads): warp 0 TMA producer, warp 1 MMA issuer (only the
 // leader CTA, rank 0, issues; both CTAs' warp 1 take part in the paired tensor-memory
-// allocation), warps 2-5 epilogue.  Synchronisation:
+// allocation), warps 2-5 epilogue (long products: 32 x 64 output boxes rounded into shared memory and
+// written by cp.async.bulk.tensor stores; short ones and the special forms: per-lane stores).  Synchronisation:
 //   full[s]   in the leader: 1 arrival (leader's expect_tx for both CTAs' bytes) + the bytes
 //             of both CTAs' loads (the peer's loads signal the leader's barrier)
 //   empty[s]  in each CTA: tcgen05.commit multicast to both CTAs when the MMAs have read stage s
