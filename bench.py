@@ -142,7 +142,7 @@ def n_params(cfg):
 
 # dram__bytes_read.sum + dram__bytes_write.sum of the representative GEMM launch of each workload
 # (ncu capture summarised in profiles/k_gemm_tc2_pair_4096x12288x12288.md), bytes per launch.
-NCU_GEMM_TRAFFIC = {"large": {"launch": "forward 4096x12288x12288", "bytes": 1.280e9, "algorithmic_bytes": 0.503e9}}
+NCU_GEMM_TRAFFIC = {"large": {"launch": "forward 4096x12288x12288", "bytes": 1.285e9, "algorithmic_bytes": 0.503e9}}
 
 
 def max_over_ranks(vals, device=None):
