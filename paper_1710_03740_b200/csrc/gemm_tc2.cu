@@ -392,44 +392,8 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUte
                     if (lane == 0 && boxes_sent >= 2) bulk_wait_group_read<1>();     // the store before last has left this box
                     __syncwarp();
                     const int colb = w.nb * TILE_N + w.n_off + bx * 64;
-#pragma unroll
-                    for (int h = 0; h < 2; h++) {
-                        uint32_t r[32], hw[16];
-                        tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * TILE_N + bx * 64 + h * 32), r);
-                        tc_wait_ld();
-                        round_pack32(r, p.relu != 0, hw);
-                        const int col0 = colb + h * 32;
-                        if (mrow && row_ok) {
-#pragma unroll
-                            for (int g8 = 0; g8 < 4; g8++) {
-                                if (col0 + g8 * 8 + 8 <= p.N) {
-                                    const uint4 mk = *(const uint4 *)(mrow + col0 + g8 * 8);
-                                    hw[4 * g8] = mask_pair(hw[4 * g8], mk.x);
-                                    hw[4 * g8 + 1] = mask_pair(hw[4 * g8 + 1], mk.y);
-                                    hw[4 * g8 + 2] = mask_pair(hw[4 * g8 + 2], mk.z);
-                                    hw[4 * g8 + 3] = mask_pair(hw[4 * g8 + 3], mk.w);
-                                }
-                            }
-                        }
-#pragma unroll
-                        for (int g8 = 0; g8 < 4; g8++) {
-                            // values outside the matrix are not stored (the tensor store clips) and must not vote
-                            if (row_ok && col0 + g8 * 8 + 8 <= p.N) {
-#pragma unroll
-                                for (int e = 0; e < 4; e++) nonfinite_acc(hw[4 * g8 + e], acc_bits);
-                            }
-                            const uint32_t piece = (uint32_t)((h * 4 + g8) ^ (lane & 7));      // 128-byte swizzle
-                            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(box + (uint32_t)(lane * 128) + (piece << 4)),
-                                         "r"(hw[4 * g8]), "r"(hw[4 * g8 + 1]), "r"(hw[4 * g8 + 2]), "r"(hw[4 * g8 + 3])
-                                         : "memory");
-                        }
-                    }
-                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the tensor store reads what the lanes wrote
-                    __syncwarp();
-                    if (lane == 0) {      // a group per box, also when the box lies outside the matrix: the wait above counts groups
-                        if (row0 < p.M && colb < p.N) tma_store_2d(&tmC, box, colb, row0);
-                        bulk_commit_group();
-                    }
+                    epilogue_box_store(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * TILE_N + bx * 64), box, &tmC, row0,
+                                       colb, p.M, p.N, p.relu != 0, mrow, row_ok, acc_bits);
                 }
                 bad |= nonfinite_any(acc_bits);
             } else {

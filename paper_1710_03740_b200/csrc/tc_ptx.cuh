@@ -548,6 +548,57 @@ __device__ __forceinline__ void bulk_wait_group_read()
 {
     asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
 }
+// Epilogue of one warp for one 32 x 64 box of the output (its 32 rows, 64 consecutive accumulator columns
+// starting at tensor-memory address taddr): each lane rounds its row's values (optional ReLU fused, optional
+// ReLU-derivative mask, inf/NaN vote into acc_bits - whole groups of 8 columns inside the matrix only, N must
+// be a multiple of 8), parks them in `box` (4 KB of shared memory, 1024-byte aligned) in the 128-byte-swizzled
+// layout of the output tensor map, and lane 0 sends the box with one tensor store and commits a bulk group
+// (always, so that callers can count groups).  The caller makes sure the box is free (bulk_wait_group_read).
+__device__ __forceinline__ void epilogue_box_store(uint32_t taddr, uint32_t box, const CUtensorMap *tmC, int row0, int colb,
+                                                   int M, int N, bool relu, const uint16_t *mrow, bool row_ok,
+                                                   uint32_t &acc_bits)
+{
+    const int lane = threadIdx.x & 31;
+#pragma unroll
+    for (int h = 0; h < 2; h++) {
+        uint32_t r[32], hw[16];
+        tc_ld32(taddr + (uint32_t)(h * 32), r);
+        tc_wait_ld();
+        round_pack32(r, relu, hw);
+        const int col0 = colb + h * 32;
+        if (mrow && row_ok) {
+#pragma unroll
+            for (int g8 = 0; g8 < 4; g8++) {
+                if (col0 + g8 * 8 + 8 <= N) {
+                    const uint4 mk = *(const uint4 *)(mrow + col0 + g8 * 8);
+                    hw[4 * g8] = mask_pair(hw[4 * g8], mk.x);
+                    hw[4 * g8 + 1] = mask_pair(hw[4 * g8 + 1], mk.y);
+                    hw[4 * g8 + 2] = mask_pair(hw[4 * g8 + 2], mk.z);
+                    hw[4 * g8 + 3] = mask_pair(hw[4 * g8 + 3], mk.w);
+                }
+            }
+        }
+#pragma unroll
+        for (int g8 = 0; g8 < 4; g8++) {
+            // values outside the matrix are not stored (the tensor store clips) and must not vote
+            if (row_ok && col0 + g8 * 8 + 8 <= N) {
+#pragma unroll
+                for (int e = 0; e < 4; e++) nonfinite_acc(hw[4 * g8 + e], acc_bits);
+            }
+            const uint32_t piece = (uint32_t)((h * 4 + g8) ^ (lane & 7));      // 128-byte swizzle
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(box + (uint32_t)(lane * 128) + (piece << 4)),
+                         "r"(hw[4 * g8]), "r"(hw[4 * g8 + 1]), "r"(hw[4 * g8 + 2]), "r"(hw[4 * g8 + 3])
+                         : "memory");
+        }
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the tensor store reads what the lanes wrote
+    __syncwarp();
+    if (lane == 0) {
+        if (row0 < M && colb < N) tma_store_2d(tmC, box, colb, row0);
+        bulk_commit_group();
+    }
+}
+
 // The same load with an L2 eviction-priority hint (policy from l2_policy()).  Operand lines marked
 // "evict last" outlive the output stores and the other kernels' streams in L2: inside the large-MLP step
 // the products run 2-2.5 % faster with both operands marked (an operand one product has just read, or
