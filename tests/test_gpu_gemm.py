@@ -253,6 +253,40 @@ def test_automatic_kernel_choice_around_the_split_thresholds(M, N, K, same_as):
         assert not np.array_equal(auto, other)          # a split sum rounds differently somewhere
 
 
+def _random_shapes(n, seed):
+    """Seeded shapes with every dimension a multiple of 8 (what the tensor-core kernels take), spread over
+    the regions of the kernel choice: few tiles with a long contraction (in-cluster split), up to 74 tiles
+    (single-CTA kernel), more (CTA pair, with and without a ragged last round), and narrow outputs."""
+    rng = np.random.default_rng(seed)
+    out = []
+    while len(out) < n:
+        kind = len(out) % 4
+        if kind == 0:      # few tiles, long K
+            M, N, K = 8 * rng.integers(32, 96), 8 * rng.integers(32, 96), 8 * rng.integers(256, 640)
+        elif kind == 1:    # mid-size
+            M, N, K = 8 * rng.integers(64, 260), 8 * rng.integers(64, 260), 8 * rng.integers(8, 96)
+        elif kind == 2:    # many tiles, short K
+            M, N, K = 8 * rng.integers(260, 420), 8 * rng.integers(260, 420), 8 * rng.integers(4, 24)
+        else:              # thin
+            M, N, K = 8 * rng.integers(1, 24), 8 * rng.integers(1, 200), 8 * rng.integers(8, 400)
+        if M * N * K <= 1.6e9:
+            out.append((int(M), int(N), int(K)))
+    return out
+
+
+@pytest.mark.parametrize("idx", range(24))
+def test_random_shapes_under_the_automatic_choice(idx):
+    """The library's own kernel choice on seeded random shapes, one of the three product forms each, with a
+    scratch buffer where the choice wants one, plus ReLU on every third: every element within the
+    acceptance rule against the oracle."""
+    from paper_1710_03740_b200 import binding as b
+    M, N, K = _random_shapes(24, 2024)[idx]
+    op = idx % 3
+    flags = b.GEMM_RELU if idx % 3 == 0 else 0
+    ws = b.mpt_gemm_workspace_bytes(op, M, N, K) > 0
+    _check_tc(op, M, N, K, flags=flags, seed=100 + idx, kernel="auto", workspace=ws)
+
+
 @pytest.mark.parametrize("kernel", ["tc", "pair"])
 @pytest.mark.parametrize("op", [0, 1, 2])
 def test_tc_gemm_run_to_run_identical(op, kernel):
